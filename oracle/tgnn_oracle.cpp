@@ -1,0 +1,736 @@
+// TEST INFRASTRUCTURE -- not part of the product path.
+//
+// Plain, slow, single-threaded CPU oracle for one chronological training step
+// of a TGN-style memory model over a mixed event batch (targets + flagged
+// auxiliary replay events), as set up by the paper's problem statement:
+//   * events e=(u,v,t,x) sorted by time, node memory m_u(t)      (Section III-A)
+//   * Message / Update recursion                                  (Eq. 1, Eq. 2)
+//   * mixed batch with an event-type mask                         (Eq. 5)
+//   * pruning set / pruned batch                                  (Eq. 10, Eq. 11)
+//   * target mask and masked loss                                 (Eq. 12, Eq. 13)
+//   * per-batch order: prune -> execute -> loss -> backprop + gradient norm
+//     -> parameter update                                         (Algorithm 2)
+// The paper leaves the model internals open; the concrete cell (GRU memory
+// updater, cosine time encoding, one multi-head temporal attention layer,
+// latest-message aggregation, MLP link-prediction head, Adam) is the textbook
+// TGN form and is written out below formula by formula.
+//
+// Everything is computed in fp64.  Two things are fp32 by definition of the
+// model state and are reproduced as such when the corresponding flag is set:
+// the argument of the time encoding (phi_f32) and the memory rows written
+// back to the table (round_state_f32).  With both flags clear the whole step
+// is a smooth fp64 function, which the finite-difference pins use.
+//
+// No blocking, fusion or reordering: every dot product is a plain loop.
+// This file shares no code with the CUDA path.  All functions are pinned by
+// tests (brute force, closed forms, invariants, finite differences).
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <vector>
+
+extern "C" {
+typedef struct {
+  int64_t num_nodes;
+  int32_t d;                // memory = time-encoding = embedding dimension
+  int32_t d_e;              // edge-feature dimension
+  int32_t k;                // most-recent neighbors per root
+  int32_t heads;            // attention heads (d % heads == 0)
+  int32_t feat_bf16;        // edge features are bf16 bit patterns (uint16) instead of fp32
+  int32_t phi_f32;          // time-encoding argument fmaf(w,(float)dt,b) formed in fp32
+  int32_t round_state_f32;  // memory rows rounded to fp32 on write-back
+  int32_t reserved;
+  double lr, beta1, beta2, eps;  // Adam
+} orc_config;
+}
+
+namespace {
+
+typedef std::vector<double> vec;
+
+// ---------------------------------------------------------------- layout ----
+// Flat parameter vector, matrices [out, in] row-major, in this order.
+struct Layout {
+  int64_t d, de, dmsg, dkv, dq;
+  int64_t time_w, time_b, gru_wi, gru_wh, gru_bi, gru_bh, wq, bq, wk, wv, bk, bv, wo, bo, w1, b1, w2, b2, total;
+  explicit Layout(const orc_config& c) {
+    d = c.d; de = c.d_e; dmsg = 3 * d + de; dkv = 2 * d + de; dq = 2 * d;
+    int64_t o = 0;
+    time_w = o; o += d;
+    time_b = o; o += d;
+    gru_wi = o; o += 3 * d * dmsg;
+    gru_wh = o; o += 3 * d * d;
+    gru_bi = o; o += 3 * d;
+    gru_bh = o; o += 3 * d;
+    wq = o; o += d * dq;
+    bq = o; o += d;
+    wk = o; o += d * dkv;
+    wv = o; o += d * dkv;
+    bk = o; o += d;
+    bv = o; o += d;
+    wo = o; o += d * 2 * d;
+    bo = o; o += d;
+    w1 = o; o += d * 2 * d;
+    b1 = o; o += d;
+    w2 = o; o += d;
+    b2 = o; o += 1;
+    total = o;
+  }
+};
+
+inline double sigmoid(double x) { return 1.0 / (1.0 + std::exp(-x)); }
+inline double softplus(double x) { return x > 0 ? x + std::log1p(std::exp(-x)) : std::log1p(std::exp(x)); }
+
+inline double bf16_to_double(uint16_t b) {
+  uint32_t u = (uint32_t)b << 16;
+  float f;
+  std::memcpy(&f, &u, 4);
+  return (double)f;
+}
+
+inline double feat_at(const orc_config& c, const void* efeat, int64_t e, int j) {
+  if (c.feat_bf16) return bf16_to_double(((const uint16_t*)efeat)[e * c.d_e + j]);
+  return (double)((const float*)efeat)[e * c.d_e + j];
+}
+
+// Time encoding  Phi(dt)_c = cos(w_c * dt + b_c).  Returns the argument and
+// the dt value that multiplies w in it (needed for d/dw).
+inline double phi_arg(const orc_config& c, double w, double b, double dt, double* dt_used) {
+  if (c.phi_f32) {
+    float dtf = (float)dt;
+    *dt_used = (double)dtf;
+    return (double)std::fmaf((float)w, dtf, (float)b);
+  }
+  *dt_used = dt;
+  return w * dt + b;
+}
+
+// ------------------------------------------------------------- step (0) ----
+// 64-bit mixer: the finaliser of the SplitMix64 generator.
+inline uint64_t mix64(uint64_t z) {
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+  return z ^ (z >> 31);
+}
+inline uint32_t hash32(uint64_t seed, int64_t batch_idx, int32_t eid) {
+  uint64_t x = seed ^ ((uint64_t)batch_idx * 0x9E3779B97F4A7C15ULL) ^ ((uint64_t)(uint32_t)eid * 0xC2B2AE3D27D4EB4FULL);
+  return (uint32_t)(mix64(x) >> 32);
+}
+
+// ------------------------------------------------------------- forward -----
+struct Inputs {
+  const orc_config* c;
+  const void* efeat;
+  // update events U (the previous kept mixed batch); keep may be null (= all kept)
+  const int32_t *u_src, *u_dst, *u_eid;
+  const double* u_t;
+  const uint8_t* u_keep;
+  int n_u;
+  // roots of the current batch's targets: rows [src | dst | neg] blocks of n_q
+  const int32_t* r_node;
+  const double* r_time;
+  int n_r;
+  const int32_t *nb_node, *nb_eid;  // [n_r, k]
+  const double* nb_ts;              // [n_r, k]
+  const int32_t* nb_cnt;            // [n_r]
+  int n_q;
+  const uint8_t* loss_mask;  // [n_q]
+};
+
+struct Tape {
+  // messages / reduction / GRU
+  std::vector<int32_t> msg_node;  // [2 n_u]
+  vec msg;                        // [2 n_u, dmsg]
+  vec msg_dt;                     // [2 n_u] dt value inside Phi
+  std::vector<int32_t> uniq, winner, node2slot;
+  vec gi, gh;        // [U, 3d]
+  vec r, z, nn, hn;  // [U, d]; hn = W_hn h + b_hn
+  vec hnew;          // [U, d]
+  vec mem_post;      // [N, d]
+  vec lu_post;       // [N]
+  // embedding
+  vec zq, Q, Z, K, V, alpha, att, cat_o, pre_o, h;
+  vec z_dt;  // [n_r, k]
+  // loss
+  vec cat1, pre1, hid1, score;  // 2*n_q pairs: pair p<n_q positive, p>=n_q negative
+  double loss;
+  double mask_sum;
+};
+
+void build_messages(const Inputs& in, const Layout& L, const double* P, const double* mem, const double* lu, Tape& T) {
+  const orc_config& c = *in.c;
+  const int64_t d = L.d, de = L.de, dm = L.dmsg;
+  T.msg_node.assign(2 * (size_t)in.n_u, -1);
+  T.msg.assign(2 * (size_t)in.n_u * dm, 0.0);
+  T.msg_dt.assign(2 * (size_t)in.n_u, 0.0);
+  for (int i = 0; i < in.n_u; ++i) {
+    if (in.u_keep && !in.u_keep[i]) continue;
+    for (int role = 0; role < 2; ++role) {
+      const int32_t self = role == 0 ? in.u_src[i] : in.u_dst[i];
+      const int32_t other = role == 0 ? in.u_dst[i] : in.u_src[i];
+      const size_t j = 2 * (size_t)i + role;
+      double* m = &T.msg[j * dm];
+      T.msg_node[j] = self;
+      for (int64_t q = 0; q < d; ++q) m[q] = mem[self * d + q];
+      for (int64_t q = 0; q < d; ++q) m[d + q] = mem[other * d + q];
+      for (int64_t q = 0; q < de; ++q) m[2 * d + q] = feat_at(c, in.efeat, in.u_eid[i], (int)q);
+      const double dt = in.u_t[i] - lu[self];
+      double dtu = 0;
+      for (int64_t q = 0; q < d; ++q) m[2 * d + de + q] = std::cos(phi_arg(c, P[L.time_w + q], P[L.time_b + q], dt, &dtu));
+      T.msg_dt[j] = dtu;
+    }
+  }
+}
+
+// Winner per node = message with the lexicographically largest (t, eid, role).
+void reduce_latest(const int32_t* msg_node, const double* t, const int32_t* eid, int n_msg, int64_t N,
+                   std::vector<int32_t>& uniq, std::vector<int32_t>& winner) {
+  std::vector<int32_t> best((size_t)N, -1);
+  for (int j = 0; j < n_msg; ++j) {
+    const int32_t n = msg_node[j];
+    if (n < 0) continue;
+    const int32_t b = best[n];
+    if (b < 0) { best[n] = j; continue; }
+    const double tj = t[j >> 1], tb = t[b >> 1];
+    const int32_t ej = eid[j >> 1], eb = eid[b >> 1];
+    const int rj = j & 1, rb = b & 1;
+    const bool greater = tj > tb || (tj == tb && (ej > eb || (ej == eb && rj > rb)));
+    if (greater) best[n] = j;
+  }
+  uniq.clear();
+  winner.clear();
+  for (int64_t n = 0; n < N; ++n)
+    if (best[n] >= 0) { uniq.push_back((int32_t)n); winner.push_back(best[n]); }
+}
+
+// GRU cell, gate order (r, z, n), separate input / hidden biases:
+//   r = s(W_ir x + b_ir + W_hr h + b_hr),  z = s(W_iz x + b_iz + W_hz h + b_hz)
+//   n = tanh(W_in x + b_in + r * (W_hn h + b_hn)),  h' = (1 - z) n + z h
+void gru_rows(const Layout& L, const double* P, const double* X, const double* H, int U, Tape& T) {
+  const int64_t d = L.d, dm = L.dmsg;
+  T.gi.assign((size_t)U * 3 * d, 0); T.gh.assign((size_t)U * 3 * d, 0);
+  T.r.assign((size_t)U * d, 0); T.z.assign((size_t)U * d, 0); T.nn.assign((size_t)U * d, 0);
+  T.hn.assign((size_t)U * d, 0); T.hnew.assign((size_t)U * d, 0);
+  for (int u = 0; u < U; ++u) {
+    const double* x = X + (size_t)u * dm;
+    const double* h = H + (size_t)u * d;
+    for (int64_t o = 0; o < 3 * d; ++o) {
+      double a = P[L.gru_bi + o];
+      for (int64_t q = 0; q < dm; ++q) a += P[L.gru_wi + o * dm + q] * x[q];
+      T.gi[(size_t)u * 3 * d + o] = a;
+      double b = P[L.gru_bh + o];
+      for (int64_t q = 0; q < d; ++q) b += P[L.gru_wh + o * d + q] * h[q];
+      T.gh[(size_t)u * 3 * d + o] = b;
+    }
+    for (int64_t q = 0; q < d; ++q) {
+      const double* gi = &T.gi[(size_t)u * 3 * d];
+      const double* gh = &T.gh[(size_t)u * 3 * d];
+      const double r = sigmoid(gi[q] + gh[q]);
+      const double z = sigmoid(gi[d + q] + gh[d + q]);
+      const double n = std::tanh(gi[2 * d + q] + r * gh[2 * d + q]);
+      T.r[(size_t)u * d + q] = r; T.z[(size_t)u * d + q] = z; T.nn[(size_t)u * d + q] = n;
+      T.hn[(size_t)u * d + q] = gh[2 * d + q];
+      T.hnew[(size_t)u * d + q] = (1.0 - z) * n + z * h[q];
+    }
+  }
+}
+
+// Steps (2)-(4): messages from U on pre-step memory, latest-message reduction,
+// GRU on the winners, then write-back (all h' computed before any write).
+void memory_update(const Inputs& in, const Layout& L, const double* P, const double* mem, const double* lu, Tape& T) {
+  const orc_config& c = *in.c;
+  const int64_t N = c.num_nodes, d = L.d, dm = L.dmsg;
+  build_messages(in, L, P, mem, lu, T);
+  reduce_latest(T.msg_node.data(), in.u_t, in.u_eid, 2 * in.n_u, N, T.uniq, T.winner);
+  const int U = (int)T.uniq.size();
+  vec X((size_t)U * dm), H((size_t)U * d);
+  for (int u = 0; u < U; ++u) {
+    std::copy(&T.msg[(size_t)T.winner[u] * dm], &T.msg[(size_t)T.winner[u] * dm] + dm, &X[(size_t)u * dm]);
+    for (int64_t q = 0; q < d; ++q) H[(size_t)u * d + q] = mem[(size_t)T.uniq[u] * d + q];
+  }
+  gru_rows(L, P, X.data(), H.data(), U, T);
+  T.mem_post.assign(mem, mem + (size_t)N * d);
+  T.lu_post.assign(lu, lu + N);
+  T.node2slot.assign((size_t)N, -1);
+  for (int u = 0; u < U; ++u) {
+    const int32_t n = T.uniq[u];
+    T.node2slot[n] = u;
+    for (int64_t q = 0; q < d; ++q) {
+      double v = T.hnew[(size_t)u * d + q];
+      if (c.round_state_f32) v = (double)(float)v;
+      T.mem_post[(size_t)n * d + q] = v;
+    }
+    T.lu_post[n] = in.u_t[T.winner[u] >> 1];
+  }
+}
+
+// Step (5): one multi-head temporal attention layer over the <=k sampled neighbors.
+void embed(const Inputs& in, const Layout& L, const double* P, const double* mem, Tape& T) {
+  const orc_config& c = *in.c;
+  const int64_t d = L.d, de = L.de, dkv = L.dkv, dq = L.dq, k = c.k, H = c.heads, dh = d / H;
+  const int R = in.n_r;
+  T.zq.assign((size_t)R * dq, 0); T.Q.assign((size_t)R * d, 0);
+  T.Z.assign((size_t)R * k * dkv, 0); T.K.assign((size_t)R * k * d, 0); T.V.assign((size_t)R * k * d, 0);
+  T.alpha.assign((size_t)R * H * k, 0); T.att.assign((size_t)R * d, 0);
+  T.cat_o.assign((size_t)R * 2 * d, 0); T.pre_o.assign((size_t)R * d, 0); T.h.assign((size_t)R * d, 0);
+  T.z_dt.assign((size_t)R * k, 0);
+  const double scale = 1.0 / std::sqrt((double)dh);
+  for (int i = 0; i < R; ++i) {
+    const int32_t n = in.r_node[i];
+    const double t = in.r_time[i];
+    const int cnt = in.nb_cnt[i];
+    double* zq = &T.zq[(size_t)i * dq];
+    double dtu;
+    for (int64_t q = 0; q < d; ++q) zq[q] = mem[(size_t)n * d + q];
+    for (int64_t q = 0; q < d; ++q) zq[d + q] = std::cos(phi_arg(c, P[L.time_w + q], P[L.time_b + q], 0.0, &dtu));
+    double* Q = &T.Q[(size_t)i * d];
+    for (int64_t o = 0; o < d; ++o) {
+      double a = P[L.bq + o];
+      for (int64_t q = 0; q < dq; ++q) a += P[L.wq + o * dq + q] * zq[q];
+      Q[o] = a;
+    }
+    for (int s = 0; s < cnt; ++s) {
+      const int32_t nb = in.nb_node[(size_t)i * k + s];
+      const int32_t e = in.nb_eid[(size_t)i * k + s];
+      const double dt = t - in.nb_ts[(size_t)i * k + s];
+      double* z = &T.Z[((size_t)i * k + s) * dkv];
+      for (int64_t q = 0; q < d; ++q) z[q] = mem[(size_t)nb * d + q];
+      for (int64_t q = 0; q < de; ++q) z[d + q] = feat_at(c, in.efeat, e, (int)q);
+      for (int64_t q = 0; q < d; ++q) z[d + de + q] = std::cos(phi_arg(c, P[L.time_w + q], P[L.time_b + q], dt, &dtu));
+      T.z_dt[(size_t)i * k + s] = dtu;
+      double* K = &T.K[((size_t)i * k + s) * d];
+      double* V = &T.V[((size_t)i * k + s) * d];
+      for (int64_t o = 0; o < d; ++o) {
+        double a = P[L.bk + o], b = P[L.bv + o];
+        for (int64_t q = 0; q < dkv; ++q) {
+          a += P[L.wk + o * dkv + q] * z[q];
+          b += P[L.wv + o * dkv + q] * z[q];
+        }
+        K[o] = a; V[o] = b;
+      }
+    }
+    double* att = &T.att[(size_t)i * d];
+    for (int64_t hh = 0; hh < H; ++hh) {
+      if (cnt == 0) break;
+      double logit[64], mx = -1e300, den = 0;
+      for (int s = 0; s < cnt; ++s) {
+        double a = 0;
+        for (int64_t q = 0; q < dh; ++q) a += Q[hh * dh + q] * T.K[((size_t)i * k + s) * d + hh * dh + q];
+        logit[s] = a * scale;
+        mx = std::max(mx, logit[s]);
+      }
+      for (int s = 0; s < cnt; ++s) { logit[s] = std::exp(logit[s] - mx); den += logit[s]; }
+      for (int s = 0; s < cnt; ++s) {
+        const double al = logit[s] / den;
+        T.alpha[((size_t)i * H + hh) * k + s] = al;
+        for (int64_t q = 0; q < dh; ++q) att[hh * dh + q] += al * T.V[((size_t)i * k + s) * d + hh * dh + q];
+      }
+    }
+    double* cat = &T.cat_o[(size_t)i * 2 * d];
+    for (int64_t q = 0; q < d; ++q) { cat[q] = att[q]; cat[d + q] = mem[(size_t)n * d + q]; }
+    for (int64_t o = 0; o < d; ++o) {
+      double a = P[L.bo + o];
+      for (int64_t q = 0; q < 2 * d; ++q) a += P[L.wo + o * 2 * d + q] * cat[q];
+      T.pre_o[(size_t)i * d + o] = a;
+      T.h[(size_t)i * d + o] = a > 0 ? a : 0;
+    }
+  }
+}
+
+// Step (6): link-prediction head and the masked mean loss of Eq. 13.
+//   score(a,b) = w2 . ReLU(W1 [a || b] + b1) + b2
+//   l_j = softplus(-score(h_src, h_dst)) + softplus(score(h_src, h_neg))
+void loss_forward(const Inputs& in, const Layout& L, const double* P, Tape& T) {
+  const int64_t d = L.d;
+  const int nq = in.n_q;
+  T.cat1.assign((size_t)2 * nq * 2 * d, 0); T.pre1.assign((size_t)2 * nq * d, 0);
+  T.hid1.assign((size_t)2 * nq * d, 0); T.score.assign((size_t)2 * nq, 0);
+  double num = 0, den = 0;
+  for (int j = 0; j < nq; ++j) {
+    for (int pn = 0; pn < 2; ++pn) {
+      const size_t p = (size_t)pn * nq + j;
+      const size_t a = j, b = (size_t)(pn == 0 ? nq : 2 * nq) + j;
+      double* cat = &T.cat1[p * 2 * d];
+      for (int64_t q = 0; q < d; ++q) { cat[q] = T.h[a * d + q]; cat[d + q] = T.h[b * d + q]; }
+      double s = P[L.b2];
+      for (int64_t o = 0; o < d; ++o) {
+        double acc = P[L.b1 + o];
+        for (int64_t q = 0; q < 2 * d; ++q) acc += P[L.w1 + o * 2 * d + q] * cat[q];
+        T.pre1[p * d + o] = acc;
+        const double hd = acc > 0 ? acc : 0;
+        T.hid1[p * d + o] = hd;
+        s += P[L.w2 + o] * hd;
+      }
+      T.score[p] = s;
+    }
+    const double m = in.loss_mask ? (in.loss_mask[j] ? 1.0 : 0.0) : 1.0;
+    num += m * (softplus(-T.score[j]) + softplus(T.score[(size_t)nq + j]));
+    den += m;
+  }
+  T.mask_sum = den;
+  T.loss = den > 0 ? num / den : 0.0;
+}
+
+void forward_all(const Inputs& in, const Layout& L, const double* P, const double* mem, const double* lu, Tape& T) {
+  memory_update(in, L, P, mem, lu, T);
+  embed(in, L, P, T.mem_post.data(), T);
+  loss_forward(in, L, P, T);
+}
+
+// ------------------------------------------------------------ backward -----
+// Exact gradient of the masked loss w.r.t. every parameter.  Memory rows
+// written by the GRU in this step depend on the GRU parameters and, through
+// the message's time encoding, on (w, b); all other table reads (including the
+// memory values inside messages and the GRU's hidden input) are constants.
+void backward_all(const Inputs& in, const Layout& L, const double* P, const Tape& T, vec& G) {
+  const orc_config& c = *in.c;
+  const int64_t N = c.num_nodes, d = L.d, de = L.de, dkv = L.dkv, dq = L.dq, dm = L.dmsg, k = c.k, H = c.heads, dh = d / H;
+  const int R = in.n_r, nq = in.n_q;
+  G.assign((size_t)L.total, 0.0);
+  vec dh_((size_t)R * d, 0.0);
+  // loss + head
+  for (int j = 0; j < nq; ++j) {
+    const double m = in.loss_mask ? (in.loss_mask[j] ? 1.0 : 0.0) : 1.0;
+    if (T.mask_sum <= 0 || m == 0) continue;
+    const double wj = m / T.mask_sum;
+    for (int pn = 0; pn < 2; ++pn) {
+      const size_t p = (size_t)pn * nq + j;
+      const size_t a = j, b = (size_t)(pn == 0 ? nq : 2 * nq) + j;
+      const double s = T.score[p];
+      const double ds = wj * (pn == 0 ? -sigmoid(-s) : sigmoid(s));
+      G[L.b2] += ds;
+      vec dcat((size_t)2 * d, 0.0);
+      for (int64_t o = 0; o < d; ++o) {
+        G[L.w2 + o] += ds * T.hid1[p * d + o];
+        const double dpre = T.pre1[p * d + o] > 0 ? ds * P[L.w2 + o] : 0.0;
+        G[L.b1 + o] += dpre;
+        for (int64_t q = 0; q < 2 * d; ++q) {
+          G[L.w1 + o * 2 * d + q] += dpre * T.cat1[p * 2 * d + q];
+          dcat[q] += P[L.w1 + o * 2 * d + q] * dpre;
+        }
+      }
+      for (int64_t q = 0; q < d; ++q) { dh_[a * d + q] += dcat[q]; dh_[b * d + q] += dcat[d + q]; }
+    }
+  }
+  // embedding
+  vec dmem((size_t)N * d, 0.0);
+  const double scale = 1.0 / std::sqrt((double)dh);
+  for (int i = 0; i < R; ++i) {
+    const int32_t n = in.r_node[i];
+    const int cnt = in.nb_cnt[i];
+    vec dcat((size_t)2 * d, 0.0);
+    for (int64_t o = 0; o < d; ++o) {
+      const double dpre = T.pre_o[(size_t)i * d + o] > 0 ? dh_[(size_t)i * d + o] : 0.0;
+      G[L.bo + o] += dpre;
+      for (int64_t q = 0; q < 2 * d; ++q) {
+        G[L.wo + o * 2 * d + q] += dpre * T.cat_o[(size_t)i * 2 * d + q];
+        dcat[q] += P[L.wo + o * 2 * d + q] * dpre;
+      }
+    }
+    for (int64_t q = 0; q < d; ++q) dmem[(size_t)n * d + q] += dcat[d + q];
+    vec dQ((size_t)d, 0.0), dK((size_t)k * d, 0.0), dV((size_t)k * d, 0.0);
+    for (int64_t hh = 0; hh < H; ++hh) {
+      if (cnt == 0) break;
+      double dal[64], dot = 0;
+      for (int s = 0; s < cnt; ++s) {
+        const double al = T.alpha[((size_t)i * H + hh) * k + s];
+        double a = 0;
+        for (int64_t q = 0; q < dh; ++q) {
+          a += dcat[hh * dh + q] * T.V[((size_t)i * k + s) * d + hh * dh + q];
+          dV[(size_t)s * d + hh * dh + q] = al * dcat[hh * dh + q];
+        }
+        dal[s] = a;
+        dot += al * a;
+      }
+      for (int s = 0; s < cnt; ++s) {
+        const double al = T.alpha[((size_t)i * H + hh) * k + s];
+        const double dlogit = al * (dal[s] - dot) * scale;
+        for (int64_t q = 0; q < dh; ++q) {
+          dQ[hh * dh + q] += dlogit * T.K[((size_t)i * k + s) * d + hh * dh + q];
+          dK[(size_t)s * d + hh * dh + q] = dlogit * T.Q[(size_t)i * d + hh * dh + q];
+        }
+      }
+    }
+    // Q = W_q [m_root || Phi(0)] + b_q
+    {
+      const double* zq = &T.zq[(size_t)i * dq];
+      vec dzq((size_t)dq, 0.0);
+      for (int64_t o = 0; o < d; ++o) {
+        G[L.bq + o] += dQ[o];
+        for (int64_t q = 0; q < dq; ++q) {
+          G[L.wq + o * dq + q] += dQ[o] * zq[q];
+          dzq[q] += P[L.wq + o * dq + q] * dQ[o];
+        }
+      }
+      for (int64_t q = 0; q < d; ++q) dmem[(size_t)n * d + q] += dzq[q];
+      for (int64_t q = 0; q < d; ++q) {
+        double dtu;
+        const double arg = phi_arg(c, P[L.time_w + q], P[L.time_b + q], 0.0, &dtu);
+        G[L.time_w + q] += -std::sin(arg) * dtu * dzq[d + q];
+        G[L.time_b + q] += -std::sin(arg) * dzq[d + q];
+      }
+    }
+    for (int s = 0; s < cnt; ++s) {
+      const double* z = &T.Z[((size_t)i * k + s) * dkv];
+      vec dz((size_t)dkv, 0.0);
+      for (int64_t o = 0; o < d; ++o) {
+        const double gk = dK[(size_t)s * d + o], gv = dV[(size_t)s * d + o];
+        G[L.bk + o] += gk;
+        G[L.bv + o] += gv;
+        for (int64_t q = 0; q < dkv; ++q) {
+          G[L.wk + o * dkv + q] += gk * z[q];
+          G[L.wv + o * dkv + q] += gv * z[q];
+          dz[q] += P[L.wk + o * dkv + q] * gk + P[L.wv + o * dkv + q] * gv;
+        }
+      }
+      const int32_t nb = in.nb_node[(size_t)i * k + s];
+      for (int64_t q = 0; q < d; ++q) dmem[(size_t)nb * d + q] += dz[q];
+      const double dt = in.r_time[i] - in.nb_ts[(size_t)i * k + s];
+      for (int64_t q = 0; q < d; ++q) {
+        double dtu;
+        const double arg = phi_arg(c, P[L.time_w + q], P[L.time_b + q], dt, &dtu);
+        G[L.time_w + q] += -std::sin(arg) * dtu * dz[d + de + q];
+        G[L.time_b + q] += -std::sin(arg) * dz[d + de + q];
+      }
+    }
+  }
+  // GRU rows written this step
+  const int U = (int)T.uniq.size();
+  for (int u = 0; u < U; ++u) {
+    const int32_t n = T.uniq[u];
+    const int32_t w = T.winner[u];
+    const double* x = &T.msg[(size_t)w * dm];
+    const double* hprev = x;  // first d entries of the message are the node's own memory
+    vec dgi((size_t)3 * d), dgh((size_t)3 * d);
+    for (int64_t q = 0; q < d; ++q) {
+      const double g = dmem[(size_t)n * d + q];
+      const double r = T.r[(size_t)u * d + q], z = T.z[(size_t)u * d + q], nn = T.nn[(size_t)u * d + q];
+      const double dn = g * (1.0 - z);
+      const double dz = g * (hprev[q] - nn);
+      const double dpn = dn * (1.0 - nn * nn);
+      const double dpz = dz * z * (1.0 - z);
+      const double dr = dpn * T.hn[(size_t)u * d + q];
+      const double dpr = dr * r * (1.0 - r);
+      dgi[q] = dpr; dgi[d + q] = dpz; dgi[2 * d + q] = dpn;
+      dgh[q] = dpr; dgh[d + q] = dpz; dgh[2 * d + q] = dpn * r;
+    }
+    vec dx((size_t)dm, 0.0);
+    for (int64_t o = 0; o < 3 * d; ++o) {
+      G[L.gru_bi + o] += dgi[o];
+      G[L.gru_bh + o] += dgh[o];
+      for (int64_t q = 0; q < dm; ++q) {
+        G[L.gru_wi + o * dm + q] += dgi[o] * x[q];
+        dx[q] += P[L.gru_wi + o * dm + q] * dgi[o];
+      }
+      for (int64_t q = 0; q < d; ++q) G[L.gru_wh + o * d + q] += dgh[o] * hprev[q];
+    }
+    const double dtu = T.msg_dt[w];
+    for (int64_t q = 0; q < d; ++q) {
+      // argument rebuilt exactly as in the forward pass
+      const double arg = c.phi_f32 ? (double)std::fmaf((float)P[L.time_w + q], (float)dtu, (float)P[L.time_b + q])
+                                   : P[L.time_w + q] * dtu + P[L.time_b + q];
+      G[L.time_w + q] += -std::sin(arg) * dtu * dx[2 * d + de + q];
+      G[L.time_b + q] += -std::sin(arg) * dx[2 * d + de + q];
+    }
+  }
+}
+
+vec to_double(const float* p, size_t n) { return vec(p, p + n); }
+
+Inputs make_inputs(const orc_config* c, const void* efeat, const int32_t* u_src, const int32_t* u_dst, const double* u_t,
+                   const int32_t* u_eid, const uint8_t* u_keep, int n_u, const int32_t* r_node, const double* r_time,
+                   int n_r, const int32_t* nb_node, const int32_t* nb_eid, const double* nb_ts, const int32_t* nb_cnt,
+                   int n_q, const uint8_t* loss_mask) {
+  Inputs in;
+  in.c = c; in.efeat = efeat;
+  in.u_src = u_src; in.u_dst = u_dst; in.u_t = u_t; in.u_eid = u_eid; in.u_keep = u_keep; in.n_u = n_u;
+  in.r_node = r_node; in.r_time = r_time; in.n_r = n_r;
+  in.nb_node = nb_node; in.nb_eid = nb_eid; in.nb_ts = nb_ts; in.nb_cnt = nb_cnt;
+  in.n_q = n_q; in.loss_mask = loss_mask;
+  return in;
+}
+
+}  // namespace
+
+// =============================================================== exports ====
+extern "C" {
+
+int64_t orc_param_count(const orc_config* c) { return Layout(*c).total; }
+
+// Offsets of the 18 tensors in the flat parameter vector, in layout order, plus the total.
+void orc_param_layout(const orc_config* c, int64_t* out19) {
+  Layout L(*c);
+  const int64_t v[19] = {L.time_w, L.time_b, L.gru_wi, L.gru_wh, L.gru_bi, L.gru_bh, L.wq, L.bq, L.wk, L.wv,
+                         L.bk, L.bv, L.wo, L.bo, L.w1, L.b1, L.w2, L.b2, L.total};
+  for (int i = 0; i < 19; ++i) out19[i] = v[i];
+}
+
+uint64_t orc_mix64(uint64_t z) { return mix64(z); }
+uint32_t orc_hash32(uint64_t seed, int64_t batch_idx, int32_t eid) { return hash32(seed, batch_idx, eid); }
+
+// Step (0), Eq. 10-11 with the workload's deterministic trigger:
+//   cnt[n] = endpoint occurrences of n in the mixed batch; T = #nodes with cnt>0;
+//   heavy = max cnt * T > 4 * 2n  (max > 4 x mean over touched nodes), unless force_heavy in {0,1};
+//   targets are always kept; a replay event is dropped iff heavy and
+//   (drop_q32 == 0xFFFFFFFF, "all", or hash32(seed, batch_idx, eid) < drop_q32).
+void orc_prune_mask(int64_t num_nodes, const int32_t* src, const int32_t* dst, const int32_t* eid, const uint8_t* is_aux,
+                    int n, int force_heavy, uint32_t drop_q32, uint64_t seed, int64_t batch_idx, uint8_t* keep_out,
+                    int32_t* heavy_out) {
+  std::vector<int64_t> cnt((size_t)num_nodes, 0);
+  for (int i = 0; i < n; ++i) { cnt[src[i]]++; cnt[dst[i]]++; }
+  int64_t mx = 0, touched = 0;
+  for (int64_t v = 0; v < num_nodes; ++v) { mx = std::max(mx, cnt[v]); touched += cnt[v] > 0; }
+  int heavy = (mx * touched > 4 * 2 * (int64_t)n) ? 1 : 0;
+  if (force_heavy == 0 || force_heavy == 1) heavy = force_heavy;
+  for (int i = 0; i < n; ++i) {
+    bool keep = true;
+    if (is_aux[i] && heavy) keep = !(drop_q32 == 0xFFFFFFFFu || hash32(seed, batch_idx, eid[i]) < drop_q32);
+    keep_out[i] = keep ? 1 : 0;
+  }
+  *heavy_out = heavy;
+}
+
+// Step (1): p = first index of the node's T-CSR slice with ts[p] >= t (found by
+// bisection); slot s < cnt is entry p-1-s; cnt = min(k, p - indptr[node]).
+void orc_sample_recent(const int64_t* indptr, const int32_t* nbr, const int32_t* eid, const double* ts,
+                       const int32_t* nodes, const double* times, int n, int k, int32_t* nbr_out, int32_t* eid_out,
+                       double* ts_out, int32_t* cnt_out) {
+  for (int i = 0; i < n; ++i) {
+    int64_t lo = indptr[nodes[i]], hi = indptr[nodes[i] + 1];
+    const int64_t base = lo;
+    while (lo < hi) {
+      const int64_t mid = lo + (hi - lo) / 2;
+      if (ts[mid] < times[i]) lo = mid + 1; else hi = mid;
+    }
+    const int64_t p = lo;
+    const int cnt = (int)std::min<int64_t>(k, p - base);
+    cnt_out[i] = cnt;
+    for (int s = 0; s < k; ++s) {
+      if (s < cnt) {
+        nbr_out[(size_t)i * k + s] = nbr[p - 1 - s];
+        eid_out[(size_t)i * k + s] = eid[p - 1 - s];
+        ts_out[(size_t)i * k + s] = ts[p - 1 - s];
+      } else {
+        nbr_out[(size_t)i * k + s] = -1;
+        eid_out[(size_t)i * k + s] = -1;
+        ts_out[(size_t)i * k + s] = 0.0;
+      }
+    }
+  }
+}
+
+// Time encoding alone (for the closed-form pins).
+void orc_time_encode(const orc_config* c, const double* w, const double* b, const double* dt, int n, double* out) {
+  for (int i = 0; i < n; ++i)
+    for (int q = 0; q < c->d; ++q) {
+      double dtu;
+      out[(size_t)i * c->d + q] = std::cos(phi_arg(*c, w[q], b[q], dt[i], &dtu));
+    }
+}
+
+// Step (2), Eq. 1: msg[2i] -> node src (role 0), msg[2i+1] -> node dst (role 1);
+// layout [m_self || m_other || x || Phi(t - last_update[self])]; dropped events give node -1, zero rows.
+void orc_build_messages(const orc_config* c, const double* params, const double* memory, const double* last_update,
+                        const void* efeat, const int32_t* src, const int32_t* dst, const double* t, const int32_t* eid,
+                        const uint8_t* keep, int n, double* msg_out, int32_t* msg_node_out) {
+  Layout L(*c);
+  Inputs in = make_inputs(c, efeat, src, dst, t, eid, keep, n, 0, 0, 0, 0, 0, 0, 0, 0, 0);
+  Tape T;
+  build_messages(in, L, params, memory, last_update, T);
+  std::copy(T.msg.begin(), T.msg.end(), msg_out);
+  std::copy(T.msg_node.begin(), T.msg_node.end(), msg_node_out);
+}
+
+// Step (3).  t and eid are per event (message j belongs to event j>>1, role j&1).
+void orc_reduce_latest(const int32_t* msg_node, const double* t, const int32_t* eid, int n_msg, int64_t num_nodes,
+                       int32_t* uniq_out, int32_t* winner_out, int32_t* n_uniq_out) {
+  std::vector<int32_t> uniq, winner;
+  reduce_latest(msg_node, t, eid, n_msg, num_nodes, uniq, winner);
+  std::copy(uniq.begin(), uniq.end(), uniq_out);
+  std::copy(winner.begin(), winner.end(), winner_out);
+  *n_uniq_out = (int32_t)uniq.size();
+}
+
+// Step (4), Eq. 2 on explicit message rows: memory[n] <- GRU(msg[winner], memory[n]),
+// last_update[n] <- t[winner>>1]; every h' is computed before any row is written.
+void orc_memory_update(const orc_config* c, const double* params, const double* msg, const double* t, const int32_t* uniq,
+                       const int32_t* winner, int n_uniq, double* memory, double* last_update) {
+  Layout L(*c);
+  const int64_t d = L.d, dm = L.dmsg;
+  vec X((size_t)n_uniq * dm), Hh((size_t)n_uniq * d);
+  for (int u = 0; u < n_uniq; ++u) {
+    std::copy(msg + (size_t)winner[u] * dm, msg + (size_t)winner[u] * dm + dm, &X[(size_t)u * dm]);
+    for (int64_t q = 0; q < d; ++q) Hh[(size_t)u * d + q] = memory[(size_t)uniq[u] * d + q];
+  }
+  Tape T;
+  gru_rows(L, params, X.data(), Hh.data(), n_uniq, T);
+  for (int u = 0; u < n_uniq; ++u) {
+    for (int64_t q = 0; q < d; ++q) {
+      double v = T.hnew[(size_t)u * d + q];
+      if (c->round_state_f32) v = (double)(float)v;
+      memory[(size_t)uniq[u] * d + q] = v;
+    }
+    last_update[uniq[u]] = t[winner[u] >> 1];
+  }
+}
+
+// Step (5).
+void orc_embed(const orc_config* c, const double* params, const double* memory, const void* efeat, const int32_t* nodes,
+               const double* times, int n, const int32_t* nbr, const int32_t* eid, const double* ts, const int32_t* cnt,
+               double* h_out) {
+  Layout L(*c);
+  Inputs in = make_inputs(c, efeat, 0, 0, 0, 0, 0, 0, nodes, times, n, nbr, eid, ts, cnt, 0, 0);
+  Tape T;
+  embed(in, L, params, memory, T);
+  std::copy(T.h.begin(), T.h.end(), h_out);
+}
+
+// Steps (2)-(6) forward plus the exact gradient, from the pre-step state.
+// Outputs (any may be null): loss, grads[P], gradnorm = sqrt(sum grads^2),
+// memory_post[N,d], last_update_post[N], h[n_r,d], uniq/winner/n_uniq.
+void orc_loss_and_grads(const orc_config* c, const double* params, const double* memory, const double* last_update,
+                        const void* efeat, const int32_t* u_src, const int32_t* u_dst, const double* u_t,
+                        const int32_t* u_eid, const uint8_t* u_keep, int n_u, const int32_t* r_node,
+                        const double* r_time, int n_r, const int32_t* nb_node, const int32_t* nb_eid,
+                        const double* nb_ts, const int32_t* nb_cnt, int n_q, const uint8_t* loss_mask, int want_grads,
+                        double* loss_out, double* grads_out, double* gradnorm_out, double* memory_post,
+                        double* last_update_post, double* h_out, int32_t* uniq_out, int32_t* winner_out,
+                        int32_t* n_uniq_out) {
+  Layout L(*c);
+  Inputs in = make_inputs(c, efeat, u_src, u_dst, u_t, u_eid, u_keep, n_u, r_node, r_time, n_r, nb_node, nb_eid, nb_ts,
+                          nb_cnt, n_q, loss_mask);
+  Tape T;
+  forward_all(in, L, params, memory, last_update, T);
+  if (loss_out) *loss_out = T.loss;
+  if (memory_post) std::copy(T.mem_post.begin(), T.mem_post.end(), memory_post);
+  if (last_update_post) std::copy(T.lu_post.begin(), T.lu_post.end(), last_update_post);
+  if (h_out) std::copy(T.h.begin(), T.h.end(), h_out);
+  if (uniq_out) std::copy(T.uniq.begin(), T.uniq.end(), uniq_out);
+  if (winner_out) std::copy(T.winner.begin(), T.winner.end(), winner_out);
+  if (n_uniq_out) *n_uniq_out = (int32_t)T.uniq.size();
+  if (want_grads) {
+    vec G;
+    backward_all(in, L, params, T, G);
+    double ss = 0;
+    for (double g : G) ss += g * g;
+    if (gradnorm_out) *gradnorm_out = std::sqrt(ss);
+    if (grads_out) std::copy(G.begin(), G.end(), grads_out);
+  }
+}
+
+// Adam, no weight decay, no clipping:
+//   step += 1; m = b1 m + (1-b1) g; v = b2 v + (1-b2) g^2;
+//   p -= lr * (m / (1 - b1^step)) / (sqrt(v / (1 - b2^step)) + eps)
+void orc_adam(const orc_config* c, int64_t n, const double* grads, double* params, double* m, double* v, int64_t* step) {
+  *step += 1;
+  const double bc1 = 1.0 - std::pow(c->beta1, (double)*step);
+  const double bc2 = 1.0 - std::pow(c->beta2, (double)*step);
+  for (int64_t i = 0; i < n; ++i) {
+    m[i] = c->beta1 * m[i] + (1.0 - c->beta1) * grads[i];
+    v[i] = c->beta2 * v[i] + (1.0 - c->beta2) * grads[i] * grads[i];
+    params[i] -= c->lr * (m[i] / bc1) / (std::sqrt(v[i] / bc2) + c->eps);
+  }
+}
+
+}  // extern "C"
