@@ -1,0 +1,368 @@
+#!/usr/bin/env python
+"""Benchmark of one chronological TGN-style training step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A "step" is one pass of the whole hot path over one batch of the synthetic
+wiki-shaped workload (9,000 nodes, 160,000 events, 172-d fp32 edge features,
+d = 100, k = 10, 2 heads, batch 600): prune mask of the mixed batch, memory
+update from the previous batch (messages, latest-event reduction, GRU), neighbor
+search, attention embedding, masked loss, backward and Adam.  The metric is
+target events per second (replay events are not counted, as in the paper's
+throughput definition).  Inputs are resident in HBM for `value`; `e2e` repeats
+the measurement through the host-buffer entry point with the per-step copies
+inside the timed region.  Every step is timed with its own CUDA event pair on
+the launching stream and L2 is flushed between steps (outside the events).
+
+With N > 1 (torchrun) every rank runs an independent replica on its own GPU:
+the step has no independent units to shard, so there is no collective on the
+data path; timing is the max over ranks.
+
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2608_16305_b200 import workload as wl  # noqa: E402
+
+METRIC = "train events/s on 1 B200 (fwd+bwd, memory+embed)"
+UNIT = "events/s"
+WORKLOAD = "wiki"
+SM_COUNT, FP32_LANES_PER_SM = 148, 128
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def aggregate_over_ranks(ms_local: float, units_local: int, device):
+    """(max over ranks of the time, sum over ranks of the units); identity without a process group."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return ms_local, units_local
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    u = torch.tensor([units_local], dtype=torch.int64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(u.item())
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def algorithmic_work(cfg: wl.WorkloadConfig, n_u: int, n_q: int, U: int):
+    """Algorithmic bytes and flops of one step (what the method must move / compute)."""
+    d, de, k = cfg.d, cfg.d_e, cfg.k
+    f = 4 if cfg.feat_dtype == "f32" else 2
+    R, NB = 3 * n_q, 3 * n_q * k
+    P = sum(int(np.prod(s)) for s in wl.param_shapes(d, de).values())
+    by = (R * 16 + NB * 16) + (2 * n_u * (2 * d * 4 + 8) + n_u * de * f) + U * (2 * d * 4 + 8) \
+        + NB * (4 * d + de * f + 16) + 2 * R * 4 * d + NB * (4 * d + de * f) + R * 4 * d + 28 * P
+    fwd = 2 * 3 * d * (cfg.d_msg + d) * U + 4 * d * cfg.d_kv * NB + 2 * d * 2 * d * R + 4 * d * R * k + 8 * d * d * R
+    return by, fwd, 2.3 * fwd
+
+
+def kv_proj_flops(cfg, n_q):
+    return 2.0 * (3 * n_q * cfg.k) * cfg.d_kv * (2 * cfg.d)
+
+
+def run_ours(args, rank, world, device):
+    from paper_2608_16305_b200 import binding as B
+    from paper_2608_16305_b200 import trainer as T
+    cfg = wl.CONFIGS[WORKLOAD]
+    stream = wl.make_stream(cfg)
+    efeat = wl.edge_feature_table_torch(cfg, device)
+    dw = T.DeviceWorkload(stream, device=device, efeat=efeat)
+    weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed)
+    math_mode = B.TGNN_MATH_TF32 if args.math == "tf32" else B.TGNN_MATH_FP32
+    tr = T.Trainer(dw, weights, math_mode=math_mode)
+    nb = cfg.num_batches - 1          # full batches only
+    K, W = args.steps, args.warmup
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)   # > 126 MB L2
+    peaks = measured_peaks()
+
+    def batch_of(i):
+        return i % nb
+
+    def reset_epoch():
+        tr.memory.zero_()
+        tr.last_update.zero_()
+
+    def run_steps(first, count, fn, timed):
+        evs = []
+        for i in range(first, first + count):
+            b = batch_of(i)
+            if b == 0:
+                reset_epoch()
+            flush.fill_(i & 0xff)
+            if timed:
+                a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                fn(b)
+                z.record()
+                evs.append((a, z))
+            else:
+                fn(b)
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(z) for a, z in evs)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    dev_step = lambda b: tr.step(b, with_update=b > 0)
+
+    # ---- device-resident inputs ----
+    run_steps(0, W, dev_step, False)
+    barrier()
+    l0 = tr.lib.kernel_launches()
+    with ClockSampler(torch.cuda.current_device()) as clk:
+        ms_dev = run_steps(W, K, dev_step, True)
+    launches = tr.lib.kernel_launches() - l0
+    barrier()
+    clocks = clk.summary()
+    loss_end = float(tr.loss.item())
+
+    # ---- host buffers: per-step H2D of the step's inputs, D2H of loss and of the pruned batch's keep mask ----
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    host = {}
+    for i in range(W + K + W + K + 4):
+        b = batch_of(i)
+        if b in host:
+            continue
+        mb = dw.mb_host[b]
+        q = dw.target_slice(b)
+        host[b] = dict(src=pin(mb.src), dst=pin(mb.dst), t=pin(mb.t), eid=pin(mb.eid), aux=pin(mb.is_aux),
+                       keep=torch.ones(mb.n, dtype=torch.uint8).pin_memory(),
+                       q_src=pin(stream.src[q]), q_dst=pin(stream.dst[q]), q_neg=pin(stream.neg[q]), q_t=pin(stream.t[q]))
+    cap = cfg.max_mixed
+    st = dict(src=torch.empty(cap, dtype=torch.int32, device=device), dst=torch.empty(cap, dtype=torch.int32, device=device),
+              eid=torch.empty(cap, dtype=torch.int32, device=device), aux=torch.empty(cap, dtype=torch.uint8, device=device),
+              keep=torch.empty(cap, dtype=torch.uint8, device=device), heavy=torch.zeros(1, dtype=torch.int32, device=device))
+    loss_h = torch.zeros(1).pin_memory()
+    gn_h = torch.zeros(1).pin_memory()
+    h2d = d2h = 0
+
+    def host_step(b):
+        nonlocal h2d, d2h
+        hb = host[b]
+        n = hb["src"].numel()
+        for kname in ("src", "dst", "eid", "aux"):
+            st[kname][:n].copy_(hb[kname], non_blocking=True)
+        tr.lib.prune_mask(st["src"][:n], st["dst"][:n], st["eid"][:n], st["aux"][:n], st["keep"][:n], st["heavy"],
+                          force_heavy=-1 if cfg.prune else 0, drop_q32=tr.drop_q32, seed=tr.prune_seed, batch_idx=b)
+        hb["keep"].copy_(st["keep"][:n], non_blocking=True)
+        if b > 0:
+            hu = host[b - 1]
+            upd = (hu["src"], hu["dst"], hu["t"], hu["eid"], hu["keep"])
+        else:
+            upd = (None,) * 5
+        tr.lib.train_step_host(*upd, hb["q_src"], hb["q_dst"], hb["q_neg"], hb["q_t"], None, loss_h, gn_h)
+        torch.cuda.current_stream().synchronize()        # the caller reads the loss every step
+        n_u = 0 if b == 0 else host[b - 1]["src"].numel()
+        h2d += n * 13 + n_u * 21 + hb["q_src"].numel() * 20
+        d2h += n + 8
+
+    reset_epoch()
+    run_steps(W + K, W, host_step, False)
+    barrier()
+    h2d = d2h = 0
+    ms_host = run_steps(W + K + W, K, host_step, True)
+    barrier()
+    h2d_step, d2h_step = h2d / K, d2h / K
+
+    # ---- per-kernel times of the same K steps (separate pass: the event pairs perturb a latency-bound step) ----
+    reset_epoch()
+    run_steps(0, W, dev_step, False)
+    tr.lib.profile_begin()
+    run_steps(W, K, dev_step, False)
+    prof = tr.lib.profile_report()
+    tot = sum(v[1] for v in prof.values()) or 1.0
+    top = sorted(prof.items(), key=lambda kv: -kv[1][1])
+
+    n_q = cfg.batch
+    ms_dev_max, units = aggregate_over_ranks(ms_dev, K * n_q, device)
+    ms_host_max, _ = aggregate_over_ranks(ms_host, K * n_q, device)
+    if rank != 0:
+        return
+    # roofline of the dominant kernel: the key/value projection GEMM of the attention layer
+    dom = "kv_proj"
+    cnt, ms_tot = prof.get(dom, (0, 0.0))
+    dur_s = (ms_tot / max(cnt, 1)) * 1e-3
+    flops = kv_proj_flops(cfg, n_q)
+    if args.math == "tf32":
+        peak, bound, peak_note = peaks["bf16_tflops"] * 0.5, "tensor", f"0.5 x {peaks['source']} bf16 burst (TF32 nominal ratio)"
+    else:
+        clk_ghz = (clocks["sm_max_mhz"] or 1965.0) / 1000.0
+        peak, bound = SM_COUNT * FP32_LANES_PER_SM * 2 * clk_ghz / 1000.0, "alu"
+        peak_note = "148 SMs x 128 fp32 lanes x 2 flop x max SM clock"
+    achieved = flops / dur_s / 1e12 if dur_s > 0 else 0.0
+    by, f_fwd, f_bwd = algorithmic_work(cfg, n_q, n_q, 450)
+    out = {
+        "metric": METRIC, "value": units / (ms_dev_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_dev_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "tf32" if args.math == "tf32" else "f32", "data": "synthetic",
+        "config": {"workload": f"{WORKLOAD}: 9000 nodes (8000+1000 bipartite), 160000 events, d_e=172 fp32, d=100, k=10, "
+                               "2 heads, batch 600, no replay",
+                   "math_mode": args.math, "l2": "512 MB buffer written between timed steps (outside the event pairs)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "inputs": "resident in HBM"},
+        "e2e": {"value": units / (ms_host_max * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d_step,
+                "d2h_bytes_per_step": d2h_step, "ms_per_step": ms_host_max / K,
+                "how": "tgnn_train_step_host with pinned host event arrays; loss read back and stream synchronised every step"},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                     "frac": achieved / peak if peak else None, "traffic": None, "peak_source": peak_note,
+                     "flops_per_launch": flops, "avg_launch_us": dur_s * 1e6, "launches": cnt,
+                     "step_algorithmic_bytes": by, "step_algorithmic_flops": f_fwd + f_bwd,
+                     "step_hbm_frac": (by / (ms_dev_max / K * 1e-3)) / (peaks["hbm_gbs"] * 1e9),
+                     "kernel_share": {k: round(v[1] / tot, 4) for k, v in top[:12]},
+                     "kernel_ms_total": round(tot, 3)},
+        "loss_last": loss_end,
+    }
+    out["cpu_baseline"] = cpu_baseline(cfg, stream, weights, budget_s=args.cpu_budget)
+    print(json.dumps(out))
+
+
+def cpu_baseline(cfg, stream, weights, budget_s=20.0, steps=None):
+    """The oracle as it stands, one thread, on consecutive batches from the middle of the epoch."""
+    from oracle import oracle as orc
+    ocfg = orc.make_config(cfg.num_nodes, cfg.d, cfg.d_e, cfg.k, cfg.heads, feat_bf16=cfg.feat_dtype == "bf16")
+    ef = stream.efeat() if cfg.d_e else None
+    state = orc.OracleState(ocfg, orc.pack_params(ocfg, weights))
+    graph = (stream.indptr, stream.nbr, stream.eid, stream.ts)
+    b0 = cfg.num_batches // 2
+    prev, done, spent = None, 0, 0.0
+    mbp = wl.mixed_batch(stream, b0 - 1)
+    prev = (mbp.src, mbp.dst, mbp.t, mbp.eid, None)
+    while (steps is None and spent < budget_s and done < 64) or (steps is not None and done < steps):
+        b = b0 + done
+        mb = wl.mixed_batch(stream, b)
+        q = slice(b * cfg.batch, (b + 1) * cfg.batch)
+        t0 = time.perf_counter()
+        keep, _ = orc.prune_mask(cfg.num_nodes, mb.src, mb.dst, mb.eid, mb.is_aux, force_heavy=-1 if cfg.prune else 0,
+                                 seed=cfg.seed, batch_idx=b)
+        state.step(graph, ef, prev, stream.src[q], stream.dst[q], stream.neg[q], stream.t[q])
+        spent += time.perf_counter() - t0
+        prev = (mb.src, mb.dst, mb.t, mb.eid, keep)
+        done += 1
+    return {"value": done * cfg.batch / spent, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": spent,
+            "sample": f"{done} consecutive steps (batches {b0}..{b0 + done - 1}) of the {cfg.name} workload, "
+                      f"single thread, host has {os.cpu_count()} cores"}
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    cfg = wl.CONFIGS[WORKLOAD]
+    stream = wl.make_stream(cfg)
+    weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed)
+    stream.efeat()
+    K, W = args.steps, args.warmup
+    per = 2                                   # oracle steps per benchmark "step" sample
+    n = min(K, 8)                             # bounded: the whole run must end within minutes
+    cpu_baseline(cfg, stream, weights, steps=min(W, 1))
+    res = cpu_baseline(cfg, stream, weights, steps=n * per)
+    ms = res["seconds"] * 1e3 / (n * per)
+    out = {"impl": "reference", "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": K,
+           "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "f64", "data": "synthetic",
+           "config": {"workload": f"{WORKLOAD}: bounded sample of {n * per} oracle steps standing for {K} steps"},
+           "cpu_baseline": {"value": res["value"], "unit": UNIT, "kind": "oracle", "cores": 1, "sample": res["sample"]},
+           "e2e": {"value": res["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--math", default=os.environ.get("TGNN_BENCH_MATH", "fp32"), choices=["fp32", "tf32"])
+    ap.add_argument("--cpu-budget", type=float, default=20.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback); use --impl reference for the CPU oracle")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        torch.distributed.init_process_group("nccl", device_id=device)
+    try:
+        run_ours(args, rank, world, device)
+    finally:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

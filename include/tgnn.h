@@ -1,0 +1,244 @@
+/*
+ * tgnn.h -- C ABI of the B200 (sm_100a) training-step library for a TGN-style
+ * memory-based temporal graph network.
+ *
+ * One chronological training step over a mixed event batch (target events plus
+ * flagged auxiliary replay events), as framed by the paper:
+ *   events e=(u,v,t,x) sorted by t, node memory m_u(t)         Section III-A
+ *   Message / Update recursion                                   Eq. 1, Eq. 2
+ *   mixed batch with an event-type mask                          Eq. 5
+ *   pruning set and pruned batch                                 Eq. 10, Eq. 11
+ *   target mask and masked loss                                  Eq. 12, Eq. 13
+ *   per-batch order (prune, execute in timestamp order, masked
+ *   loss, backprop + gradient norm g_r, parameter update)        Algorithm 2
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer BORROWED from the caller unless the
+ *     parameter name ends in `_host`.  The library owns only the workspace it
+ *     allocates in tgnn_create (sized from the capacities in tgnn_config) and
+ *     never allocates afterwards.
+ *   - All work is enqueued on the caller's stream (`stream` is a cudaStream_t
+ *     passed as void*); no call synchronises the device unless documented.
+ *   - Every function returns TGNN_OK or a negative error code; the message of
+ *     the last error of a context is available from tgnn_last_error.  Invalid
+ *     arguments are rejected on the host before anything is launched.
+ *   - A context is used from one host thread at a time, on one stream.
+ *   - Node ids are int32 in [0, num_nodes); event ids are int32 positions in
+ *     the time-sorted stream; timestamps are fp64 wherever they are compared
+ *     or subtracted.
+ *
+ * Model (the paper leaves internals open; these are the textbook forms)
+ *   d = memory = time-encoding = embedding dimension, d_e = edge-feature
+ *   dimension, d_msg = 3d + d_e, d_kv = 2d + d_e, heads H, k neighbors.
+ *   Phi(dt)_c = cos(fmaf(w_c, (float)dt, b_c)), dt formed in fp64, argument in fp32.
+ *   Parameters live in ONE flat fp32 vector, matrices [out, in] row-major, in
+ *   this order (tgnn_param_layout reports the offsets):
+ *     time_w[d] time_b[d]
+ *     gru_w_i[3d,d_msg] gru_w_h[3d,d] gru_b_i[3d] gru_b_h[3d]     gates r,z,n
+ *     w_q[d,2d] b_q[d]  w_k[d,d_kv] w_v[d,d_kv] b_k[d] b_v[d]  w_o[d,2d] b_o[d]
+ *     w_1[d,2d] b_1[d] w_2[d] b_2[1]
+ */
+#ifndef TGNN_H_
+#define TGNN_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  TGNN_OK = 0,
+  TGNN_EINVAL = -1,    /* null pointer or value out of range */
+  TGNN_ESHAPE = -2,    /* dimensions inconsistent with the configuration */
+  TGNN_ECAPACITY = -3, /* n exceeds a capacity given at tgnn_create */
+  TGNN_ESTATE = -4,    /* call out of order (graph/state not set, no forward before backward ...) */
+  TGNN_ECUDA = -5,     /* a CUDA runtime call failed; see tgnn_last_error */
+  TGNN_ETIMEOUT = -6,  /* a bounded device-side wait expired (reported through tgnn_status) */
+  TGNN_EBOUNDS = -7    /* a device-side index check failed (reported through tgnn_status) */
+};
+
+enum { TGNN_F32 = 0, TGNN_BF16 = 1 };
+
+/* math_mode: how the dense projections are computed.  Gates, softmax, loss, the
+ * time encoding and Adam are always fp32. */
+enum {
+  TGNN_MATH_FP32 = 0, /* fp32 FMA tiles */
+  TGNN_MATH_TF32 = 1  /* tcgen05 tensor cores, TF32 operands, fp32 accumulation in TMEM */
+};
+
+#if defined(__GNUC__)
+#define TGNN_API __attribute__((visibility("default")))
+#else
+#define TGNN_API
+#endif
+
+typedef struct tgnn_ctx tgnn_ctx;
+
+typedef struct {
+  int64_t num_nodes;
+  int32_t d;          /* memory / time / embedding dimension, multiple of 4 and of heads */
+  int32_t d_e;        /* edge-feature dimension, >= 0, even */
+  int32_t k;          /* neighbors per root, 1..32 */
+  int32_t heads;      /* attention heads */
+  int32_t feat_dtype; /* TGNN_F32 or TGNN_BF16 */
+  int32_t max_events; /* capacity: events in one mixed batch */
+  int32_t max_roots;  /* capacity: roots in one tgnn_embed call (3 per target event) */
+  int32_t math_mode;  /* TGNN_MATH_* */
+  float lr, beta1, beta2, eps; /* Adam */
+} tgnn_config;
+
+/* ---- life cycle --------------------------------------------------------- */
+
+/* Allocates the context and all device workspace on the current device.
+ * cfg_host is read during the call only.  On failure *out is NULL. */
+TGNN_API int tgnn_create(const tgnn_config* cfg_host, tgnn_ctx** out);
+/* Frees the workspace.  Synchronises the device.  NULL is accepted. */
+TGNN_API int tgnn_destroy(tgnn_ctx* ctx);
+/* Message of the last error recorded in ctx (static string if ctx is NULL). Never NULL. */
+TGNN_API const char* tgnn_last_error(const tgnn_ctx* ctx);
+
+/* Number of fp32 parameters, and the offsets of the 18 tensors in layout order
+ * followed by the total (out19_host has 19 entries).  Pure host computations. */
+TGNN_API int64_t tgnn_param_count(const tgnn_config* cfg_host);
+TGNN_API int tgnn_param_layout(const tgnn_config* cfg_host, int64_t* out19_host);
+
+/* Time-sorted adjacency (T-CSR) of the whole stream, both directions of every
+ * event: node n owns entries [indptr[n], indptr[n+1]) sorted by (ts, eid).
+ * indptr:int64[num_nodes+1], nbr,eid:int32[n_entries], ts:f64[n_entries].
+ * Borrowed until replaced or the context is destroyed. */
+TGNN_API int tgnn_set_graph(tgnn_ctx* ctx, const int64_t* indptr, const int32_t* nbr, const int32_t* eid, const double* ts,
+                   int64_t n_entries);
+/* Edge-feature table [num_events, d_e] row-major, fp32 or bf16 per dtype (must
+ * equal cfg.feat_dtype); may be NULL when d_e == 0.  Borrowed. */
+TGNN_API int tgnn_set_edge_features(tgnn_ctx* ctx, const void* efeat, int dtype, int64_t num_events, int d_e);
+/* Model state, mutated in place by tgnn_memory_update and tgnn_backward_step:
+ * memory:f32[num_nodes,d], last_update:f64[num_nodes], params/adam_m/adam_v:
+ * f32[param_count], step:int64[1] (Adam step counter, device).  Borrowed.
+ * Call again after changing params from outside (cached operand copies are refreshed). */
+TGNN_API int tgnn_set_state(tgnn_ctx* ctx, float* memory, double* last_update, float* params, float* adam_m, float* adam_v,
+                   int64_t* step);
+
+/* ---- the step ------------------------------------------------------------ */
+
+/* Step (0): load-aware pruning of auxiliary replay events (Eq. 10-11) on a
+ * mixed batch (Eq. 5).  cnt[v] = endpoint occurrences of node v among the n
+ * events, T = number of nodes with cnt > 0; heavy = (max cnt * T > 8 n), i.e.
+ * "max > 4 x mean over touched nodes", unless force_heavy is 0 or 1, in which
+ * case the caller's flag H (e.g. the batch-time EMA rule of Eq. 9) is used.
+ * keep_out[i] = 1 for every target event (is_aux[i] == 0; targets are never
+ * pruned).  A replay event is dropped iff heavy and (drop_q32 == 0xFFFFFFFF,
+ * meaning all of them as in Eq. 11, or hash32(seed, batch_idx, eid[i]) <
+ * drop_q32), where hash32 = top 32 bits of the SplitMix64 finaliser applied to
+ * seed ^ batch_idx*0x9E3779B97F4A7C15 ^ (uint32)eid*0xC2B2AE3D27D4EB4F.
+ * src,dst,eid:int32[n], is_aux:uint8[n] -> keep_out:uint8[n], heavy_out:int32[1]. */
+TGNN_API int tgnn_prune_mask(tgnn_ctx* ctx, const int32_t* src, const int32_t* dst, const int32_t* eid, const uint8_t* is_aux,
+                    int n, int force_heavy, uint32_t drop_q32, uint64_t seed, int64_t batch_idx, uint8_t* keep_out,
+                    int32_t* heavy_out, void* stream);
+
+/* Step (1): most-recent-k temporal neighbor search ("temporal neighborhood
+ * aggregation", Section VI-A model description).  For root i, p = first index
+ * of node nodes[i]'s T-CSR slice with ts[p] >= times[i]; cnt = min(k, p -
+ * indptr[node]); slot s < cnt is entry p-1-s (slot 0 most recent); unused
+ * slots hold nbr = eid = -1, ts = 0.
+ * nodes:int32[n], times:f64[n] -> nbr_out,eid_out:int32[n,k], ts_out:f64[n,k], cnt_out:int32[n]. */
+TGNN_API int tgnn_sample_recent(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n, int32_t* nbr_out,
+                       int32_t* eid_out, double* ts_out, int32_t* cnt_out, void* stream);
+
+/* Step (2): Message of Eq. 1 for the n update events (the previous kept mixed
+ * batch): message 2i goes to src[i] (role 0), 2i+1 to dst[i] (role 1), layout
+ * [m_self || m_other || x_eid || Phi(t - last_update[self])], memory and
+ * last_update as they stand when the kernel runs.  keep may be NULL (all kept);
+ * events with keep[i] == 0 give msg_node = -1 and zero rows.
+ * msg_node_out:int32[2n] is always written.  msg_out:f32[2n,d_msg] may be NULL:
+ * the rows then stay virtual and tgnn_memory_update gathers the winners' rows
+ * itself from the event arrays, which must stay valid until that call is enqueued. */
+TGNN_API int tgnn_build_messages(tgnn_ctx* ctx, const int32_t* src, const int32_t* dst, const double* t, const int32_t* eid,
+                        const uint8_t* keep, int n, float* msg_out, int32_t* msg_node_out, void* stream);
+
+/* Step (3): per-node latest-event reduction.  Message j belongs to event j>>1
+ * with role j&1; t,eid are per event ([n_msg/2]).  For every node with a
+ * message (msg_node >= 0) the winner is the message with the lexicographically
+ * largest (t, eid, role).  uniq_out:int32[<=n_msg] touched nodes ascending,
+ * winner_out:int32[<=n_msg] message index per unique node, n_uniq_out:int32[1]. */
+TGNN_API int tgnn_reduce_latest(tgnn_ctx* ctx, const int32_t* msg_node, const double* t, const int32_t* eid, int n_msg,
+                       int32_t* uniq_out, int32_t* winner_out, int32_t* n_uniq_out, void* stream);
+
+/* Step (4): Update of Eq. 2 as a GRU cell (gate order r,z,n; r multiplies the
+ * hidden candidate pre-activation including its bias) on the winners:
+ * memory[uniq[u]] <- GRU(msg[winner[u]], memory[uniq[u]]), last_update[uniq[u]]
+ * <- t[winner[u]>>1]; every new row is computed from pre-call memory before any
+ * row is written.  msg may be NULL if tgnn_build_messages ran with msg_out NULL
+ * (rows are gathered from its event arrays).  Activations are kept in the
+ * workspace for tgnn_backward_step.  n_uniq is a device scalar. */
+TGNN_API int tgnn_memory_update(tgnn_ctx* ctx, const float* msg, const int32_t* uniq, const int32_t* winner,
+                       const int32_t* n_uniq, void* stream);
+
+/* Step (5): one multi-head temporal attention layer.  For root i: query from
+ * [m_root || Phi(0)], keys/values from [m_nbr || x_eid || Phi(times[i] - ts)] of
+ * its cnt[i] valid neighbor slots, softmax over valid slots of q.k/sqrt(d/H) per
+ * head (zero vector if cnt = 0), h = ReLU(W_o [a || m_root] + b_o).
+ * Inputs as produced by tgnn_sample_recent -> h_out:f32[n,d].  Activations are
+ * kept for tgnn_backward_step; the neighbor arrays must stay valid until then. */
+TGNN_API int tgnn_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n, const int32_t* nbr, const int32_t* eid,
+               const double* ts, const int32_t* cnt, float* h_out, void* stream);
+
+/* Step (6): masked link-prediction loss (Eq. 13) on the rows of the last
+ * tgnn_embed call, laid out as [src | dst | neg] blocks of n_q rows:
+ *   score(a,b) = w_2 . ReLU(W_1 [a || b] + b_1) + b_2,
+ *   l_j = softplus(-score(src_j,dst_j)) + softplus(score(src_j,neg_j)),
+ *   L = sum_j M_j l_j / sum_j M_j, or 0 if no event has M_j = 1,
+ * loss_mask:uint8[n_q] (NULL = all ones) being the target mask of Eq. 12; then
+ * the exact gradient w.r.t. all parameters (rows written by the last
+ * tgnn_memory_update depend on the GRU and time-encoder parameters, all other
+ * table reads are constants), the gradient norm g_r = ||grad||_2 (Algorithm 2,
+ * "compute gradient norm") and one Adam step (step += 1, bias-corrected, no
+ * weight decay).  loss_out, gradnorm_out: f32 device scalars (may be NULL). */
+TGNN_API int tgnn_backward_step(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* loss_out, float* gradnorm_out,
+                       void* stream);
+
+/* ---- whole step, one call ------------------------------------------------- */
+
+/* Runs steps (1)-(6) in lag-one order on device-resident event arrays:
+ * the update events (previous kept batch: u_src..u_keep, n_u, may be 0) refresh
+ * memory, then the n_q target events (q_src,q_dst,q_neg:int32[n_q], q_t:f64[n_q])
+ * are sampled, embedded, scored and trained on.  Equivalent to calling the six
+ * entry points above with workspace-owned intermediates. */
+TGNN_API int tgnn_train_step(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, const double* u_t, const int32_t* u_eid,
+                    const uint8_t* u_keep, int n_u, const int32_t* q_src, const int32_t* q_dst, const int32_t* q_neg,
+                    const double* q_t, int n_q, const uint8_t* loss_mask, float* loss_out, float* gradnorm_out,
+                    void* stream);
+
+/* The same step with HOST inputs and outputs: the event arrays are copied to
+ * workspace staging buffers with cudaMemcpyAsync (pin them for overlap), and
+ * loss / gradient norm are copied back to loss_host / gradnorm_host (may be
+ * NULL).  The call returns after enqueueing; synchronise the stream before
+ * reading the two scalars or reusing the host buffers. */
+TGNN_API int tgnn_train_step_host(tgnn_ctx* ctx, const int32_t* u_src_host, const int32_t* u_dst_host, const double* u_t_host,
+                         const int32_t* u_eid_host, const uint8_t* u_keep_host, int n_u, const int32_t* q_src_host,
+                         const int32_t* q_dst_host, const int32_t* q_neg_host, const double* q_t_host, int n_q,
+                         const uint8_t* loss_mask_host, float* loss_host, float* gradnorm_host, void* stream);
+
+/* ---- debug / parity -------------------------------------------------------- */
+
+/* Copies the parameter gradient of the last tgnn_backward_step to grads_out:f32[param_count]. */
+TGNN_API int tgnn_debug_get_grads(tgnn_ctx* ctx, float* grads_out, void* stream);
+/* Device status word (0 or the first TGNN_ETIMEOUT / TGNN_EBOUNDS recorded by a
+ * kernel) copied to *status_host.  Synchronises the stream. */
+TGNN_API int tgnn_status(tgnn_ctx* ctx, int32_t* status_host, void* stream);
+/* Number of kernels this context has launched since creation (host counter). */
+TGNN_API int64_t tgnn_kernel_launches(const tgnn_ctx* ctx);
+
+/* Per-kernel timing for benchmarks (no counterpart in the paper beyond its
+ * per-phase time breakdown, Table 5).  After tgnn_profile_begin every kernel
+ * launch is bracketed by a CUDA event pair on the caller's stream until
+ * tgnn_profile_report, which synchronises the device, writes one line per kernel
+ * name ("name launches total_ms\n", NUL-terminated, truncated to size bytes)
+ * into buf_host and switches profiling off.  Creates events on first use. */
+TGNN_API int tgnn_profile_begin(tgnn_ctx* ctx);
+TGNN_API int tgnn_profile_report(tgnn_ctx* ctx, char* buf_host, int64_t size);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TGNN_H_ */

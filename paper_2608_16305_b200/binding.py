@@ -1,0 +1,274 @@
+"""Thin ctypes binding of libtgnn_b200.so: same names as the C ABI, argument
+marshalling only.  torch is used for device memory and streams; every step of
+the path runs in the library's CUDA kernels.  There is no CPU fallback: loading
+fails loudly when the shared library is missing."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtgnn_b200.so")
+
+TGNN_OK, TGNN_EINVAL, TGNN_ESHAPE, TGNN_ECAPACITY, TGNN_ESTATE, TGNN_ECUDA, TGNN_ETIMEOUT, TGNN_EBOUNDS = (
+    0, -1, -2, -3, -4, -5, -6, -7)
+TGNN_F32, TGNN_BF16 = 0, 1
+TGNN_MATH_FP32, TGNN_MATH_TF32 = 0, 1
+
+PARAM_NAMES = ("time_w", "time_b", "gru_w_i", "gru_w_h", "gru_b_i", "gru_b_h", "w_q", "b_q", "w_k", "w_v",
+               "b_k", "b_v", "w_o", "b_o", "w_1", "b_1", "w_2", "b_2")
+
+EXPORTS = ("tgnn_create", "tgnn_destroy", "tgnn_last_error", "tgnn_param_count", "tgnn_param_layout",
+           "tgnn_set_graph", "tgnn_set_edge_features", "tgnn_set_state", "tgnn_prune_mask", "tgnn_sample_recent",
+           "tgnn_build_messages", "tgnn_reduce_latest", "tgnn_memory_update", "tgnn_embed", "tgnn_backward_step",
+           "tgnn_train_step", "tgnn_train_step_host", "tgnn_debug_get_grads", "tgnn_status", "tgnn_kernel_launches", "tgnn_profile_begin",
+           "tgnn_profile_report")
+
+
+class TgnnConfig(C.Structure):
+    _fields_ = [("num_nodes", C.c_int64), ("d", C.c_int32), ("d_e", C.c_int32), ("k", C.c_int32),
+                ("heads", C.c_int32), ("feat_dtype", C.c_int32), ("max_events", C.c_int32),
+                ("max_roots", C.c_int32), ("math_mode", C.c_int32),
+                ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float)]
+
+
+class TgnnError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"tgnn error {code}: {msg}")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library():
+    """Loads the CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2608_16305_b200.build` "
+                               "(there is no CPU fallback)")
+        lib = C.CDLL(LIB_PATH)
+        vp, i32, i64, u32, u64 = C.c_void_p, C.c_int, C.c_int64, C.c_uint32, C.c_uint64
+        lib.tgnn_create.argtypes = [C.POINTER(TgnnConfig), C.POINTER(vp)]
+        lib.tgnn_destroy.argtypes = [vp]
+        lib.tgnn_last_error.argtypes = [vp]
+        lib.tgnn_last_error.restype = C.c_char_p
+        lib.tgnn_param_count.argtypes = [C.POINTER(TgnnConfig)]
+        lib.tgnn_param_count.restype = i64
+        lib.tgnn_param_layout.argtypes = [C.POINTER(TgnnConfig), vp]
+        lib.tgnn_set_graph.argtypes = [vp, vp, vp, vp, vp, i64]
+        lib.tgnn_set_edge_features.argtypes = [vp, vp, i32, i64, i32]
+        lib.tgnn_set_state.argtypes = [vp] * 7
+        lib.tgnn_prune_mask.argtypes = [vp, vp, vp, vp, vp, i32, i32, u32, u64, i64, vp, vp, vp]
+        lib.tgnn_sample_recent.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp]
+        lib.tgnn_build_messages.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
+        lib.tgnn_reduce_latest.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp]
+        lib.tgnn_memory_update.argtypes = [vp, vp, vp, vp, vp, vp]
+        lib.tgnn_embed.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
+        lib.tgnn_backward_step.argtypes = [vp, i32, vp, vp, vp, vp]
+        lib.tgnn_train_step.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, i32, vp, vp, vp, vp]
+        lib.tgnn_train_step_host.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, i32, vp, vp, vp, vp]
+        lib.tgnn_debug_get_grads.argtypes = [vp, vp, vp]
+        lib.tgnn_status.argtypes = [vp, vp, vp]
+        lib.tgnn_kernel_launches.argtypes = [vp]
+        lib.tgnn_kernel_launches.restype = i64
+        lib.tgnn_profile_begin.argtypes = [vp]
+        lib.tgnn_profile_report.argtypes = [vp, vp, i64]
+        _lib = lib
+    return _lib
+
+
+_TORCH_DT = {"i32": torch.int32, "i64": torch.int64, "f32": torch.float32, "f64": torch.float64, "u8": torch.uint8,
+             "bf16": torch.bfloat16}
+
+
+def _dp(t: Optional[torch.Tensor], dt: str, name: str):
+    """Device pointer of a contiguous CUDA tensor of the expected dtype (None -> NULL)."""
+    if t is None:
+        return None
+    if not t.is_cuda or t.dtype != _TORCH_DT[dt] or not t.is_contiguous():
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of dtype {dt}, got {t.dtype} on {t.device}")
+    return t.data_ptr()
+
+
+def _hp(t: Optional[torch.Tensor], dt: str, name: str):
+    if t is None:
+        return None
+    if t.is_cuda or t.dtype != _TORCH_DT[dt] or not t.is_contiguous():
+        raise TypeError(f"{name}: expected a contiguous host tensor of dtype {dt}")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def make_config(num_nodes, d, d_e, k, heads, feat_dtype=TGNN_F32, max_events=1024, max_roots=3072,
+                math_mode=TGNN_MATH_FP32, lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8) -> TgnnConfig:
+    return TgnnConfig(num_nodes, d, d_e, k, heads, feat_dtype, max_events, max_roots, math_mode, lr, beta1, beta2, eps)
+
+
+def param_layout(cfg: TgnnConfig) -> Dict[str, int]:
+    out = np.zeros(19, dtype=np.int64)
+    rc = load_library().tgnn_param_layout(C.byref(cfg), out.ctypes.data)
+    if rc != TGNN_OK:
+        raise TgnnError(rc, "invalid configuration")
+    lay = {n: int(out[i]) for i, n in enumerate(PARAM_NAMES)}
+    lay["total"] = int(out[18])
+    return lay
+
+
+def pack_params(cfg: TgnnConfig, weights: Dict[str, np.ndarray]) -> np.ndarray:
+    lay = param_layout(cfg)
+    flat = np.zeros(lay["total"], dtype=np.float32)
+    for n in PARAM_NAMES:
+        w = np.asarray(weights[n], dtype=np.float32).ravel()
+        flat[lay[n]:lay[n] + w.size] = w
+    return flat
+
+
+class Tgnn:
+    """One library context.  Methods mirror the C entry points one to one."""
+
+    def __init__(self, cfg: TgnnConfig):
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required (there is no CPU fallback)")
+        self.lib = load_library()
+        self.cfg = cfg
+        self._h = C.c_void_p()
+        rc = self.lib.tgnn_create(C.byref(cfg), C.byref(self._h))
+        if rc != TGNN_OK:
+            raise TgnnError(rc, "tgnn_create failed (invalid configuration, not an sm_100 device, or out of memory)")
+        self._keep = {}     # tensors the library borrows: keep them alive
+
+    def close(self):
+        if self._h:
+            self.lib.tgnn_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _ck(self, rc: int):
+        if rc != TGNN_OK:
+            raise TgnnError(rc, self.lib.tgnn_last_error(self._h).decode())
+
+    def call_raw(self, name: str, *args) -> int:
+        """Calls an entry point and returns its code without raising (error-path tests)."""
+        return getattr(self.lib, name)(self._h, *args)
+
+    def last_error(self) -> str:
+        return self.lib.tgnn_last_error(self._h).decode()
+
+    def kernel_launches(self) -> int:
+        return int(self.lib.tgnn_kernel_launches(self._h))
+
+    # ---- set-up ----
+    def set_graph(self, indptr, nbr, eid, ts):
+        self._keep["graph"] = (indptr, nbr, eid, ts)
+        self._ck(self.lib.tgnn_set_graph(self._h, _dp(indptr, "i64", "indptr"), _dp(nbr, "i32", "nbr"),
+                                         _dp(eid, "i32", "eid"), _dp(ts, "f64", "ts"), nbr.numel()))
+
+    def set_edge_features(self, efeat: Optional[torch.Tensor], num_events: int):
+        self._keep["efeat"] = efeat
+        dt = "bf16" if self.cfg.feat_dtype == TGNN_BF16 else "f32"
+        self._ck(self.lib.tgnn_set_edge_features(self._h, _dp(efeat, dt, "efeat") if self.cfg.d_e else None,
+                                                 self.cfg.feat_dtype, num_events, self.cfg.d_e))
+
+    def set_state(self, memory, last_update, params, adam_m, adam_v, step):
+        self._keep["state"] = (memory, last_update, params, adam_m, adam_v, step)
+        self._ck(self.lib.tgnn_set_state(self._h, _dp(memory, "f32", "memory"), _dp(last_update, "f64", "last_update"),
+                                         _dp(params, "f32", "params"), _dp(adam_m, "f32", "adam_m"),
+                                         _dp(adam_v, "f32", "adam_v"), _dp(step, "i64", "step")))
+
+    # ---- the step ----
+    def prune_mask(self, src, dst, eid, is_aux, keep_out, heavy_out, force_heavy=-1, drop_q32=1 << 31, seed=0,
+                   batch_idx=0):
+        self._ck(self.lib.tgnn_prune_mask(self._h, _dp(src, "i32", "src"), _dp(dst, "i32", "dst"), _dp(eid, "i32", "eid"),
+                                          _dp(is_aux, "u8", "is_aux"), src.numel(), force_heavy, drop_q32, seed,
+                                          batch_idx, _dp(keep_out, "u8", "keep_out"), _dp(heavy_out, "i32", "heavy_out"),
+                                          _stream()))
+
+    def sample_recent(self, nodes, times, nbr_out, eid_out, ts_out, cnt_out):
+        self._ck(self.lib.tgnn_sample_recent(self._h, _dp(nodes, "i32", "nodes"), _dp(times, "f64", "times"),
+                                             nodes.numel(), _dp(nbr_out, "i32", "nbr_out"), _dp(eid_out, "i32", "eid_out"),
+                                             _dp(ts_out, "f64", "ts_out"), _dp(cnt_out, "i32", "cnt_out"), _stream()))
+
+    def build_messages(self, src, dst, t, eid, keep, msg_out, msg_node_out):
+        self._keep["upd"] = (src, dst, t, eid, keep)
+        self._ck(self.lib.tgnn_build_messages(self._h, _dp(src, "i32", "src"), _dp(dst, "i32", "dst"), _dp(t, "f64", "t"),
+                                              _dp(eid, "i32", "eid"), _dp(keep, "u8", "keep"), src.numel(),
+                                              _dp(msg_out, "f32", "msg_out"), _dp(msg_node_out, "i32", "msg_node_out"),
+                                              _stream()))
+
+    def reduce_latest(self, msg_node, t, eid, uniq_out, winner_out, n_uniq_out):
+        self._ck(self.lib.tgnn_reduce_latest(self._h, _dp(msg_node, "i32", "msg_node"), _dp(t, "f64", "t"),
+                                             _dp(eid, "i32", "eid"), msg_node.numel(), _dp(uniq_out, "i32", "uniq_out"),
+                                             _dp(winner_out, "i32", "winner_out"), _dp(n_uniq_out, "i32", "n_uniq_out"),
+                                             _stream()))
+
+    def memory_update(self, msg, uniq, winner, n_uniq):
+        self._keep["upd_idx"] = (msg, uniq, winner, n_uniq)
+        self._ck(self.lib.tgnn_memory_update(self._h, _dp(msg, "f32", "msg"), _dp(uniq, "i32", "uniq"),
+                                             _dp(winner, "i32", "winner"), _dp(n_uniq, "i32", "n_uniq"), _stream()))
+
+    def embed(self, nodes, times, nbr, eid, ts, cnt, h_out):
+        self._keep["embed"] = (nodes, times, nbr, eid, ts, cnt, h_out)
+        self._ck(self.lib.tgnn_embed(self._h, _dp(nodes, "i32", "nodes"), _dp(times, "f64", "times"), nodes.numel(),
+                                     _dp(nbr, "i32", "nbr"), _dp(eid, "i32", "eid"), _dp(ts, "f64", "ts"),
+                                     _dp(cnt, "i32", "cnt"), _dp(h_out, "f32", "h_out"), _stream()))
+
+    def backward_step(self, n_q, loss_mask, loss_out, gradnorm_out):
+        self._ck(self.lib.tgnn_backward_step(self._h, n_q, _dp(loss_mask, "u8", "loss_mask"),
+                                             _dp(loss_out, "f32", "loss_out"), _dp(gradnorm_out, "f32", "gradnorm_out"),
+                                             _stream()))
+
+    def train_step(self, u_src, u_dst, u_t, u_eid, u_keep, q_src, q_dst, q_neg, q_t, loss_mask, loss_out, gradnorm_out):
+        n_u = 0 if u_src is None else u_src.numel()
+        self._ck(self.lib.tgnn_train_step(self._h, _dp(u_src, "i32", "u_src"), _dp(u_dst, "i32", "u_dst"),
+                                          _dp(u_t, "f64", "u_t"), _dp(u_eid, "i32", "u_eid"), _dp(u_keep, "u8", "u_keep"),
+                                          n_u, _dp(q_src, "i32", "q_src"), _dp(q_dst, "i32", "q_dst"),
+                                          _dp(q_neg, "i32", "q_neg"), _dp(q_t, "f64", "q_t"), q_src.numel(),
+                                          _dp(loss_mask, "u8", "loss_mask"), _dp(loss_out, "f32", "loss_out"),
+                                          _dp(gradnorm_out, "f32", "gradnorm_out"), _stream()))
+
+    def train_step_host(self, u_src, u_dst, u_t, u_eid, u_keep, q_src, q_dst, q_neg, q_t, loss_mask, loss_host,
+                        gradnorm_host):
+        n_u = 0 if u_src is None else u_src.numel()
+        self._ck(self.lib.tgnn_train_step_host(self._h, _hp(u_src, "i32", "u_src"), _hp(u_dst, "i32", "u_dst"),
+                                               _hp(u_t, "f64", "u_t"), _hp(u_eid, "i32", "u_eid"),
+                                               _hp(u_keep, "u8", "u_keep"), n_u, _hp(q_src, "i32", "q_src"),
+                                               _hp(q_dst, "i32", "q_dst"), _hp(q_neg, "i32", "q_neg"),
+                                               _hp(q_t, "f64", "q_t"), q_src.numel(), _hp(loss_mask, "u8", "loss_mask"),
+                                               _hp(loss_host, "f32", "loss_host"), _hp(gradnorm_host, "f32", "gradnorm_host"),
+                                               _stream()))
+
+    # ---- debug ----
+    def debug_get_grads(self, grads_out):
+        self._ck(self.lib.tgnn_debug_get_grads(self._h, _dp(grads_out, "f32", "grads_out"), _stream()))
+
+    def profile_begin(self):
+        self._ck(self.lib.tgnn_profile_begin(self._h))
+
+    def profile_report(self) -> Dict[str, tuple]:
+        """{kernel name: (launches, total_ms)} since profile_begin; switches profiling off."""
+        buf = C.create_string_buffer(1 << 16)
+        self._ck(self.lib.tgnn_profile_report(self._h, C.addressof(buf), len(buf)))
+        out = {}
+        for line in buf.value.decode().splitlines():
+            name, cnt, ms = line.rsplit(" ", 2)
+            out[name] = (int(cnt), float(ms))
+        return out
+
+    def status(self) -> int:
+        out = C.c_int32(0)
+        self._ck(self.lib.tgnn_status(self._h, C.addressof(out), _stream()))
+        return int(out.value)

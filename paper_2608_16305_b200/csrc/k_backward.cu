@@ -1,0 +1,436 @@
+// Step (6): masked link-prediction loss (Eq. 13), exact backward of steps (4)-(5),
+// gradient norm g_r and the Adam update.
+#include "tgnn_internal.cuh"
+#include "tgnn_device.cuh"
+
+namespace tgnn {
+namespace {
+
+constexpr unsigned FULL = 0xffffffffu;
+
+// cat1[p] = [h_src || h_dst] for p < nq (positive pairs), [h_src || h_neg] for p >= nq.
+__global__ void __launch_bounds__(256) head_gather_kernel(const float* __restrict__ h, int nq, int d,
+                                                          float* __restrict__ cat1) {
+  const int64_t total = (int64_t)2 * nq * 2 * d;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int p = (int)(e / (2 * d)), q = (int)(e % (2 * d));
+    const int j = p < nq ? p : p - nq;
+    const int row = q < d ? j : (p < nq ? nq + j : 2 * nq + j);
+    cat1[e] = h[(int64_t)row * d + (q < d ? q : q - d)];
+  }
+}
+
+// One warp per target event: both scores, the event's loss term, d loss / d score, then
+// hid1 is overwritten by d loss / d pre1.  Accumulates dw_2, db_2 and the loss.
+__global__ void __launch_bounds__(256) head_loss_kernel(float* __restrict__ hid1, const float* __restrict__ w2,
+                                                        const float* __restrict__ b2,
+                                                        const uint8_t* __restrict__ loss_mask, int nq, int d,
+                                                        float* __restrict__ g_w2, float* __restrict__ g_b2,
+                                                        float* __restrict__ loss_acc) {
+  extern __shared__ float s_gw2[];  // [d]
+  __shared__ float s_msum;
+  __shared__ float s_gb2, s_loss;
+  const int lane = threadIdx.x & 31;
+  for (int q = threadIdx.x; q < d; q += blockDim.x) s_gw2[q] = 0.f;
+  if (threadIdx.x == 0) { s_msum = 0.f; s_gb2 = 0.f; s_loss = 0.f; }
+  __syncthreads();
+  {  // every block counts the whole mask (a few KB)
+    int c = 0;
+    for (int j = threadIdx.x; j < nq; j += blockDim.x) c += loss_mask ? (loss_mask[j] != 0) : 1;
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(FULL, c, o);
+    if (lane == 0 && c) atomicAdd(&s_msum, (float)c);
+  }
+  __syncthreads();
+  const float msum = s_msum;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  for (int j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; j < nq; j += warps) {
+    const float m = (loss_mask ? (loss_mask[j] != 0) : 1) ? 1.f : 0.f;
+    const float wj = msum > 0.f ? m / msum : 0.f;
+    float* hp = hid1 + (int64_t)j * d;
+    float* hn = hid1 + (int64_t)(nq + j) * d;
+    float sp = 0.f, sn = 0.f;
+    for (int q = lane; q < d; q += 32) {
+      sp = fmaf(w2[q], hp[q], sp);
+      sn = fmaf(w2[q], hn[q], sn);
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+      sp += __shfl_xor_sync(FULL, sp, o);
+      sn += __shfl_xor_sync(FULL, sn, o);
+    }
+    sp += b2[0];
+    sn += b2[0];
+    const float dsp = -wj * sigmoidf_(-sp);
+    const float dsn = wj * sigmoidf_(sn);
+    if (lane == 0) {
+      atomicAdd(&s_loss, wj * (softplusf_(-sp) + softplusf_(sn)));
+      atomicAdd(&s_gb2, dsp + dsn);
+    }
+    for (int q = lane; q < d; q += 32) {
+      const float a = hp[q], b = hn[q];
+      if (wj != 0.f) atomicAdd(&s_gw2[q], dsp * a + dsn * b);
+      hp[q] = a > 0.f ? dsp * w2[q] : 0.f;
+      hn[q] = b > 0.f ? dsn * w2[q] : 0.f;
+    }
+  }
+  __syncthreads();
+  for (int q = threadIdx.x; q < d; q += blockDim.x)
+    if (s_gw2[q] != 0.f) atomicAdd(&g_w2[q], s_gw2[q]);
+  if (threadIdx.x == 0) {
+    if (s_gb2 != 0.f) atomicAdd(g_b2, s_gb2);
+    if (s_loss != 0.f) atomicAdd(loss_acc, s_loss);
+  }
+}
+
+// d loss / d pre_o = ReLU'(h) * d loss / d h, where dh collects the head's input gradients.
+__global__ void __launch_bounds__(256) dh_kernel(const float* __restrict__ dcat1, const float* __restrict__ h, int nq,
+                                                 int d, float* __restrict__ dpre_o) {
+  const int64_t total = (int64_t)3 * nq * d;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int i = (int)(e / d), q = (int)(e % d);
+    float g;
+    if (i < nq)
+      g = dcat1[(int64_t)i * 2 * d + q] + dcat1[(int64_t)(nq + i) * 2 * d + q];
+    else if (i < 2 * nq)
+      g = dcat1[(int64_t)(i - nq) * 2 * d + d + q];
+    else
+      g = dcat1[(int64_t)(i - nq) * 2 * d + d + q];
+    dpre_o[e] = h[e] > 0.f ? g : 0.f;
+  }
+}
+
+// One warp per root: backward of the weighted sum, the softmax and the scaled dot products.
+__global__ void __launch_bounds__(256) attention_bwd_kernel(const float* __restrict__ Q, const float* __restrict__ KV,
+                                                            const float* __restrict__ alpha,
+                                                            const float* __restrict__ dcat_o,
+                                                            const int32_t* __restrict__ cnt, int n, int d, int H, int k,
+                                                            float* __restrict__ dQ, float* __restrict__ dKV) {
+  extern __shared__ float sm[];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int i = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+  if (i >= n) return;
+  float* dl = sm + wib * H * k;  // d loss / d logit (already scaled)
+  const int dh = d / H;
+  const int c = cnt[i];
+  const float scale = rsqrtf((float)dh);
+  const float* da = dcat_o + (int64_t)i * 2 * d;
+  const float* al = alpha + (int64_t)i * H * k;
+  for (int h = 0; h < H; ++h) {
+    float dot = 0.f;
+    for (int s = 0; s < c; ++s) {
+      const float* vr = KV + ((int64_t)i * k + s) * 2 * d + d + h * dh;
+      float a = 0.f;
+      for (int e = lane; e < dh; e += 32) a = fmaf(da[h * dh + e], vr[e], a);
+      for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(FULL, a, o);
+      if (lane == 0) dl[h * k + s] = a;
+      dot = fmaf(al[h * k + s], a, dot);
+    }
+    __syncwarp();
+    if (lane < c) dl[h * k + lane] = al[h * k + lane] * (dl[h * k + lane] - dot) * scale;
+    __syncwarp();
+  }
+  for (int e = lane; e < d; e += 32) {
+    const int h = e / dh;
+    const float qe = Q[(int64_t)i * d + e], dae = da[e];
+    float dq = 0.f;
+    for (int s = 0; s < k; ++s) {
+      float* row = dKV + ((int64_t)i * k + s) * 2 * d;
+      if (s < c) {
+        const float g = dl[h * k + s];
+        dq = fmaf(g, KV[((int64_t)i * k + s) * 2 * d + e], dq);
+        row[e] = g * qe;
+        row[d + e] = al[h * k + s] * dae;
+      } else {
+        row[e] = 0.f;
+        row[d + e] = 0.f;
+      }
+    }
+    dQ[(int64_t)i * d + e] = dq;
+  }
+}
+
+// Gradient rows flowing into memory rows that the last memory update wrote: one warp per
+// source row, added into dMemU[node2slot[node]].  Rows [0, nb_rows): dZm with node = nbr;
+// rows [nb_rows, nb_rows + n): the root's own row, dcat_o[:, d:] + dzq[:, :d].
+__global__ void __launch_bounds__(256) scatter_dmem_kernel(const float* __restrict__ dZm, const float* __restrict__ dcat_o,
+                                                           const float* __restrict__ dzq,
+                                                           const int32_t* __restrict__ nbr,
+                                                           const int32_t* __restrict__ nodes, int n, int k, int d,
+                                                           const int32_t* __restrict__ node2slot,
+                                                           float* __restrict__ dMemU) {
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  const int nb_rows = n * k;
+  for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < nb_rows + n; r += warps) {
+    const int node = r < nb_rows ? nbr[r] : nodes[r - nb_rows];
+    if (node < 0) continue;
+    const int slot = node2slot[node];
+    if (slot < 0) continue;
+    float* out = dMemU + (int64_t)slot * d;
+    if (r < nb_rows) {
+      const float* g = dZm + (int64_t)r * d;
+      for (int q = lane; q < d; q += 32) atomicAdd(&out[q], g[q]);
+    } else {
+      const int i = r - nb_rows;
+      const float* g1 = dcat_o + (int64_t)i * 2 * d + d;
+      const float* g2 = dzq + (int64_t)i * 2 * d;
+      for (int q = lane; q < d; q += 32) atomicAdd(&out[q], g1[q] + g2[q]);
+    }
+  }
+}
+
+// Time-encoder gradient from a block of rows: G[r, col0 + c] is d loss / d Phi(dt_r)_c.
+//   dw_c += -sin(arg) dt_r G,  db_c += -sin(arg) G,  arg = fmaf(w_c, dt_r, b_c)
+// Thread c walks the rows of the block's chunk; one pair of atomics per block and column.
+__global__ void __launch_bounds__(128) time_grad_kernel(const float* __restrict__ G, int64_t ldg, int col0,
+                                                        const float* __restrict__ dt, int rows,
+                                                        const int32_t* __restrict__ dev_rows, int rows_per_block, int d,
+                                                        const float* __restrict__ time_w, const float* __restrict__ time_b,
+                                                        float* __restrict__ g_w, float* __restrict__ g_b) {
+  const int R = dev_rows ? min(*dev_rows, rows) : rows;
+  const int r0 = blockIdx.x * rows_per_block, r1 = min(R, r0 + rows_per_block);
+  if (r0 >= r1) return;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float w = time_w[c], b = time_b[c];
+    float gw = 0.f, gb = 0.f;
+    for (int r = r0; r < r1; ++r) {
+      const float g = G[(int64_t)r * ldg + col0 + c];
+      if (g == 0.f) continue;
+      const float dtr = dt ? dt[r] : 0.f;
+      const float sn = -sinf(time_arg(w, b, dtr)) * g;
+      gw = fmaf(sn, dtr, gw);
+      gb += sn;
+    }
+    if (gw != 0.f) atomicAdd(&g_w[c], gw);
+    if (gb != 0.f) atomicAdd(&g_b[c], gb);
+  }
+}
+
+// Backward of the GRU gates for the rows the memory update wrote.
+__global__ void __launch_bounds__(256) gru_bwd_gate_kernel(const float* __restrict__ dMemU, const float* __restrict__ X,
+                                                           int ld, int d, const float* __restrict__ g_r,
+                                                           const float* __restrict__ g_z, const float* __restrict__ g_n,
+                                                           const float* __restrict__ g_hn,
+                                                           const int32_t* __restrict__ n_uniq, int u_cap,
+                                                           float* __restrict__ dGi, float* __restrict__ dGh) {
+  const int U = min(*n_uniq, u_cap);
+  const int64_t total = (int64_t)U * d;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int u = (int)(e / d), q = (int)(e % d);
+    const float g = dMemU[e];
+    const float r = g_r[e], z = g_z[e], nn = g_n[e];
+    const float h = X[(int64_t)u * ld + q];
+    const float dn = g * (1.f - z);
+    const float dz = g * (h - nn);
+    const float dpn = dn * (1.f - nn * nn);
+    const float dpz = dz * z * (1.f - z);
+    const float dpr = dpn * g_hn[e] * r * (1.f - r);
+    float* gi = dGi + (int64_t)u * 3 * d;
+    float* gh = dGh + (int64_t)u * 3 * d;
+    gi[q] = dpr; gi[d + q] = dpz; gi[2 * d + q] = dpn;
+    gh[q] = dpr; gh[d + q] = dpz; gh[2 * d + q] = dpn * r;
+  }
+}
+
+// Sum of squares of the gradient; the last block to finish turns it into g_r, bumps the Adam
+// step counter and prepares the bias corrections.
+__global__ void __launch_bounds__(256) gradnorm_kernel(const float* __restrict__ grads, int64_t P, double* red,
+                                                       unsigned int* ticket, int64_t* step, float beta1, float beta2,
+                                                       float* __restrict__ adam_sc, const float* __restrict__ loss_acc,
+                                                       float* scalars, float* loss_out, float* gradnorm_out) {
+  __shared__ double s_part[8];
+  double acc = 0.0;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < P; e += (int64_t)gridDim.x * blockDim.x) {
+    const double g = (double)grads[e];
+    acc = fma(g, g, acc);
+  }
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(FULL, acc, o);
+  if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double b = 0.0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) b += s_part[w];
+    atomicAdd(&red[0], b);
+    __threadfence();
+    const unsigned int done = atomicAdd(ticket, 1u);
+    if (done == gridDim.x - 1) {
+      __threadfence();
+      const double ss = atomicAdd(&red[0], 0.0);
+      const float gn = (float)sqrt(ss);
+      const int64_t t = step[0] + 1;
+      step[0] = t;
+      adam_sc[0] = (float)(1.0 / (1.0 - pow((double)beta1, (double)t)));
+      adam_sc[1] = (float)(1.0 / (1.0 - pow((double)beta2, (double)t)));
+      const float loss = *loss_acc;
+      scalars[0] = loss;
+      scalars[1] = gn;
+      if (loss_out) *loss_out = loss;
+      if (gradnorm_out) *gradnorm_out = gn;
+      *ticket = 0u;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) adam_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v,
+                                                   const float* __restrict__ g, int64_t P, float lr, float beta1,
+                                                   float beta2, float eps, const float* __restrict__ adam_sc) {
+  const float c1 = adam_sc[0], c2 = adam_sc[1];
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < P; e += (int64_t)gridDim.x * blockDim.x) {
+    const float ge = g[e];
+    const float me = fmaf(beta1, m[e], (1.f - beta1) * ge);
+    const float ve = fmaf(beta2, v[e], (1.f - beta2) * ge * ge);
+    m[e] = me;
+    v[e] = ve;
+    p[e] -= lr * (me * c1) / (sqrtf(ve * c2) + eps);
+  }
+}
+
+int pick_split(int M, int N, int K) {
+  const int tiles = ((M + 63) / 64) * ((N + 63) / 64);
+  int s = (4 * 148 + tiles - 1) / tiles;
+  const int max_s = (K + 127) / 128;
+  if (s > max_s) s = max_s;
+  return s < 1 ? 1 : s;
+}
+
+// dW[N_out, K_in] += dY^T A  (+ db[N_out] += column sums of dY): a transposed product with the
+// contraction over rows (optionally a device-side count).
+int grad_w(tgnn_ctx* ctx, const float* dY, int64_t ld_dy, const float* A, int64_t ld_a, int rows, const int32_t* dev_rows,
+           int n_out, int k_in, float* dW, float* db, const char* name, cudaStream_t s) {
+  GemmArgs g = {};
+  g.A = dY; g.a_rs = 1; g.a_cs = ld_dy;  // A(m,k) = dY[k, m]
+  g.B = A; g.b_rs = ld_a; g.b_cs = 1;    // B(k,n) = A[k, n]
+  g.C = dW; g.ldc = k_in; g.M = n_out; g.N = k_in; g.K = rows; g.dev_K = dev_rows;
+  g.rowsum_out = db; g.accumulate = 1; g.split_k = pick_split(n_out, k_in, rows);
+  return launch_gemm(ctx, g, name, s);
+}
+
+// dA[rows, n_cols] = dY[rows, n_out] W[:, col0 : col0 + n_cols]   (W is [n_out, ld_w] row-major)
+int grad_in(tgnn_ctx* ctx, const float* dY, int64_t ld_dy, const float* W, int64_t ld_w, int col0, int rows,
+            const int32_t* dev_rows, int n_out, int n_cols, float* dA, int64_t ld_da, const char* name, cudaStream_t s) {
+  GemmArgs g = {};
+  g.A = dY; g.a_rs = ld_dy; g.a_cs = 1;
+  g.B = W + col0; g.b_rs = ld_w; g.b_cs = 1;
+  g.C = dA; g.ldc = ld_da; g.M = rows; g.N = n_cols; g.K = n_out; g.dev_M = dev_rows; g.split_k = 1;
+  return launch_gemm(ctx, g, name, s);
+}
+
+}  // namespace
+
+#define RC(x)            \
+  do {                   \
+    int rc__ = (x);      \
+    if (rc__) return rc__; \
+  } while (0)
+
+int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* loss_out, float* gradnorm_out,
+                    cudaStream_t s) {
+  const tgnn_config& c = ctx->cfg;
+  const ParamLayout& L = ctx->L;
+  Workspace& w = ctx->ws;
+  const int d = c.d, k = c.k, H = c.heads, de = c.d_e;
+  const int R = 3 * n_q, NB = R * k;
+  float* P = ctx->params;
+  float* G = w.grads;
+  // grads | dMemU | red | st_scalars are contiguous in the arena: one memset clears them all
+  const size_t zero_bytes = (size_t)((char*)(w.st_scalars + 4) - (char*)w.grads);
+  TGNN_CUDA_OK(ctx, cudaMemsetAsync(w.grads, 0, zero_bytes, s));
+
+  if (n_q > 0) {
+    const int64_t tot = (int64_t)2 * n_q * 2 * d;
+    {
+      KernelScope scope__(ctx, "head_gather", s);
+      head_gather_kernel<<<(int)((tot + 255) / 256), 256, 0, s>>>(ctx->e_h, n_q, d, w.cat1);
+    }
+    TGNN_LAUNCH_OK(ctx, "head_gather");
+    GemmArgs g = {};
+    g.A = w.cat1; g.a_rs = 2 * d; g.a_cs = 1;
+    g.B = P + L.w1; g.b_rs = 1; g.b_cs = 2 * d;
+    g.C = w.hid1; g.ldc = d; g.M = 2 * n_q; g.N = d; g.K = 2 * d; g.bias = P + L.b1; g.relu = 1; g.split_k = 1;
+    RC(launch_gemm(ctx, g, "head_hidden", s));
+    {
+      KernelScope scope__(ctx, "head_loss", s);
+      head_loss_kernel<<<(n_q + 7) / 8, 256, d * sizeof(float), s>>>(w.hid1, P + L.w2, P + L.b2, loss_mask, n_q, d,
+                                                                     G + L.w2, G + L.b2, w.st_scalars);
+    }
+    TGNN_LAUNCH_OK(ctx, "head_loss");
+    // hid1 now holds d loss / d pre1
+    RC(grad_w(ctx, w.hid1, d, w.cat1, 2 * d, 2 * n_q, nullptr, d, 2 * d, G + L.w1, G + L.b1, "dW_1", s));
+    RC(grad_in(ctx, w.hid1, d, P + L.w1, 2 * d, 0, 2 * n_q, nullptr, d, 2 * d, w.dcat1, 2 * d, "dcat1", s));
+    const int64_t tot2 = (int64_t)R * d;
+    {
+      KernelScope scope__(ctx, "dh", s);
+      dh_kernel<<<(int)((tot2 + 255) / 256), 256, 0, s>>>(w.dcat1, ctx->e_h, n_q, d, w.dpre_o);
+    }
+    TGNN_LAUNCH_OK(ctx, "dh");
+    RC(grad_w(ctx, w.dpre_o, d, w.cat_o, 2 * d, R, nullptr, d, 2 * d, G + L.wo, G + L.bo, "dW_o", s));
+    RC(grad_in(ctx, w.dpre_o, d, P + L.wo, 2 * d, 0, R, nullptr, d, 2 * d, w.dcat_o, 2 * d, "dcat_o", s));
+    const int wpb = 8;
+    {
+      KernelScope scope__(ctx, "attention_bwd", s);
+      attention_bwd_kernel<<<(R + wpb - 1) / wpb, wpb * 32, wpb * H * k * sizeof(float), s>>>(
+          w.Q, w.KV, w.alpha, w.dcat_o, ctx->e_cnt, R, d, H, k, w.dQ, w.dKV);
+    }
+    TGNN_LAUNCH_OK(ctx, "attention_bwd");
+    RC(grad_w(ctx, w.dQ, d, w.Zq, 2 * d, R, nullptr, d, 2 * d, G + L.wq, G + L.bq, "dW_q", s));
+    RC(grad_in(ctx, w.dQ, d, P + L.wq, 2 * d, 0, R, nullptr, d, 2 * d, w.dzq, 2 * d, "dzq", s));
+    RC(grad_w(ctx, w.dKV, 2 * d, w.Z, ctx->ld_kv, NB, nullptr, 2 * d, (int)L.dkv, G + L.wk, G + L.bk, "dW_kv", s));
+    RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, d + de, NB, nullptr, 2 * d, d, w.dZp, d, "dZ_phi", s));
+    // time-encoder gradient through the attention inputs
+    const int rpb = 64;
+    {
+      KernelScope scope__(ctx, "time_grad_z", s);
+      time_grad_kernel<<<(NB + rpb - 1) / rpb, 128, 0, s>>>(w.dZp, d, 0, w.z_dt, NB, nullptr, rpb, d, P + L.time_w,
+                                                            P + L.time_b, G + L.time_w, G + L.time_b);
+    }
+    TGNN_LAUNCH_OK(ctx, "time_grad_z");
+    {
+      KernelScope scope__(ctx, "time_grad_q", s);
+      time_grad_kernel<<<(R + rpb - 1) / rpb, 128, 0, s>>>(w.dzq, 2 * d, d, nullptr, R, nullptr, rpb, d, P + L.time_w,
+                                                           P + L.time_b, G + L.time_w, G + L.time_b);
+    }
+    TGNN_LAUNCH_OK(ctx, "time_grad_q");
+    if (ctx->have_update) {
+      RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, 0, NB, nullptr, 2 * d, d, w.dZm, d, "dZ_mem", s));
+      {
+        KernelScope scope__(ctx, "scatter_dmem", s);
+        scatter_dmem_kernel<<<(NB + R + 7) / 8, 256, 0, s>>>(w.dZm, w.dcat_o, w.dzq, ctx->e_nbr, ctx->e_nodes, R, k, d,
+                                                             w.node2slot, w.dMemU);
+      }
+      TGNN_LAUNCH_OK(ctx, "scatter_dmem");
+      const int U_cap = ctx->upd_cap;
+      const int64_t tot3 = (int64_t)U_cap * d;
+      {
+        KernelScope scope__(ctx, "gru_bwd_gate", s);
+        gru_bwd_gate_kernel<<<(int)((tot3 + 255) / 256), 256, 0, s>>>(w.dMemU, w.X, ctx->ld_msg, d, w.g_r, w.g_z, w.g_n,
+                                                                      w.g_hn, ctx->upd_n_uniq, U_cap, w.dGi, w.dGh);
+      }
+      TGNN_LAUNCH_OK(ctx, "gru_bwd_gate");
+      RC(grad_w(ctx, w.dGi, 3 * d, w.X, ctx->ld_msg, U_cap, ctx->upd_n_uniq, 3 * d, (int)L.dmsg, G + L.gru_wi,
+                G + L.gru_bi, "dW_i", s));
+      RC(grad_w(ctx, w.dGh, 3 * d, w.X, ctx->ld_msg, U_cap, ctx->upd_n_uniq, 3 * d, d, G + L.gru_wh, G + L.gru_bh,
+                "dW_h", s));
+      RC(grad_in(ctx, w.dGi, 3 * d, P + L.gru_wi, L.dmsg, 2 * d + de, U_cap, ctx->upd_n_uniq, 3 * d, d, w.dXp, d,
+                 "dX_phi", s));
+      {
+        KernelScope scope__(ctx, "time_grad_x", s);
+        time_grad_kernel<<<(U_cap + rpb - 1) / rpb, 128, 0, s>>>(w.dXp, d, 0, w.x_dt, U_cap, ctx->upd_n_uniq, rpb, d,
+                                                                 P + L.time_w, P + L.time_b, G + L.time_w, G + L.time_b);
+      }
+      TGNN_LAUNCH_OK(ctx, "time_grad_x");
+    }
+  }
+  {
+    KernelScope scope__(ctx, "gradnorm", s);
+    gradnorm_kernel<<<148, 256, 0, s>>>(G, L.total, w.red, w.counters, ctx->step, c.beta1, c.beta2, w.adam_sc,
+                                        w.st_scalars, w.st_scalars + 2, loss_out, gradnorm_out);
+  }
+  TGNN_LAUNCH_OK(ctx, "gradnorm");
+  {
+    KernelScope scope__(ctx, "adam", s);
+    adam_kernel<<<296, 256, 0, s>>>(P, ctx->adam_m, ctx->adam_v, G, L.total, c.lr, c.beta1, c.beta2, c.eps, w.adam_sc);
+  }
+  TGNN_LAUNCH_OK(ctx, "adam");
+  return TGNN_OK;
+}
+
+}  // namespace tgnn

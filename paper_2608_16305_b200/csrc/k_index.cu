@@ -1,0 +1,301 @@
+// Integer kernels: pruning mask (step 0), most-recent-k neighbor search
+// (step 1), per-node latest-event reduction (step 3).  All results are unique,
+// so they are bit-exact whatever the thread interleaving.
+#include "tgnn_internal.cuh"
+
+namespace tgnn {
+namespace {
+
+constexpr unsigned FULL = 0xffffffffu;
+
+// ---------------------------------------------------------------- step (0) --
+__device__ __forceinline__ uint64_t mix64(uint64_t z) {  // SplitMix64 finaliser
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+  return z ^ (z >> 31);
+}
+__device__ __forceinline__ uint32_t hash32(uint64_t seed, int64_t batch_idx, int32_t eid) {
+  const uint64_t x =
+      seed ^ ((uint64_t)batch_idx * 0x9E3779B97F4A7C15ULL) ^ ((uint64_t)(uint32_t)eid * 0xC2B2AE3D27D4EB4FULL);
+  return (uint32_t)(mix64(x) >> 32);
+}
+
+// One occurrence count per endpoint, warp-aggregated so a hub costs one atomic per warp.
+__device__ __forceinline__ void hist_add(int32_t* hist, int node, bool valid) {
+  const unsigned act = __ballot_sync(FULL, valid);
+  if (!valid) return;
+  const unsigned peers = __match_any_sync(act, node);
+  if ((int)(threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[node], __popc(peers));
+}
+
+constexpr int FIRST_VISIT = 0x40000000;
+
+// Single CTA: the batch has a few thousand events and the histogram lives in L2.
+__global__ void __launch_bounds__(1024) prune_mask_kernel(const int32_t* __restrict__ src, const int32_t* __restrict__ dst,
+                                                          const int32_t* __restrict__ eid,
+                                                          const uint8_t* __restrict__ is_aux, int n, int32_t* hist,
+                                                          int force_heavy, uint32_t drop_q32, uint64_t seed,
+                                                          int64_t batch_idx, uint8_t* __restrict__ keep_out,
+                                                          int32_t* __restrict__ heavy_out) {
+  __shared__ int s_max, s_touched, s_heavy;
+  if (threadIdx.x == 0) { s_max = 0; s_touched = 0; }
+  const int n_round = (n + 31) / 32 * 32;
+  for (int i = threadIdx.x; i < n_round; i += blockDim.x) {
+    const bool v = i < n;
+    hist_add(hist, v ? src[i] : 0, v);
+    hist_add(hist, v ? dst[i] : 0, v);
+  }
+  __syncthreads();
+  // max count and number of touched nodes: the first visitor of a node counts it
+  int lmax = 0, ltouched = 0;
+  for (int i = threadIdx.x; i < 2 * n; i += blockDim.x) {
+    const int node = (i & 1) ? dst[i >> 1] : src[i >> 1];
+    const int old = atomicOr(&hist[node], FIRST_VISIT);
+    lmax = max(lmax, old & (FIRST_VISIT - 1));
+    ltouched += (old & FIRST_VISIT) ? 0 : 1;
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    lmax = max(lmax, __shfl_xor_sync(FULL, lmax, o));
+    ltouched += __shfl_xor_sync(FULL, ltouched, o);
+  }
+  if ((threadIdx.x & 31) == 0) { atomicMax(&s_max, lmax); atomicAdd(&s_touched, ltouched); }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int heavy = ((int64_t)s_max * (int64_t)s_touched > 8ll * n) ? 1 : 0;
+    if (force_heavy == 0 || force_heavy == 1) heavy = force_heavy;
+    s_heavy = heavy;
+    *heavy_out = heavy;
+  }
+  __syncthreads();
+  const int heavy = s_heavy;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    bool keep = true;
+    if (is_aux[i] && heavy) keep = !(drop_q32 == 0xFFFFFFFFu || hash32(seed, batch_idx, eid[i]) < drop_q32);
+    keep_out[i] = keep ? 1 : 0;
+    hist[src[i]] = 0;  // leave the histogram clean for the next call
+    hist[dst[i]] = 0;
+  }
+}
+
+// ---------------------------------------------------------------- step (1) --
+// One warp per root.  The lower bound is found by a 32-way search: each round
+// the lanes probe 32 spread positions of the remaining range with independent
+// loads and a ballot picks the sub-range, so a hub slice of 2*10^7 entries
+// needs 5 dependent memory round trips instead of 25.
+__global__ void __launch_bounds__(256) sample_recent_kernel(const int64_t* __restrict__ indptr,
+                                                            const int32_t* __restrict__ g_nbr,
+                                                            const int32_t* __restrict__ g_eid,
+                                                            const double* __restrict__ g_ts,
+                                                            const int32_t* __restrict__ nodes,
+                                                            const double* __restrict__ times, int n, int k,
+                                                            int32_t* __restrict__ nbr_out, int32_t* __restrict__ eid_out,
+                                                            double* __restrict__ ts_out, int32_t* __restrict__ cnt_out) {
+  const int lane = threadIdx.x & 31;
+  const int root = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+  if (root >= n) return;
+  const int node = nodes[root];
+  const double t = times[root];
+  const int64_t base = indptr[node];
+  int64_t lo = base, hi = indptr[node + 1];  // the answer p lies in [lo, hi]
+  while (hi - lo > 32) {
+    const int64_t len = hi - lo;
+    const int64_t idx = lo + ((int64_t)(lane + 1) * len) / 33;  // in [lo, hi), non-decreasing in lane
+    const bool below = g_ts[idx] < t;                           // p > idx
+    const int c = __popc(__ballot_sync(FULL, below));
+    const int64_t idx_hi = __shfl_sync(FULL, idx, c < 32 ? c : 31);       // first probe with ts >= t
+    const int64_t idx_lo = __shfl_sync(FULL, idx, c > 0 ? c - 1 : 0);     // last probe with ts < t
+    if (c < 32) hi = idx_hi;
+    if (c > 0) lo = idx_lo + 1;
+  }
+  {
+    const int len = (int)(hi - lo);
+    const bool below = lane < len && g_ts[lo + lane] < t;
+    lo += __popc(__ballot_sync(FULL, below));
+  }
+  const int64_t p = lo;
+  const int cnt = (int)min((int64_t)k, p - base);
+  if (lane == 0) cnt_out[root] = cnt;
+  if (lane < k) {
+    const int64_t o = (int64_t)root * k + lane;
+    if (lane < cnt) {
+      const int64_t e = p - 1 - lane;
+      nbr_out[o] = g_nbr[e];
+      eid_out[o] = g_eid[e];
+      ts_out[o] = g_ts[e];
+    } else {
+      nbr_out[o] = -1;
+      eid_out[o] = -1;
+      ts_out[o] = 0.0;
+    }
+  }
+}
+
+__global__ void make_roots_kernel(const int32_t* __restrict__ q_src, const int32_t* __restrict__ q_dst,
+                                  const int32_t* __restrict__ q_neg, const double* __restrict__ q_t, int n_q,
+                                  int32_t* __restrict__ r_node, double* __restrict__ r_time) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= 3 * n_q) return;
+  const int j = i % n_q, blk = i / n_q;
+  r_node[i] = blk == 0 ? q_src[j] : (blk == 1 ? q_dst[j] : q_neg[j]);
+  r_time[i] = q_t[j];
+}
+
+// ---------------------------------------------------------------- step (3) --
+// fp64 -> uint64 preserving order (0 is left free as "empty" for every finite value)
+__device__ __forceinline__ unsigned long long orderable(double x) {
+  unsigned long long u = (unsigned long long)__double_as_longlong(x);
+  return (u >> 63) ? ~u : (u | 0x8000000000000000ULL);
+}
+
+// max over the lanes of `peers` (a __match_any_sync mask all of whose lanes call this)
+__device__ __forceinline__ unsigned long long peer_max(unsigned peers, unsigned long long v) {
+  unsigned long long m = v;
+  unsigned rest = peers;
+  while (rest) {
+    const int l = __ffs(rest) - 1;
+    rest &= rest - 1;
+    const unsigned long long o = __shfl_sync(peers, v, l);
+    m = o > m ? o : m;
+  }
+  return m;
+}
+
+// Single CTA.  Key order (t, eid, role) is resolved in two atomicMax passes over
+// per-node tables (time first, then eid/role among the messages that tie on
+// time); a hub's thousands of messages are pre-reduced inside each warp.
+// Then the touched nodes are compacted in ascending id order by a block scan.
+__global__ void __launch_bounds__(1024) reduce_latest_kernel(const int32_t* __restrict__ msg_node,
+                                                             const double* __restrict__ t,
+                                                             const int32_t* __restrict__ eid, int n_msg, int N,
+                                                             unsigned long long* best_t, unsigned long long* best_id,
+                                                             int32_t* win_msg, int32_t* node2slot, int32_t* prev_uniq,
+                                                             int32_t* prev_n_uniq, int32_t* __restrict__ uniq_out,
+                                                             int32_t* __restrict__ winner_out,
+                                                             int32_t* __restrict__ n_uniq_out) {
+  __shared__ int s_warp[32];
+  __shared__ int s_total;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  // forget the previous step's node -> slot map
+  const int pn = *prev_n_uniq;
+  for (int i = tid; i < pn; i += blockDim.x) node2slot[prev_uniq[i]] = -1;
+  const int n_round = (n_msg + 31) / 32 * 32;
+  for (int j = tid; j < n_round; j += blockDim.x) {
+    const int node = j < n_msg ? msg_node[j] : -1;
+    const bool v = node >= 0;
+    const unsigned act = __ballot_sync(FULL, v);
+    if (v) {
+      const unsigned peers = __match_any_sync(act, node);
+      const unsigned long long m = peer_max(peers, orderable(t[j >> 1]));
+      if (lane == __ffs(peers) - 1) atomicMax(&best_t[node], m);
+    }
+  }
+  __syncthreads();
+  for (int j = tid; j < n_round; j += blockDim.x) {
+    const int node = j < n_msg ? msg_node[j] : -1;
+    const bool v = node >= 0 && orderable(t[j >> 1]) == best_t[node];
+    const unsigned act = __ballot_sync(FULL, v);
+    if (v) {
+      const unsigned peers = __match_any_sync(act, node);
+      const unsigned long long key = (((unsigned long long)(uint32_t)eid[j >> 1]) << 1 | (unsigned)(j & 1)) + 1ULL;
+      const unsigned long long m = peer_max(peers, key);
+      if (lane == __ffs(peers) - 1) atomicMax(&best_id[node], m);
+    }
+  }
+  __syncthreads();
+  for (int j = tid; j < n_msg; j += blockDim.x) {
+    const int node = msg_node[j];
+    if (node < 0) continue;
+    const unsigned long long key = (((unsigned long long)(uint32_t)eid[j >> 1]) << 1 | (unsigned)(j & 1)) + 1ULL;
+    if (orderable(t[j >> 1]) == best_t[node] && key == best_id[node]) win_msg[node] = j;
+  }
+  __syncthreads();
+  // ascending compaction: thread i owns a contiguous chunk of node ids
+  const int chunk = (N + blockDim.x - 1) / blockDim.x;
+  const int nb = min(N, tid * chunk), ne = min(N, nb + chunk);
+  int mine = 0;
+  for (int v = nb; v < ne; ++v) mine += best_id[v] != 0ULL;
+  int incl = mine;
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(FULL, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) s_warp[wid] = incl;
+  __syncthreads();
+  if (wid == 0) {
+    int w = lane < (int)(blockDim.x >> 5) ? s_warp[lane] : 0;
+    int wi = w;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(FULL, wi, o);
+      if (lane >= o) wi += y;
+    }
+    s_warp[lane] = wi - w;  // exclusive prefix of the warp totals
+    if (lane == 31) s_total = wi;
+  }
+  __syncthreads();
+  int pos = s_warp[wid] + incl - mine;
+  for (int v = nb; v < ne; ++v) {
+    if (best_id[v] != 0ULL) {
+      uniq_out[pos] = v;
+      winner_out[pos] = win_msg[v];
+      prev_uniq[pos] = v;
+      node2slot[v] = pos;
+      best_t[v] = 0ULL;
+      best_id[v] = 0ULL;
+      ++pos;
+    }
+  }
+  if (tid == 0) { *n_uniq_out = s_total; *prev_n_uniq = s_total; }
+}
+
+}  // namespace
+
+int launch_prune_mask(tgnn_ctx* ctx, const int32_t* src, const int32_t* dst, const int32_t* eid, const uint8_t* is_aux,
+                      int n, int force_heavy, uint32_t drop_q32, uint64_t seed, int64_t batch_idx, uint8_t* keep_out,
+                      int32_t* heavy_out, cudaStream_t s) {
+  {
+    KernelScope scope__(ctx, "prune_mask", s);
+    prune_mask_kernel<<<1, 1024, 0, s>>>(src, dst, eid, is_aux, n, ctx->ws.hist, force_heavy, drop_q32, seed, batch_idx,
+                                         keep_out, heavy_out);
+  }
+  TGNN_LAUNCH_OK(ctx, "prune_mask");
+  return TGNN_OK;
+}
+
+int launch_sample_recent(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n, int32_t* nbr_out,
+                         int32_t* eid_out, double* ts_out, int32_t* cnt_out, cudaStream_t s) {
+  if (n == 0) return TGNN_OK;
+  const int warps_per_block = 8;
+  {
+    KernelScope scope__(ctx, "sample_recent", s);
+    sample_recent_kernel<<<(n + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, s>>>(
+        ctx->indptr, ctx->g_nbr, ctx->g_eid, ctx->g_ts, nodes, times, n, ctx->cfg.k, nbr_out, eid_out, ts_out, cnt_out);
+  }
+  TGNN_LAUNCH_OK(ctx, "sample_recent");
+  return TGNN_OK;
+}
+
+int launch_make_roots(tgnn_ctx* ctx, const int32_t* q_src, const int32_t* q_dst, const int32_t* q_neg,
+                      const double* q_t, int n_q, cudaStream_t s) {
+  if (n_q == 0) return TGNN_OK;
+  {
+    KernelScope scope__(ctx, "make_roots", s);
+    make_roots_kernel<<<(3 * n_q + 255) / 256, 256, 0, s>>>(q_src, q_dst, q_neg, q_t, n_q, ctx->ws.r_node, ctx->ws.r_time);
+  }
+  TGNN_LAUNCH_OK(ctx, "make_roots");
+  return TGNN_OK;
+}
+
+int launch_reduce_latest(tgnn_ctx* ctx, const int32_t* msg_node, const double* t, const int32_t* eid, int n_msg,
+                         int32_t* uniq_out, int32_t* winner_out, int32_t* n_uniq_out, cudaStream_t s) {
+  Workspace& w = ctx->ws;
+  {
+    KernelScope scope__(ctx, "reduce_latest", s);
+    reduce_latest_kernel<<<1, 1024, 0, s>>>(msg_node, t, eid, n_msg, (int)ctx->cfg.num_nodes, w.best_t, w.best_id,
+                                            w.win_msg, w.node2slot, w.prev_uniq, w.prev_n_uniq, uniq_out, winner_out,
+                                            n_uniq_out);
+  }
+  TGNN_LAUNCH_OK(ctx, "reduce_latest");
+  return TGNN_OK;
+}
+
+}  // namespace tgnn

@@ -1,0 +1,460 @@
+// C ABI: context life cycle, argument checks, and the sequencing of one training step.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <new>
+#include <string>
+
+#include "tgnn_internal.cuh"
+
+namespace tgnn {
+
+ParamLayout make_layout(int d_, int de_) {
+  ParamLayout L;
+  const int64_t d = d_, de = de_;
+  L.d = d; L.de = de; L.dmsg = 3 * d + de; L.dkv = 2 * d + de; L.dq = 2 * d;
+  int64_t o = 0;
+  L.time_w = o; o += d;
+  L.time_b = o; o += d;
+  L.gru_wi = o; o += 3 * d * L.dmsg;
+  L.gru_wh = o; o += 3 * d * d;
+  L.gru_bi = o; o += 3 * d;
+  L.gru_bh = o; o += 3 * d;
+  L.wq = o; o += d * L.dq;
+  L.bq = o; o += d;
+  L.wk = o; o += d * L.dkv;
+  L.wv = o; o += d * L.dkv;
+  L.bk = o; o += d;
+  L.bv = o; o += d;
+  L.wo = o; o += d * 2 * d;
+  L.bo = o; o += d;
+  L.w1 = o; o += d * 2 * d;
+  L.b1 = o; o += d;
+  L.w2 = o; o += d;
+  L.b2 = o; o += 1;
+  L.total = o;
+  return L;
+}
+
+int set_error(tgnn_ctx* ctx, int code, const char* fmt, ...) {
+  if (ctx) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+    va_end(ap);
+  }
+  return code;
+}
+
+namespace {
+
+int check_config(const tgnn_config* c) {
+  if (!c) return TGNN_EINVAL;
+  if (c->num_nodes <= 0 || c->num_nodes > 0x7fffffff) return TGNN_EINVAL;
+  if (c->d <= 0 || c->d % 4 != 0 || c->heads <= 0 || c->d % c->heads != 0) return TGNN_ESHAPE;
+  if (c->d_e < 0 || c->d_e % 2 != 0) return TGNN_ESHAPE;
+  if (c->k < 1 || c->k > 32 || c->heads * c->k > 1024) return TGNN_ESHAPE;
+  if (c->feat_dtype != TGNN_F32 && c->feat_dtype != TGNN_BF16) return TGNN_EINVAL;
+  if (c->max_events < 1 || c->max_roots < 3 || c->max_events > (1 << 24) || c->max_roots > (1 << 24)) return TGNN_EINVAL;
+  if (c->math_mode != TGNN_MATH_FP32 && c->math_mode != TGNN_MATH_TF32) return TGNN_EINVAL;
+  if (!(c->lr >= 0.f) || !(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f) || !(c->eps > 0.f))
+    return TGNN_EINVAL;
+  return TGNN_OK;
+}
+
+struct Carver {
+  char* base;
+  size_t off;
+  template <typename T>
+  void take(T*& p, size_t count) {
+    off = (off + 255) & ~(size_t)255;
+    p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+  }
+  // no alignment gap: keeps a group of buffers contiguous for a single memset
+  template <typename T>
+  void take_packed(T*& p, size_t count) {
+    off = (off + 15) & ~(size_t)15;
+    p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+  }
+};
+
+size_t carve(tgnn_ctx* ctx, char* base) {
+  const tgnn_config& c = ctx->cfg;
+  Workspace& w = ctx->ws;
+  const size_t N = (size_t)c.num_nodes, d = c.d, k = c.k, H = c.heads;
+  const size_t ne = c.max_events, U = ctx->U_cap, R = ctx->R_cap, NB = ctx->NB_cap, nq = ctx->nq_cap;
+  Carver cv{base, 0};
+  cv.take(w.hist, N);
+  cv.take(w.best_t, N);
+  cv.take(w.best_id, N);
+  cv.take(w.win_msg, N);
+  cv.take(w.node2slot, N);
+  cv.take(w.prev_uniq, U);
+  cv.take(w.prev_n_uniq, 4);
+  cv.take(w.msg_node, U);
+  cv.take(w.uniq, U);
+  cv.take(w.winner, U);
+  cv.take(w.n_uniq, 4);
+  cv.take(w.r_node, R);
+  cv.take(w.r_time, R);
+  cv.take(w.nb_node, NB);
+  cv.take(w.nb_eid, NB);
+  cv.take(w.nb_ts, NB);
+  cv.take(w.nb_cnt, R);
+  cv.take(w.h, R * d);
+  cv.take(w.st_u_src, ne); cv.take(w.st_u_dst, ne); cv.take(w.st_u_eid, ne);
+  cv.take(w.st_q_src, nq); cv.take(w.st_q_dst, nq); cv.take(w.st_q_neg, nq);
+  cv.take(w.st_u_t, ne); cv.take(w.st_q_t, nq);
+  cv.take(w.st_u_keep, ne); cv.take(w.st_mask, nq);
+  cv.take(w.X, U * ctx->ld_msg);
+  cv.take(w.x_dt, U);
+  cv.take(w.win_t, U);
+  cv.take(w.Gi, U * 3 * d);
+  cv.take(w.Gh, U * 3 * d);
+  cv.take(w.g_r, U * d); cv.take(w.g_z, U * d); cv.take(w.g_n, U * d); cv.take(w.g_hn, U * d);
+  cv.take(w.Z, NB * ctx->ld_kv);
+  cv.take(w.z_dt, NB);
+  cv.take(w.KV, NB * 2 * d);
+  cv.take(w.Zq, R * 2 * d);
+  cv.take(w.Q, R * d);
+  cv.take(w.alpha, R * H * k);
+  cv.take(w.cat_o, R * 2 * d);
+  cv.take(w.cat1, 2 * nq * 2 * d);
+  cv.take(w.hid1, 2 * nq * d);
+  cv.take(w.dcat1, 2 * nq * 2 * d);
+  cv.take(w.dpre_o, R * d);
+  cv.take(w.dcat_o, R * 2 * d);
+  cv.take(w.dQ, R * d);
+  cv.take(w.dzq, R * 2 * d);
+  cv.take(w.dKV, NB * 2 * d);
+  cv.take(w.dZm, NB * d);
+  cv.take(w.dZp, NB * d);
+  cv.take(w.dGi, U * 3 * d);
+  cv.take(w.dGh, U * 3 * d);
+  cv.take(w.dXp, U * d);
+  cv.take(w.adam_sc, 4);
+  cv.take(w.counters, 4);
+  cv.take(w.status, 4);
+  // cleared together at the start of every backward pass: keep these four adjacent and in this order
+  cv.take(w.grads, (size_t)ctx->L.total);
+  cv.take_packed(w.dMemU, U * d);
+  cv.take_packed(w.red, 4);
+  cv.take_packed(w.st_scalars, 4);
+  return (cv.off + 255) & ~(size_t)255;
+}
+
+inline cudaStream_t S(void* stream) { return reinterpret_cast<cudaStream_t>(stream); }
+
+}  // namespace
+}  // namespace tgnn
+
+using namespace tgnn;
+
+#define NEED(ctx, cond, code, ...)                       \
+  do {                                                   \
+    if (!(cond)) return set_error(ctx, code, __VA_ARGS__); \
+  } while (0)
+
+extern "C" {
+
+int64_t tgnn_param_count(const tgnn_config* cfg) {
+  if (check_config(cfg) != TGNN_OK) return -1;
+  return make_layout(cfg->d, cfg->d_e).total;
+}
+
+int tgnn_param_layout(const tgnn_config* cfg, int64_t* out) {
+  const int rc = check_config(cfg);
+  if (rc != TGNN_OK) return rc;
+  if (!out) return TGNN_EINVAL;
+  const ParamLayout L = make_layout(cfg->d, cfg->d_e);
+  const int64_t v[19] = {L.time_w, L.time_b, L.gru_wi, L.gru_wh, L.gru_bi, L.gru_bh, L.wq, L.bq, L.wk, L.wv,
+                         L.bk, L.bv, L.wo, L.bo, L.w1, L.b1, L.w2, L.b2, L.total};
+  for (int i = 0; i < 19; ++i) out[i] = v[i];
+  return TGNN_OK;
+}
+
+int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
+  if (!out) return TGNN_EINVAL;
+  *out = nullptr;
+  const int rc = check_config(cfg);
+  if (rc != TGNN_OK) return rc;
+  int dev = 0, cc_major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TGNN_ECUDA;
+  if (cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return TGNN_ECUDA;
+  if (cc_major != 10) return TGNN_ECUDA;  // kernels are built for sm_100a only
+  tgnn_ctx* ctx = new (std::nothrow) tgnn_ctx();
+  if (!ctx) return TGNN_ECUDA;
+  ctx->cfg = *cfg;
+  ctx->L = make_layout(cfg->d, cfg->d_e);
+  ctx->U_cap = 2 * cfg->max_events;
+  ctx->R_cap = cfg->max_roots;
+  ctx->NB_cap = cfg->max_roots * cfg->k;
+  ctx->nq_cap = cfg->max_roots / 3;
+  ctx->ld_msg = (int)((ctx->L.dmsg + 31) / 32 * 32);
+  ctx->ld_kv = (int)((ctx->L.dkv + 31) / 32 * 32);
+  ctx->arena_bytes = carve(ctx, nullptr);
+  if (cudaMalloc(&ctx->arena, ctx->arena_bytes) != cudaSuccess) {
+    cudaGetLastError();
+    delete ctx;
+    return TGNN_ECUDA;
+  }
+  carve(ctx, (char*)ctx->arena);
+  bool ok = cudaMemset(ctx->arena, 0, ctx->arena_bytes) == cudaSuccess;
+  ok = ok && cudaMemset(ctx->ws.node2slot, 0xff, sizeof(int32_t) * (size_t)cfg->num_nodes) == cudaSuccess;
+  ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+  if (!ok) {
+    cudaFree(ctx->arena);
+    delete ctx;
+    return TGNN_ECUDA;
+  }
+  snprintf(ctx->err, sizeof(ctx->err), "no error");
+  *out = ctx;
+  return TGNN_OK;
+}
+
+int tgnn_destroy(tgnn_ctx* ctx) {
+  if (!ctx) return TGNN_OK;
+  cudaDeviceSynchronize();
+  for (ProfEntry& e : ctx->prof.entries) {
+    cudaEventDestroy(e.a);
+    cudaEventDestroy(e.b);
+  }
+  cudaFree(ctx->arena);
+  delete ctx;
+  return TGNN_OK;
+}
+
+const char* tgnn_last_error(const tgnn_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+int64_t tgnn_kernel_launches(const tgnn_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int tgnn_set_graph(tgnn_ctx* ctx, const int64_t* indptr, const int32_t* nbr, const int32_t* eid, const double* ts,
+                   int64_t n_entries) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, indptr && n_entries >= 0, TGNN_EINVAL, "set_graph: null indptr or negative size");
+  NEED(ctx, n_entries == 0 || (nbr && eid && ts), TGNN_EINVAL, "set_graph: null adjacency arrays");
+  ctx->indptr = indptr; ctx->g_nbr = nbr; ctx->g_eid = eid; ctx->g_ts = ts; ctx->n_entries = n_entries;
+  return TGNN_OK;
+}
+
+int tgnn_set_edge_features(tgnn_ctx* ctx, const void* efeat, int dtype, int64_t num_events, int d_e) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, d_e == ctx->cfg.d_e, TGNN_ESHAPE, "set_edge_features: d_e %d != configured %d", d_e, ctx->cfg.d_e);
+  NEED(ctx, dtype == ctx->cfg.feat_dtype, TGNN_EINVAL, "set_edge_features: dtype differs from the configuration");
+  NEED(ctx, d_e == 0 || efeat, TGNN_EINVAL, "set_edge_features: null table");
+  NEED(ctx, num_events >= 0, TGNN_EINVAL, "set_edge_features: negative size");
+  NEED(ctx, ((uintptr_t)efeat & 3) == 0, TGNN_EINVAL, "set_edge_features: table must be 4-byte aligned");
+  ctx->efeat = efeat; ctx->num_events = num_events;
+  return TGNN_OK;
+}
+
+int tgnn_set_state(tgnn_ctx* ctx, float* memory, double* last_update, float* params, float* adam_m, float* adam_v,
+                   int64_t* step) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, memory && last_update && params && adam_m && adam_v && step, TGNN_EINVAL, "set_state: null pointer");
+  ctx->memory = memory; ctx->last_update = last_update; ctx->params = params;
+  ctx->adam_m = adam_m; ctx->adam_v = adam_v; ctx->step = step;
+  ctx->have_update = false; ctx->have_embed = false;
+  return TGNN_OK;
+}
+
+int tgnn_prune_mask(tgnn_ctx* ctx, const int32_t* src, const int32_t* dst, const int32_t* eid, const uint8_t* is_aux,
+                    int n, int force_heavy, uint32_t drop_q32, uint64_t seed, int64_t batch_idx, uint8_t* keep_out,
+                    int32_t* heavy_out, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, n >= 0, TGNN_EINVAL, "prune_mask: negative n");
+  NEED(ctx, n <= ctx->cfg.max_events, TGNN_ECAPACITY, "prune_mask: n %d > max_events %d", n, ctx->cfg.max_events);
+  NEED(ctx, heavy_out && (n == 0 || (src && dst && eid && is_aux && keep_out)), TGNN_EINVAL, "prune_mask: null pointer");
+  NEED(ctx, force_heavy >= -1 && force_heavy <= 1, TGNN_EINVAL, "prune_mask: force_heavy must be -1, 0 or 1");
+  return launch_prune_mask(ctx, src, dst, eid, is_aux, n, force_heavy, drop_q32, seed, batch_idx, keep_out, heavy_out,
+                           S(stream));
+}
+
+int tgnn_sample_recent(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n, int32_t* nbr_out,
+                       int32_t* eid_out, double* ts_out, int32_t* cnt_out, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, ctx->indptr, TGNN_ESTATE, "sample_recent: tgnn_set_graph has not been called");
+  NEED(ctx, n >= 0, TGNN_EINVAL, "sample_recent: negative n");
+  NEED(ctx, n == 0 || (nodes && times && nbr_out && eid_out && ts_out && cnt_out), TGNN_EINVAL,
+       "sample_recent: null pointer");
+  return launch_sample_recent(ctx, nodes, times, n, nbr_out, eid_out, ts_out, cnt_out, S(stream));
+}
+
+int tgnn_build_messages(tgnn_ctx* ctx, const int32_t* src, const int32_t* dst, const double* t, const int32_t* eid,
+                        const uint8_t* keep, int n, float* msg_out, int32_t* msg_node_out, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, ctx->memory, TGNN_ESTATE, "build_messages: tgnn_set_state has not been called");
+  NEED(ctx, ctx->cfg.d_e == 0 || ctx->efeat, TGNN_ESTATE, "build_messages: tgnn_set_edge_features has not been called");
+  NEED(ctx, n >= 0, TGNN_EINVAL, "build_messages: negative n");
+  NEED(ctx, n <= ctx->cfg.max_events, TGNN_ECAPACITY, "build_messages: n %d > max_events %d", n, ctx->cfg.max_events);
+  NEED(ctx, n == 0 || (src && dst && t && eid && msg_node_out), TGNN_EINVAL, "build_messages: null pointer");
+  ctx->m_src = src; ctx->m_dst = dst; ctx->m_t = t; ctx->m_eid = eid; ctx->m_keep = keep; ctx->m_n = n;
+  return launch_build_messages(ctx, src, dst, t, eid, keep, n, msg_out, msg_node_out, S(stream));
+}
+
+int tgnn_reduce_latest(tgnn_ctx* ctx, const int32_t* msg_node, const double* t, const int32_t* eid, int n_msg,
+                       int32_t* uniq_out, int32_t* winner_out, int32_t* n_uniq_out, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, n_msg >= 0 && n_msg % 2 == 0, TGNN_EINVAL, "reduce_latest: n_msg must be even and non-negative");
+  NEED(ctx, n_msg <= ctx->U_cap, TGNN_ECAPACITY, "reduce_latest: n_msg %d > 2*max_events", n_msg);
+  NEED(ctx, n_uniq_out && (n_msg == 0 || (msg_node && t && eid && uniq_out && winner_out)), TGNN_EINVAL,
+       "reduce_latest: null pointer");
+  return launch_reduce_latest(ctx, msg_node, t, eid, n_msg, uniq_out, winner_out, n_uniq_out, S(stream));
+}
+
+int tgnn_memory_update(tgnn_ctx* ctx, const float* msg, const int32_t* uniq, const int32_t* winner,
+                       const int32_t* n_uniq, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, ctx->memory, TGNN_ESTATE, "memory_update: tgnn_set_state has not been called");
+  NEED(ctx, ctx->m_src || ctx->m_n == 0, TGNN_ESTATE, "memory_update: tgnn_build_messages has not been called");
+  NEED(ctx, n_uniq && (ctx->m_n == 0 || (uniq && winner)), TGNN_EINVAL, "memory_update: null pointer");
+  ctx->upd_n_uniq = n_uniq;
+  ctx->upd_cap = ctx->U_cap < 2 * ctx->m_n ? ctx->U_cap : 2 * ctx->m_n;
+  ctx->have_update = ctx->upd_cap > 0;
+  return launch_memory_update(ctx, msg, uniq, winner, n_uniq, S(stream));
+}
+
+int tgnn_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n, const int32_t* nbr, const int32_t* eid,
+               const double* ts, const int32_t* cnt, float* h_out, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, ctx->memory, TGNN_ESTATE, "embed: tgnn_set_state has not been called");
+  NEED(ctx, ctx->cfg.d_e == 0 || ctx->efeat, TGNN_ESTATE, "embed: tgnn_set_edge_features has not been called");
+  NEED(ctx, n >= 0, TGNN_EINVAL, "embed: negative n");
+  NEED(ctx, n <= ctx->R_cap, TGNN_ECAPACITY, "embed: n %d > max_roots %d", n, ctx->R_cap);
+  NEED(ctx, n == 0 || (nodes && times && nbr && eid && ts && cnt && h_out), TGNN_EINVAL, "embed: null pointer");
+  ctx->e_nodes = nodes; ctx->e_times = times; ctx->e_nbr = nbr; ctx->e_eid = eid; ctx->e_ts = ts; ctx->e_cnt = cnt;
+  ctx->e_n = n; ctx->e_h = h_out; ctx->have_embed = true;
+  return launch_embed(ctx, nodes, times, n, nbr, eid, ts, cnt, h_out, S(stream));
+}
+
+int tgnn_backward_step(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* loss_out, float* gradnorm_out,
+                       void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, ctx->have_embed, TGNN_ESTATE, "backward_step: no tgnn_embed call to differentiate");
+  NEED(ctx, n_q >= 0 && 3 * n_q == ctx->e_n, TGNN_ESHAPE, "backward_step: the last embed call had %d rows, expected 3*n_q = %d",
+       ctx->e_n, 3 * n_q);
+  const int rc = launch_backward(ctx, n_q, loss_mask, loss_out, gradnorm_out, S(stream));
+  ctx->have_embed = false;
+  ctx->have_update = false;
+  return rc;
+}
+
+int tgnn_train_step(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, const double* u_t, const int32_t* u_eid,
+                    const uint8_t* u_keep, int n_u, const int32_t* q_src, const int32_t* q_dst, const int32_t* q_neg,
+                    const double* q_t, int n_q, const uint8_t* loss_mask, float* loss_out, float* gradnorm_out,
+                    void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, n_u >= 0 && n_q >= 0, TGNN_EINVAL, "train_step: negative size");
+  NEED(ctx, n_q <= ctx->nq_cap, TGNN_ECAPACITY, "train_step: n_q %d > max_roots/3 = %d", n_q, ctx->nq_cap);
+  NEED(ctx, n_q == 0 || (q_src && q_dst && q_neg && q_t), TGNN_EINVAL, "train_step: null target arrays");
+  Workspace& w = ctx->ws;
+  int rc;
+  ctx->have_update = false;
+  if (n_u > 0) {
+    rc = tgnn_build_messages(ctx, u_src, u_dst, u_t, u_eid, u_keep, n_u, nullptr, w.msg_node, stream);
+    if (rc) return rc;
+    rc = tgnn_reduce_latest(ctx, w.msg_node, u_t, u_eid, 2 * n_u, w.uniq, w.winner, w.n_uniq, stream);
+    if (rc) return rc;
+    rc = tgnn_memory_update(ctx, nullptr, w.uniq, w.winner, w.n_uniq, stream);
+    if (rc) return rc;
+  }
+  rc = launch_make_roots(ctx, q_src, q_dst, q_neg, q_t, n_q, S(stream));
+  if (rc) return rc;
+  rc = tgnn_sample_recent(ctx, w.r_node, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, w.nb_cnt, stream);
+  if (rc) return rc;
+  rc = tgnn_embed(ctx, w.r_node, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, w.nb_cnt, w.h, stream);
+  if (rc) return rc;
+  return tgnn_backward_step(ctx, n_q, loss_mask, loss_out, gradnorm_out, stream);
+}
+
+int tgnn_train_step_host(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, const double* u_t,
+                         const int32_t* u_eid, const uint8_t* u_keep, int n_u, const int32_t* q_src,
+                         const int32_t* q_dst, const int32_t* q_neg, const double* q_t, int n_q,
+                         const uint8_t* loss_mask, float* loss_host, float* gradnorm_host, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, n_u >= 0 && n_q >= 0, TGNN_EINVAL, "train_step_host: negative size");
+  NEED(ctx, n_u <= ctx->cfg.max_events, TGNN_ECAPACITY, "train_step_host: n_u %d > max_events", n_u);
+  NEED(ctx, n_q <= ctx->nq_cap, TGNN_ECAPACITY, "train_step_host: n_q %d > max_roots/3", n_q);
+  NEED(ctx, n_u == 0 || (u_src && u_dst && u_t && u_eid), TGNN_EINVAL, "train_step_host: null update arrays");
+  NEED(ctx, n_q == 0 || (q_src && q_dst && q_neg && q_t), TGNN_EINVAL, "train_step_host: null target arrays");
+  Workspace& w = ctx->ws;
+  cudaStream_t s = S(stream);
+  const cudaMemcpyKind H2D = cudaMemcpyHostToDevice;
+  if (n_u > 0) {
+    TGNN_CUDA_OK(ctx, cudaMemcpyAsync(w.st_u_src, u_src, sizeof(int32_t) * n_u, H2D, s));
+    TGNN_CUDA_OK(ctx, cudaMemcpyAsync(w.st_u_dst, u_dst, sizeof(int32_t) * n_u, H2D, s));
+    TGNN_CUDA_OK(ctx, cudaMemcpyAsync(w.st_u_t, u_t, sizeof(double) * n_u, H2D, s));
+    TGNN_CUDA_OK(ctx, cudaMemcpyAsync(w.st_u_eid, u_eid, sizeof(int32_t) * n_u, H2D, s));
+    if (u_keep) TGNN_CUDA_OK(ctx, cudaMemcpyAsync(w.st_u_keep, u_keep, n_u, H2D, s));
+  }
+  if (n_q > 0) {
+    TGNN_CUDA_OK(ctx, cudaMemcpyAsync(w.st_q_src, q_src, sizeof(int32_t) * n_q, H2D, s));
+    TGNN_CUDA_OK(ctx, cudaMemcpyAsync(w.st_q_dst, q_dst, sizeof(int32_t) * n_q, H2D, s));
+    TGNN_CUDA_OK(ctx, cudaMemcpyAsync(w.st_q_neg, q_neg, sizeof(int32_t) * n_q, H2D, s));
+    TGNN_CUDA_OK(ctx, cudaMemcpyAsync(w.st_q_t, q_t, sizeof(double) * n_q, H2D, s));
+    if (loss_mask) TGNN_CUDA_OK(ctx, cudaMemcpyAsync(w.st_mask, loss_mask, n_q, H2D, s));
+  }
+  const int rc = tgnn_train_step(ctx, w.st_u_src, w.st_u_dst, w.st_u_t, w.st_u_eid, u_keep ? w.st_u_keep : nullptr, n_u,
+                                 w.st_q_src, w.st_q_dst, w.st_q_neg, w.st_q_t, n_q, loss_mask ? w.st_mask : nullptr,
+                                 nullptr, nullptr, stream);
+  if (rc) return rc;
+  if (loss_host) TGNN_CUDA_OK(ctx, cudaMemcpyAsync(loss_host, w.st_scalars + 2, sizeof(float), cudaMemcpyDeviceToHost, s));
+  if (gradnorm_host)
+    TGNN_CUDA_OK(ctx, cudaMemcpyAsync(gradnorm_host, w.st_scalars + 3, sizeof(float), cudaMemcpyDeviceToHost, s));
+  return TGNN_OK;
+}
+
+int tgnn_debug_get_grads(tgnn_ctx* ctx, float* grads_out, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, grads_out, TGNN_EINVAL, "debug_get_grads: null pointer");
+  TGNN_CUDA_OK(ctx, cudaMemcpyAsync(grads_out, ctx->ws.grads, sizeof(float) * (size_t)ctx->L.total,
+                                    cudaMemcpyDeviceToDevice, S(stream)));
+  return TGNN_OK;
+}
+
+int tgnn_status(tgnn_ctx* ctx, int32_t* status_host, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, status_host, TGNN_EINVAL, "status: null pointer");
+  TGNN_CUDA_OK(ctx, cudaMemcpyAsync(status_host, ctx->ws.status, sizeof(int32_t), cudaMemcpyDeviceToHost, S(stream)));
+  TGNN_CUDA_OK(ctx, cudaStreamSynchronize(S(stream)));
+  return TGNN_OK;
+}
+
+int tgnn_profile_begin(tgnn_ctx* ctx) {
+  if (!ctx) return TGNN_EINVAL;
+  ctx->prof.used = 0;
+  ctx->prof.on = true;
+  return TGNN_OK;
+}
+
+int tgnn_profile_report(tgnn_ctx* ctx, char* buf, int64_t size) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, buf && size > 0, TGNN_EINVAL, "profile_report: null buffer");
+  ctx->prof.on = false;
+  TGNN_CUDA_OK(ctx, cudaDeviceSynchronize());
+  std::map<std::string, std::pair<long, double>> agg;
+  std::vector<std::string> order;
+  for (size_t i = 0; i < ctx->prof.used; ++i) {
+    const ProfEntry& e = ctx->prof.entries[i];
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, e.a, e.b) != cudaSuccess) { cudaGetLastError(); continue; }
+    auto it = agg.find(e.name);
+    if (it == agg.end()) { order.push_back(e.name); it = agg.emplace(e.name, std::make_pair(0L, 0.0)).first; }
+    it->second.first += 1;
+    it->second.second += ms;
+  }
+  std::string out;
+  char line[160];
+  for (const std::string& n : order) {
+    snprintf(line, sizeof(line), "%s %ld %.6f\n", n.c_str(), agg[n].first, agg[n].second);
+    out += line;
+  }
+  snprintf(buf, (size_t)size, "%s", out.c_str());
+  ctx->prof.used = 0;
+  return TGNN_OK;
+}
+
+}  // extern "C"

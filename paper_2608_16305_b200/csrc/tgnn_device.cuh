@@ -1,0 +1,45 @@
+// Small device helpers shared by the kernels.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace tgnn {
+
+// Phi(dt)_c = cos(fmaf(w_c, dt, b_c)) with the argument in fp32; cosf here is the
+// full-range accurate routine (the library is built without fast-math).
+__device__ __forceinline__ float time_arg(float w, float b, float dtf) { return fmaf(w, dtf, b); }
+__device__ __forceinline__ float time_encode(float w, float b, float dtf) { return cosf(time_arg(w, b, dtf)); }
+
+__device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + expf(-x)); }
+__device__ __forceinline__ float softplusf_(float x) { return x > 0.f ? x + log1pf(expf(-x)) : log1pf(expf(x)); }
+
+// Copy n floats with one warp: 128-bit accesses when both rows allow it.
+__device__ __forceinline__ void warp_copy_f32(float* __restrict__ dst, const float* __restrict__ src, int n, int lane) {
+  if ((((uintptr_t)dst | (uintptr_t)src) & 15) == 0 && (n & 3) == 0) {
+    const float4* s4 = reinterpret_cast<const float4*>(src);
+    float4* d4 = reinterpret_cast<float4*>(dst);
+    for (int q = lane; q < (n >> 2); q += 32) d4[q] = __ldg(s4 + q);
+  } else {
+    for (int q = lane; q < n; q += 32) dst[q] = __ldg(src + q);
+  }
+}
+
+// One edge-feature row (fp32 or bf16 table) into fp32.
+__device__ __forceinline__ void warp_copy_feat(float* __restrict__ dst, const void* __restrict__ efeat, int feat_bf16,
+                                               int64_t eid, int de, int lane) {
+  if (de == 0) return;
+  if (!feat_bf16) {
+    warp_copy_f32(dst, reinterpret_cast<const float*>(efeat) + eid * de, de, lane);
+  } else {
+    // rows are 2*de bytes, de even: 32-bit loads of bf16 pairs
+    const uint32_t* s = reinterpret_cast<const uint32_t*>(reinterpret_cast<const __nv_bfloat16*>(efeat) + eid * de);
+    for (int q = lane; q < (de >> 1); q += 32) {
+      const uint32_t v = __ldg(s + q);
+      dst[2 * q] = __uint_as_float(v << 16);
+      dst[2 * q + 1] = __uint_as_float(v & 0xffff0000u);
+    }
+  }
+}
+
+}  // namespace tgnn

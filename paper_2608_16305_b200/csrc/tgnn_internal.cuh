@@ -1,0 +1,215 @@
+// Internal declarations shared by the CUDA translation units of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/tgnn.h"
+
+namespace tgnn {
+
+// Offsets of the parameter tensors in the flat vector (order fixed by the public header).
+struct ParamLayout {
+  int64_t d, de, dmsg, dkv, dq;
+  int64_t time_w, time_b, gru_wi, gru_wh, gru_bi, gru_bh, wq, bq, wk, wv, bk, bv, wo, bo, w1, b1, w2, b2, total;
+};
+ParamLayout make_layout(int d, int d_e);
+
+// Workspace: everything the step keeps between entry points.  Row-major, fp32 unless noted.
+struct Workspace {
+  // step (0)
+  int32_t* hist;  // [N] zero between calls
+  // step (3)
+  unsigned long long* best_t;   // [N] zero between calls
+  unsigned long long* best_id;  // [N] zero between calls
+  int32_t* win_msg;             // [N]
+  int32_t* node2slot;           // [N], -1 except for the nodes updated by the last memory update
+  int32_t* prev_uniq;           // [2*max_events] nodes whose node2slot entry is set
+  int32_t* prev_n_uniq;         // [1]
+  // internal copies used by tgnn_train_step
+  int32_t* msg_node;  // [2*max_events]
+  int32_t* uniq;      // [2*max_events]
+  int32_t* winner;    // [2*max_events]
+  int32_t* n_uniq;    // [1]
+  int32_t* r_node;    // [max_roots]
+  double* r_time;     // [max_roots]
+  int32_t* nb_node;   // [max_roots*k]
+  int32_t* nb_eid;    // [max_roots*k]
+  double* nb_ts;      // [max_roots*k]
+  int32_t* nb_cnt;    // [max_roots]
+  float* h;           // [max_roots, d]
+  // host-input staging for tgnn_train_step_host
+  int32_t *st_u_src, *st_u_dst, *st_u_eid, *st_q_src, *st_q_dst, *st_q_neg;
+  double *st_u_t, *st_q_t;
+  uint8_t *st_u_keep, *st_mask;
+  float* st_scalars;  // [4] loss accumulator, spare, loss, gradient norm
+  // step (4) activations
+  float* X;        // [U_cap, ld_msg] winners' message rows (first d columns = the node's own memory)
+  float* x_dt;     // [U_cap] fp32 dt inside Phi of the winner message
+  double* win_t;   // [U_cap]
+  float* Gi;       // [U_cap, 3d]
+  float* Gh;       // [U_cap, 3d]
+  float *g_r, *g_z, *g_n, *g_hn;  // [U_cap, d]
+  // step (5) activations
+  float* Z;      // [NB_cap, ld_kv]
+  float* z_dt;   // [NB_cap]
+  float* KV;     // [NB_cap, 2d]  (K | V)
+  float* Zq;     // [R_cap, 2d]
+  float* Q;      // [R_cap, d]
+  float* alpha;  // [R_cap, H, k]
+  float* cat_o;  // [R_cap, 2d]  (a | m_root)
+  // step (6)
+  float* cat1;    // [2*nq_cap, 2d]
+  float* hid1;    // [2*nq_cap, d]  ReLU(pre1); overwritten by dpre1
+  float* dcat1;   // [2*nq_cap, 2d]
+  float* dpre_o;  // [R_cap, d]
+  float* dcat_o;  // [R_cap, 2d]
+  float* dQ;      // [R_cap, d]
+  float* dzq;     // [R_cap, 2d]
+  float* dKV;     // [NB_cap, 2d]
+  float* dZm;     // [NB_cap, d]  grad wrt the memory part of Z
+  float* dZp;     // [NB_cap, d]  grad wrt the time-encoding part of Z
+  float* dMemU;   // [U_cap, d]   grad wrt the rows written by the memory update
+  float* dGi;     // [U_cap, 3d]
+  float* dGh;     // [U_cap, 3d]
+  float* dXp;     // [U_cap, d]   grad wrt the time-encoding part of the winners' messages
+  float* grads;   // [P]
+  double* red;    // [4] sum of squares, mask sum, spare
+  float* adam_sc; // [4] bias corrections 1/(1-b1^t), 1/(1-b2^t)
+  unsigned int* counters;  // [4] "last block" tickets
+  int32_t* status;         // [1] device status word
+};
+
+// Optional per-kernel timing (tgnn_profile_begin / tgnn_profile_report): an event pair around
+// every launch while enabled.  Off by default; nothing is recorded or allocated then.
+struct ProfEntry {
+  const char* name;
+  cudaEvent_t a, b;
+};
+struct Profiler {
+  bool on = false;
+  std::vector<ProfEntry> entries;  // events are created once and reused
+  size_t used = 0;
+};
+
+}  // namespace tgnn
+
+struct tgnn_ctx {
+  tgnn_config cfg;
+  tgnn::ParamLayout L;
+  int U_cap, R_cap, NB_cap, nq_cap;
+  int ld_msg, ld_kv;  // padded leading dimensions of X and Z
+  // borrowed
+  const int64_t* indptr;
+  const int32_t *g_nbr, *g_eid;
+  const double* g_ts;
+  int64_t n_entries;
+  const void* efeat;
+  int64_t num_events;
+  float* memory;
+  double* last_update;
+  float *params, *adam_m, *adam_v;
+  int64_t* step;
+  // event arrays recorded by the last tgnn_build_messages
+  const int32_t *m_src, *m_dst, *m_eid;
+  const double* m_t;
+  const uint8_t* m_keep;
+  int m_n;
+  // arrays recorded by the last tgnn_embed
+  const int32_t *e_nodes, *e_nbr, *e_eid, *e_cnt;
+  const double *e_times, *e_ts;
+  int e_n;
+  const float* e_h;
+  // device count / capacity of the rows written by the last tgnn_memory_update
+  const int32_t* upd_n_uniq;
+  int upd_cap;
+  bool have_update, have_embed;
+  tgnn::Workspace ws;
+  void* arena;
+  size_t arena_bytes;
+  int64_t launches;
+  tgnn::Profiler prof;
+  char err[256];
+};
+
+namespace tgnn {
+
+int set_error(tgnn_ctx* ctx, int code, const char* fmt, ...);
+#define TGNN_CUDA_OK(ctx, expr)                                                              \
+  do {                                                                                       \
+    cudaError_t e__ = (expr);                                                                \
+    if (e__ != cudaSuccess) return tgnn::set_error(ctx, TGNN_ECUDA, "%s: %s", #expr, cudaGetErrorString(e__)); \
+  } while (0)
+#define TGNN_LAUNCH_OK(ctx, name)                                                            \
+  do {                                                                                       \
+    (ctx)->launches++;                                                                       \
+    cudaError_t e__ = cudaGetLastError();                                                    \
+    if (e__ != cudaSuccess) return tgnn::set_error(ctx, TGNN_ECUDA, "launch %s: %s", name, cudaGetErrorString(e__)); \
+  } while (0)
+
+// Brackets one kernel launch with events when profiling is on.
+struct KernelScope {
+  tgnn_ctx* c;
+  cudaStream_t s;
+  long idx;
+  KernelScope(tgnn_ctx* ctx, const char* name, cudaStream_t stream) : c(ctx), s(stream), idx(-1) {
+    Profiler& p = ctx->prof;
+    if (!p.on) return;
+    if (p.used == p.entries.size()) {
+      ProfEntry e{name, nullptr, nullptr};
+      if (cudaEventCreate(&e.a) != cudaSuccess || cudaEventCreate(&e.b) != cudaSuccess) return;
+      p.entries.push_back(e);
+    }
+    idx = (long)p.used++;
+    p.entries[idx].name = name;
+    cudaEventRecord(p.entries[idx].a, s);
+  }
+  ~KernelScope() {
+    if (idx >= 0) cudaEventRecord(c->prof.entries[idx].b, s);
+  }
+};
+
+// ---- integer kernels (k_index.cu) ----
+int launch_prune_mask(tgnn_ctx* ctx, const int32_t* src, const int32_t* dst, const int32_t* eid, const uint8_t* is_aux,
+                      int n, int force_heavy, uint32_t drop_q32, uint64_t seed, int64_t batch_idx, uint8_t* keep_out,
+                      int32_t* heavy_out, cudaStream_t s);
+int launch_sample_recent(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n, int32_t* nbr_out,
+                         int32_t* eid_out, double* ts_out, int32_t* cnt_out, cudaStream_t s);
+int launch_reduce_latest(tgnn_ctx* ctx, const int32_t* msg_node, const double* t, const int32_t* eid, int n_msg,
+                         int32_t* uniq_out, int32_t* winner_out, int32_t* n_uniq_out, cudaStream_t s);
+int launch_make_roots(tgnn_ctx* ctx, const int32_t* q_src, const int32_t* q_dst, const int32_t* q_neg,
+                      const double* q_t, int n_q, cudaStream_t s);
+
+// ---- memory path (k_memory.cu) ----
+int launch_build_messages(tgnn_ctx* ctx, const int32_t* src, const int32_t* dst, const double* t, const int32_t* eid,
+                          const uint8_t* keep, int n, float* msg_out, int32_t* msg_node_out, cudaStream_t s);
+int launch_memory_update(tgnn_ctx* ctx, const float* msg, const int32_t* uniq, const int32_t* winner,
+                         const int32_t* n_uniq, cudaStream_t s);
+
+// ---- embedding (k_embed.cu) ----
+int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n, const int32_t* nbr,
+                 const int32_t* eid, const double* ts, const int32_t* cnt, float* h_out, cudaStream_t s);
+
+// ---- backward + Adam (k_backward.cu) ----
+int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* loss_out, float* gradnorm_out,
+                    cudaStream_t s);
+
+// ---- dense projections (k_gemm.cu) ----
+// C[M,N] (+)= sum_k A(m,k) B(k,n) (+ bias[n]) (ReLU);  A(m,k) = A[m*a_rs + k*a_cs], B(k,n) = B[k*b_rs + n*b_cs].
+struct GemmArgs {
+  const float* A; int64_t a_rs, a_cs;
+  const float* B; int64_t b_rs, b_cs;
+  float* C; int64_t ldc;
+  int M, N, K;            // capacities when the matching device count is given
+  const int32_t* dev_M;   // optional device-side row count (<= M)
+  const int32_t* dev_K;   // optional device-side contraction length (<= K)
+  const float* bias;      // optional [N], added once
+  float* rowsum_out;      // optional [M]: += sum_k A(m,k) (bias gradient of a transposed product)
+  int relu;               // apply ReLU in the epilogue (store mode only)
+  int accumulate;         // atomicAdd into C (C must hold valid data); required when split_k > 1
+  int split_k;            // >= 1
+};
+int launch_gemm(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s);
+
+}  // namespace tgnn

@@ -1,0 +1,106 @@
+"""Device-resident workload and the per-batch driver around the C ABI.
+
+`DeviceWorkload` uploads a synthetic stream (events, T-CSR, edge features,
+mixed batches) once; `Trainer.step(b)` then issues the calls of one
+chronological training step in the lag-one order:
+
+    prune mask of mixed batch b          (step 0; kept for when b is replayed)
+    memory update from kept batch b-1    (steps 2-4)
+    sample / embed / loss / backward / Adam on the targets of batch b (steps 1,5,6)
+
+All arithmetic happens inside the library; this file only slices tensors.
+"""
+from __future__ import annotations
+
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import workload as wl
+
+
+class DeviceWorkload:
+    def __init__(self, stream: wl.EventStream, device="cuda", batches: Optional[range] = None,
+                 efeat: Optional[torch.Tensor] = None):
+        cfg = stream.cfg
+        self.cfg = cfg
+        self.stream = stream
+        dev = torch.device(device)
+        self.device = dev
+        t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+        self.src, self.dst, self.t, self.neg = t(stream.src), t(stream.dst), t(stream.t), t(stream.neg)
+        self.indptr, self.nbr, self.eid, self.ts = t(stream.indptr), t(stream.nbr), t(stream.eid), t(stream.ts)
+        if efeat is not None:
+            self.efeat = efeat
+        elif cfg.d_e == 0:
+            self.efeat = None
+        elif cfg.feat_dtype == "f32":
+            self.efeat = t(stream.efeat())
+        else:
+            self.efeat = torch.from_numpy(stream.efeat().view(np.int16)).to(dev).view(torch.bfloat16)
+        # mixed batches, concatenated; batch b occupies [off[b], off[b+1])
+        self.batches = batches if batches is not None else range(cfg.num_batches)
+        mbs = [wl.mixed_batch(stream, b) for b in self.batches]
+        self.mb_host: List[wl.MixedBatch] = mbs
+        off = np.zeros(len(mbs) + 1, dtype=np.int64)
+        np.cumsum([m.n for m in mbs], out=off[1:])
+        self.mb_off = off
+        cat = lambda f, dt: t(np.concatenate([getattr(m, f) for m in mbs]).astype(dt)) if mbs else None
+        self.mb_src, self.mb_dst = cat("src", np.int32), cat("dst", np.int32)
+        self.mb_t, self.mb_eid, self.mb_aux = cat("t", np.float64), cat("eid", np.int32), cat("is_aux", np.uint8)
+        self.mb_keep = torch.ones_like(self.mb_aux)
+        self.heavy = torch.zeros(len(mbs), dtype=torch.int32, device=dev)
+
+    def mb_slice(self, b: int):
+        i = b - self.batches.start
+        return slice(int(self.mb_off[i]), int(self.mb_off[i + 1]))
+
+    def target_slice(self, b: int):
+        return slice(b * self.cfg.batch, min((b + 1) * self.cfg.batch, self.cfg.num_events))
+
+
+class Trainer:
+    def __init__(self, dw: DeviceWorkload, weights, math_mode=B.TGNN_MATH_FP32, lr=1e-4):
+        cfg = dw.cfg
+        self.dw = dw
+        self.tcfg = B.make_config(cfg.num_nodes, cfg.d, cfg.d_e, cfg.k, cfg.heads,
+                                  feat_dtype=B.TGNN_BF16 if cfg.feat_dtype == "bf16" else B.TGNN_F32,
+                                  max_events=cfg.max_mixed, max_roots=3 * cfg.batch, math_mode=math_mode, lr=lr)
+        self.lib = B.Tgnn(self.tcfg)
+        dev = dw.device
+        P = B.param_layout(self.tcfg)["total"]
+        self.memory = torch.zeros((cfg.num_nodes, cfg.d), dtype=torch.float32, device=dev)
+        self.last_update = torch.zeros(cfg.num_nodes, dtype=torch.float64, device=dev)
+        self.params = torch.from_numpy(B.pack_params(self.tcfg, weights)).to(dev)
+        self.adam_m = torch.zeros(P, dtype=torch.float32, device=dev)
+        self.adam_v = torch.zeros(P, dtype=torch.float32, device=dev)
+        self.step_count = torch.zeros(1, dtype=torch.int64, device=dev)
+        self.loss = torch.zeros(1, dtype=torch.float32, device=dev)
+        self.gradnorm = torch.zeros(1, dtype=torch.float32, device=dev)
+        self.lib.set_graph(dw.indptr, dw.nbr, dw.eid, dw.ts)
+        self.lib.set_edge_features(dw.efeat, cfg.num_events)
+        self.lib.set_state(self.memory, self.last_update, self.params, self.adam_m, self.adam_v, self.step_count)
+        self.prune_seed = cfg.seed
+        self.drop_q32 = 1 << 31
+
+    def prune(self, b: int):
+        dw = self.dw
+        s = dw.mb_slice(b)
+        i = b - dw.batches.start
+        self.lib.prune_mask(dw.mb_src[s], dw.mb_dst[s], dw.mb_eid[s], dw.mb_aux[s], dw.mb_keep[s], dw.heavy[i:i + 1],
+                            force_heavy=-1 if dw.cfg.prune else 0, drop_q32=self.drop_q32, seed=self.prune_seed,
+                            batch_idx=b)
+
+    def step(self, b: int, with_update: bool = True):
+        """One training step on batch b (device-resident inputs)."""
+        dw = self.dw
+        self.prune(b)
+        q = dw.target_slice(b)
+        if with_update and b > dw.batches.start:
+            u = dw.mb_slice(b - 1)
+            upd = (dw.mb_src[u], dw.mb_dst[u], dw.mb_t[u], dw.mb_eid[u], dw.mb_keep[u])
+        else:
+            upd = (None, None, None, None, None)
+        self.lib.train_step(*upd, dw.src[q], dw.dst[q], dw.neg[q], dw.t[q], None, self.loss, self.gradnorm)

@@ -1,0 +1,422 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by
+element on the same seeded inputs.  Integers, indices and masks must be
+bit-exact; floats are compared teacher-forced per batch (the oracle starts each
+step from the GPU's pre-step state) with
+
+    err(x) = max|x_gpu - x_ref| / max(max|x_ref|, 1e-6)
+
+<= 2e-3 for the TF32 tensor-core mode (<= 1e-2 with bf16 features), and a much
+tighter 2e-5 for the fp32 FMA mode, per compared tensor: updated memory rows,
+embeddings h, loss, gradient norm, every gradient tensor, and the Adam update
+(checked against the oracle's Adam fed with the GPU gradient, since Adam's
+g/(|g|+eps) amplifies rounding noise of near-zero gradients without bound).
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_16305_b200 import workload as wl
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"fp32": 2e-5, "tf32": 2e-3, "tf32_bf16": 1e-2}
+
+
+def relerr(gpu, ref):
+    gpu, ref = np.asarray(gpu, np.float64), np.asarray(ref, np.float64)
+    if ref.size == 0:
+        return 0.0
+    return float(np.abs(gpu - ref).max() / max(np.abs(ref).max(), 1e-6))
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2608_16305_b200 import binding
+    binding.load_library()
+    return binding
+
+
+def dev(a, dt=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dt is not None:
+        t = t.to(dt)
+    return t.cuda()
+
+
+def orc_cfg(oracle, c, **kw):
+    return oracle.make_config(c.num_nodes, c.d, c.d_e, c.k, c.heads, feat_bf16=c.feat_dtype == "bf16", **kw)
+
+
+# ------------------------------------------------------------ set-up -------
+class Rig:
+    """A workload on the device plus a library context and an oracle configuration."""
+
+    def __init__(self, B, oracle, cfg, math="fp32", batches=None, bias_scale=0.1, lr=1e-3):
+        from paper_2608_16305_b200 import trainer
+        self.B, self.oracle, self.cfg, self.math = B, oracle, cfg, math
+        self.stream = wl.make_stream(cfg)
+        self.dw = trainer.DeviceWorkload(self.stream, batches=batches)
+        self.weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed, bias_scale=bias_scale)
+        mode = B.TGNN_MATH_FP32 if math == "fp32" else B.TGNN_MATH_TF32
+        self.tr = trainer.Trainer(self.dw, self.weights, math_mode=mode, lr=lr)
+        self.ocfg = orc_cfg(oracle, cfg, lr=lr)
+        self.graph = (self.stream.indptr, self.stream.nbr, self.stream.eid, self.stream.ts)
+        self.efeat = self.stream.efeat() if cfg.d_e else None
+        self.lay = B.param_layout(self.tr.tcfg)
+        self.shapes = wl.param_shapes(cfg.d, cfg.d_e)
+        key = math + ("_bf16" if cfg.feat_dtype == "bf16" and math != "fp32" else "")
+        self.tol = TOL[key]
+
+    def snapshot(self):
+        tr = self.tr
+        torch.cuda.synchronize()
+        return dict(memory=tr.memory.cpu().numpy().astype(np.float64), last_update=tr.last_update.cpu().numpy().copy(),
+                    params=tr.params.cpu().numpy().astype(np.float64), m=tr.adam_m.cpu().numpy().astype(np.float64),
+                    v=tr.adam_v.cpu().numpy().astype(np.float64), step=int(tr.step_count.item()))
+
+    def upd_host(self, b):
+        """Kept update events of batch b-1 as the oracle wants them (or None)."""
+        if b <= self.dw.batches.start:
+            return None
+        mb = self.dw.mb_host[b - 1 - self.dw.batches.start]
+        keep = self.dw.mb_keep[self.dw.mb_slice(b - 1)].cpu().numpy()
+        return (mb.src, mb.dst, mb.t, mb.eid, keep)
+
+    def oracle_step(self, pre, b):
+        o, s = self.oracle, self.stream
+        q = self.dw.target_slice(b)
+        nodes = np.concatenate([s.src[q], s.dst[q], s.neg[q]])
+        times = np.concatenate([s.t[q]] * 3)
+        nb = o.sample_recent(*self.graph, nodes, times, self.cfg.k)
+        upd = self.upd_host(b)
+        if upd is None:
+            z = np.zeros(0, np.int32)
+            upd = (z, z, np.zeros(0), z, None)
+        res = o.loss_and_grads(self.ocfg, pre["params"], pre["memory"], pre["last_update"], self.efeat, upd,
+                               (nodes, times) + nb, q.stop - q.start, None)
+        return res, (nodes, times) + nb
+
+    def check_step(self, b, pre, res, what=""):
+        """Compare the GPU's post-step state with the oracle's result from `pre`."""
+        tr, o, tol = self.tr, self.oracle, self.tol
+        torch.cuda.synchronize()
+        assert tr.lib.status() == 0
+        mem = tr.memory.cpu().numpy()
+        lu = tr.last_update.cpu().numpy()
+        assert np.array_equal(lu, res.last_update_post), f"{what} last_update"
+        untouched = np.ones(self.cfg.num_nodes, bool)
+        untouched[res.uniq] = False
+        assert np.array_equal(mem[untouched], pre["memory"][untouched].astype(np.float32)), f"{what} untouched rows"
+        e = relerr(mem[res.uniq], res.memory_post[res.uniq])
+        assert e <= tol, f"{what} memory rows err {e}"
+        e = abs(float(tr.loss.item()) - res.loss) / max(abs(res.loss), 1e-6)
+        assert e <= tol, f"{what} loss {tr.loss.item()} vs {res.loss}"
+        g = torch.zeros_like(tr.params)
+        tr.lib.debug_get_grads(g)
+        g = g.cpu().numpy().astype(np.float64)
+        for name in self.B.PARAM_NAMES:
+            sl = slice(self.lay[name], self.lay[name] + int(np.prod(self.shapes[name])))
+            e = relerr(g[sl], res.grads[sl])
+            assert e <= tol, f"{what} grad {name} err {e}"
+        e = abs(float(tr.gradnorm.item()) - res.gradnorm) / max(res.gradnorm, 1e-6)
+        assert e <= tol, f"{what} gradnorm {tr.gradnorm.item()} vs {res.gradnorm}"
+        # Adam, fed with the GPU's own gradient
+        p_ref, m_ref, v_ref, st = o.adam(self.ocfg, g, pre["params"], pre["m"], pre["v"], pre["step"])
+        assert int(tr.step_count.item()) == st
+        upd_gpu = tr.params.cpu().numpy().astype(np.float64) - pre["params"]
+        e = np.abs(upd_gpu - (p_ref - pre["params"])).max() / self.ocfg.lr
+        assert e <= 1e-3, f"{what} adam update err {e} (units of lr)"
+        assert relerr(tr.adam_m.cpu().numpy(), m_ref) <= 1e-5 and relerr(tr.adam_v.cpu().numpy(), v_ref) <= 1e-5
+
+
+TINY = wl.CONFIGS["tiny"]
+
+
+@pytest.fixture(scope="module")
+def tiny_rig(B, oracle):
+    return Rig(B, oracle, TINY)
+
+
+# ------------------------------------------------------------ step (0) -----
+@pytest.mark.parametrize("case", ["uniform", "hub", "mixed", "one", "ragged"])
+def test_prune_mask_bit_exact(B, oracle, case):
+    rng = np.random.default_rng(21)
+    N = 5000
+    if case == "uniform":
+        n = 600
+        src, dst = rng.permutation(N)[:n], rng.permutation(N)[:n]
+    elif case == "hub":
+        n = 4000
+        src, dst = np.zeros(n, np.int64), rng.integers(1, N, n)
+    elif case == "one":
+        n, src, dst = 1, np.array([7]), np.array([7])
+    else:
+        n = 1337 if case == "ragged" else 4800
+        p = 1.0 / np.arange(1, N + 1) ** 1.3
+        p /= p.sum()
+        src, dst = rng.choice(N, n, p=p), rng.choice(N, n, p=p)
+    eid = rng.permutation(10 * n)[:n]
+    aux = (rng.random(n) < 0.3).astype(np.uint8)
+    lib = B.Tgnn(B.make_config(N, 32, 16, 10, 2, max_events=5000, max_roots=3000))
+    d_src, d_dst, d_eid, d_aux = dev(src, torch.int32), dev(dst, torch.int32), dev(eid, torch.int32), dev(aux)
+    keep = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    heavy = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for force, q32, bidx in [(-1, 1 << 31, 0), (-1, 1 << 31, 5), (1, 1 << 30, 2), (1, 0xFFFFFFFF, 1), (0, 1 << 31, 3)]:
+        k_ref, h_ref = oracle.prune_mask(N, src, dst, eid, aux, force_heavy=force, drop_q32=q32, seed=99, batch_idx=bidx)
+        lib.prune_mask(d_src, d_dst, d_eid, d_aux, keep, heavy, force_heavy=force, drop_q32=q32, seed=99, batch_idx=bidx)
+        assert int(heavy.item()) == h_ref
+        assert np.array_equal(keep.cpu().numpy(), k_ref)
+        assert k_ref[aux == 0].all()                         # targets are never pruned
+    lib.close()
+
+
+# ------------------------------------------------------------ step (1) -----
+def test_sample_recent_bit_exact_tiny_stream(tiny_rig):
+    r = tiny_rig
+    s = r.stream
+    rng = np.random.default_rng(22)
+    nodes = np.concatenate([s.src, s.dst, s.neg[:5000], rng.integers(0, TINY.num_nodes, 3001).astype(np.int32)])
+    times = np.concatenate([s.t, s.t, s.t[:5000], rng.uniform(-1, s.t[-1] + 5, 3001)])
+    _check_sample(r.tr.lib, r.oracle, r.graph, nodes, times, TINY.k)
+
+
+def test_sample_recent_long_slices_and_ties(B, oracle):
+    # one hub with ~40k entries (several 32-way rounds), integer timestamps (ties), queries on and between ties
+    rng = np.random.default_rng(23)
+    N, E = 50, 40000
+    src = np.where(rng.random(E) < 0.9, 0, rng.integers(0, N, E)).astype(np.int32)
+    dst = rng.integers(1, N, E).astype(np.int32)
+    t = np.cumsum(rng.integers(0, 3, E)).astype(np.float64)
+    g = wl.build_tcsr(src, dst, t, N)
+    lib = B.Tgnn(B.make_config(N, 32, 16, 10, 2))
+    lib.set_graph(*[dev(a) for a in g])
+    nodes = rng.integers(0, N, 4099).astype(np.int32)
+    nodes[::3] = 0
+    times = rng.integers(-1, int(t[-1]) + 3, 4099).astype(np.float64) + rng.choice([0.0, 0.5], 4099)
+    _check_sample(lib, oracle, g, nodes, times, 10)
+    lib.close()
+
+
+def _check_sample(lib, oracle, graph, nodes, times, k):
+    n = len(nodes)
+    nb = torch.full((n, k), 77, dtype=torch.int32, device="cuda")
+    ne = torch.full((n, k), 77, dtype=torch.int32, device="cuda")
+    nt = torch.full((n, k), 7.0, dtype=torch.float64, device="cuda")
+    nc = torch.full((n,), 77, dtype=torch.int32, device="cuda")
+    lib.sample_recent(dev(nodes, torch.int32), dev(times, torch.float64), nb, ne, nt, nc)
+    ref = oracle.sample_recent(*graph, nodes, times, k)
+    for got, want in zip((nb, ne, nt, nc), ref):
+        assert np.array_equal(got.cpu().numpy(), want)
+
+
+# ----------------------------------------------------- steps (2)-(4) -------
+def _state_for_parts(r, seed=24):
+    """Random non-trivial state uploaded into the rig's trainer."""
+    rng = np.random.default_rng(seed)
+    c = r.cfg
+    mem = (rng.normal(size=(c.num_nodes, c.d)) * 0.5).astype(np.float32)
+    lu = (rng.random(c.num_nodes) * r.stream.t[2000]).astype(np.float64)
+    r.tr.memory.copy_(dev(mem))
+    r.tr.last_update.copy_(dev(lu))
+    return mem, lu
+
+
+def test_messages_reduction_and_gru_by_parts(tiny_rig):
+    r, o, c = tiny_rig, tiny_rig.oracle, TINY
+    tr = r.tr
+    mem, lu = _state_for_parts(r)
+    P = tr.params.cpu().numpy().astype(np.float64)
+    mb = r.dw.mb_host[10]
+    n = mb.n
+    rng = np.random.default_rng(25)
+    keep = (rng.random(n) < 0.85).astype(np.uint8)
+    sl = r.dw.mb_slice(10)
+    d_src, d_dst, d_t, d_eid = r.dw.mb_src[sl], r.dw.mb_dst[sl], r.dw.mb_t[sl], r.dw.mb_eid[sl]
+    d_keep = dev(keep)
+    msg = torch.zeros((2 * n, c.d_msg), dtype=torch.float32, device="cuda")
+    node = torch.zeros(2 * n, dtype=torch.int32, device="cuda")
+    tr.lib.build_messages(d_src, d_dst, d_t, d_eid, d_keep, msg, node)
+    msg_ref, node_ref = o.build_messages(r.ocfg, P, mem, lu, r.efeat, mb.src, mb.dst, mb.t, mb.eid, keep)
+    assert np.array_equal(node.cpu().numpy(), node_ref)
+    got = msg.cpu().numpy()
+    assert np.array_equal(got[:, :2 * c.d + c.d_e], msg_ref[:, :2 * c.d + c.d_e].astype(np.float32))   # pure gathers
+    assert np.abs(got[:, 2 * c.d + c.d_e:] - msg_ref[:, 2 * c.d + c.d_e:]).max() <= 2e-6                # cos in fp32
+    # reduction
+    uniq = torch.zeros(2 * n, dtype=torch.int32, device="cuda")
+    win = torch.zeros(2 * n, dtype=torch.int32, device="cuda")
+    nu = torch.zeros(1, dtype=torch.int32, device="cuda")
+    tr.lib.reduce_latest(node, d_t, d_eid, uniq, win, nu)
+    u_ref, w_ref = o.reduce_latest(node_ref, mb.t, mb.eid, c.num_nodes)
+    U = int(nu.item())
+    assert U == len(u_ref)
+    assert np.array_equal(uniq[:U].cpu().numpy(), u_ref) and np.array_equal(win[:U].cpu().numpy(), w_ref)
+    # GRU from the materialised rows, then (fresh state) from virtual rows: same result
+    mem_ref, lu_ref = o.memory_update(r.ocfg, P, msg_ref, mb.t, u_ref, w_ref, mem, lu)
+    for virtual in (False, True):
+        tr.memory.copy_(dev(mem))
+        tr.last_update.copy_(dev(lu))
+        if virtual:
+            tr.lib.build_messages(d_src, d_dst, d_t, d_eid, d_keep, None, node)
+            tr.lib.reduce_latest(node, d_t, d_eid, uniq, win, nu)
+        tr.lib.memory_update(None if virtual else msg, uniq, win, nu)
+        got_m, got_lu = tr.memory.cpu().numpy(), tr.last_update.cpu().numpy()
+        assert np.array_equal(got_lu, lu_ref)
+        assert relerr(got_m[u_ref], mem_ref[u_ref]) <= r.tol
+        rest = np.setdiff1d(np.arange(c.num_nodes), u_ref)
+        assert np.array_equal(got_m[rest], mem[rest])
+
+
+@pytest.mark.parametrize("case", ["ties_unsorted", "hub", "all_dropped", "empty"])
+def test_reduce_latest_bit_exact(B, oracle, case):
+    rng = np.random.default_rng(26)
+    N = 3000
+    lib = B.Tgnn(B.make_config(N, 32, 16, 10, 2, max_events=6000, max_roots=3000))
+    if case == "empty":
+        n = 0
+    elif case == "hub":
+        n = 5200
+    else:
+        n = 777
+    src = rng.integers(0, N, n).astype(np.int32)
+    dst = rng.integers(0, N, n).astype(np.int32)
+    if case == "hub":
+        src[rng.random(n) < 0.6] = 5
+        dst[rng.random(n) < 0.3] = 5
+    t = rng.integers(0, 40, n).astype(np.float64) - (3.0 if case == "ties_unsorted" else 0.0)   # ties, unsorted, some negative
+    eid = rng.permutation(3 * n + 1)[:n].astype(np.int32)
+    node = np.stack([src, dst], 1).reshape(-1).astype(np.int32)
+    drop = np.repeat(rng.random(n) < (1.0 if case == "all_dropped" else 0.2), 2)
+    node[drop] = -1
+    u_ref, w_ref = oracle.reduce_latest(node, t, eid, N)
+    uniq = torch.zeros(max(2 * n, 1), dtype=torch.int32, device="cuda")
+    win = torch.zeros(max(2 * n, 1), dtype=torch.int32, device="cuda")
+    nu = torch.full((1,), -5, dtype=torch.int32, device="cuda")
+    for rep in range(2):                                     # second call: the scratch tables were left clean
+        lib.reduce_latest(dev(node), dev(t), dev(eid), uniq, win, nu)
+        U = int(nu.item())
+        assert U == len(u_ref)
+        assert np.array_equal(uniq[:U].cpu().numpy(), u_ref) and np.array_equal(win[:U].cpu().numpy(), w_ref)
+    lib.close()
+
+
+# ------------------------------------------------------------ step (5) -----
+def test_embed_by_parts(tiny_rig):
+    r, o, c = tiny_rig, tiny_rig.oracle, TINY
+    tr = r.tr
+    mem, _ = _state_for_parts(r, seed=27)
+    P = tr.params.cpu().numpy().astype(np.float64)
+    s = r.stream
+    q = slice(6000, 6190)
+    nodes = np.concatenate([s.src[q], s.dst[q], s.neg[q], s.src[:7]])       # ragged count, early events with cnt < k
+    times = np.concatenate([s.t[q]] * 3 + [s.t[:7]])
+    nb = o.sample_recent(*r.graph, nodes, times, c.k)
+    assert (nb[3] == 0).any() and (nb[3] == c.k).any()
+    h = torch.zeros((len(nodes), c.d), dtype=torch.float32, device="cuda")
+    tr.lib.embed(dev(nodes), dev(times), dev(nb[0]), dev(nb[1]), dev(nb[2]), dev(nb[3]), h)
+    h_ref = o.embed(r.ocfg, P, mem, r.efeat, nodes, times, *nb)
+    assert relerr(h.cpu().numpy(), h_ref) <= r.tol
+    # the call recorded an embedding of 577 rows: a backward with a mismatching n_q is rejected on the host
+    rc = tr.lib.call_raw("tgnn_backward_step", 200, None, None, None, None)
+    assert rc == B_ESHAPE
+
+
+B_ESHAPE = -2
+
+
+# ------------------------------------------------- whole step, teacher-forced
+def _run_epoch_checks(rig, steps, check_at):
+    for b in steps:
+        pre = rig.snapshot() if b in check_at else None
+        rig.tr.step(b)
+        if pre is not None:
+            res, _ = rig.oracle_step(pre, b)
+            rig.check_step(b, pre, res, what=f"[{rig.cfg.name} batch {b}]")
+
+
+def test_tiny_epoch_teacher_forced(B, oracle):
+    rig = Rig(B, oracle, TINY)
+    nb = TINY.num_batches
+    _run_epoch_checks(rig, range(nb), {0, 1, 2, 3, 10, 37, nb // 2, nb - 2, nb - 1})
+    assert rig.tr.lib.kernel_launches() > 0
+
+
+def test_tiny_default_init_zero_biases(B, oracle):
+    rig = Rig(B, oracle, TINY, bias_scale=0.0)
+    _run_epoch_checks(rig, range(0, 6), {0, 1, 5})
+
+
+def _scaled(name, events, **kw):
+    c = wl.CONFIGS[name]
+    return wl.scaled(c, num_events=events, **kw)
+
+
+@pytest.mark.parametrize("name,events,at", [
+    ("wiki", 6000, {1, 5, 9}),          # 172-d features, d = 100: ragged tiles everywhere
+    ("reddit", 9000, {2, 8, 14}),       # replay events + pruning
+    ("lastfm", 24000, {1, 3, 5}),       # no edge features, heavy skew, batch 4000
+])
+def test_scaled_configs_teacher_forced(B, oracle, name, events, at):
+    rig = Rig(B, oracle, _scaled(name, events))
+    _run_epoch_checks(rig, range(rig.cfg.num_batches), at)
+    if rig.cfg.prune:
+        heavy = rig.dw.heavy.cpu().numpy()
+        keep = rig.dw.mb_keep.cpu().numpy()
+        aux = rig.dw.mb_aux.cpu().numpy()
+        assert keep[aux == 0].all()
+        # pruning really happened on heavy batches and only there
+        for i, b in enumerate(rig.dw.batches):
+            s = rig.dw.mb_slice(b)
+            mb = rig.dw.mb_host[i]
+            k_ref, h_ref = rig.oracle.prune_mask(rig.cfg.num_nodes, mb.src, mb.dst, mb.eid, mb.is_aux, seed=rig.cfg.seed,
+                                                 batch_idx=b)
+            assert h_ref == heavy[i] and np.array_equal(keep[s], k_ref)
+
+
+def test_bf16_feature_table(B, oracle):
+    c = wl.scaled(wl.CONFIGS["large"], num_events=20000, num_nodes=3000, batch=1000)
+    rig = Rig(B, oracle, c)
+    _run_epoch_checks(rig, range(8), {1, 4, 7})
+
+
+def test_host_buffer_entry_point_matches_device_path(B, oracle):
+    a = Rig(B, oracle, TINY)
+    b = Rig(B, oracle, TINY)
+    loss = torch.zeros(1).pin_memory()
+    gn = torch.zeros(1).pin_memory()
+    for step in range(4):
+        a.tr.step(step)
+        b.tr.prune(step)
+        q = b.dw.target_slice(step)
+        s = b.stream
+        pin = lambda x: torch.from_numpy(np.ascontiguousarray(x)).pin_memory()
+        upd = b.upd_host(step)
+        upd = tuple(pin(x) for x in upd) if upd is not None else (None,) * 5
+        b.tr.lib.train_step_host(*upd, pin(s.src[q]), pin(s.dst[q]), pin(s.neg[q]), pin(s.t[q]), None, loss, gn)
+        torch.cuda.synchronize()
+        assert float(loss.item()) == float(a.tr.loss.item()) and float(gn.item()) == float(a.tr.gradnorm.item())
+    # atomics make float sums order-dependent: compare within rounding, not bitwise
+    assert relerr(b.tr.memory.cpu().numpy(), a.tr.memory.cpu().numpy()) <= 1e-5
+    assert relerr(b.tr.params.cpu().numpy(), a.tr.params.cpu().numpy()) <= 1e-5
+
+
+# ------------------------------------------------------------ errors -------
+def test_argument_errors_are_reported_not_launched(B):
+    lib = B.Tgnn(B.make_config(100, 32, 16, 10, 2, max_events=64, max_roots=96))
+    z = torch.zeros(200, dtype=torch.int32, device="cuda")
+    zt = torch.zeros(200, dtype=torch.float64, device="cuda")
+    zu = torch.zeros(200, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.TgnnError) as e:
+        lib.sample_recent(z[:10], zt[:10], z, z, zt, z)                    # graph not set
+    assert e.value.code == B.TGNN_ESTATE
+    with pytest.raises(B.TgnnError) as e:
+        lib.prune_mask(z[:100], z[:100], z[:100], zu[:100], zu, z)         # over capacity
+    assert e.value.code == B.TGNN_ECAPACITY and "max_events" in str(e.value)
+    with pytest.raises(B.TgnnError) as e:
+        lib.backward_step(10, None, None, None)                            # nothing embedded
+    assert e.value.code == B.TGNN_ESTATE
+    assert lib.call_raw("tgnn_prune_mask", None, None, None, None, 5, -1, 0, 0, 0, None, None, None) == B.TGNN_EINVAL
+    bad = B.make_config(100, 30, 16, 10, 2)                                  # d not a multiple of 4
+    with pytest.raises(B.TgnnError):
+        B.Tgnn(bad)
+    assert lib.status() == 0
+    lib.close()
