@@ -180,29 +180,37 @@ __global__ void __launch_bounds__(256) scatter_dmem_kernel(const float* __restri
 
 // Time-encoder gradient from a block of rows: G[r, col0 + c] is d loss / d Phi(dt_r)_c.
 //   dw_c += -sin(arg) dt_r G,  db_c += -sin(arg) G,  arg = fmaf(w_c, dt_r, b_c)
-// Thread c walks the rows of the block's chunk; one pair of atomics per block and column.
+// The terms are large (dt reaches the time span of the stream) and cancel, so they are summed
+// in fp64: thread c walks the rows of the block's chunk, one pair of fp64 atomics per block
+// and column into acc[0:d] (dw) and acc[d:2d] (db).
 __global__ void __launch_bounds__(128) time_grad_kernel(const float* __restrict__ G, int64_t ldg, int col0,
                                                         const float* __restrict__ dt, int rows,
                                                         const int32_t* __restrict__ dev_rows, int rows_per_block, int d,
                                                         const float* __restrict__ time_w, const float* __restrict__ time_b,
-                                                        float* __restrict__ g_w, float* __restrict__ g_b) {
+                                                        double* __restrict__ acc) {
   const int R = dev_rows ? min(*dev_rows, rows) : rows;
   const int r0 = blockIdx.x * rows_per_block, r1 = min(R, r0 + rows_per_block);
   if (r0 >= r1) return;
   for (int c = threadIdx.x; c < d; c += blockDim.x) {
     const float w = time_w[c], b = time_b[c];
-    float gw = 0.f, gb = 0.f;
+    double gw = 0.0, gb = 0.0;
     for (int r = r0; r < r1; ++r) {
       const float g = G[(int64_t)r * ldg + col0 + c];
       if (g == 0.f) continue;
       const float dtr = dt ? dt[r] : 0.f;
-      const float sn = -sinf(time_arg(w, b, dtr)) * g;
-      gw = fmaf(sn, dtr, gw);
+      const double sn = -(double)sinf(time_arg(w, b, dtr)) * (double)g;
+      gw = fma(sn, (double)dtr, gw);
       gb += sn;
     }
-    if (gw != 0.f) atomicAdd(&g_w[c], gw);
-    if (gb != 0.f) atomicAdd(&g_b[c], gb);
+    if (gw != 0.0) atomicAdd(&acc[c], gw);
+    if (gb != 0.0) atomicAdd(&acc[d + c], gb);
   }
+}
+
+// Rounds the fp64 time-encoder sums into the fp32 gradient vector (time_w and time_b are adjacent).
+__global__ void time_grad_finish_kernel(const double* __restrict__ acc, int n, float* __restrict__ g_time) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c < n) g_time[c] = (float)acc[c];
 }
 
 // Backward of the GRU gates for the rows the memory update wrote.
@@ -274,10 +282,12 @@ __global__ void __launch_bounds__(256) adam_kernel(float* __restrict__ p, float*
                                                    const float* __restrict__ g, int64_t P, float lr, float beta1,
                                                    float beta2, float eps, const float* __restrict__ adam_sc) {
   const float c1 = adam_sc[0], c2 = adam_sc[1];
+  // 1 - beta formed in fp64 from the configured fp32 value, then rounded once
+  const float omb1 = (float)(1.0 - (double)beta1), omb2 = (float)(1.0 - (double)beta2);
   for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < P; e += (int64_t)gridDim.x * blockDim.x) {
     const float ge = g[e];
-    const float me = fmaf(beta1, m[e], (1.f - beta1) * ge);
-    const float ve = fmaf(beta2, v[e], (1.f - beta2) * ge * ge);
+    const float me = fmaf(beta1, m[e], omb1 * ge);
+    const float ve = fmaf(beta2, v[e], omb2 * ge * ge);
     m[e] = me;
     v[e] = ve;
     p[e] -= lr * (me * c1) / (sqrtf(ve * c2) + eps);
@@ -380,13 +390,13 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     {
       KernelScope scope__(ctx, "time_grad_z", s);
       time_grad_kernel<<<(NB + rpb - 1) / rpb, 128, 0, s>>>(w.dZp, d, 0, w.z_dt, NB, nullptr, rpb, d, P + L.time_w,
-                                                            P + L.time_b, G + L.time_w, G + L.time_b);
+                                                            P + L.time_b, w.tg_acc);
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_z");
     {
       KernelScope scope__(ctx, "time_grad_q", s);
       time_grad_kernel<<<(R + rpb - 1) / rpb, 128, 0, s>>>(w.dzq, 2 * d, d, nullptr, R, nullptr, rpb, d, P + L.time_w,
-                                                           P + L.time_b, G + L.time_w, G + L.time_b);
+                                                           P + L.time_b, w.tg_acc);
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_q");
     if (ctx->have_update) {
@@ -414,10 +424,17 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       {
         KernelScope scope__(ctx, "time_grad_x", s);
         time_grad_kernel<<<(U_cap + rpb - 1) / rpb, 128, 0, s>>>(w.dXp, d, 0, w.x_dt, U_cap, ctx->upd_n_uniq, rpb, d,
-                                                                 P + L.time_w, P + L.time_b, G + L.time_w, G + L.time_b);
+                                                                 P + L.time_w, P + L.time_b, w.tg_acc);
       }
       TGNN_LAUNCH_OK(ctx, "time_grad_x");
     }
+  }
+  if (n_q > 0) {
+    {
+      KernelScope scope__(ctx, "time_grad_finish", s);
+      time_grad_finish_kernel<<<(2 * d + 127) / 128, 128, 0, s>>>(w.tg_acc, 2 * d, G + L.time_w);
+    }
+    TGNN_LAUNCH_OK(ctx, "time_grad_finish");
   }
   {
     KernelScope scope__(ctx, "gradnorm", s);

@@ -138,10 +138,11 @@ size_t carve(tgnn_ctx* ctx, char* base) {
   cv.take(w.adam_sc, 4);
   cv.take(w.counters, 4);
   cv.take(w.status, 4);
-  // cleared together at the start of every backward pass: keep these four adjacent and in this order
+  // cleared together at the start of every backward pass: keep these five adjacent and in this order
   cv.take(w.grads, (size_t)ctx->L.total);
   cv.take_packed(w.dMemU, U * d);
   cv.take_packed(w.red, 4);
+  cv.take_packed(w.tg_acc, 2 * d);
   cv.take_packed(w.st_scalars, 4);
   return (cv.off + 255) & ~(size_t)255;
 }

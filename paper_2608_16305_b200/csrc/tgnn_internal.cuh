@@ -75,7 +75,8 @@ struct Workspace {
   float* dGh;     // [U_cap, 3d]
   float* dXp;     // [U_cap, d]   grad wrt the time-encoding part of the winners' messages
   float* grads;   // [P]
-  double* red;    // [4] sum of squares, mask sum, spare
+  double* red;    // [4] sum of squares, spare
+  double* tg_acc; // [2d] fp64 sums of the time-encoder gradient (dw | db)
   float* adam_sc; // [4] bias corrections 1/(1-b1^t), 1/(1-b2^t)
   unsigned int* counters;  // [4] "last block" tickets
   int32_t* status;         // [1] device status word
