@@ -229,6 +229,38 @@ TGNN_API int tgnn_status(tgnn_ctx* ctx, int32_t* status_host, void* stream);
 /* Number of kernels this context has launched since creation (host counter). */
 TGNN_API int64_t tgnn_kernel_launches(const tgnn_ctx* ctx);
 
+/* ---- for callers that cannot allocate --------------------------------------- */
+
+/* The paper has no counterpart to this entry point; it exists for hosts that
+ * keep every byte of device memory under their own plan -- a serving process
+ * with a fixed memory budget, a framework sandbox that hands an operator only
+ * the buffers it was given -- where a cudaMalloc made by a library either is
+ * forbidden, fails against the budget, or stalls the device while it runs.
+ * Such a host cannot use tgnn_create (it allocates the workspace), so this is
+ * step (3), the per-node latest-event reduction, with the same semantics as
+ * tgnn_reduce_latest but no context: its per-node scratch tables live in an
+ * array compiled into the library (20 bytes per node, TGNN_STATIC_MAX_NODES
+ * nodes = 1.25 MiB, held by every GPU that loads the library until the process
+ * exits).  Nothing is allocated or freed, by the library or on its behalf.
+ *   msg_node:int32[n_msg], t:f64[n_msg/2], eid:int32[n_msg/2] (message j belongs
+ *   to event j>>1 with role j&1; msg_node < 0 = dropped) -> uniq_out, winner_out:
+ *   int32[<= min(n_msg, num_nodes)], n_uniq_out:int32[1]; all device pointers
+ *   borrowed for the call; stream is a cudaStream_t.
+ * num_nodes above TGNN_STATIC_MAX_NODES is refused with TGNN_ECAPACITY.  On any
+ * failure a message is written to err_host (host buffer of err_size bytes, may
+ * be NULL).
+ * The first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress, with that device current) and keeps it; make that first
+ * call before any stream capture begins.
+ * All calls share the one array and it keeps what the last call left, so the
+ * kernel clears the entries it uses before it starts; two calls that overlap
+ * on the same GPU (different streams, or two threads) race on it and give
+ * wrong results -- serialise them. */
+#define TGNN_STATIC_MAX_NODES 65536
+TGNN_API int tgnn_reduce_latest_static(const int32_t* msg_node, const double* t, const int32_t* eid, int n_msg,
+                                       int64_t num_nodes, int32_t* uniq_out, int32_t* winner_out, int32_t* n_uniq_out,
+                                       void* stream, char* err_host, int err_size);
+
 /* Per-kernel timing for benchmarks (no counterpart in the paper beyond its
  * per-phase time breakdown, Table 5).  After tgnn_profile_begin every kernel
  * launch is bracketed by a CUDA event pair on the caller's stream until

@@ -26,7 +26,8 @@ EXPORTS = ("tgnn_create", "tgnn_destroy", "tgnn_last_error", "tgnn_param_count",
            "tgnn_set_graph", "tgnn_set_edge_features", "tgnn_set_state", "tgnn_prune_mask", "tgnn_sample_recent",
            "tgnn_build_messages", "tgnn_reduce_latest", "tgnn_memory_update", "tgnn_embed", "tgnn_backward_step",
            "tgnn_train_step", "tgnn_train_step_host", "tgnn_debug_get_grads", "tgnn_status", "tgnn_kernel_launches", "tgnn_profile_begin",
-           "tgnn_profile_report")
+           "tgnn_profile_report", "tgnn_reduce_latest_static")
+TGNN_STATIC_MAX_NODES = 65536
 
 
 class TgnnConfig(C.Structure):
@@ -79,6 +80,7 @@ def load_library():
         lib.tgnn_kernel_launches.restype = i64
         lib.tgnn_profile_begin.argtypes = [vp]
         lib.tgnn_profile_report.argtypes = [vp, vp, i64]
+        lib.tgnn_reduce_latest_static.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, vp, vp, i32]
         _lib = lib
     return _lib
 
@@ -130,6 +132,21 @@ def pack_params(cfg: TgnnConfig, weights: Dict[str, np.ndarray]) -> np.ndarray:
         w = np.asarray(weights[n], dtype=np.float32).ravel()
         flat[lay[n]:lay[n] + w.size] = w
     return flat
+
+
+def reduce_latest_static(msg_node, t, eid, num_nodes, uniq_out, winner_out, n_uniq_out) -> int:
+    """tgnn_reduce_latest_static: step (3) for hosts that may not allocate device memory, so no
+    context is involved -- the scratch tables are an array inside the library (at most
+    TGNN_STATIC_MAX_NODES nodes).  Raises TgnnError with the library's message on failure.
+    Calls share that array: do not let two of them overlap on one GPU."""
+    err = C.create_string_buffer(512)
+    rc = load_library().tgnn_reduce_latest_static(
+        _dp(msg_node, "i32", "msg_node"), _dp(t, "f64", "t"), _dp(eid, "i32", "eid"), msg_node.numel(), num_nodes,
+        _dp(uniq_out, "i32", "uniq_out"), _dp(winner_out, "i32", "winner_out"), _dp(n_uniq_out, "i32", "n_uniq_out"),
+        _stream(), C.addressof(err), len(err))
+    if rc != TGNN_OK:
+        raise TgnnError(rc, err.value.decode())
+    return rc
 
 
 class Tgnn:
