@@ -63,8 +63,12 @@ enum { TGNN_F32 = 0, TGNN_BF16 = 1 };
 /* math_mode: how the dense projections are computed.  Gates, softmax, loss, the
  * time encoding and Adam are always fp32. */
 enum {
-  TGNN_MATH_FP32 = 0, /* fp32 FMA tiles */
-  TGNN_MATH_TF32 = 1  /* tcgen05 tensor cores, TF32 operands, fp32 accumulation in TMEM */
+  TGNN_MATH_FP32 = 0,     /* fp32 FMA tiles */
+  TGNN_MATH_TF32 = 1,     /* tcgen05 tensor cores: every operand is split into a TF32 head and a TF32
+                             tail (3 MMAs per product, fp32 accumulation in TMEM), close to fp32 accuracy */
+  TGNN_MATH_TF32_FAST = 2 /* tcgen05 tensor cores, single TF32 pass in the forward projections (the gradient
+                             products keep the split).  Outputs stay within 2e-3, but gradient tensors whose
+                             terms cancel (time encoder, W_k) can be off by ~1e-2 of their largest entry. */
 };
 
 #if defined(__GNUC__)
@@ -77,7 +81,7 @@ typedef struct tgnn_ctx tgnn_ctx;
 
 typedef struct {
   int64_t num_nodes;
-  int32_t d;          /* memory / time / embedding dimension, multiple of 4 and of heads */
+  int32_t d;          /* memory / time / embedding dimension, <= 256, multiple of 4 and of heads */
   int32_t d_e;        /* edge-feature dimension, >= 0, even */
   int32_t k;          /* neighbors per root, 1..32 */
   int32_t heads;      /* attention heads */
@@ -223,6 +227,23 @@ TGNN_API int tgnn_train_step_host(tgnn_ctx* ctx, const int32_t* u_src_host, cons
 
 /* Copies the parameter gradient of the last tgnn_backward_step to grads_out:f32[param_count]. */
 TGNN_API int tgnn_debug_get_grads(tgnn_ctx* ctx, float* grads_out, void* stream);
+/* The ReLU branch each unit took in the last tgnn_embed / tgnn_backward_step pair, as bytes:
+ * h_gate_out:uint8[n_roots, d] (1 where h > 0), hid_gate_out:uint8[2 n_q, d] (hidden layer of the
+ * link-prediction head, positive pairs first).  A parity check needs them because the derivative
+ * of ReLU jumps at zero: a pre-activation closer to zero than the arithmetic resolves may fall on
+ * either side, and the reference must differentiate the branch the kernel took. */
+TGNN_API int tgnn_debug_get_gates(tgnn_ctx* ctx, uint8_t* h_gate_out, uint8_t* hid_gate_out, void* stream);
+/* The dense-projection kernel on its own (the one the configured math_mode selects), for
+ * parity tests: C[M,N] (+)= sum_k A(m,k) B(k,n) (+ bias[n]) (ReLU), with element strides
+ * A(m,k) = A[m*a_rs + k*a_cs], B(k,n) = B[k*b_rs + n*b_cs], C row-major with leading
+ * dimension ldc.  dev_M / dev_K (device int32, may be NULL) cap M / K at run time; bias [N]
+ * and rowsum_out [M] (+= sum_k A(m,k), the bias gradient of a transposed product) may be
+ * NULL; accumulate != 0 adds into C atomically and is required when split_k > 1; precise != 0
+ * selects the 3xTF32 head/tail split in the tensor-core mode (ignored in the fp32 mode). */
+TGNN_API int tgnn_debug_gemm(tgnn_ctx* ctx, const float* A, int64_t a_rs, int64_t a_cs, const float* B, int64_t b_rs,
+                             int64_t b_cs, float* C, int64_t ldc, int M, int N, int K, const int32_t* dev_M,
+                             const int32_t* dev_K, const float* bias, float* rowsum_out, int relu, int accumulate,
+                             int split_k, int precise, void* stream);
 /* Device status word (0 or the first TGNN_ETIMEOUT / TGNN_EBOUNDS recorded by a
  * kernel) copied to *status_host.  Synchronises the stream. */
 TGNN_API int tgnn_status(tgnn_ctx* ctx, int32_t* status_host, void* stream);

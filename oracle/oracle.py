@@ -201,8 +201,11 @@ class StepResult:
     winner: np.ndarray
 
 
-def loss_and_grads(cfg, params, memory, last_update, efeat, upd, roots, n_q, loss_mask, want_grads=True) -> StepResult:
-    """upd = (src, dst, t, eid, keep|None) of the update events; roots = (nodes, times, nbr, eid, ts, cnt)."""
+def loss_and_grads(cfg, params, memory, last_update, efeat, upd, roots, n_q, loss_mask, want_grads=True,
+                   h_gate=None, hid_gate=None, gate_eps=0.0) -> StepResult:
+    """upd = (src, dst, t, eid, keep|None) of the update events; roots = (nodes, times, nbr, eid, ts, cnt).
+    h_gate / hid_gate: ReLU branch decisions of a lower-precision run, used only for units whose
+    pre-activation lies within gate_eps * max|pre-activation| of zero (either branch is valid there)."""
     u_src, u_dst, u_t, u_eid = _i32(upd[0]), _i32(upd[1]), _f64(upd[2]), _i32(upd[3])
     u_keep = _u8(upd[4]) if upd[4] is not None else None
     n_u = len(u_src)
@@ -224,7 +227,9 @@ def loss_and_grads(cfg, params, memory, last_update, efeat, upd, roots, n_q, los
     lib().orc_loss_and_grads(C.byref(cfg), _p(_f64(params)), _p(_f64(memory)), _p(_f64(last_update)),
                              _p(_feat(cfg, efeat)), _p(u_src), _p(u_dst), _p(u_t), _p(u_eid), _p(u_keep), C.c_int(n_u),
                              _p(r_node), _p(r_time), C.c_int(n_r), _p(nb_node), _p(nb_eid), _p(nb_ts), _p(nb_cnt),
-                             C.c_int(n_q), _p(lm), C.c_int(int(want_grads)), _p(loss), _p(grads), _p(gn),
+                             C.c_int(n_q), _p(lm), _p(_u8(h_gate) if h_gate is not None else None),
+                             _p(_u8(hid_gate) if hid_gate is not None else None), C.c_double(gate_eps),
+                             C.c_int(int(want_grads)), _p(loss), _p(grads), _p(gn),
                              _p(mem_post), _p(lu_post), _p(h), _p(uniq), _p(win), _p(nu))
     return StepResult(float(loss[0]), float(gn[0]), grads, mem_post, lu_post, h, uniq[:nu[0]].copy(), win[:nu[0]].copy())
 

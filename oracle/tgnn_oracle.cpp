@@ -136,6 +136,13 @@ struct Inputs {
   const int32_t* nb_cnt;            // [n_r]
   int n_q;
   const uint8_t* loss_mask;  // [n_q]
+  // ReLU gate decisions taken elsewhere in lower precision (optional).  A pre-activation within
+  // gate_eps * max|pre-activation| of zero is closer to zero than that precision resolves, so either
+  // side of the kink is a valid outcome there; for those units (only) the given decision is used, so
+  // that both sides differentiate the same branch.  Everywhere else the fp64 sign decides.
+  const uint8_t* h_gate;    // [n_r, d]    for h = ReLU(W_o [a || m] + b_o)
+  const uint8_t* hid_gate;  // [2 n_q, d]  for the head's hidden layer
+  double gate_eps;
 };
 
 struct Tape {
@@ -154,6 +161,7 @@ struct Tape {
   vec z_dt;  // [n_r, k]
   // loss
   vec cat1, pre1, hid1, score;  // 2*n_q pairs: pair p<n_q positive, p>=n_q negative
+  std::vector<uint8_t> h_on, hid_on;  // ReLU branch taken per unit
   double loss;
   double mask_sum;
 };
@@ -333,8 +341,17 @@ void embed(const Inputs& in, const Layout& L, const double* P, const double* mem
       double a = P[L.bo + o];
       for (int64_t q = 0; q < 2 * d; ++q) a += P[L.wo + o * 2 * d + q] * cat[q];
       T.pre_o[(size_t)i * d + o] = a;
-      T.h[(size_t)i * d + o] = a > 0 ? a : 0;
     }
+  }
+  double pre_scale = 0;
+  for (double v : T.pre_o) pre_scale = std::max(pre_scale, std::fabs(v));
+  T.h_on.assign((size_t)R * d, 0);
+  for (size_t e = 0; e < (size_t)R * d; ++e) {
+    const double a = T.pre_o[e];
+    bool on = a > 0;
+    if (in.h_gate && std::fabs(a) <= in.gate_eps * pre_scale) on = in.h_gate[e] != 0;
+    T.h_on[e] = on;
+    T.h[e] = on ? a : 0;
   }
 }
 
@@ -346,19 +363,33 @@ void loss_forward(const Inputs& in, const Layout& L, const double* P, Tape& T) {
   const int nq = in.n_q;
   T.cat1.assign((size_t)2 * nq * 2 * d, 0); T.pre1.assign((size_t)2 * nq * d, 0);
   T.hid1.assign((size_t)2 * nq * d, 0); T.score.assign((size_t)2 * nq, 0);
-  double num = 0, den = 0;
+  T.hid_on.assign((size_t)2 * nq * d, 0);
   for (int j = 0; j < nq; ++j) {
     for (int pn = 0; pn < 2; ++pn) {
       const size_t p = (size_t)pn * nq + j;
       const size_t a = j, b = (size_t)(pn == 0 ? nq : 2 * nq) + j;
       double* cat = &T.cat1[p * 2 * d];
       for (int64_t q = 0; q < d; ++q) { cat[q] = T.h[a * d + q]; cat[d + q] = T.h[b * d + q]; }
-      double s = P[L.b2];
       for (int64_t o = 0; o < d; ++o) {
         double acc = P[L.b1 + o];
         for (int64_t q = 0; q < 2 * d; ++q) acc += P[L.w1 + o * 2 * d + q] * cat[q];
         T.pre1[p * d + o] = acc;
-        const double hd = acc > 0 ? acc : 0;
+      }
+    }
+  }
+  double scale = 0;
+  for (double v : T.pre1) scale = std::max(scale, std::fabs(v));
+  double num = 0, den = 0;
+  for (int j = 0; j < nq; ++j) {
+    for (int pn = 0; pn < 2; ++pn) {
+      const size_t p = (size_t)pn * nq + j;
+      double s = P[L.b2];
+      for (int64_t o = 0; o < d; ++o) {
+        const double acc = T.pre1[p * d + o];
+        bool on = acc > 0;
+        if (in.hid_gate && std::fabs(acc) <= in.gate_eps * scale) on = in.hid_gate[p * d + o] != 0;
+        T.hid_on[p * d + o] = on;
+        const double hd = on ? acc : 0;
         T.hid1[p * d + o] = hd;
         s += P[L.w2 + o] * hd;
       }
@@ -403,7 +434,7 @@ void backward_all(const Inputs& in, const Layout& L, const double* P, const Tape
       vec dcat((size_t)2 * d, 0.0);
       for (int64_t o = 0; o < d; ++o) {
         G[L.w2 + o] += ds * T.hid1[p * d + o];
-        const double dpre = T.pre1[p * d + o] > 0 ? ds * P[L.w2 + o] : 0.0;
+        const double dpre = T.hid_on[p * d + o] ? ds * P[L.w2 + o] : 0.0;
         G[L.b1 + o] += dpre;
         for (int64_t q = 0; q < 2 * d; ++q) {
           G[L.w1 + o * 2 * d + q] += dpre * T.cat1[p * 2 * d + q];
@@ -421,7 +452,7 @@ void backward_all(const Inputs& in, const Layout& L, const double* P, const Tape
     const int cnt = in.nb_cnt[i];
     vec dcat((size_t)2 * d, 0.0);
     for (int64_t o = 0; o < d; ++o) {
-      const double dpre = T.pre_o[(size_t)i * d + o] > 0 ? dh_[(size_t)i * d + o] : 0.0;
+      const double dpre = T.h_on[(size_t)i * d + o] ? dh_[(size_t)i * d + o] : 0.0;
       G[L.bo + o] += dpre;
       for (int64_t q = 0; q < 2 * d; ++q) {
         G[L.wo + o * 2 * d + q] += dpre * T.cat_o[(size_t)i * 2 * d + q];
@@ -548,6 +579,7 @@ Inputs make_inputs(const orc_config* c, const void* efeat, const int32_t* u_src,
   in.r_node = r_node; in.r_time = r_time; in.n_r = n_r;
   in.nb_node = nb_node; in.nb_eid = nb_eid; in.nb_ts = nb_ts; in.nb_cnt = nb_cnt;
   in.n_q = n_q; in.loss_mask = loss_mask;
+  in.h_gate = nullptr; in.hid_gate = nullptr; in.gate_eps = 0.0;
   return in;
 }
 
@@ -687,19 +719,21 @@ void orc_embed(const orc_config* c, const double* params, const double* memory, 
 }
 
 // Steps (2)-(6) forward plus the exact gradient, from the pre-step state.
-// Outputs (any may be null): loss, grads[P], gradnorm = sqrt(sum grads^2),
+// h_gate / hid_gate / gate_eps (optional): see Inputs.  Outputs (any may be null): loss, grads[P], gradnorm = sqrt(sum grads^2),
 // memory_post[N,d], last_update_post[N], h[n_r,d], uniq/winner/n_uniq.
 void orc_loss_and_grads(const orc_config* c, const double* params, const double* memory, const double* last_update,
                         const void* efeat, const int32_t* u_src, const int32_t* u_dst, const double* u_t,
                         const int32_t* u_eid, const uint8_t* u_keep, int n_u, const int32_t* r_node,
                         const double* r_time, int n_r, const int32_t* nb_node, const int32_t* nb_eid,
-                        const double* nb_ts, const int32_t* nb_cnt, int n_q, const uint8_t* loss_mask, int want_grads,
+                        const double* nb_ts, const int32_t* nb_cnt, int n_q, const uint8_t* loss_mask,
+                        const uint8_t* h_gate, const uint8_t* hid_gate, double gate_eps, int want_grads,
                         double* loss_out, double* grads_out, double* gradnorm_out, double* memory_post,
                         double* last_update_post, double* h_out, int32_t* uniq_out, int32_t* winner_out,
                         int32_t* n_uniq_out) {
   Layout L(*c);
   Inputs in = make_inputs(c, efeat, u_src, u_dst, u_t, u_eid, u_keep, n_u, r_node, r_time, n_r, nb_node, nb_eid, nb_ts,
                           nb_cnt, n_q, loss_mask);
+  in.h_gate = h_gate; in.hid_gate = hid_gate; in.gate_eps = gate_eps;
   Tape T;
   forward_all(in, L, params, memory, last_update, T);
   if (loss_out) *loss_out = T.loss;

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libtgnn_b200.so")
 TGNN_OK, TGNN_EINVAL, TGNN_ESHAPE, TGNN_ECAPACITY, TGNN_ESTATE, TGNN_ECUDA, TGNN_ETIMEOUT, TGNN_EBOUNDS = (
     0, -1, -2, -3, -4, -5, -6, -7)
 TGNN_F32, TGNN_BF16 = 0, 1
-TGNN_MATH_FP32, TGNN_MATH_TF32 = 0, 1
+TGNN_MATH_FP32, TGNN_MATH_TF32, TGNN_MATH_TF32_FAST = 0, 1, 2
 
 PARAM_NAMES = ("time_w", "time_b", "gru_w_i", "gru_w_h", "gru_b_i", "gru_b_h", "w_q", "b_q", "w_k", "w_v",
                "b_k", "b_v", "w_o", "b_o", "w_1", "b_1", "w_2", "b_2")
@@ -26,7 +26,7 @@ EXPORTS = ("tgnn_create", "tgnn_destroy", "tgnn_last_error", "tgnn_param_count",
            "tgnn_set_graph", "tgnn_set_edge_features", "tgnn_set_state", "tgnn_prune_mask", "tgnn_sample_recent",
            "tgnn_build_messages", "tgnn_reduce_latest", "tgnn_memory_update", "tgnn_embed", "tgnn_backward_step",
            "tgnn_train_step", "tgnn_train_step_host", "tgnn_debug_get_grads", "tgnn_status", "tgnn_kernel_launches", "tgnn_profile_begin",
-           "tgnn_profile_report", "tgnn_reduce_latest_static")
+           "tgnn_profile_report", "tgnn_reduce_latest_static", "tgnn_debug_gemm", "tgnn_debug_get_gates")
 TGNN_STATIC_MAX_NODES = 65536
 
 
@@ -80,6 +80,9 @@ def load_library():
         lib.tgnn_kernel_launches.restype = i64
         lib.tgnn_profile_begin.argtypes = [vp]
         lib.tgnn_profile_report.argtypes = [vp, vp, i64]
+        lib.tgnn_debug_gemm.argtypes = [vp, vp, i64, i64, vp, i64, i64, vp, i64, i32, i32, i32, vp, vp, vp, vp, i32, i32, i32, i32,
+                                        vp]
+        lib.tgnn_debug_get_gates.argtypes = [vp, vp, vp, vp]
         lib.tgnn_reduce_latest_static.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, vp, vp, i32]
         _lib = lib
     return _lib
@@ -271,6 +274,18 @@ class Tgnn:
     # ---- debug ----
     def debug_get_grads(self, grads_out):
         self._ck(self.lib.tgnn_debug_get_grads(self._h, _dp(grads_out, "f32", "grads_out"), _stream()))
+
+    def debug_gemm(self, A, a_rs, a_cs, Bm, b_rs, b_cs, Cm, ldc, M, N, K, dev_M=None, dev_K=None, bias=None,
+                   rowsum_out=None, relu=False, accumulate=False, split_k=1, precise=False):
+        self._ck(self.lib.tgnn_debug_gemm(self._h, _dp(A, "f32", "A"), a_rs, a_cs, _dp(Bm, "f32", "B"), b_rs, b_cs,
+                                          _dp(Cm, "f32", "C"), ldc, M, N, K, _dp(dev_M, "i32", "dev_M"),
+                                          _dp(dev_K, "i32", "dev_K"), _dp(bias, "f32", "bias"),
+                                          _dp(rowsum_out, "f32", "rowsum_out"), int(relu), int(accumulate), split_k,
+                                          int(precise), _stream()))
+
+    def debug_get_gates(self, h_gate_out, hid_gate_out):
+        self._ck(self.lib.tgnn_debug_get_gates(self._h, _dp(h_gate_out, "u8", "h_gate_out"),
+                                               _dp(hid_gate_out, "u8", "hid_gate_out"), _stream()))
 
     def profile_begin(self):
         self._ck(self.lib.tgnn_profile_begin(self._h))

@@ -26,7 +26,7 @@ __global__ void __launch_bounds__(256) head_loss_kernel(float* __restrict__ hid1
                                                         const float* __restrict__ b2,
                                                         const uint8_t* __restrict__ loss_mask, int nq, int d,
                                                         float* __restrict__ g_w2, float* __restrict__ g_b2,
-                                                        float* __restrict__ loss_acc) {
+                                                        float* __restrict__ loss_acc, uint8_t* __restrict__ hid_gate) {
   extern __shared__ float s_gw2[];  // [d]
   __shared__ float s_msum;
   __shared__ float s_gb2, s_loss;
@@ -70,6 +70,8 @@ __global__ void __launch_bounds__(256) head_loss_kernel(float* __restrict__ hid1
       if (wj != 0.f) atomicAdd(&s_gw2[q], dsp * a + dsn * b);
       hp[q] = a > 0.f ? dsp * w2[q] : 0.f;
       hn[q] = b > 0.f ? dsn * w2[q] : 0.f;
+      hid_gate[(int64_t)j * d + q] = a > 0.f;
+      hid_gate[(int64_t)(nq + j) * d + q] = b > 0.f;
     }
   }
   __syncthreads();
@@ -178,32 +180,55 @@ __global__ void __launch_bounds__(256) scatter_dmem_kernel(const float* __restri
   }
 }
 
-// Time-encoder gradient from a block of rows: G[r, col0 + c] is d loss / d Phi(dt_r)_c.
-//   dw_c += -sin(arg) dt_r G,  db_c += -sin(arg) G,  arg = fmaf(w_c, dt_r, b_c)
-// The terms are large (dt reaches the time span of the stream) and cancel, so they are summed
-// in fp64: thread c walks the rows of the block's chunk, one pair of fp64 atomics per block
-// and column into acc[0:d] (dw) and acc[d:2d] (db).
-__global__ void __launch_bounds__(128) time_grad_kernel(const float* __restrict__ G, int64_t ldg, int col0,
-                                                        const float* __restrict__ dt, int rows,
-                                                        const int32_t* __restrict__ dev_rows, int rows_per_block, int d,
-                                                        const float* __restrict__ time_w, const float* __restrict__ time_b,
-                                                        double* __restrict__ acc) {
+// Time-encoder gradient: G[r, col0 + c] is d loss / d Phi(dt_r)_c and S[r, c] = sin(arg) was kept by
+// the forward pass (S == nullptr: every row has dt = 0, sin(arg) = sin(b_c)).
+//   dw_c += -S dt_r G,   db_c += -S G
+// The terms are large (dt reaches the time span of the stream) and cancel, so they are summed in
+// fp64.  Block = 8 warps over 64 rows; lanes own columns c = lane + 32 j; the warps' partial sums
+// meet in shared memory and leave as one pair of fp64 atomics per block and column into acc[0:d]
+// (dw) and acc[d:2d] (db).  Dynamic shared memory: 8 * 2 * d doubles.
+constexpr int TG_ROWS = 64, TG_MAXJ = 8;
+__global__ void __launch_bounds__(256) time_grad_kernel(const float* __restrict__ G, int64_t ldg, int col0,
+                                                        const float* __restrict__ S, const float* __restrict__ dt,
+                                                        int rows, const int32_t* __restrict__ dev_rows, int d,
+                                                        const float* __restrict__ time_b, double* __restrict__ acc) {
+  extern __shared__ double s_part[];  // [8][2][d]
   const int R = dev_rows ? min(*dev_rows, rows) : rows;
-  const int r0 = blockIdx.x * rows_per_block, r1 = min(R, r0 + rows_per_block);
+  const int r0 = blockIdx.x * TG_ROWS, r1 = min(R, r0 + TG_ROWS);
   if (r0 >= r1) return;
-  for (int c = threadIdx.x; c < d; c += blockDim.x) {
-    const float w = time_w[c], b = time_b[c];
-    double gw = 0.0, gb = 0.0;
-    for (int r = r0; r < r1; ++r) {
-      const float g = G[(int64_t)r * ldg + col0 + c];
-      if (g == 0.f) continue;
-      const float dtr = dt ? dt[r] : 0.f;
-      const double sn = -(double)sinf(time_arg(w, b, dtr)) * (double)g;
-      gw = fma(sn, (double)dtr, gw);
-      gb += sn;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  double gw[TG_MAXJ], gb[TG_MAXJ];
+  float sb[TG_MAXJ];
+#pragma unroll
+  for (int j = 0; j < TG_MAXJ; ++j) {
+    gw[j] = 0.0; gb[j] = 0.0;
+    const int c = lane + 32 * j;
+    sb[j] = (S == nullptr && c < d) ? sinf(time_b[c]) : 0.f;
+  }
+  for (int r = r0 + wid; r < r1; r += 8) {
+    const float dtr = dt ? dt[r] : 0.f;
+#pragma unroll
+    for (int j = 0; j < TG_MAXJ; ++j) {
+      const int c = lane + 32 * j;
+      if (c < d) {
+        const float g = G[(int64_t)r * ldg + col0 + c];
+        const float sn = S ? S[(int64_t)r * d + c] : sb[j];
+        const double t = -(double)sn * (double)g;
+        gw[j] = fma(t, (double)dtr, gw[j]);
+        gb[j] += t;
+      }
     }
-    if (gw != 0.0) atomicAdd(&acc[c], gw);
-    if (gb != 0.0) atomicAdd(&acc[d + c], gb);
+  }
+#pragma unroll
+  for (int j = 0; j < TG_MAXJ; ++j) {
+    const int c = lane + 32 * j;
+    if (c < d) { s_part[(wid * 2 + 0) * d + c] = gw[j]; s_part[(wid * 2 + 1) * d + c] = gb[j]; }
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < 2 * d; e += blockDim.x) {
+    double t = 0.0;
+    for (int w = 0; w < 8; ++w) t += s_part[w * 2 * d + e];
+    if (t != 0.0) atomicAdd(&acc[e], t);
   }
 }
 
@@ -294,6 +319,11 @@ __global__ void __launch_bounds__(256) adam_kernel(float* __restrict__ p, float*
   }
 }
 
+__global__ void gate_bytes_kernel(const float* __restrict__ h, int64_t n, uint8_t* __restrict__ out) {
+  const int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (e < n) out[e] = h[e] > 0.f;
+}
+
 int pick_split(int M, int N, int K) {
   const int tiles = ((M + 63) / 64) * ((N + 63) / 64);
   int s = (4 * 148 + tiles - 1) / tiles;
@@ -310,7 +340,7 @@ int grad_w(tgnn_ctx* ctx, const float* dY, int64_t ld_dy, const float* A, int64_
   g.A = dY; g.a_rs = 1; g.a_cs = ld_dy;  // A(m,k) = dY[k, m]
   g.B = A; g.b_rs = ld_a; g.b_cs = 1;    // B(k,n) = A[k, n]
   g.C = dW; g.ldc = k_in; g.M = n_out; g.N = k_in; g.K = rows; g.dev_K = dev_rows;
-  g.rowsum_out = db; g.accumulate = 1; g.split_k = pick_split(n_out, k_in, rows);
+  g.rowsum_out = db; g.accumulate = 1; g.split_k = pick_split(n_out, k_in, rows); g.precise = 1;
   return launch_gemm(ctx, g, name, s);
 }
 
@@ -320,11 +350,22 @@ int grad_in(tgnn_ctx* ctx, const float* dY, int64_t ld_dy, const float* W, int64
   GemmArgs g = {};
   g.A = dY; g.a_rs = ld_dy; g.a_cs = 1;
   g.B = W + col0; g.b_rs = ld_w; g.b_cs = 1;
-  g.C = dA; g.ldc = ld_da; g.M = rows; g.N = n_cols; g.K = n_out; g.dev_M = dev_rows; g.split_k = 1;
+  g.C = dA; g.ldc = ld_da; g.M = rows; g.N = n_cols; g.K = n_out; g.dev_M = dev_rows; g.split_k = 1; g.precise = 1;
   return launch_gemm(ctx, g, name, s);
 }
 
 }  // namespace
+
+int launch_get_gates(tgnn_ctx* ctx, uint8_t* h_gate_out, uint8_t* hid_gate_out, cudaStream_t s) {
+  const int64_t n = (int64_t)ctx->e_n * ctx->cfg.d;
+  if (n > 0) {
+    gate_bytes_kernel<<<(int)((n + 255) / 256), 256, 0, s>>>(ctx->e_h, n, h_gate_out);
+    TGNN_LAUNCH_OK(ctx, "gate_bytes");
+    const size_t m = (size_t)2 * (ctx->e_n / 3) * ctx->cfg.d;
+    TGNN_CUDA_OK(ctx, cudaMemcpyAsync(hid_gate_out, ctx->ws.hid_gate, m, cudaMemcpyDeviceToDevice, s));
+  }
+  return TGNN_OK;
+}
 
 #define RC(x)            \
   do {                   \
@@ -360,7 +401,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     {
       KernelScope scope__(ctx, "head_loss", s);
       head_loss_kernel<<<(n_q + 7) / 8, 256, d * sizeof(float), s>>>(w.hid1, P + L.w2, P + L.b2, loss_mask, n_q, d,
-                                                                     G + L.w2, G + L.b2, w.st_scalars);
+                                                                     G + L.w2, G + L.b2, w.st_scalars, w.hid_gate);
     }
     TGNN_LAUNCH_OK(ctx, "head_loss");
     // hid1 now holds d loss / d pre1
@@ -386,17 +427,17 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     RC(grad_w(ctx, w.dKV, 2 * d, w.Z, ctx->ld_kv, NB, nullptr, 2 * d, (int)L.dkv, G + L.wk, G + L.bk, "dW_kv", s));
     RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, d + de, NB, nullptr, 2 * d, d, w.dZp, d, "dZ_phi", s));
     // time-encoder gradient through the attention inputs
-    const int rpb = 64;
+    const size_t tg_smem = (size_t)8 * 2 * d * sizeof(double);
     {
       KernelScope scope__(ctx, "time_grad_z", s);
-      time_grad_kernel<<<(NB + rpb - 1) / rpb, 128, 0, s>>>(w.dZp, d, 0, w.z_dt, NB, nullptr, rpb, d, P + L.time_w,
-                                                            P + L.time_b, w.tg_acc);
+      time_grad_kernel<<<(NB + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, s>>>(w.dZp, d, 0, w.Zsin, w.z_dt, NB, nullptr, d,
+                                                                          P + L.time_b, w.tg_acc);
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_z");
     {
       KernelScope scope__(ctx, "time_grad_q", s);
-      time_grad_kernel<<<(R + rpb - 1) / rpb, 128, 0, s>>>(w.dzq, 2 * d, d, nullptr, R, nullptr, rpb, d, P + L.time_w,
-                                                           P + L.time_b, w.tg_acc);
+      time_grad_kernel<<<(R + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, s>>>(w.dzq, 2 * d, d, nullptr, nullptr, R, nullptr, d,
+                                                                         P + L.time_b, w.tg_acc);
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_q");
     if (ctx->have_update) {
@@ -423,8 +464,8 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
                  "dX_phi", s));
       {
         KernelScope scope__(ctx, "time_grad_x", s);
-        time_grad_kernel<<<(U_cap + rpb - 1) / rpb, 128, 0, s>>>(w.dXp, d, 0, w.x_dt, U_cap, ctx->upd_n_uniq, rpb, d,
-                                                                 P + L.time_w, P + L.time_b, w.tg_acc);
+        time_grad_kernel<<<(U_cap + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, s>>>(w.dXp, d, 0, w.Xsin, w.x_dt, U_cap,
+                                                                             ctx->upd_n_uniq, d, P + L.time_b, w.tg_acc);
       }
       TGNN_LAUNCH_OK(ctx, "time_grad_x");
     }

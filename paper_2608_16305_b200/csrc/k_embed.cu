@@ -16,6 +16,7 @@ __global__ void __launch_bounds__(256) gather_z_kernel(const float* __restrict__
                                                        int n, const int32_t* __restrict__ nbr,
                                                        const int32_t* __restrict__ eid, const double* __restrict__ ts,
                                                        int ld, float* __restrict__ Z, float* __restrict__ z_dt,
+                                                       float* __restrict__ Zsin,
                                                        float* __restrict__ Zq, float* __restrict__ cat_o) {
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
@@ -27,6 +28,7 @@ __global__ void __launch_bounds__(256) gather_z_kernel(const float* __restrict__
       const int nb = nbr[r];
       if (nb < 0) {
         for (int q = lane; q < ld; q += 32) row[q] = 0.f;
+        for (int q = lane; q < d; q += 32) Zsin[(int64_t)r * d + q] = 0.f;
         if (lane == 0) z_dt[r] = 0.f;
         continue;
       }
@@ -34,7 +36,7 @@ __global__ void __launch_bounds__(256) gather_z_kernel(const float* __restrict__
       warp_copy_f32(row, memory + (int64_t)nb * d, d, lane);
       warp_copy_feat(row + d, efeat, feat_bf16, eid[r], de, lane);
       float* phi = row + d + de;
-      for (int q = lane; q < d; q += 32) phi[q] = time_encode(time_w[q], time_b[q], dtf);
+      for (int q = lane; q < d; q += 32) time_encode_sc(time_w[q], time_b[q], dtf, &phi[q], &Zsin[(int64_t)r * d + q]);
       for (int q = dkv + lane; q < ld; q += 32) row[q] = 0.f;
       if (lane == 0) z_dt[r] = dtf;
     } else {
@@ -103,7 +105,7 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
     KernelScope scope__(ctx, "gather_z", s);
     gather_z_kernel<<<(rows + 7) / 8, 256, 0, s>>>(ctx->memory, ctx->efeat, c.feat_dtype == TGNN_BF16,
                                                    ctx->params + L.time_w, ctx->params + L.time_b, d, c.d_e, k, nodes,
-                                                   times, n, nbr, eid, ts, ctx->ld_kv, w.Z, w.z_dt, w.Zq, w.cat_o);
+                                                   times, n, nbr, eid, ts, ctx->ld_kv, w.Z, w.z_dt, w.Zsin, w.Zq, w.cat_o);
   }
   TGNN_LAUNCH_OK(ctx, "gather_z");
   GemmArgs g = {};

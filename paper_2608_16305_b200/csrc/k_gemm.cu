@@ -89,6 +89,12 @@ __global__ void __launch_bounds__(NT) gemm_fp32_kernel(GemmArgs g) {
 int launch_gemm(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s) {
   if (g.M <= 0 || g.N <= 0) return TGNN_OK;
   if (g.split_k > 1 && !g.accumulate) return set_error(ctx, TGNN_EINVAL, "gemm %s: split_k needs accumulate", name);
+  if (ctx->cfg.math_mode != TGNN_MATH_FP32) {
+    GemmArgs gp = g;
+    if (ctx->cfg.math_mode == TGNN_MATH_TF32) gp.precise = 1;
+    const int rc = launch_gemm_tf32(ctx, gp, name, s);
+    if (rc != 1) return rc;  // 1: shape not handled by the tensor-core kernel, use the FMA tiles
+  }
   dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.split_k < 1 ? 1 : g.split_k);
   GemmArgs a = g;
   if (a.split_k < 1) a.split_k = 1;

@@ -1,0 +1,483 @@
+// Dense projections on the 5th-generation tensor cores (TGNN_MATH_TF32).
+//
+// One CTA computes a 128 x BN tile of C = A B over a range of the contraction
+// (split-K across blockIdx.z) with tcgen05.mma.kind::tf32: fp32 operands rounded to
+// TF32 (round-to-nearest, by the producer warps, so there is no truncation bias),
+// fp32 accumulation in tensor memory.  With `precise` set every operand is split into
+// a TF32 head and a TF32 tail (x = hi + lo) and three MMAs (lo*hi, hi*lo, hi*hi) give
+// close to fp32 accuracy; the gradient products, whose terms cancel, use it.
+//
+// Warp roles:
+//   G producer groups of 4 warps.  Group g fills the stages of contraction blocks
+//     i = g, g + G, ...: global -> registers (all 128-bit loads of a block issued before
+//     the first use) -> round to TF32 -> shared memory in the swizzled canonical layout
+//     the MMA descriptors expect.  Several blocks are therefore in flight at once.
+//     Afterwards all groups run the epilogue (tcgen05.ld of the 32 TMEM lanes their warp
+//     may touch, bias / ReLU / store or atomic accumulate), sharing the columns.
+//   1 MMA warp: allocates tensor memory; one lane issues the MMAs and commits.
+// A ring of (A tile, B tile) stages is handed over through mbarriers: full[s] (128
+// producer arrivals) and empty[s] (tcgen05.commit).  Every wait is bounded; on expiry
+// the kernel records TGNN_ETIMEOUT in the status word, stops waiting, frees its tensor
+// memory and returns.
+//
+// Operands may be K-major (contraction index contiguous) or MN-major (row/column index
+// contiguous), so the forward projections (activations [M,K] x weights [N,K]), the
+// input gradients (dY [M,N'] x W [N',K]) and the weight gradients (dY^T x A, contraction
+// over rows) all run here without a transposed copy.
+#include "tgnn_internal.cuh"
+
+namespace tgnn {
+namespace {
+
+constexpr int BM = 128;    // rows of C per CTA (UMMA M)
+constexpr int BK = 32;     // contraction elements per stage: one 128-byte swizzle row of fp32
+constexpr int UMMA_K = 8;  // tf32
+constexpr int GROUP = 128; // threads per producer group
+constexpr unsigned SPIN_LIMIT = 1u << 24;
+constexpr unsigned FULL = 0xffffffffu;
+
+enum { MAJOR_K = 0, MAJOR_MN = 1 };
+
+struct TcArgs {
+  const float* A; int64_t lda; int a_major;
+  const float* B; int64_t ldb; int b_major;
+  float* C; int64_t ldc;
+  int M, N, K;
+  const int32_t* dev_M;
+  const int32_t* dev_K;
+  const float* bias;
+  float* rowsum_out;
+  int relu, accumulate, split_k;
+  int32_t* status;
+};
+
+template <int BN_T, bool PRECISE>
+struct Cfg {
+  static constexpr int STAGES = PRECISE ? (BN_T > 128 ? 2 : 3) : 4;
+  static constexpr int GROUPS = STAGES < 3 ? STAGES : 3;
+  static constexpr int THREADS = GROUPS * GROUP + 32;
+  static constexpr int A_BYTES = BM * 128, B_BYTES = BN_T * 128;
+  static constexpr int COPIES = PRECISE ? 2 : 1;  // head (+ tail) copy of each operand tile
+  static constexpr int STAGE_BYTES = COPIES * (A_BYTES + B_BYTES);
+  static constexpr int SMEM = 1024 + STAGES * STAGE_BYTES;
+  static constexpr uint32_t TMEM_COLS = BN_T <= 128 ? 128 : 256;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Bounded wait on a phase parity.  Returns false if the limit was reached.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (unsigned it = 0; it < SPIN_LIMIT; ++it) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+
+// Loads and stores are volatile asm so that the compiler keeps every load of a block ahead of
+// the first store (it otherwise sinks each load next to its use and serialises the round trips).
+__device__ __forceinline__ float4 ldg_v4(const float* p) {
+  float4 v;
+  asm volatile("ld.global.nc.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ float ldg_f(const float* p) {
+  float v;
+  asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void sts_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+// Round-to-nearest (ties away from zero) to the 10 mantissa bits of TF32: add half an ulp to the
+// magnitude and clear the 13 low bits.  Same result as cvt.rna.tf32.f32 for finite inputs, but on
+// the integer pipe at full rate (the conversion pipe would bound the producers).
+__device__ __forceinline__ uint32_t to_tf32(float x) { return (__float_as_uint(x) + 0x1000u) & 0xffffe000u; }
+
+template <bool PRECISE>
+__device__ __forceinline__ void store_chunk(uint32_t addr, uint32_t tail_offset, const float4& v) {
+  const uint32_t h0 = to_tf32(v.x), h1 = to_tf32(v.y), h2 = to_tf32(v.z), h3 = to_tf32(v.w);
+  sts_v4(addr, h0, h1, h2, h3);
+  if (PRECISE) {
+    sts_v4(addr + tail_offset, to_tf32(v.x - __uint_as_float(h0)), to_tf32(v.y - __uint_as_float(h1)),
+           to_tf32(v.z - __uint_as_float(h2)), to_tf32(v.w - __uint_as_float(h3)));
+  }
+}
+
+// 64-bit shared-memory matrix descriptor.  layout: 2 = 128-byte swizzle on 16-byte chunks (K-major
+// operands), 1 = 128-byte swizzle with a 32-byte base (the only layout for MN-major 32-bit operands).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;  // descriptor version for this architecture
+  d |= (uint64_t)layout << 61;
+  return d;
+}
+
+// One producer group (128 threads, index t) fills one operand tile for contraction block [k0, k0+32).
+//   K-major:  rows [r0, r0 + rows_t) x 32 k; row r lives at (r/8)*1024 + (r%8)*128, its 16-byte
+//             chunk c at position c ^ (r%8).
+//   MN-major: 32 k-rows x rows_t (MN) values in atoms of 4 k-rows x 32 values (512 B); k-row kk, MN
+//             atom a, chunk c lives at (kk/4)*(atoms*512) + a*512 + (kk%4)*128 + ((c ^ 2*(kk%4))*16):
+//             the swizzle exchanges 32-byte pairs of chunks (address bits 5-6 ^= bits 7-8).
+// rows_t is a multiple of 32 (MN-major) or of 8 (K-major); chunks outside the valid range are zero.
+template <int ROWS_MAX, bool PRECISE>
+__device__ __forceinline__ void load_tile(uint32_t tile, uint32_t tail_offset, const float* __restrict__ P, int64_t ld,
+                                          int major, int r0, int R, int rows_t, int k0, int k1, bool vec, int t,
+                                          float4* rowsum) {
+  constexpr int ITERS = ROWS_MAX * 8 / GROUP;
+  float4 v[ITERS];
+  if (major == MAJOR_K) {
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+      const int idx = t + i * GROUP;
+      const int r = idx >> 3, c = idx & 7;
+      const int gr = r0 + r, gk = k0 + 4 * c;
+      v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (r < rows_t && gr < R && gk < k1) {
+        const float* p = P + (int64_t)gr * ld + gk;
+        if (vec && gk + 3 < k1) {
+          v[i] = ldg_v4(p);
+        } else {
+          v[i].x = ldg_f(p);
+          if (gk + 1 < k1) v[i].y = ldg_f(p + 1);
+          if (gk + 2 < k1) v[i].z = ldg_f(p + 2);
+          if (gk + 3 < k1) v[i].w = ldg_f(p + 3);
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+      const int idx = t + i * GROUP;
+      const int r = idx >> 3, c = idx & 7;
+      if (r < rows_t) store_chunk<PRECISE>(tile + (r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4), tail_offset, v[i]);
+    }
+  } else {
+    const int cpr = rows_t >> 2;  // 16-byte chunks per k-row (multiple of 8)
+    const int atoms = rows_t >> 5;
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+      const int idx = t + i * GROUP;
+      const int kk = idx / cpr, cm = idx - kk * cpr;
+      const int gk = k0 + kk, gr = r0 + 4 * cm;
+      v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (kk < BK && gk < k1 && gr < R) {
+        const float* p = P + (int64_t)gk * ld + gr;
+        if (vec && gr + 3 < R) {
+          v[i] = ldg_v4(p);
+        } else {
+          v[i].x = ldg_f(p);
+          if (gr + 1 < R) v[i].y = ldg_f(p + 1);
+          if (gr + 2 < R) v[i].z = ldg_f(p + 2);
+          if (gr + 3 < R) v[i].w = ldg_f(p + 3);
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+      const int idx = t + i * GROUP;
+      const int kk = idx / cpr, cm = idx - kk * cpr;
+      if (kk < BK) {
+        const int a = cm >> 3, c = cm & 7;
+        store_chunk<PRECISE>(tile + (kk >> 2) * (atoms * 512) + a * 512 + (kk & 3) * 128 + ((c ^ ((kk & 3) << 1)) << 4),
+                             tail_offset, v[i]);
+        if (rowsum && rows_t == BM) {  // cm == t % 32 for every i: per-thread sums of 4 rows of C
+          rowsum->x += v[i].x; rowsum->y += v[i].y; rowsum->z += v[i].z; rowsum->w += v[i].w;
+        }
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void mma_tf32(uint32_t tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc)
+      : "memory");
+}
+
+// grid: (n tiles, m tiles, split_k).  Dynamic shared memory: Cfg::SMEM bytes.
+template <int BN_T, bool PRECISE>
+__global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kernel(TcArgs g) {
+  using C_ = Cfg<BN_T, PRECISE>;
+  constexpr int STAGES = C_::STAGES, GROUPS = C_::GROUPS, THREADS = C_::THREADS;
+  constexpr int MMA_WARP = GROUPS * 4;
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) uint64_t s_full[STAGES], s_empty[STAGES], s_accum;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+  __shared__ float s_rowsum[BM];
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int M = g.dev_M ? min(*g.dev_M, g.M) : g.M;
+  const int K = g.dev_K ? min(*g.dev_K, g.K) : g.K;
+  const int m0 = blockIdx.y * BM;
+  const int bn = min(BN_T, ((g.N + gridDim.x - 1) / gridDim.x + 31) / 32 * 32);  // columns per n-tile
+  const int n0 = blockIdx.x * bn;
+  if (m0 >= M || n0 >= g.N) return;
+  const int n_valid = min(bn, g.N - n0);
+  // MMA N: multiple of 16; MN-major B tiles are loaded in whole 32-column atoms
+  const int n_mma = (n_valid + 15) / 16 * 16;
+  const int b_rows = g.b_major == MAJOR_MN ? (n_valid + 31) / 32 * 32 : (n_mma + 7) / 8 * 8;
+  const int nkb_total = (K + BK - 1) / BK;
+  const int per = (nkb_total + g.split_k - 1) / g.split_k;
+  const int kb0 = blockIdx.z * per, kb1 = min(nkb_total, kb0 + per);
+  const int nkb = kb1 - kb0;
+
+  if (nkb <= 0) {  // nothing to contract: store mode still owes bias (+ReLU)
+    if (!g.accumulate && blockIdx.z == 0) {
+      for (int e = tid; e < BM * n_valid; e += THREADS) {
+        const int r = e / n_valid, c = e - r * n_valid;
+        if (m0 + r < M) {
+          float v = g.bias ? g.bias[n0 + c] : 0.f;
+          if (g.relu) v = fmaxf(v, 0.f);
+          g.C[(int64_t)(m0 + r) * g.ldc + n0 + c] = v;
+        }
+      }
+    }
+    return;
+  }
+
+  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t smem_base = smem_u32(smem);
+
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&s_full[s]), GROUP);
+      mbar_init(smem_u32(&s_empty[s]), 1);
+    }
+    mbar_init(smem_u32(&s_accum), 1);
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (tid < BM) s_rowsum[tid] = 0.f;
+  if (warp == MMA_WARP) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)),
+                 "r"(C_::TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = s_tmem;
+
+  if (warp < MMA_WARP) {
+    // ------------------------------------------------------------ producers
+    const int grp = warp >> 2, t = tid & (GROUP - 1);
+    const bool a_vec = (((uintptr_t)g.A & 15) == 0) && (g.lda % 4 == 0);
+    const bool b_vec = (((uintptr_t)g.B & 15) == 0) && (g.ldb % 4 == 0);
+    const bool want_rowsum = g.rowsum_out != nullptr && blockIdx.x == 0 && g.a_major == MAJOR_MN;
+    float4 rs = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int k_end = min(K, kb1 * BK);
+    bool ok = true;
+    for (int i = grp; i < nkb; i += GROUPS) {
+      const int s = i % STAGES;
+      if (i >= STAGES) {
+        ok = mbar_wait(smem_u32(&s_empty[s]), ((i / STAGES) - 1) & 1);
+        if (!ok) break;
+      }
+      const uint32_t a_tile = smem_base + s * C_::STAGE_BYTES;
+      const uint32_t b_tile = a_tile + C_::COPIES * C_::A_BYTES;
+      const int k0 = (kb0 + i) * BK;
+      load_tile<BM, PRECISE>(a_tile, C_::A_BYTES, g.A, g.lda, g.a_major, m0, M, BM, k0, k_end, a_vec, t,
+                             want_rowsum ? &rs : nullptr);
+      load_tile<BN_T, PRECISE>(b_tile, C_::B_BYTES, g.B, g.ldb, g.b_major, n0, g.N, b_rows, k0, k_end, b_vec, t, nullptr);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(smem_u32(&s_full[s]));
+    }
+    if (!ok) { s_abort = 1; atomicCAS(g.status, 0, TGNN_ETIMEOUT); }
+    if (want_rowsum) {  // the thread's chunks cover rows 4*(t%32) .. +3 of the tile
+      const int r = 4 * (t & 31);
+      atomicAdd(&s_rowsum[r], rs.x); atomicAdd(&s_rowsum[r + 1], rs.y);
+      atomicAdd(&s_rowsum[r + 2], rs.z); atomicAdd(&s_rowsum[r + 3], rs.w);
+    }
+    // ------------------------------------------------------------ epilogue
+    if (ok) ok = mbar_wait(smem_u32(&s_accum), 0);
+    if (!ok) { s_abort = 1; atomicCAS(g.status, 0, TGNN_ETIMEOUT); }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("bar.sync 1, %0;" ::"n"(GROUPS * GROUP) : "memory");  // all producers: s_rowsum complete
+    if (want_rowsum && tid < BM && m0 + tid < M && s_rowsum[tid] != 0.f) atomicAdd(&g.rowsum_out[m0 + tid], s_rowsum[tid]);
+    if (__all_sync(FULL, ok && !s_abort)) {  // warp-uniform: the TMEM loads are warp-collective
+      const int q4 = warp & 3;               // the TMEM lane quarter this warp may access
+      const int row = m0 + q4 * 32 + lane;
+      const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16);
+      const bool c_vec = (((uintptr_t)g.C & 15) == 0) && (g.ldc % 4 == 0) && (n0 % 4 == 0);
+      for (int c0 = grp * 16; c0 < n_mma; c0 += GROUPS * 16) {
+        uint32_t r[16];
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+            : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+              "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+            : "r"(taddr + (uint32_t)c0));
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (row < M) {
+          float* crow = g.C + (int64_t)row * g.ldc + n0 + c0;
+#pragma unroll
+          for (int q = 0; q < 16; q += 4) {
+            if (c0 + q >= n_valid) break;
+            float4 v = make_float4(__uint_as_float(r[q]), __uint_as_float(r[q + 1]), __uint_as_float(r[q + 2]),
+                                   __uint_as_float(r[q + 3]));
+            if (g.bias && blockIdx.z == 0) {
+              const float* bp = g.bias + n0 + c0 + q;
+              v.x += bp[0];
+              if (c0 + q + 1 < n_valid) v.y += bp[1];
+              if (c0 + q + 2 < n_valid) v.z += bp[2];
+              if (c0 + q + 3 < n_valid) v.w += bp[3];
+            }
+            const bool full4 = c0 + q + 3 < n_valid;
+            if (g.accumulate) {
+              if (full4 && c_vec) {
+                atomicAdd(reinterpret_cast<float4*>(crow + q), v);
+              } else {
+                atomicAdd(crow + q, v.x);
+                if (c0 + q + 1 < n_valid) atomicAdd(crow + q + 1, v.y);
+                if (c0 + q + 2 < n_valid) atomicAdd(crow + q + 2, v.z);
+                if (c0 + q + 3 < n_valid) atomicAdd(crow + q + 3, v.w);
+              }
+            } else {
+              if (g.relu) { v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); v.z = fmaxf(v.z, 0.f); v.w = fmaxf(v.w, 0.f); }
+              if (full4 && c_vec) {
+                *reinterpret_cast<float4*>(crow + q) = v;
+              } else {
+                crow[q] = v.x;
+                if (c0 + q + 1 < n_valid) crow[q + 1] = v.y;
+                if (c0 + q + 2 < n_valid) crow[q + 2] = v.z;
+                if (c0 + q + 3 < n_valid) crow[q + 3] = v.w;
+              }
+            }
+          }
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ MMA issuer
+    // instruction descriptor: D fp32, A/B tf32, majors, N >> 3, M >> 4
+    const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)g.a_major << 15) | ((uint32_t)g.b_major << 16) |
+                           ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    const int b_atoms = b_rows >> 5;
+    bool ok = true;
+    for (int i = 0; i < nkb && ok; ++i) {
+      const int s = i % STAGES;
+      ok = mbar_wait(smem_u32(&s_full[s]), (i / STAGES) & 1);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      if (lane == 0) {
+        const uint32_t a_addr = smem_base + s * C_::STAGE_BYTES;
+        const uint32_t b_addr = a_addr + C_::COPIES * C_::A_BYTES;
+#pragma unroll
+        for (int k = 0; k < BK / UMMA_K; ++k) {
+          // K-major: 8-row x 128 B atoms 1024 B apart (SBO); one MMA advances 32 B inside the swizzle row.
+          // MN-major: 4-k-row atoms of 512 B; MN atoms 512 B apart (LBO), k-groups atoms*512 B apart
+          // (SBO); one MMA consumes two k-groups.
+          const uint32_t a_off = g.a_major == MAJOR_K ? k * 32 : k * 2 * (BM / 32) * 512;
+          const uint32_t b_off = g.b_major == MAJOR_K ? k * 32 : k * 2 * b_atoms * 512;
+          const uint32_t a_lbo = g.a_major == MAJOR_K ? 16 : 512, a_sbo = g.a_major == MAJOR_K ? 1024 : (BM / 32) * 512;
+          const uint32_t b_lbo = g.b_major == MAJOR_K ? 16 : 512, b_sbo = g.b_major == MAJOR_K ? 1024 : b_atoms * 512;
+          const uint32_t a_lay = g.a_major == MAJOR_K ? 2 : 1, b_lay = g.b_major == MAJOR_K ? 2 : 1;
+          const uint64_t da = make_desc(a_addr + a_off, a_lbo, a_sbo, a_lay);
+          const uint64_t db = make_desc(b_addr + b_off, b_lbo, b_sbo, b_lay);
+          const uint32_t first = (i > 0 || k > 0) ? 1u : 0u;
+          if (PRECISE) {
+            const uint64_t da_lo = make_desc(a_addr + C_::A_BYTES + a_off, a_lbo, a_sbo, a_lay);
+            const uint64_t db_lo = make_desc(b_addr + C_::B_BYTES + b_off, b_lbo, b_sbo, b_lay);
+            mma_tf32(tmem, da_lo, db, idesc, first);  // tail(A) * head(B)
+            mma_tf32(tmem, da, db_lo, idesc, 1u);     // head(A) * tail(B)
+            mma_tf32(tmem, da, db, idesc, 1u);        // head(A) * head(B)
+          } else {
+            mma_tf32(tmem, da, db, idesc, first);
+          }
+        }
+        // frees the stage for the producers once the MMAs that read it have completed
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s_empty[s]))
+                     : "memory");
+      }
+      __syncwarp();
+    }
+    if (lane == 0) {
+      if (ok)
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s_accum))
+                     : "memory");
+      else { s_abort = 1; atomicCAS(g.status, 0, TGNN_ETIMEOUT); }
+    }
+    __syncwarp();
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == MMA_WARP) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C_::TMEM_COLS) : "memory");
+  }
+}
+
+template <int BN_T, bool PRECISE>
+int launch_tc(tgnn_ctx* ctx, const TcArgs& a, int n_tiles, const char* name, cudaStream_t s) {
+  using C_ = Cfg<BN_T, PRECISE>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(gemm_tf32_kernel<BN_T, PRECISE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           C_::SMEM));
+    attr_set = true;
+  }
+  dim3 grid(n_tiles, (a.M + BM - 1) / BM, a.split_k);
+  {
+    KernelScope scope__(ctx, name, s);
+    gemm_tf32_kernel<BN_T, PRECISE><<<grid, C_::THREADS, C_::SMEM, s>>>(a);
+  }
+  TGNN_LAUNCH_OK(ctx, name);
+  return TGNN_OK;
+}
+
+}  // namespace
+
+// Returns TGNN_OK after launching, or 1 if the product does not fit this kernel (caller falls back to the FMA tiles).
+int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s) {
+  TcArgs a = {};
+  if (g.a_cs == 1) { a.a_major = MAJOR_K; a.lda = g.a_rs; }
+  else if (g.a_rs == 1) { a.a_major = MAJOR_MN; a.lda = g.a_cs; }
+  else return 1;
+  if (g.b_rs == 1) { a.b_major = MAJOR_K; a.ldb = g.b_cs; }
+  else if (g.b_cs == 1) { a.b_major = MAJOR_MN; a.ldb = g.b_rs; }
+  else return 1;
+  if (g.rowsum_out && a.a_major != MAJOR_MN) return 1;
+  a.A = g.A; a.B = g.B; a.C = g.C; a.ldc = g.ldc;
+  a.M = g.M; a.N = g.N; a.K = g.K; a.dev_M = g.dev_M; a.dev_K = g.dev_K;
+  a.bias = g.bias; a.rowsum_out = g.rowsum_out; a.relu = g.relu; a.accumulate = g.accumulate;
+  a.status = ctx->ws.status;
+  // n-tiles of at most 256 columns, balanced, whole 32-column atoms
+  const int n_tiles = (g.N + 255) / 256;
+  a.split_k = 1;
+  if (g.accumulate && g.split_k > 1) {  // the caller allows split-K: one wave of CTAs, >= 4 stages of work each
+    const int tiles = n_tiles * ((g.M + BM - 1) / BM);
+    const int max_s = (g.K + 4 * BK - 1) / (4 * BK);
+    a.split_k = (148 + tiles - 1) / tiles;
+    if (a.split_k > max_s) a.split_k = max_s;
+    if (a.split_k < 1) a.split_k = 1;
+  }
+  const int bn = ((g.N + n_tiles - 1) / n_tiles + 31) / 32 * 32;
+  if (g.precise) {
+    if (bn <= 128) return launch_tc<128, true>(ctx, a, n_tiles, name, s);
+    return launch_tc<256, true>(ctx, a, n_tiles, name, s);
+  }
+  if (bn <= 128) return launch_tc<128, false>(ctx, a, n_tiles, name, s);
+  return launch_tc<256, false>(ctx, a, n_tiles, name, s);
+}
+
+}  // namespace tgnn

@@ -10,12 +10,17 @@ namespace {
 __device__ __forceinline__ void write_message_row(float* __restrict__ row, const float* __restrict__ memory,
                                                   const void* __restrict__ efeat, int feat_bf16,
                                                   const float* __restrict__ time_w, const float* __restrict__ time_b,
-                                                  int d, int de, int self, int other, int eid, float dtf, int lane) {
+                                                  int d, int de, int self, int other, int eid, float dtf, int lane,
+                                                  float* __restrict__ sin_row) {
   warp_copy_f32(row, memory + (int64_t)self * d, d, lane);
   warp_copy_f32(row + d, memory + (int64_t)other * d, d, lane);
   warp_copy_feat(row + 2 * d, efeat, feat_bf16, eid, de, lane);
   float* phi = row + 2 * d + de;
-  for (int q = lane; q < d; q += 32) phi[q] = time_encode(time_w[q], time_b[q], dtf);
+  if (sin_row == nullptr) {
+    for (int q = lane; q < d; q += 32) phi[q] = time_encode(time_w[q], time_b[q], dtf);
+  } else {
+    for (int q = lane; q < d; q += 32) time_encode_sc(time_w[q], time_b[q], dtf, &phi[q], &sin_row[q]);
+  }
 }
 
 // One warp per message j = 2i + role.
@@ -45,7 +50,7 @@ __global__ void __launch_bounds__(256) build_messages_kernel(const float* __rest
       continue;
     }
     const float dtf = (float)(t[i] - last_update[self]);
-    write_message_row(row, memory, efeat, feat_bf16, time_w, time_b, d, de, self, other, eid[i], dtf, lane);
+    write_message_row(row, memory, efeat, feat_bf16, time_w, time_b, d, de, self, other, eid[i], dtf, lane, nullptr);
   }
 }
 
@@ -61,7 +66,7 @@ __global__ void __launch_bounds__(256) gather_winner_kernel(const float* __restr
                                                             const int32_t* __restrict__ winner,
                                                             const int32_t* __restrict__ n_uniq, int u_cap, int ld,
                                                             float* __restrict__ X, float* __restrict__ x_dt,
-                                                            double* __restrict__ win_t) {
+                                                            float* __restrict__ Xsin, double* __restrict__ win_t) {
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   const int U = min(*n_uniq, u_cap);
@@ -73,10 +78,13 @@ __global__ void __launch_bounds__(256) gather_winner_kernel(const float* __restr
     const double ti = t[i];
     const float dtf = (float)(ti - last_update[self]);
     float* row = X + (int64_t)u * ld;
-    if (msg != nullptr)
+    float* sin_row = Xsin + (int64_t)u * d;
+    if (msg != nullptr) {
       warp_copy_f32(row, msg + (int64_t)j * dm, dm, lane);
-    else
-      write_message_row(row, memory, efeat, feat_bf16, time_w, time_b, d, de, self, other, eid[i], dtf, lane);
+      for (int q = lane; q < d; q += 32) sin_row[q] = sinf(time_arg(time_w[q], time_b[q], dtf));
+    } else {
+      write_message_row(row, memory, efeat, feat_bf16, time_w, time_b, d, de, self, other, eid[i], dtf, lane, sin_row);
+    }
     for (int q = dm + lane; q < ld; q += 32) row[q] = 0.f;
     if (lane == 0) { x_dt[u] = dtf; win_t[u] = ti; }
   }
@@ -140,7 +148,7 @@ int launch_memory_update(tgnn_ctx* ctx, const float* msg, const int32_t* uniq, c
                                                          c.feat_dtype == TGNN_BF16, ctx->params + L.time_w,
                                                          ctx->params + L.time_b, d, c.d_e, ctx->m_src, ctx->m_dst, ctx->m_t,
                                                          ctx->m_eid, msg, uniq, winner, n_uniq, U_cap, ctx->ld_msg, w.X,
-                                                         w.x_dt, w.win_t);
+                                                         w.x_dt, w.Xsin, w.win_t);
   }
   TGNN_LAUNCH_OK(ctx, "gather_winner");
   GemmArgs g = {};

@@ -52,12 +52,12 @@ namespace {
 int check_config(const tgnn_config* c) {
   if (!c) return TGNN_EINVAL;
   if (c->num_nodes <= 0 || c->num_nodes > 0x7fffffff) return TGNN_EINVAL;
-  if (c->d <= 0 || c->d % 4 != 0 || c->heads <= 0 || c->d % c->heads != 0) return TGNN_ESHAPE;
+  if (c->d <= 0 || c->d > 256 || c->d % 4 != 0 || c->heads <= 0 || c->d % c->heads != 0) return TGNN_ESHAPE;
   if (c->d_e < 0 || c->d_e % 2 != 0) return TGNN_ESHAPE;
   if (c->k < 1 || c->k > 32 || c->heads * c->k > 1024) return TGNN_ESHAPE;
   if (c->feat_dtype != TGNN_F32 && c->feat_dtype != TGNN_BF16) return TGNN_EINVAL;
   if (c->max_events < 1 || c->max_roots < 3 || c->max_events > (1 << 24) || c->max_roots > (1 << 24)) return TGNN_EINVAL;
-  if (c->math_mode != TGNN_MATH_FP32 && c->math_mode != TGNN_MATH_TF32) return TGNN_EINVAL;
+  if (c->math_mode != TGNN_MATH_FP32 && c->math_mode != TGNN_MATH_TF32 && c->math_mode != TGNN_MATH_TF32_FAST) return TGNN_EINVAL;
   if (!(c->lr >= 0.f) || !(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f) || !(c->eps > 0.f))
     return TGNN_EINVAL;
   return TGNN_OK;
@@ -111,12 +111,14 @@ size_t carve(tgnn_ctx* ctx, char* base) {
   cv.take(w.st_u_keep, ne); cv.take(w.st_mask, nq);
   cv.take(w.X, U * ctx->ld_msg);
   cv.take(w.x_dt, U);
+  cv.take(w.Xsin, U * d);
   cv.take(w.win_t, U);
   cv.take(w.Gi, U * 3 * d);
   cv.take(w.Gh, U * 3 * d);
   cv.take(w.g_r, U * d); cv.take(w.g_z, U * d); cv.take(w.g_n, U * d); cv.take(w.g_hn, U * d);
   cv.take(w.Z, NB * ctx->ld_kv);
   cv.take(w.z_dt, NB);
+  cv.take(w.Zsin, NB * d);
   cv.take(w.KV, NB * 2 * d);
   cv.take(w.Zq, R * 2 * d);
   cv.take(w.Q, R * d);
@@ -124,6 +126,7 @@ size_t carve(tgnn_ctx* ctx, char* base) {
   cv.take(w.cat_o, R * 2 * d);
   cv.take(w.cat1, 2 * nq * 2 * d);
   cv.take(w.hid1, 2 * nq * d);
+  cv.take(w.hid_gate, 2 * nq * d);
   cv.take(w.dcat1, 2 * nq * 2 * d);
   cv.take(w.dpre_o, R * d);
   cv.take(w.dcat_o, R * 2 * d);
@@ -414,6 +417,26 @@ int tgnn_debug_get_grads(tgnn_ctx* ctx, float* grads_out, void* stream) {
   TGNN_CUDA_OK(ctx, cudaMemcpyAsync(grads_out, ctx->ws.grads, sizeof(float) * (size_t)ctx->L.total,
                                     cudaMemcpyDeviceToDevice, S(stream)));
   return TGNN_OK;
+}
+
+int tgnn_debug_get_gates(tgnn_ctx* ctx, uint8_t* h_gate_out, uint8_t* hid_gate_out, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, h_gate_out && hid_gate_out, TGNN_EINVAL, "debug_get_gates: null pointer");
+  NEED(ctx, ctx->e_h && ctx->e_n % 3 == 0, TGNN_ESTATE, "debug_get_gates: no embedding / backward pass recorded");
+  return launch_get_gates(ctx, h_gate_out, hid_gate_out, S(stream));
+}
+
+int tgnn_debug_gemm(tgnn_ctx* ctx, const float* A, int64_t a_rs, int64_t a_cs, const float* B, int64_t b_rs, int64_t b_cs,
+                    float* C, int64_t ldc, int M, int N, int K, const int32_t* dev_M, const int32_t* dev_K,
+                    const float* bias, float* rowsum_out, int relu, int accumulate, int split_k, int precise,
+                    void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, A && B && C && M >= 0 && N >= 0 && K >= 0, TGNN_EINVAL, "debug_gemm: null pointer or negative size");
+  GemmArgs g = {};
+  g.A = A; g.a_rs = a_rs; g.a_cs = a_cs; g.B = B; g.b_rs = b_rs; g.b_cs = b_cs; g.C = C; g.ldc = ldc;
+  g.M = M; g.N = N; g.K = K; g.dev_M = dev_M; g.dev_K = dev_K; g.bias = bias; g.rowsum_out = rowsum_out;
+  g.relu = relu; g.accumulate = accumulate; g.split_k = split_k < 1 ? 1 : split_k; g.precise = precise;
+  return launch_gemm(ctx, g, "debug_gemm", S(stream));
 }
 
 int tgnn_status(tgnn_ctx* ctx, int32_t* status_host, void* stream) {

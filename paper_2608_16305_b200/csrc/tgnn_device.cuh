@@ -10,6 +10,10 @@ namespace tgnn {
 // full-range accurate routine (the library is built without fast-math).
 __device__ __forceinline__ float time_arg(float w, float b, float dtf) { return fmaf(w, dtf, b); }
 __device__ __forceinline__ float time_encode(float w, float b, float dtf) { return cosf(time_arg(w, b, dtf)); }
+// cos and sin of the same argument at once; the sine is kept for the backward pass (d Phi / d arg = -sin).
+__device__ __forceinline__ void time_encode_sc(float w, float b, float dtf, float* cos_out, float* sin_out) {
+  sincosf(time_arg(w, b, dtf), sin_out, cos_out);
+}
 
 __device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + expf(-x)); }
 __device__ __forceinline__ float softplusf_(float x) { return x > 0.f ? x + log1pf(expf(-x)) : log1pf(expf(x)); }

@@ -47,6 +47,7 @@ struct Workspace {
   // step (4) activations
   float* X;        // [U_cap, ld_msg] winners' message rows (first d columns = the node's own memory)
   float* x_dt;     // [U_cap] fp32 dt inside Phi of the winner message
+  float* Xsin;     // [U_cap, d] sin of the time-encoding arguments of the winner messages
   double* win_t;   // [U_cap]
   float* Gi;       // [U_cap, 3d]
   float* Gh;       // [U_cap, 3d]
@@ -54,6 +55,7 @@ struct Workspace {
   // step (5) activations
   float* Z;      // [NB_cap, ld_kv]
   float* z_dt;   // [NB_cap]
+  float* Zsin;   // [NB_cap, d] sin of the time-encoding arguments of Z (zero for empty slots)
   float* KV;     // [NB_cap, 2d]  (K | V)
   float* Zq;     // [R_cap, 2d]
   float* Q;      // [R_cap, d]
@@ -62,6 +64,7 @@ struct Workspace {
   // step (6)
   float* cat1;    // [2*nq_cap, 2d]
   float* hid1;    // [2*nq_cap, d]  ReLU(pre1); overwritten by dpre1
+  uint8_t* hid_gate;  // [2*nq_cap, d] 1 where the head's hidden unit was active
   float* dcat1;   // [2*nq_cap, 2d]
   float* dpre_o;  // [R_cap, d]
   float* dcat_o;  // [R_cap, 2d]
@@ -196,6 +199,8 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
 int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* loss_out, float* gradnorm_out,
                     cudaStream_t s);
 
+int launch_get_gates(tgnn_ctx* ctx, uint8_t* h_gate_out, uint8_t* hid_gate_out, cudaStream_t s);
+
 // ---- dense projections (k_gemm.cu) ----
 // C[M,N] (+)= sum_k A(m,k) B(k,n) (+ bias[n]) (ReLU);  A(m,k) = A[m*a_rs + k*a_cs], B(k,n) = B[k*b_rs + n*b_cs].
 struct GemmArgs {
@@ -210,7 +215,9 @@ struct GemmArgs {
   int relu;               // apply ReLU in the epilogue (store mode only)
   int accumulate;         // atomicAdd into C (C must hold valid data); required when split_k > 1
   int split_k;            // >= 1
+  int precise;            // tensor-core mode only: 3xTF32 head/tail split, close to fp32 accuracy
 };
 int launch_gemm(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s);
+int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s);  // k_gemm_tc.cu
 
 }  // namespace tgnn

@@ -501,6 +501,28 @@ def test_gradient_against_central_differences(oracle, seed):
     assert abs(base.gradnorm - math.sqrt((base.grads ** 2).sum())) < 1e-14
 
 
+def test_relu_gate_hints_apply_only_inside_the_window(oracle):
+    cfg = small_cfg(oracle, N=20, phi_f32=False, round_state_f32=False)
+    W = weights(cfg)
+    c = _full_case(oracle, cfg, W)
+    args = (cfg, c["P"], c["mem"], c["lu"], c["ef"], c["upd"], c["roots"], c["n_q"], None)
+    base = oracle.loss_and_grads(*args)
+    R, nq, d = len(c["roots"][0]), c["n_q"], cfg.d
+    own_h = (base.h > 0).astype(np.uint8)
+    zeros_h, zeros_hid = np.zeros((R, d), np.uint8), np.zeros((2 * nq, d), np.uint8)
+    # a zero-width window ignores the hints entirely
+    r = oracle.loss_and_grads(*args, h_gate=zeros_h, hid_gate=zeros_hid, gate_eps=0.0)
+    assert r.loss == base.loss and np.array_equal(r.grads, base.grads)
+    # a narrow window around zero touches no unit of this case: wrong hints change nothing
+    r = oracle.loss_and_grads(*args, h_gate=1 - own_h, hid_gate=zeros_hid, gate_eps=1e-9)
+    assert r.loss == base.loss and np.array_equal(r.grads, base.grads)
+    # a window covering everything with all gates closed switches every unit off: h = 0, score = b_2
+    r = oracle.loss_and_grads(*args, h_gate=zeros_h, hid_gate=zeros_hid, gate_eps=1.0)
+    assert not r.h.any()
+    b2 = float(W["b_2"][0])
+    assert abs(r.loss - (math.log1p(math.exp(-b2)) + math.log1p(math.exp(b2)))) < 1e-12
+
+
 # --------------------------------------------------------------- Adam ------
 def test_adam_first_step_closed_form(oracle):
     cfg = small_cfg(oracle, lr=1e-3)
