@@ -382,7 +382,12 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
   const int R = 3 * n_q, NB = R * k;
   float* P = ctx->params;
   float* G = w.grads;
-  // grads | dMemU | red | st_scalars are contiguous in the arena: one memset clears them all
+  // The chain loss -> head -> output projection -> attention -> inputs -> memory rows -> GRU is
+  // sequential and stays on the caller's stream s.  Weight-gradient products and time-encoder sums
+  // are leaves of that chain: they go to the two side streams as soon as their operands exist and
+  // are joined back before the gradient norm.
+  cudaStream_t sa = ctx->side[0], sb = ctx->side[1];
+  // grads | dMemU | red | tg_acc | st_scalars are contiguous in the arena: one memset clears them all
   const size_t zero_bytes = (size_t)((char*)(w.st_scalars + 4) - (char*)w.grads);
   TGNN_CUDA_OK(ctx, cudaMemsetAsync(w.grads, 0, zero_bytes, s));
 
@@ -405,7 +410,8 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     }
     TGNN_LAUNCH_OK(ctx, "head_loss");
     // hid1 now holds d loss / d pre1
-    RC(grad_w(ctx, w.hid1, d, w.cat1, 2 * d, 2 * n_q, nullptr, d, 2 * d, G + L.w1, G + L.b1, "dW_1", s));
+    RC(fork_to(ctx, s, sa));
+    RC(grad_w(ctx, w.hid1, d, w.cat1, 2 * d, 2 * n_q, nullptr, d, 2 * d, G + L.w1, G + L.b1, "dW_1", sa));
     RC(grad_in(ctx, w.hid1, d, P + L.w1, 2 * d, 0, 2 * n_q, nullptr, d, 2 * d, w.dcat1, 2 * d, "dcat1", s));
     const int64_t tot2 = (int64_t)R * d;
     {
@@ -413,7 +419,8 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       dh_kernel<<<(int)((tot2 + 255) / 256), 256, 0, s>>>(w.dcat1, ctx->e_h, n_q, d, w.dpre_o);
     }
     TGNN_LAUNCH_OK(ctx, "dh");
-    RC(grad_w(ctx, w.dpre_o, d, w.cat_o, 2 * d, R, nullptr, d, 2 * d, G + L.wo, G + L.bo, "dW_o", s));
+    RC(fork_to(ctx, s, sb));
+    RC(grad_w(ctx, w.dpre_o, d, w.cat_o, 2 * d, R, nullptr, d, 2 * d, G + L.wo, G + L.bo, "dW_o", sb));
     RC(grad_in(ctx, w.dpre_o, d, P + L.wo, 2 * d, 0, R, nullptr, d, 2 * d, w.dcat_o, 2 * d, "dcat_o", s));
     const int wpb = 8;
     {
@@ -422,22 +429,25 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
           w.Q, w.KV, w.alpha, w.dcat_o, ctx->e_cnt, R, d, H, k, w.dQ, w.dKV);
     }
     TGNN_LAUNCH_OK(ctx, "attention_bwd");
-    RC(grad_w(ctx, w.dQ, d, w.Zq, 2 * d, R, nullptr, d, 2 * d, G + L.wq, G + L.bq, "dW_q", s));
-    RC(grad_in(ctx, w.dQ, d, P + L.wq, 2 * d, 0, R, nullptr, d, 2 * d, w.dzq, 2 * d, "dzq", s));
-    RC(grad_w(ctx, w.dKV, 2 * d, w.Z, ctx->ld_kv, NB, nullptr, 2 * d, (int)L.dkv, G + L.wk, G + L.bk, "dW_kv", s));
-    RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, d + de, NB, nullptr, 2 * d, d, w.dZp, d, "dZ_phi", s));
-    // time-encoder gradient through the attention inputs
+    RC(fork_to(ctx, s, sa));
+    RC(fork_to(ctx, s, sb));
+    RC(grad_w(ctx, w.dKV, 2 * d, w.Z, ctx->ld_kv, NB, nullptr, 2 * d, (int)L.dkv, G + L.wk, G + L.bk, "dW_kv", sa));
+    RC(grad_w(ctx, w.dQ, d, w.Zq, 2 * d, R, nullptr, d, 2 * d, G + L.wq, G + L.bq, "dW_q", sb));
+    // time-encoder gradient through the attention inputs (side stream b)
     const size_t tg_smem = (size_t)8 * 2 * d * sizeof(double);
+    RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, d + de, NB, nullptr, 2 * d, d, w.dZp, d, "dZ_phi", sb));
     {
-      KernelScope scope__(ctx, "time_grad_z", s);
-      time_grad_kernel<<<(NB + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, s>>>(w.dZp, d, 0, w.Zsin, w.z_dt, NB, nullptr, d,
-                                                                          P + L.time_b, w.tg_acc);
+      KernelScope scope__(ctx, "time_grad_z", sb);
+      time_grad_kernel<<<(NB + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, sb>>>(w.dZp, d, 0, w.Zsin, w.z_dt, NB, nullptr, d,
+                                                                           P + L.time_b, w.tg_acc);
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_z");
+    RC(grad_in(ctx, w.dQ, d, P + L.wq, 2 * d, 0, R, nullptr, d, 2 * d, w.dzq, 2 * d, "dzq", s));
+    RC(fork_to(ctx, s, sb));
     {
-      KernelScope scope__(ctx, "time_grad_q", s);
-      time_grad_kernel<<<(R + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, s>>>(w.dzq, 2 * d, d, nullptr, nullptr, R, nullptr, d,
-                                                                         P + L.time_b, w.tg_acc);
+      KernelScope scope__(ctx, "time_grad_q", sb);
+      time_grad_kernel<<<(R + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, sb>>>(w.dzq, 2 * d, d, nullptr, nullptr, R, nullptr, d,
+                                                                          P + L.time_b, w.tg_acc);
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_q");
     if (ctx->have_update) {
@@ -456,10 +466,12 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
                                                                       w.g_hn, ctx->upd_n_uniq, U_cap, w.dGi, w.dGh);
       }
       TGNN_LAUNCH_OK(ctx, "gru_bwd_gate");
+      RC(fork_to(ctx, s, sa));
+      RC(fork_to(ctx, s, sb));
       RC(grad_w(ctx, w.dGi, 3 * d, w.X, ctx->ld_msg, U_cap, ctx->upd_n_uniq, 3 * d, (int)L.dmsg, G + L.gru_wi,
-                G + L.gru_bi, "dW_i", s));
+                G + L.gru_bi, "dW_i", sa));
       RC(grad_w(ctx, w.dGh, 3 * d, w.X, ctx->ld_msg, U_cap, ctx->upd_n_uniq, 3 * d, d, G + L.gru_wh, G + L.gru_bh,
-                "dW_h", s));
+                "dW_h", sb));
       RC(grad_in(ctx, w.dGi, 3 * d, P + L.gru_wi, L.dmsg, 2 * d + de, U_cap, ctx->upd_n_uniq, 3 * d, d, w.dXp, d,
                  "dX_phi", s));
       {
@@ -469,8 +481,8 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       }
       TGNN_LAUNCH_OK(ctx, "time_grad_x");
     }
-  }
-  if (n_q > 0) {
+    RC(fork_to(ctx, sa, s));  // join
+    RC(fork_to(ctx, sb, s));
     {
       KernelScope scope__(ctx, "time_grad_finish", s);
       time_grad_finish_kernel<<<(2 * d + 127) / 128, 128, 0, s>>>(w.tg_acc, 2 * d, G + L.time_w);

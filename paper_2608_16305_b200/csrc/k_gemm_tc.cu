@@ -461,8 +461,12 @@ int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStr
   a.M = g.M; a.N = g.N; a.K = g.K; a.dev_M = g.dev_M; a.dev_K = g.dev_K;
   a.bias = g.bias; a.rowsum_out = g.rowsum_out; a.relu = g.relu; a.accumulate = g.accumulate;
   a.status = ctx->ws.status;
-  // n-tiles of at most 256 columns, balanced, whole 32-column atoms
-  const int n_tiles = (g.N + 255) / 256;
+  // n-tiles of at most 256 columns, balanced, whole 32-column atoms; narrower tiles (down to 64
+  // columns) when the product would otherwise occupy only a few SMs
+  int n_tiles = (g.N + 255) / 256;
+  const int m_tiles = (g.M + BM - 1) / BM;
+  if (!(g.accumulate && g.split_k > 1))
+    while (m_tiles * n_tiles < 96 && ((g.N + n_tiles - 1) / n_tiles + 31) / 32 * 32 > 64) ++n_tiles;
   a.split_k = 1;
   if (g.accumulate && g.split_k > 1) {  // the caller allows split-K: one wave of CTAs, >= 4 stages of work each
     const int tiles = n_tiles * ((g.M + BM - 1) / BM);

@@ -156,10 +156,14 @@ int launch_memory_update(tgnn_ctx* ctx, const float* msg, const int32_t* uniq, c
   g.B = ctx->params + L.gru_wi; g.b_rs = 1; g.b_cs = L.dmsg;  // B(k,n) = W_i[n,k]
   g.C = w.Gi; g.ldc = 3 * d; g.M = U_cap; g.N = 3 * d; g.K = (int)L.dmsg; g.dev_M = n_uniq;
   g.bias = ctx->params + L.gru_bi; g.split_k = 1;
-  int rc = launch_gemm(ctx, g, "gru_gi", s);
+  int rc = fork_to(ctx, s, ctx->side[0]);  // the hidden-state product runs beside the input product
+  if (rc) return rc;
+  rc = launch_gemm(ctx, g, "gru_gi", s);
   if (rc) return rc;
   g.B = ctx->params + L.gru_wh; g.b_cs = d; g.C = w.Gh; g.K = d; g.bias = ctx->params + L.gru_bh;
-  rc = launch_gemm(ctx, g, "gru_gh", s);
+  rc = launch_gemm(ctx, g, "gru_gh", ctx->side[0]);
+  if (rc) return rc;
+  rc = fork_to(ctx, ctx->side[0], s);
   if (rc) return rc;
   const int64_t total = (int64_t)U_cap * d;
   {

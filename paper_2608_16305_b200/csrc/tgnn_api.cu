@@ -214,6 +214,15 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
     delete ctx;
     return TGNN_ECUDA;
   }
+  ctx->ev_next = 0;
+  for (int i = 0; ok && i < 2; ++i) ok = cudaStreamCreateWithFlags(&ctx->side[i], cudaStreamNonBlocking) == cudaSuccess;
+  for (int i = 0; ok && i < 16; ++i) ok = cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    cudaFree(ctx->arena);
+    delete ctx;
+    return TGNN_ECUDA;
+  }
   snprintf(ctx->err, sizeof(ctx->err), "no error");
   *out = ctx;
   return TGNN_OK;
@@ -226,6 +235,8 @@ int tgnn_destroy(tgnn_ctx* ctx) {
     cudaEventDestroy(e.a);
     cudaEventDestroy(e.b);
   }
+  for (int i = 0; i < 2; ++i) cudaStreamDestroy(ctx->side[i]);
+  for (int i = 0; i < 16; ++i) cudaEventDestroy(ctx->ev[i]);
   cudaFree(ctx->arena);
   delete ctx;
   return TGNN_OK;
@@ -357,6 +368,14 @@ int tgnn_train_step(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, c
   Workspace& w = ctx->ws;
   int rc;
   ctx->have_update = false;
+  // the neighbor search reads only the static graph: it runs beside the memory update
+  cudaStream_t side = ctx->side[1];
+  rc = fork_to(ctx, S(stream), side);
+  if (rc) return rc;
+  rc = launch_make_roots(ctx, q_src, q_dst, q_neg, q_t, n_q, side);
+  if (rc) return rc;
+  rc = tgnn_sample_recent(ctx, w.r_node, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, w.nb_cnt, side);
+  if (rc) return rc;
   if (n_u > 0) {
     rc = tgnn_build_messages(ctx, u_src, u_dst, u_t, u_eid, u_keep, n_u, nullptr, w.msg_node, stream);
     if (rc) return rc;
@@ -365,9 +384,7 @@ int tgnn_train_step(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, c
     rc = tgnn_memory_update(ctx, nullptr, w.uniq, w.winner, w.n_uniq, stream);
     if (rc) return rc;
   }
-  rc = launch_make_roots(ctx, q_src, q_dst, q_neg, q_t, n_q, S(stream));
-  if (rc) return rc;
-  rc = tgnn_sample_recent(ctx, w.r_node, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, w.nb_cnt, stream);
+  rc = fork_to(ctx, side, S(stream));  // join
   if (rc) return rc;
   rc = tgnn_embed(ctx, w.r_node, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, w.nb_cnt, w.h, stream);
   if (rc) return rc;

@@ -132,6 +132,12 @@ struct tgnn_ctx {
   tgnn::Workspace ws;
   void* arena;
   size_t arena_bytes;
+  // Two internal streams for kernels that do not lie on the step's critical chain (weight-gradient
+  // products, the neighbor search next to the memory update, ...).  They are forked from and joined
+  // back into the caller's stream with events, so the caller still sees one ordered stream of work.
+  cudaStream_t side[2];
+  cudaEvent_t ev[16];
+  int ev_next;
   int64_t launches;
   tgnn::Profiler prof;
   char err[256];
@@ -151,6 +157,15 @@ int set_error(tgnn_ctx* ctx, int code, const char* fmt, ...);
     cudaError_t e__ = cudaGetLastError();                                                    \
     if (e__ != cudaSuccess) return tgnn::set_error(ctx, TGNN_ECUDA, "launch %s: %s", name, cudaGetErrorString(e__)); \
   } while (0)
+
+// side[i] waits for everything enqueued so far on `from`.
+inline int fork_to(tgnn_ctx* ctx, cudaStream_t from, cudaStream_t to) {
+  cudaEvent_t e = ctx->ev[ctx->ev_next];
+  ctx->ev_next = (ctx->ev_next + 1) % 16;
+  if (cudaEventRecord(e, from) != cudaSuccess || cudaStreamWaitEvent(to, e, 0) != cudaSuccess)
+    return set_error(ctx, TGNN_ECUDA, "stream fork/join failed: %s", cudaGetErrorString(cudaGetLastError()));
+  return TGNN_OK;
+}
 
 // Brackets one kernel launch with events when profiling is on.
 struct KernelScope {
