@@ -207,11 +207,21 @@ TGNN_API int tgnn_backward_step(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask
  * the update events (previous kept batch: u_src..u_keep, n_u, may be 0) refresh
  * memory, then the n_q target events (q_src,q_dst,q_neg:int32[n_q], q_t:f64[n_q])
  * are sampled, embedded, scored and trained on.  Equivalent to calling the six
- * entry points above with workspace-owned intermediates. */
+ * entry points above with workspace-owned intermediates.  The inputs are first
+ * copied into fixed staging buffers by the first kernel of the step; treat them
+ * as borrowed until the stream has passed that kernel.
+ * Graph replay: the second call with the same (n_u, n_q, keep / mask presence,
+ * output pointers) records the step's launch sequence with CUDA stream capture
+ * on `stream` (which therefore must not be the legacy default stream; if capture
+ * is refused the library silently keeps launching kernel by kernel) and later
+ * calls replay the instantiated graph.  tgnn_set_graph_replay(ctx, 0) turns this
+ * off.  Profiling (tgnn_profile_begin) always uses plain launches. */
 TGNN_API int tgnn_train_step(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, const double* u_t, const int32_t* u_eid,
                     const uint8_t* u_keep, int n_u, const int32_t* q_src, const int32_t* q_dst, const int32_t* q_neg,
                     const double* q_t, int n_q, const uint8_t* loss_mask, float* loss_out, float* gradnorm_out,
                     void* stream);
+
+TGNN_API int tgnn_set_graph_replay(tgnn_ctx* ctx, int enable);
 
 /* The same step with HOST inputs and outputs: the event arrays are copied to
  * workspace staging buffers with cudaMemcpyAsync (pin them for overlap), and

@@ -26,7 +26,7 @@ EXPORTS = ("tgnn_create", "tgnn_destroy", "tgnn_last_error", "tgnn_param_count",
            "tgnn_set_graph", "tgnn_set_edge_features", "tgnn_set_state", "tgnn_prune_mask", "tgnn_sample_recent",
            "tgnn_build_messages", "tgnn_reduce_latest", "tgnn_memory_update", "tgnn_embed", "tgnn_backward_step",
            "tgnn_train_step", "tgnn_train_step_host", "tgnn_debug_get_grads", "tgnn_status", "tgnn_kernel_launches", "tgnn_profile_begin",
-           "tgnn_profile_report", "tgnn_reduce_latest_static", "tgnn_debug_gemm", "tgnn_debug_get_gates")
+           "tgnn_profile_report", "tgnn_reduce_latest_static", "tgnn_debug_gemm", "tgnn_debug_get_gates", "tgnn_set_graph_replay")
 TGNN_STATIC_MAX_NODES = 65536
 
 
@@ -83,6 +83,7 @@ def load_library():
         lib.tgnn_debug_gemm.argtypes = [vp, vp, i64, i64, vp, i64, i64, vp, i64, i32, i32, i32, vp, vp, vp, vp, i32, i32, i32, i32,
                                         vp]
         lib.tgnn_debug_get_gates.argtypes = [vp, vp, vp, vp]
+        lib.tgnn_set_graph_replay.argtypes = [vp, i32]
         lib.tgnn_reduce_latest_static.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, vp, vp, i32]
         _lib = lib
     return _lib
@@ -270,6 +271,9 @@ class Tgnn:
                                                _hp(q_t, "f64", "q_t"), q_src.numel(), _hp(loss_mask, "u8", "loss_mask"),
                                                _hp(loss_host, "f32", "loss_host"), _hp(gradnorm_host, "f32", "gradnorm_host"),
                                                _stream()))
+
+    def set_graph_replay(self, enable: bool):
+        self._ck(self.lib.tgnn_set_graph_replay(self._h, int(enable)))
 
     # ---- debug ----
     def debug_get_grads(self, grads_out):

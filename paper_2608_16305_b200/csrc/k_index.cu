@@ -140,6 +140,35 @@ __global__ void make_roots_kernel(const int32_t* __restrict__ q_src, const int32
   r_time[i] = q_t[j];
 }
 
+// Copies one step's event arrays into the context's fixed staging buffers (so that the rest of the
+// step always sees the same addresses).  Sources equal to their destination are skipped.
+struct StageArgs {
+  const int32_t *u_src, *u_dst, *u_eid, *q_src, *q_dst, *q_neg;
+  const double *u_t, *q_t;
+  const uint8_t *u_keep, *mask;
+  int32_t *d_u_src, *d_u_dst, *d_u_eid, *d_q_src, *d_q_dst, *d_q_neg;
+  double *d_u_t, *d_q_t;
+  uint8_t *d_u_keep, *d_mask;
+  int n_u, n_q;
+};
+__global__ void __launch_bounds__(256) stage_inputs_kernel(StageArgs a) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < a.n_u) {
+    if (a.u_src != a.d_u_src) a.d_u_src[i] = a.u_src[i];
+    if (a.u_dst != a.d_u_dst) a.d_u_dst[i] = a.u_dst[i];
+    if (a.u_eid != a.d_u_eid) a.d_u_eid[i] = a.u_eid[i];
+    if (a.u_t != a.d_u_t) a.d_u_t[i] = a.u_t[i];
+    if (a.u_keep && a.u_keep != a.d_u_keep) a.d_u_keep[i] = a.u_keep[i];
+  }
+  if (i < a.n_q) {
+    if (a.q_src != a.d_q_src) a.d_q_src[i] = a.q_src[i];
+    if (a.q_dst != a.d_q_dst) a.d_q_dst[i] = a.q_dst[i];
+    if (a.q_neg != a.d_q_neg) a.d_q_neg[i] = a.q_neg[i];
+    if (a.q_t != a.d_q_t) a.d_q_t[i] = a.q_t[i];
+    if (a.mask && a.mask != a.d_mask) a.d_mask[i] = a.mask[i];
+  }
+}
+
 // ---------------------------------------------------------------- step (3) --
 // fp64 -> uint64 preserving order (0 is left free as "empty" for every finite value)
 __device__ __forceinline__ unsigned long long orderable(double x) {
@@ -271,6 +300,23 @@ int launch_sample_recent(tgnn_ctx* ctx, const int32_t* nodes, const double* time
         ctx->indptr, ctx->g_nbr, ctx->g_eid, ctx->g_ts, nodes, times, n, ctx->cfg.k, nbr_out, eid_out, ts_out, cnt_out);
   }
   TGNN_LAUNCH_OK(ctx, "sample_recent");
+  return TGNN_OK;
+}
+
+int launch_stage_inputs(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, const double* u_t,
+                        const int32_t* u_eid, const uint8_t* u_keep, int n_u, const int32_t* q_src, const int32_t* q_dst,
+                        const int32_t* q_neg, const double* q_t, int n_q, const uint8_t* loss_mask, cudaStream_t s) {
+  const int n = n_u > n_q ? n_u : n_q;
+  if (n == 0) return TGNN_OK;
+  Workspace& w = ctx->ws;
+  StageArgs a = {u_src, u_dst, u_eid, q_src, q_dst, q_neg, u_t, q_t, u_keep, loss_mask,
+                 w.st_u_src, w.st_u_dst, w.st_u_eid, w.st_q_src, w.st_q_dst, w.st_q_neg, w.st_u_t, w.st_q_t,
+                 w.st_u_keep, w.st_mask, n_u, n_q};
+  {
+    KernelScope scope__(ctx, "stage_inputs", s);
+    stage_inputs_kernel<<<(n + 255) / 256, 256, 0, s>>>(a);
+  }
+  TGNN_LAUNCH_OK(ctx, "stage_inputs");
   return TGNN_OK;
 }
 

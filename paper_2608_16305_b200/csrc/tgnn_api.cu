@@ -215,8 +215,10 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
     return TGNN_ECUDA;
   }
   ctx->ev_next = 0;
+  ctx->n_graphs = 0;
+  ctx->graphs_enabled = 1;
   for (int i = 0; ok && i < 2; ++i) ok = cudaStreamCreateWithFlags(&ctx->side[i], cudaStreamNonBlocking) == cudaSuccess;
-  for (int i = 0; ok && i < 16; ++i) ok = cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; ok && i < 32; ++i) ok = cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     cudaFree(ctx->arena);
@@ -235,8 +237,10 @@ int tgnn_destroy(tgnn_ctx* ctx) {
     cudaEventDestroy(e.a);
     cudaEventDestroy(e.b);
   }
+  for (int i = 0; i < ctx->n_graphs; ++i)
+    if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
   for (int i = 0; i < 2; ++i) cudaStreamDestroy(ctx->side[i]);
-  for (int i = 0; i < 16; ++i) cudaEventDestroy(ctx->ev[i]);
+  for (int i = 0; i < 32; ++i) cudaEventDestroy(ctx->ev[i]);
   cudaFree(ctx->arena);
   delete ctx;
   return TGNN_OK;
@@ -357,14 +361,11 @@ int tgnn_backward_step(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* 
   return rc;
 }
 
-int tgnn_train_step(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, const double* u_t, const int32_t* u_eid,
-                    const uint8_t* u_keep, int n_u, const int32_t* q_src, const int32_t* q_dst, const int32_t* q_neg,
-                    const double* q_t, int n_q, const uint8_t* loss_mask, float* loss_out, float* gradnorm_out,
-                    void* stream) {
-  if (!ctx) return TGNN_EINVAL;
-  NEED(ctx, n_u >= 0 && n_q >= 0, TGNN_EINVAL, "train_step: negative size");
-  NEED(ctx, n_q <= ctx->nq_cap, TGNN_ECAPACITY, "train_step: n_q %d > max_roots/3 = %d", n_q, ctx->nq_cap);
-  NEED(ctx, n_q == 0 || (q_src && q_dst && q_neg && q_t), TGNN_EINVAL, "train_step: null target arrays");
+namespace {
+
+// The launch sequence of one step on fixed (staging) input addresses.
+int step_body(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q, bool has_mask, float* loss_out, float* gradnorm_out,
+              void* stream) {
   Workspace& w = ctx->ws;
   int rc;
   ctx->have_update = false;
@@ -372,14 +373,15 @@ int tgnn_train_step(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, c
   cudaStream_t side = ctx->side[1];
   rc = fork_to(ctx, S(stream), side);
   if (rc) return rc;
-  rc = launch_make_roots(ctx, q_src, q_dst, q_neg, q_t, n_q, side);
+  rc = launch_make_roots(ctx, w.st_q_src, w.st_q_dst, w.st_q_neg, w.st_q_t, n_q, side);
   if (rc) return rc;
   rc = tgnn_sample_recent(ctx, w.r_node, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, w.nb_cnt, side);
   if (rc) return rc;
   if (n_u > 0) {
-    rc = tgnn_build_messages(ctx, u_src, u_dst, u_t, u_eid, u_keep, n_u, nullptr, w.msg_node, stream);
+    rc = tgnn_build_messages(ctx, w.st_u_src, w.st_u_dst, w.st_u_t, w.st_u_eid, has_keep ? w.st_u_keep : nullptr, n_u,
+                             nullptr, w.msg_node, stream);
     if (rc) return rc;
-    rc = tgnn_reduce_latest(ctx, w.msg_node, u_t, u_eid, 2 * n_u, w.uniq, w.winner, w.n_uniq, stream);
+    rc = tgnn_reduce_latest(ctx, w.msg_node, w.st_u_t, w.st_u_eid, 2 * n_u, w.uniq, w.winner, w.n_uniq, stream);
     if (rc) return rc;
     rc = tgnn_memory_update(ctx, nullptr, w.uniq, w.winner, w.n_uniq, stream);
     if (rc) return rc;
@@ -388,7 +390,96 @@ int tgnn_train_step(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, c
   if (rc) return rc;
   rc = tgnn_embed(ctx, w.r_node, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, w.nb_cnt, w.h, stream);
   if (rc) return rc;
-  return tgnn_backward_step(ctx, n_q, loss_mask, loss_out, gradnorm_out, stream);
+  return tgnn_backward_step(ctx, n_q, has_mask ? w.st_mask : nullptr, loss_out, gradnorm_out, stream);
+}
+
+// Host-side bookkeeping that step_body leaves behind, reproduced after a graph replay.
+void after_replay(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q) {
+  Workspace& w = ctx->ws;
+  ctx->m_src = w.st_u_src; ctx->m_dst = w.st_u_dst; ctx->m_t = w.st_u_t; ctx->m_eid = w.st_u_eid;
+  ctx->m_keep = has_keep ? w.st_u_keep : nullptr; ctx->m_n = n_u;
+  ctx->upd_n_uniq = w.n_uniq;
+  ctx->upd_cap = ctx->U_cap < 2 * n_u ? ctx->U_cap : 2 * n_u;
+  ctx->e_nodes = w.r_node; ctx->e_times = w.r_time; ctx->e_nbr = w.nb_node; ctx->e_eid = w.nb_eid;
+  ctx->e_ts = w.nb_ts; ctx->e_cnt = w.nb_cnt; ctx->e_n = 3 * n_q; ctx->e_h = w.h;
+  ctx->have_embed = false; ctx->have_update = false;
+}
+
+}  // namespace
+
+int tgnn_set_graph_replay(tgnn_ctx* ctx, int enable) {
+  if (!ctx) return TGNN_EINVAL;
+  ctx->graphs_enabled = enable ? 1 : 0;
+  return TGNN_OK;
+}
+
+int tgnn_train_step(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, const double* u_t, const int32_t* u_eid,
+                    const uint8_t* u_keep, int n_u, const int32_t* q_src, const int32_t* q_dst, const int32_t* q_neg,
+                    const double* q_t, int n_q, const uint8_t* loss_mask, float* loss_out, float* gradnorm_out,
+                    void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, n_u >= 0 && n_q >= 0, TGNN_EINVAL, "train_step: negative size");
+  NEED(ctx, n_u <= ctx->cfg.max_events, TGNN_ECAPACITY, "train_step: n_u %d > max_events %d", n_u, ctx->cfg.max_events);
+  NEED(ctx, n_q <= ctx->nq_cap, TGNN_ECAPACITY, "train_step: n_q %d > max_roots/3 = %d", n_q, ctx->nq_cap);
+  NEED(ctx, n_u == 0 || (u_src && u_dst && u_t && u_eid), TGNN_EINVAL, "train_step: null update arrays");
+  NEED(ctx, n_q == 0 || (q_src && q_dst && q_neg && q_t), TGNN_EINVAL, "train_step: null target arrays");
+  NEED(ctx, ctx->memory && ctx->indptr, TGNN_ESTATE, "train_step: tgnn_set_state / tgnn_set_graph have not been called");
+  const bool has_keep = n_u > 0 && u_keep != nullptr, has_mask = n_q > 0 && loss_mask != nullptr;
+  int rc = launch_stage_inputs(ctx, u_src, u_dst, u_t, u_eid, u_keep, n_u, q_src, q_dst, q_neg, q_t, n_q, loss_mask,
+                               S(stream));
+  if (rc) return rc;
+  if (!ctx->graphs_enabled || ctx->prof.on)
+    return step_body(ctx, n_u, has_keep, n_q, has_mask, loss_out, gradnorm_out, stream);
+
+  tgnn_ctx::StepGraph* e = nullptr;
+  for (int i = 0; i < ctx->n_graphs; ++i) {
+    tgnn_ctx::StepGraph& c = ctx->graphs[i];
+    if (c.n_u == n_u && c.n_q == n_q && c.has_keep == (int)has_keep && c.has_mask == (int)has_mask &&
+        c.loss_out == loss_out && c.gradnorm_out == gradnorm_out) { e = &c; break; }
+  }
+  if (!e) {
+    if (ctx->n_graphs == 8) return step_body(ctx, n_u, has_keep, n_q, has_mask, loss_out, gradnorm_out, stream);
+    e = &ctx->graphs[ctx->n_graphs++];
+    *e = tgnn_ctx::StepGraph{n_u, n_q, (int)has_keep, (int)has_mask, loss_out, gradnorm_out, 0, 0, nullptr};
+  }
+  if (e->exec) {
+    TGNN_CUDA_OK(ctx, cudaGraphLaunch(e->exec, S(stream)));
+    ctx->launches += e->kernels;
+    after_replay(ctx, n_u, has_keep, n_q);
+    return TGNN_OK;
+  }
+  if (e->seen++ == 0)  // first time: plain launches (also performs one-time kernel attribute set-up)
+    return step_body(ctx, n_u, has_keep, n_q, has_mask, loss_out, gradnorm_out, stream);
+  // second time: record the launches into a graph, then run it
+  if (cudaStreamBeginCapture(S(stream), cudaStreamCaptureModeRelaxed) != cudaSuccess) {
+    cudaGetLastError();  // e.g. the legacy default stream cannot capture: stay with plain launches
+    ctx->graphs_enabled = 0;
+    return step_body(ctx, n_u, has_keep, n_q, has_mask, loss_out, gradnorm_out, stream);
+  }
+  const int64_t l0 = ctx->launches;
+  rc = step_body(ctx, n_u, has_keep, n_q, has_mask, loss_out, gradnorm_out, stream);
+  cudaGraph_t graph = nullptr;
+  const cudaError_t ce = cudaStreamEndCapture(S(stream), &graph);
+  if (rc != TGNN_OK || ce != cudaSuccess || !graph) {
+    cudaGetLastError();
+    if (graph) cudaGraphDestroy(graph);
+    ctx->graphs_enabled = 0;
+    if (rc != TGNN_OK) return rc;
+    return set_error(ctx, TGNN_ECUDA, "train_step: stream capture failed: %s", cudaGetErrorString(ce));
+  }
+  e->kernels = ctx->launches - l0;
+  cudaGraphExec_t exec = nullptr;
+  const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (ie != cudaSuccess || !exec) {
+    cudaGetLastError();
+    ctx->graphs_enabled = 0;
+    return set_error(ctx, TGNN_ECUDA, "train_step: graph instantiation failed: %s", cudaGetErrorString(ie));
+  }
+  e->exec = exec;
+  TGNN_CUDA_OK(ctx, cudaGraphLaunch(e->exec, S(stream)));
+  after_replay(ctx, n_u, has_keep, n_q);
+  return TGNN_OK;
 }
 
 int tgnn_train_step_host(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, const double* u_t,

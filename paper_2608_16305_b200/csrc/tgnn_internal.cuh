@@ -136,8 +136,21 @@ struct tgnn_ctx {
   // products, the neighbor search next to the memory update, ...).  They are forked from and joined
   // back into the caller's stream with events, so the caller still sees one ordered stream of work.
   cudaStream_t side[2];
-  cudaEvent_t ev[16];
+  cudaEvent_t ev[32];
   int ev_next;
+  // Replay of a whole training step as a CUDA graph: tgnn_train_step copies its inputs into the
+  // fixed staging buffers and, for a shape signature it has already run once, captures the launch
+  // sequence on the caller's stream and replays it from then on.
+  struct StepGraph {
+    int n_u, n_q, has_keep, has_mask;
+    float *loss_out, *gradnorm_out;
+    int seen;
+    int64_t kernels;
+    cudaGraphExec_t exec;
+  };
+  StepGraph graphs[8];
+  int n_graphs;
+  int graphs_enabled;
   int64_t launches;
   tgnn::Profiler prof;
   char err[256];
@@ -161,7 +174,7 @@ int set_error(tgnn_ctx* ctx, int code, const char* fmt, ...);
 // side[i] waits for everything enqueued so far on `from`.
 inline int fork_to(tgnn_ctx* ctx, cudaStream_t from, cudaStream_t to) {
   cudaEvent_t e = ctx->ev[ctx->ev_next];
-  ctx->ev_next = (ctx->ev_next + 1) % 16;
+  ctx->ev_next = (ctx->ev_next + 1) % 32;
   if (cudaEventRecord(e, from) != cudaSuccess || cudaStreamWaitEvent(to, e, 0) != cudaSuccess)
     return set_error(ctx, TGNN_ECUDA, "stream fork/join failed: %s", cudaGetErrorString(cudaGetLastError()));
   return TGNN_OK;
@@ -197,6 +210,9 @@ int launch_sample_recent(tgnn_ctx* ctx, const int32_t* nodes, const double* time
                          int32_t* eid_out, double* ts_out, int32_t* cnt_out, cudaStream_t s);
 int launch_reduce_latest(tgnn_ctx* ctx, const int32_t* msg_node, const double* t, const int32_t* eid, int n_msg,
                          int32_t* uniq_out, int32_t* winner_out, int32_t* n_uniq_out, cudaStream_t s);
+int launch_stage_inputs(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, const double* u_t,
+                        const int32_t* u_eid, const uint8_t* u_keep, int n_u, const int32_t* q_src, const int32_t* q_dst,
+                        const int32_t* q_neg, const double* q_t, int n_q, const uint8_t* loss_mask, cudaStream_t s);
 int launch_make_roots(tgnn_ctx* ctx, const int32_t* q_src, const int32_t* q_dst, const int32_t* q_neg,
                       const double* q_t, int n_q, cudaStream_t s);
 

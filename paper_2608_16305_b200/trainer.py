@@ -84,6 +84,20 @@ class Trainer:
         self.lib.set_state(self.memory, self.last_update, self.params, self.adam_m, self.adam_v, self.step_count)
         self.prune_seed = cfg.seed
         self.drop_q32 = 1 << 31
+        # The library replays a step as a CUDA graph, which it records by stream capture; the legacy
+        # default stream cannot capture, so when the caller is on it the step runs on this stream,
+        # ordered after / before the caller's stream with events.
+        self.stream = torch.cuda.Stream(device=dev)
+
+    def _run(self, fn):
+        cur = torch.cuda.current_stream()
+        if cur != torch.cuda.default_stream():
+            return fn()
+        self.stream.wait_stream(cur)
+        with torch.cuda.stream(self.stream):
+            out = fn()
+        cur.wait_stream(self.stream)
+        return out
 
     def prune(self, b: int):
         dw = self.dw
@@ -95,6 +109,9 @@ class Trainer:
 
     def step(self, b: int, with_update: bool = True):
         """One training step on batch b (device-resident inputs)."""
+        return self._run(lambda: self._step(b, with_update))
+
+    def _step(self, b: int, with_update: bool):
         dw = self.dw
         self.prune(b)
         q = dw.target_slice(b)

@@ -90,6 +90,7 @@ class Rig:
     def gpu_gates(self, b):
         q = self.dw.target_slice(b)
         nq = q.stop - q.start
+        torch.cuda.synchronize()
         hg = torch.zeros((3 * nq, self.cfg.d), dtype=torch.uint8, device="cuda")
         dg = torch.zeros((2 * nq, self.cfg.d), dtype=torch.uint8, device="cuda")
         self.tr.lib.debug_get_gates(hg, dg)
