@@ -100,45 +100,66 @@ __global__ void __launch_bounds__(256) dh_kernel(const float* __restrict__ dcat1
   }
 }
 
-// One warp per root: backward of the weighted sum, the softmax and the scaled dot products.
+// One warp per root: backward of the weighted sum, the softmax and the scaled dot products, on the
+// root's K | V rows staged in shared memory.  Lane p < H*k owns the (head, slot) pair p for the
+// probability and logit gradients; afterwards the lanes own columns and write dQ and the dK | dV rows.
 __global__ void __launch_bounds__(256) attention_bwd_kernel(const float* __restrict__ Q, const float* __restrict__ KV,
                                                             const float* __restrict__ alpha,
                                                             const float* __restrict__ dcat_o,
                                                             const int32_t* __restrict__ cnt, int n, int d, int H, int k,
                                                             float* __restrict__ dQ, float* __restrict__ dKV) {
-  extern __shared__ float sm[];
+  extern __shared__ __align__(16) float sm[];
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   const int i = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
   if (i >= n) return;
-  float* dl = sm + wib * H * k;  // d loss / d logit (already scaled)
+  float* Ks = sm + wib * attn_warp_floats(d, H, k);
+  float* Vs = Ks + k * d;
+  float* Qs = Vs + k * d;
+  float* das = Qs + d;       // d loss / d a
+  float* al = das + d;       // probabilities
+  float* dal = al + H * k;   // d loss / d probability
+  float* dl = dal + H * k;   // d loss / d logit, already scaled
   const int dh = d / H;
   const int c = cnt[i];
   const float scale = rsqrtf((float)dh);
-  const float* da = dcat_o + (int64_t)i * 2 * d;
-  const float* al = alpha + (int64_t)i * H * k;
-  for (int h = 0; h < H; ++h) {
-    float dot = 0.f;
-    for (int s = 0; s < c; ++s) {
-      const float* vr = KV + ((int64_t)i * k + s) * 2 * d + d + h * dh;
-      float a = 0.f;
-      for (int e = lane; e < dh; e += 32) a = fmaf(da[h * dh + e], vr[e], a);
-      for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(FULL, a, o);
-      if (lane == 0) dl[h * k + s] = a;
-      dot = fmaf(al[h * k + s], a, dot);
-    }
-    __syncwarp();
-    if (lane < c) dl[h * k + lane] = al[h * k + lane] * (dl[h * k + lane] - dot) * scale;
-    __syncwarp();
+  attn_stage(Ks, Vs, Qs, Q, KV, i, c, d, k, lane);
+  {
+    const float4* g4 = reinterpret_cast<const float4*>(dcat_o + (int64_t)i * 2 * d);
+    for (int e = lane; e < (d >> 2); e += 32) reinterpret_cast<float4*>(das)[e] = __ldg(g4 + e);
+    for (int p = lane; p < H * k; p += 32) al[p] = alpha[(int64_t)i * H * k + p];
   }
+  __syncwarp();
+  for (int p = lane; p < H * k; p += 32) {
+    const int h = p / k, s = p - h * k;
+    float a = 0.f;
+    if (s < c) {
+      const float* vr = Vs + s * d + h * dh;
+      const float* gr = das + h * dh;
+      for (int e = 0; e < dh; ++e) a = fmaf(gr[e], vr[e], a);
+    }
+    dal[p] = a;
+  }
+  __syncwarp();
+  for (int p = lane; p < H * k; p += 32) {
+    const int h = p / k, s = p - h * k;
+    float g = 0.f;
+    if (s < c) {
+      float dot = 0.f;
+      for (int t = 0; t < c; ++t) dot = fmaf(al[h * k + t], dal[h * k + t], dot);
+      g = al[p] * (dal[p] - dot) * scale;
+    }
+    dl[p] = g;
+  }
+  __syncwarp();
   for (int e = lane; e < d; e += 32) {
     const int h = e / dh;
-    const float qe = Q[(int64_t)i * d + e], dae = da[e];
+    const float qe = Qs[e], dae = das[e];
     float dq = 0.f;
     for (int s = 0; s < k; ++s) {
       float* row = dKV + ((int64_t)i * k + s) * 2 * d;
       if (s < c) {
         const float g = dl[h * k + s];
-        dq = fmaf(g, KV[((int64_t)i * k + s) * 2 * d + e], dq);
+        dq = fmaf(g, Ks[s * d + e], dq);
         row[e] = g * qe;
         row[d + e] = al[h * k + s] * dae;
       } else {
@@ -232,12 +253,6 @@ __global__ void __launch_bounds__(256) time_grad_kernel(const float* __restrict_
   }
 }
 
-// Rounds the fp64 time-encoder sums into the fp32 gradient vector (time_w and time_b are adjacent).
-__global__ void time_grad_finish_kernel(const double* __restrict__ acc, int n, float* __restrict__ g_time) {
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c < n) g_time[c] = (float)acc[c];
-}
-
 // Backward of the GRU gates for the rows the memory update wrote.
 __global__ void __launch_bounds__(256) gru_bwd_gate_kernel(const float* __restrict__ dMemU, const float* __restrict__ X,
                                                            int ld, int d, const float* __restrict__ g_r,
@@ -266,14 +281,25 @@ __global__ void __launch_bounds__(256) gru_bwd_gate_kernel(const float* __restri
 
 // Sum of squares of the gradient; the last block to finish turns it into g_r, bumps the Adam
 // step counter and prepares the bias corrections.
-__global__ void __launch_bounds__(256) gradnorm_kernel(const float* __restrict__ grads, int64_t P, double* red,
+// The time-encoder entries [t_off, t_off + t_n) are taken from their fp64 sums tg_acc (rounded once)
+// and written back into grads by block 0, so the update kernel finds them there.
+__global__ void __launch_bounds__(256) gradnorm_kernel(float* __restrict__ grads, int64_t P,
+                                                       const double* __restrict__ tg_acc, int64_t t_off, int t_n,
+                                                       double* red,
                                                        unsigned int* ticket, int64_t* step, float beta1, float beta2,
                                                        float* __restrict__ adam_sc, const float* __restrict__ loss_acc,
                                                        float* scalars, float* loss_out, float* gradnorm_out) {
   __shared__ double s_part[8];
   double acc = 0.0;
   for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < P; e += (int64_t)gridDim.x * blockDim.x) {
-    const double g = (double)grads[e];
+    double g;
+    if (e >= t_off && e < t_off + t_n) {
+      const float gt = (float)tg_acc[e - t_off];
+      grads[e] = gt;  // same value from whichever block owns e
+      g = (double)gt;
+    } else {
+      g = (double)grads[e];
+    }
     acc = fma(g, g, acc);
   }
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(FULL, acc, o);
@@ -388,8 +414,10 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
   // are joined back before the gradient norm.
   cudaStream_t sa = ctx->side[0], sb = ctx->side[1];
   // grads | dMemU | red | tg_acc | st_scalars are contiguous in the arena: one memset clears them all
-  const size_t zero_bytes = (size_t)((char*)(w.st_scalars + 4) - (char*)w.grads);
-  TGNN_CUDA_OK(ctx, cudaMemsetAsync(w.grads, 0, zero_bytes, s));
+  if (!ctx->grads_zeroed) {
+    const size_t zero_bytes = (size_t)((char*)(w.st_scalars + 4) - (char*)w.grads);
+    TGNN_CUDA_OK(ctx, cudaMemsetAsync(w.grads, 0, zero_bytes, s));
+  }
 
   if (n_q > 0) {
     const int64_t tot = (int64_t)2 * n_q * 2 * d;
@@ -422,10 +450,18 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     RC(fork_to(ctx, s, sb));
     RC(grad_w(ctx, w.dpre_o, d, w.cat_o, 2 * d, R, nullptr, d, 2 * d, G + L.wo, G + L.bo, "dW_o", sb));
     RC(grad_in(ctx, w.dpre_o, d, P + L.wo, 2 * d, 0, R, nullptr, d, 2 * d, w.dcat_o, 2 * d, "dcat_o", s));
-    const int wpb = 8;
+    const int wpb = attn_warps_per_block(d, H, k);
+    {
+      static int attr_bytes = 0;
+      const int need = (int)attn_smem_bytes(d, H, k, wpb);
+      if (attr_bytes < need) {
+        TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(attention_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, need));
+        attr_bytes = need;
+      }
+    }
     {
       KernelScope scope__(ctx, "attention_bwd", s);
-      attention_bwd_kernel<<<(R + wpb - 1) / wpb, wpb * 32, wpb * H * k * sizeof(float), s>>>(
+      attention_bwd_kernel<<<(R + wpb - 1) / wpb, wpb * 32, attn_smem_bytes(d, H, k, wpb), s>>>(
           w.Q, w.KV, w.alpha, w.dcat_o, ctx->e_cnt, R, d, H, k, w.dQ, w.dKV);
     }
     TGNN_LAUNCH_OK(ctx, "attention_bwd");
@@ -483,15 +519,10 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     }
     RC(fork_to(ctx, sa, s));  // join
     RC(fork_to(ctx, sb, s));
-    {
-      KernelScope scope__(ctx, "time_grad_finish", s);
-      time_grad_finish_kernel<<<(2 * d + 127) / 128, 128, 0, s>>>(w.tg_acc, 2 * d, G + L.time_w);
-    }
-    TGNN_LAUNCH_OK(ctx, "time_grad_finish");
   }
   {
     KernelScope scope__(ctx, "gradnorm", s);
-    gradnorm_kernel<<<148, 256, 0, s>>>(G, L.total, w.red, w.counters, ctx->step, c.beta1, c.beta2, w.adam_sc,
+    gradnorm_kernel<<<148, 256, 0, s>>>(G, L.total, w.tg_acc, L.time_w, n_q > 0 ? 2 * d : 0, w.red, w.counters, ctx->step, c.beta1, c.beta2, w.adam_sc,
                                         w.st_scalars, w.st_scalars + 2, loss_out, gradnorm_out);
   }
   TGNN_LAUNCH_OK(ctx, "gradnorm");

@@ -2,10 +2,18 @@
 #include "tgnn_internal.cuh"
 #include "tgnn_device.cuh"
 
+// Raises a kernel's dynamic shared-memory limit once (the attention kernels stage > 48 KB per block).
+#define RC_ATTR(ctx, kernel, bytes)                                                                                   \
+  do {                                                                                                                \
+    static int done__ = 0;                                                                                            \
+    if (done__ < (int)(bytes)) {                                                                                      \
+      TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(bytes)));     \
+      done__ = (int)(bytes);                                                                                          \
+    }                                                                                                                 \
+  } while (0)
+
 namespace tgnn {
 namespace {
-
-constexpr unsigned FULL = 0xffffffffu;
 
 // One warp per row.  Rows [0, n*k): neighbor rows z = [m_nbr || x_eid || Phi(t - ts)] (zero if the slot
 // is empty).  Rows [n*k, n*k + n): per root, z_q = [m_root || Phi(0)] and the memory half of cat_o.
@@ -49,44 +57,55 @@ __global__ void __launch_bounds__(256) gather_z_kernel(const float* __restrict__
   }
 }
 
-// One warp per root: logits, softmax over the valid slots, weighted sum of V into cat_o[:, :d].
-// Dynamic shared memory: warps_per_block * H * k floats.
+// One warp per root.  Lane p < H*k owns the (head, slot) pair p: it forms the scaled dot product
+// from shared memory, then the softmax over the head's valid slots; afterwards the lanes own output
+// columns and accumulate the weighted sum of V into cat_o[:, :d].
 __global__ void __launch_bounds__(256) attention_fwd_kernel(const float* __restrict__ Q, const float* __restrict__ KV,
                                                             const int32_t* __restrict__ cnt, int n, int d, int H, int k,
                                                             float* __restrict__ alpha, float* __restrict__ cat_o) {
-  extern __shared__ float sm[];
+  extern __shared__ __align__(16) float sm[];
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   const int i = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
   if (i >= n) return;
-  float* al = sm + wib * H * k;
+  float* Ks = sm + wib * attn_warp_floats(d, H, k);
+  float* Vs = Ks + k * d;
+  float* Qs = Vs + k * d;
+  float* al = Qs + 2 * d;  // logits
+  float* pr = al + H * k;  // probabilities
   const int dh = d / H;
   const int c = cnt[i];
   const float scale = rsqrtf((float)dh);
-  const float* q = Q + (int64_t)i * d;
-  for (int h = 0; h < H; ++h) {
-    float mx = -INFINITY;
-    for (int s = 0; s < c; ++s) {
-      const float* kr = KV + ((int64_t)i * k + s) * 2 * d + h * dh;
-      float a = 0.f;
-      for (int e = lane; e < dh; e += 32) a = fmaf(q[h * dh + e], kr[e], a);
-      for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(FULL, a, o);
+  attn_stage(Ks, Vs, Qs, Q, KV, i, c, d, k, lane);
+  __syncwarp();
+  for (int p = lane; p < H * k; p += 32) {
+    const int h = p / k, s = p - h * k;
+    float a = 0.f;
+    if (s < c) {
+      const float* kr = Ks + s * d + h * dh;
+      const float* qr = Qs + h * dh;
+      for (int e = 0; e < dh; ++e) a = fmaf(qr[e], kr[e], a);
       a *= scale;
-      if (lane == 0) al[h * k + s] = a;
-      mx = fmaxf(mx, a);
     }
-    __syncwarp();
-    float den = 0.f;
-    for (int s = 0; s < c; ++s) den += expf(al[h * k + s] - mx);
-    __syncwarp();
-    if (lane < c) al[h * k + lane] = expf(al[h * k + lane] - mx) / den;
-    if (lane >= c && lane < k) al[h * k + lane] = 0.f;
-    __syncwarp();
-    if (lane < k) alpha[((int64_t)i * H + h) * k + lane] = al[h * k + lane];
+    al[p] = a;
   }
+  __syncwarp();
+  for (int p = lane; p < H * k; p += 32) {
+    const int h = p / k, s = p - h * k;
+    float out = 0.f;
+    if (s < c) {
+      float mx = -INFINITY, den = 0.f;
+      for (int t = 0; t < c; ++t) mx = fmaxf(mx, al[h * k + t]);
+      for (int t = 0; t < c; ++t) den += expf(al[h * k + t] - mx);
+      out = expf(al[p] - mx) / den;
+    }
+    pr[p] = out;
+    alpha[(int64_t)i * H * k + p] = out;
+  }
+  __syncwarp();
   for (int e = lane; e < d; e += 32) {
     const int h = e / dh;
     float a = 0.f;
-    for (int s = 0; s < c; ++s) a = fmaf(al[h * k + s], KV[((int64_t)i * k + s) * 2 * d + d + e], a);
+    for (int s = 0; s < c; ++s) a = fmaf(pr[h * k + s], Vs[s * d + e], a);
     cat_o[(int64_t)i * 2 * d + e] = a;
   }
 }
@@ -125,10 +144,11 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
   if (rc) return rc;
   rc = fork_to(ctx, ctx->side[0], s);
   if (rc) return rc;
-  const int wpb = 8;
+  const int wpb = attn_warps_per_block(d, H, k);
+  RC_ATTR(ctx, attention_fwd_kernel, attn_smem_bytes(d, H, k, wpb));
   {
     KernelScope scope__(ctx, "attention_fwd", s);
-    attention_fwd_kernel<<<(n + wpb - 1) / wpb, wpb * 32, wpb * H * k * sizeof(float), s>>>(w.Q, w.KV, cnt, n, d, H, k,
+    attention_fwd_kernel<<<(n + wpb - 1) / wpb, wpb * 32, attn_smem_bytes(d, H, k, wpb), s>>>(w.Q, w.KV, cnt, n, d, H, k,
                                                                                            w.alpha, w.cat_o);
   }
   TGNN_LAUNCH_OK(ctx, "attention_fwd");

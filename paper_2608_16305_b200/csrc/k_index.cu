@@ -193,7 +193,19 @@ __device__ __forceinline__ unsigned long long peer_max(unsigned peers, unsigned 
 // per-node tables (time first, then eid/role among the messages that tie on
 // time); a hub's thousands of messages are pre-reduced inside each warp.
 // Then the touched nodes are compacted in ascending id order by a block scan.
+// msg_node may be null: the node of message j is then read from the event arrays (src for role 0,
+// dst for role 1, none if keep[j>>1] == 0), which saves materialising it.
+__device__ __forceinline__ int message_node(const int32_t* __restrict__ msg_node, const int32_t* __restrict__ src,
+                                            const int32_t* __restrict__ dst, const uint8_t* __restrict__ keep, int j) {
+  if (msg_node) return msg_node[j];
+  if (keep && !keep[j >> 1]) return -1;
+  return (j & 1) ? dst[j >> 1] : src[j >> 1];
+}
+
 __global__ void __launch_bounds__(1024) reduce_latest_kernel(const int32_t* __restrict__ msg_node,
+                                                             const int32_t* __restrict__ ev_src,
+                                                             const int32_t* __restrict__ ev_dst,
+                                                             const uint8_t* __restrict__ ev_keep,
                                                              const double* __restrict__ t,
                                                              const int32_t* __restrict__ eid, int n_msg, int N,
                                                              unsigned long long* best_t, unsigned long long* best_id,
@@ -209,7 +221,7 @@ __global__ void __launch_bounds__(1024) reduce_latest_kernel(const int32_t* __re
   for (int i = tid; i < pn; i += blockDim.x) node2slot[prev_uniq[i]] = -1;
   const int n_round = (n_msg + 31) / 32 * 32;
   for (int j = tid; j < n_round; j += blockDim.x) {
-    const int node = j < n_msg ? msg_node[j] : -1;
+    const int node = j < n_msg ? message_node(msg_node, ev_src, ev_dst, ev_keep, j) : -1;
     const bool v = node >= 0;
     const unsigned act = __ballot_sync(FULL, v);
     if (v) {
@@ -220,7 +232,7 @@ __global__ void __launch_bounds__(1024) reduce_latest_kernel(const int32_t* __re
   }
   __syncthreads();
   for (int j = tid; j < n_round; j += blockDim.x) {
-    const int node = j < n_msg ? msg_node[j] : -1;
+    const int node = j < n_msg ? message_node(msg_node, ev_src, ev_dst, ev_keep, j) : -1;
     const bool v = node >= 0 && orderable(t[j >> 1]) == best_t[node];
     const unsigned act = __ballot_sync(FULL, v);
     if (v) {
@@ -232,7 +244,7 @@ __global__ void __launch_bounds__(1024) reduce_latest_kernel(const int32_t* __re
   }
   __syncthreads();
   for (int j = tid; j < n_msg; j += blockDim.x) {
-    const int node = msg_node[j];
+    const int node = message_node(msg_node, ev_src, ev_dst, ev_keep, j);
     if (node < 0) continue;
     const unsigned long long key = (((unsigned long long)(uint32_t)eid[j >> 1]) << 1 | (unsigned)(j & 1)) + 1ULL;
     if (orderable(t[j >> 1]) == best_t[node] && key == best_id[node]) win_msg[node] = j;
@@ -333,10 +345,17 @@ int launch_make_roots(tgnn_ctx* ctx, const int32_t* q_src, const int32_t* q_dst,
 
 int launch_reduce_latest(tgnn_ctx* ctx, const int32_t* msg_node, const double* t, const int32_t* eid, int n_msg,
                          int32_t* uniq_out, int32_t* winner_out, int32_t* n_uniq_out, cudaStream_t s) {
+  return launch_reduce_latest_events(ctx, msg_node, nullptr, nullptr, nullptr, t, eid, n_msg, uniq_out, winner_out,
+                                     n_uniq_out, s);
+}
+
+int launch_reduce_latest_events(tgnn_ctx* ctx, const int32_t* msg_node, const int32_t* src, const int32_t* dst,
+                                const uint8_t* keep, const double* t, const int32_t* eid, int n_msg, int32_t* uniq_out,
+                                int32_t* winner_out, int32_t* n_uniq_out, cudaStream_t s) {
   Workspace& w = ctx->ws;
   {
     KernelScope scope__(ctx, "reduce_latest", s);
-    reduce_latest_kernel<<<1, 1024, 0, s>>>(msg_node, t, eid, n_msg, (int)ctx->cfg.num_nodes, w.best_t, w.best_id,
+    reduce_latest_kernel<<<1, 1024, 0, s>>>(msg_node, src, dst, keep, t, eid, n_msg, (int)ctx->cfg.num_nodes, w.best_t, w.best_id,
                                             w.win_msg, w.node2slot, w.prev_uniq, w.prev_n_uniq, uniq_out, winner_out,
                                             n_uniq_out);
   }

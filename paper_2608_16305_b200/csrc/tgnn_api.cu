@@ -276,7 +276,7 @@ int tgnn_set_state(tgnn_ctx* ctx, float* memory, double* last_update, float* par
   NEED(ctx, memory && last_update && params && adam_m && adam_v && step, TGNN_EINVAL, "set_state: null pointer");
   ctx->memory = memory; ctx->last_update = last_update; ctx->params = params;
   ctx->adam_m = adam_m; ctx->adam_v = adam_v; ctx->step = step;
-  ctx->have_update = false; ctx->have_embed = false;
+  ctx->have_update = false; ctx->have_embed = false; ctx->grads_zeroed = false;
   return TGNN_OK;
 }
 
@@ -358,6 +358,7 @@ int tgnn_backward_step(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* 
   const int rc = launch_backward(ctx, n_q, loss_mask, loss_out, gradnorm_out, S(stream));
   ctx->have_embed = false;
   ctx->have_update = false;
+  ctx->grads_zeroed = false;
   return rc;
 }
 
@@ -373,15 +374,21 @@ int step_body(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q, bool has_mask, flo
   cudaStream_t side = ctx->side[1];
   rc = fork_to(ctx, S(stream), side);
   if (rc) return rc;
+  {  // clear the gradient block off the critical chain (grads | dMemU | red | tg_acc | scalars, contiguous)
+    const size_t zero_bytes = (size_t)((char*)(w.st_scalars + 4) - (char*)w.grads);
+    TGNN_CUDA_OK(ctx, cudaMemsetAsync(w.grads, 0, zero_bytes, side));
+    ctx->grads_zeroed = true;
+  }
   rc = launch_make_roots(ctx, w.st_q_src, w.st_q_dst, w.st_q_neg, w.st_q_t, n_q, side);
   if (rc) return rc;
   rc = tgnn_sample_recent(ctx, w.r_node, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, w.nb_cnt, side);
   if (rc) return rc;
   if (n_u > 0) {
-    rc = tgnn_build_messages(ctx, w.st_u_src, w.st_u_dst, w.st_u_t, w.st_u_eid, has_keep ? w.st_u_keep : nullptr, n_u,
-                             nullptr, w.msg_node, stream);
-    if (rc) return rc;
-    rc = tgnn_reduce_latest(ctx, w.msg_node, w.st_u_t, w.st_u_eid, 2 * n_u, w.uniq, w.winner, w.n_uniq, stream);
+    // messages stay virtual: the reduction reads the event arrays, the memory update gathers the winners
+    ctx->m_src = w.st_u_src; ctx->m_dst = w.st_u_dst; ctx->m_t = w.st_u_t; ctx->m_eid = w.st_u_eid;
+    ctx->m_keep = has_keep ? w.st_u_keep : nullptr; ctx->m_n = n_u;
+    rc = launch_reduce_latest_events(ctx, nullptr, w.st_u_src, w.st_u_dst, ctx->m_keep, w.st_u_t, w.st_u_eid, 2 * n_u,
+                                     w.uniq, w.winner, w.n_uniq, S(stream));
     if (rc) return rc;
     rc = tgnn_memory_update(ctx, nullptr, w.uniq, w.winner, w.n_uniq, stream);
     if (rc) return rc;
@@ -402,7 +409,7 @@ void after_replay(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q) {
   ctx->upd_cap = ctx->U_cap < 2 * n_u ? ctx->U_cap : 2 * n_u;
   ctx->e_nodes = w.r_node; ctx->e_times = w.r_time; ctx->e_nbr = w.nb_node; ctx->e_eid = w.nb_eid;
   ctx->e_ts = w.nb_ts; ctx->e_cnt = w.nb_cnt; ctx->e_n = 3 * n_q; ctx->e_h = w.h;
-  ctx->have_embed = false; ctx->have_update = false;
+  ctx->have_embed = false; ctx->have_update = false; ctx->grads_zeroed = false;
 }
 
 }  // namespace

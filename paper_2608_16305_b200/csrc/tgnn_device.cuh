@@ -46,4 +46,30 @@ __device__ __forceinline__ void warp_copy_feat(float* __restrict__ dst, const vo
   }
 }
 
+// ---- attention kernels: per-warp shared-memory staging --------------------------------------------
+// Floats one warp needs: K and V rows of the root's k slots, two d-vectors (query, upstream gradient)
+// and three H*k scratch vectors, rounded to whole 16-byte chunks.
+__host__ __device__ inline int attn_warp_floats(int d, int H, int k) { return 2 * k * d + 2 * d + ((3 * H * k + 3) & ~3); }
+inline int attn_warps_per_block(int d, int H, int k) {
+  const int per = attn_warp_floats(d, H, k) * 4;
+  int w = (200 * 1024) / per;
+  return w > 8 ? 8 : (w < 1 ? 1 : w);
+}
+inline size_t attn_smem_bytes(int d, int H, int k, int warps) { return (size_t)warps * attn_warp_floats(d, H, k) * 4; }
+
+// Stage the root's valid K | V rows and its query in shared memory with coalesced 128-bit loads.
+__device__ __forceinline__ void attn_stage(float* Ks, float* Vs, float* Qs, const float* __restrict__ Q,
+                                           const float* __restrict__ KV, int i, int c, int d, int k, int lane) {
+  const int d4 = d >> 2;
+  const float4* q4 = reinterpret_cast<const float4*>(Q + (int64_t)i * d);
+  for (int e = lane; e < d4; e += 32) reinterpret_cast<float4*>(Qs)[e] = __ldg(q4 + e);
+  const float4* kv4 = reinterpret_cast<const float4*>(KV + (int64_t)i * k * 2 * d);
+  for (int e = lane; e < c * 2 * d4; e += 32) {
+    const int s = e / (2 * d4), r = e - s * 2 * d4;
+    const float4 v = __ldg(kv4 + e);
+    if (r < d4) reinterpret_cast<float4*>(Ks + s * d)[r] = v;
+    else reinterpret_cast<float4*>(Vs + s * d)[r - d4] = v;
+  }
+}
+
 }  // namespace tgnn

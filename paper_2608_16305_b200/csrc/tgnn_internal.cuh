@@ -129,6 +129,7 @@ struct tgnn_ctx {
   const int32_t* upd_n_uniq;
   int upd_cap;
   bool have_update, have_embed;
+  bool grads_zeroed;  // tgnn_train_step cleared the gradient block ahead of the backward pass
   tgnn::Workspace ws;
   void* arena;
   size_t arena_bytes;
@@ -210,6 +211,9 @@ int launch_sample_recent(tgnn_ctx* ctx, const int32_t* nodes, const double* time
                          int32_t* eid_out, double* ts_out, int32_t* cnt_out, cudaStream_t s);
 int launch_reduce_latest(tgnn_ctx* ctx, const int32_t* msg_node, const double* t, const int32_t* eid, int n_msg,
                          int32_t* uniq_out, int32_t* winner_out, int32_t* n_uniq_out, cudaStream_t s);
+int launch_reduce_latest_events(tgnn_ctx* ctx, const int32_t* msg_node, const int32_t* src, const int32_t* dst,
+                                const uint8_t* keep, const double* t, const int32_t* eid, int n_msg, int32_t* uniq_out,
+                                int32_t* winner_out, int32_t* n_uniq_out, cudaStream_t s);
 int launch_stage_inputs(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, const double* u_t,
                         const int32_t* u_eid, const uint8_t* u_keep, int n_u, const int32_t* q_src, const int32_t* q_dst,
                         const int32_t* q_neg, const double* q_t, int n_q, const uint8_t* loss_mask, cudaStream_t s);
