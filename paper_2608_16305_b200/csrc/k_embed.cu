@@ -15,17 +15,22 @@
 namespace tgnn {
 namespace {
 
-// One warp per row.  Rows [0, n*k): neighbor rows z = [m_nbr || x_eid || Phi(t - ts)] (zero if the slot
-// is empty).  Rows [n*k, n*k + n): per root, z_q = [m_root || Phi(0)] and the memory half of cat_o.
-__global__ void __launch_bounds__(256) gather_z_kernel(const float* __restrict__ memory, const void* __restrict__ efeat,
-                                                       int feat_bf16, const float* __restrict__ time_w,
-                                                       const float* __restrict__ time_b, int d, int de, int k,
-                                                       const int32_t* __restrict__ nodes, const double* __restrict__ times,
-                                                       int n, const int32_t* __restrict__ nbr,
-                                                       const int32_t* __restrict__ eid, const double* __restrict__ ts,
-                                                       int ld, float* __restrict__ Z, float* __restrict__ z_dt,
-                                                       float* __restrict__ Zsin,
-                                                       float* __restrict__ Zq, float* __restrict__ cat_o) {
+// The attention inputs are gathered in two kernels.  The static part of a neighbor row z = [m_nbr ||
+// x_eid || Phi(t - ts)] -- edge features, time encoding and its sine -- depends only on the sampled
+// neighbors and the parameters, so it can run beside the memory update; the memory part has to wait
+// for it.  One warp per row in both.
+//
+// Static part.  Rows [0, n*k): columns [d, ld) of Z (zero row if the slot is empty), Zsin, z_dt.
+// Rows [n*k, n*k + n): the Phi(0) half of z_q.
+__global__ void __launch_bounds__(256) gather_z_static_kernel(const void* __restrict__ efeat, int feat_bf16,
+                                                              const float* __restrict__ time_w,
+                                                              const float* __restrict__ time_b, int d, int de, int k,
+                                                              const double* __restrict__ times, int n,
+                                                              const int32_t* __restrict__ nbr,
+                                                              const int32_t* __restrict__ eid,
+                                                              const double* __restrict__ ts, int ld,
+                                                              float* __restrict__ Z, float* __restrict__ z_dt,
+                                                              float* __restrict__ Zsin, float* __restrict__ Zq) {
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   const int nb_rows = n * k;
@@ -33,15 +38,13 @@ __global__ void __launch_bounds__(256) gather_z_kernel(const float* __restrict__
   for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < nb_rows + n; r += warps) {
     if (r < nb_rows) {
       float* row = Z + (int64_t)r * ld;
-      const int nb = nbr[r];
-      if (nb < 0) {
-        for (int q = lane; q < ld; q += 32) row[q] = 0.f;
+      if (nbr[r] < 0) {
+        for (int q = lane; q < ld; q += 32) row[q] = 0.f;  // the memory part too: nobody else writes this row
         for (int q = lane; q < d; q += 32) Zsin[(int64_t)r * d + q] = 0.f;
         if (lane == 0) z_dt[r] = 0.f;
         continue;
       }
       const float dtf = (float)(times[r / k] - ts[r]);
-      warp_copy_f32(row, memory + (int64_t)nb * d, d, lane);
       warp_copy_feat(row + d, efeat, feat_bf16, eid[r], de, lane);
       float* phi = row + d + de;
       for (int q = lane; q < d; q += 32) time_encode_sc(time_w[q], time_b[q], dtf, &phi[q], &Zsin[(int64_t)r * d + q]);
@@ -49,10 +52,30 @@ __global__ void __launch_bounds__(256) gather_z_kernel(const float* __restrict__
       if (lane == 0) z_dt[r] = dtf;
     } else {
       const int i = r - nb_rows;
+      for (int q = lane; q < d; q += 32) Zq[(int64_t)i * 2 * d + d + q] = time_encode(time_w[q], time_b[q], 0.f);
+    }
+  }
+}
+
+// Memory part.  Rows [0, n*k): columns [0, d) of Z for the valid slots.  Rows [n*k, n*k + n): the
+// memory half of z_q and of cat_o.
+__global__ void __launch_bounds__(256) gather_z_memory_kernel(const float* __restrict__ memory, int d, int k,
+                                                              const int32_t* __restrict__ nodes, int n,
+                                                              const int32_t* __restrict__ nbr, int ld,
+                                                              float* __restrict__ Z, float* __restrict__ Zq,
+                                                              float* __restrict__ cat_o) {
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  const int nb_rows = n * k;
+  for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < nb_rows + n; r += warps) {
+    if (r < nb_rows) {
+      const int nb = nbr[r];
+      if (nb >= 0) warp_copy_f32(Z + (int64_t)r * ld, memory + (int64_t)nb * d, d, lane);
+    } else {
+      const int i = r - nb_rows;
       const float* m = memory + (int64_t)nodes[i] * d;
       warp_copy_f32(Zq + (int64_t)i * 2 * d, m, d, lane);
       warp_copy_f32(cat_o + (int64_t)i * 2 * d + d, m, d, lane);
-      for (int q = lane; q < d; q += 32) Zq[(int64_t)i * 2 * d + d + q] = time_encode(time_w[q], time_b[q], 0.f);
     }
   }
 }
@@ -112,6 +135,23 @@ __global__ void __launch_bounds__(256) attention_fwd_kernel(const float* __restr
 
 }  // namespace
 
+int launch_embed_static(tgnn_ctx* ctx, const double* times, int n, const int32_t* nbr, const int32_t* eid,
+                        const double* ts, cudaStream_t s) {
+  if (n == 0) return TGNN_OK;
+  const tgnn_config& c = ctx->cfg;
+  const ParamLayout& L = ctx->L;
+  Workspace& w = ctx->ws;
+  const int rows = n * c.k + n;
+  {
+    KernelScope scope__(ctx, "gather_z_static", s);
+    gather_z_static_kernel<<<(rows + 7) / 8, 256, 0, s>>>(ctx->efeat, c.feat_dtype == TGNN_BF16, ctx->params + L.time_w,
+                                                          ctx->params + L.time_b, c.d, c.d_e, c.k, times, n, nbr, eid, ts,
+                                                          ctx->ld_kv, w.Z, w.z_dt, w.Zsin, w.Zq);
+  }
+  TGNN_LAUNCH_OK(ctx, "gather_z_static");
+  return TGNN_OK;
+}
+
 int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n, const int32_t* nbr,
                  const int32_t* eid, const double* ts, const int32_t* cnt, float* h_out, cudaStream_t s) {
   if (n == 0) return TGNN_OK;
@@ -120,13 +160,16 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
   Workspace& w = ctx->ws;
   const int d = c.d, k = c.k, H = c.heads;
   const int rows = n * k + n;
-  {
-    KernelScope scope__(ctx, "gather_z", s);
-    gather_z_kernel<<<(rows + 7) / 8, 256, 0, s>>>(ctx->memory, ctx->efeat, c.feat_dtype == TGNN_BF16,
-                                                   ctx->params + L.time_w, ctx->params + L.time_b, d, c.d_e, k, nodes,
-                                                   times, n, nbr, eid, ts, ctx->ld_kv, w.Z, w.z_dt, w.Zsin, w.Zq, w.cat_o);
+  if (!ctx->z_static_done) {
+    const int rc0 = launch_embed_static(ctx, times, n, nbr, eid, ts, s);
+    if (rc0) return rc0;
   }
-  TGNN_LAUNCH_OK(ctx, "gather_z");
+  ctx->z_static_done = false;
+  {
+    KernelScope scope__(ctx, "gather_z_memory", s);
+    gather_z_memory_kernel<<<(rows + 7) / 8, 256, 0, s>>>(ctx->memory, d, k, nodes, n, nbr, ctx->ld_kv, w.Z, w.Zq, w.cat_o);
+  }
+  TGNN_LAUNCH_OK(ctx, "gather_z_memory");
   GemmArgs g = {};
   g.A = w.Z; g.a_rs = ctx->ld_kv; g.a_cs = 1;
   g.B = ctx->params + L.wk; g.b_rs = 1; g.b_cs = L.dkv;  // rows of [W_k; W_v]

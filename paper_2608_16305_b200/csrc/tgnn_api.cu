@@ -383,6 +383,11 @@ int step_body(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q, bool has_mask, flo
   if (rc) return rc;
   rc = tgnn_sample_recent(ctx, w.r_node, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, w.nb_cnt, side);
   if (rc) return rc;
+  // edge features and time encodings of the sampled neighbors do not depend on memory either
+  NEED(ctx, ctx->cfg.d_e == 0 || ctx->efeat, TGNN_ESTATE, "train_step: tgnn_set_edge_features has not been called");
+  rc = launch_embed_static(ctx, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, side);
+  if (rc) return rc;
+  ctx->z_static_done = true;
   if (n_u > 0) {
     // messages stay virtual: the reduction reads the event arrays, the memory update gathers the winners
     ctx->m_src = w.st_u_src; ctx->m_dst = w.st_u_dst; ctx->m_t = w.st_u_t; ctx->m_eid = w.st_u_eid;

@@ -129,6 +129,7 @@ struct tgnn_ctx {
   const int32_t* upd_n_uniq;
   int upd_cap;
   bool have_update, have_embed;
+  bool z_static_done; // tgnn_train_step already gathered the memory-independent part of the attention inputs
   bool grads_zeroed;  // tgnn_train_step cleared the gradient block ahead of the backward pass
   tgnn::Workspace ws;
   void* arena;
@@ -229,6 +230,9 @@ int launch_memory_update(tgnn_ctx* ctx, const float* msg, const int32_t* uniq, c
 // ---- embedding (k_embed.cu) ----
 int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n, const int32_t* nbr,
                  const int32_t* eid, const double* ts, const int32_t* cnt, float* h_out, cudaStream_t s);
+
+int launch_embed_static(tgnn_ctx* ctx, const double* times, int n, const int32_t* nbr, const int32_t* eid,
+                        const double* ts, cudaStream_t s);
 
 // ---- backward + Adam (k_backward.cu) ----
 int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* loss_out, float* gradnorm_out,

@@ -59,18 +59,29 @@ class Rig:
         from paper_2608_16305_b200 import trainer
         self.B, self.oracle, self.cfg, self.math = B, oracle, cfg, math
         self.stream = wl.make_stream(cfg)
-        self.dw = trainer.DeviceWorkload(self.stream, batches=batches)
+        efeat_dev = None
+        self.compact = cfg.num_events * cfg.d_e > 2_000_000_000   # too big for a host copy: fetch rows per step
+        if cfg.num_events * cfg.d_e > 20_000_000:      # big table: generate it on the device (bit-identical)
+            efeat_dev = wl.edge_feature_table_torch(cfg, "cuda")
+            if not self.compact:
+                self.stream._efeat = self._to_host(efeat_dev)
+        self.efeat_dev = efeat_dev
+        self.dw = trainer.DeviceWorkload(self.stream, batches=batches, efeat=efeat_dev)
         self.weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed, bias_scale=bias_scale)
         mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST}[math]
         self.tr = trainer.Trainer(self.dw, self.weights, math_mode=mode, lr=lr)
         f32 = lambda x: float(np.float32(x))      # the library's configuration holds fp32 hyper-parameters
         self.ocfg = orc_cfg(oracle, cfg, lr=f32(lr), beta1=f32(0.9), beta2=f32(0.999), eps=f32(1e-8))
         self.graph = (self.stream.indptr, self.stream.nbr, self.stream.eid, self.stream.ts)
-        self.efeat = self.stream.efeat() if cfg.d_e else None
+        self.efeat = self.stream.efeat() if (cfg.d_e and not self.compact) else None
         self.lay = B.param_layout(self.tr.tcfg)
         self.shapes = wl.param_shapes(cfg.d, cfg.d_e)
         key = math + ("_bf16" if cfg.feat_dtype == "bf16" and math != "fp32" else "")
         self.tol = TOL[key]
+
+    def _to_host(self, t):
+        host = t.cpu()
+        return host.view(torch.int16).numpy().view(np.uint16) if self.cfg.feat_dtype == "bf16" else host.numpy()
 
     def snapshot(self):
         tr = self.tr
@@ -107,12 +118,22 @@ class Rig:
         if upd is None:
             z = np.zeros(0, np.int32)
             upd = (z, z, np.zeros(0), z, None)
+        efeat = self.efeat
+        roots = (nodes, times) + nb
+        if self.compact:
+            # the oracle indexes the feature table by event id: hand it only the rows this step touches,
+            # with ids renumbered monotonically (the (t, eid) order of the reduction is unchanged)
+            ids = np.unique(np.concatenate([np.asarray(upd[3], np.int64), nb[1][nb[1] >= 0].astype(np.int64)]))
+            efeat = self._to_host(self.efeat_dev[torch.from_numpy(ids).cuda()])
+            remap = lambda e: np.where(e >= 0, np.searchsorted(ids, np.maximum(e, 0)), -1).astype(np.int32)
+            upd = (upd[0], upd[1], upd[2], remap(np.asarray(upd[3])), upd[4])
+            roots = (nodes, times, nb[0], remap(nb[1]), nb[2], nb[3])
         kw = {}
         if gates is not None:
             kw = dict(h_gate=gates[0], hid_gate=gates[1], gate_eps=GATE_EPS[self.math])
-        res = o.loss_and_grads(self.ocfg, pre["params"], pre["memory"], pre["last_update"], self.efeat, upd,
-                               (nodes, times) + nb, q.stop - q.start, None, **kw)
-        return res, (nodes, times) + nb
+        res = o.loss_and_grads(self.ocfg, pre["params"], pre["memory"], pre["last_update"], efeat, upd,
+                               roots, q.stop - q.start, None, **kw)
+        return res, roots
 
     def check_step(self, b, pre, res, what=""):
         """Compare the GPU's post-step state with the oracle's result from `pre`."""
@@ -446,3 +467,59 @@ def test_argument_errors_are_reported_not_launched(B):
         B.Tgnn(bad)
     assert lib.status() == 0
     lib.close()
+
+
+# ------------------------------------------ full-size workloads, bench launch configuration
+# The same teacher-forced comparison at the sizes the benchmark spec names, driven the way bench.py drives
+# it: tensor-core mode, the whole step replayed as a CUDA graph on a capturable stream.  The oracle
+# needs seconds per step at these sizes, so only a few sampled steps are compared; every other step
+# still has to keep the device status clean.
+def _full_size(B, oracle, cfg, check_at, last, math="tf32"):
+    rig = Rig(B, oracle, cfg, math=math, batches=range(0, last + 1), bias_scale=0.0, lr=1e-4)
+    for b in range(last + 1):
+        pre = rig.snapshot() if b in check_at else None
+        rig.tr.step(b)
+        if pre is not None:
+            res, _ = rig.oracle_step(pre, b, rig.gpu_gates(b))
+            rig.check_step(b, pre, res, what=f"[{cfg.name} full size, batch {b}]")
+    torch.cuda.synchronize()
+    assert rig.tr.lib.status() == 0
+    return rig
+
+
+@pytest.mark.slow
+def test_wiki_full_size_graph_replay(B, oracle):
+    cfg = wl.CONFIGS["wiki"]
+    rig = _full_size(B, oracle, cfg, {0, 1, 2, 150, cfg.num_batches - 1}, cfg.num_batches - 1)
+    # the last batch is ragged (160000 = 266 * 600 + 400): a different shape signature was captured
+    assert cfg.num_events % cfg.batch != 0
+    assert rig.tr.lib.kernel_launches() > 30 * cfg.num_batches
+
+
+@pytest.mark.slow
+def test_reddit_full_size_replay_and_pruning(B, oracle):
+    cfg = wl.CONFIGS["reddit"]
+    rig = _full_size(B, oracle, cfg, {3, 400}, 400)
+    heavy = rig.dw.heavy.cpu().numpy()
+    keep = rig.dw.mb_keep.cpu().numpy()
+    aux = rig.dw.mb_aux.cpu().numpy()
+    assert keep[aux == 0].all() and 0 < heavy.sum() and (keep[aux == 1] == 0).any()
+
+
+@pytest.mark.slow
+def test_lastfm_full_size_hub_contention(B, oracle):
+    cfg = wl.CONFIGS["lastfm"]
+    rig = _full_size(B, oracle, cfg, {2, 60}, 60)
+    top = np.bincount(np.concatenate([rig.stream.src, rig.stream.dst])).max() / (2 * cfg.num_events)
+    assert top > 0.3                       # one node takes a third of all endpoint slots
+
+
+@pytest.mark.slow
+def test_large_full_size_bf16(B, oracle):
+    # 17,000 nodes, 50 M events, 18.6 GB of bf16 edge features resident in HBM (generated on the device),
+    # batch 4,000, 20 % replay with pruning; about a minute of host set-up (T-CSR over 10^8 entries).  The
+    # feature table is too big for a host copy, so the oracle gets the rows each compared step touches.
+    cfg = wl.CONFIGS["large"]
+    last = cfg.num_batches - 1
+    rig = _full_size(B, oracle, cfg, {5, last}, last)
+    assert rig.compact and rig.efeat_dev.numel() * 2 > 18e9
