@@ -300,6 +300,9 @@ TGNN_API int tgnn_reduce_latest_static(const int32_t* msg_node, const double* t,
  * into buf_host and switches profiling off.  Creates events on first use. */
 TGNN_API int tgnn_profile_begin(tgnn_ctx* ctx);
 TGNN_API int tgnn_profile_report(tgnn_ctx* ctx, char* buf_host, int64_t size);
+/* Same recording, reported launch by launch in issue order: "name start_us duration_us\n", start
+ * relative to the first recorded launch (the internal side streams make launches overlap). */
+TGNN_API int tgnn_profile_timeline(tgnn_ctx* ctx, char* buf_host, int64_t size);
 
 #ifdef __cplusplus
 }

@@ -26,7 +26,7 @@ EXPORTS = ("tgnn_create", "tgnn_destroy", "tgnn_last_error", "tgnn_param_count",
            "tgnn_set_graph", "tgnn_set_edge_features", "tgnn_set_state", "tgnn_prune_mask", "tgnn_sample_recent",
            "tgnn_build_messages", "tgnn_reduce_latest", "tgnn_memory_update", "tgnn_embed", "tgnn_backward_step",
            "tgnn_train_step", "tgnn_train_step_host", "tgnn_debug_get_grads", "tgnn_status", "tgnn_kernel_launches", "tgnn_profile_begin",
-           "tgnn_profile_report", "tgnn_reduce_latest_static", "tgnn_debug_gemm", "tgnn_debug_get_gates", "tgnn_set_graph_replay")
+           "tgnn_profile_report", "tgnn_reduce_latest_static", "tgnn_debug_gemm", "tgnn_debug_get_gates", "tgnn_set_graph_replay", "tgnn_profile_timeline")
 TGNN_STATIC_MAX_NODES = 65536
 
 
@@ -80,6 +80,7 @@ def load_library():
         lib.tgnn_kernel_launches.restype = i64
         lib.tgnn_profile_begin.argtypes = [vp]
         lib.tgnn_profile_report.argtypes = [vp, vp, i64]
+        lib.tgnn_profile_timeline.argtypes = [vp, vp, i64]
         lib.tgnn_debug_gemm.argtypes = [vp, vp, i64, i64, vp, i64, i64, vp, i64, i32, i32, i32, vp, vp, vp, vp, i32, i32, i32, i32,
                                         vp]
         lib.tgnn_debug_get_gates.argtypes = [vp, vp, vp, vp]
@@ -286,6 +287,16 @@ class Tgnn:
                                           _dp(dev_K, "i32", "dev_K"), _dp(bias, "f32", "bias"),
                                           _dp(rowsum_out, "f32", "rowsum_out"), int(relu), int(accumulate), split_k,
                                           int(precise), _stream()))
+
+    def profile_timeline(self):
+        """[(kernel name, start_us, duration_us)] in issue order since profile_begin; switches profiling off."""
+        buf = C.create_string_buffer(1 << 20)
+        self._ck(self.lib.tgnn_profile_timeline(self._h, C.addressof(buf), len(buf)))
+        out = []
+        for line in buf.value.decode().splitlines():
+            name, t0, dt = line.rsplit(" ", 2)
+            out.append((name, float(t0), float(dt)))
+        return out
 
     def debug_get_gates(self, h_gate_out, hid_gate_out):
         self._ck(self.lib.tgnn_debug_get_gates(self._h, _dp(h_gate_out, "u8", "h_gate_out"),

@@ -190,7 +190,7 @@ __global__ void __launch_bounds__(256) scatter_dmem_kernel(const float* __restri
     if (slot < 0) continue;
     float* out = dMemU + (int64_t)slot * d;
     if (r < nb_rows) {
-      const float* g = dZm + (int64_t)r * d;
+      const float* g = dZm + (int64_t)r * 2 * d;  // memory half of the [NB, 2d] gradient rows
       for (int q = lane; q < d; q += 32) atomicAdd(&out[q], g[q]);
     } else {
       const int i = r - nb_rows;
@@ -372,11 +372,13 @@ int grad_w(tgnn_ctx* ctx, const float* dY, int64_t ld_dy, const float* A, int64_
 
 // dA[rows, n_cols] = dY[rows, n_out] W[:, col0 : col0 + n_cols]   (W is [n_out, ld_w] row-major)
 int grad_in(tgnn_ctx* ctx, const float* dY, int64_t ld_dy, const float* W, int64_t ld_w, int col0, int rows,
-            const int32_t* dev_rows, int n_out, int n_cols, float* dA, int64_t ld_da, const char* name, cudaStream_t s) {
+            const int32_t* dev_rows, int n_out, int n_cols, float* dA, int64_t ld_da, const char* name, cudaStream_t s,
+            int site = 0) {
   GemmArgs g = {};
   g.A = dY; g.a_rs = ld_dy; g.a_cs = 1;
   g.B = W + col0; g.b_rs = ld_w; g.b_cs = 1;
   g.C = dA; g.ldc = ld_da; g.M = rows; g.N = n_cols; g.K = n_out; g.dev_M = dev_rows; g.split_k = 1; g.precise = 1;
+  g.site = site;
   return launch_gemm(ctx, g, name, s);
 }
 
@@ -430,6 +432,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     g.A = w.cat1; g.a_rs = 2 * d; g.a_cs = 1;
     g.B = P + L.w1; g.b_rs = 1; g.b_cs = 2 * d;
     g.C = w.hid1; g.ldc = d; g.M = 2 * n_q; g.N = d; g.K = 2 * d; g.bias = P + L.b1; g.relu = 1; g.split_k = 1;
+    g.site = SITE_HEAD + 1;
     RC(launch_gemm(ctx, g, "head_hidden", s));
     {
       KernelScope scope__(ctx, "head_loss", s);
@@ -440,7 +443,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     // hid1 now holds d loss / d pre1
     RC(fork_to(ctx, s, sa));
     RC(grad_w(ctx, w.hid1, d, w.cat1, 2 * d, 2 * n_q, nullptr, d, 2 * d, G + L.w1, G + L.b1, "dW_1", sa));
-    RC(grad_in(ctx, w.hid1, d, P + L.w1, 2 * d, 0, 2 * n_q, nullptr, d, 2 * d, w.dcat1, 2 * d, "dcat1", s));
+    RC(grad_in(ctx, w.hid1, d, P + L.w1, 2 * d, 0, 2 * n_q, nullptr, d, 2 * d, w.dcat1, 2 * d, "dcat1", s, SITE_DCAT1 + 1));
     const int64_t tot2 = (int64_t)R * d;
     {
       KernelScope scope__(ctx, "dh", s);
@@ -449,7 +452,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     TGNN_LAUNCH_OK(ctx, "dh");
     RC(fork_to(ctx, s, sb));
     RC(grad_w(ctx, w.dpre_o, d, w.cat_o, 2 * d, R, nullptr, d, 2 * d, G + L.wo, G + L.bo, "dW_o", sb));
-    RC(grad_in(ctx, w.dpre_o, d, P + L.wo, 2 * d, 0, R, nullptr, d, 2 * d, w.dcat_o, 2 * d, "dcat_o", s));
+    RC(grad_in(ctx, w.dpre_o, d, P + L.wo, 2 * d, 0, R, nullptr, d, 2 * d, w.dcat_o, 2 * d, "dcat_o", s, SITE_DCATO + 1));
     const int wpb = attn_warps_per_block(d, H, k);
     {
       static int attr_bytes = 0;
@@ -471,14 +474,23 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     RC(grad_w(ctx, w.dQ, d, w.Zq, 2 * d, R, nullptr, d, 2 * d, G + L.wq, G + L.bq, "dW_q", sb));
     // time-encoder gradient through the attention inputs (side stream b)
     const size_t tg_smem = (size_t)8 * 2 * d * sizeof(double);
-    RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, d + de, NB, nullptr, 2 * d, d, w.dZp, d, "dZ_phi", sb));
+    // gradient w.r.t. the memory columns and the time-encoding columns of Z, side by side in dZmp.  With the
+    // weight images at hand it is one product on the caller's stream (the scatter below needs its first
+    // half); otherwise the two column ranges of W_kv are two strided products.
+    const bool merged_dz = ctx->cfg.math_mode != TGNN_MATH_FP32 && ctx->images_fresh && ctx->images != nullptr;
+    if (merged_dz) {
+      RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, 0, NB, nullptr, 2 * d, 2 * d, w.dZmp, 2 * d, "dZ", s, SITE_DZ + 1));
+      RC(fork_to(ctx, s, sb));
+    } else {
+      RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, d + de, NB, nullptr, 2 * d, d, w.dZmp + d, 2 * d, "dZ_phi", sb));
+    }
     {
       KernelScope scope__(ctx, "time_grad_z", sb);
-      time_grad_kernel<<<(NB + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, sb>>>(w.dZp, d, 0, w.Zsin, w.z_dt, NB, nullptr, d,
-                                                                           P + L.time_b, w.tg_acc);
+      time_grad_kernel<<<(NB + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, sb>>>(w.dZmp, 2 * d, d, w.Zsin, w.z_dt, NB, nullptr,
+                                                                           d, P + L.time_b, w.tg_acc);
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_z");
-    RC(grad_in(ctx, w.dQ, d, P + L.wq, 2 * d, 0, R, nullptr, d, 2 * d, w.dzq, 2 * d, "dzq", s));
+    RC(grad_in(ctx, w.dQ, d, P + L.wq, 2 * d, 0, R, nullptr, d, 2 * d, w.dzq, 2 * d, "dzq", s, SITE_DZQ + 1));
     RC(fork_to(ctx, s, sb));
     {
       KernelScope scope__(ctx, "time_grad_q", sb);
@@ -487,10 +499,11 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_q");
     if (ctx->have_update) {
-      RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, 0, NB, nullptr, 2 * d, d, w.dZm, d, "dZ_mem", s));
+      if (!merged_dz)
+        RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, 0, NB, nullptr, 2 * d, d, w.dZmp, 2 * d, "dZ_mem", s));
       {
         KernelScope scope__(ctx, "scatter_dmem", s);
-        scatter_dmem_kernel<<<(NB + R + 7) / 8, 256, 0, s>>>(w.dZm, w.dcat_o, w.dzq, ctx->e_nbr, ctx->e_nodes, R, k, d,
+        scatter_dmem_kernel<<<(NB + R + 7) / 8, 256, 0, s>>>(w.dZmp, w.dcat_o, w.dzq, ctx->e_nbr, ctx->e_nodes, R, k, d,
                                                              w.node2slot, w.dMemU);
       }
       TGNN_LAUNCH_OK(ctx, "scatter_dmem");
@@ -509,7 +522,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       RC(grad_w(ctx, w.dGh, 3 * d, w.X, ctx->ld_msg, U_cap, ctx->upd_n_uniq, 3 * d, d, G + L.gru_wh, G + L.gru_bh,
                 "dW_h", sb));
       RC(grad_in(ctx, w.dGi, 3 * d, P + L.gru_wi, L.dmsg, 2 * d + de, U_cap, ctx->upd_n_uniq, 3 * d, d, w.dXp, d,
-                 "dX_phi", s));
+                 "dX_phi", s, SITE_DXPHI + 1));
       {
         KernelScope scope__(ctx, "time_grad_x", s);
         time_grad_kernel<<<(U_cap + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, s>>>(w.dXp, d, 0, w.Xsin, w.x_dt, U_cap,

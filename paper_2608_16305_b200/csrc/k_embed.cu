@@ -174,7 +174,7 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
   g.A = w.Z; g.a_rs = ctx->ld_kv; g.a_cs = 1;
   g.B = ctx->params + L.wk; g.b_rs = 1; g.b_cs = L.dkv;  // rows of [W_k; W_v]
   g.C = w.KV; g.ldc = 2 * d; g.M = n * k; g.N = 2 * d; g.K = (int)L.dkv;
-  g.bias = ctx->params + L.bk; g.split_k = 1;
+  g.bias = ctx->params + L.bk; g.split_k = 1; g.site = SITE_KV + 1;
   int rc = fork_to(ctx, s, ctx->side[0]);  // the query projection runs beside the key/value projection
   if (rc) return rc;
   rc = launch_gemm(ctx, g, "kv_proj", s);
@@ -182,7 +182,7 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
   g = GemmArgs{};
   g.A = w.Zq; g.a_rs = 2 * d; g.a_cs = 1;
   g.B = ctx->params + L.wq; g.b_rs = 1; g.b_cs = 2 * d;
-  g.C = w.Q; g.ldc = d; g.M = n; g.N = d; g.K = 2 * d; g.bias = ctx->params + L.bq; g.split_k = 1;
+  g.C = w.Q; g.ldc = d; g.M = n; g.N = d; g.K = 2 * d; g.bias = ctx->params + L.bq; g.split_k = 1; g.site = SITE_Q + 1;
   rc = launch_gemm(ctx, g, "q_proj", ctx->side[0]);
   if (rc) return rc;
   rc = fork_to(ctx, ctx->side[0], s);
@@ -198,7 +198,7 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
   g = GemmArgs{};
   g.A = w.cat_o; g.a_rs = 2 * d; g.a_cs = 1;
   g.B = ctx->params + L.wo; g.b_rs = 1; g.b_cs = 2 * d;
-  g.C = h_out; g.ldc = d; g.M = n; g.N = d; g.K = 2 * d; g.bias = ctx->params + L.bo; g.relu = 1; g.split_k = 1;
+  g.C = h_out; g.ldc = d; g.M = n; g.N = d; g.K = 2 * d; g.bias = ctx->params + L.bo; g.relu = 1; g.split_k = 1; g.site = SITE_OUT + 1;
   return launch_gemm(ctx, g, "out_proj", s);
 }
 

@@ -49,6 +49,10 @@ struct TcArgs {
   float* rowsum_out;
   int relu, accumulate, split_k;
   int32_t* status;
+  // B operand prepared as shared-memory images (see WeightSite): image of n-tile x, contraction block
+  // kb at b_image + x * b_tile_stride + kb * (COPIES * B_BYTES); nullptr: B goes through registers
+  const unsigned char* b_image;
+  int64_t b_tile_stride;
 };
 
 template <int BN_T, bool PRECISE>
@@ -260,7 +264,7 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kern
 
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(smem_u32(&s_full[s]), GROUP);
+      mbar_init(smem_u32(&s_full[s]), GROUP + (g.b_image ? 1 : 0));
       mbar_init(smem_u32(&s_empty[s]), 1);
     }
     mbar_init(smem_u32(&s_accum), 1);
@@ -299,7 +303,19 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kern
       const int k0 = (kb0 + i) * BK;
       load_tile<BM, PRECISE>(a_tile, C_::A_BYTES, g.A, g.lda, g.a_major, m0, M, BM, k0, k_end, a_vec, t,
                              want_rowsum ? &rs : nullptr);
-      load_tile<BN_T, PRECISE>(b_tile, C_::B_BYTES, g.B, g.ldb, g.b_major, n0, g.N, b_rows, k0, k_end, b_vec, t, nullptr);
+      if (g.b_image != nullptr) {
+        if (t == 0) {  // one bulk asynchronous copy brings the whole B tile (head and tail); it signals full[s] itself
+          constexpr uint32_t bytes = C_::COPIES * C_::B_BYTES;
+          const unsigned char* src = g.b_image + blockIdx.x * g.b_tile_stride + (int64_t)(kb0 + i) * bytes;
+          const uint32_t bar = smem_u32(&s_full[s]);
+          asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+          asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                       ::"r"(b_tile), "l"(src), "r"(bytes), "r"(bar)
+                       : "memory");
+        }
+      } else {
+        load_tile<BN_T, PRECISE>(b_tile, C_::B_BYTES, g.B, g.ldb, g.b_major, n0, g.N, b_rows, k0, k_end, b_vec, t, nullptr);
+      }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       mbar_arrive(smem_u32(&s_full[s]));
     }
@@ -427,6 +443,69 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kern
   }
 }
 
+// n-tiles of at most 256 columns, balanced, in whole 32-column atoms; narrower tiles (down to 64
+// columns) when a store-mode product would otherwise occupy only a few SMs.
+void tile_plan(int M, int N, bool split_accumulate, int* n_tiles, int* bn) {
+  int nt = (N + 255) / 256;
+  const int m_tiles = (M + BM - 1) / BM;
+  if (!split_accumulate)
+    while (m_tiles * nt < 96 && ((N + nt - 1) / nt + 31) / 32 * 32 > 64) ++nt;
+  *n_tiles = nt;
+  *bn = ((N + nt - 1) / nt + 31) / 32 * 32;
+}
+
+// Writes the B-operand images of every weight site from the current parameters.  One thread per
+// 16-byte chunk: the same rounding / head-tail split and the same swizzled placement as load_tile.
+__global__ void __launch_bounds__(256) prep_weights_kernel(const WeightSite* __restrict__ sites,
+                                                           const float* __restrict__ params,
+                                                           unsigned char* __restrict__ images) {
+  const WeightSite st = sites[blockIdx.y];
+  const int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (idx >= st.chunks) return;
+  const int per_tile_kb = st.bn_t * 8;  // logical chunks per (tile, k-block)
+  const int cidx = (int)(idx % per_tile_kb);
+  const int64_t tk = idx / per_tile_kb;
+  const int kb = (int)(tk % st.nkb), tile = (int)(tk / st.nkb);
+  const int n0 = tile * st.bn;
+  const int n_valid = min(st.bn, st.N - n0);
+  const int n_mma = (n_valid + 15) / 16 * 16;
+  const int copies = st.precise ? 2 : 1;
+  const int b_bytes = st.bn_t * 128;
+  unsigned char* img = images + st.image_off + ((int64_t)tile * st.nkb + kb) * copies * b_bytes;
+  const float* W = params + st.w_off;
+  float v[4] = {0.f, 0.f, 0.f, 0.f};
+  uint32_t off;
+  if (st.major == MAJOR_K) {
+    const int r = cidx >> 3, c = cidx & 7;
+    const int n = n0 + r, k = kb * BK + 4 * c;
+    if (r < (n_mma + 7) / 8 * 8 && n < st.N)
+      for (int e = 0; e < 4; ++e)
+        if (k + e < st.K) v[e] = W[(int64_t)n * st.ld + k + e];
+    off = (r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4);
+  } else {
+    const int b_rows = (n_valid + 31) / 32 * 32;
+    const int cpr = b_rows >> 2, atoms = b_rows >> 5;
+    const int kk = cidx / cpr, cm = cidx - kk * cpr;
+    if (kk >= BK) return;  // beyond the region this tile uses
+    const int k = kb * BK + kk;
+    for (int e = 0; e < 4; ++e) {
+      const int n = n0 + 4 * cm + e;
+      if (k < st.K && n < st.N) {
+        const int col = n < st.n_split ? st.col0 + n : st.col1 + (n - st.n_split);
+        v[e] = W[(int64_t)k * st.ld + col];
+      }
+    }
+    const int a = cm >> 3, c = cm & 7;
+    off = (kk >> 2) * (atoms * 512) + a * 512 + (kk & 3) * 128 + ((c ^ ((kk & 3) << 1)) << 4);
+  }
+  const uint32_t h0 = to_tf32(v[0]), h1 = to_tf32(v[1]), h2 = to_tf32(v[2]), h3 = to_tf32(v[3]);
+  *reinterpret_cast<uint4*>(img + off) = make_uint4(h0, h1, h2, h3);
+  if (st.precise)
+    *reinterpret_cast<uint4*>(img + b_bytes + off) =
+        make_uint4(to_tf32(v[0] - __uint_as_float(h0)), to_tf32(v[1] - __uint_as_float(h1)),
+                   to_tf32(v[2] - __uint_as_float(h2)), to_tf32(v[3] - __uint_as_float(h3)));
+}
+
 template <int BN_T, bool PRECISE>
 int launch_tc(tgnn_ctx* ctx, const TcArgs& a, int n_tiles, const char* name, cudaStream_t s) {
   using C_ = Cfg<BN_T, PRECISE>;
@@ -461,12 +540,16 @@ int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStr
   a.M = g.M; a.N = g.N; a.K = g.K; a.dev_M = g.dev_M; a.dev_K = g.dev_K;
   a.bias = g.bias; a.rowsum_out = g.rowsum_out; a.relu = g.relu; a.accumulate = g.accumulate;
   a.status = ctx->ws.status;
-  // n-tiles of at most 256 columns, balanced, whole 32-column atoms; narrower tiles (down to 64
-  // columns) when the product would otherwise occupy only a few SMs
-  int n_tiles = (g.N + 255) / 256;
-  const int m_tiles = (g.M + BM - 1) / BM;
-  if (!(g.accumulate && g.split_k > 1))
-    while (m_tiles * n_tiles < 96 && ((g.N + n_tiles - 1) / n_tiles + 31) / 32 * 32 > 64) ++n_tiles;
+  int n_tiles, bn;
+  bool precise = g.precise != 0;
+  tile_plan(g.M, g.N, g.accumulate && g.split_k > 1, &n_tiles, &bn);
+  if (g.site > 0 && ctx->images_fresh && ctx->images) {  // B is a weight matrix whose images are up to date
+    const WeightSite& st = ctx->sites[g.site - 1];
+    n_tiles = st.n_tiles; bn = st.bn; precise = st.precise != 0;
+    a.b_image = ctx->images + st.image_off;
+    a.b_tile_stride = (int64_t)st.nkb * (st.precise ? 2 : 1) * st.bn_t * 128;
+    a.b_major = st.major;
+  }
   a.split_k = 1;
   if (g.accumulate && g.split_k > 1) {  // the caller allows split-K: one wave of CTAs, >= 4 stages of work each
     const int tiles = n_tiles * ((g.M + BM - 1) / BM);
@@ -475,13 +558,64 @@ int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStr
     if (a.split_k > max_s) a.split_k = max_s;
     if (a.split_k < 1) a.split_k = 1;
   }
-  const int bn = ((g.N + n_tiles - 1) / n_tiles + 31) / 32 * 32;
-  if (g.precise) {
+  if (precise) {
     if (bn <= 128) return launch_tc<128, true>(ctx, a, n_tiles, name, s);
     return launch_tc<256, true>(ctx, a, n_tiles, name, s);
   }
   if (bn <= 128) return launch_tc<128, false>(ctx, a, n_tiles, name, s);
   return launch_tc<256, false>(ctx, a, n_tiles, name, s);
+}
+
+}  // namespace tgnn
+
+namespace tgnn {
+
+size_t plan_weight_sites(tgnn_ctx* ctx) {
+  const ParamLayout& L = ctx->L;
+  const int d = (int)L.d, de = (int)L.de;
+  const bool all_precise = ctx->cfg.math_mode == TGNN_MATH_TF32;
+  struct Def { int id; int64_t w_off, ld; int major, N, K, col0, n_split, col1, M_cap, split_acc, grad; };
+  const int U = ctx->U_cap, R = ctx->R_cap, NB = ctx->NB_cap, Q2 = 2 * ctx->nq_cap;
+  const Def defs[SITE_COUNT] = {
+      {SITE_GI, L.gru_wi, L.dmsg, MAJOR_K, 3 * d, (int)L.dmsg, 0, 0, 0, U, 1, 0},
+      {SITE_GH, L.gru_wh, d, MAJOR_K, 3 * d, d, 0, 0, 0, U, 0, 0},
+      {SITE_KV, L.wk, L.dkv, MAJOR_K, 2 * d, (int)L.dkv, 0, 0, 0, NB, 0, 0},
+      {SITE_Q, L.wq, 2 * d, MAJOR_K, d, 2 * d, 0, 0, 0, R, 0, 0},
+      {SITE_OUT, L.wo, 2 * d, MAJOR_K, d, 2 * d, 0, 0, 0, R, 0, 0},
+      {SITE_HEAD, L.w1, 2 * d, MAJOR_K, d, 2 * d, 0, 0, 0, Q2, 0, 0},
+      {SITE_DCAT1, L.w1, 2 * d, MAJOR_MN, 2 * d, d, 0, 2 * d, 0, Q2, 0, 1},
+      {SITE_DCATO, L.wo, 2 * d, MAJOR_MN, 2 * d, d, 0, 2 * d, 0, R, 0, 1},
+      {SITE_DZQ, L.wq, 2 * d, MAJOR_MN, 2 * d, d, 0, 2 * d, 0, R, 0, 1},
+      {SITE_DZ, L.wk, L.dkv, MAJOR_MN, 2 * d, 2 * d, 0, d, d + de, NB, 0, 1},
+      {SITE_DXPHI, L.gru_wi, L.dmsg, MAJOR_MN, d, 3 * d, 2 * d + de, d, 0, U, 0, 1},
+  };
+  size_t off = 0;
+  for (const Def& f : defs) {
+    WeightSite& st = ctx->sites[f.id];
+    st.w_off = f.w_off; st.ld = f.ld; st.major = f.major; st.N = f.N; st.K = f.K;
+    st.col0 = f.col0; st.n_split = f.n_split; st.col1 = f.col1;
+    st.precise = (all_precise || f.grad) ? 1 : 0;
+    tile_plan(f.M_cap, f.N, f.split_acc != 0, &st.n_tiles, &st.bn);
+    st.bn_t = st.bn <= 128 ? 128 : 256;
+    st.nkb = (f.K + BK - 1) / BK;
+    st.image_off = (int64_t)off;
+    st.chunks = (int64_t)st.n_tiles * st.nkb * st.bn_t * 8;
+    off += (size_t)st.n_tiles * st.nkb * (st.precise ? 2 : 1) * st.bn_t * 128;
+  }
+  return off;
+}
+
+int launch_prep_weights(tgnn_ctx* ctx, cudaStream_t s) {
+  if (!ctx->images || ctx->cfg.math_mode == TGNN_MATH_FP32) return TGNN_OK;
+  int64_t mx = 0;
+  for (int i = 0; i < SITE_COUNT; ++i) mx = ctx->sites[i].chunks > mx ? ctx->sites[i].chunks : mx;
+  dim3 grid((unsigned)((mx + 255) / 256), SITE_COUNT);
+  {
+    KernelScope scope__(ctx, "prep_weights", s);
+    prep_weights_kernel<<<grid, 256, 0, s>>>(ctx->sites_dev, ctx->params, ctx->images);
+  }
+  TGNN_LAUNCH_OK(ctx, "prep_weights");
+  return TGNN_OK;
 }
 
 }  // namespace tgnn

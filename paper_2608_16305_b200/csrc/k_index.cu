@@ -212,13 +212,73 @@ __global__ void __launch_bounds__(1024) reduce_latest_kernel(const int32_t* __re
                                                              int32_t* win_msg, int32_t* node2slot, int32_t* prev_uniq,
                                                              int32_t* prev_n_uniq, int32_t* __restrict__ uniq_out,
                                                              int32_t* __restrict__ winner_out,
-                                                             int32_t* __restrict__ n_uniq_out) {
+                                                             int32_t* __restrict__ n_uniq_out, int smem_nodes) {
+  extern __shared__ int s_last[];  // [smem_nodes]: last message index per node (fast path)
   __shared__ int s_warp[32];
   __shared__ int s_total;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   // forget the previous step's node -> slot map
   const int pn = *prev_n_uniq;
   for (int i = tid; i < pn; i += blockDim.x) node2slot[prev_uniq[i]] = -1;
+  // Fast path.  A mixed batch arrives sorted by (t, eid) (Eq. 5), and then the key order of the
+  // messages is their index order: the winner of a node is simply its last message.  One shared-memory
+  // atomicMax per warp and node replaces the two global passes.  Unsorted input takes the general path.
+  if (smem_nodes >= N) {
+    bool sorted = true;
+    const int n_ev = n_msg >> 1;
+    for (int i = tid; i + 1 < n_ev; i += blockDim.x)
+      sorted = sorted && (t[i] < t[i + 1] || (t[i] == t[i + 1] && eid[i] < eid[i + 1]));
+    if (__syncthreads_and(sorted)) {
+      for (int v = tid; v < N; v += blockDim.x) s_last[v] = -1;
+      __syncthreads();
+      const int n_round = (n_msg + 31) / 32 * 32;
+      for (int j = tid; j < n_round; j += blockDim.x) {
+        const int node = j < n_msg ? message_node(msg_node, ev_src, ev_dst, ev_keep, j) : -1;
+        const bool v = node >= 0;
+        const unsigned act = __ballot_sync(FULL, v);
+        if (v) {
+          const unsigned peers = __match_any_sync(act, node);
+          if (lane == 31 - __clz(peers)) atomicMax(&s_last[node], j);  // the highest lane holds the largest j
+        }
+      }
+      __syncthreads();
+      const int chunk = (N + blockDim.x - 1) / blockDim.x;
+      const int nb = min(N, tid * chunk), ne = min(N, nb + chunk);
+      int mine = 0;
+      for (int v = nb; v < ne; ++v) mine += s_last[v] >= 0;
+      int incl = mine;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(FULL, incl, o);
+        if (lane >= o) incl += y;
+      }
+      if (lane == 31) s_warp[wid] = incl;
+      __syncthreads();
+      if (wid == 0) {
+        const int w = lane < (int)(blockDim.x >> 5) ? s_warp[lane] : 0;
+        int wi = w;
+        for (int o = 1; o < 32; o <<= 1) {
+          const int y = __shfl_up_sync(FULL, wi, o);
+          if (lane >= o) wi += y;
+        }
+        s_warp[lane] = wi - w;
+        if (lane == 31) s_total = wi;
+      }
+      __syncthreads();
+      int pos = s_warp[wid] + incl - mine;
+      for (int v = nb; v < ne; ++v) {
+        const int j = s_last[v];
+        if (j >= 0) {
+          uniq_out[pos] = v;
+          winner_out[pos] = j;
+          prev_uniq[pos] = v;
+          node2slot[v] = pos;
+          ++pos;
+        }
+      }
+      if (tid == 0) { *n_uniq_out = s_total; *prev_n_uniq = s_total; }
+      return;
+    }
+  }
   const int n_round = (n_msg + 31) / 32 * 32;
   for (int j = tid; j < n_round; j += blockDim.x) {
     const int node = j < n_msg ? message_node(msg_node, ev_src, ev_dst, ev_keep, j) : -1;
@@ -353,11 +413,20 @@ int launch_reduce_latest_events(tgnn_ctx* ctx, const int32_t* msg_node, const in
                                 const uint8_t* keep, const double* t, const int32_t* eid, int n_msg, int32_t* uniq_out,
                                 int32_t* winner_out, int32_t* n_uniq_out, cudaStream_t s) {
   Workspace& w = ctx->ws;
+  // shared-memory table of the fast path: 4 bytes per node, when it fits
+  const int N = (int)ctx->cfg.num_nodes;
+  const int smem_nodes = (size_t)N * 4 <= 200 * 1024 ? N : 0;
+  static int attr_bytes = 0;
+  if (smem_nodes * 4 > attr_bytes) {
+    TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(reduce_latest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_nodes * 4));
+    attr_bytes = smem_nodes * 4;
+  }
   {
     KernelScope scope__(ctx, "reduce_latest", s);
-    reduce_latest_kernel<<<1, 1024, 0, s>>>(msg_node, src, dst, keep, t, eid, n_msg, (int)ctx->cfg.num_nodes, w.best_t, w.best_id,
-                                            w.win_msg, w.node2slot, w.prev_uniq, w.prev_n_uniq, uniq_out, winner_out,
-                                            n_uniq_out);
+    reduce_latest_kernel<<<1, 1024, (size_t)smem_nodes * 4, s>>>(msg_node, src, dst, keep, t, eid, n_msg, N, w.best_t,
+                                                                 w.best_id, w.win_msg, w.node2slot, w.prev_uniq,
+                                                                 w.prev_n_uniq, uniq_out, winner_out, n_uniq_out,
+                                                                 smem_nodes);
   }
   TGNN_LAUNCH_OK(ctx, "reduce_latest");
   return TGNN_OK;

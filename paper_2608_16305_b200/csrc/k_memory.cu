@@ -157,14 +157,14 @@ int launch_memory_update(tgnn_ctx* ctx, const float* msg, const int32_t* uniq, c
   g.C = w.Gi; g.ldc = 3 * d; g.M = U_cap; g.N = 3 * d; g.K = (int)L.dmsg; g.dev_M = n_uniq;
   g.bias = ctx->params + L.gru_bi;
   // few rows, long contraction: split the contraction over CTAs and accumulate into a cleared Gi
-  g.accumulate = 1; g.split_k = 4;
+  g.accumulate = 1; g.split_k = 4; g.site = SITE_GI + 1;
   TGNN_CUDA_OK(ctx, cudaMemsetAsync(w.Gi, 0, sizeof(float) * (size_t)U_cap * 3 * d, s));
   int rc = fork_to(ctx, s, ctx->side[0]);  // the hidden-state product runs beside the input product
   if (rc) return rc;
   rc = launch_gemm(ctx, g, "gru_gi", s);
   if (rc) return rc;
   g.B = ctx->params + L.gru_wh; g.b_cs = d; g.C = w.Gh; g.K = d; g.bias = ctx->params + L.gru_bh;
-  g.accumulate = 0; g.split_k = 1;
+  g.accumulate = 0; g.split_k = 1; g.site = SITE_GH + 1;
   rc = launch_gemm(ctx, g, "gru_gh", ctx->side[0]);
   if (rc) return rc;
   rc = fork_to(ctx, ctx->side[0], s);

@@ -133,8 +133,7 @@ size_t carve(tgnn_ctx* ctx, char* base) {
   cv.take(w.dQ, R * d);
   cv.take(w.dzq, R * 2 * d);
   cv.take(w.dKV, NB * 2 * d);
-  cv.take(w.dZm, NB * d);
-  cv.take(w.dZp, NB * d);
+  cv.take(w.dZmp, NB * 2 * d);
   cv.take(w.dGi, U * 3 * d);
   cv.take(w.dGh, U * 3 * d);
   cv.take(w.dXp, U * d);
@@ -214,6 +213,14 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
     delete ctx;
     return TGNN_ECUDA;
   }
+  ctx->images = nullptr; ctx->sites_dev = nullptr; ctx->images_fresh = false;
+  if (ok && cfg->math_mode != TGNN_MATH_FP32) {
+    ctx->images_bytes = plan_weight_sites(ctx);
+    ok = cudaMalloc((void**)&ctx->images, ctx->images_bytes) == cudaSuccess &&
+         cudaMemset(ctx->images, 0, ctx->images_bytes) == cudaSuccess &&
+         cudaMalloc((void**)&ctx->sites_dev, sizeof(ctx->sites)) == cudaSuccess &&
+         cudaMemcpy(ctx->sites_dev, ctx->sites, sizeof(ctx->sites), cudaMemcpyHostToDevice) == cudaSuccess;
+  }
   ctx->ev_next = 0;
   ctx->n_graphs = 0;
   ctx->graphs_enabled = 1;
@@ -221,6 +228,8 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
   for (int i = 0; ok && i < 32; ++i) ok = cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
+    cudaFree(ctx->images);
+    cudaFree(ctx->sites_dev);
     cudaFree(ctx->arena);
     delete ctx;
     return TGNN_ECUDA;
@@ -241,6 +250,8 @@ int tgnn_destroy(tgnn_ctx* ctx) {
     if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
   for (int i = 0; i < 2; ++i) cudaStreamDestroy(ctx->side[i]);
   for (int i = 0; i < 32; ++i) cudaEventDestroy(ctx->ev[i]);
+  cudaFree(ctx->images);
+  cudaFree(ctx->sites_dev);
   cudaFree(ctx->arena);
   delete ctx;
   return TGNN_OK;
@@ -276,7 +287,7 @@ int tgnn_set_state(tgnn_ctx* ctx, float* memory, double* last_update, float* par
   NEED(ctx, memory && last_update && params && adam_m && adam_v && step, TGNN_EINVAL, "set_state: null pointer");
   ctx->memory = memory; ctx->last_update = last_update; ctx->params = params;
   ctx->adam_m = adam_m; ctx->adam_v = adam_v; ctx->step = step;
-  ctx->have_update = false; ctx->have_embed = false; ctx->grads_zeroed = false;
+  ctx->have_update = false; ctx->have_embed = false; ctx->grads_zeroed = false; ctx->images_fresh = false;
   return TGNN_OK;
 }
 
@@ -359,6 +370,7 @@ int tgnn_backward_step(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* 
   ctx->have_embed = false;
   ctx->have_update = false;
   ctx->grads_zeroed = false;
+  ctx->images_fresh = false;  // Adam has changed the parameters
   return rc;
 }
 
@@ -370,6 +382,14 @@ int step_body(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q, bool has_mask, flo
   Workspace& w = ctx->ws;
   int rc;
   ctx->have_update = false;
+  // the weights' B-operand images for this step's projections: written beside the first kernels
+  const bool prep = ctx->images != nullptr;
+  if (prep) {
+    rc = fork_to(ctx, S(stream), ctx->side[0]);
+    if (rc) return rc;
+    rc = launch_prep_weights(ctx, ctx->side[0]);
+    if (rc) return rc;
+  }
   // the neighbor search reads only the static graph: it runs beside the memory update
   cudaStream_t side = ctx->side[1];
   rc = fork_to(ctx, S(stream), side);
@@ -395,8 +415,17 @@ int step_body(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q, bool has_mask, flo
     rc = launch_reduce_latest_events(ctx, nullptr, w.st_u_src, w.st_u_dst, ctx->m_keep, w.st_u_t, w.st_u_eid, 2 * n_u,
                                      w.uniq, w.winner, w.n_uniq, S(stream));
     if (rc) return rc;
+    if (prep) {
+      rc = fork_to(ctx, ctx->side[0], S(stream));
+      if (rc) return rc;
+      ctx->images_fresh = true;
+    }
     rc = tgnn_memory_update(ctx, nullptr, w.uniq, w.winner, w.n_uniq, stream);
     if (rc) return rc;
+  } else if (prep) {
+    rc = fork_to(ctx, ctx->side[0], S(stream));
+    if (rc) return rc;
+    ctx->images_fresh = true;
   }
   rc = fork_to(ctx, side, S(stream));  // join
   if (rc) return rc;
@@ -414,7 +443,7 @@ void after_replay(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q) {
   ctx->upd_cap = ctx->U_cap < 2 * n_u ? ctx->U_cap : 2 * n_u;
   ctx->e_nodes = w.r_node; ctx->e_times = w.r_time; ctx->e_nbr = w.nb_node; ctx->e_eid = w.nb_eid;
   ctx->e_ts = w.nb_ts; ctx->e_cnt = w.nb_cnt; ctx->e_n = 3 * n_q; ctx->e_h = w.h;
-  ctx->have_embed = false; ctx->have_update = false; ctx->grads_zeroed = false;
+  ctx->have_embed = false; ctx->have_update = false; ctx->grads_zeroed = false; ctx->images_fresh = false;
 }
 
 }  // namespace
@@ -571,6 +600,26 @@ int tgnn_profile_begin(tgnn_ctx* ctx) {
   if (!ctx) return TGNN_EINVAL;
   ctx->prof.used = 0;
   ctx->prof.on = true;
+  return TGNN_OK;
+}
+
+int tgnn_profile_timeline(tgnn_ctx* ctx, char* buf, int64_t size) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, buf && size > 0, TGNN_EINVAL, "profile_timeline: null buffer");
+  ctx->prof.on = false;
+  TGNN_CUDA_OK(ctx, cudaDeviceSynchronize());
+  std::string out;
+  char line[160];
+  for (size_t i = 0; i < ctx->prof.used; ++i) {
+    const ProfEntry& e = ctx->prof.entries[i];
+    float t0 = 0.f, dt = 0.f;
+    if (cudaEventElapsedTime(&t0, ctx->prof.entries[0].a, e.a) != cudaSuccess ||
+        cudaEventElapsedTime(&dt, e.a, e.b) != cudaSuccess) { cudaGetLastError(); continue; }
+    snprintf(line, sizeof(line), "%s %.3f %.3f\n", e.name, t0 * 1e3, dt * 1e3);
+    out += line;
+  }
+  snprintf(buf, (size_t)size, "%s", out.c_str());
+  ctx->prof.used = 0;
   return TGNN_OK;
 }
 

@@ -71,8 +71,7 @@ struct Workspace {
   float* dQ;      // [R_cap, d]
   float* dzq;     // [R_cap, 2d]
   float* dKV;     // [NB_cap, 2d]
-  float* dZm;     // [NB_cap, d]  grad wrt the memory part of Z
-  float* dZp;     // [NB_cap, d]  grad wrt the time-encoding part of Z
+  float* dZmp;    // [NB_cap, 2d] grad wrt the memory part (cols [0,d)) and the time-encoding part (cols [d,2d)) of Z
   float* dMemU;   // [U_cap, d]   grad wrt the rows written by the memory update
   float* dGi;     // [U_cap, 3d]
   float* dGh;     // [U_cap, 3d]
@@ -95,6 +94,27 @@ struct Profiler {
   bool on = false;
   std::vector<ProfEntry> entries;  // events are created once and reused
   size_t used = 0;
+};
+
+// A weight matrix in its role as the B operand of one projection, with the tiling the tensor-core
+// kernel will use for it.  Once per step the weights are written out as "images": for every n-tile and
+// contraction block the exact bytes of the shared-memory B tile (TF32 head, then TF32 tail, already
+// swizzled), so that a CTA fetches a stage's B operand with one bulk asynchronous copy instead of
+// loading, splitting and storing it through registers in every CTA.
+enum WeightSiteId {
+  SITE_GI = 0, SITE_GH, SITE_KV, SITE_Q, SITE_OUT, SITE_HEAD,   // forward: B(k,n) = W[n*ld + k]
+  SITE_DCAT1, SITE_DCATO, SITE_DZQ, SITE_DZ, SITE_DXPHI,        // input gradients: B(k,n) = W[k*ld + col(n)]
+  SITE_COUNT
+};
+struct WeightSite {
+  int64_t w_off, ld;
+  int major;                 // 0: K-major (forward), 1: MN-major (input gradient)
+  int N, K;                  // columns of C, contraction length
+  int col0, n_split, col1;   // MN-major: col(n) = n < n_split ? col0 + n : col1 + (n - n_split)
+  int precise;
+  int n_tiles, bn, bn_t, nkb;
+  int64_t image_off;         // byte offset of the site's images in the image buffer
+  int64_t chunks;            // 16-byte chunks the preparation kernel writes for this site
 };
 
 }  // namespace tgnn
@@ -129,6 +149,11 @@ struct tgnn_ctx {
   const int32_t* upd_n_uniq;
   int upd_cap;
   bool have_update, have_embed;
+  tgnn::WeightSite sites[tgnn::SITE_COUNT];
+  tgnn::WeightSite* sites_dev;   // device copy
+  unsigned char* images;         // device buffer of all sites' images
+  size_t images_bytes;
+  bool images_fresh;             // images match the current parameters (set by the step, cleared by Adam)
   bool z_static_done; // tgnn_train_step already gathered the memory-independent part of the attention inputs
   bool grads_zeroed;  // tgnn_train_step cleared the gradient block ahead of the backward pass
   tgnn::Workspace ws;
@@ -254,9 +279,12 @@ struct GemmArgs {
   int relu;               // apply ReLU in the epilogue (store mode only)
   int accumulate;         // atomicAdd into C (C must hold valid data); required when split_k > 1
   int split_k;            // >= 1
+  int site;               // WeightSiteId + 1 when B is that weight matrix (0: none); lets the kernel use its image
   int precise;            // tensor-core mode only: 3xTF32 head/tail split, close to fp32 accuracy
 };
 int launch_gemm(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s);
 int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s);  // k_gemm_tc.cu
+size_t plan_weight_sites(tgnn_ctx* ctx);                       // fills ctx->sites, returns the image bytes needed
+int launch_prep_weights(tgnn_ctx* ctx, cudaStream_t s);        // writes all images from the current parameters
 
 }  // namespace tgnn

@@ -309,24 +309,26 @@ def test_messages_reduction_and_gru_by_parts(tiny_rig):
         assert np.array_equal(got_m[rest], mem[rest])
 
 
-@pytest.mark.parametrize("case", ["ties_unsorted", "hub", "all_dropped", "empty"])
+@pytest.mark.parametrize("case", ["ties_unsorted", "hub", "sorted_hub", "all_dropped", "empty"])
 def test_reduce_latest_bit_exact(B, oracle, case):
     rng = np.random.default_rng(26)
     N = 3000
     lib = B.Tgnn(B.make_config(N, 32, 16, 10, 2, max_events=6000, max_roots=3000))
     if case == "empty":
         n = 0
-    elif case == "hub":
+    elif case in ("hub", "sorted_hub"):
         n = 5200
     else:
         n = 777
     src = rng.integers(0, N, n).astype(np.int32)
     dst = rng.integers(0, N, n).astype(np.int32)
-    if case == "hub":
+    if case in ("hub", "sorted_hub"):
         src[rng.random(n) < 0.6] = 5
         dst[rng.random(n) < 0.3] = 5
     t = rng.integers(0, 40, n).astype(np.float64) - (3.0 if case == "ties_unsorted" else 0.0)   # ties, unsorted, some negative
     eid = rng.permutation(3 * n + 1)[:n].astype(np.int32)
+    if case == "sorted_hub":          # a batch sorted by (t, eid), as mixed batches are: the shared-memory fast path
+        t, eid = np.sort(t), np.sort(eid)
     node = np.stack([src, dst], 1).reshape(-1).astype(np.int32)
     drop = np.repeat(rng.random(n) < (1.0 if case == "all_dropped" else 0.2), 2)
     node[drop] = -1
