@@ -266,6 +266,9 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
         peak, bound = SM_COUNT * FP32_LANES_PER_SM * 2 * clk_ghz / 1000.0, "alu"
         peak_note = "148 SMs x 128 fp32 lanes x 2 flop x max SM clock"
     achieved = flops / dur_s / 1e12 if dur_s > 0 else 0.0
+    # dram__bytes_read.sum + dram__bytes_write.sum of one key/value-projection launch on this workload
+    # (ncu --set full, summarised in profiles/gemm_tf32_kv_proj_wiki.md; tensor-core mode only)
+    traffic = 28.6e6 + 0.08e6 if args.math == "tf32" else None
     by, f_fwd, f_bwd = algorithmic_work(cfg, n_q, n_q, 450)
     out = {
         "metric": METRIC, "value": units / (ms_dev_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
@@ -283,7 +286,8 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                     "frac": achieved / peak if peak else None, "traffic": None, "peak_source": peak_note,
+                     "frac": achieved / peak if peak else None, "traffic": traffic, "peak_source": peak_note,
+                     "algorithmic_bytes_per_launch": 3 * n_q * cfg.k * (cfg.d_kv * 4 + 2 * cfg.d * 4) + 2 * cfg.d * cfg.d_kv * 4,
                      "flops_per_launch": flops, "avg_launch_us": dur_s * 1e6, "launches": cnt,
                      "step_algorithmic_bytes": by, "step_algorithmic_flops": f_fwd + f_bwd,
                      "step_hbm_frac": (by / (ms_dev_max / K * 1e-3)) / (peaks["hbm_gbs"] * 1e9),
