@@ -471,33 +471,37 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     RC(fork_to(ctx, s, sa));
     RC(fork_to(ctx, s, sb));
     RC(grad_w(ctx, w.dKV, 2 * d, w.Z, ctx->ld_kv, NB, nullptr, 2 * d, (int)L.dkv, G + L.wk, G + L.bk, "dW_kv", sa));
-    RC(grad_w(ctx, w.dQ, d, w.Zq, 2 * d, R, nullptr, d, 2 * d, G + L.wq, G + L.bq, "dW_q", sb));
     // time-encoder gradient through the attention inputs (side stream b)
     const size_t tg_smem = (size_t)8 * 2 * d * sizeof(double);
     // gradient w.r.t. the memory columns and the time-encoding columns of Z, side by side in dZmp.  With the
     // weight images at hand it is one product on the caller's stream (the scatter below needs its first
     // half); otherwise the two column ranges of W_kv are two strided products.
     const bool merged_dz = ctx->cfg.math_mode != TGNN_MATH_FP32 && ctx->images_fresh && ctx->images != nullptr;
-    if (merged_dz) {
-      RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, 0, NB, nullptr, 2 * d, 2 * d, w.dZmp, 2 * d, "dZ", s, SITE_DZ + 1));
-      RC(fork_to(ctx, s, sb));
-    } else {
-      RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, d + de, NB, nullptr, 2 * d, d, w.dZmp + d, 2 * d, "dZ_phi", sb));
-    }
-    {
-      KernelScope scope__(ctx, "time_grad_z", sb);
-      time_grad_kernel<<<(NB + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, sb>>>(w.dZmp, 2 * d, d, w.Zsin, w.z_dt, NB, nullptr,
-                                                                           d, P + L.time_b, w.tg_acc);
-    }
-    TGNN_LAUNCH_OK(ctx, "time_grad_z");
-    RC(grad_in(ctx, w.dQ, d, P + L.wq, 2 * d, 0, R, nullptr, d, 2 * d, w.dzq, 2 * d, "dzq", s, SITE_DZQ + 1));
-    RC(fork_to(ctx, s, sb));
+    // the query-side input gradient does not depend on dZ: it runs on side stream b next to it
+    RC(grad_in(ctx, w.dQ, d, P + L.wq, 2 * d, 0, R, nullptr, d, 2 * d, w.dzq, 2 * d, "dzq", sb, SITE_DZQ + 1));
+    cudaEvent_t dzq_done = mark_stream(ctx, sb);  // waited for by the scatter further down
+    RC(grad_w(ctx, w.dQ, d, w.Zq, 2 * d, R, nullptr, d, 2 * d, G + L.wq, G + L.bq, "dW_q", sb));
     {
       KernelScope scope__(ctx, "time_grad_q", sb);
       time_grad_kernel<<<(R + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, sb>>>(w.dzq, 2 * d, d, nullptr, nullptr, R, nullptr, d,
                                                                           P + L.time_b, w.tg_acc);
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_q");
+    cudaStream_t s_tgz = sb;  // where the time-encoder sum over the neighbor rows runs
+    if (merged_dz) {
+      RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, 0, NB, nullptr, 2 * d, 2 * d, w.dZmp, 2 * d, "dZ", s, SITE_DZ + 1));
+      RC(fork_to(ctx, s, sa));
+      s_tgz = sa;
+    } else {
+      RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, d + de, NB, nullptr, 2 * d, d, w.dZmp + d, 2 * d, "dZ_phi", sb));
+    }
+    {
+      KernelScope scope__(ctx, "time_grad_z", s_tgz);
+      time_grad_kernel<<<(NB + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, s_tgz>>>(w.dZmp, 2 * d, d, w.Zsin, w.z_dt, NB, nullptr,
+                                                                              d, P + L.time_b, w.tg_acc);
+    }
+    TGNN_LAUNCH_OK(ctx, "time_grad_z");
+    RC(wait_mark(ctx, s, dzq_done));  // the scatter below needs dzq
     if (ctx->have_update) {
       if (!merged_dz)
         RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, 0, NB, nullptr, 2 * d, d, w.dZmp, 2 * d, "dZ_mem", s));

@@ -140,12 +140,12 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 //             atom a, chunk c lives at (kk/4)*(atoms*512) + a*512 + (kk%4)*128 + ((c ^ 2*(kk%4))*16):
 //             the swizzle exchanges 32-byte pairs of chunks (address bits 5-6 ^= bits 7-8).
 // rows_t is a multiple of 32 (MN-major) or of 8 (K-major); chunks outside the valid range are zero.
-template <int ROWS_MAX, bool PRECISE>
-__device__ __forceinline__ void load_tile(uint32_t tile, uint32_t tail_offset, const float* __restrict__ P, int64_t ld,
-                                          int major, int r0, int R, int rows_t, int k0, int k1, bool vec, int t,
-                                          float4* rowsum) {
+// The tile is filled in two steps so that a producer can have the loads of its next block in flight
+// while it waits for a free stage and stores the current one.
+template <int ROWS_MAX>
+__device__ __forceinline__ void load_regs(float4 (&v)[ROWS_MAX * 8 / GROUP], const float* __restrict__ P, int64_t ld,
+                                          int major, int r0, int R, int rows_t, int k0, int k1, bool vec, int t) {
   constexpr int ITERS = ROWS_MAX * 8 / GROUP;
-  float4 v[ITERS];
   if (major == MAJOR_K) {
 #pragma unroll
     for (int i = 0; i < ITERS; ++i) {
@@ -165,15 +165,8 @@ __device__ __forceinline__ void load_tile(uint32_t tile, uint32_t tail_offset, c
         }
       }
     }
-#pragma unroll
-    for (int i = 0; i < ITERS; ++i) {
-      const int idx = t + i * GROUP;
-      const int r = idx >> 3, c = idx & 7;
-      if (r < rows_t) store_chunk<PRECISE>(tile + (r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4), tail_offset, v[i]);
-    }
   } else {
     const int cpr = rows_t >> 2;  // 16-byte chunks per k-row (multiple of 8)
-    const int atoms = rows_t >> 5;
 #pragma unroll
     for (int i = 0; i < ITERS; ++i) {
       const int idx = t + i * GROUP;
@@ -192,6 +185,23 @@ __device__ __forceinline__ void load_tile(uint32_t tile, uint32_t tail_offset, c
         }
       }
     }
+  }
+}
+
+template <int ROWS_MAX, bool PRECISE>
+__device__ __forceinline__ void store_regs(const float4 (&v)[ROWS_MAX * 8 / GROUP], uint32_t tile, uint32_t tail_offset,
+                                           int major, int rows_t, int t, float4* rowsum) {
+  constexpr int ITERS = ROWS_MAX * 8 / GROUP;
+  if (major == MAJOR_K) {
+#pragma unroll
+    for (int i = 0; i < ITERS; ++i) {
+      const int idx = t + i * GROUP;
+      const int r = idx >> 3, c = idx & 7;
+      if (r < rows_t) store_chunk<PRECISE>(tile + (r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4), tail_offset, v[i]);
+    }
+  } else {
+    const int cpr = rows_t >> 2;
+    const int atoms = rows_t >> 5;
 #pragma unroll
     for (int i = 0; i < ITERS; ++i) {
       const int idx = t + i * GROUP;
@@ -206,6 +216,15 @@ __device__ __forceinline__ void load_tile(uint32_t tile, uint32_t tail_offset, c
       }
     }
   }
+}
+
+template <int ROWS_MAX, bool PRECISE>
+__device__ __forceinline__ void load_tile(uint32_t tile, uint32_t tail_offset, const float* __restrict__ P, int64_t ld,
+                                          int major, int r0, int R, int rows_t, int k0, int k1, bool vec, int t,
+                                          float4* rowsum) {
+  float4 v[ROWS_MAX * 8 / GROUP];
+  load_regs<ROWS_MAX>(v, P, ld, major, r0, R, rows_t, k0, k1, vec, t);
+  store_regs<ROWS_MAX, PRECISE>(v, tile, tail_offset, major, rows_t, t, rowsum);
 }
 
 __device__ __forceinline__ void mma_tf32(uint32_t tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
@@ -292,8 +311,13 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kern
     float4 rs = make_float4(0.f, 0.f, 0.f, 0.f);
     const int k_end = min(K, kb1 * BK);
     bool ok = true;
+    // The A registers of the group's next block are loaded before it waits for the current stage,
+    // so that round trip overlaps the wait, the stores and the MMAs of the blocks in between.
+    float4 va[BM * 8 / GROUP], vn[BM * 8 / GROUP];
+    if (grp < nkb) load_regs<BM>(va, g.A, g.lda, g.a_major, m0, M, BM, (kb0 + grp) * BK, k_end, a_vec, t);
     for (int i = grp; i < nkb; i += GROUPS) {
       const int s = i % STAGES;
+      if (i + GROUPS < nkb) load_regs<BM>(vn, g.A, g.lda, g.a_major, m0, M, BM, (kb0 + i + GROUPS) * BK, k_end, a_vec, t);
       if (i >= STAGES) {
         ok = mbar_wait(smem_u32(&s_empty[s]), ((i / STAGES) - 1) & 1);
         if (!ok) break;
@@ -301,8 +325,6 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kern
       const uint32_t a_tile = smem_base + s * C_::STAGE_BYTES;
       const uint32_t b_tile = a_tile + C_::COPIES * C_::A_BYTES;
       const int k0 = (kb0 + i) * BK;
-      load_tile<BM, PRECISE>(a_tile, C_::A_BYTES, g.A, g.lda, g.a_major, m0, M, BM, k0, k_end, a_vec, t,
-                             want_rowsum ? &rs : nullptr);
       if (g.b_image != nullptr) {
         if (t == 0) {  // one bulk asynchronous copy brings the whole B tile (head and tail); it signals full[s] itself
           constexpr uint32_t bytes = C_::COPIES * C_::B_BYTES;
@@ -313,11 +335,14 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kern
                        ::"r"(b_tile), "l"(src), "r"(bytes), "r"(bar)
                        : "memory");
         }
-      } else {
-        load_tile<BN_T, PRECISE>(b_tile, C_::B_BYTES, g.B, g.ldb, g.b_major, n0, g.N, b_rows, k0, k_end, b_vec, t, nullptr);
       }
+      store_regs<BM, PRECISE>(va, a_tile, C_::A_BYTES, g.a_major, BM, t, want_rowsum ? &rs : nullptr);
+      if (g.b_image == nullptr)
+        load_tile<BN_T, PRECISE>(b_tile, C_::B_BYTES, g.B, g.ldb, g.b_major, n0, g.N, b_rows, k0, k_end, b_vec, t, nullptr);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       mbar_arrive(smem_u32(&s_full[s]));
+#pragma unroll
+      for (int q = 0; q < BM * 8 / GROUP; ++q) va[q] = vn[q];
     }
     if (!ok) { s_abort = 1; atomicCAS(g.status, 0, TGNN_ETIMEOUT); }
     if (want_rowsum) {  // the thread's chunks cover rows 4*(t%32) .. +3 of the tile

@@ -207,6 +207,18 @@ inline int fork_to(tgnn_ctx* ctx, cudaStream_t from, cudaStream_t to) {
   return TGNN_OK;
 }
 
+// The two halves of fork_to, for a dependency that is recorded now and waited for later.
+inline cudaEvent_t mark_stream(tgnn_ctx* ctx, cudaStream_t on) {
+  cudaEvent_t e = ctx->ev[ctx->ev_next];
+  ctx->ev_next = (ctx->ev_next + 1) % 32;
+  return cudaEventRecord(e, on) == cudaSuccess ? e : nullptr;
+}
+inline int wait_mark(tgnn_ctx* ctx, cudaStream_t waiter, cudaEvent_t e) {
+  if (!e || cudaStreamWaitEvent(waiter, e, 0) != cudaSuccess)
+    return set_error(ctx, TGNN_ECUDA, "stream fork/join failed: %s", cudaGetErrorString(cudaGetLastError()));
+  return TGNN_OK;
+}
+
 // Brackets one kernel launch with events when profiling is on.
 struct KernelScope {
   tgnn_ctx* c;

@@ -88,6 +88,9 @@ class Trainer:
         # default stream cannot capture, so when the caller is on it the step runs on this stream,
         # ordered after / before the caller's stream with events.
         self.stream = torch.cuda.Stream(device=dev)
+        # The prune mask of batch b is consumed only when b is replayed as the update batch of step b+1,
+        # so it runs on a stream of its own beside step b and is waited for at the start of step b+1.
+        self.prune_stream = torch.cuda.Stream(device=dev)
 
     def _run(self, fn):
         cur = torch.cuda.current_stream()
@@ -113,7 +116,11 @@ class Trainer:
 
     def _step(self, b: int, with_update: bool):
         dw = self.dw
-        self.prune(b)
+        cur = torch.cuda.current_stream()
+        cur.wait_stream(self.prune_stream)          # keep mask of batch b-1 is complete
+        self.prune_stream.wait_stream(cur)          # inputs uploaded on this stream are visible
+        with torch.cuda.stream(self.prune_stream):
+            self.prune(b)
         q = dw.target_slice(b)
         if with_update and b > dw.batches.start:
             u = dw.mb_slice(b - 1)
