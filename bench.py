@@ -192,22 +192,12 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
     clocks = clk.summary()
     loss_end = float(tr.loss.item())
 
-    # ---- host buffers: per-step H2D of the step's inputs, D2H of loss and of the pruned batch's keep mask ----
-    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    # ---- host buffers: one streaming call per mixed batch (packed H2D of the batch, D2H of loss and gradient norm) ----
     host = {}
-    for i in range(W + K + W + K + 4):
-        b = batch_of(i)
-        if b in host:
-            continue
-        mb = dw.mb_host[b]
-        q = dw.target_slice(b)
-        host[b] = dict(src=pin(mb.src), dst=pin(mb.dst), t=pin(mb.t), eid=pin(mb.eid), aux=pin(mb.is_aux),
-                       keep=torch.ones(mb.n, dtype=torch.uint8).pin_memory(),
-                       q_src=pin(stream.src[q]), q_dst=pin(stream.dst[q]), q_neg=pin(stream.neg[q]), q_t=pin(stream.t[q]))
-    cap = cfg.max_mixed
-    st = dict(src=torch.empty(cap, dtype=torch.int32, device=device), dst=torch.empty(cap, dtype=torch.int32, device=device),
-              eid=torch.empty(cap, dtype=torch.int32, device=device), aux=torch.empty(cap, dtype=torch.uint8, device=device),
-              keep=torch.empty(cap, dtype=torch.uint8, device=device), heavy=torch.zeros(1, dtype=torch.int32, device=device))
+    for i in range(W + K, W + K + W + K):
+        bb = batch_of(i)
+        if bb not in host:
+            host[bb] = tr.host_batch(bb)
     loss_h = torch.zeros(1).pin_memory()
     gn_h = torch.zeros(1).pin_memory()
     h2d = d2h = 0
@@ -215,24 +205,16 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
     def host_step(b):
         nonlocal h2d, d2h
         hb = host[b]
-        n = hb["src"].numel()
-        for kname in ("src", "dst", "eid", "aux"):
-            st[kname][:n].copy_(hb[kname], non_blocking=True)
-        tr.lib.prune_mask(st["src"][:n], st["dst"][:n], st["eid"][:n], st["aux"][:n], st["keep"][:n], st["heavy"],
-                          force_heavy=-1 if cfg.prune else 0, drop_q32=tr.drop_q32, seed=tr.prune_seed, batch_idx=b)
-        hb["keep"].copy_(st["keep"][:n], non_blocking=True)
-        if b > 0:
-            hu = host[b - 1]
-            upd = (hu["src"], hu["dst"], hu["t"], hu["eid"], hu["keep"])
-        else:
-            upd = (None,) * 5
-        tr.lib.train_step_host(*upd, hb["q_src"], hb["q_dst"], hb["q_neg"], hb["q_t"], None, loss_h, gn_h)
+        if b == 0:
+            tr.lib.set_state(tr.memory, tr.last_update, tr.params, tr.adam_m, tr.adam_v, tr.step_count)  # restart the stream
+        tr.step_host(b, hb, loss_h, gn_h)
         torch.cuda.current_stream().synchronize()        # the caller reads the loss every step
-        n_u = 0 if b == 0 else host[b - 1]["src"].numel()
-        h2d += n * 13 + n_u * 21 + hb["q_src"].numel() * 20
-        d2h += n + 8
+        n, nq = hb["src"].numel(), hb["neg"].numel()
+        h2d += 21 * n + 20 * nq
+        d2h += 8
 
     reset_epoch()
+    tr.lib.set_state(tr.memory, tr.last_update, tr.params, tr.adam_m, tr.adam_v, tr.step_count)
     run_steps(W + K, W, host_step, False)
     barrier()
     h2d = d2h = 0
@@ -282,7 +264,7 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
                    "inputs": "resident in HBM"},
         "e2e": {"value": units / (ms_host_max * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d_step,
                 "d2h_bytes_per_step": d2h_step, "ms_per_step": ms_host_max / K,
-                "how": "tgnn_train_step_host with pinned host event arrays; loss read back and stream synchronised every step"},
+                "how": "tgnn_step_mixed_host: one call per mixed batch from host arrays (packed copy), loss and gradient norm read back, stream synchronised every step"},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",

@@ -233,6 +233,19 @@ TGNN_API int tgnn_train_step_host(tgnn_ctx* ctx, const int32_t* u_src_host, cons
                          const int32_t* q_dst_host, const int32_t* q_neg_host, const double* q_t_host, int n_q,
                          const uint8_t* loss_mask_host, float* loss_host, float* gradnorm_host, void* stream);
 
+/* The streaming form of the step, host inputs: one call per mixed batch (Eq. 5), in stream order.
+ * The call copies the batch to the device as one packed block, computes its prune mask (step 0,
+ * arguments as in tgnn_prune_mask) beside the rest of the step, and trains on its target events
+ * (is_aux == 0, in batch order; neg_host holds one negative destination per target event) after the
+ * PREVIOUS call's batch, as kept by its mask, has updated memory (lag-one order).  The batch then
+ * stays on the device for the next call.  tgnn_set_state restarts the sequence (no previous batch).
+ * Host arrays may be pageable and are free for reuse when the call returns; loss_host /
+ * gradnorm_host (may be NULL) are written by asynchronous copies: synchronise the stream first. */
+TGNN_API int tgnn_step_mixed_host(tgnn_ctx* ctx, const int32_t* src_host, const int32_t* dst_host, const double* t_host,
+                                  const int32_t* eid_host, const uint8_t* is_aux_host, int n, const int32_t* neg_host,
+                                  int force_heavy, uint32_t drop_q32, uint64_t seed, int64_t batch_idx,
+                                  float* loss_host, float* gradnorm_host, void* stream);
+
 /* ---- debug / parity -------------------------------------------------------- */
 
 /* Copies the parameter gradient of the last tgnn_backward_step to grads_out:f32[param_count]. */

@@ -26,7 +26,7 @@ EXPORTS = ("tgnn_create", "tgnn_destroy", "tgnn_last_error", "tgnn_param_count",
            "tgnn_set_graph", "tgnn_set_edge_features", "tgnn_set_state", "tgnn_prune_mask", "tgnn_sample_recent",
            "tgnn_build_messages", "tgnn_reduce_latest", "tgnn_memory_update", "tgnn_embed", "tgnn_backward_step",
            "tgnn_train_step", "tgnn_train_step_host", "tgnn_debug_get_grads", "tgnn_status", "tgnn_kernel_launches", "tgnn_profile_begin",
-           "tgnn_profile_report", "tgnn_reduce_latest_static", "tgnn_debug_gemm", "tgnn_debug_get_gates", "tgnn_set_graph_replay", "tgnn_profile_timeline")
+           "tgnn_profile_report", "tgnn_reduce_latest_static", "tgnn_debug_gemm", "tgnn_debug_get_gates", "tgnn_set_graph_replay", "tgnn_profile_timeline", "tgnn_step_mixed_host")
 TGNN_STATIC_MAX_NODES = 65536
 
 
@@ -84,6 +84,7 @@ def load_library():
         lib.tgnn_debug_gemm.argtypes = [vp, vp, i64, i64, vp, i64, i64, vp, i64, i32, i32, i32, vp, vp, vp, vp, i32, i32, i32, i32,
                                         vp]
         lib.tgnn_debug_get_gates.argtypes = [vp, vp, vp, vp]
+        lib.tgnn_step_mixed_host.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, i32, u32, u64, i64, vp, vp, vp]
         lib.tgnn_set_graph_replay.argtypes = [vp, i32]
         lib.tgnn_reduce_latest_static.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, vp, vp, i32]
         _lib = lib
@@ -272,6 +273,14 @@ class Tgnn:
                                                _hp(q_t, "f64", "q_t"), q_src.numel(), _hp(loss_mask, "u8", "loss_mask"),
                                                _hp(loss_host, "f32", "loss_host"), _hp(gradnorm_host, "f32", "gradnorm_host"),
                                                _stream()))
+
+    def step_mixed_host(self, src, dst, t, eid, is_aux, neg, loss_host, gradnorm_host, force_heavy=-1,
+                        drop_q32=1 << 31, seed=0, batch_idx=0):
+        self._ck(self.lib.tgnn_step_mixed_host(self._h, _hp(src, "i32", "src"), _hp(dst, "i32", "dst"), _hp(t, "f64", "t"),
+                                               _hp(eid, "i32", "eid"), _hp(is_aux, "u8", "is_aux"), src.numel(),
+                                               _hp(neg, "i32", "neg"), force_heavy, drop_q32, seed, batch_idx,
+                                               _hp(loss_host, "f32", "loss_host"),
+                                               _hp(gradnorm_host, "f32", "gradnorm_host"), _stream()))
 
     def set_graph_replay(self, enable: bool):
         self._ck(self.lib.tgnn_set_graph_replay(self._h, int(enable)))

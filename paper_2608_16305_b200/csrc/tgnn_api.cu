@@ -213,6 +213,32 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
     delete ctx;
     return TGNN_ECUDA;
   }
+  {
+    const size_t ne = (size_t)cfg->max_events, nq = (size_t)ctx->nq_cap;
+    ctx->pack_bytes = (8 * ne + 8 * nq + 12 * ne + 12 * nq + ne + 63) & ~(size_t)63;
+    const size_t slot_bytes = (((12 + 8 + 2) * ne) + 255) & ~(size_t)255;
+    unsigned char* base = nullptr;
+    ctx->mixed_cur = -1;
+    ctx->pack_dev = nullptr; ctx->pack_host[0] = ctx->pack_host[1] = nullptr; ctx->heavy_dev = nullptr;
+    ok = ok && cudaMalloc((void**)&ctx->pack_dev, ctx->pack_bytes + 2 * slot_bytes + 256) == cudaSuccess;
+    if (ok) {
+      base = ctx->pack_dev + ctx->pack_bytes;
+      for (int i = 0; i < 2; ++i) {
+        unsigned char* p = base + i * slot_bytes;
+        ctx->mixed[i].t = (double*)p; p += 8 * ne;
+        ctx->mixed[i].src = (int32_t*)p; p += 4 * ne;
+        ctx->mixed[i].dst = (int32_t*)p; p += 4 * ne;
+        ctx->mixed[i].eid = (int32_t*)p; p += 4 * ne;
+        ctx->mixed[i].aux = p; p += ne;
+        ctx->mixed[i].keep = p;
+        ctx->mixed[i].n = 0;
+      }
+      ctx->heavy_dev = (int32_t*)(base + 2 * slot_bytes);
+    }
+    for (int i = 0; ok && i < 2; ++i)
+      ok = cudaHostAlloc((void**)&ctx->pack_host[i], ctx->pack_bytes, cudaHostAllocDefault) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ctx->pack_done[i], cudaEventDisableTiming) == cudaSuccess;
+  }
   ctx->images = nullptr; ctx->sites_dev = nullptr; ctx->images_fresh = false;
   if (ok && cfg->math_mode != TGNN_MATH_FP32) {
     ctx->images_bytes = plan_weight_sites(ctx);
@@ -230,6 +256,8 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
     cudaGetLastError();
     cudaFree(ctx->images);
     cudaFree(ctx->sites_dev);
+    cudaFree(ctx->pack_dev);
+    for (int i = 0; i < 2; ++i) if (ctx->pack_host[i]) cudaFreeHost(ctx->pack_host[i]);
     cudaFree(ctx->arena);
     delete ctx;
     return TGNN_ECUDA;
@@ -252,6 +280,11 @@ int tgnn_destroy(tgnn_ctx* ctx) {
   for (int i = 0; i < 32; ++i) cudaEventDestroy(ctx->ev[i]);
   cudaFree(ctx->images);
   cudaFree(ctx->sites_dev);
+  cudaFree(ctx->pack_dev);
+  for (int i = 0; i < 2; ++i) {
+    if (ctx->pack_host[i]) cudaFreeHost(ctx->pack_host[i]);
+    cudaEventDestroy(ctx->pack_done[i]);
+  }
   cudaFree(ctx->arena);
   delete ctx;
   return TGNN_OK;
@@ -288,6 +321,7 @@ int tgnn_set_state(tgnn_ctx* ctx, float* memory, double* last_update, float* par
   ctx->memory = memory; ctx->last_update = last_update; ctx->params = params;
   ctx->adam_m = adam_m; ctx->adam_v = adam_v; ctx->step = step;
   ctx->have_update = false; ctx->have_embed = false; ctx->grads_zeroed = false; ctx->images_fresh = false;
+  ctx->mixed_cur = -1;
   return TGNN_OK;
 }
 
@@ -520,6 +554,65 @@ int tgnn_train_step(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, c
   e->exec = exec;
   TGNN_CUDA_OK(ctx, cudaGraphLaunch(e->exec, S(stream)));
   after_replay(ctx, n_u, has_keep, n_q);
+  return TGNN_OK;
+}
+
+int tgnn_step_mixed_host(tgnn_ctx* ctx, const int32_t* src, const int32_t* dst, const double* t, const int32_t* eid,
+                         const uint8_t* is_aux, int n, const int32_t* neg, int force_heavy, uint32_t drop_q32,
+                         uint64_t seed, int64_t batch_idx, float* loss_host, float* gradnorm_host, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, n >= 0, TGNN_EINVAL, "step_mixed_host: negative n");
+  NEED(ctx, n <= ctx->cfg.max_events, TGNN_ECAPACITY, "step_mixed_host: n %d > max_events %d", n, ctx->cfg.max_events);
+  NEED(ctx, n == 0 || (src && dst && t && eid && is_aux), TGNN_EINVAL, "step_mixed_host: null batch arrays");
+  NEED(ctx, force_heavy >= -1 && force_heavy <= 1, TGNN_EINVAL, "step_mixed_host: force_heavy must be -1, 0 or 1");
+  int n_q = 0;
+  for (int i = 0; i < n; ++i) n_q += is_aux[i] == 0;
+  NEED(ctx, n_q <= ctx->nq_cap, TGNN_ECAPACITY, "step_mixed_host: %d target events > max_roots/3 = %d", n_q, ctx->nq_cap);
+  NEED(ctx, n_q == 0 || neg, TGNN_EINVAL, "step_mixed_host: null negatives");
+  cudaStream_t s = S(stream);
+  const int slot = ctx->mixed_cur < 0 ? 0 : 1 - ctx->mixed_cur;
+  // pack: one block, one copy
+  unsigned char* pk = ctx->pack_host[slot];
+  TGNN_CUDA_OK(ctx, cudaEventSynchronize(ctx->pack_done[slot]));  // the copy that last used this buffer has finished
+  double* p_t = reinterpret_cast<double*>(pk);
+  double* p_qt = p_t + n;
+  int32_t* p_i = reinterpret_cast<int32_t*>(p_qt + n_q);
+  int32_t* p_q = p_i + 3 * (size_t)n;
+  uint8_t* p_aux = reinterpret_cast<uint8_t*>(p_q + 3 * (size_t)n_q);
+  memcpy(p_t, t, sizeof(double) * n);
+  memcpy(p_i, src, sizeof(int32_t) * n);
+  memcpy(p_i + n, dst, sizeof(int32_t) * n);
+  memcpy(p_i + 2 * (size_t)n, eid, sizeof(int32_t) * n);
+  memcpy(p_aux, is_aux, n);
+  for (int i = 0, j = 0; i < n; ++i)
+    if (!is_aux[i]) { p_qt[j] = t[i]; p_q[j] = src[i]; p_q[n_q + j] = dst[i]; p_q[2 * (size_t)n_q + j] = neg[j]; ++j; }
+  const size_t bytes = (size_t)(p_aux + n - pk);
+  if (bytes > 0) TGNN_CUDA_OK(ctx, cudaMemcpyAsync(ctx->pack_dev, pk, bytes, cudaMemcpyHostToDevice, s));
+  TGNN_CUDA_OK(ctx, cudaEventRecord(ctx->pack_done[slot], s));
+  // the previous call's prune ran on a side stream: its keep mask is needed from here on
+  int rc = fork_to(ctx, ctx->side[1], s);
+  if (rc) return rc;
+  rc = launch_unpack_mixed(ctx, ctx->pack_dev, n, n_q, slot, s);
+  if (rc) return rc;
+  ctx->mixed[slot].n = n;
+  if (n > 0) {  // step (0) for this batch, beside the step: its result is first read by the next call
+    rc = fork_to(ctx, s, ctx->side[1]);
+    if (rc) return rc;
+    const tgnn_ctx::MixedSlot& m = ctx->mixed[slot];
+    rc = launch_prune_mask(ctx, m.src, m.dst, m.eid, m.aux, n, force_heavy, drop_q32, seed, batch_idx, m.keep,
+                           ctx->heavy_dev, ctx->side[1]);
+    if (rc) return rc;
+  }
+  const tgnn_ctx::MixedSlot* u = ctx->mixed_cur >= 0 ? &ctx->mixed[ctx->mixed_cur] : nullptr;
+  Workspace& w = ctx->ws;
+  rc = tgnn_train_step(ctx, u ? u->src : nullptr, u ? u->dst : nullptr, u ? u->t : nullptr, u ? u->eid : nullptr,
+                       u ? u->keep : nullptr, u ? u->n : 0, w.st_q_src, w.st_q_dst, w.st_q_neg, w.st_q_t, n_q, nullptr,
+                       nullptr, nullptr, stream);
+  if (rc) return rc;
+  ctx->mixed_cur = slot;
+  if (loss_host) TGNN_CUDA_OK(ctx, cudaMemcpyAsync(loss_host, w.st_scalars + 2, sizeof(float), cudaMemcpyDeviceToHost, s));
+  if (gradnorm_host)
+    TGNN_CUDA_OK(ctx, cudaMemcpyAsync(gradnorm_host, w.st_scalars + 3, sizeof(float), cudaMemcpyDeviceToHost, s));
   return TGNN_OK;
 }
 

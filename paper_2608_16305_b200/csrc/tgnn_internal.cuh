@@ -149,6 +149,22 @@ struct tgnn_ctx {
   const int32_t* upd_n_uniq;
   int upd_cap;
   bool have_update, have_embed;
+  // tgnn_step_mixed_host: the mixed batch of the current call stays on the device (two slots, used
+  // alternately) because it is the update batch of the next call; host inputs travel as one packed
+  // block through two pinned buffers.
+  struct MixedSlot {
+    int32_t *src, *dst, *eid;
+    double* t;
+    uint8_t *aux, *keep;
+    int n;
+  };
+  MixedSlot mixed[2];
+  int mixed_cur;              // slot written by the last call (-1: none yet)
+  unsigned char* pack_host[2];
+  cudaEvent_t pack_done[2];
+  unsigned char* pack_dev;
+  size_t pack_bytes;
+  int32_t* heavy_dev;
   tgnn::WeightSite sites[tgnn::SITE_COUNT];
   tgnn::WeightSite* sites_dev;   // device copy
   unsigned char* images;         // device buffer of all sites' images
@@ -255,6 +271,7 @@ int launch_reduce_latest_events(tgnn_ctx* ctx, const int32_t* msg_node, const in
 int launch_stage_inputs(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, const double* u_t,
                         const int32_t* u_eid, const uint8_t* u_keep, int n_u, const int32_t* q_src, const int32_t* q_dst,
                         const int32_t* q_neg, const double* q_t, int n_q, const uint8_t* loss_mask, cudaStream_t s);
+int launch_unpack_mixed(tgnn_ctx* ctx, const unsigned char* packed, int n, int n_q, int slot, cudaStream_t s);
 int launch_make_roots(tgnn_ctx* ctx, const int32_t* q_src, const int32_t* q_dst, const int32_t* q_neg,
                       const double* q_t, int n_q, cudaStream_t s);
 

@@ -110,6 +110,22 @@ class Trainer:
                             force_heavy=-1 if dw.cfg.prune else 0, drop_q32=self.drop_q32, seed=self.prune_seed,
                             batch_idx=b)
 
+    def host_batch(self, b: int):
+        """Pinned host copies of mixed batch b and of its targets' negatives (what a data loader would hand over)."""
+        dw = self.dw
+        mb = dw.mb_host[b - dw.batches.start]
+        pin = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a, dtype=dt)).pin_memory()
+        q = dw.target_slice(b)
+        return dict(src=pin(mb.src, np.int32), dst=pin(mb.dst, np.int32), t=pin(mb.t, np.float64),
+                    eid=pin(mb.eid, np.int32), aux=pin(mb.is_aux, np.uint8), neg=pin(dw.stream.neg[q], np.int32))
+
+    def step_host(self, b: int, hb, loss_host, gradnorm_host):
+        """One training step fed from host memory: a single call of the streaming entry point per mixed batch."""
+        cfg = self.dw.cfg
+        return self._run(lambda: self.lib.step_mixed_host(
+            hb["src"], hb["dst"], hb["t"], hb["eid"], hb["aux"], hb["neg"], loss_host, gradnorm_host,
+            force_heavy=-1 if cfg.prune else 0, drop_q32=self.drop_q32, seed=self.prune_seed, batch_idx=b))
+
     def step(self, b: int, with_update: bool = True):
         """One training step on batch b (device-resident inputs)."""
         return self._run(lambda: self._step(b, with_update))

@@ -448,6 +448,30 @@ def test_host_buffer_entry_point_matches_device_path(B, oracle):
     assert relerr(b.tr.params.cpu().numpy(), a.tr.params.cpu().numpy()) <= 2e-3
 
 
+def test_streaming_host_entry_point_matches_device_path(B, oracle):
+    # replay + pruning workload: the streaming call keeps each batch (and its prune mask) on the device for the
+    # next call, so agreement over several steps checks the slot hand-over and the mask as well
+    cfg = _scaled("reddit", 9000)
+    a = Rig(B, oracle, cfg, math="tf32")
+    b = Rig(B, oracle, cfg, math="tf32")
+    loss = torch.zeros(1).pin_memory()
+    gn = torch.zeros(1).pin_memory()
+    for step in range(cfg.num_batches):
+        # two training runs drift apart chaotically (atomics order -> rounding -> Adam), so the second run is
+        # put on the first one's state before every step; its previous batch and prune mask remain its own
+        for name in ("memory", "last_update", "params", "adam_m", "adam_v", "step_count"):
+            getattr(b.tr, name).copy_(getattr(a.tr, name))
+        torch.cuda.synchronize()
+        a.tr.step(step)
+        b.tr.step_host(step, b.tr.host_batch(step), loss, gn)
+        torch.cuda.synchronize()
+        assert abs(float(loss.item()) - float(a.tr.loss.item())) <= 1e-5 * abs(float(loss.item())), step
+        assert abs(float(gn.item()) - float(a.tr.gradnorm.item())) <= 1e-4 * abs(float(gn.item())), step
+        assert np.array_equal(b.tr.last_update.cpu().numpy(), a.tr.last_update.cpu().numpy())   # same events kept
+        assert relerr(b.tr.memory.cpu().numpy(), a.tr.memory.cpu().numpy()) <= 1e-5
+    assert a.dw.heavy.sum().item() > 0
+
+
 # ------------------------------------------------------------ errors -------
 def test_argument_errors_are_reported_not_launched(B):
     lib = B.Tgnn(B.make_config(100, 32, 16, 10, 2, max_events=64, max_roots=96))
