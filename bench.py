@@ -128,10 +128,11 @@ def kv_proj_flops(cfg, n_q):
 def run_ours(args, rank, world, device):
     from paper_2608_16305_b200 import binding as B
     from paper_2608_16305_b200 import trainer as T
-    cfg = wl.CONFIGS[WORKLOAD]
+    cfg = wl.CONFIGS[args.workload]
     stream = wl.make_stream(cfg)
     efeat = wl.edge_feature_table_torch(cfg, device)
-    dw = T.DeviceWorkload(stream, device=device, efeat=efeat)
+    n_need = 2 * (args.steps + args.warmup) + 8
+    dw = T.DeviceWorkload(stream, device=device, efeat=efeat, batches=range(0, min(cfg.num_batches, n_need)))
     weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed)
     math_mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST}[args.math]
     tr = T.Trainer(dw, weights, math_mode=math_mode)
@@ -144,7 +145,7 @@ def run_ours(args, rank, world, device):
 
 def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr):
     from paper_2608_16305_b200 import binding as B
-    nb = cfg.num_batches - 1          # full batches only
+    nb = len(dw.batches) - 1          # full batches only
     K, W = args.steps, args.warmup
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)   # > 126 MB L2
     peaks = measured_peaks()
@@ -250,14 +251,15 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
     achieved = flops / dur_s / 1e12 if dur_s > 0 else 0.0
     # dram__bytes_read.sum + dram__bytes_write.sum of one key/value-projection launch on this workload
     # (ncu --set full, summarised in profiles/gemm_tf32_kv_proj_wiki.md; tensor-core mode only)
-    traffic = 28.6e6 + 0.08e6 if args.math == "tf32" else None
-    by, f_fwd, f_bwd = algorithmic_work(cfg, n_q, n_q, 450)
+    traffic = 28.6e6 + 0.08e6 if (args.math == "tf32" and cfg.name == WORKLOAD) else None
+    by, f_fwd, f_bwd = algorithmic_work(cfg, cfg.max_mixed, n_q, min(2 * cfg.max_mixed, cfg.num_nodes) // 2)
     out = {
         "metric": METRIC, "value": units / (ms_dev_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_dev_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32" if args.math == "fp32" else "tf32", "data": "synthetic",
-        "config": {"workload": f"{WORKLOAD}: 9000 nodes (8000+1000 bipartite), 160000 events, d_e=172 fp32, d=100, k=10, "
-                               "2 heads, batch 600, no replay",
+        "config": {"workload": f"{cfg.name}: {cfg.num_nodes} nodes" + (f" ({cfg.num_src}+{cfg.num_nodes - cfg.num_src} bipartite)" if cfg.num_src else "")
+                               + f", {cfg.num_events} events, d_e={cfg.d_e} {cfg.feat_dtype}, d={cfg.d}, k={cfg.k}, {cfg.heads} heads, "
+                               f"batch {cfg.batch}, replay {cfg.replay_frac:g}" + (" with pruning" if cfg.prune else ""),
                    "math_mode": args.math, "l2": "512 MB buffer written between timed steps (outside the event pairs)",
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "launch": "kernel by kernel" if args.no_graph else "CUDA graph replay of the step (captured by the library)",
@@ -277,7 +279,7 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
                      "kernel_ms_total": round(tot, 3)},
         "loss_last": loss_end,
     }
-    out["cpu_baseline"] = cpu_baseline(cfg, stream, weights, budget_s=args.cpu_budget)
+    out["cpu_baseline"] = cpu_baseline(cfg, stream, weights, budget_s=args.cpu_budget) if args.cpu_budget > 0 else None
     print(json.dumps(out))
 
 
@@ -339,6 +341,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--math", default=os.environ.get("TGNN_BENCH_MATH", "tf32"), choices=["fp32", "tf32", "tf32fast"])
     ap.add_argument("--cpu-budget", type=float, default=20.0)
+    ap.add_argument("--workload", default=WORKLOAD, choices=sorted(wl.CONFIGS), help="default: the benchmark workload (wiki)")
     ap.add_argument("--no-graph", action="store_true", help="launch kernel by kernel instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
