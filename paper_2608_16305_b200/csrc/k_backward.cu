@@ -279,28 +279,45 @@ __global__ void __launch_bounds__(256) gru_bwd_gate_kernel(const float* __restri
   }
 }
 
-// Sum of squares of the gradient; the last block to finish turns it into g_r, bumps the Adam
-// step counter and prepares the bias corrections.
+// Gradient norm g_r and the Adam update in one pass over the parameters.  Adam does not depend on the
+// norm (no clipping), so each thread squares its gradient entries into the block's partial sum and
+// updates the same entries; the last block to finish turns the sum into g_r and bumps the step counter
+// (every block has read the counter before it takes its ticket).
 // The time-encoder entries [t_off, t_off + t_n) are taken from their fp64 sums tg_acc (rounded once)
-// and written back into grads by block 0, so the update kernel finds them there.
-__global__ void __launch_bounds__(256) gradnorm_kernel(float* __restrict__ grads, int64_t P,
-                                                       const double* __restrict__ tg_acc, int64_t t_off, int t_n,
-                                                       double* red,
-                                                       unsigned int* ticket, int64_t* step, float beta1, float beta2,
-                                                       float* __restrict__ adam_sc, const float* __restrict__ loss_acc,
-                                                       float* scalars, float* loss_out, float* gradnorm_out) {
+// and written into grads, where the debug export finds them.
+__global__ void __launch_bounds__(256) gradnorm_adam_kernel(float* __restrict__ grads, int64_t P,
+                                                            const double* __restrict__ tg_acc, int64_t t_off, int t_n,
+                                                            double* red, unsigned int* ticket, int64_t* step,
+                                                            float* __restrict__ p, float* __restrict__ m,
+                                                            float* __restrict__ v, float lr, float beta1, float beta2,
+                                                            float eps, const float* __restrict__ loss_acc, float* scalars,
+                                                            float* loss_out, float* gradnorm_out) {
   __shared__ double s_part[8];
+  __shared__ float s_c1, s_c2;
+  if (threadIdx.x == 0) {
+    const double t = (double)(step[0] + 1);
+    s_c1 = (float)(1.0 / (1.0 - pow((double)beta1, t)));
+    s_c2 = (float)(1.0 / (1.0 - pow((double)beta2, t)));
+  }
+  __syncthreads();
+  const float c1 = s_c1, c2 = s_c2;
+  // 1 - beta formed in fp64 from the configured fp32 value, then rounded once
+  const float omb1 = (float)(1.0 - (double)beta1), omb2 = (float)(1.0 - (double)beta2);
   double acc = 0.0;
   for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < P; e += (int64_t)gridDim.x * blockDim.x) {
-    double g;
+    float ge;
     if (e >= t_off && e < t_off + t_n) {
-      const float gt = (float)tg_acc[e - t_off];
-      grads[e] = gt;  // same value from whichever block owns e
-      g = (double)gt;
+      ge = (float)tg_acc[e - t_off];
+      grads[e] = ge;
     } else {
-      g = (double)grads[e];
+      ge = grads[e];
     }
-    acc = fma(g, g, acc);
+    acc = fma((double)ge, (double)ge, acc);
+    const float me = fmaf(beta1, m[e], omb1 * ge);
+    const float ve = fmaf(beta2, v[e], omb2 * ge * ge);
+    m[e] = me;
+    v[e] = ve;
+    p[e] -= lr * (me * c1) / (sqrtf(ve * c2) + eps);
   }
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(FULL, acc, o);
   if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = acc;
@@ -315,10 +332,7 @@ __global__ void __launch_bounds__(256) gradnorm_kernel(float* __restrict__ grads
       __threadfence();
       const double ss = atomicAdd(&red[0], 0.0);
       const float gn = (float)sqrt(ss);
-      const int64_t t = step[0] + 1;
-      step[0] = t;
-      adam_sc[0] = (float)(1.0 / (1.0 - pow((double)beta1, (double)t)));
-      adam_sc[1] = (float)(1.0 / (1.0 - pow((double)beta2, (double)t)));
+      step[0] = step[0] + 1;
       const float loss = *loss_acc;
       scalars[0] = loss;
       scalars[1] = gn;
@@ -326,22 +340,6 @@ __global__ void __launch_bounds__(256) gradnorm_kernel(float* __restrict__ grads
       if (gradnorm_out) *gradnorm_out = gn;
       *ticket = 0u;
     }
-  }
-}
-
-__global__ void __launch_bounds__(256) adam_kernel(float* __restrict__ p, float* __restrict__ m, float* __restrict__ v,
-                                                   const float* __restrict__ g, int64_t P, float lr, float beta1,
-                                                   float beta2, float eps, const float* __restrict__ adam_sc) {
-  const float c1 = adam_sc[0], c2 = adam_sc[1];
-  // 1 - beta formed in fp64 from the configured fp32 value, then rounded once
-  const float omb1 = (float)(1.0 - (double)beta1), omb2 = (float)(1.0 - (double)beta2);
-  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < P; e += (int64_t)gridDim.x * blockDim.x) {
-    const float ge = g[e];
-    const float me = fmaf(beta1, m[e], omb1 * ge);
-    const float ve = fmaf(beta2, v[e], omb2 * ge * ge);
-    m[e] = me;
-    v[e] = ve;
-    p[e] -= lr * (me * c1) / (sqrtf(ve * c2) + eps);
   }
 }
 
@@ -538,16 +536,12 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     RC(fork_to(ctx, sb, s));
   }
   {
-    KernelScope scope__(ctx, "gradnorm", s);
-    gradnorm_kernel<<<148, 256, 0, s>>>(G, L.total, w.tg_acc, L.time_w, n_q > 0 ? 2 * d : 0, w.red, w.counters, ctx->step, c.beta1, c.beta2, w.adam_sc,
-                                        w.st_scalars, w.st_scalars + 2, loss_out, gradnorm_out);
+    KernelScope scope__(ctx, "gradnorm_adam", s);
+    gradnorm_adam_kernel<<<296, 256, 0, s>>>(G, L.total, w.tg_acc, L.time_w, n_q > 0 ? 2 * d : 0, w.red, w.counters,
+                                             ctx->step, P, ctx->adam_m, ctx->adam_v, c.lr, c.beta1, c.beta2, c.eps,
+                                             w.st_scalars, w.st_scalars + 2, loss_out, gradnorm_out);
   }
-  TGNN_LAUNCH_OK(ctx, "gradnorm");
-  {
-    KernelScope scope__(ctx, "adam", s);
-    adam_kernel<<<296, 256, 0, s>>>(P, ctx->adam_m, ctx->adam_v, G, L.total, c.lr, c.beta1, c.beta2, c.eps, w.adam_sc);
-  }
-  TGNN_LAUNCH_OK(ctx, "adam");
+  TGNN_LAUNCH_OK(ctx, "gradnorm_adam");
   return TGNN_OK;
 }
 

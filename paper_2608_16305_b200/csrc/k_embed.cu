@@ -165,18 +165,28 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
     if (rc0) return rc0;
   }
   ctx->z_static_done = false;
+  // In the tensor-core modes the key/value projection reads the neighbors' memory rows straight from
+  // the table (row-indirect A), so the copy of those rows into Z -- still needed by the backward pass,
+  // like the root rows by the query and output projections -- leaves the critical chain for a side stream.
+  const bool indirect = c.math_mode != TGNN_MATH_FP32;
+  int rc = fork_to(ctx, s, ctx->side[0]);
+  if (rc) return rc;
+  cudaStream_t sg = indirect ? ctx->side[0] : s;
   {
-    KernelScope scope__(ctx, "gather_z_memory", s);
-    gather_z_memory_kernel<<<(rows + 7) / 8, 256, 0, s>>>(ctx->memory, d, k, nodes, n, nbr, ctx->ld_kv, w.Z, w.Zq, w.cat_o);
+    KernelScope scope__(ctx, "gather_z_memory", sg);
+    gather_z_memory_kernel<<<(rows + 7) / 8, 256, 0, sg>>>(ctx->memory, d, k, nodes, n, nbr, ctx->ld_kv, w.Z, w.Zq, w.cat_o);
   }
   TGNN_LAUNCH_OK(ctx, "gather_z_memory");
+  if (!indirect) {  // the query projection below runs on the side stream and needs the rows just gathered
+    rc = fork_to(ctx, s, ctx->side[0]);
+    if (rc) return rc;
+  }
   GemmArgs g = {};
   g.A = w.Z; g.a_rs = ctx->ld_kv; g.a_cs = 1;
   g.B = ctx->params + L.wk; g.b_rs = 1; g.b_cs = L.dkv;  // rows of [W_k; W_v]
   g.C = w.KV; g.ldc = 2 * d; g.M = n * k; g.N = 2 * d; g.K = (int)L.dkv;
   g.bias = ctx->params + L.bk; g.split_k = 1; g.site = SITE_KV + 1;
-  int rc = fork_to(ctx, s, ctx->side[0]);  // the query projection runs beside the key/value projection
-  if (rc) return rc;
+  if (indirect) { g.a_idx = nbr; g.a_tab = ctx->memory; g.a_tab_cols = d; }
   rc = launch_gemm(ctx, g, "kv_proj", s);
   if (rc) return rc;
   g = GemmArgs{};

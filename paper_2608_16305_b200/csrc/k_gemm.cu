@@ -95,6 +95,7 @@ int launch_gemm(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t
     const int rc = launch_gemm_tf32(ctx, gp, name, s);
     if (rc != 1) return rc;  // 1: shape not handled by the tensor-core kernel, use the FMA tiles
   }
+  if (g.a_idx) return set_error(ctx, TGNN_EINVAL, "gemm %s: row-indirect A needs the tensor-core path", name);
   dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.split_k < 1 ? 1 : g.split_k);
   GemmArgs a = g;
   if (a.split_k < 1) a.split_k = 1;

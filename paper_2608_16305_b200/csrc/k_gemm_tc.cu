@@ -53,6 +53,12 @@ struct TcArgs {
   // kb at b_image + x * b_tile_stride + kb * (COPIES * B_BYTES); nullptr: B goes through registers
   const unsigned char* b_image;
   int64_t b_tile_stride;
+  // Row-indirect leading columns of a K-major A: A(m, k) for k < a_tab_cols is a_tab[a_idx[m] * a_tab_cols + k]
+  // (zero if a_idx[m] < 0) instead of A[m * lda + k]; nullptr: plain A.  Lets the key/value projection
+  // read the neighbors' memory rows straight from the table.
+  const int32_t* a_idx;
+  const float* a_tab;
+  int a_tab_cols;
 };
 
 template <int BN_T, bool PRECISE>
@@ -144,7 +150,9 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 // while it waits for a free stage and stores the current one.
 template <int ROWS_MAX>
 __device__ __forceinline__ void load_regs(float4 (&v)[ROWS_MAX * 8 / GROUP], const float* __restrict__ P, int64_t ld,
-                                          int major, int r0, int R, int rows_t, int k0, int k1, bool vec, int t) {
+                                          int major, int r0, int R, int rows_t, int k0, int k1, bool vec, int t,
+                                          const int32_t* tab_row = nullptr, const float* __restrict__ tab = nullptr,
+                                          int tab_cols = 0) {
   constexpr int ITERS = ROWS_MAX * 8 / GROUP;
   if (major == MAJOR_K) {
 #pragma unroll
@@ -155,6 +163,10 @@ __device__ __forceinline__ void load_regs(float4 (&v)[ROWS_MAX * 8 / GROUP], con
       v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
       if (r < rows_t && gr < R && gk < k1) {
         const float* p = P + (int64_t)gr * ld + gk;
+        if (tab_row != nullptr && gk < tab_cols) {  // tab_cols is a multiple of 4: the chunk is all table or all A
+          if (tab_row[i] < 0) continue;
+          p = tab + (int64_t)tab_row[i] * tab_cols + gk;
+        }
         if (vec && gk + 3 < k1) {
           v[i] = ldg_v4(p);
         } else {
@@ -314,10 +326,23 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kern
     // The A registers of the group's next block are loaded before it waits for the current stage,
     // so that round trip overlaps the wait, the stores and the MMAs of the blocks in between.
     float4 va[BM * 8 / GROUP], vn[BM * 8 / GROUP];
-    if (grp < nkb) load_regs<BM>(va, g.A, g.lda, g.a_major, m0, M, BM, (kb0 + grp) * BK, k_end, a_vec, t);
+    int32_t tab_row[BM * 8 / GROUP];  // table row of each of the thread's A rows (row-indirect mode)
+    const int32_t* trp = nullptr;
+    if (g.a_idx != nullptr && g.a_major == MAJOR_K) {
+#pragma unroll
+      for (int q = 0; q < BM * 8 / GROUP; ++q) {
+        const int gr = m0 + ((t + q * GROUP) >> 3);
+        tab_row[q] = gr < M ? g.a_idx[gr] : -1;
+      }
+      trp = tab_row;
+    }
+    if (grp < nkb)
+      load_regs<BM>(va, g.A, g.lda, g.a_major, m0, M, BM, (kb0 + grp) * BK, k_end, a_vec, t, trp, g.a_tab, g.a_tab_cols);
     for (int i = grp; i < nkb; i += GROUPS) {
       const int s = i % STAGES;
-      if (i + GROUPS < nkb) load_regs<BM>(vn, g.A, g.lda, g.a_major, m0, M, BM, (kb0 + i + GROUPS) * BK, k_end, a_vec, t);
+      if (i + GROUPS < nkb)
+        load_regs<BM>(vn, g.A, g.lda, g.a_major, m0, M, BM, (kb0 + i + GROUPS) * BK, k_end, a_vec, t, trp, g.a_tab,
+                      g.a_tab_cols);
       if (i >= STAGES) {
         ok = mbar_wait(smem_u32(&s_empty[s]), ((i / STAGES) - 1) & 1);
         if (!ok) break;
@@ -565,6 +590,11 @@ int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStr
   a.M = g.M; a.N = g.N; a.K = g.K; a.dev_M = g.dev_M; a.dev_K = g.dev_K;
   a.bias = g.bias; a.rowsum_out = g.rowsum_out; a.relu = g.relu; a.accumulate = g.accumulate;
   a.status = ctx->ws.status;
+  if (g.a_idx && a.a_major == MAJOR_K && g.a_tab_cols % 4 == 0 && (((uintptr_t)g.a_tab & 15) == 0)) {
+    a.a_idx = g.a_idx; a.a_tab = g.a_tab; a.a_tab_cols = g.a_tab_cols;
+  } else if (g.a_idx) {
+    return 1;
+  }
   int n_tiles, bn;
   bool precise = g.precise != 0;
   tile_plan(g.M, g.N, g.accumulate && g.split_k > 1, &n_tiles, &bn);

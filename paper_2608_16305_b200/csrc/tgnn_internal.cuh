@@ -308,6 +308,9 @@ struct GemmArgs {
   int relu;               // apply ReLU in the epilogue (store mode only)
   int accumulate;         // atomicAdd into C (C must hold valid data); required when split_k > 1
   int split_k;            // >= 1
+  const int32_t* a_idx;   // optional (tensor-core path, K-major A): leading a_tab_cols columns of row m come from
+  const float* a_tab;     //   a_tab[a_idx[m] * a_tab_cols + k] (zero row if a_idx[m] < 0) instead of A
+  int a_tab_cols;
   int site;               // WeightSiteId + 1 when B is that weight matrix (0: none); lets the kernel use its image
   int precise;            // tensor-core mode only: 3xTF32 head/tail split, close to fp32 accuracy
 };
