@@ -33,6 +33,7 @@ constexpr int BM = 128;    // rows of C per CTA (UMMA M)
 constexpr int BK = 32;     // contraction elements per stage: one 128-byte swizzle row of fp32
 constexpr int UMMA_K = 8;  // tf32
 constexpr int GROUP = 128; // threads per producer group
+constexpr int EPI_PITCH = 36;  // floats between rows of an epilogue staging square (16-byte aligned, bank-staggered)
 constexpr unsigned SPIN_LIMIT = 1u << 24;
 constexpr unsigned FULL = 0xffffffffu;
 
@@ -148,32 +149,44 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 // rows_t is a multiple of 32 (MN-major) or of 8 (K-major); chunks outside the valid range are zero.
 // The tile is filled in two steps so that a producer can have the loads of its next block in flight
 // while it waits for a free stage and stores the current one.
-template <int ROWS_MAX>
-__device__ __forceinline__ void load_regs(float4 (&v)[ROWS_MAX * 8 / GROUP], const float* __restrict__ P, int64_t ld,
-                                          int major, int r0, int R, int rows_t, int k0, int k1, bool vec, int t,
-                                          const int32_t* tab_row = nullptr, const float* __restrict__ tab = nullptr,
-                                          int tab_cols = 0) {
+// FAST (every chunk is wholly inside or wholly outside the operand, pointers 16-byte aligned): the
+// loads are unconditional -- an out-of-range chunk reads the operand's first chunk instead and is
+// zeroed at store time from the returned mask -- so nothing between the loads depends on a loaded
+// value and all of a block's round trips overlap.  Otherwise chunks are read element by element
+// under their bounds checks.
+template <int ROWS_MAX, bool FAST>
+__device__ __forceinline__ uint32_t load_regs(float4 (&v)[ROWS_MAX * 8 / GROUP], const float* __restrict__ P, int64_t ld,
+                                              int major, int r0, int R, int rows_t, int k0, int k1, bool vec, int t,
+                                              const int32_t* tab_row = nullptr, const float* __restrict__ tab = nullptr,
+                                              int tab_cols = 0) {
   constexpr int ITERS = ROWS_MAX * 8 / GROUP;
+  uint32_t mask = 0;
   if (major == MAJOR_K) {
 #pragma unroll
     for (int i = 0; i < ITERS; ++i) {
       const int idx = t + i * GROUP;
       const int r = idx >> 3, c = idx & 7;
       const int gr = r0 + r, gk = k0 + 4 * c;
-      v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (r < rows_t && gr < R && gk < k1) {
-        const float* p = P + (int64_t)gr * ld + gk;
-        if (tab_row != nullptr && gk < tab_cols) {  // tab_cols is a multiple of 4: the chunk is all table or all A
-          if (tab_row[i] < 0) continue;
-          p = tab + (int64_t)tab_row[i] * tab_cols + gk;
-        }
-        if (vec && gk + 3 < k1) {
-          v[i] = ldg_v4(p);
-        } else {
-          v[i].x = ldg_f(p);
-          if (gk + 1 < k1) v[i].y = ldg_f(p + 1);
-          if (gk + 2 < k1) v[i].z = ldg_f(p + 2);
-          if (gk + 3 < k1) v[i].w = ldg_f(p + 3);
+      bool valid = r < rows_t && gr < R && gk < k1;
+      const float* p = P + (int64_t)gr * ld + gk;
+      if (tab_row != nullptr && gk < tab_cols) {  // tab_cols is a multiple of 4: the chunk is all table or all A
+        valid = valid && tab_row[i] >= 0;
+        p = tab + (int64_t)tab_row[i] * tab_cols + gk;
+      }
+      if (FAST) {
+        v[i] = ldg_v4(valid ? p : P);
+        mask |= (valid ? 1u : 0u) << i;
+      } else {
+        v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid) {
+          if (vec && gk + 3 < k1) {
+            v[i] = ldg_v4(p);
+          } else {
+            v[i].x = ldg_f(p);
+            if (gk + 1 < k1) v[i].y = ldg_f(p + 1);
+            if (gk + 2 < k1) v[i].z = ldg_f(p + 2);
+            if (gk + 3 < k1) v[i].w = ldg_f(p + 3);
+          }
         }
       }
     }
@@ -184,32 +197,40 @@ __device__ __forceinline__ void load_regs(float4 (&v)[ROWS_MAX * 8 / GROUP], con
       const int idx = t + i * GROUP;
       const int kk = idx / cpr, cm = idx - kk * cpr;
       const int gk = k0 + kk, gr = r0 + 4 * cm;
-      v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (kk < BK && gk < k1 && gr < R) {
-        const float* p = P + (int64_t)gk * ld + gr;
-        if (vec && gr + 3 < R) {
-          v[i] = ldg_v4(p);
-        } else {
-          v[i].x = ldg_f(p);
-          if (gr + 1 < R) v[i].y = ldg_f(p + 1);
-          if (gr + 2 < R) v[i].z = ldg_f(p + 2);
-          if (gr + 3 < R) v[i].w = ldg_f(p + 3);
+      const bool valid = kk < BK && gk < k1 && gr < R;
+      const float* p = P + (int64_t)gk * ld + gr;
+      if (FAST) {
+        v[i] = ldg_v4(valid ? p : P);
+        mask |= (valid ? 1u : 0u) << i;
+      } else {
+        v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid) {
+          if (vec && gr + 3 < R) {
+            v[i] = ldg_v4(p);
+          } else {
+            v[i].x = ldg_f(p);
+            if (gr + 1 < R) v[i].y = ldg_f(p + 1);
+            if (gr + 2 < R) v[i].z = ldg_f(p + 2);
+            if (gr + 3 < R) v[i].w = ldg_f(p + 3);
+          }
         }
       }
     }
   }
+  return FAST ? mask : 0xffffffffu;
 }
 
 template <int ROWS_MAX, bool PRECISE>
-__device__ __forceinline__ void store_regs(const float4 (&v)[ROWS_MAX * 8 / GROUP], uint32_t tile, uint32_t tail_offset,
-                                           int major, int rows_t, int t, float4* rowsum) {
+__device__ __forceinline__ void store_regs(const float4 (&v)[ROWS_MAX * 8 / GROUP], uint32_t mask, uint32_t tile,
+                                           uint32_t tail_offset, int major, int rows_t, int t, float4* rowsum) {
   constexpr int ITERS = ROWS_MAX * 8 / GROUP;
   if (major == MAJOR_K) {
 #pragma unroll
     for (int i = 0; i < ITERS; ++i) {
       const int idx = t + i * GROUP;
       const int r = idx >> 3, c = idx & 7;
-      if (r < rows_t) store_chunk<PRECISE>(tile + (r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4), tail_offset, v[i]);
+      const float4 x = (mask >> i) & 1u ? v[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+      if (r < rows_t) store_chunk<PRECISE>(tile + (r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4), tail_offset, x);
     }
   } else {
     const int cpr = rows_t >> 2;
@@ -220,23 +241,24 @@ __device__ __forceinline__ void store_regs(const float4 (&v)[ROWS_MAX * 8 / GROU
       const int kk = idx / cpr, cm = idx - kk * cpr;
       if (kk < BK) {
         const int a = cm >> 3, c = cm & 7;
+        const float4 x = (mask >> i) & 1u ? v[i] : make_float4(0.f, 0.f, 0.f, 0.f);
         store_chunk<PRECISE>(tile + (kk >> 2) * (atoms * 512) + a * 512 + (kk & 3) * 128 + ((c ^ ((kk & 3) << 1)) << 4),
-                             tail_offset, v[i]);
+                             tail_offset, x);
         if (rowsum && rows_t == BM) {  // cm == t % 32 for every i: per-thread sums of 4 rows of C
-          rowsum->x += v[i].x; rowsum->y += v[i].y; rowsum->z += v[i].z; rowsum->w += v[i].w;
+          rowsum->x += x.x; rowsum->y += x.y; rowsum->z += x.z; rowsum->w += x.w;
         }
       }
     }
   }
 }
 
-template <int ROWS_MAX, bool PRECISE>
+template <int ROWS_MAX, bool PRECISE, bool FAST>
 __device__ __forceinline__ void load_tile(uint32_t tile, uint32_t tail_offset, const float* __restrict__ P, int64_t ld,
                                           int major, int r0, int R, int rows_t, int k0, int k1, bool vec, int t,
                                           float4* rowsum) {
   float4 v[ROWS_MAX * 8 / GROUP];
-  load_regs<ROWS_MAX>(v, P, ld, major, r0, R, rows_t, k0, k1, vec, t);
-  store_regs<ROWS_MAX, PRECISE>(v, tile, tail_offset, major, rows_t, t, rowsum);
+  const uint32_t mask = load_regs<ROWS_MAX, FAST>(v, P, ld, major, r0, R, rows_t, k0, k1, vec, t);
+  store_regs<ROWS_MAX, PRECISE>(v, mask, tile, tail_offset, major, rows_t, t, rowsum);
 }
 
 __device__ __forceinline__ void mma_tf32(uint32_t tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
@@ -249,7 +271,7 @@ __device__ __forceinline__ void mma_tf32(uint32_t tmem, uint64_t da, uint64_t db
 }
 
 // grid: (n tiles, m tiles, split_k).  Dynamic shared memory: Cfg::SMEM bytes.
-template <int BN_T, bool PRECISE>
+template <int BN_T, bool PRECISE, bool FAST>
 __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kernel(TcArgs g) {
   using C_ = Cfg<BN_T, PRECISE>;
   constexpr int STAGES = C_::STAGES, GROUPS = C_::GROUPS, THREADS = C_::THREADS;
@@ -336,13 +358,15 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kern
       }
       trp = tab_row;
     }
+    uint32_t ma = 0, mn = 0;
     if (grp < nkb)
-      load_regs<BM>(va, g.A, g.lda, g.a_major, m0, M, BM, (kb0 + grp) * BK, k_end, a_vec, t, trp, g.a_tab, g.a_tab_cols);
+      ma = load_regs<BM, FAST>(va, g.A, g.lda, g.a_major, m0, M, BM, (kb0 + grp) * BK, k_end, a_vec, t, trp, g.a_tab,
+                               g.a_tab_cols);
     for (int i = grp; i < nkb; i += GROUPS) {
       const int s = i % STAGES;
       if (i + GROUPS < nkb)
-        load_regs<BM>(vn, g.A, g.lda, g.a_major, m0, M, BM, (kb0 + i + GROUPS) * BK, k_end, a_vec, t, trp, g.a_tab,
-                      g.a_tab_cols);
+        mn = load_regs<BM, FAST>(vn, g.A, g.lda, g.a_major, m0, M, BM, (kb0 + i + GROUPS) * BK, k_end, a_vec, t, trp,
+                                 g.a_tab, g.a_tab_cols);
       if (i >= STAGES) {
         ok = mbar_wait(smem_u32(&s_empty[s]), ((i / STAGES) - 1) & 1);
         if (!ok) break;
@@ -361,13 +385,14 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kern
                        : "memory");
         }
       }
-      store_regs<BM, PRECISE>(va, a_tile, C_::A_BYTES, g.a_major, BM, t, want_rowsum ? &rs : nullptr);
+      store_regs<BM, PRECISE>(va, ma, a_tile, C_::A_BYTES, g.a_major, BM, t, want_rowsum ? &rs : nullptr);
       if (g.b_image == nullptr)
-        load_tile<BN_T, PRECISE>(b_tile, C_::B_BYTES, g.B, g.ldb, g.b_major, n0, g.N, b_rows, k0, k_end, b_vec, t, nullptr);
+        load_tile<BN_T, PRECISE, FAST>(b_tile, C_::B_BYTES, g.B, g.ldb, g.b_major, n0, g.N, b_rows, k0, k_end, b_vec, t, nullptr);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       mbar_arrive(smem_u32(&s_full[s]));
 #pragma unroll
       for (int q = 0; q < BM * 8 / GROUP; ++q) va[q] = vn[q];
+      ma = mn;
     }
     if (!ok) { s_abort = 1; atomicCAS(g.status, 0, TGNN_ETIMEOUT); }
     if (want_rowsum) {  // the thread's chunks cover rows 4*(t%32) .. +3 of the tile
@@ -382,55 +407,71 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kern
     asm volatile("bar.sync 1, %0;" ::"n"(GROUPS * GROUP) : "memory");  // all producers: s_rowsum complete
     if (want_rowsum && tid < BM && m0 + tid < M && s_rowsum[tid] != 0.f) atomicAdd(&g.rowsum_out[m0 + tid], s_rowsum[tid]);
     if (__all_sync(FULL, ok && !s_abort)) {  // warp-uniform: the TMEM loads are warp-collective
-      const int q4 = warp & 3;               // the TMEM lane quarter this warp may access
-      const int row = m0 + q4 * 32 + lane;
+      // Each warp moves 32 rows x 32 columns at a time: TMEM -> registers (one row per lane) -> its
+      // own staging square in the now idle pipeline memory -> global, re-read so that 8 lanes cover
+      // 128 contiguous bytes of one row of C (whole sectors per request; a lane-per-row store would
+      // touch 32 rows with 16 bytes each).
+      const int q4 = warp & 3;  // the TMEM lane quarter this warp may access
       const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16);
-      const bool c_vec = (((uintptr_t)g.C & 15) == 0) && (g.ldc % 4 == 0) && (n0 % 4 == 0);
-      for (int c0 = grp * 16; c0 < n_mma; c0 += GROUPS * 16) {
-        uint32_t r[16];
+      float* stg = reinterpret_cast<float*>(smem) + warp * (32 * EPI_PITCH);
+      const bool c_vec = (((uintptr_t)g.C & 15) == 0) && (g.ldc % 4 == 0);
+      const int sub = lane >> 3, ch = lane & 7;
+      for (int c0 = grp * 32; c0 < n_valid; c0 += GROUPS * 32) {
+        uint32_t r[32];
         asm volatile(
-            "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+            "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+            "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
             : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-              "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+              "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+              "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+              "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
             : "r"(taddr + (uint32_t)c0));
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (row < M) {
-          float* crow = g.C + (int64_t)row * g.ldc + n0 + c0;
 #pragma unroll
-          for (int q = 0; q < 16; q += 4) {
-            if (c0 + q >= n_valid) break;
-            float4 v = make_float4(__uint_as_float(r[q]), __uint_as_float(r[q + 1]), __uint_as_float(r[q + 2]),
-                                   __uint_as_float(r[q + 3]));
-            if (g.bias && blockIdx.z == 0) {
-              const float* bp = g.bias + n0 + c0 + q;
-              v.x += bp[0];
-              if (c0 + q + 1 < n_valid) v.y += bp[1];
-              if (c0 + q + 2 < n_valid) v.z += bp[2];
-              if (c0 + q + 3 < n_valid) v.w += bp[3];
-            }
-            const bool full4 = c0 + q + 3 < n_valid;
+        for (int q = 0; q < 8; ++q)
+          *reinterpret_cast<uint4*>(stg + lane * EPI_PITCH + 4 * q) = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+        __syncwarp();
+        const int col = c0 + 4 * ch;  // first of this lane's 4 columns, relative to the tile
+        float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (g.bias && blockIdx.z == 0 && col < n_valid) {
+          const float* bp = g.bias + n0 + col;
+          b4.x = bp[0];
+          if (col + 1 < n_valid) b4.y = bp[1];
+          if (col + 2 < n_valid) b4.z = bp[2];
+          if (col + 3 < n_valid) b4.w = bp[3];
+        }
+        const bool full4 = col + 3 < n_valid;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int rr = j * 4 + sub;
+          const int row = m0 + q4 * 32 + rr;
+          float4 v = *reinterpret_cast<const float4*>(stg + rr * EPI_PITCH + 4 * ch);
+          if (row < M && col < n_valid) {
+            v.x += b4.x; v.y += b4.y; v.z += b4.z; v.w += b4.w;
+            float* cp = g.C + (int64_t)row * g.ldc + n0 + col;
             if (g.accumulate) {
               if (full4 && c_vec) {
-                atomicAdd(reinterpret_cast<float4*>(crow + q), v);
+                atomicAdd(reinterpret_cast<float4*>(cp), v);
               } else {
-                atomicAdd(crow + q, v.x);
-                if (c0 + q + 1 < n_valid) atomicAdd(crow + q + 1, v.y);
-                if (c0 + q + 2 < n_valid) atomicAdd(crow + q + 2, v.z);
-                if (c0 + q + 3 < n_valid) atomicAdd(crow + q + 3, v.w);
+                atomicAdd(cp, v.x);
+                if (col + 1 < n_valid) atomicAdd(cp + 1, v.y);
+                if (col + 2 < n_valid) atomicAdd(cp + 2, v.z);
+                if (col + 3 < n_valid) atomicAdd(cp + 3, v.w);
               }
             } else {
               if (g.relu) { v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); v.z = fmaxf(v.z, 0.f); v.w = fmaxf(v.w, 0.f); }
               if (full4 && c_vec) {
-                *reinterpret_cast<float4*>(crow + q) = v;
+                *reinterpret_cast<float4*>(cp) = v;
               } else {
-                crow[q] = v.x;
-                if (c0 + q + 1 < n_valid) crow[q + 1] = v.y;
-                if (c0 + q + 2 < n_valid) crow[q + 2] = v.z;
-                if (c0 + q + 3 < n_valid) crow[q + 3] = v.w;
+                cp[0] = v.x;
+                if (col + 1 < n_valid) cp[1] = v.y;
+                if (col + 2 < n_valid) cp[2] = v.z;
+                if (col + 3 < n_valid) cp[3] = v.w;
               }
             }
           }
         }
+        __syncwarp();
       }
     }
   } else {
@@ -556,19 +597,19 @@ __global__ void __launch_bounds__(256) prep_weights_kernel(const WeightSite* __r
                    to_tf32(v[2] - __uint_as_float(h2)), to_tf32(v[3] - __uint_as_float(h3)));
 }
 
-template <int BN_T, bool PRECISE>
+template <int BN_T, bool PRECISE, bool FAST>
 int launch_tc(tgnn_ctx* ctx, const TcArgs& a, int n_tiles, const char* name, cudaStream_t s) {
   using C_ = Cfg<BN_T, PRECISE>;
   static bool attr_set = false;
   if (!attr_set) {
-    TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(gemm_tf32_kernel<BN_T, PRECISE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(gemm_tf32_kernel<BN_T, PRECISE, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            C_::SMEM));
     attr_set = true;
   }
   dim3 grid(n_tiles, (a.M + BM - 1) / BM, a.split_k);
   {
     KernelScope scope__(ctx, name, s);
-    gemm_tf32_kernel<BN_T, PRECISE><<<grid, C_::THREADS, C_::SMEM, s>>>(a);
+    gemm_tf32_kernel<BN_T, PRECISE, FAST><<<grid, C_::THREADS, C_::SMEM, s>>>(a);
   }
   TGNN_LAUNCH_OK(ctx, name);
   return TGNN_OK;
@@ -613,12 +654,25 @@ int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStr
     if (a.split_k > max_s) a.split_k = max_s;
     if (a.split_k < 1) a.split_k = 1;
   }
-  if (precise) {
-    if (bn <= 128) return launch_tc<128, true>(ctx, a, n_tiles, name, s);
-    return launch_tc<256, true>(ctx, a, n_tiles, name, s);
+  // whole-chunk operands: 16-byte aligned rows, and the dimension the 16-byte chunks run along is a
+  // multiple of 4 and known on the host
+  const auto whole = [](const float* p, int64_t ld, int major, int k, const int* dev_k, int mn, const int* dev_mn) {
+    if (((uintptr_t)p & 15) != 0 || ld % 4 != 0) return false;
+    return major == MAJOR_K ? (k % 4 == 0 && dev_k == nullptr) : (mn % 4 == 0 && dev_mn == nullptr);
+  };
+  const bool fast = whole(a.A, a.lda, a.a_major, a.K, a.dev_K, a.M, a.dev_M) &&
+                    (a.b_image != nullptr || whole(a.B, a.ldb, a.b_major, a.K, a.dev_K, a.N, nullptr));
+  const int sel = (precise ? 4 : 0) | (bn <= 128 ? 0 : 2) | (fast ? 1 : 0);
+  switch (sel) {
+    case 0: return launch_tc<128, false, false>(ctx, a, n_tiles, name, s);
+    case 1: return launch_tc<128, false, true>(ctx, a, n_tiles, name, s);
+    case 2: return launch_tc<256, false, false>(ctx, a, n_tiles, name, s);
+    case 3: return launch_tc<256, false, true>(ctx, a, n_tiles, name, s);
+    case 4: return launch_tc<128, true, false>(ctx, a, n_tiles, name, s);
+    case 5: return launch_tc<128, true, true>(ctx, a, n_tiles, name, s);
+    case 6: return launch_tc<256, true, false>(ctx, a, n_tiles, name, s);
+    default: return launch_tc<256, true, true>(ctx, a, n_tiles, name, s);
   }
-  if (bn <= 128) return launch_tc<128, false>(ctx, a, n_tiles, name, s);
-  return launch_tc<256, false>(ctx, a, n_tiles, name, s);
 }
 
 }  // namespace tgnn
