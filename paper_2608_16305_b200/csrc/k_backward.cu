@@ -100,6 +100,184 @@ __global__ void __launch_bounds__(256) dh_kernel(const float* __restrict__ dcat1
   }
 }
 
+// The whole link-prediction head for a group of 4 target events (8 pairs: 4 positive, 4 negative) in one
+// block: gather [h_a || h_b], hidden layer, scores, the masked loss (Eq. 13), and the backward pass down to
+// d loss / d pre_o of the 12 embedding rows involved.  W_1 stays in shared memory (row pitch 2d+1: both the
+// forward sweep, threads over hidden units, and the backward sweep, threads over input columns, are free
+// of bank conflicts) while the block walks over its groups.  Also leaves what the leaves of the chain
+// need: cat1 and d loss / d pre1 (for dW_1, db_1), the hidden gates, and the sums for dw_2, db_2 and the loss.
+// Rows of hsT: 0-3 source, 4-7 destination, 8-11 negative.  Dynamic shared memory: head_fused_smem(d) bytes.
+constexpr int HF_EV = 4, HF_THREADS = 512;
+__host__ __device__ inline int head_fused_w_floats(int d) { return (d * (2 * d + 1) + 3) & ~3; }
+inline size_t head_fused_smem(int d) {
+  return (size_t)(head_fused_w_floats(d) + 12 * d + 12 * d + 8 * d + 8 * 2 * d + d) * sizeof(float);
+}
+
+__global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __restrict__ h, const float* __restrict__ W1,
+                                                                const float* __restrict__ b1,
+                                                                const float* __restrict__ w2, const float* __restrict__ b2,
+                                                                const uint8_t* __restrict__ loss_mask, int nq, int d,
+                                                                float* __restrict__ cat1, float* __restrict__ dpre1,
+                                                                uint8_t* __restrict__ hid_gate,
+                                                                float* __restrict__ dpre_o, float* __restrict__ g_w2,
+                                                                float* __restrict__ g_b2, float* __restrict__ loss_acc) {
+  extern __shared__ __align__(16) float sm[];
+  __shared__ float s_msum, s_gb2, s_loss;
+  const int PW = 2 * d + 1;
+  float* W1s = sm;                              // [d][2d+1]
+  float* hsT = W1s + head_fused_w_floats(d);    // [d][12]   embedding rows, transposed
+  float* part = hsT + 12 * d;                   // [d][12]   W_1a h_src | W_1b h_dst | W_1b h_neg per event
+  float* dh1T = part + 12 * d;                  // [d][8]    d loss / d pre1, transposed
+  float* dc = dh1T + 8 * d;                     // [2d][8]   partial input gradients of the lower half of j
+  float* gw2 = dc + 16 * d;                     // [d]
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  {  // W_1 [d][2d] -> padded rows; 2d is a multiple of 4 and the parameter block is 16-byte aligned
+    const int n4 = d * 2 * d / 4, row4 = 2 * d / 4;
+    const bool vec = (((uintptr_t)W1) & 15) == 0;
+    for (int e = tid; e < n4; e += blockDim.x) {
+      const int j = e / row4, c = 4 * (e - j * row4);
+      float4 v;
+      if (vec) v = __ldg(reinterpret_cast<const float4*>(W1) + e);
+      else v = make_float4(W1[4 * e], W1[4 * e + 1], W1[4 * e + 2], W1[4 * e + 3]);
+      float* dst = W1s + j * PW + c;
+      dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+    }
+  }
+  for (int q = tid; q < d; q += blockDim.x) gw2[q] = 0.f;
+  if (tid == 0) { s_msum = 0.f; s_gb2 = 0.f; s_loss = 0.f; }
+  __syncthreads();
+  {  // every block counts the whole mask (a few KB)
+    int c = 0;
+    for (int j = tid; j < nq; j += blockDim.x) c += loss_mask ? (loss_mask[j] != 0) : 1;
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(FULL, c, o);
+    if (lane == 0 && c) atomicAdd(&s_msum, (float)c);
+  }
+  __syncthreads();
+  const float msum = s_msum;
+  const float bias2 = b2[0];
+  const int groups = (nq + HF_EV - 1) / HF_EV;
+  for (int grp = blockIdx.x; grp < groups; grp += gridDim.x) {
+    const int ev0 = grp * HF_EV;
+    for (int e = tid; e < 12 * d; e += blockDim.x) {
+      const int r = e / d, q = e - r * d;
+      const int ev = ev0 + (r & 3), blk = r >> 2;
+      float v = 0.f;
+      if (ev < nq) {
+        v = h[((int64_t)blk * nq + ev) * d + q];
+        if (blk == 0) {
+          cat1[(int64_t)ev * 2 * d + q] = v;
+          cat1[(int64_t)(nq + ev) * 2 * d + q] = v;
+        } else if (blk == 1) {
+          cat1[(int64_t)ev * 2 * d + d + q] = v;
+        } else {
+          cat1[(int64_t)(nq + ev) * 2 * d + d + q] = v;
+        }
+      }
+      hsT[q * 12 + r] = v;
+    }
+    __syncthreads();
+    // hidden layer in three parts: a thread owns hidden unit j and one block of 4 embedding rows (the
+    // source rows serve the positive and the negative pair of their event, so their part is formed once)
+    for (int it = tid; it < 3 * d; it += blockDim.x) {
+      const int blk = it / d, j = it - blk * d;
+      const float* wr = W1s + j * PW + (blk ? d : 0);
+      const float* hb = hsT + 4 * blk;
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 4
+      for (int c = 0; c < d; ++c) {
+        const float x = wr[c];
+        const float4 v = *reinterpret_cast<const float4*>(hb + c * 12);
+        a0 = fmaf(x, v.x, a0); a1 = fmaf(x, v.y, a1); a2 = fmaf(x, v.z, a2); a3 = fmaf(x, v.w, a3);
+      }
+      *reinterpret_cast<float4*>(part + j * 12 + 4 * blk) = make_float4(a0, a1, a2, a3);
+    }
+    __syncthreads();
+    // scores, loss terms and d loss / d pre1: one warp per pair
+    for (int p = wid; p < 8; p += (blockDim.x >> 5)) {
+      const int half = p >> 2, e4 = p & 3, ev = ev0 + e4;
+      const bool valid = ev < nq;
+      const int o_col = 4 + 4 * half + e4;  // the pair's second row: destination or negative
+      float sc = 0.f;
+      for (int q = lane; q < d; q += 32) {
+        const float a = fmaxf(part[q * 12 + e4] + part[q * 12 + o_col] + b1[q], 0.f);
+        sc = fmaf(w2[q], a, sc);
+      }
+      for (int o = 16; o > 0; o >>= 1) sc += __shfl_xor_sync(FULL, sc, o);
+      sc += bias2;
+      const float m = valid && (loss_mask ? (loss_mask[ev] != 0) : true) ? 1.f : 0.f;
+      const float wj = msum > 0.f ? m / msum : 0.f;
+      const float ds = half == 0 ? -wj * sigmoidf_(-sc) : wj * sigmoidf_(sc);
+      if (lane == 0 && wj != 0.f) {
+        atomicAdd(&s_loss, wj * (half == 0 ? softplusf_(-sc) : softplusf_(sc)));
+        atomicAdd(&s_gb2, ds);
+      }
+      const int64_t row = (int64_t)half * nq + ev;
+      for (int q = lane; q < d; q += 32) {
+        const float a = fmaxf(part[q * 12 + e4] + part[q * 12 + o_col] + b1[q], 0.f);
+        if (wj != 0.f) atomicAdd(&gw2[q], ds * a);
+        const float dv = a > 0.f ? ds * w2[q] : 0.f;
+        dh1T[q * 8 + p] = dv;
+        if (valid) {
+          dpre1[row * d + q] = dv;
+          hid_gate[row * d + q] = a > 0.f;
+        }
+      }
+    }
+    __syncthreads();
+    // input gradient: a thread owns column c of [h_a || h_b] for all 8 pairs over one half of the hidden
+    // units; the lower half parks its sums in shared memory, the upper half adds them and folds the pairs
+    // into the embedding rows (the source row collects its positive and its negative pair)
+    const int jh = (d + 1) / 2;
+    for (int base = 0; base < 4 * d; base += blockDim.x) {  // items [0, 2d): lower half of j, [2d, 4d): upper half
+      const int it = base + tid;
+      const bool act = it < 4 * d;
+      const int hi = act ? it / (2 * d) : 0, c = act ? it - hi * 2 * d : 0;
+      float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      if (act) {
+        const int j0 = hi ? jh : 0, j1 = hi ? d : jh;
+#pragma unroll 4
+        for (int j = j0; j < j1; ++j) {
+          const float x = W1s[j * PW + c];
+          const float4 u = *reinterpret_cast<const float4*>(dh1T + j * 8);
+          const float4 v = *reinterpret_cast<const float4*>(dh1T + j * 8 + 4);
+          a[0] = fmaf(x, u.x, a[0]); a[1] = fmaf(x, u.y, a[1]); a[2] = fmaf(x, u.z, a[2]); a[3] = fmaf(x, u.w, a[3]);
+          a[4] = fmaf(x, v.x, a[4]); a[5] = fmaf(x, v.y, a[5]); a[6] = fmaf(x, v.z, a[6]); a[7] = fmaf(x, v.w, a[7]);
+        }
+        if (hi == 0) {
+          *reinterpret_cast<float4*>(dc + c * 8) = make_float4(a[0], a[1], a[2], a[3]);
+          *reinterpret_cast<float4*>(dc + c * 8 + 4) = make_float4(a[4], a[5], a[6], a[7]);
+        }
+      }
+      __syncthreads();
+      if (act && hi == 1) {
+        const float4 u = *reinterpret_cast<const float4*>(dc + c * 8);
+        const float4 v = *reinterpret_cast<const float4*>(dc + c * 8 + 4);
+        a[0] += u.x; a[1] += u.y; a[2] += u.z; a[3] += u.w;
+        a[4] += v.x; a[5] += v.y; a[6] += v.z; a[7] += v.w;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int ev = ev0 + e;
+          if (ev >= nq) break;
+          if (c < d) {
+            dpre_o[(int64_t)ev * d + c] = hsT[c * 12 + e] > 0.f ? a[e] + a[4 + e] : 0.f;
+          } else {
+            const int q = c - d;
+            dpre_o[((int64_t)nq + ev) * d + q] = hsT[q * 12 + 4 + e] > 0.f ? a[e] : 0.f;
+            dpre_o[((int64_t)2 * nq + ev) * d + q] = hsT[q * 12 + 8 + e] > 0.f ? a[4 + e] : 0.f;
+          }
+        }
+      }
+    }
+    __syncthreads();
+  }
+  for (int q = tid; q < d; q += blockDim.x)
+    if (gw2[q] != 0.f) atomicAdd(&g_w2[q], gw2[q]);
+  if (tid == 0) {
+    if (s_gb2 != 0.f) atomicAdd(g_b2, s_gb2);
+    if (s_loss != 0.f) atomicAdd(loss_acc, s_loss);
+  }
+}
+
 // One warp per root: backward of the weighted sum, the softmax and the scaled dot products, on the
 // root's K | V rows staged in shared memory.  Lane p < H*k owns the (head, slot) pair p for the
 // probability and logit gradients; afterwards the lanes own columns and write dQ and the dK | dV rows.
@@ -205,17 +383,24 @@ __global__ void __launch_bounds__(256) scatter_dmem_kernel(const float* __restri
 // the forward pass (S == nullptr: every row has dt = 0, sin(arg) = sin(b_c)).
 //   dw_c += -S dt_r G,   db_c += -S G
 // The terms are large (dt reaches the time span of the stream) and cancel, so they are summed in
-// fp64.  Block = 8 warps over 64 rows; lanes own columns c = lane + 32 j; the warps' partial sums
+// fp64.  Block = 8 warps over rows_per_block rows; lanes own columns c = lane + 32 j; the warps' partial sums
 // meet in shared memory and leave as one pair of fp64 atomics per block and column into acc[0:d]
 // (dw) and acc[d:2d] (db).  Dynamic shared memory: 8 * 2 * d doubles.
-constexpr int TG_ROWS = 64, TG_MAXJ = 8;
+constexpr int TG_MAXJ = 8;
+// rows per block: 64 for long inputs, fewer (down to one per warp) when that is needed to fill the machine
+inline int tg_rows_per_block(int rows) {
+  int r = 64;
+  while (r > 8 && (rows + r - 1) / r < 296) r >>= 1;
+  return r;
+}
 __global__ void __launch_bounds__(256) time_grad_kernel(const float* __restrict__ G, int64_t ldg, int col0,
                                                         const float* __restrict__ S, const float* __restrict__ dt,
                                                         int rows, const int32_t* __restrict__ dev_rows, int d,
-                                                        const float* __restrict__ time_b, double* __restrict__ acc) {
+                                                        const float* __restrict__ time_b, double* __restrict__ acc,
+                                                        int rows_per_block) {
   extern __shared__ double s_part[];  // [8][2][d]
   const int R = dev_rows ? min(*dev_rows, rows) : rows;
-  const int r0 = blockIdx.x * TG_ROWS, r1 = min(R, r0 + TG_ROWS);
+  const int r0 = blockIdx.x * rows_per_block, r1 = min(R, r0 + rows_per_block);
   if (r0 >= r1) return;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   double gw[TG_MAXJ], gb[TG_MAXJ];
@@ -420,34 +605,55 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
   }
 
   if (n_q > 0) {
-    const int64_t tot = (int64_t)2 * n_q * 2 * d;
-    {
-      KernelScope scope__(ctx, "head_gather", s);
-      head_gather_kernel<<<(int)((tot + 255) / 256), 256, 0, s>>>(ctx->e_h, n_q, d, w.cat1);
+    // One block does the head forward and backward for 4 events at a time when W_1 fits in shared memory
+    // beside the staging rows; wider models take the projections through the GEMM path instead.
+    const size_t hf_smem = head_fused_smem(d);
+    if (hf_smem <= 200 * 1024) {
+      static size_t attr_bytes = 0;
+      if (attr_bytes < hf_smem) {
+        TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(head_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hf_smem));
+        attr_bytes = hf_smem;
+      }
+      const int groups = (n_q + HF_EV - 1) / HF_EV;
+      {
+        KernelScope scope__(ctx, "head_fused", s);
+        head_fused_kernel<<<groups < 296 ? groups : 296, HF_THREADS, hf_smem, s>>>(
+            ctx->e_h, P + L.w1, P + L.b1, P + L.w2, P + L.b2, loss_mask, n_q, d, w.cat1, w.hid1, w.hid_gate, w.dpre_o,
+            G + L.w2, G + L.b2, w.st_scalars);
+      }
+      TGNN_LAUNCH_OK(ctx, "head_fused");
+      RC(fork_to(ctx, s, sa));
+      RC(grad_w(ctx, w.hid1, d, w.cat1, 2 * d, 2 * n_q, nullptr, d, 2 * d, G + L.w1, G + L.b1, "dW_1", sa));
+    } else {
+      const int64_t tot = (int64_t)2 * n_q * 2 * d;
+      {
+        KernelScope scope__(ctx, "head_gather", s);
+        head_gather_kernel<<<(int)((tot + 255) / 256), 256, 0, s>>>(ctx->e_h, n_q, d, w.cat1);
+      }
+      TGNN_LAUNCH_OK(ctx, "head_gather");
+      GemmArgs g = {};
+      g.A = w.cat1; g.a_rs = 2 * d; g.a_cs = 1;
+      g.B = P + L.w1; g.b_rs = 1; g.b_cs = 2 * d;
+      g.C = w.hid1; g.ldc = d; g.M = 2 * n_q; g.N = d; g.K = 2 * d; g.bias = P + L.b1; g.relu = 1; g.split_k = 1;
+      g.site = SITE_HEAD + 1;
+      RC(launch_gemm(ctx, g, "head_hidden", s));
+      {
+        KernelScope scope__(ctx, "head_loss", s);
+        head_loss_kernel<<<(n_q + 7) / 8, 256, d * sizeof(float), s>>>(w.hid1, P + L.w2, P + L.b2, loss_mask, n_q, d,
+                                                                       G + L.w2, G + L.b2, w.st_scalars, w.hid_gate);
+      }
+      TGNN_LAUNCH_OK(ctx, "head_loss");
+      // hid1 now holds d loss / d pre1
+      RC(fork_to(ctx, s, sa));
+      RC(grad_w(ctx, w.hid1, d, w.cat1, 2 * d, 2 * n_q, nullptr, d, 2 * d, G + L.w1, G + L.b1, "dW_1", sa));
+      RC(grad_in(ctx, w.hid1, d, P + L.w1, 2 * d, 0, 2 * n_q, nullptr, d, 2 * d, w.dcat1, 2 * d, "dcat1", s, SITE_DCAT1 + 1));
+      const int64_t tot2 = (int64_t)R * d;
+      {
+        KernelScope scope__(ctx, "dh", s);
+        dh_kernel<<<(int)((tot2 + 255) / 256), 256, 0, s>>>(w.dcat1, ctx->e_h, n_q, d, w.dpre_o);
+      }
+      TGNN_LAUNCH_OK(ctx, "dh");
     }
-    TGNN_LAUNCH_OK(ctx, "head_gather");
-    GemmArgs g = {};
-    g.A = w.cat1; g.a_rs = 2 * d; g.a_cs = 1;
-    g.B = P + L.w1; g.b_rs = 1; g.b_cs = 2 * d;
-    g.C = w.hid1; g.ldc = d; g.M = 2 * n_q; g.N = d; g.K = 2 * d; g.bias = P + L.b1; g.relu = 1; g.split_k = 1;
-    g.site = SITE_HEAD + 1;
-    RC(launch_gemm(ctx, g, "head_hidden", s));
-    {
-      KernelScope scope__(ctx, "head_loss", s);
-      head_loss_kernel<<<(n_q + 7) / 8, 256, d * sizeof(float), s>>>(w.hid1, P + L.w2, P + L.b2, loss_mask, n_q, d,
-                                                                     G + L.w2, G + L.b2, w.st_scalars, w.hid_gate);
-    }
-    TGNN_LAUNCH_OK(ctx, "head_loss");
-    // hid1 now holds d loss / d pre1
-    RC(fork_to(ctx, s, sa));
-    RC(grad_w(ctx, w.hid1, d, w.cat1, 2 * d, 2 * n_q, nullptr, d, 2 * d, G + L.w1, G + L.b1, "dW_1", sa));
-    RC(grad_in(ctx, w.hid1, d, P + L.w1, 2 * d, 0, 2 * n_q, nullptr, d, 2 * d, w.dcat1, 2 * d, "dcat1", s, SITE_DCAT1 + 1));
-    const int64_t tot2 = (int64_t)R * d;
-    {
-      KernelScope scope__(ctx, "dh", s);
-      dh_kernel<<<(int)((tot2 + 255) / 256), 256, 0, s>>>(w.dcat1, ctx->e_h, n_q, d, w.dpre_o);
-    }
-    TGNN_LAUNCH_OK(ctx, "dh");
     RC(fork_to(ctx, s, sb));
     RC(grad_w(ctx, w.dpre_o, d, w.cat_o, 2 * d, R, nullptr, d, 2 * d, G + L.wo, G + L.bo, "dW_o", sb));
     RC(grad_in(ctx, w.dpre_o, d, P + L.wo, 2 * d, 0, R, nullptr, d, 2 * d, w.dcat_o, 2 * d, "dcat_o", s, SITE_DCATO + 1));
@@ -481,8 +687,9 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     RC(grad_w(ctx, w.dQ, d, w.Zq, 2 * d, R, nullptr, d, 2 * d, G + L.wq, G + L.bq, "dW_q", sb));
     {
       KernelScope scope__(ctx, "time_grad_q", sb);
-      time_grad_kernel<<<(R + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, sb>>>(w.dzq, 2 * d, d, nullptr, nullptr, R, nullptr, d,
-                                                                          P + L.time_b, w.tg_acc);
+      const int rpb = tg_rows_per_block(R);
+      time_grad_kernel<<<(R + rpb - 1) / rpb, 256, tg_smem, sb>>>(w.dzq, 2 * d, d, nullptr, nullptr, R, nullptr, d,
+                                                                  P + L.time_b, w.tg_acc, rpb);
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_q");
     cudaStream_t s_tgz = sb;  // where the time-encoder sum over the neighbor rows runs
@@ -495,8 +702,9 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     }
     {
       KernelScope scope__(ctx, "time_grad_z", s_tgz);
-      time_grad_kernel<<<(NB + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, s_tgz>>>(w.dZmp, 2 * d, d, w.Zsin, w.z_dt, NB, nullptr,
-                                                                              d, P + L.time_b, w.tg_acc);
+      const int rpb = tg_rows_per_block(NB);
+      time_grad_kernel<<<(NB + rpb - 1) / rpb, 256, tg_smem, s_tgz>>>(w.dZmp, 2 * d, d, w.Zsin, w.z_dt, NB, nullptr, d,
+                                                                      P + L.time_b, w.tg_acc, rpb);
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_z");
     RC(wait_mark(ctx, s, dzq_done));  // the scatter below needs dzq
@@ -527,8 +735,9 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
                  "dX_phi", s, SITE_DXPHI + 1));
       {
         KernelScope scope__(ctx, "time_grad_x", s);
-        time_grad_kernel<<<(U_cap + TG_ROWS - 1) / TG_ROWS, 256, tg_smem, s>>>(w.dXp, d, 0, w.Xsin, w.x_dt, U_cap,
-                                                                             ctx->upd_n_uniq, d, P + L.time_b, w.tg_acc);
+        const int rpb = tg_rows_per_block(U_cap);
+        time_grad_kernel<<<(U_cap + rpb - 1) / rpb, 256, tg_smem, s>>>(w.dXp, d, 0, w.Xsin, w.x_dt, U_cap, ctx->upd_n_uniq,
+                                                                       d, P + L.time_b, w.tg_acc, rpb);
       }
       TGNN_LAUNCH_OK(ctx, "time_grad_x");
     }

@@ -420,6 +420,18 @@ def test_scaled_configs_teacher_forced(B, oracle, name, events, at, math):
 
 
 @pytest.mark.parametrize("math", ["fp32", "tf32"])
+@pytest.mark.parametrize("d,batch", [
+    (160, 150),   # W_1 no longer fits in shared memory: the head runs as separate projection kernels
+    (100, 150),   # fused head, last group of 4 events ragged (150 = 37 * 4 + 2)
+    (32, 2501),   # fused head walking several groups per block; odd batch
+])
+def test_head_paths_wide_and_ragged(B, oracle, math, d, batch):
+    c = wl.scaled(wl.CONFIGS["wiki"], num_events=4 * batch, num_nodes=1200, num_src=1000, d=d, batch=batch)
+    rig = Rig(B, oracle, c, math=math)
+    _run_epoch_checks(rig, range(4), {1, 3})
+
+
+@pytest.mark.parametrize("math", ["fp32", "tf32"])
 def test_bf16_feature_table(B, oracle, math):
     c = wl.scaled(wl.CONFIGS["large"], num_events=20000, num_nodes=3000, batch=1000)
     rig = Rig(B, oracle, c, math=math)
