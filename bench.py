@@ -223,6 +223,24 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
     barrier()
     h2d_step, d2h_step = h2d / K, d2h / K
 
+    # ---- optional: the same steps under the adaptive runtime controller (Algorithm 2) ----
+    adaptive = None
+    if args.adaptive:
+        ctl = B.Controller(alpha=0.1, beta=0.1, tau_g=1.6, tau_c=0.5, K=6)
+        logs = []
+        reset_epoch()
+        ad_step = lambda b: logs.append(tr.step_adaptive(b, ctl))
+        run_steps(0, W, ad_step, False)
+        logs.clear()
+        ms_ad = run_steps(W, K, ad_step, True)
+        adaptive = {"value": K * cfg.batch / (ms_ad * 1e-3), "unit": UNIT, "ms_per_step": ms_ad / K,
+                    "heavy_batches": sum(l["heavy"] for l in logs),
+                    "boundaries": sum(l["boundary"] for l in logs),
+                    "refresh_skipped": sum(1 for l in logs if l["sync"] == 0),
+                    "constants": "K=6, tau_g=1.6, tau_c=0.5 (the paper's), alpha=beta=0.1 (unstated there)",
+                    "how": "Trainer.step_adaptive: controller decisions on the host, one synchronisation per step "
+                           "to read the gradient norm and the step's device time"}
+
     # ---- per-kernel times of the same K steps (separate pass: the event pairs perturb a latency-bound step) ----
     reset_epoch()
     run_steps(0, W, dev_step, False)
@@ -279,6 +297,8 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
                      "kernel_ms_total": round(tot, 3)},
         "loss_last": loss_end,
     }
+    if adaptive is not None:
+        out["adaptive"] = adaptive
     out["cpu_baseline"] = cpu_baseline(cfg, stream, weights, budget_s=args.cpu_budget) if args.cpu_budget > 0 else None
     print(json.dumps(out))
 
@@ -342,6 +362,8 @@ def main():
     ap.add_argument("--math", default=os.environ.get("TGNN_BENCH_MATH", "tf32"), choices=["fp32", "tf32", "tf32fast"])
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--workload", default=WORKLOAD, choices=sorted(wl.CONFIGS), help="default: the benchmark workload (wiki)")
+    ap.add_argument("--adaptive", action="store_true",
+                    help="also time the steps under the adaptive runtime controller (adds an 'adaptive' object)")
     ap.add_argument("--no-graph", action="store_true", help="launch kernel by kernel instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)

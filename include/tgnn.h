@@ -317,6 +317,35 @@ TGNN_API int tgnn_profile_report(tgnn_ctx* ctx, char* buf_host, int64_t size);
  * relative to the first recorded launch (the internal side streams make launches overlap). */
 TGNN_API int tgnn_profile_timeline(tgnn_ctx* ctx, char* buf_host, int64_t size);
 
+/* ---- adaptive runtime controller (Eq. 6-9, Algorithm 2): host-side, no GPU work -------------
+ * Keeps the exponential moving averages of the gradient norm g_r (Eq. 6, factor alpha) and of
+ * the measured batch time c_r (Eq. 8, factor beta) and takes the two per-batch decisions of
+ * Algorithm 2.  An average that is exactly 0 restarts from the next sample.  All arithmetic is
+ * fp64.  Every pointer is a HOST pointer; the object is owned by the caller between create and
+ * destroy and is not thread-safe.
+ *
+ * tgnn_controller_create   alpha, beta in (0, 1]; tau_g, tau_c > 0; K >= 1 (candidate cache-refresh
+ *                          boundaries are the batches r with r % K == 0); else TGNN_EINVAL
+ *                          (TGNN_ECAPACITY if the host allocation fails).
+ * tgnn_controller_begin_batch   the decisions before batch r (r >= 0) runs:
+ *     *boundary_out = 1 if r is a candidate boundary, else 0;
+ *     *sync_out     = S_r of Eq. 7 at a boundary (0: skip the refresh, when r > 0, the gradient
+ *                     average is > 0 and the last norm is < tau_g * average; else 1), -1 elsewhere;
+ *     *heavy_out    = H_r of Eq. 9 (1 when r > 0, the time average is > 0 and the last batch time
+ *                     is > tau_c * average; else 0) -- pass it as force_heavy, with
+ *                     drop_q32 = 0xFFFFFFFF, to prune every pure replay event of the batch (Eq. 10-11).
+ *     On one GPU there is no remote cache: S_r is reported for the log only.
+ * tgnn_controller_end_batch     folds g_r (>= 0) and c_r (>= 0, any unit) into the averages after
+ *                          the batch; NaN or negative values are refused with TGNN_EINVAL.
+ * tgnn_controller_state    out_host[4] = {g average, last g, c average, last c}. */
+typedef struct tgnn_controller tgnn_controller;
+TGNN_API int tgnn_controller_create(double alpha, double beta, double tau_g, double tau_c, int K, tgnn_controller** out);
+TGNN_API int tgnn_controller_destroy(tgnn_controller* ctl);
+TGNN_API int tgnn_controller_begin_batch(tgnn_controller* ctl, int64_t r, int* boundary_out, int* sync_out,
+                                         int* heavy_out);
+TGNN_API int tgnn_controller_end_batch(tgnn_controller* ctl, double g_r, double c_r);
+TGNN_API int tgnn_controller_state(const tgnn_controller* ctl, double* out_host);
+
 #ifdef __cplusplus
 }
 #endif

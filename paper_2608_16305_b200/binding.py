@@ -26,7 +26,9 @@ EXPORTS = ("tgnn_create", "tgnn_destroy", "tgnn_last_error", "tgnn_param_count",
            "tgnn_set_graph", "tgnn_set_edge_features", "tgnn_set_state", "tgnn_prune_mask", "tgnn_sample_recent",
            "tgnn_build_messages", "tgnn_reduce_latest", "tgnn_memory_update", "tgnn_embed", "tgnn_backward_step",
            "tgnn_train_step", "tgnn_train_step_host", "tgnn_debug_get_grads", "tgnn_status", "tgnn_kernel_launches", "tgnn_profile_begin",
-           "tgnn_profile_report", "tgnn_reduce_latest_static", "tgnn_debug_gemm", "tgnn_debug_get_gates", "tgnn_set_graph_replay", "tgnn_profile_timeline", "tgnn_step_mixed_host")
+           "tgnn_profile_report", "tgnn_reduce_latest_static", "tgnn_debug_gemm", "tgnn_debug_get_gates", "tgnn_set_graph_replay", "tgnn_profile_timeline", "tgnn_step_mixed_host",
+           "tgnn_controller_create", "tgnn_controller_destroy", "tgnn_controller_begin_batch",
+           "tgnn_controller_end_batch", "tgnn_controller_state")
 TGNN_STATIC_MAX_NODES = 65536
 
 
@@ -87,6 +89,12 @@ def load_library():
         lib.tgnn_step_mixed_host.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, i32, u32, u64, i64, vp, vp, vp]
         lib.tgnn_set_graph_replay.argtypes = [vp, i32]
         lib.tgnn_reduce_latest_static.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, vp, vp, i32]
+        f64 = C.c_double
+        lib.tgnn_controller_create.argtypes = [f64, f64, f64, f64, i32, C.POINTER(vp)]
+        lib.tgnn_controller_destroy.argtypes = [vp]
+        lib.tgnn_controller_begin_batch.argtypes = [vp, i64, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
+        lib.tgnn_controller_end_batch.argtypes = [vp, f64, f64]
+        lib.tgnn_controller_state.argtypes = [vp, C.POINTER(f64)]
         _lib = lib
     return _lib
 
@@ -153,6 +161,48 @@ def reduce_latest_static(msg_node, t, eid, num_nodes, uniq_out, winner_out, n_un
     if rc != TGNN_OK:
         raise TgnnError(rc, err.value.decode())
     return rc
+
+
+class Controller:
+    """The adaptive runtime controller (host-side; mirrors the tgnn_controller_* entry points)."""
+
+    def __init__(self, alpha: float, beta: float, tau_g: float, tau_c: float, K: int):
+        self.lib = load_library()
+        self._h = C.c_void_p()
+        rc = self.lib.tgnn_controller_create(alpha, beta, tau_g, tau_c, K, C.byref(self._h))
+        if rc != TGNN_OK:
+            raise TgnnError(rc, "tgnn_controller_create: parameter out of range")
+
+    def close(self):
+        if self._h:
+            self.lib.tgnn_controller_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def begin_batch(self, r: int):
+        """(boundary, S_r or -1, H_r) for batch r."""
+        b, s, h = C.c_int(), C.c_int(), C.c_int()
+        rc = self.lib.tgnn_controller_begin_batch(self._h, r, C.byref(b), C.byref(s), C.byref(h))
+        if rc != TGNN_OK:
+            raise TgnnError(rc, "tgnn_controller_begin_batch: invalid argument")
+        return b.value, s.value, h.value
+
+    def end_batch(self, g_r: float, c_r: float):
+        rc = self.lib.tgnn_controller_end_batch(self._h, g_r, c_r)
+        if rc != TGNN_OK:
+            raise TgnnError(rc, "tgnn_controller_end_batch: invalid argument")
+
+    def state(self):
+        out = (C.c_double * 4)()
+        rc = self.lib.tgnn_controller_state(self._h, out)
+        if rc != TGNN_OK:
+            raise TgnnError(rc, "tgnn_controller_state: invalid argument")
+        return tuple(out)
 
 
 class Tgnn:

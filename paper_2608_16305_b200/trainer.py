@@ -102,13 +102,17 @@ class Trainer:
         cur.wait_stream(self.stream)
         return out
 
-    def prune(self, b: int):
+    def prune(self, b: int, force_heavy: Optional[int] = None, drop_q32: Optional[int] = None):
+        """Keep mask of mixed batch b.  Default: the workload's own rule (count trigger, hashed half);
+        force_heavy / drop_q32 override it (the adaptive controller passes its H and "all")."""
         dw = self.dw
         s = dw.mb_slice(b)
         i = b - dw.batches.start
+        if force_heavy is None:
+            force_heavy = -1 if dw.cfg.prune else 0
         self.lib.prune_mask(dw.mb_src[s], dw.mb_dst[s], dw.mb_eid[s], dw.mb_aux[s], dw.mb_keep[s], dw.heavy[i:i + 1],
-                            force_heavy=-1 if dw.cfg.prune else 0, drop_q32=self.drop_q32, seed=self.prune_seed,
-                            batch_idx=b)
+                            force_heavy=force_heavy, drop_q32=self.drop_q32 if drop_q32 is None else drop_q32,
+                            seed=self.prune_seed, batch_idx=b)
 
     def host_batch(self, b: int):
         """Pinned host copies of mixed batch b and of its targets' negatives (what a data loader would hand over)."""
@@ -126,17 +130,42 @@ class Trainer:
             hb["src"], hb["dst"], hb["t"], hb["eid"], hb["aux"], hb["neg"], loss_host, gradnorm_host,
             force_heavy=-1 if cfg.prune else 0, drop_q32=self.drop_q32, seed=self.prune_seed, batch_idx=b))
 
-    def step(self, b: int, with_update: bool = True):
+    def step(self, b: int, with_update: bool = True, force_heavy: Optional[int] = None,
+             drop_q32: Optional[int] = None):
         """One training step on batch b (device-resident inputs)."""
-        return self._run(lambda: self._step(b, with_update))
+        return self._run(lambda: self._step(b, with_update, force_heavy, drop_q32))
 
-    def _step(self, b: int, with_update: bool):
+    def step_adaptive(self, b: int, ctl: "B.Controller", batch_time: Optional[float] = None):
+        """One step under the adaptive runtime controller (Algorithm 2).
+
+        Before the step the controller decides S_r (logged only: one GPU has no remote cache to
+        refresh) and H_r; under H_r = 1 every pure replay event of mixed batch b is pruned
+        (Eq. 10-11).  After it, the gradient norm and the step's device time (CUDA events, ms;
+        or `batch_time` when the caller supplies its own measurement) feed the controller's
+        averages.  Reads two scalars back, so it synchronises once per step.
+        """
+        r = b - self.dw.batches.start
+        boundary, sync, heavy = ctl.begin_batch(r)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+        def run():
+            e0.record()
+            self._step(b, True, heavy, 0xFFFFFFFF)
+            e1.record()
+        self._run(run)
+        e1.synchronize()
+        c = float(e0.elapsed_time(e1)) if batch_time is None else float(batch_time)
+        g = float(self.gradnorm.item())
+        ctl.end_batch(g, c)
+        return dict(r=r, boundary=boundary, sync=sync, heavy=heavy, g=g, c=c)
+
+    def _step(self, b: int, with_update: bool, force_heavy: Optional[int] = None, drop_q32: Optional[int] = None):
         dw = self.dw
         cur = torch.cuda.current_stream()
         cur.wait_stream(self.prune_stream)          # keep mask of batch b-1 is complete
         self.prune_stream.wait_stream(cur)          # inputs uploaded on this stream are visible
         with torch.cuda.stream(self.prune_stream):
-            self.prune(b)
+            self.prune(b, force_heavy, drop_q32)
         q = dw.target_slice(b)
         if with_update and b > dw.batches.start:
             u = dw.mb_slice(b - 1)

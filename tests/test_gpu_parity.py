@@ -438,6 +438,42 @@ def test_bf16_feature_table(B, oracle, math):
     _run_epoch_checks(rig, range(8), {1, 4, 7})
 
 
+def test_adaptive_controller_drives_pruning(B, oracle):
+    """Algorithm 2 end to end: the library's controller decides H_r from the batch times it is fed, a heavy
+    batch loses every pure replay event (Eq. 10-11) and nothing else, the next step's memory update uses
+    exactly the kept events, and the decisions equal the oracle controller's on the same measurements."""
+    from oracle import controller as oc
+    rig = Rig(B, oracle, _scaled("reddit", 9000))
+    alpha, beta, tau_g, tau_c, K = 0.1, 0.1, 1.6, 1.5, 3
+    ctl = B.Controller(alpha, beta, tau_g, tau_c, K)
+    ref = oc.ControllerOracle(alpha, beta, tau_g, tau_c, K)
+    nb = rig.cfg.num_batches
+    times = [1.0] * nb
+    times[3] = 4.0          # a straggling batch: the one after it runs in heavy-load mode
+    times[9] = 3.0
+    heavy_seen = []
+    for b in range(nb):
+        pre = rig.snapshot() if b in (4, 5, 10) else None
+        log = rig.tr.step_adaptive(b, ctl, batch_time=times[b])
+        bd, s, h = ref.begin_batch(b)
+        assert (log["boundary"], log["sync"], log["heavy"]) == (bd, -1 if s is None else s, h), b
+        ref.end_batch(log["g"], times[b])
+        assert ctl.state() == (ref.g_bar, ref.g_last, ref.c_bar, ref.c_prev)
+        heavy_seen.append(h)
+        torch.cuda.synchronize()
+        mb = rig.dw.mb_host[b]
+        keep = rig.dw.mb_keep[rig.dw.mb_slice(b)].cpu().numpy()
+        k_ref, _ = oracle.prune_mask(rig.cfg.num_nodes, mb.src, mb.dst, mb.eid, mb.is_aux, seed=rig.cfg.seed, batch_idx=b,
+                                     force_heavy=h, drop_q32=0xFFFFFFFF)
+        assert np.array_equal(keep, k_ref), b
+        assert np.array_equal(keep, (mb.is_aux == 0) if h else np.ones_like(keep)), b
+        if pre is not None:   # steps 5 and 10 update memory from the pruned batches 4 and 9... and 4 from the unpruned 3
+            res, _ = rig.oracle_step(pre, b, rig.gpu_gates(b))
+            rig.check_step(b, pre, res, what=f"[adaptive batch {b}]")
+    assert heavy_seen[4] == 1 and heavy_seen[10] == 1 and sum(heavy_seen) == 2
+    assert any(m.is_aux.any() for m in rig.dw.mb_host[4:5])   # the heavy batch did have replay events to lose
+
+
 def test_host_buffer_entry_point_matches_device_path(B, oracle):
     a = Rig(B, oracle, TINY)
     b = Rig(B, oracle, TINY)
