@@ -241,6 +241,9 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
                     "how": "Trainer.step_adaptive: controller decisions on the host, one synchronisation per step "
                            "to read the gradient norm and the step's device time"}
 
+    # ---- optional: the offline preprocessing pass (Algorithm 1 + Eq. 5) on this workload's stream ----
+    preprocess = preprocess_pass(cfg, stream, dw, device) if args.preprocess else None
+
     # ---- per-kernel times of the same K steps (separate pass: the event pairs perturb a latency-bound step) ----
     reset_epoch()
     run_steps(0, W, dev_step, False)
@@ -299,8 +302,58 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
     }
     if adaptive is not None:
         out["adaptive"] = adaptive
+    if preprocess is not None:
+        out["preprocess"] = preprocess
     out["cpu_baseline"] = cpu_baseline(cfg, stream, weights, budget_s=args.cpu_budget) if args.cpu_budget > 0 else None
     print(json.dumps(out))
+
+
+def preprocess_pass(cfg, stream, dw, device, P=8, K=6, reps=5):
+    """Backward dependency scan for all P workers and windows, then worker 0's mixed batches; the oracle's
+    scan is timed on a bounded number of (worker, window) pairs."""
+    from paper_2608_16305_b200 import binding as B
+    from oracle import scan as osc
+    E, nb, N = cfg.num_events, cfg.num_batches, cfg.num_nodes
+    Q = (nb + K - 1) // K
+    owner_h = (np.arange(N, dtype=np.int64) * 2654435761 % 2 ** 32 % P).astype(np.int32)
+    owner = torch.from_numpy(owner_h).to(device)
+    role = torch.empty((P, E), dtype=torch.uint8, device=device)
+    n_sync = torch.empty((P, Q), dtype=torch.int32, device=device)
+    scratch = torch.empty(B.backward_scan_scratch(E, cfg.batch, K, N, P), dtype=torch.int32, device=device)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    off = torch.empty(nb + 1, dtype=torch.int32, device=device)
+    toff = torch.empty(nb + 1, dtype=torch.int32, device=device)
+    i32 = lambda: torch.empty(E, dtype=torch.int32, device=device)
+    f64 = lambda: torch.empty(E, dtype=torch.float64, device=device)
+    mb = (i32(), i32(), f64(), i32(), torch.empty(E, dtype=torch.uint8, device=device))
+    tg = (i32(), i32(), f64(), i32(), i32())
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    ms_scan, ms_build = [], []
+    for _ in range(reps + 2):
+        a, b_, c = ev(), ev(), ev()
+        a.record()
+        B.backward_scan(dw.src, dw.dst, cfg.batch, K, owner, P, role, n_sync, None, scratch, status)
+        b_.record()
+        B.build_mixed(dw.src, dw.dst, dw.t, dw.neg, cfg.batch, role[0], off, toff, mb, tg, status)
+        c.record()
+        torch.cuda.synchronize()
+        ms_scan.append(a.elapsed_time(b_))
+        ms_build.append(b_.elapsed_time(c))
+    ms_scan, ms_build = float(np.median(ms_scan[2:])), float(np.median(ms_build[2:]))
+    aux_frac = float((role == 2).sum().item()) / float(max((role == 1).sum().item(), 1))
+    t0, pairs = time.perf_counter(), 0
+    for q in range(Q):
+        osc.backward_scan(stream.src, stream.dst, owner_h, q % P, cfg.batch, K, q)
+        pairs += 1
+        if time.perf_counter() - t0 > 5.0:
+            break
+    cpu_s = time.perf_counter() - t0
+    return {"workers": P, "K": K, "windows": Q, "scan_ms": ms_scan, "build_mixed_ms": ms_build,
+            "scan_events_per_s": P * E / (ms_scan * 1e-3), "aux_per_target": aux_frac,
+            "n_sync_mean": float(n_sync.float().mean().item()),
+            "cpu_oracle_events_per_s": pairs * K * cfg.batch / cpu_s, "cpu_oracle_sample": f"{pairs} (worker, window) scans",
+            "how": "tgnn_backward_scan over all workers and windows (hash partition), tgnn_build_mixed for worker 0; "
+                   "CUDA events, median of %d" % reps}
 
 
 def cpu_baseline(cfg, stream, weights, budget_s=20.0, steps=None):
@@ -362,6 +415,8 @@ def main():
     ap.add_argument("--math", default=os.environ.get("TGNN_BENCH_MATH", "tf32"), choices=["fp32", "tf32", "tf32fast"])
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--workload", default=WORKLOAD, choices=sorted(wl.CONFIGS), help="default: the benchmark workload (wiki)")
+    ap.add_argument("--preprocess", action="store_true",
+                    help="also time the backward dependency scan and mixed-batch construction (adds a 'preprocess' object)")
     ap.add_argument("--adaptive", action="store_true",
                     help="also time the steps under the adaptive runtime controller (adds an 'adaptive' object)")
     ap.add_argument("--no-graph", action="store_true", help="launch kernel by kernel instead of replaying a CUDA graph")

@@ -346,6 +346,53 @@ TGNN_API int tgnn_controller_begin_batch(tgnn_controller* ctl, int64_t r, int* b
 TGNN_API int tgnn_controller_end_batch(tgnn_controller* ctl, double g_r, double c_r);
 TGNN_API int tgnn_controller_state(const tgnn_controller* ctl, double* out_host);
 
+/* ---- offline preprocessing: backward dependency scan and mixed batches (Algorithm 1, Eq. 5) ----
+ * Stateless (no context); every pointer is a DEVICE pointer borrowed for the call unless named
+ * *_host; work is enqueued on `stream` (a cudaStream_t) and nothing is allocated.  On failure a
+ * message is written to err_host (host buffer of err_size bytes, may be NULL).
+ *
+ * The stream is src/dst[num_events] in timestamp order, cut into global batches of `batch` events
+ * (the last may be short); window W_q holds batches qK .. qK+K-1 (the last may hold fewer); owner[n]
+ * in [0, P) is the node ownership map pi.  nb = ceil(num_events / batch), Q = ceil(nb / K).
+ *
+ * tgnn_backward_scan runs Algorithm 1 for every worker p and window q:
+ *   role_out[p * num_events + e] = 1 if e is a target event of worker p (pi(src) = p), 2 if it is an
+ *       auxiliary replay event of p in its window, 0 if p's mixed batches do not contain it;
+ *   n_sync_out[p * Q + q]        = |N_sync| of (p, q), the candidate boundary refresh set;
+ *   sync_out[(p * Q + q) * num_nodes + n] = 1 if n is in that set, else 0 (may be NULL);
+ *   scratch  int32[tgnn_backward_scan_scratch(...)]: per-block node tables, contents undefined after;
+ *   status_out  device int32: zeroed by the call, set to 1 if a window's relaxation did not settle
+ *       within its event count (cannot happen; the loop is bounded all the same).
+ * Within a batch the walk is reverse chronological as between batches; the target events' remote
+ * destinations enter the frontier before their batch is walked, as in the listing.
+ * Errors: TGNN_EINVAL (null pointer, size < 1), TGNN_ECAPACITY (K * batch or P * Q out of int range),
+ * TGNN_ECUDA.  num_events = 0 is a no-op. */
+#define TGNN_SCAN_MAX_BLOCKS 592
+TGNN_API int64_t tgnn_backward_scan_scratch(int64_t num_events, int batch, int K, int64_t num_nodes, int P);
+TGNN_API int tgnn_backward_scan(const int32_t* src, const int32_t* dst, int64_t num_events, int batch, int K,
+                                const int32_t* owner, int64_t num_nodes, int P, uint8_t* role_out,
+                                int32_t* n_sync_out, uint8_t* sync_out, int32_t* scratch, int32_t* status_out,
+                                void* stream, char* err_host, int64_t err_size);
+
+/* tgnn_build_mixed forms one worker's mixed batches (Eq. 5) from its row of role_out: for every global
+ * batch s the events with role != 0, in timestamp order, with the event-type mask, and the target
+ * events among them.
+ *   role            uint8[num_events], one worker's row;   neg  int32[num_events] negatives per event or NULL;
+ *   mb_off_out      int32[nb + 1]: mixed batch s occupies [mb_off[s], mb_off[s+1]) of mb_src, mb_dst, mb_t,
+ *                   mb_eid (stream position of the event), mb_aux (1 = auxiliary replay event);
+ *   tgt_off_out     int32[nb + 1]: the targets of batch s occupy [tgt_off[s], tgt_off[s+1]) of tgt_src,
+ *                   tgt_dst, tgt_t, tgt_neg (may be NULL; -1 where neg is NULL), tgt_eid;
+ *   cap_mixed, cap_tgt  elements available in the mb_* / tgt_* arrays (num_events always suffices);
+ *   status_out      device int32: zeroed by the call, set to 2 if a capacity was too small (the events
+ *                   beyond it are not written).
+ * Errors: TGNN_EINVAL, TGNN_ECAPACITY (num_events beyond int32), TGNN_ECUDA. */
+TGNN_API int tgnn_build_mixed(const int32_t* src, const int32_t* dst, const double* t, const int32_t* neg,
+                              int64_t num_events, int batch, const uint8_t* role, int32_t* mb_off_out,
+                              int32_t* tgt_off_out, int64_t cap_mixed, int64_t cap_tgt, int32_t* mb_src, int32_t* mb_dst,
+                              double* mb_t, int32_t* mb_eid, uint8_t* mb_aux, int32_t* tgt_src, int32_t* tgt_dst,
+                              double* tgt_t, int32_t* tgt_neg, int32_t* tgt_eid, int32_t* status_out, void* stream,
+                              char* err_host, int64_t err_size);
+
 #ifdef __cplusplus
 }
 #endif

@@ -28,7 +28,8 @@ EXPORTS = ("tgnn_create", "tgnn_destroy", "tgnn_last_error", "tgnn_param_count",
            "tgnn_train_step", "tgnn_train_step_host", "tgnn_debug_get_grads", "tgnn_status", "tgnn_kernel_launches", "tgnn_profile_begin",
            "tgnn_profile_report", "tgnn_reduce_latest_static", "tgnn_debug_gemm", "tgnn_debug_get_gates", "tgnn_set_graph_replay", "tgnn_profile_timeline", "tgnn_step_mixed_host",
            "tgnn_controller_create", "tgnn_controller_destroy", "tgnn_controller_begin_batch",
-           "tgnn_controller_end_batch", "tgnn_controller_state")
+           "tgnn_controller_end_batch", "tgnn_controller_state", "tgnn_backward_scan_scratch", "tgnn_backward_scan",
+           "tgnn_build_mixed")
 TGNN_STATIC_MAX_NODES = 65536
 
 
@@ -95,6 +96,10 @@ def load_library():
         lib.tgnn_controller_begin_batch.argtypes = [vp, i64, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
         lib.tgnn_controller_end_batch.argtypes = [vp, f64, f64]
         lib.tgnn_controller_state.argtypes = [vp, C.POINTER(f64)]
+        lib.tgnn_backward_scan_scratch.argtypes = [i64, i32, i32, i64, i32]
+        lib.tgnn_backward_scan_scratch.restype = i64
+        lib.tgnn_backward_scan.argtypes = [vp, vp, i64, i32, i32, vp, i64, i32, vp, vp, vp, vp, vp, vp, vp, i64]
+        lib.tgnn_build_mixed.argtypes = [vp, vp, vp, vp, i64, i32, vp, vp, vp, i64, i64] + [vp] * 11 + [vp, vp, i64]
         _lib = lib
     return _lib
 
@@ -157,6 +162,43 @@ def reduce_latest_static(msg_node, t, eid, num_nodes, uniq_out, winner_out, n_un
     rc = load_library().tgnn_reduce_latest_static(
         _dp(msg_node, "i32", "msg_node"), _dp(t, "f64", "t"), _dp(eid, "i32", "eid"), msg_node.numel(), num_nodes,
         _dp(uniq_out, "i32", "uniq_out"), _dp(winner_out, "i32", "winner_out"), _dp(n_uniq_out, "i32", "n_uniq_out"),
+        _stream(), C.addressof(err), len(err))
+    if rc != TGNN_OK:
+        raise TgnnError(rc, err.value.decode())
+    return rc
+
+
+def backward_scan_scratch(num_events: int, batch: int, K: int, num_nodes: int, P: int) -> int:
+    """int32 elements tgnn_backward_scan needs as scratch."""
+    n = load_library().tgnn_backward_scan_scratch(num_events, batch, K, num_nodes, P)
+    if n < 0:
+        raise TgnnError(TGNN_EINVAL, "tgnn_backward_scan_scratch: size out of range")
+    return n
+
+
+def backward_scan(src, dst, batch: int, K: int, owner, P: int, role_out, n_sync_out, sync_out, scratch, status_out) -> int:
+    """tgnn_backward_scan: Algorithm 1 for every worker and window (device tensors; sync_out may be None)."""
+    err = C.create_string_buffer(512)
+    rc = load_library().tgnn_backward_scan(
+        _dp(src, "i32", "src"), _dp(dst, "i32", "dst"), src.numel(), batch, K, _dp(owner, "i32", "owner"), owner.numel(), P,
+        _dp(role_out, "u8", "role_out"), _dp(n_sync_out, "i32", "n_sync_out"), _dp(sync_out, "u8", "sync_out"),
+        _dp(scratch, "i32", "scratch"), _dp(status_out, "i32", "status_out"), _stream(), C.addressof(err), len(err))
+    if rc != TGNN_OK:
+        raise TgnnError(rc, err.value.decode())
+    return rc
+
+
+def build_mixed(src, dst, t, neg, batch: int, role, mb_off_out, tgt_off_out, mb, tgt, status_out) -> int:
+    """tgnn_build_mixed: one worker's mixed batches (Eq. 5).  mb = (src, dst, t, eid, aux) output tensors,
+    tgt = (src, dst, t, neg or None, eid) output tensors."""
+    err = C.create_string_buffer(512)
+    rc = load_library().tgnn_build_mixed(
+        _dp(src, "i32", "src"), _dp(dst, "i32", "dst"), _dp(t, "f64", "t"), _dp(neg, "i32", "neg"), src.numel(), batch,
+        _dp(role, "u8", "role"), _dp(mb_off_out, "i32", "mb_off_out"), _dp(tgt_off_out, "i32", "tgt_off_out"),
+        mb[0].numel(), tgt[0].numel(),
+        _dp(mb[0], "i32", "mb_src"), _dp(mb[1], "i32", "mb_dst"), _dp(mb[2], "f64", "mb_t"), _dp(mb[3], "i32", "mb_eid"),
+        _dp(mb[4], "u8", "mb_aux"), _dp(tgt[0], "i32", "tgt_src"), _dp(tgt[1], "i32", "tgt_dst"), _dp(tgt[2], "f64", "tgt_t"),
+        _dp(tgt[3], "i32", "tgt_neg"), _dp(tgt[4], "i32", "tgt_eid"), _dp(status_out, "i32", "status_out"),
         _stream(), C.addressof(err), len(err))
     if rc != TGNN_OK:
         raise TgnnError(rc, err.value.decode())

@@ -50,8 +50,10 @@ class DeviceWorkload:
         cat = lambda f, dt: t(np.concatenate([getattr(m, f) for m in mbs]).astype(dt)) if mbs else None
         self.mb_src, self.mb_dst = cat("src", np.int32), cat("dst", np.int32)
         self.mb_t, self.mb_eid, self.mb_aux = cat("t", np.float64), cat("eid", np.int32), cat("is_aux", np.uint8)
-        self.mb_keep = torch.ones_like(self.mb_aux)
+        self.mb_keep = torch.ones_like(self.mb_aux) if mbs else None
         self.heavy = torch.zeros(len(mbs), dtype=torch.int32, device=dev)
+        self.max_mixed = cfg.max_mixed      # capacities the library context is created with
+        self.max_targets = cfg.batch
 
     def mb_slice(self, b: int):
         i = b - self.batches.start
@@ -60,6 +62,71 @@ class DeviceWorkload:
     def target_slice(self, b: int):
         return slice(b * self.cfg.batch, min((b + 1) * self.cfg.batch, self.cfg.num_events))
 
+    def targets(self, b: int):
+        """Device tensors (src, dst, neg, t) of the target events of batch b."""
+        q = self.target_slice(b)
+        return self.src[q], self.dst[q], self.neg[q], self.t[q]
+
+    def targets_host(self, b: int):
+        q = self.target_slice(b)
+        s = self.stream
+        return s.src[q], s.dst[q], s.neg[q], s.t[q]
+
+
+class PartitionedWorkload(DeviceWorkload):
+    """Worker p's view of the stream under a node partition: its mixed batches come from the
+    backward dependency scan (Algorithm 1) instead of the resampled replay sets, its targets are the
+    source-owned events of each global batch.  The scan and the batch construction run on the device."""
+
+    def __init__(self, stream: wl.EventStream, owner: np.ndarray, P: int, p: int, K: int, device="cuda",
+                 efeat: Optional[torch.Tensor] = None):
+        super().__init__(stream, device=device, batches=range(0, 0), efeat=efeat)
+        cfg = self.cfg
+        dev = self.device
+        E, nb = cfg.num_events, cfg.num_batches
+        Q = (nb + K - 1) // K
+        self.owner = torch.from_numpy(np.ascontiguousarray(owner, dtype=np.int32)).to(dev)
+        self.P, self.p, self.K = P, p, K
+        self.role = torch.empty((P, E), dtype=torch.uint8, device=dev)
+        self.n_sync = torch.empty((P, Q), dtype=torch.int32, device=dev)
+        scratch = torch.empty(B.backward_scan_scratch(E, cfg.batch, K, cfg.num_nodes, P), dtype=torch.int32, device=dev)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        B.backward_scan(self.src, self.dst, cfg.batch, K, self.owner, P, self.role, self.n_sync, None, scratch, status)
+        off = torch.empty(nb + 1, dtype=torch.int32, device=dev)
+        toff = torch.empty(nb + 1, dtype=torch.int32, device=dev)
+        i32 = lambda: torch.empty(E, dtype=torch.int32, device=dev)
+        mb = (i32(), i32(), torch.empty(E, dtype=torch.float64, device=dev), i32(), torch.empty(E, dtype=torch.uint8, device=dev))
+        tg = (i32(), i32(), torch.empty(E, dtype=torch.float64, device=dev), i32(), i32())
+        status2 = torch.zeros(1, dtype=torch.int32, device=dev)
+        B.build_mixed(self.src, self.dst, self.t, self.neg, cfg.batch, self.role[p], off, toff, mb, tg, status2)
+        torch.cuda.synchronize(dev)
+        if int(status.item()) or int(status2.item()):
+            raise RuntimeError("backward scan / mixed-batch construction reported a device-side error")
+        self.mb_off = off.cpu().numpy().astype(np.int64)
+        self.tgt_off = toff.cpu().numpy().astype(np.int64)
+        n_m, n_t = int(self.mb_off[-1]), int(self.tgt_off[-1])
+        self.mb_src, self.mb_dst, self.mb_t, self.mb_eid, self.mb_aux = (x[:n_m].clone() for x in mb)
+        self.tgt_src, self.tgt_dst, self.tgt_t, self.tgt_neg, self.tgt_eid = (x[:n_t].clone() for x in tg)
+        self.mb_keep = torch.ones_like(self.mb_aux)
+        self.batches = range(0, nb)
+        self.heavy = torch.zeros(nb, dtype=torch.int32, device=dev)
+        self.max_mixed = max(1, int(np.diff(self.mb_off).max()))
+        self.max_targets = max(1, int(np.diff(self.tgt_off).max()))
+        h = [x.cpu().numpy() for x in (self.mb_src, self.mb_dst, self.mb_t, self.mb_eid, self.mb_aux)]
+        self.mb_host = [wl.MixedBatch(b, *(a[self.mb_off[b]:self.mb_off[b + 1]] for a in h)) for b in range(nb)]
+        self._tgt_host = [x.cpu().numpy() for x in (self.tgt_src, self.tgt_dst, self.tgt_neg, self.tgt_t)]
+
+    def _tslice(self, b: int):
+        return slice(int(self.tgt_off[b]), int(self.tgt_off[b + 1]))
+
+    def targets(self, b: int):
+        q = self._tslice(b)
+        return self.tgt_src[q], self.tgt_dst[q], self.tgt_neg[q], self.tgt_t[q]
+
+    def targets_host(self, b: int):
+        q = self._tslice(b)
+        return tuple(a[q] for a in self._tgt_host)
+
 
 class Trainer:
     def __init__(self, dw: DeviceWorkload, weights, math_mode=B.TGNN_MATH_FP32, lr=1e-4):
@@ -67,7 +134,7 @@ class Trainer:
         self.dw = dw
         self.tcfg = B.make_config(cfg.num_nodes, cfg.d, cfg.d_e, cfg.k, cfg.heads,
                                   feat_dtype=B.TGNN_BF16 if cfg.feat_dtype == "bf16" else B.TGNN_F32,
-                                  max_events=cfg.max_mixed, max_roots=3 * cfg.batch, math_mode=math_mode, lr=lr)
+                                  max_events=dw.max_mixed, max_roots=3 * dw.max_targets, math_mode=math_mode, lr=lr)
         self.lib = B.Tgnn(self.tcfg)
         dev = dw.device
         P = B.param_layout(self.tcfg)["total"]
@@ -119,9 +186,8 @@ class Trainer:
         dw = self.dw
         mb = dw.mb_host[b - dw.batches.start]
         pin = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a, dtype=dt)).pin_memory()
-        q = dw.target_slice(b)
         return dict(src=pin(mb.src, np.int32), dst=pin(mb.dst, np.int32), t=pin(mb.t, np.float64),
-                    eid=pin(mb.eid, np.int32), aux=pin(mb.is_aux, np.uint8), neg=pin(dw.stream.neg[q], np.int32))
+                    eid=pin(mb.eid, np.int32), aux=pin(mb.is_aux, np.uint8), neg=pin(dw.targets_host(b)[2], np.int32))
 
     def step_host(self, b: int, hb, loss_host, gradnorm_host):
         """One training step fed from host memory: a single call of the streaming entry point per mixed batch."""
@@ -166,10 +232,10 @@ class Trainer:
         self.prune_stream.wait_stream(cur)          # inputs uploaded on this stream are visible
         with torch.cuda.stream(self.prune_stream):
             self.prune(b, force_heavy, drop_q32)
-        q = dw.target_slice(b)
+        tsrc, tdst, tneg, tt = dw.targets(b)
         if with_update and b > dw.batches.start:
             u = dw.mb_slice(b - 1)
             upd = (dw.mb_src[u], dw.mb_dst[u], dw.mb_t[u], dw.mb_eid[u], dw.mb_keep[u])
         else:
             upd = (None, None, None, None, None)
-        self.lib.train_step(*upd, dw.src[q], dw.dst[q], dw.neg[q], dw.t[q], None, self.loss, self.gradnorm)
+        self.lib.train_step(*upd, tsrc, tdst, tneg, tt, None, self.loss, self.gradnorm)

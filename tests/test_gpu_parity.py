@@ -55,7 +55,7 @@ def orc_cfg(oracle, c, **kw):
 class Rig:
     """A workload on the device plus a library context and an oracle configuration."""
 
-    def __init__(self, B, oracle, cfg, math="fp32", batches=None, bias_scale=0.1, lr=1e-3):
+    def __init__(self, B, oracle, cfg, math="fp32", batches=None, bias_scale=0.1, lr=1e-3, partition=None):
         from paper_2608_16305_b200 import trainer
         self.B, self.oracle, self.cfg, self.math = B, oracle, cfg, math
         self.stream = wl.make_stream(cfg)
@@ -66,7 +66,10 @@ class Rig:
             if not self.compact:
                 self.stream._efeat = self._to_host(efeat_dev)
         self.efeat_dev = efeat_dev
-        self.dw = trainer.DeviceWorkload(self.stream, batches=batches, efeat=efeat_dev)
+        if partition is None:
+            self.dw = trainer.DeviceWorkload(self.stream, batches=batches, efeat=efeat_dev)
+        else:   # (owner, P, p, K): worker p's mixed batches from the backward dependency scan
+            self.dw = trainer.PartitionedWorkload(self.stream, *partition, efeat=efeat_dev)
         self.weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed, bias_scale=bias_scale)
         mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST}[math]
         self.tr = trainer.Trainer(self.dw, self.weights, math_mode=mode, lr=lr)
@@ -99,8 +102,7 @@ class Rig:
         return (mb.src, mb.dst, mb.t, mb.eid, keep)
 
     def gpu_gates(self, b):
-        q = self.dw.target_slice(b)
-        nq = q.stop - q.start
+        nq = len(self.dw.targets_host(b)[0])
         torch.cuda.synchronize()
         hg = torch.zeros((3 * nq, self.cfg.d), dtype=torch.uint8, device="cuda")
         dg = torch.zeros((2 * nq, self.cfg.d), dtype=torch.uint8, device="cuda")
@@ -109,10 +111,10 @@ class Rig:
         return hg.cpu().numpy(), dg.cpu().numpy()
 
     def oracle_step(self, pre, b, gates=None):
-        o, s = self.oracle, self.stream
-        q = self.dw.target_slice(b)
-        nodes = np.concatenate([s.src[q], s.dst[q], s.neg[q]])
-        times = np.concatenate([s.t[q]] * 3)
+        o = self.oracle
+        t_src, t_dst, t_neg, t_t = self.dw.targets_host(b)
+        nodes = np.concatenate([t_src, t_dst, t_neg])
+        times = np.concatenate([t_t] * 3)
         nb = o.sample_recent(*self.graph, nodes, times, self.cfg.k)
         upd = self.upd_host(b)
         if upd is None:
@@ -132,7 +134,7 @@ class Rig:
         if gates is not None:
             kw = dict(h_gate=gates[0], hid_gate=gates[1], gate_eps=GATE_EPS[self.math])
         res = o.loss_and_grads(self.ocfg, pre["params"], pre["memory"], pre["last_update"], efeat, upd,
-                               roots, q.stop - q.start, None, **kw)
+                               roots, len(t_src), None, **kw)
         return res, roots
 
     def check_step(self, b, pre, res, what=""):
@@ -472,6 +474,25 @@ def test_adaptive_controller_drives_pruning(B, oracle):
             rig.check_step(b, pre, res, what=f"[adaptive batch {b}]")
     assert heavy_seen[4] == 1 and heavy_seen[10] == 1 and sum(heavy_seen) == 2
     assert any(m.is_aux.any() for m in rig.dw.mb_host[4:5])   # the heavy batch did have replay events to lose
+
+
+@pytest.mark.parametrize("p", [0, 2])
+def test_partitioned_worker_steps_on_scanned_mixed_batches(B, oracle, p):
+    """Worker p of a 3-way node partition trains on the mixed batches that the backward dependency scan
+    (Algorithm 1) built on the device: its targets are the source-owned events (variable count per batch),
+    the memory update replays targets and auxiliary events alike, and each step matches the oracle."""
+    cfg = _scaled("reddit", 7200)
+    owner = (np.arange(cfg.num_nodes) * 2654435761 % 2 ** 32 % 3).astype(np.int32)
+    rig = Rig(B, oracle, cfg, math="tf32", partition=(owner, 3, p, 4))
+    dw = rig.dw
+    src, dst = rig.stream.src, rig.stream.dst
+    for b in range(cfg.num_batches):
+        mb = dw.mb_host[b]
+        assert np.array_equal(owner[src[mb.eid]] != p, mb.is_aux == 1)           # the event-type mask is the ownership test
+        assert np.array_equal(dw.targets_host(b)[0], mb.src[mb.is_aux == 0])     # targets = the non-auxiliary events, in order
+        assert np.all(np.diff(mb.t) >= 0)                                        # timestamp order (Eq. 5)
+    assert sum(int(m.is_aux.sum()) for m in dw.mb_host) > 0
+    _run_epoch_checks(rig, range(cfg.num_batches), {1, 4, 7, cfg.num_batches - 1})
 
 
 def test_host_buffer_entry_point_matches_device_path(B, oracle):
