@@ -125,6 +125,17 @@ def kv_proj_flops(cfg, n_q):
     return 2.0 * (3 * n_q * cfg.k) * cfg.d_kv * (2 * cfg.d)
 
 
+def algorithmic_work_jodie(cfg: wl.WorkloadConfig, n_u: int, n_q: int, U: int):
+    """The same accounting for the time-projection model: no neighbor search, no attention."""
+    d, de = cfg.d, cfg.d_e
+    f = 4 if cfg.feat_dtype == "f32" else 2
+    R = 3 * n_q
+    P = sum(int(np.prod(s)) for s in wl.param_shapes(d, de, "jodie").values())
+    by = (2 * n_u * (2 * d * 4 + 8) + n_u * de * f) + U * (2 * d * 4 + 8) + 2 * R * (4 * d + 8) + 28 * P
+    fwd = 2 * d * (cfg.d_msg + d) * U + 2 * R * d + 2 * (2 * n_q) * 2 * d * d
+    return by, fwd, 2.0 * fwd
+
+
 def run_ours(args, rank, world, device):
     from paper_2608_16305_b200 import binding as B
     from paper_2608_16305_b200 import trainer as T
@@ -133,9 +144,9 @@ def run_ours(args, rank, world, device):
     efeat = wl.edge_feature_table_torch(cfg, device)
     n_need = 2 * (args.steps + args.warmup) + 8
     dw = T.DeviceWorkload(stream, device=device, efeat=efeat, batches=range(0, min(cfg.num_batches, n_need)))
-    weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed)
+    weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed, model=args.model)
     math_mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST}[args.math]
-    tr = T.Trainer(dw, weights, math_mode=math_mode)
+    tr = T.Trainer(dw, weights, math_mode=math_mode, model=args.model)
     if args.no_graph:
         tr.lib.set_graph_replay(False)
     torch.cuda.synchronize()
@@ -259,10 +270,12 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
     if rank != 0:
         return
     # roofline of the dominant kernel: the key/value projection GEMM of the attention layer
-    dom = "kv_proj"
+    jodie = args.model == "jodie"
+    U_est = min(2 * cfg.max_mixed, cfg.num_nodes) // 2
+    dom = "gru_gi" if jodie else "kv_proj"      # time-projection model: the update cell's input product dominates
     cnt, ms_tot = prof.get(dom, (0, 0.0))
     dur_s = (ms_tot / max(cnt, 1)) * 1e-3
-    flops = kv_proj_flops(cfg, n_q)
+    flops = 2.0 * U_est * cfg.d_msg * cfg.d if jodie else kv_proj_flops(cfg, n_q)
     if args.math != "fp32":
         peak, bound, peak_note = peaks["bf16_tflops"] * 0.5, "tensor", f"0.5 x {peaks['source']} bf16 burst (TF32 nominal ratio)"
     else:
@@ -272,8 +285,8 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
     achieved = flops / dur_s / 1e12 if dur_s > 0 else 0.0
     # dram__bytes_read.sum + dram__bytes_write.sum of one key/value-projection launch on this workload
     # (ncu --set full, summarised in profiles/gemm_tf32_kv_proj_wiki.md; tensor-core mode only)
-    traffic = 28.6e6 + 0.08e6 if (args.math == "tf32" and cfg.name == WORKLOAD) else None
-    by, f_fwd, f_bwd = algorithmic_work(cfg, cfg.max_mixed, n_q, min(2 * cfg.max_mixed, cfg.num_nodes) // 2)
+    traffic = 28.6e6 + 0.08e6 if (args.math == "tf32" and cfg.name == WORKLOAD and not jodie) else None
+    by, f_fwd, f_bwd = (algorithmic_work_jodie if jodie else algorithmic_work)(cfg, cfg.max_mixed, n_q, U_est)
     out = {
         "metric": METRIC, "value": units / (ms_dev_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_dev_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -281,6 +294,7 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
         "config": {"workload": f"{cfg.name}: {cfg.num_nodes} nodes" + (f" ({cfg.num_src}+{cfg.num_nodes - cfg.num_src} bipartite)" if cfg.num_src else "")
                                + f", {cfg.num_events} events, d_e={cfg.d_e} {cfg.feat_dtype}, d={cfg.d}, k={cfg.k}, {cfg.heads} heads, "
                                f"batch {cfg.batch}, replay {cfg.replay_frac:g}" + (" with pruning" if cfg.prune else ""),
+                   "model": "JODIE-style (recurrent cell + time projection)" if jodie else "TGN-style (GRU + temporal attention)",
                    "math_mode": args.math, "l2": "512 MB buffer written between timed steps (outside the event pairs)",
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "launch": "kernel by kernel" if args.no_graph else "CUDA graph replay of the step (captured by the library)",
@@ -292,7 +306,8 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
         "clocks": clocks,
         "roofline": {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak if peak else None, "traffic": traffic, "peak_source": peak_note,
-                     "algorithmic_bytes_per_launch": 3 * n_q * cfg.k * (cfg.d_kv * 4 + 2 * cfg.d * 4) + 2 * cfg.d * cfg.d_kv * 4,
+                     "algorithmic_bytes_per_launch": (U_est * (cfg.d_msg + cfg.d) * 4 + cfg.d * cfg.d_msg * 4) if jodie else
+                     3 * n_q * cfg.k * (cfg.d_kv * 4 + 2 * cfg.d * 4) + 2 * cfg.d * cfg.d_kv * 4,
                      "flops_per_launch": flops, "avg_launch_us": dur_s * 1e6, "launches": cnt,
                      "step_algorithmic_bytes": by, "step_algorithmic_flops": f_fwd + f_bwd,
                      "step_hbm_frac": (by / (ms_dev_max / K * 1e-3)) / (peaks["hbm_gbs"] * 1e9),
@@ -304,7 +319,7 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
         out["adaptive"] = adaptive
     if preprocess is not None:
         out["preprocess"] = preprocess
-    out["cpu_baseline"] = cpu_baseline(cfg, stream, weights, budget_s=args.cpu_budget) if args.cpu_budget > 0 else None
+    out["cpu_baseline"] = cpu_baseline(cfg, stream, weights, budget_s=args.cpu_budget, model=args.model) if args.cpu_budget > 0 else None
     print(json.dumps(out))
 
 
@@ -356,11 +371,13 @@ def preprocess_pass(cfg, stream, dw, device, P=8, K=6, reps=5):
                    "CUDA events, median of %d" % reps}
 
 
-def cpu_baseline(cfg, stream, weights, budget_s=20.0, steps=None):
+def cpu_baseline(cfg, stream, weights, budget_s=20.0, steps=None, model="tgn"):
     """The oracle as it stands, one thread, on consecutive batches from the middle of the epoch."""
     from oracle import oracle as orc
     ocfg = orc.make_config(cfg.num_nodes, cfg.d, cfg.d_e, cfg.k, cfg.heads, feat_bf16=cfg.feat_dtype == "bf16")
     ef = stream.efeat() if cfg.d_e else None
+    if model == "jodie":
+        return cpu_baseline_jodie(cfg, stream, weights, ocfg, ef, budget_s, steps)
     state = orc.OracleState(ocfg, orc.pack_params(ocfg, weights))
     graph = (stream.indptr, stream.nbr, stream.eid, stream.ts)
     b0 = cfg.num_batches // 2
@@ -383,24 +400,52 @@ def cpu_baseline(cfg, stream, weights, budget_s=20.0, steps=None):
                       f"single thread, host has {os.cpu_count()} cores"}
 
 
+def cpu_baseline_jodie(cfg, stream, weights, ocfg, ef, budget_s, steps):
+    """The time-projection model's oracle (numpy, one process; its matrix products may use several threads)."""
+    from oracle import jodie as oj
+    from oracle import oracle as orc
+    p = oj.pack(cfg.d, cfg.d_e, weights)
+    m, v, st = np.zeros_like(p), np.zeros_like(p), 0
+    mem, lu = np.zeros((cfg.num_nodes, cfg.d)), np.zeros(cfg.num_nodes)
+    b0 = cfg.num_batches // 2
+    mbp = wl.mixed_batch(stream, b0 - 1)
+    prev, done, spent = (mbp.src, mbp.dst, mbp.t, mbp.eid, None), 0, 0.0
+    while (steps is None and spent < budget_s and done < 64) or (steps is not None and done < steps):
+        b = b0 + done
+        mb = wl.mixed_batch(stream, b)
+        q = slice(b * cfg.batch, (b + 1) * cfg.batch)
+        t0 = time.perf_counter()
+        keep, _ = orc.prune_mask(cfg.num_nodes, mb.src, mb.dst, mb.eid, mb.is_aux, force_heavy=-1 if cfg.prune else 0,
+                                 seed=cfg.seed, batch_idx=b)
+        res = oj.step(ocfg, p, mem, lu, ef, prev, (stream.src[q], stream.dst[q], stream.neg[q], stream.t[q]))
+        p, m, v, st = orc.adam(ocfg, res.grads, p, m, v, st)
+        mem, lu = res.memory_post, res.last_update_post
+        spent += time.perf_counter() - t0
+        prev = (mb.src, mb.dst, mb.t, mb.eid, keep)
+        done += 1
+    return {"value": done * cfg.batch / spent, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle", "seconds": spent,
+            "sample": f"{done} consecutive steps (batches {b0}..{b0 + done - 1}) of the {cfg.name} workload, numpy "
+                      f"(BLAS threads as configured on the host, {os.cpu_count()} cores)"}
+
+
 def run_reference(args, rank, world):
     if rank != 0:
         return
     cfg = wl.CONFIGS[WORKLOAD]
     stream = wl.make_stream(cfg)
-    weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed)
+    weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed, model=args.model)
     stream.efeat()
     K, W = args.steps, args.warmup
     per = 2                                   # oracle steps per benchmark "step" sample
     n = min(K, 8)                             # bounded: the whole run must end within minutes
-    cpu_baseline(cfg, stream, weights, steps=min(W, 1))
-    res = cpu_baseline(cfg, stream, weights, steps=n * per)
+    cpu_baseline(cfg, stream, weights, steps=min(W, 1), model=args.model)
+    res = cpu_baseline(cfg, stream, weights, steps=n * per, model=args.model)
     ms = res["seconds"] * 1e3 / (n * per)
     out = {"impl": "reference", "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": K,
            "warmup": W, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": "f64", "data": "synthetic",
            "config": {"workload": f"{WORKLOAD}: bounded sample of {n * per} oracle steps standing for {K} steps"},
-           "cpu_baseline": {"value": res["value"], "unit": UNIT, "kind": "oracle", "cores": 1, "sample": res["sample"]},
+           "cpu_baseline": {"value": res["value"], "unit": UNIT, "kind": "oracle", "cores": res["cores"], "sample": res["sample"]},
            "e2e": {"value": res["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
     print(json.dumps(out))
@@ -415,6 +460,8 @@ def main():
     ap.add_argument("--math", default=os.environ.get("TGNN_BENCH_MATH", "tf32"), choices=["fp32", "tf32", "tf32fast"])
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--workload", default=WORKLOAD, choices=sorted(wl.CONFIGS), help="default: the benchmark workload (wiki)")
+    ap.add_argument("--model", default="tgn", choices=["tgn", "jodie"],
+                    help="tgn: GRU + temporal attention (the benchmark's model); jodie: recurrent cell + time projection")
     ap.add_argument("--preprocess", action="store_true",
                     help="also time the backward dependency scan and mixed-batch construction (adds a 'preprocess' object)")
     ap.add_argument("--adaptive", action="store_true",

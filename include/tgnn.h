@@ -71,6 +71,15 @@ enum {
                              terms cancel (time encoder, W_k) can be off by ~1e-2 of their largest entry. */
 };
 
+/* model: which memory-based model the step trains.  Steps (0)-(3), the head, the loss and Adam are
+ * shared; steps (4)-(5) and their backward differ. */
+enum {
+  TGNN_MODEL_TGN = 0,   /* GRU memory update + one temporal attention layer over the k most recent neighbors */
+  TGNN_MODEL_JODIE = 1  /* plain recurrent cell  m' = tanh(W_i msg + b_i + W_h m + b_h)  and the
+                           time-projected embedding  h(n, t) = m_n * (1 + dt w_p + b_p),
+                           dt = fp32(t - last_update[n]); no neighbor sampling, no attention */
+};
+
 #if defined(__GNUC__)
 #define TGNN_API __attribute__((visibility("default")))
 #else
@@ -90,6 +99,7 @@ typedef struct {
   int32_t max_roots;  /* capacity: roots in one tgnn_embed call (3 per target event) */
   int32_t math_mode;  /* TGNN_MATH_* */
   float lr, beta1, beta2, eps; /* Adam */
+  int32_t model;      /* TGNN_MODEL_* */
 } tgnn_config;
 
 /* ---- life cycle --------------------------------------------------------- */
@@ -102,10 +112,14 @@ TGNN_API int tgnn_destroy(tgnn_ctx* ctx);
 /* Message of the last error recorded in ctx (static string if ctx is NULL). Never NULL. */
 TGNN_API const char* tgnn_last_error(const tgnn_ctx* ctx);
 
-/* Number of fp32 parameters, and the offsets of the 18 tensors in layout order
- * followed by the total (out19_host has 19 entries).  Pure host computations. */
+/* Number of fp32 parameters, and the offsets of the 20 tensors followed by the total (out21_host has
+ * 21 entries): time_w, time_b, update-cell W_i [g*d, d_msg], W_h [g*d, d], b_i, b_h (g = 3 gates for
+ * the GRU, 1 for the plain cell), W_q, b_q, W_k, W_v, b_k, b_v, W_o, b_o, W_1, b_1, w_2, b_2, then the
+ * projection's w_p, b_p.  Tensors a model does not have are empty (the attention block for
+ * TGNN_MODEL_JODIE, the projection for TGNN_MODEL_TGN); in memory w_p, b_p sit between b_o and W_1.
+ * Pure host computations. */
 TGNN_API int64_t tgnn_param_count(const tgnn_config* cfg_host);
-TGNN_API int tgnn_param_layout(const tgnn_config* cfg_host, int64_t* out19_host);
+TGNN_API int tgnn_param_layout(const tgnn_config* cfg_host, int64_t* out21_host);
 
 /* Time-sorted adjacency (T-CSR) of the whole stream, both directions of every
  * event: node n owns entries [indptr[n], indptr[n+1]) sorted by (ts, eid).
@@ -169,7 +183,7 @@ TGNN_API int tgnn_reduce_latest(tgnn_ctx* ctx, const int32_t* msg_node, const do
                        int32_t* uniq_out, int32_t* winner_out, int32_t* n_uniq_out, void* stream);
 
 /* Step (4): Update of Eq. 2 as a GRU cell (gate order r,z,n; r multiplies the
- * hidden candidate pre-activation including its bias) on the winners:
+ * hidden candidate pre-activation including its bias; TGNN_MODEL_JODIE: the plain tanh cell) on the winners:
  * memory[uniq[u]] <- GRU(msg[winner[u]], memory[uniq[u]]), last_update[uniq[u]]
  * <- t[winner[u]>>1]; every new row is computed from pre-call memory before any
  * row is written.  msg may be NULL if tgnn_build_messages ran with msg_out NULL
@@ -183,7 +197,9 @@ TGNN_API int tgnn_memory_update(tgnn_ctx* ctx, const float* msg, const int32_t* 
  * its cnt[i] valid neighbor slots, softmax over valid slots of q.k/sqrt(d/H) per
  * head (zero vector if cnt = 0), h = ReLU(W_o [a || m_root] + b_o).
  * Inputs as produced by tgnn_sample_recent -> h_out:f32[n,d].  Activations are
- * kept for tgnn_backward_step; the neighbor arrays must stay valid until then. */
+ * kept for tgnn_backward_step; the neighbor arrays must stay valid until then.
+ * TGNN_MODEL_JODIE: h[i] = memory[nodes[i]] * (1 + dt w_p + b_p) with dt = fp32(times[i] -
+ * last_update[nodes[i]]); nbr, eid, ts, cnt are ignored and may be NULL. */
 TGNN_API int tgnn_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n, const int32_t* nbr, const int32_t* eid,
                const double* ts, const int32_t* cnt, float* h_out, void* stream);
 

@@ -21,6 +21,12 @@ TGNN_MATH_FP32, TGNN_MATH_TF32, TGNN_MATH_TF32_FAST = 0, 1, 2
 
 PARAM_NAMES = ("time_w", "time_b", "gru_w_i", "gru_w_h", "gru_b_i", "gru_b_h", "w_q", "b_q", "w_k", "w_v",
                "b_k", "b_v", "w_o", "b_o", "w_1", "b_1", "w_2", "b_2")
+# the time-projection model: plain recurrent cell in the update-cell slots, no attention block, w_p | b_p
+PARAM_NAMES_JODIE = ("time_w", "time_b", "rnn_w_i", "rnn_w_h", "rnn_b_i", "rnn_b_h", "proj_w", "proj_b",
+                     "w_1", "b_1", "w_2", "b_2")
+_JODIE_SLOT = {"time_w": 0, "time_b": 1, "rnn_w_i": 2, "rnn_w_h": 3, "rnn_b_i": 4, "rnn_b_h": 5, "proj_w": 18, "proj_b": 19,
+               "w_1": 14, "b_1": 15, "w_2": 16, "b_2": 17}
+TGNN_MODEL_TGN, TGNN_MODEL_JODIE = 0, 1
 
 EXPORTS = ("tgnn_create", "tgnn_destroy", "tgnn_last_error", "tgnn_param_count", "tgnn_param_layout",
            "tgnn_set_graph", "tgnn_set_edge_features", "tgnn_set_state", "tgnn_prune_mask", "tgnn_sample_recent",
@@ -37,7 +43,8 @@ class TgnnConfig(C.Structure):
     _fields_ = [("num_nodes", C.c_int64), ("d", C.c_int32), ("d_e", C.c_int32), ("k", C.c_int32),
                 ("heads", C.c_int32), ("feat_dtype", C.c_int32), ("max_events", C.c_int32),
                 ("max_roots", C.c_int32), ("math_mode", C.c_int32),
-                ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float)]
+                ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("model", C.c_int32)]
 
 
 class TgnnError(RuntimeError):
@@ -130,24 +137,33 @@ def _stream() -> int:
 
 
 def make_config(num_nodes, d, d_e, k, heads, feat_dtype=TGNN_F32, max_events=1024, max_roots=3072,
-                math_mode=TGNN_MATH_FP32, lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8) -> TgnnConfig:
-    return TgnnConfig(num_nodes, d, d_e, k, heads, feat_dtype, max_events, max_roots, math_mode, lr, beta1, beta2, eps)
+                math_mode=TGNN_MATH_FP32, lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8, model=TGNN_MODEL_TGN) -> TgnnConfig:
+    return TgnnConfig(num_nodes, d, d_e, k, heads, feat_dtype, max_events, max_roots, math_mode, lr, beta1, beta2, eps,
+                      model)
+
+
+def param_names(cfg: TgnnConfig):
+    """Names of the model's parameter tensors in memory order."""
+    return PARAM_NAMES_JODIE if cfg.model == TGNN_MODEL_JODIE else PARAM_NAMES
 
 
 def param_layout(cfg: TgnnConfig) -> Dict[str, int]:
-    out = np.zeros(19, dtype=np.int64)
+    out = np.zeros(21, dtype=np.int64)
     rc = load_library().tgnn_param_layout(C.byref(cfg), out.ctypes.data)
     if rc != TGNN_OK:
         raise TgnnError(rc, "invalid configuration")
-    lay = {n: int(out[i]) for i, n in enumerate(PARAM_NAMES)}
-    lay["total"] = int(out[18])
+    if cfg.model == TGNN_MODEL_JODIE:
+        lay = {n: int(out[_JODIE_SLOT[n]]) for n in PARAM_NAMES_JODIE}
+    else:
+        lay = {n: int(out[i]) for i, n in enumerate(PARAM_NAMES)}
+    lay["total"] = int(out[20])
     return lay
 
 
 def pack_params(cfg: TgnnConfig, weights: Dict[str, np.ndarray]) -> np.ndarray:
     lay = param_layout(cfg)
     flat = np.zeros(lay["total"], dtype=np.float32)
-    for n in PARAM_NAMES:
+    for n in param_names(cfg):
         w = np.asarray(weights[n], dtype=np.float32).ravel()
         flat[lay[n]:lay[n] + w.size] = w
     return flat

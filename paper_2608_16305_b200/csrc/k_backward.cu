@@ -85,7 +85,7 @@ __global__ void __launch_bounds__(256) head_loss_kernel(float* __restrict__ hid1
 
 // d loss / d pre_o = ReLU'(h) * d loss / d h, where dh collects the head's input gradients.
 __global__ void __launch_bounds__(256) dh_kernel(const float* __restrict__ dcat1, const float* __restrict__ h, int nq,
-                                                 int d, float* __restrict__ dpre_o) {
+                                                 int d, float* __restrict__ dpre_o, int relu_out) {
   const int64_t total = (int64_t)3 * nq * d;
   for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
     const int i = (int)(e / d), q = (int)(e % d);
@@ -96,7 +96,7 @@ __global__ void __launch_bounds__(256) dh_kernel(const float* __restrict__ dcat1
       g = dcat1[(int64_t)(i - nq) * 2 * d + d + q];
     else
       g = dcat1[(int64_t)(i - nq) * 2 * d + d + q];
-    dpre_o[e] = h[e] > 0.f ? g : 0.f;
+    dpre_o[e] = (!relu_out || h[e] > 0.f) ? g : 0.f;
   }
 }
 
@@ -107,6 +107,8 @@ __global__ void __launch_bounds__(256) dh_kernel(const float* __restrict__ dcat1
 // of bank conflicts) while the block walks over its groups.  Also leaves what the leaves of the chain
 // need: cat1 and d loss / d pre1 (for dW_1, db_1), the hidden gates, and the sums for dw_2, db_2 and the loss.
 // Rows of hsT: 0-3 source, 4-7 destination, 8-11 negative.  Dynamic shared memory: head_fused_smem(d) bytes.
+// relu_out: the embedding rows are outputs of a ReLU layer (attention model) and dpre_o is masked by it;
+// otherwise dpre_o is the plain gradient with respect to the embedding rows.
 constexpr int HF_EV = 4, HF_THREADS = 512;
 __host__ __device__ inline int head_fused_w_floats(int d) { return (d * (2 * d + 1) + 3) & ~3; }
 inline size_t head_fused_smem(int d) {
@@ -120,7 +122,8 @@ __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __r
                                                                 float* __restrict__ cat1, float* __restrict__ dpre1,
                                                                 uint8_t* __restrict__ hid_gate,
                                                                 float* __restrict__ dpre_o, float* __restrict__ g_w2,
-                                                                float* __restrict__ g_b2, float* __restrict__ loss_acc) {
+                                                                float* __restrict__ g_b2, float* __restrict__ loss_acc,
+                                                                int relu_out) {
   extern __shared__ __align__(16) float sm[];
   __shared__ float s_msum, s_gb2, s_loss;
   const int PW = 2 * d + 1;
@@ -259,11 +262,11 @@ __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __r
           const int ev = ev0 + e;
           if (ev >= nq) break;
           if (c < d) {
-            dpre_o[(int64_t)ev * d + c] = hsT[c * 12 + e] > 0.f ? a[e] + a[4 + e] : 0.f;
+            dpre_o[(int64_t)ev * d + c] = (!relu_out || hsT[c * 12 + e] > 0.f) ? a[e] + a[4 + e] : 0.f;
           } else {
             const int q = c - d;
-            dpre_o[((int64_t)nq + ev) * d + q] = hsT[q * 12 + 4 + e] > 0.f ? a[e] : 0.f;
-            dpre_o[((int64_t)2 * nq + ev) * d + q] = hsT[q * 12 + 8 + e] > 0.f ? a[4 + e] : 0.f;
+            dpre_o[((int64_t)nq + ev) * d + q] = (!relu_out || hsT[q * 12 + 4 + e] > 0.f) ? a[e] : 0.f;
+            dpre_o[((int64_t)2 * nq + ev) * d + q] = (!relu_out || hsT[q * 12 + 8 + e] > 0.f) ? a[4 + e] : 0.f;
           }
         }
       }
@@ -438,6 +441,68 @@ __global__ void __launch_bounds__(256) time_grad_kernel(const float* __restrict_
   }
 }
 
+// Backward of the time-projected embedding h = m * (1 + dt w_p + b_p), one warp per root:
+//   dw_p += dh m dt,  db_p += dh m   (fp64 block sums, then one pair of fp64 atomics per block and column into
+//                                     acc[0:d] and acc[d:2d]: dt spans the stream and the terms cancel)
+//   dm = dh (1 + dt w_p + b_p) is added to the row's slot of dMemU when the node's memory row was written
+//   by this step's update (all other table rows are constants).
+// Dynamic shared memory: 8 * 2 * d doubles.
+__global__ void __launch_bounds__(256) jodie_embed_bwd_kernel(const float* __restrict__ dh, const float* __restrict__ memory,
+                                                              const double* __restrict__ last_update,
+                                                              const float* __restrict__ proj_w,
+                                                              const float* __restrict__ proj_b,
+                                                              const int32_t* __restrict__ nodes,
+                                                              const double* __restrict__ times, int n, int d,
+                                                              const int32_t* __restrict__ node2slot, int have_update,
+                                                              float* __restrict__ dMemU, double* __restrict__ acc) {
+  extern __shared__ double s_part[];  // [8][2][d]
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  double gw[TG_MAXJ], gb[TG_MAXJ];
+#pragma unroll
+  for (int j = 0; j < TG_MAXJ; ++j) { gw[j] = 0.0; gb[j] = 0.0; }
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  for (int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
+    const int node = nodes[i];
+    const float dt = (float)(times[i] - last_update[node]);
+    const int slot = have_update ? node2slot[node] : -1;
+#pragma unroll
+    for (int j = 0; j < TG_MAXJ; ++j) {
+      const int c = lane + 32 * j;
+      if (c < d) {
+        const float g = dh[(int64_t)i * d + c];
+        const float m = memory[(int64_t)node * d + c];
+        const double t = (double)g * (double)m;
+        gw[j] = fma(t, (double)dt, gw[j]);
+        gb[j] += t;
+        if (slot >= 0) atomicAdd(&dMemU[(int64_t)slot * d + c], g * (1.f + fmaf(dt, proj_w[c], proj_b[c])));
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < TG_MAXJ; ++j) {
+    const int c = lane + 32 * j;
+    if (c < d) { s_part[(wid * 2 + 0) * d + c] = gw[j]; s_part[(wid * 2 + 1) * d + c] = gb[j]; }
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < 2 * d; e += blockDim.x) {
+    double t = 0.0;
+    for (int w = 0; w < 8; ++w) t += s_part[w * 2 * d + e];
+    if (t != 0.0) atomicAdd(&acc[e], t);
+  }
+}
+
+// Backward of the plain recurrent cell for the rows the memory update wrote: d pre = dm' (1 - m'^2).
+__global__ void __launch_bounds__(256) rnn_bwd_gate_kernel(const float* __restrict__ dMemU, const float* __restrict__ g_n,
+                                                           const int32_t* __restrict__ n_uniq, int u_cap, int d,
+                                                           float* __restrict__ dG) {
+  const int U = min(*n_uniq, u_cap);
+  const int64_t total = (int64_t)U * d;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const float m = g_n[e];
+    dG[e] = dMemU[e] * (1.f - m * m);
+  }
+}
+
 // Backward of the GRU gates for the rows the memory update wrote.
 __global__ void __launch_bounds__(256) gru_bwd_gate_kernel(const float* __restrict__ dMemU, const float* __restrict__ X,
                                                            int ld, int d, const float* __restrict__ g_r,
@@ -468,11 +533,11 @@ __global__ void __launch_bounds__(256) gru_bwd_gate_kernel(const float* __restri
 // norm (no clipping), so each thread squares its gradient entries into the block's partial sum and
 // updates the same entries; the last block to finish turns the sum into g_r and bumps the step counter
 // (every block has read the counter before it takes its ticket).
-// The time-encoder entries [t_off, t_off + t_n) are taken from their fp64 sums tg_acc (rounded once)
-// and written into grads, where the debug export finds them.
+// The time-encoder entries [t_off, t_off + t_n) and the time projection's [p_off, p_off + p_n) are taken
+// from their fp64 sums tg_acc (rounded once) and written into grads, where the debug export finds them.
 __global__ void __launch_bounds__(256) gradnorm_adam_kernel(float* __restrict__ grads, int64_t P,
                                                             const double* __restrict__ tg_acc, int64_t t_off, int t_n,
-                                                            double* red, unsigned int* ticket, int64_t* step,
+                                                            int64_t p_off, int p_n, double* red, unsigned int* ticket, int64_t* step,
                                                             float* __restrict__ p, float* __restrict__ m,
                                                             float* __restrict__ v, float lr, float beta1, float beta2,
                                                             float eps, const float* __restrict__ loss_acc, float* scalars,
@@ -493,6 +558,9 @@ __global__ void __launch_bounds__(256) gradnorm_adam_kernel(float* __restrict__ 
     float ge;
     if (e >= t_off && e < t_off + t_n) {
       ge = (float)tg_acc[e - t_off];
+      grads[e] = ge;
+    } else if (e >= p_off && e < p_off + p_n) {  // the projection's w_p | b_p, summed in fp64 behind the time encoder's
+      ge = (float)tg_acc[t_n + (e - p_off)];
       grads[e] = ge;
     } else {
       ge = grads[e];
@@ -607,6 +675,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
   if (n_q > 0) {
     // One block does the head forward and backward for 4 events at a time when W_1 fits in shared memory
     // beside the staging rows; wider models take the projections through the GEMM path instead.
+    const int relu_out = c.model == TGNN_MODEL_TGN ? 1 : 0;
     const size_t hf_smem = head_fused_smem(d);
     if (hf_smem <= 200 * 1024) {
       static size_t attr_bytes = 0;
@@ -619,7 +688,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
         KernelScope scope__(ctx, "head_fused", s);
         head_fused_kernel<<<groups < 296 ? groups : 296, HF_THREADS, hf_smem, s>>>(
             ctx->e_h, P + L.w1, P + L.b1, P + L.w2, P + L.b2, loss_mask, n_q, d, w.cat1, w.hid1, w.hid_gate, w.dpre_o,
-            G + L.w2, G + L.b2, w.st_scalars);
+            G + L.w2, G + L.b2, w.st_scalars, relu_out);
       }
       TGNN_LAUNCH_OK(ctx, "head_fused");
       RC(fork_to(ctx, s, sa));
@@ -650,10 +719,46 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       const int64_t tot2 = (int64_t)R * d;
       {
         KernelScope scope__(ctx, "dh", s);
-        dh_kernel<<<(int)((tot2 + 255) / 256), 256, 0, s>>>(w.dcat1, ctx->e_h, n_q, d, w.dpre_o);
+        dh_kernel<<<(int)((tot2 + 255) / 256), 256, 0, s>>>(w.dcat1, ctx->e_h, n_q, d, w.dpre_o, relu_out);
       }
       TGNN_LAUNCH_OK(ctx, "dh");
     }
+    if (c.model == TGNN_MODEL_JODIE) {
+      // embedding -> memory rows written by this step -> recurrent cell -> its weights and the time encoder
+      const size_t tg_smem = (size_t)8 * 2 * d * sizeof(double);
+      {
+        KernelScope scope__(ctx, "jodie_embed_bwd", s);
+        jodie_embed_bwd_kernel<<<(R + 7) / 8 < 592 ? (R + 7) / 8 : 592, 256, tg_smem, s>>>(
+            w.dpre_o, ctx->memory, ctx->last_update, P + L.proj_w, P + L.proj_b, ctx->e_nodes, ctx->e_times, R, d,
+            w.node2slot, ctx->have_update ? 1 : 0, w.dMemU, w.tg_acc + 2 * d);
+      }
+      TGNN_LAUNCH_OK(ctx, "jodie_embed_bwd");
+      if (ctx->have_update) {
+        const int U_cap = ctx->upd_cap;
+        const int64_t tot3 = (int64_t)U_cap * d;
+        {
+          KernelScope scope__(ctx, "rnn_bwd_gate", s);
+          rnn_bwd_gate_kernel<<<(int)((tot3 + 255) / 256), 256, 0, s>>>(w.dMemU, w.g_n, ctx->upd_n_uniq, U_cap, d, w.dGi);
+        }
+        TGNN_LAUNCH_OK(ctx, "rnn_bwd_gate");
+        RC(fork_to(ctx, s, sa));
+        RC(fork_to(ctx, s, sb));
+        RC(grad_w(ctx, w.dGi, d, w.X, ctx->ld_msg, U_cap, ctx->upd_n_uniq, d, (int)L.dmsg, G + L.gru_wi, G + L.gru_bi,
+                  "dW_i", sa));
+        RC(grad_w(ctx, w.dGi, d, w.X, ctx->ld_msg, U_cap, ctx->upd_n_uniq, d, d, G + L.gru_wh, G + L.gru_bh, "dW_h", sb));
+        RC(grad_in(ctx, w.dGi, d, P + L.gru_wi, L.dmsg, 2 * d + de, U_cap, ctx->upd_n_uniq, d, d, w.dXp, d, "dX_phi", s,
+                   SITE_DXPHI + 1));
+        {
+          KernelScope scope__(ctx, "time_grad_x", s);
+          const int rpb = tg_rows_per_block(U_cap);
+          time_grad_kernel<<<(U_cap + rpb - 1) / rpb, 256, tg_smem, s>>>(w.dXp, d, 0, w.Xsin, w.x_dt, U_cap,
+                                                                         ctx->upd_n_uniq, d, P + L.time_b, w.tg_acc, rpb);
+        }
+        TGNN_LAUNCH_OK(ctx, "time_grad_x");
+      }
+      RC(fork_to(ctx, sa, s));  // join
+      RC(fork_to(ctx, sb, s));
+    } else {
     RC(fork_to(ctx, s, sb));
     RC(grad_w(ctx, w.dpre_o, d, w.cat_o, 2 * d, R, nullptr, d, 2 * d, G + L.wo, G + L.bo, "dW_o", sb));
     RC(grad_in(ctx, w.dpre_o, d, P + L.wo, 2 * d, 0, R, nullptr, d, 2 * d, w.dcat_o, 2 * d, "dcat_o", s, SITE_DCATO + 1));
@@ -743,10 +848,12 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     }
     RC(fork_to(ctx, sa, s));  // join
     RC(fork_to(ctx, sb, s));
+    }  // attention model
   }
   {
     KernelScope scope__(ctx, "gradnorm_adam", s);
-    gradnorm_adam_kernel<<<296, 256, 0, s>>>(G, L.total, w.tg_acc, L.time_w, n_q > 0 ? 2 * d : 0, w.red, w.counters,
+    const int p_n = (n_q > 0 && c.model == TGNN_MODEL_JODIE) ? 2 * d : 0;
+    gradnorm_adam_kernel<<<296, 256, 0, s>>>(G, L.total, w.tg_acc, L.time_w, n_q > 0 ? 2 * d : 0, L.proj_w, p_n, w.red, w.counters,
                                              ctx->step, P, ctx->adam_m, ctx->adam_v, c.lr, c.beta1, c.beta2, c.eps,
                                              w.st_scalars, w.st_scalars + 2, loss_out, gradnorm_out);
   }

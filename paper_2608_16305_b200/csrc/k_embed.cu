@@ -133,6 +133,35 @@ __global__ void __launch_bounds__(256) attention_fwd_kernel(const float* __restr
   }
 }
 
+// Time-projected embedding: h[i] = memory[node_i] * (1 + dt_i w_p + b_p), dt_i = fp32(t_i - last_update[node_i]).
+// One warp per root, 128-bit accesses (d is a multiple of 4, rows 16-byte aligned).
+__global__ void __launch_bounds__(256) jodie_embed_kernel(const float* __restrict__ memory,
+                                                          const double* __restrict__ last_update,
+                                                          const float* __restrict__ proj_w,
+                                                          const float* __restrict__ proj_b,
+                                                          const int32_t* __restrict__ nodes,
+                                                          const double* __restrict__ times, int n, int d,
+                                                          float* __restrict__ h) {
+  const int lane = threadIdx.x & 31;
+  const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (i >= n) return;
+  const int node = nodes[i];
+  const float dt = (float)(times[i] - last_update[node]);
+  const float4* m4 = reinterpret_cast<const float4*>(memory + (int64_t)node * d);
+  float4* h4 = reinterpret_cast<float4*>(h + (int64_t)i * d);
+  for (int q = lane; q < (d >> 2); q += 32) {
+    const float4 m = __ldg(m4 + q);
+    const float4 w = *reinterpret_cast<const float4*>(proj_w + 4 * q);
+    const float4 b = *reinterpret_cast<const float4*>(proj_b + 4 * q);
+    float4 o;
+    o.x = m.x * (1.f + fmaf(dt, w.x, b.x));
+    o.y = m.y * (1.f + fmaf(dt, w.y, b.y));
+    o.z = m.z * (1.f + fmaf(dt, w.z, b.z));
+    o.w = m.w * (1.f + fmaf(dt, w.w, b.w));
+    h4[q] = o;
+  }
+}
+
 }  // namespace
 
 int launch_embed_static(tgnn_ctx* ctx, const double* times, int n, const int32_t* nbr, const int32_t* eid,
@@ -159,6 +188,15 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
   const ParamLayout& L = ctx->L;
   Workspace& w = ctx->ws;
   const int d = c.d, k = c.k, H = c.heads;
+  if (c.model == TGNN_MODEL_JODIE) {
+    {
+      KernelScope scope__(ctx, "jodie_embed", s);
+      jodie_embed_kernel<<<(n + 7) / 8, 256, 0, s>>>(ctx->memory, ctx->last_update, ctx->params + L.proj_w,
+                                                     ctx->params + L.proj_b, nodes, times, n, d, h_out);
+    }
+    TGNN_LAUNCH_OK(ctx, "jodie_embed");
+    return TGNN_OK;
+  }
   const int rows = n * k + n;
   if (!ctx->z_static_done) {
     const int rc0 = launch_embed_static(ctx, times, n, nbr, eid, ts, s);

@@ -685,22 +685,29 @@ size_t plan_weight_sites(tgnn_ctx* ctx) {
   const bool all_precise = ctx->cfg.math_mode == TGNN_MATH_TF32;
   struct Def { int id; int64_t w_off, ld; int major, N, K, col0, n_split, col1, M_cap, split_acc, grad; };
   const int U = ctx->U_cap, R = ctx->R_cap, NB = ctx->NB_cap, Q2 = 2 * ctx->nq_cap;
+  const int gd = (int)L.gates * d;              // rows of the update cell's matrices
+  const int att = L.wo > L.wq ? 1 : 0;          // the attention block is empty for the time-projection model
   const Def defs[SITE_COUNT] = {
-      {SITE_GI, L.gru_wi, L.dmsg, MAJOR_K, 3 * d, (int)L.dmsg, 0, 0, 0, U, 1, 0},
-      {SITE_GH, L.gru_wh, d, MAJOR_K, 3 * d, d, 0, 0, 0, U, 0, 0},
-      {SITE_KV, L.wk, L.dkv, MAJOR_K, 2 * d, (int)L.dkv, 0, 0, 0, NB, 0, 0},
-      {SITE_Q, L.wq, 2 * d, MAJOR_K, d, 2 * d, 0, 0, 0, R, 0, 0},
-      {SITE_OUT, L.wo, 2 * d, MAJOR_K, d, 2 * d, 0, 0, 0, R, 0, 0},
+      {SITE_GI, L.gru_wi, L.dmsg, MAJOR_K, gd, (int)L.dmsg, 0, 0, 0, U, 1, 0},
+      {SITE_GH, L.gru_wh, d, MAJOR_K, gd, d, 0, 0, 0, U, 0, 0},
+      {SITE_KV, L.wk, L.dkv, MAJOR_K, att * 2 * d, (int)L.dkv, 0, 0, 0, NB, 0, 0},
+      {SITE_Q, L.wq, 2 * d, MAJOR_K, att * d, 2 * d, 0, 0, 0, R, 0, 0},
+      {SITE_OUT, L.wo, 2 * d, MAJOR_K, att * d, 2 * d, 0, 0, 0, R, 0, 0},
       {SITE_HEAD, L.w1, 2 * d, MAJOR_K, d, 2 * d, 0, 0, 0, Q2, 0, 0},
       {SITE_DCAT1, L.w1, 2 * d, MAJOR_MN, 2 * d, d, 0, 2 * d, 0, Q2, 0, 1},
-      {SITE_DCATO, L.wo, 2 * d, MAJOR_MN, 2 * d, d, 0, 2 * d, 0, R, 0, 1},
-      {SITE_DZQ, L.wq, 2 * d, MAJOR_MN, 2 * d, d, 0, 2 * d, 0, R, 0, 1},
-      {SITE_DZ, L.wk, L.dkv, MAJOR_MN, 2 * d, 2 * d, 0, d, d + de, NB, 0, 1},
-      {SITE_DXPHI, L.gru_wi, L.dmsg, MAJOR_MN, d, 3 * d, 2 * d + de, d, 0, U, 0, 1},
+      {SITE_DCATO, L.wo, 2 * d, MAJOR_MN, att * 2 * d, d, 0, 2 * d, 0, R, 0, 1},
+      {SITE_DZQ, L.wq, 2 * d, MAJOR_MN, att * 2 * d, d, 0, 2 * d, 0, R, 0, 1},
+      {SITE_DZ, L.wk, L.dkv, MAJOR_MN, att * 2 * d, 2 * d, 0, d, d + de, NB, 0, 1},
+      {SITE_DXPHI, L.gru_wi, L.dmsg, MAJOR_MN, d, gd, 2 * d + de, d, 0, U, 0, 1},
   };
   size_t off = 0;
   for (const Def& f : defs) {
     WeightSite& st = ctx->sites[f.id];
+    if (f.N == 0) {  // a projection this model does not have: an empty image
+      st = WeightSite{};
+      st.image_off = (int64_t)off;
+      continue;
+    }
     st.w_off = f.w_off; st.ld = f.ld; st.major = f.major; st.N = f.N; st.K = f.K;
     st.col0 = f.col0; st.n_split = f.n_split; st.col1 = f.col1;
     st.precise = (all_precise || f.grad) ? 1 : 0;

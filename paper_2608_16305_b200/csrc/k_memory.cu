@@ -117,6 +117,25 @@ __global__ void __launch_bounds__(256) gru_gate_kernel(const float* __restrict__
   }
 }
 
+// The plain recurrent cell and write-back: m' = tanh(Gi + Gh) with Gi = W_i x + b_i, Gh = W_h h + b_h
+// (row pitch d).  The new row is kept in g_n for the backward pass (d tanh = 1 - m'^2).
+__global__ void __launch_bounds__(256) rnn_gate_kernel(const float* __restrict__ Gi, const float* __restrict__ Gh, int d,
+                                                       const int32_t* __restrict__ uniq, const double* __restrict__ win_t,
+                                                       const int32_t* __restrict__ n_uniq, int u_cap,
+                                                       float* __restrict__ g_n, float* __restrict__ memory,
+                                                       double* __restrict__ last_update) {
+  const int U = min(*n_uniq, u_cap);
+  const int64_t total = (int64_t)U * d;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int u = (int)(e / d), q = (int)(e % d);
+    const float hnew = tanhf(Gi[e] + Gh[e]);
+    g_n[e] = hnew;
+    const int node = uniq[u];
+    memory[(int64_t)node * d + q] = hnew;
+    if (q == 0) last_update[node] = win_t[u];
+  }
+}
+
 }  // namespace
 
 int launch_build_messages(tgnn_ctx* ctx, const int32_t* src, const int32_t* dst, const double* t, const int32_t* eid,
@@ -141,6 +160,7 @@ int launch_memory_update(tgnn_ctx* ctx, const float* msg, const int32_t* uniq, c
   const ParamLayout& L = ctx->L;
   Workspace& w = ctx->ws;
   const int d = c.d, U_cap = min(ctx->U_cap, 2 * ctx->m_n);
+  const int gd = (int)L.gates * d;  // rows of the cell's matrices: 3d (GRU) or d (plain cell)
   if (U_cap == 0) return TGNN_OK;
   {
     KernelScope scope__(ctx, "gather_winner", s);
@@ -154,11 +174,11 @@ int launch_memory_update(tgnn_ctx* ctx, const float* msg, const int32_t* uniq, c
   GemmArgs g = {};
   g.A = w.X; g.a_rs = ctx->ld_msg; g.a_cs = 1;
   g.B = ctx->params + L.gru_wi; g.b_rs = 1; g.b_cs = L.dmsg;  // B(k,n) = W_i[n,k]
-  g.C = w.Gi; g.ldc = 3 * d; g.M = U_cap; g.N = 3 * d; g.K = (int)L.dmsg; g.dev_M = n_uniq;
+  g.C = w.Gi; g.ldc = gd; g.M = U_cap; g.N = gd; g.K = (int)L.dmsg; g.dev_M = n_uniq;
   g.bias = ctx->params + L.gru_bi;
   // few rows, long contraction: split the contraction over CTAs and accumulate into a cleared Gi
   g.accumulate = 1; g.split_k = 4; g.site = SITE_GI + 1;
-  TGNN_CUDA_OK(ctx, cudaMemsetAsync(w.Gi, 0, sizeof(float) * (size_t)U_cap * 3 * d, s));
+  TGNN_CUDA_OK(ctx, cudaMemsetAsync(w.Gi, 0, sizeof(float) * (size_t)U_cap * gd, s));
   int rc = fork_to(ctx, s, ctx->side[0]);  // the hidden-state product runs beside the input product
   if (rc) return rc;
   rc = launch_gemm(ctx, g, "gru_gi", s);
@@ -170,6 +190,15 @@ int launch_memory_update(tgnn_ctx* ctx, const float* msg, const int32_t* uniq, c
   rc = fork_to(ctx, ctx->side[0], s);
   if (rc) return rc;
   const int64_t total = (int64_t)U_cap * d;
+  if (c.model == TGNN_MODEL_JODIE) {
+    {
+      KernelScope scope__(ctx, "rnn_gate", s);
+      rnn_gate_kernel<<<(int)((total + 255) / 256), 256, 0, s>>>(w.Gi, w.Gh, d, uniq, w.win_t, n_uniq, U_cap, w.g_n,
+                                                                 ctx->memory, ctx->last_update);
+    }
+    TGNN_LAUNCH_OK(ctx, "rnn_gate");
+    return TGNN_OK;
+  }
   {
     KernelScope scope__(ctx, "gru_gate", s);
     gru_gate_kernel<<<(int)((total + 255) / 256), 256, 0, s>>>(w.Gi, w.Gh, w.X, ctx->ld_msg, d, uniq, w.win_t, n_uniq,

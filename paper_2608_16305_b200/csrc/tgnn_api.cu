@@ -10,25 +10,29 @@
 
 namespace tgnn {
 
-ParamLayout make_layout(int d_, int de_) {
+ParamLayout make_layout(int d_, int de_, int model) {
   ParamLayout L;
   const int64_t d = d_, de = de_;
-  L.d = d; L.de = de; L.dmsg = 3 * d + de; L.dkv = 2 * d + de; L.dq = 2 * d;
+  const bool jodie = model == TGNN_MODEL_JODIE;
+  const int64_t g = jodie ? 1 : 3, att = jodie ? 0 : 1, prj = jodie ? 1 : 0;
+  L.d = d; L.de = de; L.dmsg = 3 * d + de; L.dkv = 2 * d + de; L.dq = 2 * d; L.gates = g;
   int64_t o = 0;
   L.time_w = o; o += d;
   L.time_b = o; o += d;
-  L.gru_wi = o; o += 3 * d * L.dmsg;
-  L.gru_wh = o; o += 3 * d * d;
-  L.gru_bi = o; o += 3 * d;
-  L.gru_bh = o; o += 3 * d;
-  L.wq = o; o += d * L.dq;
-  L.bq = o; o += d;
-  L.wk = o; o += d * L.dkv;
-  L.wv = o; o += d * L.dkv;
-  L.bk = o; o += d;
-  L.bv = o; o += d;
-  L.wo = o; o += d * 2 * d;
-  L.bo = o; o += d;
+  L.gru_wi = o; o += g * d * L.dmsg;
+  L.gru_wh = o; o += g * d * d;
+  L.gru_bi = o; o += g * d;
+  L.gru_bh = o; o += g * d;
+  L.wq = o; o += att * d * L.dq;
+  L.bq = o; o += att * d;
+  L.wk = o; o += att * d * L.dkv;
+  L.wv = o; o += att * d * L.dkv;
+  L.bk = o; o += att * d;
+  L.bv = o; o += att * d;
+  L.wo = o; o += att * d * 2 * d;
+  L.bo = o; o += att * d;
+  L.proj_w = o; o += prj * d;
+  L.proj_b = o; o += prj * d;
   L.w1 = o; o += d * 2 * d;
   L.b1 = o; o += d;
   L.w2 = o; o += d;
@@ -58,6 +62,7 @@ int check_config(const tgnn_config* c) {
   if (c->feat_dtype != TGNN_F32 && c->feat_dtype != TGNN_BF16) return TGNN_EINVAL;
   if (c->max_events < 1 || c->max_roots < 3 || c->max_events > (1 << 24) || c->max_roots > (1 << 24)) return TGNN_EINVAL;
   if (c->math_mode != TGNN_MATH_FP32 && c->math_mode != TGNN_MATH_TF32 && c->math_mode != TGNN_MATH_TF32_FAST) return TGNN_EINVAL;
+  if (c->model != TGNN_MODEL_TGN && c->model != TGNN_MODEL_JODIE) return TGNN_EINVAL;
   if (!(c->lr >= 0.f) || !(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f) || !(c->eps > 0.f))
     return TGNN_EINVAL;
   return TGNN_OK;
@@ -144,7 +149,7 @@ size_t carve(tgnn_ctx* ctx, char* base) {
   cv.take(w.grads, (size_t)ctx->L.total);
   cv.take_packed(w.dMemU, U * d);
   cv.take_packed(w.red, 4);
-  cv.take_packed(w.tg_acc, 2 * d);
+  cv.take_packed(w.tg_acc, 4 * d);  // time encoder dw | db, time projection dw_p | db_p
   cv.take_packed(w.st_scalars, 4);
   return (cv.off + 255) & ~(size_t)255;
 }
@@ -165,17 +170,17 @@ extern "C" {
 
 int64_t tgnn_param_count(const tgnn_config* cfg) {
   if (check_config(cfg) != TGNN_OK) return -1;
-  return make_layout(cfg->d, cfg->d_e).total;
+  return make_layout(cfg->d, cfg->d_e, cfg->model).total;
 }
 
 int tgnn_param_layout(const tgnn_config* cfg, int64_t* out) {
   const int rc = check_config(cfg);
   if (rc != TGNN_OK) return rc;
   if (!out) return TGNN_EINVAL;
-  const ParamLayout L = make_layout(cfg->d, cfg->d_e);
-  const int64_t v[19] = {L.time_w, L.time_b, L.gru_wi, L.gru_wh, L.gru_bi, L.gru_bh, L.wq, L.bq, L.wk, L.wv,
-                         L.bk, L.bv, L.wo, L.bo, L.w1, L.b1, L.w2, L.b2, L.total};
-  for (int i = 0; i < 19; ++i) out[i] = v[i];
+  const ParamLayout L = make_layout(cfg->d, cfg->d_e, cfg->model);
+  const int64_t v[21] = {L.time_w, L.time_b, L.gru_wi, L.gru_wh, L.gru_bi, L.gru_bh, L.wq, L.bq, L.wk, L.wv, L.bk,
+                         L.bv, L.wo, L.bo, L.w1, L.b1, L.w2, L.b2, L.proj_w, L.proj_b, L.total};
+  for (int i = 0; i < 21; ++i) out[i] = v[i];
   return TGNN_OK;
 }
 
@@ -191,7 +196,7 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
   tgnn_ctx* ctx = new (std::nothrow) tgnn_ctx();
   if (!ctx) return TGNN_ECUDA;
   ctx->cfg = *cfg;
-  ctx->L = make_layout(cfg->d, cfg->d_e);
+  ctx->L = make_layout(cfg->d, cfg->d_e, cfg->model);
   ctx->U_cap = 2 * cfg->max_events;
   ctx->R_cap = cfg->max_roots;
   ctx->NB_cap = cfg->max_roots * cfg->k;
@@ -388,7 +393,9 @@ int tgnn_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n, 
   NEED(ctx, ctx->cfg.d_e == 0 || ctx->efeat, TGNN_ESTATE, "embed: tgnn_set_edge_features has not been called");
   NEED(ctx, n >= 0, TGNN_EINVAL, "embed: negative n");
   NEED(ctx, n <= ctx->R_cap, TGNN_ECAPACITY, "embed: n %d > max_roots %d", n, ctx->R_cap);
-  NEED(ctx, n == 0 || (nodes && times && nbr && eid && ts && cnt && h_out), TGNN_EINVAL, "embed: null pointer");
+  const bool needs_nbrs = ctx->cfg.model == TGNN_MODEL_TGN;
+  NEED(ctx, n == 0 || (nodes && times && h_out && (!needs_nbrs || (nbr && eid && ts && cnt))), TGNN_EINVAL,
+       "embed: null pointer");
   ctx->e_nodes = nodes; ctx->e_times = times; ctx->e_nbr = nbr; ctx->e_eid = eid; ctx->e_ts = ts; ctx->e_cnt = cnt;
   ctx->e_n = n; ctx->e_h = h_out; ctx->have_embed = true;
   return launch_embed(ctx, nodes, times, n, nbr, eid, ts, cnt, h_out, S(stream));
@@ -435,13 +442,15 @@ int step_body(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q, bool has_mask, flo
   }
   rc = launch_make_roots(ctx, w.st_q_src, w.st_q_dst, w.st_q_neg, w.st_q_t, n_q, side);
   if (rc) return rc;
-  rc = tgnn_sample_recent(ctx, w.r_node, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, w.nb_cnt, side);
-  if (rc) return rc;
-  // edge features and time encodings of the sampled neighbors do not depend on memory either
   NEED(ctx, ctx->cfg.d_e == 0 || ctx->efeat, TGNN_ESTATE, "train_step: tgnn_set_edge_features has not been called");
-  rc = launch_embed_static(ctx, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, side);
-  if (rc) return rc;
-  ctx->z_static_done = true;
+  if (ctx->cfg.model == TGNN_MODEL_TGN) {  // the time-projected embedding samples no neighbors
+    rc = tgnn_sample_recent(ctx, w.r_node, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, w.nb_cnt, side);
+    if (rc) return rc;
+    // edge features and time encodings of the sampled neighbors do not depend on memory either
+    rc = launch_embed_static(ctx, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, side);
+    if (rc) return rc;
+    ctx->z_static_done = true;
+  }
   if (n_u > 0) {
     // messages stay virtual: the reduction reads the event arrays, the memory update gathers the winners
     ctx->m_src = w.st_u_src; ctx->m_dst = w.st_u_dst; ctx->m_t = w.st_u_t; ctx->m_eid = w.st_u_eid;

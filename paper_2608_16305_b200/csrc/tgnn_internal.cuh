@@ -12,9 +12,11 @@ namespace tgnn {
 // Offsets of the parameter tensors in the flat vector (order fixed by the public header).
 struct ParamLayout {
   int64_t d, de, dmsg, dkv, dq;
-  int64_t time_w, time_b, gru_wi, gru_wh, gru_bi, gru_bh, wq, bq, wk, wv, bk, bv, wo, bo, w1, b1, w2, b2, total;
+  int64_t gates;  // rows of the update cell's matrices in units of d: 3 (GRU) or 1 (plain recurrent cell)
+  int64_t time_w, time_b, gru_wi, gru_wh, gru_bi, gru_bh, wq, bq, wk, wv, bk, bv, wo, bo, proj_w, proj_b, w1, b1, w2, b2,
+      total;
 };
-ParamLayout make_layout(int d, int d_e);
+ParamLayout make_layout(int d, int d_e, int model);
 
 // Workspace: everything the step keeps between entry points.  Row-major, fp32 unless noted.
 struct Workspace {

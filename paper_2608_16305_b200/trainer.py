@@ -129,12 +129,13 @@ class PartitionedWorkload(DeviceWorkload):
 
 
 class Trainer:
-    def __init__(self, dw: DeviceWorkload, weights, math_mode=B.TGNN_MATH_FP32, lr=1e-4):
+    def __init__(self, dw: DeviceWorkload, weights, math_mode=B.TGNN_MATH_FP32, lr=1e-4, model: str = "tgn"):
         cfg = dw.cfg
         self.dw = dw
         self.tcfg = B.make_config(cfg.num_nodes, cfg.d, cfg.d_e, cfg.k, cfg.heads,
                                   feat_dtype=B.TGNN_BF16 if cfg.feat_dtype == "bf16" else B.TGNN_F32,
-                                  max_events=dw.max_mixed, max_roots=3 * dw.max_targets, math_mode=math_mode, lr=lr)
+                                  max_events=dw.max_mixed, max_roots=3 * dw.max_targets, math_mode=math_mode, lr=lr,
+                                  model=B.TGNN_MODEL_JODIE if model == "jodie" else B.TGNN_MODEL_TGN)
         self.lib = B.Tgnn(self.tcfg)
         dev = dw.device
         P = B.param_layout(self.tcfg)["total"]

@@ -297,8 +297,15 @@ PARAM_SHAPES = (
 )
 
 
-def param_shapes(d: int, d_e: int) -> Dict[str, tuple]:
+def param_shapes(d: int, d_e: int, model: str = "tgn") -> Dict[str, tuple]:
     d_msg, d_kv = 3 * d + d_e, 2 * d + d_e
+    if model == "jodie":   # plain recurrent cell, time projection (w_p, b_p), the same head
+        return {
+            "time_w": (d,), "time_b": (d,),
+            "rnn_w_i": (d, d_msg), "rnn_w_h": (d, d), "rnn_b_i": (d,), "rnn_b_h": (d,),
+            "proj_w": (d,), "proj_b": (d,),
+            "w_1": (d, 2 * d), "b_1": (d,), "w_2": (d,), "b_2": (1,),
+        }
     return {
         "time_w": (d,), "time_b": (d,),
         "gru_w_i": (3 * d, d_msg), "gru_w_h": (3 * d, d), "gru_b_i": (3 * d,), "gru_b_h": (3 * d,),
@@ -309,11 +316,12 @@ def param_shapes(d: int, d_e: int) -> Dict[str, tuple]:
     }
 
 
-def make_weights(d: int, d_e: int, seed: int, bias_scale: float = 0.0) -> Dict[str, np.ndarray]:
-    """Named fp32 tensors; matrices are [out, in] row-major."""
+def make_weights(d: int, d_e: int, seed: int, bias_scale: float = 0.0, model: str = "tgn") -> Dict[str, np.ndarray]:
+    """Named fp32 tensors; matrices are [out, in] row-major.  The time projection's slope w_p multiplies raw
+    time differences (hundreds to thousands of mean gaps), so it is drawn 1000 times smaller than the biases."""
     rng = np.random.Generator(np.random.Philox(key=np.array([seed, 0xBEEF], dtype=np.uint64)))
     out: Dict[str, np.ndarray] = {}
-    for name, shape in param_shapes(d, d_e).items():
+    for name, shape in param_shapes(d, d_e, model).items():
         if name == "time_w":
             c = np.arange(d, dtype=np.float64)
             out[name] = (10.0 ** (-9.0 * c / max(d - 1, 1))).astype(np.float32)
@@ -325,5 +333,5 @@ def make_weights(d: int, d_e: int, seed: int, bias_scale: float = 0.0) -> Dict[s
             out[name] = rng.uniform(-a, a, size=shape).astype(np.float32)
         else:
             v = rng.uniform(-bias_scale, bias_scale, size=shape) if bias_scale > 0 else np.zeros(shape)
-            out[name] = v.astype(np.float32)
+            out[name] = (v * (1e-3 if name == "proj_w" else 1.0)).astype(np.float32)
     return out

@@ -7,6 +7,7 @@ import subprocess
 import sys
 
 import numpy as np
+import pytest
 import torch
 
 from paper_2608_16305_b200 import workload as wl
@@ -147,3 +148,21 @@ print("ok", rank)
         out, err = p.communicate(timeout=120)
         assert p.returncode == 0, err.decode()[-2000:]
         assert b"ok" in out
+
+
+def test_jodie_layout_matches_the_oracles_and_tgn_layout_is_unchanged():
+    from oracle import jodie as oj
+    from paper_2608_16305_b200 import binding
+    for name in ("tiny", "wiki", "lastfm"):
+        c = wl.CONFIGS[name]
+        cfg = binding.make_config(c.num_nodes, c.d, c.d_e, c.k, c.heads, model=binding.TGNN_MODEL_JODIE)
+        lay, ref = binding.param_layout(cfg), oj.param_layout(c.d, c.d_e)
+        assert lay == {k: ref[k] for k in lay}
+        shapes = wl.param_shapes(c.d, c.d_e, "jodie")
+        assert tuple(shapes) == binding.PARAM_NAMES_JODIE == oj.PARAM_NAMES
+        assert sum(int(np.prod(s)) for s in shapes.values()) == lay["total"]
+        w = wl.make_weights(c.d, c.d_e, c.seed, bias_scale=0.1, model="jodie")
+        flat = binding.pack_params(cfg, w)
+        assert np.array_equal(flat, oj.pack(c.d, c.d_e, w).astype(np.float32))
+    with pytest.raises(binding.TgnnError):
+        binding.param_layout(binding.make_config(100, 32, 16, 10, 2, model=7))

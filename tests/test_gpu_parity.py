@@ -55,7 +55,7 @@ def orc_cfg(oracle, c, **kw):
 class Rig:
     """A workload on the device plus a library context and an oracle configuration."""
 
-    def __init__(self, B, oracle, cfg, math="fp32", batches=None, bias_scale=0.1, lr=1e-3, partition=None):
+    def __init__(self, B, oracle, cfg, math="fp32", batches=None, bias_scale=0.1, lr=1e-3, partition=None, model="tgn"):
         from paper_2608_16305_b200 import trainer
         self.B, self.oracle, self.cfg, self.math = B, oracle, cfg, math
         self.stream = wl.make_stream(cfg)
@@ -70,15 +70,16 @@ class Rig:
             self.dw = trainer.DeviceWorkload(self.stream, batches=batches, efeat=efeat_dev)
         else:   # (owner, P, p, K): worker p's mixed batches from the backward dependency scan
             self.dw = trainer.PartitionedWorkload(self.stream, *partition, efeat=efeat_dev)
-        self.weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed, bias_scale=bias_scale)
+        self.model = model
+        self.weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed, bias_scale=bias_scale, model=model)
         mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST}[math]
-        self.tr = trainer.Trainer(self.dw, self.weights, math_mode=mode, lr=lr)
+        self.tr = trainer.Trainer(self.dw, self.weights, math_mode=mode, lr=lr, model=model)
         f32 = lambda x: float(np.float32(x))      # the library's configuration holds fp32 hyper-parameters
         self.ocfg = orc_cfg(oracle, cfg, lr=f32(lr), beta1=f32(0.9), beta2=f32(0.999), eps=f32(1e-8))
         self.graph = (self.stream.indptr, self.stream.nbr, self.stream.eid, self.stream.ts)
         self.efeat = self.stream.efeat() if (cfg.d_e and not self.compact) else None
         self.lay = B.param_layout(self.tr.tcfg)
-        self.shapes = wl.param_shapes(cfg.d, cfg.d_e)
+        self.shapes = wl.param_shapes(cfg.d, cfg.d_e, model)
         key = math + ("_bf16" if cfg.feat_dtype == "bf16" and math != "fp32" else "")
         self.tol = TOL[key]
 
@@ -115,6 +116,16 @@ class Rig:
         t_src, t_dst, t_neg, t_t = self.dw.targets_host(b)
         nodes = np.concatenate([t_src, t_dst, t_neg])
         times = np.concatenate([t_t] * 3)
+        if self.model == "jodie":
+            from oracle import jodie as oj
+            upd = self.upd_host(b)
+            if upd is None:
+                z = np.zeros(0, np.int32)
+                upd = (z, z, np.zeros(0), z, None)
+            hint = {} if gates is None else dict(hid_gate=gates[1], gate_eps=GATE_EPS[self.math])
+            res = oj.step(self.ocfg, pre["params"], pre["memory"], pre["last_update"], self.efeat, upd,
+                          (t_src, t_dst, t_neg, t_t), None, **hint)
+            return res, (nodes, times)
         nb = o.sample_recent(*self.graph, nodes, times, self.cfg.k)
         upd = self.upd_host(b)
         if upd is None:
@@ -159,7 +170,7 @@ class Rig:
         # logit gradients of a root sum to zero); what both sides hold is rounding residue.  Such a
         # tensor is measured on the scale of the gradient as a whole: floor = 1e-3 x largest entry.
         floor = 1e-3 * np.abs(res.grads).max()
-        for name in self.B.PARAM_NAMES:
+        for name in self.B.param_names(self.tr.tcfg):
             sl = slice(self.lay[name], self.lay[name] + int(np.prod(self.shapes[name])))
             e = float(np.abs(g[sl] - res.grads[sl]).max() / max(np.abs(res.grads[sl]).max(), floor, 1e-6))
             assert e <= tol, f"{what} grad {name} err {e}"
@@ -493,6 +504,43 @@ def test_partitioned_worker_steps_on_scanned_mixed_batches(B, oracle, p):
         assert np.all(np.diff(mb.t) >= 0)                                        # timestamp order (Eq. 5)
     assert sum(int(m.is_aux.sum()) for m in dw.mb_host) > 0
     _run_epoch_checks(rig, range(cfg.num_batches), {1, 4, 7, cfg.num_batches - 1})
+
+
+@pytest.mark.parametrize("math", ["fp32", "tf32"])
+@pytest.mark.parametrize("name,events,at", [
+    ("tiny", 4000, {0, 1, 2, 7, 19}),
+    ("wiki", 6000, {1, 5, 9}),
+    ("reddit", 9000, {2, 8, 14}),       # replay events + pruning
+    ("lastfm", 24000, {1, 3, 5}),       # no edge features, batch 4000
+])
+def test_jodie_variant_teacher_forced(B, oracle, name, events, at, math):
+    """The paper's second model: recurrent-cell memory update and time-projected embedding, same head, loss and Adam."""
+    from oracle import jodie as oj
+    rig = Rig(B, oracle, _scaled(name, events), math=math, model="jodie")
+    lay = oj.param_layout(rig.cfg.d, rig.cfg.d_e)
+    assert all(rig.lay[n] == lay[n] for n in oj.PARAM_NAMES) and rig.lay["total"] == lay["total"]
+    _run_epoch_checks(rig, range(rig.cfg.num_batches), at)
+    assert rig.tr.lib.kernel_launches() > 0
+
+
+def test_jodie_by_parts_and_wide_model(B, oracle):
+    """Entry point by entry point (no whole-step call), a model too wide for the fused head, and the embedding alone."""
+    from oracle import jodie as oj
+    c = wl.scaled(wl.CONFIGS["wiki"], num_events=1200, num_nodes=1200, num_src=1000, d=160, batch=300)
+    rig = Rig(B, oracle, c, math="tf32", model="jodie")
+    _run_epoch_checks(rig, range(4), {1, 3})
+    # the embedding entry point with the neighbor arrays left out
+    tr, s = rig.tr, rig.stream
+    nodes = dev(np.concatenate([s.src[:50], s.dst[:50]]), torch.int32)
+    times = dev(np.full(100, s.t[-1] + 3.5), torch.float64)
+    h = torch.zeros((100, c.d), dtype=torch.float32, device="cuda")
+    tr.lib.embed(nodes, times, None, None, None, None, h)
+    torch.cuda.synchronize()
+    W = oj.unpack(c.d, c.d_e, tr.params.cpu().numpy().astype(np.float64))
+    mem, lu = tr.memory.cpu().numpy().astype(np.float64), tr.last_update.cpu().numpy()
+    n = nodes.cpu().numpy()
+    dt = (times.cpu().numpy() - lu[n]).astype(np.float32).astype(np.float64)
+    assert relerr(h.cpu().numpy(), oj.time_projection(mem[n], dt, W["proj_w"], W["proj_b"])) <= 1e-6
 
 
 def test_host_buffer_entry_point_matches_device_path(B, oracle):
