@@ -155,7 +155,7 @@ class Trainer:
         # The library replays a step as a CUDA graph, which it records by stream capture; the legacy
         # default stream cannot capture, so when the caller is on it the step runs on this stream,
         # ordered after / before the caller's stream with events.
-        self.stream = torch.cuda.Stream(device=dev)
+        self.stream = torch.cuda.Stream(device=dev, priority=-1)
         # The prune mask of batch b is consumed only when b is replayed as the update batch of step b+1,
         # so it runs on a stream of its own beside step b and is waited for at the start of step b+1.
         self.prune_stream = torch.cuda.Stream(device=dev)
