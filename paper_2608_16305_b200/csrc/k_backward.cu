@@ -686,7 +686,9 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       const int groups = (n_q + HF_EV - 1) / HF_EV;
       {
         KernelScope scope__(ctx, "head_fused", s);
-        head_fused_kernel<<<groups < 296 ? groups : 296, HF_THREADS, hf_smem, s>>>(
+        // one block per SM (148) walking its groups, or two per SM when there are groups for all of them: a grid
+        // a little above the SM count would leave a few SMs with two blocks and everyone waiting for those
+        head_fused_kernel<<<groups <= 148 ? groups : (groups < 296 ? 148 : 296), HF_THREADS, hf_smem, s>>>(
             ctx->e_h, P + L.w1, P + L.b1, P + L.w2, P + L.b2, loss_mask, n_q, d, w.cat1, w.hid1, w.hid_gate, w.dpre_o,
             G + L.w2, G + L.b2, w.st_scalars, relu_out);
       }
