@@ -390,11 +390,12 @@ __global__ void __launch_bounds__(256) scatter_dmem_kernel(const float* __restri
 // meet in shared memory and leave as one pair of fp64 atomics per block and column into acc[0:d]
 // (dw) and acc[d:2d] (db).  Dynamic shared memory: 8 * 2 * d doubles.
 constexpr int TG_MAXJ = 8;
-// rows per block: 64 for long inputs, fewer (down to one per warp) when that is needed to fill the machine
+// Rows per block: every block ends with one fp64 atomic per column onto the same 2d addresses, and those
+// serialise, so the grid is kept to about one block per SM (rows per block a multiple of the 8 warps);
+// inside a block each warp walks its rows four at a time so that their loads overlap.
 inline int tg_rows_per_block(int rows) {
-  int r = 64;
-  while (r > 8 && (rows + r - 1) / r < 296) r >>= 1;
-  return r;
+  const int r = (rows + 147) / 148;
+  return r < 8 ? 8 : (r + 7) / 8 * 8;
 }
 __global__ void __launch_bounds__(256) time_grad_kernel(const float* __restrict__ G, int64_t ldg, int col0,
                                                         const float* __restrict__ S, const float* __restrict__ dt,
@@ -414,16 +415,27 @@ __global__ void __launch_bounds__(256) time_grad_kernel(const float* __restrict_
     const int c = lane + 32 * j;
     sb[j] = (S == nullptr && c < d) ? sinf(time_b[c]) : 0.f;
   }
-  for (int r = r0 + wid; r < r1; r += 8) {
-    const float dtr = dt ? dt[r] : 0.f;
+  for (int rb = r0 + wid; rb < r1; rb += 32) {  // rows rb, rb + 8, rb + 16, rb + 24: loads first, sums after
+    float g[4][TG_MAXJ], sn[4][TG_MAXJ], dtr[4];
 #pragma unroll
-    for (int j = 0; j < TG_MAXJ; ++j) {
-      const int c = lane + 32 * j;
-      if (c < d) {
-        const float g = G[(int64_t)r * ldg + col0 + c];
-        const float sn = S ? S[(int64_t)r * d + c] : sb[j];
-        const double t = -(double)sn * (double)g;
-        gw[j] = fma(t, (double)dtr, gw[j]);
+    for (int u = 0; u < 4; ++u) {
+      const int r = rb + 8 * u;
+      const bool in = r < r1;
+      dtr[u] = (in && dt) ? dt[r] : 0.f;
+#pragma unroll
+      for (int j = 0; j < TG_MAXJ; ++j) {
+        const int c = lane + 32 * j;
+        const bool ok = in && c < d;
+        g[u][j] = ok ? G[(int64_t)r * ldg + col0 + c] : 0.f;
+        sn[u][j] = ok ? (S ? S[(int64_t)r * d + c] : sb[j]) : 0.f;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+#pragma unroll
+      for (int j = 0; j < TG_MAXJ; ++j) {
+        const double t = -(double)sn[u][j] * (double)g[u][j];
+        gw[j] = fma(t, (double)dtr[u], gw[j]);
         gb[j] += t;
       }
     }
@@ -730,7 +742,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       const size_t tg_smem = (size_t)8 * 2 * d * sizeof(double);
       {
         KernelScope scope__(ctx, "jodie_embed_bwd", s);
-        jodie_embed_bwd_kernel<<<(R + 7) / 8 < 592 ? (R + 7) / 8 : 592, 256, tg_smem, s>>>(
+        jodie_embed_bwd_kernel<<<(R + 7) / 8 < 148 ? (R + 7) / 8 : 148, 256, tg_smem, s>>>(
             w.dpre_o, ctx->memory, ctx->last_update, P + L.proj_w, P + L.proj_b, ctx->e_nodes, ctx->e_times, R, d,
             w.node2slot, ctx->have_update ? 1 : 0, w.dMemU, w.tg_acc + 2 * d);
       }
