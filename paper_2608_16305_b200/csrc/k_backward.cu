@@ -566,23 +566,55 @@ __global__ void __launch_bounds__(256) gradnorm_adam_kernel(float* __restrict__ 
   // 1 - beta formed in fp64 from the configured fp32 value, then rounded once
   const float omb1 = (float)(1.0 - (double)beta1), omb2 = (float)(1.0 - (double)beta2);
   double acc = 0.0;
-  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < P; e += (int64_t)gridDim.x * blockDim.x) {
+  // one parameter: gradient (from the fp64 sums where those exist), sum of squares, Adam
+  auto one = [&](int64_t e, float ge, float& pe, float& me, float& ve) {
+    acc = fma((double)ge, (double)ge, acc);
+    me = fmaf(beta1, me, omb1 * ge);
+    ve = fmaf(beta2, ve, omb2 * ge * ge);
+    pe -= lr * (me * c1) / (sqrtf(ve * c2) + eps);
+  };
+  // groups of four consecutive parameters with 128-bit accesses (the arrays are 16-byte aligned; the ranges
+  // taken from the fp64 sums start and end on multiples of four because d is one), then the last P % 4
+  const bool vec = ((((uintptr_t)grads | (uintptr_t)p | (uintptr_t)m | (uintptr_t)v) & 15) == 0) && (t_off % 4 == 0) &&
+                   (t_n % 4 == 0) && (p_off % 4 == 0) && (p_n % 4 == 0);
+  const int64_t P4 = vec ? P / 4 : 0;
+  for (int64_t q = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; q < P4; q += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t e = 4 * q;
+    float4 g4;
+    if (e >= t_off && e < t_off + t_n) {
+      const double* a = tg_acc + (e - t_off);
+      g4 = make_float4((float)a[0], (float)a[1], (float)a[2], (float)a[3]);
+      reinterpret_cast<float4*>(grads)[q] = g4;
+    } else if (e >= p_off && e < p_off + p_n) {  // the projection's w_p | b_p, summed in fp64 behind the time encoder's
+      const double* a = tg_acc + t_n + (e - p_off);
+      g4 = make_float4((float)a[0], (float)a[1], (float)a[2], (float)a[3]);
+      reinterpret_cast<float4*>(grads)[q] = g4;
+    } else {
+      g4 = reinterpret_cast<const float4*>(grads)[q];
+    }
+    float4 p4 = reinterpret_cast<float4*>(p)[q], m4 = reinterpret_cast<float4*>(m)[q], v4 = reinterpret_cast<float4*>(v)[q];
+    one(e, g4.x, p4.x, m4.x, v4.x);
+    one(e + 1, g4.y, p4.y, m4.y, v4.y);
+    one(e + 2, g4.z, p4.z, m4.z, v4.z);
+    one(e + 3, g4.w, p4.w, m4.w, v4.w);
+    reinterpret_cast<float4*>(p)[q] = p4;
+    reinterpret_cast<float4*>(m)[q] = m4;
+    reinterpret_cast<float4*>(v)[q] = v4;
+  }
+  for (int64_t e = 4 * P4 + blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < P; e += (int64_t)gridDim.x * blockDim.x) {
     float ge;
     if (e >= t_off && e < t_off + t_n) {
       ge = (float)tg_acc[e - t_off];
       grads[e] = ge;
-    } else if (e >= p_off && e < p_off + p_n) {  // the projection's w_p | b_p, summed in fp64 behind the time encoder's
+    } else if (e >= p_off && e < p_off + p_n) {
       ge = (float)tg_acc[t_n + (e - p_off)];
       grads[e] = ge;
     } else {
       ge = grads[e];
     }
-    acc = fma((double)ge, (double)ge, acc);
-    const float me = fmaf(beta1, m[e], omb1 * ge);
-    const float ve = fmaf(beta2, v[e], omb2 * ge * ge);
-    m[e] = me;
-    v[e] = ve;
-    p[e] -= lr * (me * c1) / (sqrtf(ve * c2) + eps);
+    float pe = p[e], me = m[e], ve = v[e];
+    one(e, ge, pe, me, ve);
+    p[e] = pe; m[e] = me; v[e] = ve;
   }
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(FULL, acc, o);
   if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = acc;
