@@ -151,22 +151,32 @@ struct StageArgs {
   uint8_t *d_u_keep, *d_mask;
   int n_u, n_q;
 };
+// All loads are issued before the first store (the pointers may alias as far as the compiler knows, so
+// written one array after the other every load would wait for the store before it).
 __global__ void __launch_bounds__(256) stage_inputs_kernel(StageArgs a) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < a.n_u) {
-    if (a.u_src != a.d_u_src) a.d_u_src[i] = a.u_src[i];
-    if (a.u_dst != a.d_u_dst) a.d_u_dst[i] = a.u_dst[i];
-    if (a.u_eid != a.d_u_eid) a.d_u_eid[i] = a.u_eid[i];
-    if (a.u_t != a.d_u_t) a.d_u_t[i] = a.u_t[i];
-    if (a.u_keep && a.u_keep != a.d_u_keep) a.d_u_keep[i] = a.u_keep[i];
-  }
-  if (i < a.n_q) {
-    if (a.q_src != a.d_q_src) a.d_q_src[i] = a.q_src[i];
-    if (a.q_dst != a.d_q_dst) a.d_q_dst[i] = a.q_dst[i];
-    if (a.q_neg != a.d_q_neg) a.d_q_neg[i] = a.q_neg[i];
-    if (a.q_t != a.d_q_t) a.d_q_t[i] = a.q_t[i];
-    if (a.mask && a.mask != a.d_mask) a.d_mask[i] = a.mask[i];
-  }
+  const bool u = i < a.n_u, q = i < a.n_q;
+  // an array that is already in place is not copied
+  const bool c0 = u && a.u_src != a.d_u_src, c1 = u && a.u_dst != a.d_u_dst, c2 = u && a.u_eid != a.d_u_eid;
+  const bool c3 = u && a.u_t != a.d_u_t, c4 = u && a.u_keep && a.u_keep != a.d_u_keep;
+  const bool e0 = q && a.q_src != a.d_q_src, e1 = q && a.q_dst != a.d_q_dst, e2 = q && a.q_neg != a.d_q_neg;
+  const bool e3 = q && a.q_t != a.d_q_t, e4 = q && a.mask && a.mask != a.d_mask;
+  const int32_t s0 = c0 ? a.u_src[i] : 0, s1 = c1 ? a.u_dst[i] : 0, s2 = c2 ? a.u_eid[i] : 0;
+  const double s3 = c3 ? a.u_t[i] : 0.0;
+  const uint8_t s4 = c4 ? a.u_keep[i] : 0;
+  const int32_t t0 = e0 ? a.q_src[i] : 0, t1 = e1 ? a.q_dst[i] : 0, t2 = e2 ? a.q_neg[i] : 0;
+  const double t3 = e3 ? a.q_t[i] : 0.0;
+  const uint8_t t4 = e4 ? a.mask[i] : 0;
+  if (c0) a.d_u_src[i] = s0;
+  if (c1) a.d_u_dst[i] = s1;
+  if (c2) a.d_u_eid[i] = s2;
+  if (c3) a.d_u_t[i] = s3;
+  if (c4) a.d_u_keep[i] = s4;
+  if (e0) a.d_q_src[i] = t0;
+  if (e1) a.d_q_dst[i] = t1;
+  if (e2) a.d_q_neg[i] = t2;
+  if (e3) a.d_q_t[i] = t3;
+  if (e4) a.d_mask[i] = t4;
 }
 
 // Packed host block of tgnn_step_mixed_host: [t f64 n][q_t f64 nq][src,dst,eid i32 n each]
