@@ -303,13 +303,13 @@ __global__ void __launch_bounds__(256) attention_bwd_kernel(const float* __restr
   const int dh = d / H;
   const int c = cnt[i];
   const float scale = rsqrtf((float)dh);
-  attn_stage(Ks, Vs, Qs, Q, KV, i, c, d, k, lane);
+  attn_stage_issue(Ks, Vs, Qs, Q, KV, i, c, d, k, lane);
   {
-    const float4* g4 = reinterpret_cast<const float4*>(dcat_o + (int64_t)i * 2 * d);
-    for (int e = lane; e < (d >> 2); e += 32) reinterpret_cast<float4*>(das)[e] = __ldg(g4 + e);
+    const float* g = dcat_o + (int64_t)i * 2 * d;
+    for (int e = lane; e < (d >> 2); e += 32) cp_async16(das + 4 * e, g + 4 * e);
     for (int p = lane; p < H * k; p += 32) al[p] = alpha[(int64_t)i * H * k + p];
   }
-  __syncwarp();
+  attn_stage_wait();
   for (int p = lane; p < H * k; p += 32) {
     const int h = p / k, s = p - h * k;
     float a = 0.f;

@@ -98,8 +98,8 @@ __global__ void __launch_bounds__(256) attention_fwd_kernel(const float* __restr
   const int dh = d / H;
   const int c = cnt[i];
   const float scale = rsqrtf((float)dh);
-  attn_stage(Ks, Vs, Qs, Q, KV, i, c, d, k, lane);
-  __syncwarp();
+  attn_stage_issue(Ks, Vs, Qs, Q, KV, i, c, d, k, lane);
+  attn_stage_wait();
   for (int p = lane; p < H * k; p += 32) {
     const int h = p / k, s = p - h * k;
     float a = 0.f;

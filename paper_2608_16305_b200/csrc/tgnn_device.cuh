@@ -57,19 +57,30 @@ inline int attn_warps_per_block(int d, int H, int k) {
 }
 inline size_t attn_smem_bytes(int d, int H, int k, int warps) { return (size_t)warps * attn_warp_floats(d, H, k) * 4; }
 
-// Stage the root's valid K | V rows and its query in shared memory with coalesced 128-bit loads.
-__device__ __forceinline__ void attn_stage(float* Ks, float* Vs, float* Qs, const float* __restrict__ Q,
-                                           const float* __restrict__ KV, int i, int c, int d, int k, int lane) {
+// Stage the root's valid K | V rows and its query in shared memory: asynchronous 16-byte copies, all
+// issued before the single wait, so the whole 8 KB of a root costs one round trip instead of one per
+// loop iteration.  Rows are 16-byte aligned (d is a multiple of 4).  Ends with the copies complete and
+// visible to the warp (attn_stage_wait; other loads of the caller can be put between issue and wait).
+__device__ __forceinline__ void cp_async16(float* smem_dst, const float* gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+__device__ __forceinline__ void attn_stage_issue(float* Ks, float* Vs, float* Qs, const float* __restrict__ Q,
+                                                 const float* __restrict__ KV, int i, int c, int d, int k, int lane) {
   const int d4 = d >> 2;
-  const float4* q4 = reinterpret_cast<const float4*>(Q + (int64_t)i * d);
-  for (int e = lane; e < d4; e += 32) reinterpret_cast<float4*>(Qs)[e] = __ldg(q4 + e);
-  const float4* kv4 = reinterpret_cast<const float4*>(KV + (int64_t)i * k * 2 * d);
+  const float* q = Q + (int64_t)i * d;
+  for (int e = lane; e < d4; e += 32) cp_async16(Qs + 4 * e, q + 4 * e);
+  const float* kv = KV + (int64_t)i * k * 2 * d;
   for (int e = lane; e < c * 2 * d4; e += 32) {
     const int s = e / (2 * d4), r = e - s * 2 * d4;
-    const float4 v = __ldg(kv4 + e);
-    if (r < d4) reinterpret_cast<float4*>(Ks + s * d)[r] = v;
-    else reinterpret_cast<float4*>(Vs + s * d)[r - d4] = v;
+    cp_async16(r < d4 ? Ks + s * d + 4 * r : Vs + s * d + 4 * (r - d4), kv + 4 * e);
   }
+}
+__device__ __forceinline__ void attn_stage_wait() {
+  cp_async_wait_all();
+  __syncwarp();
 }
 
 }  // namespace tgnn
