@@ -364,20 +364,36 @@ __global__ void __launch_bounds__(256) scatter_dmem_kernel(const float* __restri
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   const int nb_rows = n * k;
+  const int d4 = d >> 2;  // <= 64: at most two 16-byte pieces per lane
   for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < nb_rows + n; r += warps) {
-    const int node = r < nb_rows ? nbr[r] : nodes[r - nb_rows];
+    // the row's gradient is requested before it is known whether its node was updated (most were not):
+    // the index chain node -> slot and the row loads overlap
+    const bool isn = r < nb_rows;
+    const int i = r - nb_rows;
+    float4 g[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int q4 = lane + 32 * u;
+      g[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (q4 < d4) {
+        if (isn) {
+          g[u] = __ldg(reinterpret_cast<const float4*>(dZm + (int64_t)r * 2 * d) + q4);  // memory half of the row
+        } else {
+          const float4 a = __ldg(reinterpret_cast<const float4*>(dcat_o + (int64_t)i * 2 * d + d) + q4);
+          const float4 b = __ldg(reinterpret_cast<const float4*>(dzq + (int64_t)i * 2 * d) + q4);
+          g[u] = make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+        }
+      }
+    }
+    const int node = isn ? nbr[r] : nodes[i];
     if (node < 0) continue;
     const int slot = node2slot[node];
     if (slot < 0) continue;
-    float* out = dMemU + (int64_t)slot * d;
-    if (r < nb_rows) {
-      const float* g = dZm + (int64_t)r * 2 * d;  // memory half of the [NB, 2d] gradient rows
-      for (int q = lane; q < d; q += 32) atomicAdd(&out[q], g[q]);
-    } else {
-      const int i = r - nb_rows;
-      const float* g1 = dcat_o + (int64_t)i * 2 * d + d;
-      const float* g2 = dzq + (int64_t)i * 2 * d;
-      for (int q = lane; q < d; q += 32) atomicAdd(&out[q], g1[q] + g2[q]);
+    float4* out = reinterpret_cast<float4*>(dMemU + (int64_t)slot * d);
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int q4 = lane + 32 * u;
+      if (q4 < d4) atomicAdd(out + q4, g[u]);
     }
   }
 }
