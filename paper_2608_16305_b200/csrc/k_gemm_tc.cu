@@ -24,6 +24,10 @@
 // contiguous), so the forward projections (activations [M,K] x weights [N,K]), the
 // input gradients (dY [M,N'] x W [N',K]) and the weight gradients (dY^T x A, contraction
 // over rows) all run here without a transposed copy.
+#include <cuda.h>
+
+#include <cstdlib>
+
 #include "tgnn_internal.cuh"
 
 namespace tgnn {
@@ -60,18 +64,26 @@ struct TcArgs {
   const int32_t* a_idx;
   const float* a_tab;
   int a_tab_cols;
+  // K-major A as a tiled tensor map (box 32 x 128, 128-byte swizzle): the tensor-memory-access unit brings
+  // whole activation tiles into shared memory; a_tma = 0: A goes through registers
+  int a_tma;
+  CUtensorMap a_map;
 };
 
-template <int BN_T, bool PRECISE>
+template <int BN_T, bool PRECISE, bool TMA = false>
 struct Cfg {
   static constexpr int STAGES = PRECISE ? (BN_T > 128 ? 2 : 3) : 4;
+  // A group's consecutive blocks must not be more than one use of a stage apart (the waits tell phases apart
+  // by parity only), so there are never more groups than stages.
   static constexpr int GROUPS = STAGES < 3 ? STAGES : 3;
+  static_assert(GROUPS <= STAGES, "a producer group may not lap a stage");
   static constexpr int THREADS = GROUPS * GROUP + 32;
   static constexpr int A_BYTES = BM * 128, B_BYTES = BN_T * 128;
   static constexpr int COPIES = PRECISE ? 2 : 1;  // head (+ tail) copy of each operand tile
   static constexpr int STAGE_BYTES = COPIES * (A_BYTES + B_BYTES);
   static constexpr int SMEM = 1024 + STAGES * STAGE_BYTES;
   static constexpr uint32_t TMEM_COLS = BN_T <= 128 ? 128 : 256;
+  static_assert(SMEM <= 227 * 1024, "shared memory budget");
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -271,13 +283,13 @@ __device__ __forceinline__ void mma_tf32(uint32_t tmem, uint64_t da, uint64_t db
 }
 
 // grid: (n tiles, m tiles, split_k).  Dynamic shared memory: Cfg::SMEM bytes.
-template <int BN_T, bool PRECISE, bool FAST>
-__global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kernel(TcArgs g) {
-  using C_ = Cfg<BN_T, PRECISE>;
+template <int BN_T, bool PRECISE, bool FAST, bool TMA>
+__global__ void __launch_bounds__(Cfg<BN_T, PRECISE, TMA>::THREADS, 1) gemm_tf32_kernel(const __grid_constant__ TcArgs g) {
+  using C_ = Cfg<BN_T, PRECISE, TMA>;
   constexpr int STAGES = C_::STAGES, GROUPS = C_::GROUPS, THREADS = C_::THREADS;
   constexpr int MMA_WARP = GROUPS * 4;
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) uint64_t s_full[STAGES], s_empty[STAGES], s_accum;
+  __shared__ __align__(8) uint64_t s_full[STAGES], s_empty[STAGES], s_accum, s_raw[STAGES];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
   __shared__ float s_rowsum[BM];
@@ -321,6 +333,7 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kern
       mbar_init(smem_u32(&s_empty[s]), 1);
     }
     mbar_init(smem_u32(&s_accum), 1);
+    for (int r = 0; r < STAGES; ++r) mbar_init(smem_u32(&s_raw[r]), 1);
     s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -359,6 +372,68 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kern
       trp = tab_row;
     }
     uint32_t ma = 0, mn = 0;
+    // The B tile of block i into stage s: one bulk asynchronous copy of the prepared image (head and tail);
+    // it signals full[s] itself.
+    auto b_image_copy = [&](int i, int s, uint32_t b_tile) {
+      constexpr uint32_t bytes = C_::COPIES * C_::B_BYTES;
+      const unsigned char* src = g.b_image + blockIdx.x * g.b_tile_stride + (int64_t)(kb0 + i) * bytes;
+      const uint32_t bar = smem_u32(&s_full[s]);
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(b_tile), "l"(src), "r"(bytes), "r"(bar)
+                   : "memory");
+    };
+    if constexpr (TMA) {
+      // A arrives as whole tiles: once the stage is free, one thread of the group asks the tensor-memory-access
+      // unit for block i (box 32 x 128 at column k, row m0; rows and columns outside the matrix come back as
+      // zeros) straight into the stage's head tile, already in its 128-byte-swizzled layout.  When the tile
+      // has landed every thread rounds its own chunks in place and writes their tails -- shared memory to
+      // shared memory, no thread touches another's chunk.  Blocks that overlap the row-indirect columns still
+      // go through registers from global memory.
+      auto by_tma = [&](int i) { return !(g.a_idx != nullptr && (kb0 + i) * BK < g.a_tab_cols); };
+      for (int i = grp; i < nkb; i += GROUPS) {
+        const int s = i % STAGES;
+        const bool tile = by_tma(i);
+        if (!tile)
+          ma = load_regs<BM, FAST>(va, g.A, g.lda, g.a_major, m0, M, BM, (kb0 + i) * BK, k_end, a_vec, t, trp, g.a_tab,
+                                   g.a_tab_cols);
+        if (i >= STAGES) {
+          ok = mbar_wait(smem_u32(&s_empty[s]), ((i / STAGES) - 1) & 1);
+          if (!ok) break;
+        }
+        const uint32_t a_tile = smem_base + s * C_::STAGE_BYTES;
+        const uint32_t b_tile = a_tile + C_::COPIES * C_::A_BYTES;
+        const uint32_t raw_bar = smem_u32(&s_raw[s]);
+        if (t == 0) {
+          if (tile) {
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(raw_bar), "r"((uint32_t)C_::A_BYTES)
+                         : "memory");
+            asm volatile(
+                "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                ::"r"(a_tile), "l"(&g.a_map), "r"((kb0 + i) * BK), "r"(m0), "r"(raw_bar)
+                : "memory");
+          }
+          b_image_copy(i, s, b_tile);
+        }
+        if (tile) {
+          int before = 0;  // tile blocks that used this stage (and its tile barrier) before block i: the phase
+          for (int j = s; j < i; j += STAGES) before += by_tma(j) ? 1 : 0;
+          ok = mbar_wait(raw_bar, before & 1);
+          if (!ok) break;
+#pragma unroll
+          for (int q = 0; q < BM * 8 / GROUP; ++q) {
+            const int idx = t + q * GROUP, r = idx >> 3, c = idx & 7;
+            const uint32_t addr = a_tile + r * 128 + ((c ^ (r & 7)) << 4);
+            asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
+                         : "=f"(va[q].x), "=f"(va[q].y), "=f"(va[q].z), "=f"(va[q].w) : "r"(addr) : "memory");
+          }
+          ma = 0xffffffffu;
+        }
+        store_regs<BM, PRECISE>(va, ma, a_tile, C_::A_BYTES, MAJOR_K, BM, t, nullptr);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(smem_u32(&s_full[s]));
+      }
+    } else {
     if (grp < nkb)
       ma = load_regs<BM, FAST>(va, g.A, g.lda, g.a_major, m0, M, BM, (kb0 + grp) * BK, k_end, a_vec, t, trp, g.a_tab,
                                g.a_tab_cols);
@@ -374,17 +449,7 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kern
       const uint32_t a_tile = smem_base + s * C_::STAGE_BYTES;
       const uint32_t b_tile = a_tile + C_::COPIES * C_::A_BYTES;
       const int k0 = (kb0 + i) * BK;
-      if (g.b_image != nullptr) {
-        if (t == 0) {  // one bulk asynchronous copy brings the whole B tile (head and tail); it signals full[s] itself
-          constexpr uint32_t bytes = C_::COPIES * C_::B_BYTES;
-          const unsigned char* src = g.b_image + blockIdx.x * g.b_tile_stride + (int64_t)(kb0 + i) * bytes;
-          const uint32_t bar = smem_u32(&s_full[s]);
-          asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-          asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                       ::"r"(b_tile), "l"(src), "r"(bytes), "r"(bar)
-                       : "memory");
-        }
-      }
+      if (g.b_image != nullptr && t == 0) b_image_copy(i, s, b_tile);
       store_regs<BM, PRECISE>(va, ma, a_tile, C_::A_BYTES, g.a_major, BM, t, want_rowsum ? &rs : nullptr);
       if (g.b_image == nullptr)
         load_tile<BN_T, PRECISE, FAST>(b_tile, C_::B_BYTES, g.B, g.ldb, g.b_major, n0, g.N, b_rows, k0, k_end, b_vec, t, nullptr);
@@ -393,6 +458,7 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE>::THREADS, 1) gemm_tf32_kern
 #pragma unroll
       for (int q = 0; q < BM * 8 / GROUP; ++q) va[q] = vn[q];
       ma = mn;
+    }
     }
     if (!ok) { s_abort = 1; atomicCAS(g.status, 0, TGNN_ETIMEOUT); }
     if (want_rowsum) {  // the thread's chunks cover rows 4*(t%32) .. +3 of the tile
@@ -597,22 +663,50 @@ __global__ void __launch_bounds__(256) prep_weights_kernel(const WeightSite* __r
                    to_tf32(v[2] - __uint_as_float(h2)), to_tf32(v[3] - __uint_as_float(h3)));
 }
 
-template <int BN_T, bool PRECISE, bool FAST>
+template <int BN_T, bool PRECISE, bool FAST, bool TMA>
 int launch_tc(tgnn_ctx* ctx, const TcArgs& a, int n_tiles, const char* name, cudaStream_t s) {
-  using C_ = Cfg<BN_T, PRECISE>;
+  using C_ = Cfg<BN_T, PRECISE, TMA>;
   static bool attr_set = false;
   if (!attr_set) {
-    TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(gemm_tf32_kernel<BN_T, PRECISE, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           C_::SMEM));
+    TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(gemm_tf32_kernel<BN_T, PRECISE, FAST, TMA>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM));
     attr_set = true;
   }
   dim3 grid(n_tiles, (a.M + BM - 1) / BM, a.split_k);
   {
     KernelScope scope__(ctx, name, s);
-    gemm_tf32_kernel<BN_T, PRECISE, FAST><<<grid, C_::THREADS, C_::SMEM, s>>>(a);
+    gemm_tf32_kernel<BN_T, PRECISE, FAST, TMA><<<grid, C_::THREADS, C_::SMEM, s>>>(a);
   }
   TGNN_LAUNCH_OK(ctx, name);
   return TGNN_OK;
+}
+
+// Tiled tensor map of a row-major fp32 matrix [rows, cols] (row pitch ld floats): boxes of 32 columns x 128
+// rows, 128-byte swizzle, zeros outside.  The driver's encoder is looked up once through the runtime (no link
+// against the driver library).  Returns false if it is unavailable or refuses the shape.
+bool encode_a_map(CUtensorMap* map, const float* base, int64_t rows, int64_t cols, int64_t ld) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn enc = nullptr;
+  static bool looked = false;
+  if (!looked) {
+    looked = true;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      enc = reinterpret_cast<EncodeFn>(fn);
+    (void)cudaGetLastError();
+  }
+  if (!enc || rows <= 0 || cols <= 0) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
+  const cuuint32_t box[2] = {BK, BM};
+  const cuuint32_t elem[2] = {1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, elem,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace
@@ -662,16 +756,27 @@ int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStr
   };
   const bool fast = whole(a.A, a.lda, a.a_major, a.K, a.dev_K, a.M, a.dev_M) &&
                     (a.b_image != nullptr || whole(a.B, a.ldb, a.b_major, a.K, a.dev_K, a.N, nullptr));
+  // activations as TMA tiles: K-major whole-chunk A beside a prepared weight image
+  static const bool tma_off = getenv("TGNN_NO_TMA") != nullptr;  // debugging aid: activations through registers
+  if (!tma_off && fast && a.a_major == MAJOR_K && a.b_image != nullptr && encode_a_map(&a.a_map, a.A, a.M, a.K, a.lda)) {
+    a.a_tma = 1;
+    if (precise) {
+      if (bn <= 128) return launch_tc<128, true, true, true>(ctx, a, n_tiles, name, s);
+      return launch_tc<256, true, true, true>(ctx, a, n_tiles, name, s);
+    }
+    if (bn <= 128) return launch_tc<128, false, true, true>(ctx, a, n_tiles, name, s);
+    return launch_tc<256, false, true, true>(ctx, a, n_tiles, name, s);
+  }
   const int sel = (precise ? 4 : 0) | (bn <= 128 ? 0 : 2) | (fast ? 1 : 0);
   switch (sel) {
-    case 0: return launch_tc<128, false, false>(ctx, a, n_tiles, name, s);
-    case 1: return launch_tc<128, false, true>(ctx, a, n_tiles, name, s);
-    case 2: return launch_tc<256, false, false>(ctx, a, n_tiles, name, s);
-    case 3: return launch_tc<256, false, true>(ctx, a, n_tiles, name, s);
-    case 4: return launch_tc<128, true, false>(ctx, a, n_tiles, name, s);
-    case 5: return launch_tc<128, true, true>(ctx, a, n_tiles, name, s);
-    case 6: return launch_tc<256, true, false>(ctx, a, n_tiles, name, s);
-    default: return launch_tc<256, true, true>(ctx, a, n_tiles, name, s);
+    case 0: return launch_tc<128, false, false, false>(ctx, a, n_tiles, name, s);
+    case 1: return launch_tc<128, false, true, false>(ctx, a, n_tiles, name, s);
+    case 2: return launch_tc<256, false, false, false>(ctx, a, n_tiles, name, s);
+    case 3: return launch_tc<256, false, true, false>(ctx, a, n_tiles, name, s);
+    case 4: return launch_tc<128, true, false, false>(ctx, a, n_tiles, name, s);
+    case 5: return launch_tc<128, true, true, false>(ctx, a, n_tiles, name, s);
+    case 6: return launch_tc<256, true, false, false>(ctx, a, n_tiles, name, s);
+    default: return launch_tc<256, true, true, false>(ctx, a, n_tiles, name, s);
   }
 }
 
