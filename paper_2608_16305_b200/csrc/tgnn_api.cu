@@ -423,6 +423,16 @@ int step_body(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q, bool has_mask, flo
   Workspace& w = ctx->ws;
   int rc;
   ctx->have_update = false;
+  // While per-kernel timing is on, everything is issued on the caller's stream: the event pair around a
+  // launch then times that kernel alone instead of the kernel plus whatever shares the machine with it.
+  struct SideGuard {
+    tgnn_ctx* c;
+    cudaStream_t s0, s1;
+    SideGuard(tgnn_ctx* c_, cudaStream_t main) : c(c_), s0(c_->side[0]), s1(c_->side[1]) {
+      if (c->prof.on) c->side[0] = c->side[1] = main;
+    }
+    ~SideGuard() { c->side[0] = s0; c->side[1] = s1; }
+  } side_guard(ctx, S(stream));
   // the weights' B-operand images for this step's projections: written beside the first kernels
   const bool prep = ctx->images != nullptr;
   if (prep) {
