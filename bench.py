@@ -285,7 +285,7 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
     achieved = flops / dur_s / 1e12 if dur_s > 0 else 0.0
     # dram__bytes_read.sum + dram__bytes_write.sum of one key/value-projection launch on this workload
     # (ncu --set full, summarised in profiles/gemm_tf32_kv_proj_wiki.md; tensor-core mode only)
-    traffic = 28.6e6 + 0.08e6 if (args.math == "tf32" and cfg.name == WORKLOAD and not jodie) else None
+    traffic = 22.0e6 + 0.002e6 if (args.math == "tf32" and cfg.name == WORKLOAD and not jodie) else None
     by, f_fwd, f_bwd = (algorithmic_work_jodie if jodie else algorithmic_work)(cfg, cfg.max_mixed, n_q, U_est)
     out = {
         "metric": METRIC, "value": units / (ms_dev_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,

@@ -68,9 +68,13 @@ struct TcArgs {
   // whole activation tiles into shared memory; a_tma = 0: A goes through registers
   int a_tma;
   CUtensorMap a_map;
+  // both operands MN-major (weight gradients): A and B as four-dimensional views of their row-major matrices
+  // whose boxes land in the operand tiles' atom layout (see encode_mn_map); b_box_atoms = 32-column atoms per B box
+  CUtensorMap b_map;
+  int b_box_atoms;
 };
 
-template <int BN_T, bool PRECISE, bool TMA = false>
+template <int BN_T, bool PRECISE, int TMA = 0>
 struct Cfg {
   static constexpr int STAGES = PRECISE ? (BN_T > 128 ? 2 : 3) : 4;
   // A group's consecutive blocks must not be more than one use of a stage apart (the waits tell phases apart
@@ -283,7 +287,7 @@ __device__ __forceinline__ void mma_tf32(uint32_t tmem, uint64_t da, uint64_t db
 }
 
 // grid: (n tiles, m tiles, split_k).  Dynamic shared memory: Cfg::SMEM bytes.
-template <int BN_T, bool PRECISE, bool FAST, bool TMA>
+template <int BN_T, bool PRECISE, bool FAST, int TMA>
 __global__ void __launch_bounds__(Cfg<BN_T, PRECISE, TMA>::THREADS, 1) gemm_tf32_kernel(const __grid_constant__ TcArgs g) {
   using C_ = Cfg<BN_T, PRECISE, TMA>;
   constexpr int STAGES = C_::STAGES, GROUPS = C_::GROUPS, THREADS = C_::THREADS;
@@ -304,7 +308,8 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE, TMA>::THREADS, 1) gemm_tf32
   const int n_valid = min(bn, g.N - n0);
   // MMA N: multiple of 16; MN-major B tiles are loaded in whole 32-column atoms
   const int n_mma = (n_valid + 15) / 16 * 16;
-  const int b_rows = g.b_major == MAJOR_MN ? (n_valid + 31) / 32 * 32 : (n_mma + 7) / 8 * 8;
+  const int b_rows = TMA == 2 ? g.b_box_atoms * 32  // the tile's layout is the box's, whatever part of it is valid
+                              : (g.b_major == MAJOR_MN ? (n_valid + 31) / 32 * 32 : (n_mma + 7) / 8 * 8);
   const int nkb_total = (K + BK - 1) / BK;
   const int per = (nkb_total + g.split_k - 1) / g.split_k;
   const int kb0 = blockIdx.z * per, kb1 = min(nkb_total, kb0 + per);
@@ -383,7 +388,62 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE, TMA>::THREADS, 1) gemm_tf32
                    ::"r"(b_tile), "l"(src), "r"(bytes), "r"(bar)
                    : "memory");
     };
-    if constexpr (TMA) {
+    if constexpr (TMA == 2) {
+      // Weight gradients: both operands are transposed views (contraction over rows).  One thread asks for the
+      // block's two boxes -- 32 contraction rows x 128 (A) or 32 x b_rows (B) values, delivered as atoms of
+      // 4 rows x 32 values with the 32-byte swizzle, i.e. in the operand tiles' own layout -- and when they have
+      // landed every thread rounds / splits its own chunks in place.  Values beyond the matrix edge inside the
+      // last atom are whatever follows in memory: they only reach rows / columns of C that are never stored.
+      const int b_atoms = b_rows >> 5, b_cpr = b_rows >> 2;
+      const uint32_t b_bytes = (uint32_t)b_rows * 128;
+      for (int i = grp; i < nkb; i += GROUPS) {
+        const int s = i % STAGES;
+        if (i >= STAGES) {
+          ok = mbar_wait(smem_u32(&s_empty[s]), ((i / STAGES) - 1) & 1);
+          if (!ok) break;
+        }
+        const uint32_t a_tile = smem_base + s * C_::STAGE_BYTES;
+        const uint32_t b_tile = a_tile + C_::COPIES * C_::A_BYTES;
+        const uint32_t raw_bar = smem_u32(&s_raw[s]);
+        if (t == 0) {
+          asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(raw_bar), "r"((uint32_t)C_::A_BYTES + b_bytes)
+                       : "memory");
+          asm volatile(
+              "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+              ::"r"(a_tile), "l"(&g.a_map), "r"(0), "r"(0), "r"(m0 >> 5), "r"((kb0 + i) * (BK / 4)), "r"(raw_bar)
+              : "memory");
+          asm volatile(
+              "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+              ::"r"(b_tile), "l"(&g.b_map), "r"(0), "r"(0), "r"(n0 >> 5), "r"((kb0 + i) * (BK / 4)), "r"(raw_bar)
+              : "memory");
+        }
+        ok = mbar_wait(raw_bar, (i / STAGES) & 1);
+        if (!ok) break;
+        // A: 32 rows x 128 values = 1024 chunks, 8 per thread; chunk (kk, cm) lives where store_regs would put it
+#pragma unroll
+        for (int q = 0; q < BM * 8 / GROUP; ++q) {
+          const int idx = t + q * GROUP;
+          const int kk = idx >> 5, cm = idx & 31;
+          const uint32_t addr = a_tile + (kk >> 2) * ((BM / 32) * 512) + (cm >> 3) * 512 + (kk & 3) * 128 +
+                                (((cm & 7) ^ ((kk & 3) << 1)) << 4);
+          float4 x;
+          asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w) : "r"(addr) : "memory");
+          store_chunk<PRECISE>(addr, C_::A_BYTES, x);
+          if (want_rowsum) { rs.x += x.x; rs.y += x.y; rs.z += x.z; rs.w += x.w; }  // cm == t % 32 for every q
+        }
+        // B: 32 rows x b_rows values
+        for (int idx = t; idx < BK * b_cpr; idx += GROUP) {
+          const int kk = idx / b_cpr, cm = idx - kk * b_cpr;
+          const uint32_t addr = b_tile + (kk >> 2) * (b_atoms * 512) + (cm >> 3) * 512 + (kk & 3) * 128 +
+                                (((cm & 7) ^ ((kk & 3) << 1)) << 4);
+          float4 x;
+          asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w) : "r"(addr) : "memory");
+          store_chunk<PRECISE>(addr, C_::B_BYTES, x);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(smem_u32(&s_full[s]));
+      }
+    } else if constexpr (TMA == 1) {
       // A arrives as whole tiles: once the stage is free, one thread of the group asks the tensor-memory-access
       // unit for block i (box 32 x 128 at column k, row m0; rows and columns outside the matrix come back as
       // zeros) straight into the stage's head tile, already in its 128-byte-swizzled layout.  When the tile
@@ -663,7 +723,7 @@ __global__ void __launch_bounds__(256) prep_weights_kernel(const WeightSite* __r
                    to_tf32(v[2] - __uint_as_float(h2)), to_tf32(v[3] - __uint_as_float(h3)));
 }
 
-template <int BN_T, bool PRECISE, bool FAST, bool TMA>
+template <int BN_T, bool PRECISE, bool FAST, int TMA>
 int launch_tc(tgnn_ctx* ctx, const TcArgs& a, int n_tiles, const char* name, cudaStream_t s) {
   using C_ = Cfg<BN_T, PRECISE, TMA>;
   static bool attr_set = false;
@@ -709,6 +769,38 @@ bool encode_a_map(CUtensorMap* map, const float* base, int64_t rows, int64_t col
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+}  // namespace
+
+namespace {
+// A row-major fp32 matrix [rows (contraction), cols] as the transposed operand of a product: a four-dimensional
+// view (value within a 32-wide atom, row within a group of 4, atom, group) whose box of 32 x 4 x atoms x 8 lands
+// in shared memory exactly as the MN-major operand tile is laid out: groups of 4 contraction rows, inside a group
+// one 512-byte atom per 32 columns, 32-byte swizzle.  rows must be a multiple of 4; the last atom of a row may run
+// past the row end (into the next row, or up to 124 bytes past the matrix).
+bool encode_mn_map(CUtensorMap* map, const float* base, int64_t rows, int64_t cols, int64_t ld, int box_atoms) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn enc = nullptr;
+  static bool looked = false;
+  if (!looked) {
+    looked = true;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      enc = reinterpret_cast<EncodeFn>(fn);
+    (void)cudaGetLastError();
+  }
+  if (!enc || rows <= 0 || cols <= 0 || rows % 4 != 0 || box_atoms < 1 || box_atoms > 8) return false;
+  const cuuint64_t dims[4] = {32, 4, (cuuint64_t)((cols + 31) / 32), (cuuint64_t)(rows / 4)};
+  const cuuint64_t strides[3] = {(cuuint64_t)ld * 4, 128, (cuuint64_t)ld * 16};
+  const cuuint32_t box[4] = {32, 4, (cuuint32_t)box_atoms, BK / 4};
+  const cuuint32_t elem[4] = {1, 1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(base), dims, strides, box, elem,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 }  // namespace
 
 // Returns TGNN_OK after launching, or 1 if the product does not fit this kernel (caller falls back to the FMA tiles).
@@ -761,22 +853,31 @@ int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStr
   if (!tma_off && fast && a.a_major == MAJOR_K && a.b_image != nullptr && encode_a_map(&a.a_map, a.A, a.M, a.K, a.lda)) {
     a.a_tma = 1;
     if (precise) {
-      if (bn <= 128) return launch_tc<128, true, true, true>(ctx, a, n_tiles, name, s);
-      return launch_tc<256, true, true, true>(ctx, a, n_tiles, name, s);
+      if (bn <= 128) return launch_tc<128, true, true, 1>(ctx, a, n_tiles, name, s);
+      return launch_tc<256, true, true, 1>(ctx, a, n_tiles, name, s);
     }
-    if (bn <= 128) return launch_tc<128, false, true, true>(ctx, a, n_tiles, name, s);
-    return launch_tc<256, false, true, true>(ctx, a, n_tiles, name, s);
+    if (bn <= 128) return launch_tc<128, false, true, 1>(ctx, a, n_tiles, name, s);
+    return launch_tc<256, false, true, 1>(ctx, a, n_tiles, name, s);
+  }
+  // weight gradients: both operands transposed, contraction length static and a multiple of 4
+  if (!tma_off && fast && precise && a.a_major == MAJOR_MN && a.b_major == MAJOR_MN && a.b_image == nullptr &&
+      a.dev_K == nullptr && a.K % 4 == 0 && bn % 32 == 0 &&
+      encode_mn_map(&a.a_map, a.A, a.K, a.M, a.lda, BM / 32) && encode_mn_map(&a.b_map, a.B, a.K, a.N, a.ldb, bn / 32)) {
+    a.a_tma = 2;
+    a.b_box_atoms = bn / 32;
+    if (bn <= 128) return launch_tc<128, true, true, 2>(ctx, a, n_tiles, name, s);
+    return launch_tc<256, true, true, 2>(ctx, a, n_tiles, name, s);
   }
   const int sel = (precise ? 4 : 0) | (bn <= 128 ? 0 : 2) | (fast ? 1 : 0);
   switch (sel) {
-    case 0: return launch_tc<128, false, false, false>(ctx, a, n_tiles, name, s);
-    case 1: return launch_tc<128, false, true, false>(ctx, a, n_tiles, name, s);
-    case 2: return launch_tc<256, false, false, false>(ctx, a, n_tiles, name, s);
-    case 3: return launch_tc<256, false, true, false>(ctx, a, n_tiles, name, s);
-    case 4: return launch_tc<128, true, false, false>(ctx, a, n_tiles, name, s);
-    case 5: return launch_tc<128, true, true, false>(ctx, a, n_tiles, name, s);
-    case 6: return launch_tc<256, true, false, false>(ctx, a, n_tiles, name, s);
-    default: return launch_tc<256, true, true, false>(ctx, a, n_tiles, name, s);
+    case 0: return launch_tc<128, false, false, 0>(ctx, a, n_tiles, name, s);
+    case 1: return launch_tc<128, false, true, 0>(ctx, a, n_tiles, name, s);
+    case 2: return launch_tc<256, false, false, 0>(ctx, a, n_tiles, name, s);
+    case 3: return launch_tc<256, false, true, 0>(ctx, a, n_tiles, name, s);
+    case 4: return launch_tc<128, true, false, 0>(ctx, a, n_tiles, name, s);
+    case 5: return launch_tc<128, true, true, 0>(ctx, a, n_tiles, name, s);
+    case 6: return launch_tc<256, true, false, 0>(ctx, a, n_tiles, name, s);
+    default: return launch_tc<256, true, true, 0>(ctx, a, n_tiles, name, s);
   }
 }
 

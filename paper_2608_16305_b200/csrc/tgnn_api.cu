@@ -151,7 +151,8 @@ size_t carve(tgnn_ctx* ctx, char* base) {
   cv.take_packed(w.red, 4);
   cv.take_packed(w.tg_acc, 4 * d);  // time encoder dw | db, time projection dw_p | db_p
   cv.take_packed(w.st_scalars, 4);
-  return (cv.off + 255) & ~(size_t)255;
+  // 256 bytes of slack: a tiled load of a transposed operand may run up to 124 bytes past the end of its matrix
+  return ((cv.off + 255) & ~(size_t)255) + 256;
 }
 
 inline cudaStream_t S(void* stream) { return reinterpret_cast<cudaStream_t>(stream); }
