@@ -678,6 +678,7 @@ int grad_w(tgnn_ctx* ctx, const float* dY, int64_t ld_dy, const float* A, int64_
   g.B = A; g.b_rs = ld_a; g.b_cs = 1;    // B(k,n) = A[k, n]
   g.C = dW; g.ldc = k_in; g.M = n_out; g.N = k_in; g.K = rows; g.dev_K = dev_rows;
   g.rowsum_out = db; g.accumulate = 1; g.split_k = pick_split(n_out, k_in, rows); g.precise = 1;
+  g.tail_slack = 1;  // dY and the saved activations are workspace buffers
   return launch_gemm(ctx, g, name, s);
 }
 

@@ -862,6 +862,7 @@ int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStr
   // weight gradients: both operands transposed, contraction length static and a multiple of 4
   if (!tma_off && fast && precise && a.a_major == MAJOR_MN && a.b_major == MAJOR_MN && a.b_image == nullptr &&
       a.dev_K == nullptr && a.K % 4 == 0 && bn % 32 == 0 &&
+      (g.tail_slack || ((a.M + 31) / 32 * 32 <= a.lda && (a.N + 31) / 32 * 32 <= a.ldb)) &&  // no read past a caller's matrix
       encode_mn_map(&a.a_map, a.A, a.K, a.M, a.lda, BM / 32) && encode_mn_map(&a.b_map, a.B, a.K, a.N, a.ldb, bn / 32)) {
     a.a_tma = 2;
     a.b_box_atoms = bn / 32;

@@ -315,6 +315,8 @@ struct GemmArgs {
   int a_tab_cols;
   int site;               // WeightSiteId + 1 when B is that weight matrix (0: none); lets the kernel use its image
   int precise;            // tensor-core mode only: 3xTF32 head/tail split, close to fp32 accuracy
+  int tail_slack;         // both operands live in the workspace arena: a tiled load may read up to 124 bytes past
+                          //   the end of a matrix whose width is not a multiple of 32 (the arena ends in slack)
 };
 int launch_gemm(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s);
 int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s);  // k_gemm_tc.cu

@@ -85,3 +85,31 @@ def test_projection_matches_definition(mode, shape):
             ref2 = A[:, :K - 37].astype(np.float64) @ Bm[:K - 37].astype(np.float64)
             assert np.abs(got - ref2).max() <= tol * scale
     lib.close()
+
+
+@pytest.mark.parametrize("M,N,K,pad", [
+    (192, 352, 4096, 0),     # widths are whole 32-column atoms
+    (200, 372, 5000, 28),    # ragged widths inside padded rows: the last atom of a row reads the padding
+    (100, 200, 1200, 24),    # one tile, split-K, several contraction blocks per CTA
+    (128, 256, 36, 0),       # contraction shorter than two blocks, a full 256-column tile
+])
+def test_transposed_products_by_tiles(M, N, K, pad):
+    """Weight-gradient shaped products (both operands transposed, contraction over rows) whose operands are
+    delivered by the tensor-memory-access unit: widths that are whole atoms, or rows padded far enough that the
+    last atom stays inside the matrix (the library does not read past a caller's buffer)."""
+    from paper_2608_16305_b200 import binding as B
+    rng = np.random.default_rng(M + 7 * N + 13 * K)
+    lib = B.Tgnn(B.make_config(100, 32, 16, 10, 2, math_mode=B.TGNN_MATH_TF32))
+    A, Bm, A_dev, sa, B_dev, sb = _operands(rng, M, N, K, "mn", "mn", pad=pad)
+    ref = A.astype(np.float64) @ Bm.astype(np.float64)
+    scale = np.abs(ref).max()
+    C0 = rng.normal(size=(M, N)).astype(np.float32)
+    for split in (1, 8):
+        C = torch.from_numpy(C0.copy()).cuda()
+        rs = torch.zeros(M, dtype=torch.float32, device="cuda")
+        lib.debug_gemm(A_dev, *sa, B_dev, *sb, C, N, M, N, K, rowsum_out=rs, accumulate=True, split_k=split, precise=True)
+        torch.cuda.synchronize()
+        assert lib.status() == 0
+        assert np.abs(C.cpu().numpy() - (ref + C0)).max() <= 1e-4 * scale
+        assert np.abs(rs.cpu().numpy() - A.astype(np.float64).sum(1)).max() <= 1e-4 * max(np.abs(A).sum(1).max(), 1.0)
+    lib.close()
