@@ -850,7 +850,10 @@ int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStr
                     (a.b_image != nullptr || whole(a.B, a.ldb, a.b_major, a.K, a.dev_K, a.N, nullptr));
   // activations as TMA tiles: K-major whole-chunk A beside a prepared weight image
   static const bool tma_off = getenv("TGNN_NO_TMA") != nullptr;  // debugging aid: activations through registers
-  if (!tma_off && fast && a.a_major == MAJOR_K && a.b_image != nullptr && encode_a_map(&a.a_map, a.A, a.M, a.K, a.lda)) {
+  // (tiles need 16-byte aligned rows only: a ragged contraction length is the tensor map's edge, filled with zeros)
+  const auto aligned = [](const float* p, int64_t ld) { return ((uintptr_t)p & 15) == 0 && ld % 4 == 0; };
+  if (!tma_off && aligned(a.A, a.lda) && a.dev_K == nullptr && a.a_major == MAJOR_K && a.b_image != nullptr &&
+      encode_a_map(&a.a_map, a.A, a.M, a.K, a.lda)) {
     a.a_tma = 1;
     if (precise) {
       if (bn <= 128) return launch_tc<128, true, true, 1>(ctx, a, n_tiles, name, s);
@@ -860,7 +863,8 @@ int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStr
     return launch_tc<256, false, true, 1>(ctx, a, n_tiles, name, s);
   }
   // weight gradients: both operands transposed, contraction length static and a multiple of 4
-  if (!tma_off && fast && precise && a.a_major == MAJOR_MN && a.b_major == MAJOR_MN && a.b_image == nullptr &&
+  if (!tma_off && aligned(a.A, a.lda) && aligned(a.B, a.ldb) && precise && a.a_major == MAJOR_MN && a.b_major == MAJOR_MN &&
+      a.b_image == nullptr &&
       a.dev_K == nullptr && a.K % 4 == 0 && bn % 32 == 0 &&
       (g.tail_slack || ((a.M + 31) / 32 * 32 <= a.lda && (a.N + 31) / 32 * 32 <= a.ldb)) &&  // no read past a caller's matrix
       encode_mn_map(&a.a_map, a.A, a.K, a.M, a.lda, BM / 32) && encode_mn_map(&a.b_map, a.B, a.K, a.N, a.ldb, bn / 32)) {
