@@ -109,10 +109,13 @@ __global__ void __launch_bounds__(256) dh_kernel(const float* __restrict__ dcat1
 // Rows of hsT: 0-3 source, 4-7 destination, 8-11 negative.  Dynamic shared memory: head_fused_smem(d) bytes.
 // relu_out: the embedding rows are outputs of a ReLU layer (attention model) and dpre_o is masked by it;
 // otherwise dpre_o is the plain gradient with respect to the embedding rows.
-constexpr int HF_EV = 4, HF_THREADS = 512;
+// Two teams of 512 threads share the block's copy of W_1 and work on two groups side by side (their phases
+// are latency-bound, so the teams overlap almost for free, and a batch of 600 events -- 150 groups -- fits
+// 75 blocks with nothing left over for a second round).  Team barriers are the named barriers 1 and 2.
+constexpr int HF_EV = 4, HF_TEAM = 512, HF_TEAMS = 2, HF_THREADS = HF_TEAM * HF_TEAMS;
 __host__ __device__ inline int head_fused_w_floats(int d) { return (d * (2 * d + 1) + 3) & ~3; }
 inline size_t head_fused_smem(int d) {
-  return (size_t)(head_fused_w_floats(d) + 12 * d + 12 * d + 8 * d + 8 * 2 * d + d) * sizeof(float);
+  return (size_t)(head_fused_w_floats(d) + HF_TEAMS * (12 * d + 12 * d + 8 * d + 8 * 2 * d) + d) * sizeof(float);
 }
 
 __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __restrict__ h, const float* __restrict__ W1,
@@ -127,13 +130,15 @@ __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __r
   extern __shared__ __align__(16) float sm[];
   __shared__ float s_msum, s_gb2, s_loss;
   const int PW = 2 * d + 1;
-  float* W1s = sm;                              // [d][2d+1]
-  float* hsT = W1s + head_fused_w_floats(d);    // [d][12]   embedding rows, transposed
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int team = tid / HF_TEAM, tt = tid - team * HF_TEAM, wid = tt >> 5;  // team, thread and warp within the team
+  float* W1s = sm;                                                         // [d][2d+1]  (shared by the teams)
+  float* gw2 = W1s + head_fused_w_floats(d);                               // [d]        (shared)
+  float* hsT = gw2 + d + team * (12 * d + 12 * d + 8 * d + 16 * d);        // [d][12]   embedding rows, transposed
   float* part = hsT + 12 * d;                   // [d][12]   W_1a h_src | W_1b h_dst | W_1b h_neg per event
   float* dh1T = part + 12 * d;                  // [d][8]    d loss / d pre1, transposed
   float* dc = dh1T + 8 * d;                     // [2d][8]   partial input gradients of the lower half of j
-  float* gw2 = dc + 16 * d;                     // [d]
-  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  auto team_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "n"(HF_TEAM) : "memory"); };
   {  // W_1 [d][2d] -> padded rows; 2d is a multiple of 4 and the parameter block is 16-byte aligned
     const int n4 = d * 2 * d / 4, row4 = 2 * d / 4;
     const bool vec = (((uintptr_t)W1) & 15) == 0;
@@ -159,9 +164,9 @@ __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __r
   const float msum = s_msum;
   const float bias2 = b2[0];
   const int groups = (nq + HF_EV - 1) / HF_EV;
-  for (int grp = blockIdx.x; grp < groups; grp += gridDim.x) {
+  for (int grp = blockIdx.x * HF_TEAMS + team; grp < groups; grp += gridDim.x * HF_TEAMS) {
     const int ev0 = grp * HF_EV;
-    for (int e = tid; e < 12 * d; e += blockDim.x) {
+    for (int e = tt; e < 12 * d; e += HF_TEAM) {
       const int r = e / d, q = e - r * d;
       const int ev = ev0 + (r & 3), blk = r >> 2;
       float v = 0.f;
@@ -178,10 +183,10 @@ __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __r
       }
       hsT[q * 12 + r] = v;
     }
-    __syncthreads();
+    team_sync();
     // hidden layer in three parts: a thread owns hidden unit j and one block of 4 embedding rows (the
     // source rows serve the positive and the negative pair of their event, so their part is formed once)
-    for (int it = tid; it < 3 * d; it += blockDim.x) {
+    for (int it = tt; it < 3 * d; it += HF_TEAM) {
       const int blk = it / d, j = it - blk * d;
       const float* wr = W1s + j * PW + (blk ? d : 0);
       const float* hb = hsT + 4 * blk;
@@ -194,9 +199,9 @@ __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __r
       }
       *reinterpret_cast<float4*>(part + j * 12 + 4 * blk) = make_float4(a0, a1, a2, a3);
     }
-    __syncthreads();
+    team_sync();
     // scores, loss terms and d loss / d pre1: one warp per pair
-    for (int p = wid; p < 8; p += (blockDim.x >> 5)) {
+    for (int p = wid; p < 8; p += (HF_TEAM >> 5)) {
       const int half = p >> 2, e4 = p & 3, ev = ev0 + e4;
       const bool valid = ev < nq;
       const int o_col = 4 + 4 * half + e4;  // the pair's second row: destination or negative
@@ -226,13 +231,13 @@ __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __r
         }
       }
     }
-    __syncthreads();
+    team_sync();
     // input gradient: a thread owns column c of [h_a || h_b] for all 8 pairs over one half of the hidden
     // units; the lower half parks its sums in shared memory, the upper half adds them and folds the pairs
     // into the embedding rows (the source row collects its positive and its negative pair)
     const int jh = (d + 1) / 2;
-    for (int base = 0; base < 4 * d; base += blockDim.x) {  // items [0, 2d): lower half of j, [2d, 4d): upper half
-      const int it = base + tid;
+    for (int base = 0; base < 4 * d; base += HF_TEAM) {  // items [0, 2d): lower half of j, [2d, 4d): upper half
+      const int it = base + tt;
       const bool act = it < 4 * d;
       const int hi = act ? it / (2 * d) : 0, c = act ? it - hi * 2 * d : 0;
       float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -251,7 +256,7 @@ __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __r
           *reinterpret_cast<float4*>(dc + c * 8 + 4) = make_float4(a[4], a[5], a[6], a[7]);
         }
       }
-      __syncthreads();
+      team_sync();
       if (act && hi == 1) {
         const float4 u = *reinterpret_cast<const float4*>(dc + c * 8);
         const float4 v = *reinterpret_cast<const float4*>(dc + c * 8 + 4);
@@ -271,8 +276,9 @@ __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __r
         }
       }
     }
-    __syncthreads();
+    team_sync();
   }
+  __syncthreads();  // both teams are through: the block's sums are complete
   for (int q = tid; q < d; q += blockDim.x)
     if (gw2[q] != 0.f) atomicAdd(&g_w2[q], gw2[q]);
   if (tid == 0) {
@@ -747,9 +753,8 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       const int groups = (n_q + HF_EV - 1) / HF_EV;
       {
         KernelScope scope__(ctx, "head_fused", s);
-        // one block per SM (148) walking its groups, or two per SM when there are groups for all of them: a grid
-        // a little above the SM count would leave a few SMs with two blocks and everyone waiting for those
-        head_fused_kernel<<<groups <= 148 ? groups : (groups < 296 ? 148 : 296), HF_THREADS, hf_smem, s>>>(
+        // two groups per block side by side; at most one block per SM
+        head_fused_kernel<<<(groups + HF_TEAMS - 1) / HF_TEAMS < 148 ? (groups + HF_TEAMS - 1) / HF_TEAMS : 148, HF_THREADS, hf_smem, s>>>(
             ctx->e_h, P + L.w1, P + L.b1, P + L.w2, P + L.b2, loss_mask, n_q, d, w.cat1, w.hid1, w.hid_gate, w.dpre_o,
             G + L.w2, G + L.b2, w.st_scalars, relu_out);
       }
