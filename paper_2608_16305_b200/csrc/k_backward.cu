@@ -404,6 +404,85 @@ __global__ void __launch_bounds__(256) scatter_dmem_kernel(const float* __restri
   }
 }
 
+// The same scatter for batches in which many rows hit few nodes (hub nodes: tens of thousands of rows onto one
+// updated row serialise on its atomics).  A block takes SC_ROWS consecutive rows and first sums them per slot in
+// a small shared-memory table (SC_WAYS entries, claimed by compare-and-swap; a row whose slot finds its entry
+// taken by another slot goes to global memory directly), then adds every claimed entry to dMemU once.
+// Dynamic shared memory: SC_WAYS * d floats.
+constexpr int SC_ROWS = 128, SC_WAYS = 16;
+__global__ void __launch_bounds__(256) scatter_dmem_cached_kernel(const float* __restrict__ dZm,
+                                                                  const float* __restrict__ dcat_o,
+                                                                  const float* __restrict__ dzq,
+                                                                  const int32_t* __restrict__ nbr,
+                                                                  const int32_t* __restrict__ nodes, int n, int k, int d,
+                                                                  const int32_t* __restrict__ node2slot,
+                                                                  float* __restrict__ dMemU) {
+  extern __shared__ __align__(16) float s_acc[];  // [SC_WAYS][d]
+  __shared__ int s_id[SC_WAYS];
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const int nb_rows = n * k, total = nb_rows + n;
+  const int d4 = d >> 2;
+  for (int e = threadIdx.x; e < SC_WAYS * d; e += blockDim.x) s_acc[e] = 0.f;
+  if (threadIdx.x < SC_WAYS) s_id[threadIdx.x] = -1;
+  __syncthreads();
+  const int r_end = min(total, (int)(blockIdx.x + 1) * SC_ROWS);
+  for (int r = blockIdx.x * SC_ROWS + wid; r < r_end; r += 8) {
+    const bool isn = r < nb_rows;
+    const int i = r - nb_rows;
+    float4 g[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int q4 = lane + 32 * u;
+      g[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (q4 < d4) {
+        if (isn) {
+          g[u] = __ldg(reinterpret_cast<const float4*>(dZm + (int64_t)r * 2 * d) + q4);
+        } else {
+          const float4 a = __ldg(reinterpret_cast<const float4*>(dcat_o + (int64_t)i * 2 * d + d) + q4);
+          const float4 b = __ldg(reinterpret_cast<const float4*>(dzq + (int64_t)i * 2 * d) + q4);
+          g[u] = make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+        }
+      }
+    }
+    const int node = isn ? nbr[r] : nodes[i];
+    if (node < 0) continue;
+    const int slot = node2slot[node];
+    if (slot < 0) continue;
+    const int way = slot % SC_WAYS;
+    int owner = 0;
+    if (lane == 0) {
+      owner = atomicCAS(&s_id[way], -1, slot);
+      if (owner == -1) owner = slot;  // claimed now
+    }
+    owner = __shfl_sync(FULL, owner, 0);
+    if (owner == slot) {
+      float* acc = s_acc + way * d;
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int q4 = lane + 32 * u;
+        if (q4 < d4) {
+          atomicAdd(acc + 4 * q4, g[u].x); atomicAdd(acc + 4 * q4 + 1, g[u].y);
+          atomicAdd(acc + 4 * q4 + 2, g[u].z); atomicAdd(acc + 4 * q4 + 3, g[u].w);
+        }
+      }
+    } else {
+      float4* out = reinterpret_cast<float4*>(dMemU + (int64_t)slot * d);
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int q4 = lane + 32 * u;
+        if (q4 < d4) atomicAdd(out + q4, g[u]);
+      }
+    }
+  }
+  __syncthreads();
+  for (int w = wid; w < SC_WAYS; w += 8) {
+    const int slot = s_id[w];
+    if (slot < 0) continue;
+    float4* out = reinterpret_cast<float4*>(dMemU + (int64_t)slot * d);
+    for (int q4 = lane; q4 < d4; q4 += 32) atomicAdd(out + q4, *reinterpret_cast<const float4*>(s_acc + w * d + 4 * q4));
+  }
+}
+
 // Time-encoder gradient: G[r, col0 + c] is d loss / d Phi(dt_r)_c and S[r, c] = sin(arg) was kept by
 // the forward pass (S == nullptr: every row has dt = 0, sin(arg) = sin(b_c)).
 //   dw_c += -S dt_r G,   db_c += -S G
@@ -886,8 +965,13 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
         RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, 0, NB, nullptr, 2 * d, d, w.dZmp, 2 * d, "dZ_mem", s));
       {
         KernelScope scope__(ctx, "scatter_dmem", s);
-        scatter_dmem_kernel<<<(NB + R + 7) / 8, 256, 0, s>>>(w.dZmp, w.dcat_o, w.dzq, ctx->e_nbr, ctx->e_nodes, R, k, d,
-                                                             w.node2slot, w.dMemU);
+        // many rows per node (small node set, large batch): sum per block first, the hub rows would serialise
+        if ((int64_t)NB >= 4 * c.num_nodes)
+          scatter_dmem_cached_kernel<<<(NB + R + SC_ROWS - 1) / SC_ROWS, 256, (size_t)SC_WAYS * d * sizeof(float), s>>>(
+              w.dZmp, w.dcat_o, w.dzq, ctx->e_nbr, ctx->e_nodes, R, k, d, w.node2slot, w.dMemU);
+        else
+          scatter_dmem_kernel<<<(NB + R + 7) / 8, 256, 0, s>>>(w.dZmp, w.dcat_o, w.dzq, ctx->e_nbr, ctx->e_nodes, R, k, d,
+                                                               w.node2slot, w.dMemU);
       }
       TGNN_LAUNCH_OK(ctx, "scatter_dmem");
       const int U_cap = ctx->upd_cap;
