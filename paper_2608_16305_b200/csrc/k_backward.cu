@@ -508,43 +508,56 @@ __global__ void __launch_bounds__(256) time_grad_kernel(const float* __restrict_
   const int r0 = blockIdx.x * rows_per_block, r1 = min(R, r0 + rows_per_block);
   if (r0 >= r1) return;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  double gw[TG_MAXJ], gb[TG_MAXJ];
-  float sb[TG_MAXJ];
+  // a lane owns columns 4 (lane + 32 v) .. + 3, v = 0, 1 (d <= 256): 128-bit loads of G and S (d, ldg and col0 are
+  // multiples of 4 and the rows 16-byte aligned)
+  double gw[2][4], gb[2][4];
+  float4 sb[2];
 #pragma unroll
-  for (int j = 0; j < TG_MAXJ; ++j) {
-    gw[j] = 0.0; gb[j] = 0.0;
-    const int c = lane + 32 * j;
-    sb[j] = (S == nullptr && c < d) ? sinf(time_b[c]) : 0.f;
+  for (int v = 0; v < 2; ++v) {
+    const int c = 4 * (lane + 32 * v);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { gw[v][e] = 0.0; gb[v][e] = 0.0; }
+    sb[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (S == nullptr && c < d) sb[v] = make_float4(sinf(time_b[c]), sinf(time_b[c + 1]), sinf(time_b[c + 2]), sinf(time_b[c + 3]));
   }
   for (int rb = r0 + wid; rb < r1; rb += 32) {  // rows rb, rb + 8, rb + 16, rb + 24: loads first, sums after
-    float g[4][TG_MAXJ], sn[4][TG_MAXJ], dtr[4];
+    float4 g[4][2], sn[4][2];
+    float dtr[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int r = rb + 8 * u;
       const bool in = r < r1;
       dtr[u] = (in && dt) ? dt[r] : 0.f;
 #pragma unroll
-      for (int j = 0; j < TG_MAXJ; ++j) {
-        const int c = lane + 32 * j;
+      for (int v = 0; v < 2; ++v) {
+        const int c = 4 * (lane + 32 * v);
         const bool ok = in && c < d;
-        g[u][j] = ok ? G[(int64_t)r * ldg + col0 + c] : 0.f;
-        sn[u][j] = ok ? (S ? S[(int64_t)r * d + c] : sb[j]) : 0.f;
+        g[u][v] = ok ? __ldg(reinterpret_cast<const float4*>(G + (int64_t)r * ldg + col0 + c)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        sn[u][v] = ok ? (S ? __ldg(reinterpret_cast<const float4*>(S + (int64_t)r * d + c)) : sb[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
 #pragma unroll
-      for (int j = 0; j < TG_MAXJ; ++j) {
-        const double t = -(double)sn[u][j] * (double)g[u][j];
-        gw[j] = fma(t, (double)dtr[u], gw[j]);
-        gb[j] += t;
+      for (int v = 0; v < 2; ++v) {
+        const float ge[4] = {g[u][v].x, g[u][v].y, g[u][v].z, g[u][v].w};
+        const float se[4] = {sn[u][v].x, sn[u][v].y, sn[u][v].z, sn[u][v].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const double t = -(double)se[e] * (double)ge[e];
+          gw[v][e] = fma(t, (double)dtr[u], gw[v][e]);
+          gb[v][e] += t;
+        }
       }
     }
   }
 #pragma unroll
-  for (int j = 0; j < TG_MAXJ; ++j) {
-    const int c = lane + 32 * j;
-    if (c < d) { s_part[(wid * 2 + 0) * d + c] = gw[j]; s_part[(wid * 2 + 1) * d + c] = gb[j]; }
+  for (int v = 0; v < 2; ++v) {
+    const int c = 4 * (lane + 32 * v);
+    if (c < d) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) { s_part[(wid * 2 + 0) * d + c + e] = gw[v][e]; s_part[(wid * 2 + 1) * d + c + e] = gb[v][e]; }
+    }
   }
   __syncthreads();
   for (int e = threadIdx.x; e < 2 * d; e += blockDim.x) {
