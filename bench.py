@@ -309,6 +309,10 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
                      "algorithmic_bytes_per_launch": (U_est * (cfg.d_msg + cfg.d) * 4 + cfg.d * cfg.d_msg * 4) if jodie else
                      3 * n_q * cfg.k * (cfg.d_kv * 4 + 2 * cfg.d * 4) + 2 * cfg.d * cfg.d_kv * 4,
                      "flops_per_launch": flops, "avg_launch_us": dur_s * 1e6, "launches": cnt,
+                     # the default mode splits every operand into a TF32 head and tail: three tensor-core passes
+                     # per algorithmic product (not counted in "achieved"; shown here for the pipe's real load)
+                     "tensor_passes": 3 if args.math == "tf32" else 1,
+                     "issued_frac": (achieved * (3 if args.math == "tf32" else 1) / peak) if (peak and args.math != "fp32") else None,
                      "step_algorithmic_bytes": by, "step_algorithmic_flops": f_fwd + f_bwd,
                      "step_hbm_frac": (by / (ms_dev_max / K * 1e-3)) / (peaks["hbm_gbs"] * 1e9),
                      "kernel_share": {k: round(v[1] / tot, 4) for k, v in top[:12]},
