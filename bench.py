@@ -143,7 +143,8 @@ def run_ours(args, rank, world, device):
     stream = wl.make_stream(cfg)
     efeat = wl.edge_feature_table_torch(cfg, device)
     n_need = 2 * (args.steps + args.warmup) + 8
-    dw = T.DeviceWorkload(stream, device=device, efeat=efeat, batches=range(0, min(cfg.num_batches, n_need)))
+    dw = T.DeviceWorkload(stream, device=device, efeat=efeat, batches=range(0, min(cfg.num_batches, n_need)),
+                          embed_aux=args.embed_aux)
     weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed, model=args.model)
     math_mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST}[args.math]
     tr = T.Trainer(dw, weights, math_mode=math_mode, model=args.model)
@@ -222,7 +223,7 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
         tr.step_host(b, hb, loss_h, gn_h)
         torch.cuda.current_stream().synchronize()        # the caller reads the loss every step
         n, nq = hb["src"].numel(), hb["neg"].numel()
-        h2d += 21 * n + 20 * nq
+        h2d += 21 * n + 20 * nq + (nq if args.embed_aux else 0)    # + the target mask when every event is scored
         d2h += 8
 
     reset_epoch()
@@ -264,9 +265,10 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
     tot = sum(v[1] for v in prof.values()) or 1.0
     top = sorted(prof.items(), key=lambda kv: -kv[1][1])
 
-    n_q = cfg.batch
-    ms_dev_max, units = aggregate_over_ranks(ms_dev, K * n_q, device)
-    ms_host_max, _ = aggregate_over_ranks(ms_host, K * n_q, device)
+    # throughput counts target events only; with every event scored the roots are the whole mixed batch
+    ms_dev_max, units = aggregate_over_ranks(ms_dev, K * cfg.batch, device)
+    ms_host_max, _ = aggregate_over_ranks(ms_host, K * cfg.batch, device)
+    n_q = cfg.max_mixed if args.embed_aux else cfg.batch
     if rank != 0:
         return
     # roofline of the dominant kernel: the key/value projection GEMM of the attention layer
@@ -295,6 +297,8 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
                                + f", {cfg.num_events} events, d_e={cfg.d_e} {cfg.feat_dtype}, d={cfg.d}, k={cfg.k}, {cfg.heads} heads, "
                                f"batch {cfg.batch}, replay {cfg.replay_frac:g}" + (" with pruning" if cfg.prune else ""),
                    "model": "JODIE-style (recurrent cell + time projection)" if jodie else "TGN-style (GRU + temporal attention)",
+                   "scored_events": "every event of the mixed batch, auxiliary events under loss weight 0" if args.embed_aux
+                                    else "target events only",
                    "math_mode": args.math, "l2": "512 MB buffer written between timed steps (outside the event pairs)",
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "launch": "kernel by kernel" if args.no_graph else "CUDA graph replay of the step (captured by the library)",
@@ -323,7 +327,9 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
         out["adaptive"] = adaptive
     if preprocess is not None:
         out["preprocess"] = preprocess
-    out["cpu_baseline"] = cpu_baseline(cfg, stream, weights, budget_s=args.cpu_budget, model=args.model) if args.cpu_budget > 0 else None
+    # the host baseline times the default costing (target events only)
+    out["cpu_baseline"] = (cpu_baseline(cfg, stream, weights, budget_s=args.cpu_budget, model=args.model)
+                           if args.cpu_budget > 0 and not args.embed_aux else None)
     print(json.dumps(out))
 
 
@@ -470,6 +476,9 @@ def main():
                     help="also time the backward dependency scan and mixed-batch construction (adds a 'preprocess' object)")
     ap.add_argument("--adaptive", action="store_true",
                     help="also time the steps under the adaptive runtime controller (adds an 'adaptive' object)")
+    ap.add_argument("--embed-aux", action="store_true",
+                    help="embed and score every event of the mixed batch (auxiliary events under loss weight 0) "
+                         "instead of the target events only: the costing in which replay events pay the forward pass")
     ap.add_argument("--no-graph", action="store_true", help="launch kernel by kernel instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)

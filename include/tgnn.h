@@ -100,6 +100,12 @@ typedef struct {
   int32_t math_mode;  /* TGNN_MATH_* */
   float lr, beta1, beta2, eps; /* Adam */
   int32_t model;      /* TGNN_MODEL_* */
+  int32_t embed_aux;  /* 0: tgnn_step_mixed_host embeds and scores the target events only (auxiliary events
+                         carry loss weight 0, so their embeddings cannot change the result);
+                         1: it embeds and scores EVERY event of the mixed batch and applies the target
+                         mask of Eq. 12 in the loss (Eq. 13), the cost model of the workload analysis
+                         in which auxiliary events pay the forward pass too.  Loss, gradients and
+                         state are the same either way up to summation order. */
 } tgnn_config;
 
 /* ---- life cycle --------------------------------------------------------- */
@@ -252,7 +258,9 @@ TGNN_API int tgnn_train_step_host(tgnn_ctx* ctx, const int32_t* u_src_host, cons
 /* The streaming form of the step, host inputs: one call per mixed batch (Eq. 5), in stream order.
  * The call copies the batch to the device as one packed block, computes its prune mask (step 0,
  * arguments as in tgnn_prune_mask) beside the rest of the step, and trains on its target events
- * (is_aux == 0, in batch order; neg_host holds one negative destination per target event) after the
+ * (is_aux == 0, in batch order; neg_host holds one negative destination per target event; with
+ * cfg.embed_aux = 1 every event of the batch is embedded and scored under the mask 1 - is_aux, neg_host
+ * holds one negative per EVENT and max_roots must cover 3 n) after the
  * PREVIOUS call's batch, as kept by its mask, has updated memory (lag-one order).  The batch then
  * stays on the device for the next call.  tgnn_set_state restarts the sequence (no previous batch).
  * Host arrays may be pageable and are free for reuse when the call returns; loss_host /

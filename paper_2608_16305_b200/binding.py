@@ -44,7 +44,7 @@ class TgnnConfig(C.Structure):
                 ("heads", C.c_int32), ("feat_dtype", C.c_int32), ("max_events", C.c_int32),
                 ("max_roots", C.c_int32), ("math_mode", C.c_int32),
                 ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
-                ("model", C.c_int32)]
+                ("model", C.c_int32), ("embed_aux", C.c_int32)]
 
 
 class TgnnError(RuntimeError):
@@ -137,9 +137,10 @@ def _stream() -> int:
 
 
 def make_config(num_nodes, d, d_e, k, heads, feat_dtype=TGNN_F32, max_events=1024, max_roots=3072,
-                math_mode=TGNN_MATH_FP32, lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8, model=TGNN_MODEL_TGN) -> TgnnConfig:
+                math_mode=TGNN_MATH_FP32, lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8, model=TGNN_MODEL_TGN,
+                embed_aux=0) -> TgnnConfig:
     return TgnnConfig(num_nodes, d, d_e, k, heads, feat_dtype, max_events, max_roots, math_mode, lr, beta1, beta2, eps,
-                      model)
+                      model, int(embed_aux))
 
 
 def param_names(cfg: TgnnConfig):

@@ -741,14 +741,13 @@ int launch_tc(tgnn_ctx* ctx, const TcArgs& a, int n_tiles, const char* name, cud
   return TGNN_OK;
 }
 
-// Tiled tensor map of a row-major fp32 matrix [rows, cols] (row pitch ld floats): boxes of 32 columns x 128
-// rows, 128-byte swizzle, zeros outside.  The driver's encoder is looked up once through the runtime (no link
-// against the driver library).  Returns false if it is unavailable or refuses the shape.
-bool encode_a_map(CUtensorMap* map, const float* base, int64_t rows, int64_t cols, int64_t ld) {
-  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-  static EncodeFn enc = nullptr;
+// The driver's tensor-map encoder, looked up once through the runtime (no link against the driver library);
+// nullptr if it is unavailable.
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+TensorMapEncodeFn tensor_map_encoder() {
+  static TensorMapEncodeFn enc = nullptr;
   static bool looked = false;
   if (!looked) {
     looked = true;
@@ -756,9 +755,16 @@ bool encode_a_map(CUtensorMap* map, const float* base, int64_t rows, int64_t col
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) == cudaSuccess &&
         q == cudaDriverEntryPointSuccess)
-      enc = reinterpret_cast<EncodeFn>(fn);
+      enc = reinterpret_cast<TensorMapEncodeFn>(fn);
     (void)cudaGetLastError();
   }
+  return enc;
+}
+
+// Tiled tensor map of a row-major fp32 matrix [rows, cols] (row pitch ld floats): boxes of 32 columns x 128
+// rows, 128-byte swizzle, zeros outside.  Returns false if the encoder is unavailable or refuses the shape.
+bool encode_a_map(CUtensorMap* map, const float* base, int64_t rows, int64_t cols, int64_t ld) {
+  const TensorMapEncodeFn enc = tensor_map_encoder();
   if (!enc || rows <= 0 || cols <= 0) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
@@ -778,20 +784,7 @@ namespace {
 // one 512-byte atom per 32 columns, 32-byte swizzle.  rows must be a multiple of 4; the last atom of a row may run
 // past the row end (into the next row, or up to 124 bytes past the matrix).
 bool encode_mn_map(CUtensorMap* map, const float* base, int64_t rows, int64_t cols, int64_t ld, int box_atoms) {
-  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-  static EncodeFn enc = nullptr;
-  static bool looked = false;
-  if (!looked) {
-    looked = true;
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      enc = reinterpret_cast<EncodeFn>(fn);
-    (void)cudaGetLastError();
-  }
+  const TensorMapEncodeFn enc = tensor_map_encoder();
   if (!enc || rows <= 0 || cols <= 0 || rows % 4 != 0 || box_atoms < 1 || box_atoms > 8) return false;
   const cuuint64_t dims[4] = {32, 4, (cuuint64_t)((cols + 31) / 32), (cuuint64_t)(rows / 4)};
   const cuuint64_t strides[3] = {(cuuint64_t)ld * 4, 128, (cuuint64_t)ld * 16};

@@ -180,11 +180,12 @@ __global__ void __launch_bounds__(256) stage_inputs_kernel(StageArgs a) {
 }
 
 // Packed host block of tgnn_step_mixed_host: [t f64 n][q_t f64 nq][src,dst,eid i32 n each]
-// [q_src,q_dst,q_neg i32 nq each][is_aux u8 n].  Scattered into the mixed-batch slot and the target staging.
+// [q_src,q_dst,q_neg i32 nq each][is_aux u8 n][loss mask u8 nq, only if q_mask != nullptr].  Scattered into
+// the mixed-batch slot and the target staging.
 __global__ void __launch_bounds__(256) unpack_mixed_kernel(const unsigned char* __restrict__ pk, int n, int nq,
                                                            int32_t* src, int32_t* dst, int32_t* eid, double* t,
                                                            uint8_t* aux, uint8_t* keep, int32_t* q_src, int32_t* q_dst,
-                                                           int32_t* q_neg, double* q_t) {
+                                                           int32_t* q_neg, double* q_t, uint8_t* q_mask) {
   const double* p_t = reinterpret_cast<const double*>(pk);
   const double* p_qt = p_t + n;
   const int32_t* p_i = reinterpret_cast<const int32_t*>(p_qt + nq);
@@ -195,7 +196,10 @@ __global__ void __launch_bounds__(256) unpack_mixed_kernel(const unsigned char* 
     t[i] = p_t[i]; src[i] = p_i[i]; dst[i] = p_i[n + i]; eid[i] = p_i[2 * n + i];
     aux[i] = p_aux[i]; keep[i] = 1;
   }
-  if (i < nq) { q_t[i] = p_qt[i]; q_src[i] = p_q[i]; q_dst[i] = p_q[nq + i]; q_neg[i] = p_q[2 * nq + i]; }
+  if (i < nq) {
+    q_t[i] = p_qt[i]; q_src[i] = p_q[i]; q_dst[i] = p_q[nq + i]; q_neg[i] = p_q[2 * nq + i];
+    if (q_mask) q_mask[i] = p_aux[n + i];
+  }
 }
 
 // ---------------------------------------------------------------- step (3) --
@@ -421,7 +425,8 @@ int launch_stage_inputs(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_ds
   return TGNN_OK;
 }
 
-int launch_unpack_mixed(tgnn_ctx* ctx, const unsigned char* packed, int n, int n_q, int slot, cudaStream_t s) {
+int launch_unpack_mixed(tgnn_ctx* ctx, const unsigned char* packed, int n, int n_q, bool with_mask, int slot,
+                        cudaStream_t s) {
   const int m = n > n_q ? n : n_q;
   if (m == 0) return TGNN_OK;
   Workspace& w = ctx->ws;
@@ -429,7 +434,8 @@ int launch_unpack_mixed(tgnn_ctx* ctx, const unsigned char* packed, int n, int n
   {
     KernelScope scope__(ctx, "unpack_mixed", s);
     unpack_mixed_kernel<<<(m + 255) / 256, 256, 0, s>>>(packed, n, n_q, ms.src, ms.dst, ms.eid, ms.t, ms.aux, ms.keep,
-                                                        w.st_q_src, w.st_q_dst, w.st_q_neg, w.st_q_t);
+                                                        w.st_q_src, w.st_q_dst, w.st_q_neg, w.st_q_t,
+                                                        with_mask ? w.st_mask : nullptr);
   }
   TGNN_LAUNCH_OK(ctx, "unpack_mixed");
   return TGNN_OK;

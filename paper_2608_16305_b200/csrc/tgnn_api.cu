@@ -63,6 +63,7 @@ int check_config(const tgnn_config* c) {
   if (c->max_events < 1 || c->max_roots < 3 || c->max_events > (1 << 24) || c->max_roots > (1 << 24)) return TGNN_EINVAL;
   if (c->math_mode != TGNN_MATH_FP32 && c->math_mode != TGNN_MATH_TF32 && c->math_mode != TGNN_MATH_TF32_FAST) return TGNN_EINVAL;
   if (c->model != TGNN_MODEL_TGN && c->model != TGNN_MODEL_JODIE) return TGNN_EINVAL;
+  if (c->embed_aux != 0 && c->embed_aux != 1) return TGNN_EINVAL;
   if (!(c->lr >= 0.f) || !(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f) || !(c->eps > 0.f))
     return TGNN_EINVAL;
   return TGNN_OK;
@@ -221,7 +222,7 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
   }
   {
     const size_t ne = (size_t)cfg->max_events, nq = (size_t)ctx->nq_cap;
-    ctx->pack_bytes = (8 * ne + 8 * nq + 12 * ne + 12 * nq + ne + 63) & ~(size_t)63;
+    ctx->pack_bytes = (8 * ne + 8 * nq + 12 * ne + 12 * nq + ne + nq + 63) & ~(size_t)63;
     const size_t slot_bytes = (((12 + 8 + 2) * ne) + 255) & ~(size_t)255;
     unsigned char* base = nullptr;
     ctx->mixed_cur = -1;
@@ -585,9 +586,10 @@ int tgnn_step_mixed_host(tgnn_ctx* ctx, const int32_t* src, const int32_t* dst, 
   NEED(ctx, n <= ctx->cfg.max_events, TGNN_ECAPACITY, "step_mixed_host: n %d > max_events %d", n, ctx->cfg.max_events);
   NEED(ctx, n == 0 || (src && dst && t && eid && is_aux), TGNN_EINVAL, "step_mixed_host: null batch arrays");
   NEED(ctx, force_heavy >= -1 && force_heavy <= 1, TGNN_EINVAL, "step_mixed_host: force_heavy must be -1, 0 or 1");
+  const bool all = ctx->cfg.embed_aux != 0;  // every event is a root; the loss mask is 1 - is_aux
   int n_q = 0;
-  for (int i = 0; i < n; ++i) n_q += is_aux[i] == 0;
-  NEED(ctx, n_q <= ctx->nq_cap, TGNN_ECAPACITY, "step_mixed_host: %d target events > max_roots/3 = %d", n_q, ctx->nq_cap);
+  for (int i = 0; i < n; ++i) n_q += all || is_aux[i] == 0;
+  NEED(ctx, n_q <= ctx->nq_cap, TGNN_ECAPACITY, "step_mixed_host: %d scored events > max_roots/3 = %d", n_q, ctx->nq_cap);
   NEED(ctx, n_q == 0 || neg, TGNN_EINVAL, "step_mixed_host: null negatives");
   cudaStream_t s = S(stream);
   const int slot = ctx->mixed_cur < 0 ? 0 : 1 - ctx->mixed_cur;
@@ -599,20 +601,25 @@ int tgnn_step_mixed_host(tgnn_ctx* ctx, const int32_t* src, const int32_t* dst, 
   int32_t* p_i = reinterpret_cast<int32_t*>(p_qt + n_q);
   int32_t* p_q = p_i + 3 * (size_t)n;
   uint8_t* p_aux = reinterpret_cast<uint8_t*>(p_q + 3 * (size_t)n_q);
+  uint8_t* p_mask = p_aux + n;  // [n_q], present only when every event is scored
   memcpy(p_t, t, sizeof(double) * n);
   memcpy(p_i, src, sizeof(int32_t) * n);
   memcpy(p_i + n, dst, sizeof(int32_t) * n);
   memcpy(p_i + 2 * (size_t)n, eid, sizeof(int32_t) * n);
   memcpy(p_aux, is_aux, n);
   for (int i = 0, j = 0; i < n; ++i)
-    if (!is_aux[i]) { p_qt[j] = t[i]; p_q[j] = src[i]; p_q[n_q + j] = dst[i]; p_q[2 * (size_t)n_q + j] = neg[j]; ++j; }
-  const size_t bytes = (size_t)(p_aux + n - pk);
+    if (all || !is_aux[i]) {
+      p_qt[j] = t[i]; p_q[j] = src[i]; p_q[n_q + j] = dst[i]; p_q[2 * (size_t)n_q + j] = neg[j];
+      if (all) p_mask[j] = is_aux[i] ? 0 : 1;
+      ++j;
+    }
+  const size_t bytes = (size_t)(p_aux + n + (all ? n_q : 0) - pk);
   if (bytes > 0) TGNN_CUDA_OK(ctx, cudaMemcpyAsync(ctx->pack_dev, pk, bytes, cudaMemcpyHostToDevice, s));
   TGNN_CUDA_OK(ctx, cudaEventRecord(ctx->pack_done[slot], s));
   // the previous call's prune ran on a side stream: its keep mask is needed from here on
   int rc = fork_to(ctx, ctx->side[1], s);
   if (rc) return rc;
-  rc = launch_unpack_mixed(ctx, ctx->pack_dev, n, n_q, slot, s);
+  rc = launch_unpack_mixed(ctx, ctx->pack_dev, n, n_q, all, slot, s);
   if (rc) return rc;
   ctx->mixed[slot].n = n;
   if (n > 0) {  // step (0) for this batch, beside the step: its result is first read by the next call
@@ -626,8 +633,8 @@ int tgnn_step_mixed_host(tgnn_ctx* ctx, const int32_t* src, const int32_t* dst, 
   const tgnn_ctx::MixedSlot* u = ctx->mixed_cur >= 0 ? &ctx->mixed[ctx->mixed_cur] : nullptr;
   Workspace& w = ctx->ws;
   rc = tgnn_train_step(ctx, u ? u->src : nullptr, u ? u->dst : nullptr, u ? u->t : nullptr, u ? u->eid : nullptr,
-                       u ? u->keep : nullptr, u ? u->n : 0, w.st_q_src, w.st_q_dst, w.st_q_neg, w.st_q_t, n_q, nullptr,
-                       nullptr, nullptr, stream);
+                       u ? u->keep : nullptr, u ? u->n : 0, w.st_q_src, w.st_q_dst, w.st_q_neg, w.st_q_t, n_q,
+                       all ? w.st_mask : nullptr, nullptr, nullptr, stream);
   if (rc) return rc;
   ctx->mixed_cur = slot;
   if (loss_host) TGNN_CUDA_OK(ctx, cudaMemcpyAsync(loss_host, w.st_scalars + 2, sizeof(float), cudaMemcpyDeviceToHost, s));

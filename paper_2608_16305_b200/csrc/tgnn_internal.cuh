@@ -273,7 +273,8 @@ int launch_reduce_latest_events(tgnn_ctx* ctx, const int32_t* msg_node, const in
 int launch_stage_inputs(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, const double* u_t,
                         const int32_t* u_eid, const uint8_t* u_keep, int n_u, const int32_t* q_src, const int32_t* q_dst,
                         const int32_t* q_neg, const double* q_t, int n_q, const uint8_t* loss_mask, cudaStream_t s);
-int launch_unpack_mixed(tgnn_ctx* ctx, const unsigned char* packed, int n, int n_q, int slot, cudaStream_t s);
+int launch_unpack_mixed(tgnn_ctx* ctx, const unsigned char* packed, int n, int n_q, bool with_mask, int slot,
+                        cudaStream_t s);
 int launch_make_roots(tgnn_ctx* ctx, const int32_t* q_src, const int32_t* q_dst, const int32_t* q_neg,
                       const double* q_t, int n_q, cudaStream_t s);
 

@@ -22,10 +22,17 @@ from . import workload as wl
 
 
 class DeviceWorkload:
+    """The event stream, its neighbor index and its mixed batches on the device.
+
+    embed_aux: every event of a mixed batch is embedded and scored, auxiliary events under loss weight 0
+    (the target mask of Eq. 12 applied in Eq. 13), instead of the target events only; the negative of an
+    event is the stream's negative for its event id either way."""
+
     def __init__(self, stream: wl.EventStream, device="cuda", batches: Optional[range] = None,
-                 efeat: Optional[torch.Tensor] = None):
+                 efeat: Optional[torch.Tensor] = None, embed_aux: bool = False):
         cfg = stream.cfg
         self.cfg = cfg
+        self.embed_aux = bool(embed_aux)
         self.stream = stream
         dev = torch.device(device)
         self.device = dev
@@ -53,7 +60,14 @@ class DeviceWorkload:
         self.mb_keep = torch.ones_like(self.mb_aux) if mbs else None
         self.heavy = torch.zeros(len(mbs), dtype=torch.int32, device=dev)
         self.max_mixed = cfg.max_mixed      # capacities the library context is created with
-        self.max_targets = cfg.batch
+        self.max_targets = cfg.max_mixed if self.embed_aux else cfg.batch
+        self._scored_arrays()
+
+    def _scored_arrays(self):
+        """Negatives and loss mask per mixed-batch event (used when every event is scored)."""
+        if self.embed_aux and self.mb_aux is not None:
+            self.mb_neg = self.neg[self.mb_eid.long()].contiguous()
+            self.mb_lmask = (1 - self.mb_aux).contiguous()
 
     def mb_slice(self, b: int):
         i = b - self.batches.start
@@ -63,14 +77,34 @@ class DeviceWorkload:
         return slice(b * self.cfg.batch, min((b + 1) * self.cfg.batch, self.cfg.num_events))
 
     def targets(self, b: int):
-        """Device tensors (src, dst, neg, t) of the target events of batch b."""
+        """Device tensors (src, dst, neg, t) of the scored events of batch b: its target events, or every
+        event of the mixed batch under embed_aux."""
+        if self.embed_aux:
+            m = self.mb_slice(b)
+            return self.mb_src[m], self.mb_dst[m], self.mb_neg[m], self.mb_t[m]
+        return self._targets(b)
+
+    def _targets(self, b: int):
         q = self.target_slice(b)
         return self.src[q], self.dst[q], self.neg[q], self.t[q]
 
+    def loss_mask(self, b: int):
+        """Target mask (Eq. 12) over the scored events of batch b; None when all of them are targets."""
+        return self.mb_lmask[self.mb_slice(b)] if self.embed_aux else None
+
     def targets_host(self, b: int):
+        if self.embed_aux:
+            mb = self.mb_host[b - self.batches.start]
+            return mb.src, mb.dst, self.stream.neg[mb.eid], mb.t
+        return self._targets_host(b)
+
+    def _targets_host(self, b: int):
         q = self.target_slice(b)
         s = self.stream
         return s.src[q], s.dst[q], s.neg[q], s.t[q]
+
+    def loss_mask_host(self, b: int):
+        return (1 - self.mb_host[b - self.batches.start].is_aux).astype(np.uint8) if self.embed_aux else None
 
 
 class PartitionedWorkload(DeviceWorkload):
@@ -79,8 +113,8 @@ class PartitionedWorkload(DeviceWorkload):
     source-owned events of each global batch.  The scan and the batch construction run on the device."""
 
     def __init__(self, stream: wl.EventStream, owner: np.ndarray, P: int, p: int, K: int, device="cuda",
-                 efeat: Optional[torch.Tensor] = None):
-        super().__init__(stream, device=device, batches=range(0, 0), efeat=efeat)
+                 efeat: Optional[torch.Tensor] = None, embed_aux: bool = False):
+        super().__init__(stream, device=device, batches=range(0, 0), efeat=efeat, embed_aux=embed_aux)
         cfg = self.cfg
         dev = self.device
         E, nb = cfg.num_events, cfg.num_batches
@@ -111,7 +145,8 @@ class PartitionedWorkload(DeviceWorkload):
         self.batches = range(0, nb)
         self.heavy = torch.zeros(nb, dtype=torch.int32, device=dev)
         self.max_mixed = max(1, int(np.diff(self.mb_off).max()))
-        self.max_targets = max(1, int(np.diff(self.tgt_off).max()))
+        self.max_targets = self.max_mixed if self.embed_aux else max(1, int(np.diff(self.tgt_off).max()))
+        self._scored_arrays()
         h = [x.cpu().numpy() for x in (self.mb_src, self.mb_dst, self.mb_t, self.mb_eid, self.mb_aux)]
         self.mb_host = [wl.MixedBatch(b, *(a[self.mb_off[b]:self.mb_off[b + 1]] for a in h)) for b in range(nb)]
         self._tgt_host = [x.cpu().numpy() for x in (self.tgt_src, self.tgt_dst, self.tgt_neg, self.tgt_t)]
@@ -119,11 +154,11 @@ class PartitionedWorkload(DeviceWorkload):
     def _tslice(self, b: int):
         return slice(int(self.tgt_off[b]), int(self.tgt_off[b + 1]))
 
-    def targets(self, b: int):
+    def _targets(self, b: int):
         q = self._tslice(b)
         return self.tgt_src[q], self.tgt_dst[q], self.tgt_neg[q], self.tgt_t[q]
 
-    def targets_host(self, b: int):
+    def _targets_host(self, b: int):
         q = self._tslice(b)
         return tuple(a[q] for a in self._tgt_host)
 
@@ -135,7 +170,8 @@ class Trainer:
         self.tcfg = B.make_config(cfg.num_nodes, cfg.d, cfg.d_e, cfg.k, cfg.heads,
                                   feat_dtype=B.TGNN_BF16 if cfg.feat_dtype == "bf16" else B.TGNN_F32,
                                   max_events=dw.max_mixed, max_roots=3 * dw.max_targets, math_mode=math_mode, lr=lr,
-                                  model=B.TGNN_MODEL_JODIE if model == "jodie" else B.TGNN_MODEL_TGN)
+                                  model=B.TGNN_MODEL_JODIE if model == "jodie" else B.TGNN_MODEL_TGN,
+                                  embed_aux=dw.embed_aux)
         self.lib = B.Tgnn(self.tcfg)
         dev = dw.device
         P = B.param_layout(self.tcfg)["total"]
@@ -239,4 +275,4 @@ class Trainer:
             upd = (dw.mb_src[u], dw.mb_dst[u], dw.mb_t[u], dw.mb_eid[u], dw.mb_keep[u])
         else:
             upd = (None, None, None, None, None)
-        self.lib.train_step(*upd, tsrc, tdst, tneg, tt, None, self.loss, self.gradnorm)
+        self.lib.train_step(*upd, tsrc, tdst, tneg, tt, dw.loss_mask(b), self.loss, self.gradnorm)

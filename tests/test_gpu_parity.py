@@ -55,7 +55,8 @@ def orc_cfg(oracle, c, **kw):
 class Rig:
     """A workload on the device plus a library context and an oracle configuration."""
 
-    def __init__(self, B, oracle, cfg, math="fp32", batches=None, bias_scale=0.1, lr=1e-3, partition=None, model="tgn"):
+    def __init__(self, B, oracle, cfg, math="fp32", batches=None, bias_scale=0.1, lr=1e-3, partition=None, model="tgn",
+                 embed_aux=False):
         from paper_2608_16305_b200 import trainer
         self.B, self.oracle, self.cfg, self.math = B, oracle, cfg, math
         self.stream = wl.make_stream(cfg)
@@ -67,9 +68,9 @@ class Rig:
                 self.stream._efeat = self._to_host(efeat_dev)
         self.efeat_dev = efeat_dev
         if partition is None:
-            self.dw = trainer.DeviceWorkload(self.stream, batches=batches, efeat=efeat_dev)
+            self.dw = trainer.DeviceWorkload(self.stream, batches=batches, efeat=efeat_dev, embed_aux=embed_aux)
         else:   # (owner, P, p, K): worker p's mixed batches from the backward dependency scan
-            self.dw = trainer.PartitionedWorkload(self.stream, *partition, efeat=efeat_dev)
+            self.dw = trainer.PartitionedWorkload(self.stream, *partition, efeat=efeat_dev, embed_aux=embed_aux)
         self.model = model
         self.weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed, bias_scale=bias_scale, model=model)
         mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST}[math]
@@ -111,9 +112,11 @@ class Rig:
         torch.cuda.synchronize()
         return hg.cpu().numpy(), dg.cpu().numpy()
 
-    def oracle_step(self, pre, b, gates=None):
+    def oracle_step(self, pre, b, gates=None, loss_mask="workload"):
         o = self.oracle
         t_src, t_dst, t_neg, t_t = self.dw.targets_host(b)
+        if isinstance(loss_mask, str):
+            loss_mask = self.dw.loss_mask_host(b)
         nodes = np.concatenate([t_src, t_dst, t_neg])
         times = np.concatenate([t_t] * 3)
         if self.model == "jodie":
@@ -124,7 +127,7 @@ class Rig:
                 upd = (z, z, np.zeros(0), z, None)
             hint = {} if gates is None else dict(hid_gate=gates[1], gate_eps=GATE_EPS[self.math])
             res = oj.step(self.ocfg, pre["params"], pre["memory"], pre["last_update"], self.efeat, upd,
-                          (t_src, t_dst, t_neg, t_t), None, **hint)
+                          (t_src, t_dst, t_neg, t_t), loss_mask, **hint)
             return res, (nodes, times)
         nb = o.sample_recent(*self.graph, nodes, times, self.cfg.k)
         upd = self.upd_host(b)
@@ -145,7 +148,7 @@ class Rig:
         if gates is not None:
             kw = dict(h_gate=gates[0], hid_gate=gates[1], gate_eps=GATE_EPS[self.math])
         res = o.loss_and_grads(self.ocfg, pre["params"], pre["memory"], pre["last_update"], efeat, upd,
-                               roots, len(t_src), None, **kw)
+                               roots, len(t_src), loss_mask, **kw)
         return res, roots
 
     def check_step(self, b, pre, res, what=""):
@@ -506,6 +509,74 @@ def test_partitioned_worker_steps_on_scanned_mixed_batches(B, oracle, p):
     _run_epoch_checks(rig, range(cfg.num_batches), {1, 4, 7, cfg.num_batches - 1})
 
 
+# ------------------------------------------------- masked loss (Eq. 12-13)
+@pytest.mark.parametrize("model", ["tgn", "jodie"])
+@pytest.mark.parametrize("mask_kind", ["random", "none_set", "one_set"])
+def test_masked_loss_with_caller_mask(B, oracle, model, mask_kind):
+    """The step under an arbitrary target mask: masked events add nothing to the loss or to any gradient,
+    the mean runs over the unmasked ones, and a mask with no event set gives loss 0, a zero gradient and an
+    Adam step on a zero gradient (the memory update of the previous batch still happens)."""
+    rig = Rig(B, oracle, TINY, model=model)
+    tr, dw = rig.tr, rig.dw
+    rng = np.random.default_rng(5)
+    for b in range(4):
+        nq = len(dw.targets_host(b)[0])
+        mask = {"random": (rng.random(nq) < 0.4), "none_set": np.zeros(nq, bool),
+                "one_set": np.arange(nq) == nq // 3}[mask_kind].astype(np.uint8)
+        pre = rig.snapshot()
+        u = dw.mb_slice(b - 1) if b > 0 else None
+        upd = (dw.mb_src[u], dw.mb_dst[u], dw.mb_t[u], dw.mb_eid[u], dw.mb_keep[u]) if b > 0 else (None,) * 5
+        m_dev = torch.from_numpy(mask).cuda()
+        tr._run(lambda: tr.lib.train_step(*upd, *dw.targets(b), m_dev, tr.loss, tr.gradnorm))
+        res, _ = rig.oracle_step(pre, b, rig.gpu_gates(b), loss_mask=mask)
+        rig.check_step(b, pre, res, what=f"[{model} {mask_kind} batch {b}]")
+        if mask_kind == "none_set":
+            assert float(tr.loss.item()) == 0.0 and float(tr.gradnorm.item()) == 0.0
+
+
+@pytest.mark.parametrize("math", ["fp32", "tf32"])
+def test_every_event_scored_under_the_target_mask(B, oracle, math):
+    """embed_aux: every event of the mixed batch is a root (auxiliary events too, the costing in which replay
+    events pay the forward pass) and Eq. 13 weighs auxiliary events 0.  Each step matches the oracle on the
+    same roots and mask, and loss and gradient norm equal those of the target-only path from the same state."""
+    cfg = _scaled("reddit", 9000)
+    rig = Rig(B, oracle, cfg, math=math, embed_aux=True)
+    ref = Rig(B, oracle, cfg, math=math)
+    assert rig.tr.tcfg.embed_aux == 1 and rig.dw.max_targets == cfg.max_mixed
+    for b in range(cfg.num_batches):
+        mb = rig.dw.mb_host[b]
+        assert len(rig.dw.targets_host(b)[0]) == mb.n and int(rig.dw.loss_mask_host(b).sum()) == int((mb.is_aux == 0).sum())
+        for name in ("memory", "last_update", "params", "adam_m", "adam_v", "step_count"):
+            getattr(ref.tr, name).copy_(getattr(rig.tr, name))
+        pre = rig.snapshot() if b in {1, 6, 13} else None
+        rig.tr.step(b)
+        ref.tr.step(b)
+        torch.cuda.synchronize()
+        if pre is not None:
+            res, _ = rig.oracle_step(pre, b, rig.gpu_gates(b))
+            rig.check_step(b, pre, res, what=f"[embed_aux batch {b}]")
+        tol = 1e-5 if math == "fp32" else 1e-4
+        assert abs(float(rig.tr.loss.item()) - float(ref.tr.loss.item())) <= tol * abs(float(ref.tr.loss.item())), b
+        assert abs(float(rig.tr.gradnorm.item()) - float(ref.tr.gradnorm.item())) <= 10 * tol * float(ref.tr.gradnorm.item()), b
+        assert np.array_equal(rig.tr.last_update.cpu().numpy(), ref.tr.last_update.cpu().numpy())
+    assert sum(int(m.is_aux.sum()) for m in rig.dw.mb_host) > 0
+
+
+def test_partitioned_worker_scoring_every_event(B, oracle):
+    """The scanned mixed batches of one worker with every event scored: roots and mask come from the
+    device-built batch (the negatives by event id), and the steps match the oracle."""
+    cfg = _scaled("reddit", 7200)
+    owner = (np.arange(cfg.num_nodes) * 2654435761 % 2 ** 32 % 3).astype(np.int32)
+    rig = Rig(B, oracle, cfg, math="tf32", partition=(owner, 3, 1, 4), embed_aux=True)
+    for b in range(cfg.num_batches):
+        mb = rig.dw.mb_host[b]
+        s, d, n, t = rig.dw.targets_host(b)
+        assert np.array_equal(s, mb.src) and np.array_equal(n, rig.stream.neg[mb.eid])
+        assert np.array_equal(rig.dw.loss_mask_host(b), 1 - mb.is_aux)
+    _run_epoch_checks(rig, range(cfg.num_batches), {2, 5, cfg.num_batches - 1})
+
+
+
 @pytest.mark.parametrize("math", ["fp32", "tf32"])
 @pytest.mark.parametrize("name,events,at", [
     ("tiny", 4000, {0, 1, 2, 7, 19}),
@@ -565,12 +636,14 @@ def test_host_buffer_entry_point_matches_device_path(B, oracle):
     assert relerr(b.tr.params.cpu().numpy(), a.tr.params.cpu().numpy()) <= 2e-3
 
 
-def test_streaming_host_entry_point_matches_device_path(B, oracle):
+@pytest.mark.parametrize("embed_aux", [False, True])
+def test_streaming_host_entry_point_matches_device_path(B, oracle, embed_aux):
     # replay + pruning workload: the streaming call keeps each batch (and its prune mask) on the device for the
-    # next call, so agreement over several steps checks the slot hand-over and the mask as well
+    # next call, so agreement over several steps checks the slot hand-over and the mask as well; with every
+    # event scored the call also builds the roots and the target mask of the whole mixed batch
     cfg = _scaled("reddit", 9000)
-    a = Rig(B, oracle, cfg, math="tf32")
-    b = Rig(B, oracle, cfg, math="tf32")
+    a = Rig(B, oracle, cfg, math="tf32", embed_aux=embed_aux)
+    b = Rig(B, oracle, cfg, math="tf32", embed_aux=embed_aux)
     loss = torch.zeros(1).pin_memory()
     gn = torch.zeros(1).pin_memory()
     for step in range(cfg.num_batches):
@@ -613,7 +686,7 @@ def test_argument_errors_are_reported_not_launched(B):
 
 
 # ------------------------------------------ full-size workloads, bench launch configuration
-# The same teacher-forced comparison at the sizes the benchmark spec names, driven the way bench.py drives
+# The same teacher-forced comparison at the full sizes of the named workloads, driven the way bench.py drives
 # it: tensor-core mode, the whole step replayed as a CUDA graph on a capturable stream.  The oracle
 # needs seconds per step at these sizes, so only a few sampled steps are compared; every other step
 # still has to keep the device status clean.
