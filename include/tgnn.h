@@ -245,6 +245,23 @@ TGNN_API int tgnn_train_step(tgnn_ctx* ctx, const int32_t* u_src, const int32_t*
 
 TGNN_API int tgnn_set_graph_replay(tgnn_ctx* ctx, int enable);
 
+/* ---- gradient synchronisation across workers (Algorithm 2: the gradient norm g_r "is computed from
+ * the synchronised model gradients") ------------------------------------------------------------
+ * tgnn_set_grad_sync(ctx, 1): from now on tgnn_backward_step / tgnn_train_step and the host forms stop
+ * after the gradient: the complete fp32 gradient of the step is left in the context's gradient buffer,
+ * the loss is written, gradnorm_out receives the norm of the LOCAL gradient, and parameters, Adam
+ * moments and the step counter are untouched.  The caller reduces the buffer across workers in stream
+ * order (e.g. an NCCL all-reduce on the same stream) and calls tgnn_apply_gradient, which multiplies the
+ * buffer by `scale` (1 / workers for a mean; the product is stored), computes g_r = ||gradient||_2 into
+ * gradnorm_out (f32 device scalar, may be NULL) and performs the Adam step (step += 1).  A new step
+ * before the pending gradient is applied is refused with TGNN_ESTATE.  tgnn_set_grad_sync(ctx, 0)
+ * returns to the fused form; switching drops recorded step graphs (they are recorded again).
+ * tgnn_grad_buffer: *grads_dev_out = the buffer (device, param_count floats, owned by the context and
+ * valid for its lifetime; layout = the parameter layout), *count_out = param_count.  Both host pointers. */
+TGNN_API int tgnn_set_grad_sync(tgnn_ctx* ctx, int defer);
+TGNN_API int tgnn_grad_buffer(tgnn_ctx* ctx, float** grads_dev_out, int64_t* count_out);
+TGNN_API int tgnn_apply_gradient(tgnn_ctx* ctx, float scale, float* gradnorm_out, void* stream);
+
 /* The same step with HOST inputs and outputs: the event arrays are copied to
  * workspace staging buffers with cudaMemcpyAsync (pin them for overlap), and
  * loss / gradient norm are copied back to loss_host / gradnorm_host (may be
@@ -416,6 +433,37 @@ TGNN_API int tgnn_build_mixed(const int32_t* src, const int32_t* dst, const doub
                               double* mb_t, int32_t* mb_eid, uint8_t* mb_aux, int32_t* tgt_src, int32_t* tgt_dst,
                               double* tgt_t, int32_t* tgt_neg, int32_t* tgt_eid, int32_t* status_out, void* stream,
                               char* err_host, int64_t err_size);
+
+/* ---- boundary cache refresh (dynamic cache synchronisation: at an executed boundary, S_r = 1, worker p
+ * fetches the state of every node in N_sync[p] from the worker that owns it) -------------------------
+ * Stateless, device pointers, work enqueued on `stream`, nothing allocated; errors as above.  The
+ * exchange between the workers' processes is the caller's (one all-to-all of packed rows); these
+ * entry points compute who sends what and move the rows on each GPU.  A node's state is its memory
+ * row and its last-update time; a packed row is d + 2 floats (the row, then the low and high halves
+ * of the fp64 time), so d must be even and memory / packed 8-byte aligned.
+ *
+ * tgnn_refresh_plan: worker `me`'s plan for every window from tgnn_backward_scan's sync_out flags
+ *   (uint8[P, Q, num_nodes]) and the ownership map:
+ *   recv_nodes[q * cap + i], recv_off[q * (P + 1) + o]: the nodes of N_sync[me] in window q, grouped by
+ *       owner o (group o occupies [recv_off[o], recv_off[o + 1])), ascending ids within a group;
+ *   send_nodes / send_off: the nodes owned by `me` that worker r requests, grouped by r, ascending;
+ *       group r of `me`'s send list equals group `me` of worker r's receive list, element by element.
+ *   cap = elements per window in recv_nodes / send_nodes (the sum of the window's N_sync sizes over
+ *       all workers always suffices); status_out: device int32, zeroed by the call, 2 if cap was too
+ *       small (the excess is not written), 3 if a worker's N_sync names a node it owns (skipped).
+ * tgnn_pack_rows:   packed[i] = state of nodes[i]      (n rows; what an owner sends)
+ * tgnn_unpack_rows: state of nodes[i] = packed[i]      (n rows; what a requester received; nodes must be
+ *       distinct or the result for a repeated node is one of its rows)
+ *   status: device int32, NOT zeroed by these two; 4 is recorded for a node id outside [0, num_nodes)
+ *   (packed as zeros / not written). */
+TGNN_API int tgnn_refresh_plan(const uint8_t* sync, const int32_t* owner, int64_t num_nodes, int P, int Q, int me,
+                               int64_t cap, int32_t* recv_nodes, int32_t* recv_off, int32_t* send_nodes,
+                               int32_t* send_off, int32_t* status_out, void* stream, char* err_host, int64_t err_size);
+TGNN_API int tgnn_pack_rows(const float* memory, const double* last_update, int64_t num_nodes, int d,
+                            const int32_t* nodes, int n, float* packed, int32_t* status, void* stream, char* err_host,
+                            int64_t err_size);
+TGNN_API int tgnn_unpack_rows(float* memory, double* last_update, int64_t num_nodes, int d, const int32_t* nodes, int n,
+                              const float* packed, int32_t* status, void* stream, char* err_host, int64_t err_size);
 
 #ifdef __cplusplus
 }

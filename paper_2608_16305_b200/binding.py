@@ -35,7 +35,8 @@ EXPORTS = ("tgnn_create", "tgnn_destroy", "tgnn_last_error", "tgnn_param_count",
            "tgnn_profile_report", "tgnn_reduce_latest_static", "tgnn_debug_gemm", "tgnn_debug_get_gates", "tgnn_set_graph_replay", "tgnn_profile_timeline", "tgnn_step_mixed_host",
            "tgnn_controller_create", "tgnn_controller_destroy", "tgnn_controller_begin_batch",
            "tgnn_controller_end_batch", "tgnn_controller_state", "tgnn_backward_scan_scratch", "tgnn_backward_scan",
-           "tgnn_build_mixed")
+           "tgnn_build_mixed", "tgnn_set_grad_sync", "tgnn_grad_buffer", "tgnn_apply_gradient", "tgnn_refresh_plan",
+           "tgnn_pack_rows", "tgnn_unpack_rows")
 TGNN_STATIC_MAX_NODES = 65536
 
 
@@ -107,6 +108,12 @@ def load_library():
         lib.tgnn_backward_scan_scratch.restype = i64
         lib.tgnn_backward_scan.argtypes = [vp, vp, i64, i32, i32, vp, i64, i32, vp, vp, vp, vp, vp, vp, vp, i64]
         lib.tgnn_build_mixed.argtypes = [vp, vp, vp, vp, i64, i32, vp, vp, vp, i64, i64] + [vp] * 11 + [vp, vp, i64]
+        lib.tgnn_set_grad_sync.argtypes = [vp, i32]
+        lib.tgnn_grad_buffer.argtypes = [vp, C.POINTER(vp), C.POINTER(i64)]
+        lib.tgnn_apply_gradient.argtypes = [vp, C.c_float, vp, vp]
+        lib.tgnn_refresh_plan.argtypes = [vp, vp, i64, i32, i32, i32, i64, vp, vp, vp, vp, vp, vp, vp, i64]
+        lib.tgnn_pack_rows.argtypes = [vp, vp, i64, i32, vp, i32, vp, vp, vp, vp, i64]
+        lib.tgnn_unpack_rows.argtypes = [vp, vp, i64, i32, vp, i32, vp, vp, vp, vp, i64]
         _lib = lib
     return _lib
 
@@ -222,11 +229,47 @@ def build_mixed(src, dst, t, neg, batch: int, role, mb_off_out, tgt_off_out, mb,
     return rc
 
 
+def refresh_plan(sync, owner, P: int, Q: int, me: int, cap: int, recv_nodes, recv_off, send_nodes, send_off, status_out) -> int:
+    """tgnn_refresh_plan: worker `me`'s receive and send lists for every window (device tensors)."""
+    err = C.create_string_buffer(512)
+    rc = load_library().tgnn_refresh_plan(
+        _dp(sync, "u8", "sync"), _dp(owner, "i32", "owner"), owner.numel(), P, Q, me, cap,
+        _dp(recv_nodes, "i32", "recv_nodes"), _dp(recv_off, "i32", "recv_off"), _dp(send_nodes, "i32", "send_nodes"),
+        _dp(send_off, "i32", "send_off"), _dp(status_out, "i32", "status_out"), _stream(), C.addressof(err), len(err))
+    if rc != TGNN_OK:
+        raise TgnnError(rc, err.value.decode())
+    return rc
+
+
+def _rows(fn, memory, last_update, nodes, packed, status) -> int:
+    err = C.create_string_buffer(512)
+    n = 0 if nodes is None else nodes.numel()
+    if n and packed.numel() < n * (memory.shape[1] + 2):
+        raise TgnnError(TGNN_EINVAL, "packed buffer too small")
+    rc = fn(_dp(memory, "f32", "memory"), _dp(last_update, "f64", "last_update"), memory.shape[0], memory.shape[1],
+            _dp(nodes, "i32", "nodes"), n, _dp(packed, "f32", "packed"), _dp(status, "i32", "status"), _stream(),
+            C.addressof(err), len(err))
+    if rc != TGNN_OK:
+        raise TgnnError(rc, err.value.decode())
+    return rc
+
+
+def pack_rows(memory, last_update, nodes, packed, status) -> int:
+    """tgnn_pack_rows: packed[i] = (memory row, last-update time) of nodes[i], d + 2 floats per row."""
+    return _rows(load_library().tgnn_pack_rows, memory, last_update, nodes, packed, status)
+
+
+def unpack_rows(memory, last_update, nodes, packed, status) -> int:
+    """tgnn_unpack_rows: the state of nodes[i] becomes packed[i]."""
+    return _rows(load_library().tgnn_unpack_rows, memory, last_update, nodes, packed, status)
+
+
 class Controller:
     """The adaptive runtime controller (host-side; mirrors the tgnn_controller_* entry points)."""
 
     def __init__(self, alpha: float, beta: float, tau_g: float, tau_c: float, K: int):
         self.lib = load_library()
+        self.K = int(K)
         self._h = C.c_void_p()
         rc = self.lib.tgnn_controller_create(alpha, beta, tau_g, tau_c, K, C.byref(self._h))
         if rc != TGNN_OK:
@@ -393,6 +436,22 @@ class Tgnn:
 
     def set_graph_replay(self, enable: bool):
         self._ck(self.lib.tgnn_set_graph_replay(self._h, int(enable)))
+
+    def set_grad_sync(self, defer: bool):
+        """Steps stop after the gradient (to be reduced across workers); apply_gradient finishes them."""
+        self._ck(self.lib.tgnn_set_grad_sync(self._h, int(defer)))
+
+    def grad_buffer(self) -> torch.Tensor:
+        """The context's gradient buffer as a float32 CUDA tensor (a view; valid while the context lives)."""
+        ptr, n = C.c_void_p(), C.c_int64()
+        self._ck(self.lib.tgnn_grad_buffer(self._h, C.byref(ptr), C.byref(n)))
+
+        class _Mem:   # the CUDA array interface: torch wraps the pointer without copying
+            __cuda_array_interface__ = {"shape": (n.value,), "typestr": "<f4", "data": (ptr.value, False), "version": 2}
+        return torch.as_tensor(_Mem(), device=torch.device("cuda", torch.cuda.current_device()))
+
+    def apply_gradient(self, scale: float, gradnorm_out):
+        self._ck(self.lib.tgnn_apply_gradient(self._h, float(scale), _dp(gradnorm_out, "f32", "gradnorm_out"), _stream()))
 
     # ---- debug ----
     def debug_get_grads(self, grads_out):

@@ -661,13 +661,16 @@ __global__ void __launch_bounds__(256) gru_bwd_gate_kernel(const float* __restri
 // (every block has read the counter before it takes its ticket).
 // The time-encoder entries [t_off, t_off + t_n) and the time projection's [p_off, p_off + p_n) are taken
 // from their fp64 sums tg_acc (rounded once) and written into grads, where the debug export finds them.
+// apply = 0 stops after the gradient and its norm (parameters, moments and the step counter stay): the
+// caller synchronises the gradient across workers and comes back with t_n = p_n = 0 and gscale = 1 / workers;
+// a gscale other than 1 multiplies every gradient entry first and stores the product.
 __global__ void __launch_bounds__(256) gradnorm_adam_kernel(float* __restrict__ grads, int64_t P,
                                                             const double* __restrict__ tg_acc, int64_t t_off, int t_n,
                                                             int64_t p_off, int p_n, double* red, unsigned int* ticket, int64_t* step,
                                                             float* __restrict__ p, float* __restrict__ m,
                                                             float* __restrict__ v, float lr, float beta1, float beta2,
                                                             float eps, const float* __restrict__ loss_acc, float* scalars,
-                                                            float* loss_out, float* gradnorm_out) {
+                                                            float* loss_out, float* gradnorm_out, float gscale, int apply) {
   __shared__ double s_part[8];
   __shared__ float s_c1, s_c2;
   if (threadIdx.x == 0) {
@@ -683,6 +686,7 @@ __global__ void __launch_bounds__(256) gradnorm_adam_kernel(float* __restrict__ 
   // one parameter: gradient (from the fp64 sums where those exist), sum of squares, Adam
   auto one = [&](int64_t e, float ge, float& pe, float& me, float& ve) {
     acc = fma((double)ge, (double)ge, acc);
+    if (!apply) return;
     me = fmaf(beta1, me, omb1 * ge);
     ve = fmaf(beta2, ve, omb2 * ge * ge);
     pe -= lr * (me * c1) / (sqrtf(ve * c2) + eps);
@@ -706,14 +710,21 @@ __global__ void __launch_bounds__(256) gradnorm_adam_kernel(float* __restrict__ 
     } else {
       g4 = reinterpret_cast<const float4*>(grads)[q];
     }
-    float4 p4 = reinterpret_cast<float4*>(p)[q], m4 = reinterpret_cast<float4*>(m)[q], v4 = reinterpret_cast<float4*>(v)[q];
+    if (gscale != 1.f) {
+      g4 = make_float4(g4.x * gscale, g4.y * gscale, g4.z * gscale, g4.w * gscale);
+      reinterpret_cast<float4*>(grads)[q] = g4;
+    }
+    float4 p4 = make_float4(0.f, 0.f, 0.f, 0.f), m4 = p4, v4 = p4;
+    if (apply) { p4 = reinterpret_cast<float4*>(p)[q]; m4 = reinterpret_cast<float4*>(m)[q]; v4 = reinterpret_cast<float4*>(v)[q]; }
     one(e, g4.x, p4.x, m4.x, v4.x);
     one(e + 1, g4.y, p4.y, m4.y, v4.y);
     one(e + 2, g4.z, p4.z, m4.z, v4.z);
     one(e + 3, g4.w, p4.w, m4.w, v4.w);
-    reinterpret_cast<float4*>(p)[q] = p4;
-    reinterpret_cast<float4*>(m)[q] = m4;
-    reinterpret_cast<float4*>(v)[q] = v4;
+    if (apply) {
+      reinterpret_cast<float4*>(p)[q] = p4;
+      reinterpret_cast<float4*>(m)[q] = m4;
+      reinterpret_cast<float4*>(v)[q] = v4;
+    }
   }
   for (int64_t e = 4 * P4 + blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < P; e += (int64_t)gridDim.x * blockDim.x) {
     float ge;
@@ -726,9 +737,14 @@ __global__ void __launch_bounds__(256) gradnorm_adam_kernel(float* __restrict__ 
     } else {
       ge = grads[e];
     }
-    float pe = p[e], me = m[e], ve = v[e];
+    if (gscale != 1.f) {
+      ge *= gscale;
+      grads[e] = ge;
+    }
+    float pe = 0.f, me = 0.f, ve = 0.f;
+    if (apply) { pe = p[e]; me = m[e]; ve = v[e]; }
     one(e, ge, pe, me, ve);
-    p[e] = pe; m[e] = me; v[e] = ve;
+    if (apply) { p[e] = pe; m[e] = me; v[e] = ve; }
   }
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(FULL, acc, o);
   if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = acc;
@@ -743,7 +759,7 @@ __global__ void __launch_bounds__(256) gradnorm_adam_kernel(float* __restrict__ 
       __threadfence();
       const double ss = atomicAdd(&red[0], 0.0);
       const float gn = (float)sqrt(ss);
-      step[0] = step[0] + 1;
+      if (apply) step[0] = step[0] + 1;
       const float loss = *loss_acc;
       scalars[0] = loss;
       scalars[1] = gn;
@@ -1020,9 +1036,24 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     const int p_n = (n_q > 0 && c.model == TGNN_MODEL_JODIE) ? 2 * d : 0;
     gradnorm_adam_kernel<<<296, 256, 0, s>>>(G, L.total, w.tg_acc, L.time_w, n_q > 0 ? 2 * d : 0, L.proj_w, p_n, w.red, w.counters,
                                              ctx->step, P, ctx->adam_m, ctx->adam_v, c.lr, c.beta1, c.beta2, c.eps,
-                                             w.st_scalars, w.st_scalars + 2, loss_out, gradnorm_out);
+                                             w.st_scalars, w.st_scalars + 2, loss_out, gradnorm_out, 1.f, ctx->defer_adam ? 0 : 1);
   }
   TGNN_LAUNCH_OK(ctx, "gradnorm_adam");
+  return TGNN_OK;
+}
+
+// The second half of a step whose gradient was left for synchronisation: norm of gscale * gradient and Adam.
+int launch_apply_gradient(tgnn_ctx* ctx, float gscale, float* gradnorm_out, cudaStream_t s) {
+  const tgnn_config& c = ctx->cfg;
+  Workspace& w = ctx->ws;
+  TGNN_CUDA_OK(ctx, cudaMemsetAsync(w.red, 0, sizeof(double), s));
+  {
+    KernelScope scope__(ctx, "apply_gradient", s);
+    gradnorm_adam_kernel<<<296, 256, 0, s>>>(w.grads, ctx->L.total, w.tg_acc, 0, 0, 0, 0, w.red, w.counters, ctx->step,
+                                             ctx->params, ctx->adam_m, ctx->adam_v, c.lr, c.beta1, c.beta2, c.eps,
+                                             w.st_scalars, w.st_scalars + 2, nullptr, gradnorm_out, gscale, 1);
+  }
+  TGNN_LAUNCH_OK(ctx, "apply_gradient");
   return TGNN_OK;
 }
 

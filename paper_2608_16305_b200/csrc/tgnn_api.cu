@@ -257,6 +257,8 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
   ctx->ev_next = 0;
   ctx->n_graphs = 0;
   ctx->graphs_enabled = 1;
+  ctx->defer_adam = 0;
+  ctx->grad_pending = false;
   for (int i = 0; ok && i < 2; ++i) ok = cudaStreamCreateWithFlags(&ctx->side[i], cudaStreamNonBlocking) == cudaSuccess;
   for (int i = 0; ok && i < 32; ++i) ok = cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
@@ -328,6 +330,7 @@ int tgnn_set_state(tgnn_ctx* ctx, float* memory, double* last_update, float* par
   ctx->memory = memory; ctx->last_update = last_update; ctx->params = params;
   ctx->adam_m = adam_m; ctx->adam_v = adam_v; ctx->step = step;
   ctx->have_update = false; ctx->have_embed = false; ctx->grads_zeroed = false; ctx->images_fresh = false;
+  ctx->grad_pending = false;
   ctx->mixed_cur = -1;
   return TGNN_OK;
 }
@@ -409,7 +412,9 @@ int tgnn_backward_step(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* 
   NEED(ctx, ctx->have_embed, TGNN_ESTATE, "backward_step: no tgnn_embed call to differentiate");
   NEED(ctx, n_q >= 0 && 3 * n_q == ctx->e_n, TGNN_ESHAPE, "backward_step: the last embed call had %d rows, expected 3*n_q = %d",
        ctx->e_n, 3 * n_q);
+  NEED(ctx, !ctx->grad_pending, TGNN_ESTATE, "backward_step: the previous step's gradient has not been applied (tgnn_apply_gradient)");
   const int rc = launch_backward(ctx, n_q, loss_mask, loss_out, gradnorm_out, S(stream));
+  ctx->grad_pending = ctx->defer_adam != 0 && rc == TGNN_OK;
   ctx->have_embed = false;
   ctx->have_update = false;
   ctx->grads_zeroed = false;
@@ -499,9 +504,41 @@ void after_replay(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q) {
   ctx->e_nodes = w.r_node; ctx->e_times = w.r_time; ctx->e_nbr = w.nb_node; ctx->e_eid = w.nb_eid;
   ctx->e_ts = w.nb_ts; ctx->e_cnt = w.nb_cnt; ctx->e_n = 3 * n_q; ctx->e_h = w.h;
   ctx->have_embed = false; ctx->have_update = false; ctx->grads_zeroed = false; ctx->images_fresh = false;
+  ctx->grad_pending = ctx->defer_adam != 0;
 }
 
 }  // namespace
+
+int tgnn_set_grad_sync(tgnn_ctx* ctx, int defer) {
+  if (!ctx) return TGNN_EINVAL;
+  if ((defer != 0) == (ctx->defer_adam != 0)) return TGNN_OK;
+  // recorded steps end with the fused norm + Adam launch of the other mode: drop them
+  for (int i = 0; i < ctx->n_graphs; ++i)
+    if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
+  ctx->n_graphs = 0;
+  ctx->defer_adam = defer ? 1 : 0;
+  ctx->grad_pending = false;
+  return TGNN_OK;
+}
+
+int tgnn_grad_buffer(tgnn_ctx* ctx, float** grads_dev_out, int64_t* count_out) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, grads_dev_out && count_out, TGNN_EINVAL, "grad_buffer: null pointer");
+  *grads_dev_out = ctx->ws.grads;
+  *count_out = ctx->L.total;
+  return TGNN_OK;
+}
+
+int tgnn_apply_gradient(tgnn_ctx* ctx, float scale, float* gradnorm_out, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, ctx->defer_adam, TGNN_ESTATE, "apply_gradient: the context applies Adam inside the step (tgnn_set_grad_sync(ctx, 1) first)");
+  NEED(ctx, ctx->grad_pending, TGNN_ESTATE, "apply_gradient: no step has left a gradient to apply");
+  NEED(ctx, scale == scale && scale != 0.f, TGNN_EINVAL, "apply_gradient: scale must be a non-zero number");
+  const int rc = launch_apply_gradient(ctx, scale, gradnorm_out, S(stream));
+  ctx->grad_pending = false;
+  ctx->images_fresh = false;  // Adam has changed the parameters
+  return rc;
+}
 
 int tgnn_set_graph_replay(tgnn_ctx* ctx, int enable) {
   if (!ctx) return TGNN_EINVAL;
@@ -520,6 +557,7 @@ int tgnn_train_step(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, c
   NEED(ctx, n_u == 0 || (u_src && u_dst && u_t && u_eid), TGNN_EINVAL, "train_step: null update arrays");
   NEED(ctx, n_q == 0 || (q_src && q_dst && q_neg && q_t), TGNN_EINVAL, "train_step: null target arrays");
   NEED(ctx, ctx->memory && ctx->indptr, TGNN_ESTATE, "train_step: tgnn_set_state / tgnn_set_graph have not been called");
+  NEED(ctx, !ctx->grad_pending, TGNN_ESTATE, "train_step: the previous step's gradient has not been applied (tgnn_apply_gradient)");
   const bool has_keep = n_u > 0 && u_keep != nullptr, has_mask = n_q > 0 && loss_mask != nullptr;
   int rc = launch_stage_inputs(ctx, u_src, u_dst, u_t, u_eid, u_keep, n_u, q_src, q_dst, q_neg, q_t, n_q, loss_mask,
                                S(stream));

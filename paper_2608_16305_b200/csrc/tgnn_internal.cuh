@@ -196,6 +196,10 @@ struct tgnn_ctx {
   StepGraph graphs[8];
   int n_graphs;
   int graphs_enabled;
+  // Gradient synchronisation across workers: the step stops after the gradient, the caller reduces
+  // the buffer and tgnn_apply_gradient finishes the step.
+  int defer_adam;
+  bool grad_pending;
   int64_t launches;
   tgnn::Profiler prof;
   char err[256];
@@ -292,6 +296,7 @@ int launch_embed_static(tgnn_ctx* ctx, const double* times, int n, const int32_t
                         const double* ts, cudaStream_t s);
 
 // ---- backward + Adam (k_backward.cu) ----
+int launch_apply_gradient(tgnn_ctx* ctx, float gscale, float* gradnorm_out, cudaStream_t s);
 int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* loss_out, float* gradnorm_out,
                     cudaStream_t s);
 

@@ -113,7 +113,7 @@ class PartitionedWorkload(DeviceWorkload):
     source-owned events of each global batch.  The scan and the batch construction run on the device."""
 
     def __init__(self, stream: wl.EventStream, owner: np.ndarray, P: int, p: int, K: int, device="cuda",
-                 efeat: Optional[torch.Tensor] = None, embed_aux: bool = False):
+                 efeat: Optional[torch.Tensor] = None, embed_aux: bool = False, keep_sync: bool = False):
         super().__init__(stream, device=device, batches=range(0, 0), efeat=efeat, embed_aux=embed_aux)
         cfg = self.cfg
         dev = self.device
@@ -123,9 +123,11 @@ class PartitionedWorkload(DeviceWorkload):
         self.P, self.p, self.K = P, p, K
         self.role = torch.empty((P, E), dtype=torch.uint8, device=dev)
         self.n_sync = torch.empty((P, Q), dtype=torch.int32, device=dev)
+        # N_sync membership flags of every (worker, window): the input of the boundary refresh plan
+        self.sync = torch.empty((P, Q, cfg.num_nodes), dtype=torch.uint8, device=dev) if keep_sync else None
         scratch = torch.empty(B.backward_scan_scratch(E, cfg.batch, K, cfg.num_nodes, P), dtype=torch.int32, device=dev)
         status = torch.zeros(1, dtype=torch.int32, device=dev)
-        B.backward_scan(self.src, self.dst, cfg.batch, K, self.owner, P, self.role, self.n_sync, None, scratch, status)
+        B.backward_scan(self.src, self.dst, cfg.batch, K, self.owner, P, self.role, self.n_sync, self.sync, scratch, status)
         off = torch.empty(nb + 1, dtype=torch.int32, device=dev)
         toff = torch.empty(nb + 1, dtype=torch.int32, device=dev)
         i32 = lambda: torch.empty(E, dtype=torch.int32, device=dev)
@@ -150,6 +152,13 @@ class PartitionedWorkload(DeviceWorkload):
         h = [x.cpu().numpy() for x in (self.mb_src, self.mb_dst, self.mb_t, self.mb_eid, self.mb_aux)]
         self.mb_host = [wl.MixedBatch(b, *(a[self.mb_off[b]:self.mb_off[b + 1]] for a in h)) for b in range(nb)]
         self._tgt_host = [x.cpu().numpy() for x in (self.tgt_src, self.tgt_dst, self.tgt_neg, self.tgt_t)]
+
+    def refresh_plan(self):
+        """This worker's boundary refresh plan for every window (needs keep_sync=True)."""
+        from . import distributed as D
+        if self.sync is None:
+            raise RuntimeError("the workload was built without the N_sync flags (keep_sync=True)")
+        return D.RefreshPlan(self.sync, self.owner, self.n_sync.cpu().numpy(), self.P, self.p)
 
     def _tslice(self, b: int):
         return slice(int(self.tgt_off[b]), int(self.tgt_off[b + 1]))
@@ -255,6 +264,49 @@ class Trainer:
             e0.record()
             self._step(b, True, heavy, 0xFFFFFFFF)
             e1.record()
+        self._run(run)
+        e1.synchronize()
+        c = float(e0.elapsed_time(e1)) if batch_time is None else float(batch_time)
+        g = float(self.gradnorm.item())
+        ctl.end_batch(g, c)
+        return dict(r=r, boundary=boundary, sync=sync, heavy=heavy, g=g, c=c)
+
+    def step_distributed(self, b: int, ctl: "B.Controller", refresh=None, group=None, reduce_gradient=None,
+                         batch_time: Optional[float] = None):
+        """One step of one worker among several (Algorithm 2 with its exchanges).
+
+        At a candidate boundary the coordinator's decision S_r is broadcast and, if 1, the boundary
+        refresh of the window that starts here runs on the tables as they stand (the lag-one update of
+        the previous batch is applied after it, by this worker's own mixed batch).  The step then stops
+        after the gradient; the workers' gradients are summed (`reduce_gradient(buffer)`, default an
+        all-reduce over `group`), and norm and Adam run on their mean, so g_r is the same number on every
+        worker.  Requires lib.set_grad_sync(True).
+        """
+        from . import distributed as D
+        import torch.distributed as dist
+        r = b - self.dw.batches.start
+        boundary, sync, heavy = ctl.begin_batch(r)
+        multi = dist.is_available() and dist.is_initialized()
+        if boundary and refresh is not None:
+            if multi:
+                sync = D.broadcast_decision(sync, self.dw.device, group)
+            if sync:
+                self._run(lambda: refresh.run(r // ctl.K, self.memory, self.last_update))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        world = dist.get_world_size(group) if multi else 1
+
+        def run():
+            e0.record()
+            self._step(b, True, heavy, 0xFFFFFFFF)
+            e1.record()                                     # the worker's own batch time excludes the wait for the others
+            g = self.lib.grad_buffer()
+            if reduce_gradient is not None:
+                world_ = reduce_gradient(g)
+            else:
+                if world > 1:
+                    dist.all_reduce(g, op=dist.ReduceOp.SUM, group=group)
+                world_ = world
+            self.lib.apply_gradient(1.0 / world_, self.gradnorm)
         self._run(run)
         e1.synchronize()
         c = float(e0.elapsed_time(e1)) if batch_time is None else float(batch_time)

@@ -169,6 +169,14 @@ class Rig:
         g = torch.zeros_like(tr.params)
         tr.lib.debug_get_grads(g)
         g = g.cpu().numpy().astype(np.float64)
+        self.check_grads(g, res, what)
+        e = abs(float(tr.gradnorm.item()) - res.gradnorm) / max(res.gradnorm, 1e-6)
+        assert e <= tol, f"{what} gradnorm {tr.gradnorm.item()} vs {res.gradnorm}"
+        self.check_adam(g, pre, what)
+
+    def check_grads(self, g, res, what=""):
+        """A gradient (fp64 copy of the GPU's) against the oracle's, tensor by tensor."""
+        tol = self.tol
         # b_k's gradient is identically zero in exact arithmetic (softmax is shift invariant, so the
         # logit gradients of a root sum to zero); what both sides hold is rounding residue.  Such a
         # tensor is measured on the scale of the gradient as a whole: floor = 1e-3 x largest entry.
@@ -177,9 +185,10 @@ class Rig:
             sl = slice(self.lay[name], self.lay[name] + int(np.prod(self.shapes[name])))
             e = float(np.abs(g[sl] - res.grads[sl]).max() / max(np.abs(res.grads[sl]).max(), floor, 1e-6))
             assert e <= tol, f"{what} grad {name} err {e}"
-        e = abs(float(tr.gradnorm.item()) - res.gradnorm) / max(res.gradnorm, 1e-6)
-        assert e <= tol, f"{what} gradnorm {tr.gradnorm.item()} vs {res.gradnorm}"
-        # Adam, fed with the GPU's own gradient
+
+    def check_adam(self, g, pre, what=""):
+        """The GPU's parameter update against the oracle's Adam fed with the gradient g the GPU applied."""
+        tr, o = self.tr, self.oracle
         p_ref, m_ref, v_ref, st = o.adam(self.ocfg, g, pre["params"], pre["m"], pre["v"], pre["step"])
         assert int(tr.step_count.item()) == st
         upd_gpu = tr.params.cpu().numpy().astype(np.float64) - pre["params"]
@@ -507,6 +516,136 @@ def test_partitioned_worker_steps_on_scanned_mixed_batches(B, oracle, p):
         assert np.all(np.diff(mb.t) >= 0)                                        # timestamp order (Eq. 5)
     assert sum(int(m.is_aux.sum()) for m in dw.mb_host) > 0
     _run_epoch_checks(rig, range(cfg.num_batches), {1, 4, 7, cfg.num_batches - 1})
+
+
+# ------------------------------------------------- gradient synchronisation across workers
+def test_deferred_gradient_then_apply_equals_the_fused_step(B, oracle):
+    """With gradient synchronisation on, a step leaves its complete gradient in the context's buffer and
+    touches neither parameters nor Adam state; tgnn_apply_gradient then finishes it.  Against a second
+    context that runs the fused step from the same state: same gradient, same loss, same norm; the applied
+    update is the oracle's Adam on scale x the buffer.  Steps are replayed as CUDA graphs from the third on."""
+    cfg = _scaled("reddit", 9000)
+    a = Rig(B, oracle, cfg, math="tf32")
+    b = Rig(B, oracle, cfg, math="tf32")
+    b.tr.lib.set_grad_sync(True)
+    names = ("memory", "last_update", "params", "adam_m", "adam_v", "step_count")
+    for step in range(8):
+        for name in names:
+            getattr(b.tr, name).copy_(getattr(a.tr, name))
+        pre = b.snapshot()
+        a.tr.step(step)
+        b.tr.step(step)
+        torch.cuda.synchronize()
+        assert np.array_equal(b.tr.params.cpu().numpy(), pre["params"].astype(np.float32))
+        assert int(b.tr.step_count.item()) == pre["step"] and np.array_equal(b.tr.adam_m.cpu().numpy(), pre["m"].astype(np.float32))
+        ga = torch.zeros_like(a.tr.params)
+        a.tr.lib.debug_get_grads(ga)
+        gb = b.tr.lib.grad_buffer()
+        assert gb.numel() == ga.numel()
+        assert relerr(gb.cpu().numpy(), ga.cpu().numpy()) <= 1e-4
+        assert abs(float(b.tr.loss.item()) - float(a.tr.loss.item())) <= 1e-5 * abs(float(a.tr.loss.item()))
+        assert abs(float(b.tr.gradnorm.item()) - float(a.tr.gradnorm.item())) <= 1e-4 * float(a.tr.gradnorm.item())
+        assert relerr(b.tr.memory.cpu().numpy(), a.tr.memory.cpu().numpy()) <= 1e-5
+        # a new step while the gradient is pending is refused on the host
+        with pytest.raises(B.TgnnError) as ei:
+            b.tr.lib.train_step(None, None, None, None, None, *b.dw.targets(step), None, b.tr.loss, b.tr.gradnorm)
+        assert ei.value.code == B.TGNN_ESTATE
+        scale = 1.0 if step % 2 == 0 else 0.5
+        g_local = gb.cpu().numpy().astype(np.float64)
+        b.tr._run(lambda: b.tr.lib.apply_gradient(scale, b.tr.gradnorm))
+        torch.cuda.synchronize()
+        g_applied = b.tr.lib.grad_buffer().cpu().numpy().astype(np.float64)
+        assert np.array_equal(g_applied, g_local * scale)                     # the product is stored (exact for 1 and 1/2)
+        want = np.sqrt(np.sum(g_applied * g_applied))
+        assert abs(float(b.tr.gradnorm.item()) - want) <= 1e-6 * want
+        b.check_adam(g_applied, pre, what=f"[deferred step {step}]")
+        with pytest.raises(B.TgnnError):
+            b.tr.lib.apply_gradient(1.0, b.tr.gradnorm)                       # nothing pending any more
+    with pytest.raises(B.TgnnError):
+        a.tr.lib.apply_gradient(1.0, a.tr.gradnorm)                           # fused mode has nothing to apply
+    # back to the fused form: the next step applies Adam by itself again
+    b.tr.lib.set_grad_sync(False)
+    st = int(b.tr.step_count.item())
+    b.tr.step(8)
+    torch.cuda.synchronize()
+    assert int(b.tr.step_count.item()) == st + 1
+
+
+def test_two_emulated_workers_with_synchronised_gradient_match_oracle(B, oracle):
+    """Two workers of a 2-way node partition on one device, run one after the other: each steps on its
+    scanned mixed batch up to the gradient, the all-reduce is written out (both buffers receive the sum),
+    each applies the mean.  Local gradients match the oracle's per worker, g_r matches the norm of the
+    oracle's mean gradient and is the same number on both, the update is Adam on the mean, and the two
+    replicas of the parameters stay bitwise identical."""
+    from oracle import refresh as orf
+    cfg = _scaled("reddit", 7200)
+    owner = (np.arange(cfg.num_nodes) * 2654435761 % 2 ** 32 % 2).astype(np.int32)
+    rigs = [Rig(B, oracle, cfg, math="tf32", partition=(owner, 2, p, 4)) for p in range(2)]
+    for r in rigs:
+        r.tr.lib.set_grad_sync(True)
+    check = {1, 4, 9, cfg.num_batches - 1}
+    for b in range(cfg.num_batches):
+        pres = [r.snapshot() for r in rigs] if b in check else None
+        for r in rigs:
+            r.tr.step(b)
+        bufs = [r.tr.lib.grad_buffer() for r in rigs]
+        local = [x.clone() for x in bufs]
+        losses = [float(r.tr.loss.item()) for r in rigs]
+        total = bufs[0] + bufs[1]
+        for r, buf in zip(rigs, bufs):
+            buf.copy_(total)
+            r.tr._run(lambda r=r: r.tr.lib.apply_gradient(0.5, r.tr.gradnorm))
+        torch.cuda.synchronize()
+        for name in ("params", "adam_m", "adam_v", "step_count"):
+            assert torch.equal(getattr(rigs[0].tr, name), getattr(rigs[1].tr, name)), (b, name)
+        assert float(rigs[0].tr.gradnorm.item()) == float(rigs[1].tr.gradnorm.item())
+        if pres is not None:
+            res = [r.oracle_step(pre, b, r.gpu_gates(b))[0] for r, pre in zip(rigs, pres)]
+            for p, r in enumerate(rigs):
+                r.check_grads(local[p].cpu().numpy().astype(np.float64), res[p], what=f"[worker {p} batch {b}]")
+                assert abs(losses[p] - res[p].loss) <= r.tol * max(abs(res[p].loss), 1e-6)
+                assert relerr(r.tr.memory.cpu().numpy()[res[p].uniq], res[p].memory_post[res[p].uniq]) <= r.tol
+            mean, g = orf.synchronised_gradient([x.grads for x in res])
+            assert abs(float(rigs[0].tr.gradnorm.item()) - g) <= rigs[0].tol * g
+            applied = bufs[0].cpu().numpy().astype(np.float64)
+            assert np.array_equal(applied, (total * 0.5).cpu().numpy().astype(np.float64))
+            for r, pre in zip(rigs, pres):
+                r.check_adam(applied, pre, what=f"[synchronised batch {b}]")
+
+
+def test_distributed_step_of_a_single_worker_runs_refresh_decisions_and_applies_its_own_gradient(B, oracle):
+    """Trainer.step_distributed without a process group: the controller's boundary decisions are taken, the
+    refresh callback runs exactly at the executed boundaries with the window index, the gradient hook sees
+    the context's buffer, and the step equals the fused step of a second context."""
+    cfg = _scaled("reddit", 9000)
+    a = Rig(B, oracle, cfg, math="tf32")
+    b = Rig(B, oracle, cfg, math="tf32")
+    b.tr.lib.set_grad_sync(True)
+    ctl = B.Controller(alpha=0.1, beta=0.1, tau_g=1.6, tau_c=1e9, K=3)
+
+    class Probe:
+        def __init__(self):
+            self.calls = []
+
+        def run(self, q, memory, last_update):
+            self.calls.append(q)
+    probe, seen, logs = Probe(), [], []
+
+    def reduce(buf):
+        seen.append(buf.data_ptr())
+        return 1
+    for step in range(10):
+        for name in ("memory", "last_update", "params", "adam_m", "adam_v", "step_count"):
+            getattr(b.tr, name).copy_(getattr(a.tr, name))
+        pre = b.snapshot()
+        a.tr.step(step, force_heavy=0)
+        logs.append(b.tr.step_distributed(step, ctl, refresh=probe, reduce_gradient=reduce, batch_time=1.0))
+        torch.cuda.synchronize()
+        assert abs(float(b.tr.gradnorm.item()) - float(a.tr.gradnorm.item())) <= 1e-4 * float(a.tr.gradnorm.item())
+        b.check_adam(b.tr.lib.grad_buffer().cpu().numpy().astype(np.float64), pre, what=f"[step {step}]")
+    assert [l["boundary"] for l in logs] == [1 if r % 3 == 0 else 0 for r in range(10)]
+    assert probe.calls == [l["r"] // 3 for l in logs if l["boundary"] and l["sync"]] and 0 in probe.calls
+    assert len(set(seen)) == 1 and len(seen) == 10
 
 
 # ------------------------------------------------- masked loss (Eq. 12-13)

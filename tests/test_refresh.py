@@ -143,3 +143,94 @@ def test_synchronised_gradient_of_two_half_batches_is_the_full_batch_gradient(or
     assert np.abs(mean - full.grads).max() <= 1e-12 * scale
     assert abs(g - full.gradnorm) <= 1e-12 * full.gradnorm
     assert abs(0.5 * (a.loss + c.loss) - full.loss) <= 1e-13
+
+
+def test_two_rank_refresh_flag_and_gradient_sum_over_gloo():
+    """The host side of the exchanges with two CPU processes: split sizes and routing of the all-to-all
+    from each rank's plan, the coordinator's flag, and the gradient all-reduce followed by the apply call.
+    The row movers are replaced by index copies (the kernels are covered on the GPU); the tables after the
+    refresh must equal the oracle's."""
+    import socket
+    import subprocess
+    import sys
+    root = os.path.dirname(HERE)
+    code = r"""
+import os, sys, numpy as np, torch, torch.distributed as dist
+sys.path.insert(0, %r)
+from oracle import refresh as orf, scan as osc
+from paper_2608_16305_b200 import distributed as D
+rank = int(os.environ["RANK"])
+dist.init_process_group("gloo", rank=rank, world_size=2, init_method="tcp://127.0.0.1:" + os.environ["PORT"])
+rng = np.random.default_rng(5)                       # same stream on both ranks
+P, N, E, Bsz, K, d = 2, 80, 400, 20, 4, 6
+src, dst = rng.integers(0, N, E), rng.integers(0, N, E)
+owner = rng.integers(0, P, N)
+Q = (E // Bsz + K - 1) // K
+mem = [rng.standard_normal((N, d)).astype(np.float32) for _ in range(P)]
+lu = [rng.random(N) * 50 for _ in range(P)]
+sets = [[osc.backward_scan(src, dst, owner, p, Bsz, K, q)[2] for p in range(P)] for q in range(Q)]
+cap = max(sum(len(s) for s in sets[q]) for q in range(Q))
+rn, sn = np.zeros((Q, cap), np.int32), np.zeros((Q, cap), np.int32)
+ro, so = np.zeros((Q, P + 1), np.int64), np.zeros((Q, P + 1), np.int64)
+for q in range(Q):
+    plan = orf.refresh_plan(sets[q], owner)
+    r_list = [plan[o][rank] for o in range(P)]
+    s_list = [plan[rank][r] for r in range(P)]
+    ro[q, 1:], so[q, 1:] = np.cumsum([len(x) for x in r_list]), np.cumsum([len(x) for x in s_list])
+    rn[q, :ro[q, -1]], sn[q, :so[q, -1]] = sum(r_list, []), sum(s_list, [])
+plan = D.RefreshPlan.from_lists(torch.from_numpy(rn), ro, torch.from_numpy(sn), so, P, rank)
+
+def pack(memory, last_update, nodes, packed, status):
+    n = nodes.numel()
+    rows = packed[:n * (d + 2)].view(n, d + 2)
+    rows[:, :d] = memory[nodes.long()]
+    rows[:, d:] = last_update[nodes.long()].view(torch.float32).view(n, 2)
+
+def unpack(memory, last_update, nodes, packed, status):
+    n = nodes.numel()
+    rows = packed[:n * (d + 2)].view(n, d + 2)
+    memory[nodes.long()] = rows[:, :d]
+    last_update[nodes.long()] = rows[:, d:].contiguous().view(torch.float64).view(n)
+
+ref = D.BoundaryRefresh(plan, d, pack=pack, unpack=unpack)
+my_mem, my_lu = torch.from_numpy(mem[rank].copy()), torch.from_numpy(lu[rank].copy())
+moved = 0
+for q in range(Q):
+    # the coordinator (rank 0) decides; rank 1's own opinion is overruled
+    s = D.broadcast_decision(q %% 2 if rank == 0 else 1 - q %% 2, torch.device("cpu"))
+    assert s == q %% 2
+    if s:
+        ref.run(q, my_mem, my_lu)
+        mem, lu = orf.boundary_refresh(mem, lu, sets[q], owner)
+    assert np.array_equal(my_mem.numpy(), mem[rank]) and np.array_equal(my_lu.numpy(), lu[rank]), q
+moved = ref.rows_received
+assert moved == sum(len(sets[q][rank]) for q in range(Q) if q %% 2) and moved > 0
+
+class FakeLib:                                          # records what the gradient synchronisation asks of the library
+    def __init__(self):
+        self.g = torch.arange(5, dtype=torch.float32) * (rank + 1)
+        self.applied = None
+    def grad_buffer(self):
+        return self.g
+    def apply_gradient(self, scale, out):
+        self.applied = (scale, self.g.clone())
+lib = FakeLib()
+D.synchronise_gradient(lib, None)
+scale, g = lib.applied
+mean, norm = orf.synchronised_gradient([np.arange(5.0), 2 * np.arange(5.0)])
+assert scale == 0.5 and np.array_equal(g.numpy() * scale, mean.astype(np.float32))
+dist.barrier()
+print("ok", rank)
+""" % root
+    sock = socket.socket()
+    sock.bind(("127.0.0.1", 0))
+    port = sock.getsockname()[1]
+    sock.close()
+    procs = []
+    for r in range(2):
+        env = dict(os.environ, RANK=str(r), PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, "-c", code], env=env, stdout=subprocess.PIPE, stderr=subprocess.PIPE))
+    for p in procs:
+        out, err = p.communicate(timeout=180)
+        assert p.returncode == 0, err.decode()[-3000:]
+        assert b"ok" in out
