@@ -333,6 +333,89 @@ def _run_ours_on_stream(args, rank, world, device, cfg, stream, dw, weights, tr)
     print(json.dumps(out))
 
 
+def run_partitioned(args, rank, world, device):
+    """The multi-worker form of the step, one worker per GPU: worker `rank` of a `world`-way node partition
+    trains on its scanned mixed batches (Algorithm 1, Eq. 5) under the adaptive controller (Algorithm 2), with
+    the boundary cache refresh as an all-to-all of packed rows and the gradient all-reduced before Adam.
+    Throughput counts the original events of the global batches processed (each is some worker's target)."""
+    import torch.distributed as dist
+    from paper_2608_16305_b200 import binding as B
+    from paper_2608_16305_b200 import distributed as D
+    from paper_2608_16305_b200 import trainer as T
+    cfg = wl.CONFIGS[args.workload]
+    stream = wl.make_stream(cfg)
+    efeat = wl.edge_feature_table_torch(cfg, device)
+    K_sync = 6
+    owner = (np.arange(cfg.num_nodes, dtype=np.int64) * 2654435761 % 2 ** 32 % world).astype(np.int32)
+    t0 = time.time()
+    dw = T.PartitionedWorkload(stream, owner, world, rank, K_sync, device=device, efeat=efeat, keep_sync=True)
+    refresh = D.BoundaryRefresh(dw.refresh_plan(), cfg.d)
+    torch.cuda.synchronize()
+    prep_s = time.time() - t0
+    weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed, model=args.model)
+    math_mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST}[args.math]
+    tr = T.Trainer(dw, weights, math_mode=math_mode, model=args.model)
+    tr.lib.set_grad_sync(True)
+    ctl = B.Controller(alpha=0.1, beta=0.1, tau_g=1.6, tau_c=0.5, K=K_sync)
+    nb = len(dw.batches) - 1
+    K, W = args.steps, args.warmup
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)
+    logs = []
+
+    def run_steps(first, count):
+        ms = 0.0
+        for i in range(first, first + count):
+            b = i % nb
+            if b == 0:
+                tr.memory.zero_()
+                tr.last_update.zero_()
+            flush.fill_(i & 0xff)
+            a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            logs.append(tr.step_distributed(b, ctl, refresh=refresh))
+            z.record()
+            z.synchronize()
+            ms += a.elapsed_time(z)
+        return ms
+
+    def barrier():
+        if dist.is_initialized():
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    with torch.cuda.stream(tr.stream):
+        run_steps(0, W)
+        barrier()
+        logs.clear()
+        l0 = tr.lib.kernel_launches()
+        with ClockSampler(torch.cuda.current_device()) as clk:
+            ms = run_steps(W, K)
+        launches = tr.lib.kernel_launches() - l0
+        barrier()
+    ms_max, units = aggregate_over_ranks(ms, K * cfg.batch if rank == 0 else 0, device)
+    if int(refresh.status.item()) or tr.lib.status():
+        raise SystemExit("device status set during the partitioned run")
+    if rank != 0:
+        return
+    print(json.dumps({
+        "metric": METRIC, "value": units / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_max / K, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+        "dtype": "f32" if args.math == "fp32" else "tf32", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: {cfg.num_nodes} nodes, {cfg.num_events} events, batch {cfg.batch} (global), "
+                               f"{world}-way hashed node partition, source-owned targets, K = {K_sync}",
+                   "parallelism": f"{world} partitioned worker(s): scanned mixed batches, boundary refresh (all-to-all of "
+                                  "packed rows), gradient all-reduce, adaptive controller",
+                   "math_mode": args.math, "l2": "512 MB buffer written between timed steps",
+                   "inputs": "resident in HBM", "preprocess_s": round(prep_s, 3)},
+        "e2e": None, "gpu_launches": int(launches), "clocks": clk.summary(),
+        "worker0": {"mixed_events_per_step": float(np.diff(dw.mb_off).mean()), "targets_per_step": float(np.diff(dw.tgt_off).mean()),
+                    "boundaries": sum(l["boundary"] for l in logs), "refreshes": sum(1 for l in logs if l["boundary"] and l["sync"]),
+                    "rows_received": refresh.rows_received, "rows_sent": refresh.rows_sent,
+                    "heavy_batches": sum(l["heavy"] for l in logs)},
+        "loss_last": float(tr.loss.item()),
+    }))
+
+
 def preprocess_pass(cfg, stream, dw, device, P=8, K=6, reps=5):
     """Backward dependency scan for all P workers and windows, then worker 0's mixed batches; the oracle's
     scan is timed on a bounded number of (worker, window) pairs."""
@@ -373,12 +456,91 @@ def preprocess_pass(cfg, stream, dw, device, P=8, K=6, reps=5):
         if time.perf_counter() - t0 > 5.0:
             break
     cpu_s = time.perf_counter() - t0
-    return {"workers": P, "K": K, "windows": Q, "scan_ms": ms_scan, "build_mixed_ms": ms_build,
+    refresh = refresh_pass(cfg, dw, device, owner, P, K, Q, reps)
+    return {"workers": P, "K": K, "windows": Q, "scan_ms": ms_scan, "build_mixed_ms": ms_build, "refresh": refresh,
             "scan_events_per_s": P * E / (ms_scan * 1e-3), "aux_per_target": aux_frac,
             "n_sync_mean": float(n_sync.float().mean().item()),
             "cpu_oracle_events_per_s": pairs * K * cfg.batch / cpu_s, "cpu_oracle_sample": f"{pairs} (worker, window) scans",
             "how": "tgnn_backward_scan over all workers and windows (hash partition), tgnn_build_mixed for worker 0; "
                    "CUDA events, median of %d" % reps}
+
+
+def refresh_pass(cfg, dw, device, owner, P, K, Q, reps):
+    """The boundary refresh's device work: worker 0's exchange plan for every window, and the two row movers,
+    on a window of this workload and on a table larger than L2 (where their HBM rate means something)."""
+    from paper_2608_16305_b200 import binding as B
+    from paper_2608_16305_b200 import distributed as D
+    N, d = cfg.num_nodes, cfg.d
+    E = cfg.num_events
+    role = torch.empty((P, E), dtype=torch.uint8, device=device)
+    n_sync = torch.empty((P, Q), dtype=torch.int32, device=device)
+    sync = torch.empty((P, Q, N), dtype=torch.uint8, device=device)
+    scratch = torch.empty(B.backward_scan_scratch(E, cfg.batch, K, N, P), dtype=torch.int32, device=device)
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    B.backward_scan(dw.src, dw.dst, cfg.batch, K, owner, P, role, n_sync, sync, scratch, status)
+    n_sync_h = n_sync.cpu().numpy()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    plan, ms_plan = None, []
+    for _ in range(reps + 2):
+        a, z = ev(), ev()
+        a.record()
+        plan = D.RefreshPlan(sync, owner, n_sync_h, P, 0)
+        z.record()
+        torch.cuda.synchronize()
+        ms_plan.append(a.elapsed_time(z))
+    # a window of this workload: what worker 0 sends and receives at its busiest boundary
+    q = int(np.argmax(plan.recv_off[:, -1] + plan.send_off[:, -1]))
+    mem = torch.randn((N, d), dtype=torch.float32, device=device)
+    lu = torch.rand(N, dtype=torch.float64, device=device)
+    ref = D.BoundaryRefresh(plan, d)
+    # a table larger than L2: 2 M rows, a random three quarters of them moved
+    Nbig = 2_000_000
+    big = torch.randn((Nbig, d), dtype=torch.float32, device=device)
+    big_t = torch.rand(Nbig, dtype=torch.float64, device=device)
+    nodes = torch.randperm(Nbig, device=device)[:Nbig * 3 // 4].to(torch.int32).contiguous()
+    packed = torch.empty(nodes.numel() * (d + 2), dtype=torch.float32, device=device)
+    st = torch.zeros(1, dtype=torch.int32, device=device)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=device)
+    t = {"pack_window": [], "unpack_window": [], "pack_big": [], "unpack_big": []}
+    for i in range(reps + 2):
+        flush.fill_(i)
+        e = [ev() for _ in range(3)]
+        e[0].record()
+        ref.pack(q, mem, lu)
+        e[1].record()
+        ref.unpack(q, mem, lu)
+        e[2].record()
+        torch.cuda.synchronize()
+        t["pack_window"].append(e[0].elapsed_time(e[1]))
+        t["unpack_window"].append(e[1].elapsed_time(e[2]))
+        flush.fill_(i + 1)
+        e = [ev() for _ in range(2)]
+        e[0].record()
+        B.pack_rows(big, big_t, nodes, packed, st)
+        e[1].record()
+        torch.cuda.synchronize()
+        t["pack_big"].append(e[0].elapsed_time(e[1]))
+        flush.fill_(i + 2)
+        e = [ev() for _ in range(2)]
+        e[0].record()
+        B.unpack_rows(big, big_t, nodes, packed, st)
+        e[1].record()
+        torch.cuda.synchronize()
+        t["unpack_big"].append(e[0].elapsed_time(e[1]))
+    med = {k: float(np.median(v[2:])) for k, v in t.items()}
+    row_bytes = 2 * (4 * d + 8) + 4               # state read + state written + the node id
+    big_bytes = nodes.numel() * row_bytes
+    peaks = measured_peaks()
+    assert int(st.item()) == 0 and int(ref.status.item()) == 0
+    return {"plan_ms_all_windows": float(np.median(ms_plan[2:])), "window": q,
+            "window_rows_sent": int(plan.send_off[q, -1]), "window_rows_received": int(plan.recv_off[q, -1]),
+            "pack_window_us": med["pack_window"] * 1e3, "unpack_window_us": med["unpack_window"] * 1e3,
+            "bytes_per_row": row_bytes, "big_rows": int(nodes.numel()),
+            "pack_big_gbs": big_bytes / (med["pack_big"] * 1e-3) / 1e9, "unpack_big_gbs": big_bytes / (med["unpack_big"] * 1e-3) / 1e9,
+            "hbm_peak_gbs": peaks["hbm_gbs"], "pack_big_frac": big_bytes / (med["pack_big"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "unpack_big_frac": big_bytes / (med["unpack_big"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "how": "tgnn_refresh_plan for worker 0 over all windows; tgnn_pack_rows / tgnn_unpack_rows on worker 0's busiest "
+                   "window and on 1.5 M random rows of a 2 M-row table (L2 flushed before each), CUDA events, median"}
 
 
 def cpu_baseline(cfg, stream, weights, budget_s=20.0, steps=None, model="tgn"):
@@ -479,6 +641,9 @@ def main():
     ap.add_argument("--embed-aux", action="store_true",
                     help="embed and score every event of the mixed batch (auxiliary events under loss weight 0) "
                          "instead of the target events only: the costing in which replay events pay the forward pass")
+    ap.add_argument("--partitioned", action="store_true",
+                    help="run the multi-worker form instead of independent replicas: one node-partitioned worker per "
+                         "GPU with boundary refresh and gradient all-reduce (strong scaling over the same stream)")
     ap.add_argument("--no-graph", action="store_true", help="launch kernel by kernel instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -492,12 +657,13 @@ def main():
         raise SystemExit("bench.py needs a CUDA device (no CPU fallback); use --impl reference for the CPU oracle")
     torch.cuda.set_device(local)
     device = torch.device("cuda", local)
-    if world > 1:
+    group = world > 1 or (args.partitioned and "RANK" in os.environ)     # a launcher's single rank also gets its group
+    if group:
         torch.distributed.init_process_group("nccl", device_id=device)
     try:
-        run_ours(args, rank, world, device)
+        (run_partitioned if args.partitioned else run_ours)(args, rank, world, device)
     finally:
-        if world > 1:
+        if group:
             torch.distributed.destroy_process_group()
 
 

@@ -8,8 +8,8 @@
 //   * packing the rows to send into one contiguous buffer, and writing received rows into the table.
 // A packed row is d + 2 floats: the memory row, then the two halves of the fp64 time.
 //
-// Both row kernels move 2 x (4 d + 8) bytes per row and nothing else: they are bound by HBM (and, for
-// the gather side, by the row-granular access pattern: one 4d-byte segment per node).
+// Both row kernels move 2 x (4 d + 8) bytes per row and nothing else: they are bound by HBM (and by the
+// row-granular access pattern on the table side: one 4d-byte segment per node, wherever it lies).
 #include <cstdarg>
 #include <cstdio>
 
@@ -87,47 +87,116 @@ __global__ void __launch_bounds__(1024) refresh_plan_kernel(const uint8_t* __res
   }
 }
 
-// One warp per row; lanes move 8-byte pieces (a packed row starts on an 8-byte boundary: d is even).
+// A warp moves ROWS rows at a time in 8-byte pieces (a packed row starts on an 8-byte boundary: d is
+// even): all pieces of all its rows are loaded before the first is stored, so that ROWS x J independent
+// loads per lane are in flight.  J = ceil((d / 2 + 1) / 32) pieces per lane and row; piece d / 2 is the time.
+constexpr int ROWS = 4;
+
+template <int J>
 __global__ void __launch_bounds__(256) pack_rows_kernel(const float* __restrict__ memory, const double* __restrict__ last_update,
                                                         int64_t N, int d, const int32_t* __restrict__ nodes, int n,
                                                         float* __restrict__ packed, int32_t* status) {
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int row0 = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * ROWS;
   const int lane = threadIdx.x & 31;
-  if (row >= n) return;
-  const int node = nodes[row];
-  float2* dst = reinterpret_cast<float2*>(packed + (int64_t)row * (d + 2));
-  if (node < 0 || node >= N) {
-    if (lane == 0) atomicMax(status, 4);
-    for (int j = lane; j < d / 2 + 1; j += 32) dst[j] = make_float2(0.f, 0.f);
-    return;
+  if (row0 >= n) return;
+  const int h = d >> 1;
+  int my = (lane < ROWS && row0 + lane < n) ? nodes[row0 + lane] : -1;
+  if (lane < ROWS && row0 + lane < n && (my < 0 || my >= N)) {
+    atomicMax(status, 4);
+    my = -1;
   }
-  const float2* src = reinterpret_cast<const float2*>(memory + (int64_t)node * d);
-  for (int j = lane; j < d / 2; j += 32) dst[j] = src[j];
-  if (lane == 0) {
-    const long long bits = __double_as_longlong(last_update[node]);
-    dst[d / 2] = make_float2(__int_as_float((int)(bits & 0xffffffffll)), __int_as_float((int)(bits >> 32)));
+  float2 v[ROWS][J];
+#pragma unroll
+  for (int r = 0; r < ROWS; ++r) {
+    const int node = __shfl_sync(FULL, my, r);
+    const float2* src = reinterpret_cast<const float2*>(memory + (int64_t)(node < 0 ? 0 : node) * d);
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+      const int c = lane + 32 * j;
+      v[r][j] = make_float2(0.f, 0.f);
+      if (node >= 0) {
+        if (c < h) {
+          v[r][j] = src[c];
+        } else if (c == h) {
+          const long long bits = __double_as_longlong(last_update[node]);
+          v[r][j] = make_float2(__int_as_float((int)(bits & 0xffffffffll)), __int_as_float((int)(bits >> 32)));
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < ROWS; ++r) {
+    if (row0 + r >= n) break;
+    float2* dst = reinterpret_cast<float2*>(packed + (int64_t)(row0 + r) * (d + 2));
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+      const int c = lane + 32 * j;
+      if (c <= h) dst[c] = v[r][j];      // an out-of-range node id packs as zeros
+    }
   }
 }
 
+template <int J>
 __global__ void __launch_bounds__(256) unpack_rows_kernel(float* __restrict__ memory, double* __restrict__ last_update,
                                                           int64_t N, int d, const int32_t* __restrict__ nodes, int n,
                                                           const float* __restrict__ packed, int32_t* status) {
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int row0 = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * ROWS;
   const int lane = threadIdx.x & 31;
-  if (row >= n) return;
-  const int node = nodes[row];
-  if (node < 0 || node >= N) {
-    if (lane == 0) atomicMax(status, 4);
-    return;
+  if (row0 >= n) return;
+  const int h = d >> 1;
+  int my = (lane < ROWS && row0 + lane < n) ? nodes[row0 + lane] : -1;
+  if (lane < ROWS && row0 + lane < n && (my < 0 || my >= N)) {
+    atomicMax(status, 4);
+    my = -1;
   }
-  const float2* src = reinterpret_cast<const float2*>(packed + (int64_t)row * (d + 2));
-  float2* dst = reinterpret_cast<float2*>(memory + (int64_t)node * d);
-  for (int j = lane; j < d / 2; j += 32) dst[j] = src[j];
-  if (lane == 0) {
-    const float2 t = src[d / 2];
-    const long long bits = ((long long)__float_as_int(t.y) << 32) | (unsigned int)__float_as_int(t.x);
-    last_update[node] = __longlong_as_double(bits);
+  float2 v[ROWS][J];
+#pragma unroll
+  for (int r = 0; r < ROWS; ++r) {
+    const float2* src = reinterpret_cast<const float2*>(packed + (int64_t)(row0 + r) * (d + 2));
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+      const int c = lane + 32 * j;
+      v[r][j] = (row0 + r < n && c <= h) ? src[c] : make_float2(0.f, 0.f);
+    }
   }
+#pragma unroll
+  for (int r = 0; r < ROWS; ++r) {
+    const int node = __shfl_sync(FULL, my, r);
+    if (node < 0) continue;             // beyond n, or an id outside the table: not written
+    float2* dst = reinterpret_cast<float2*>(memory + (int64_t)node * d);
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+      const int c = lane + 32 * j;
+      if (c < h) {
+        dst[c] = v[r][j];
+      } else if (c == h) {
+        const long long bits = ((long long)__float_as_int(v[r][j].y) << 32) | (unsigned int)__float_as_int(v[r][j].x);
+        last_update[node] = __longlong_as_double(bits);
+      }
+    }
+  }
+}
+
+constexpr int kMaxD = 32 * 2 * 8 - 2;   // J <= 8 pieces per lane
+
+template <bool PACK>
+cudaError_t launch_rows(const float* memory_in, float* memory_out, const double* lu_in, double* lu_out, int64_t N, int d,
+                        const int32_t* nodes, int n, const float* packed_in, float* packed_out, int32_t* status,
+                        cudaStream_t s) {
+  const int J = (d / 2 + 1 + 31) / 32;
+  const int grid = (n + 8 * ROWS - 1) / (8 * ROWS);
+#define TGNN_ROWS_CASE(JJ)                                                                                              \
+  case JJ:                                                                                                              \
+    if (PACK) pack_rows_kernel<JJ><<<grid, 256, 0, s>>>(memory_in, lu_in, N, d, nodes, n, packed_out, status);         \
+    else unpack_rows_kernel<JJ><<<grid, 256, 0, s>>>(memory_out, lu_out, N, d, nodes, n, packed_in, status);           \
+    break;
+  switch (J) {
+    TGNN_ROWS_CASE(1) TGNN_ROWS_CASE(2) TGNN_ROWS_CASE(3) TGNN_ROWS_CASE(4) TGNN_ROWS_CASE(5) TGNN_ROWS_CASE(6)
+    TGNN_ROWS_CASE(7) TGNN_ROWS_CASE(8)
+    default: return cudaErrorInvalidValue;
+  }
+#undef TGNN_ROWS_CASE
+  return cudaGetLastError();
 }
 
 }  // namespace
@@ -156,7 +225,8 @@ int tgnn_refresh_plan(const uint8_t* sync, const int32_t* owner, int64_t num_nod
 
 static int check_rows(const char* who, const void* memory, const void* last_update, int64_t num_nodes, int d,
                       const void* nodes, int n, const void* packed, const void* status, char* err_host, int64_t err_size) {
-  if (num_nodes < 1 || d < 2 || (d & 1) || n < 0) return fail(err_host, err_size, TGNN_EINVAL, "%s: size out of range (d must be even)", who);
+  if (num_nodes < 1 || d < 2 || (d & 1) || d > kMaxD || n < 0)
+    return fail(err_host, err_size, TGNN_EINVAL, "%s: size out of range (d must be even and at most %d)", who, kMaxD);
   if (!status || !memory || !last_update || (n > 0 && (!nodes || !packed)))
     return fail(err_host, err_size, TGNN_EINVAL, "%s: null pointer", who);
   if ((((uintptr_t)memory | (uintptr_t)packed) & 7) != 0)
@@ -169,8 +239,8 @@ int tgnn_pack_rows(const float* memory, const double* last_update, int64_t num_n
   const int rc = check_rows("tgnn_pack_rows", memory, last_update, num_nodes, d, nodes, n, packed, status, err_host, err_size);
   if (rc) return rc;
   if (n == 0) return TGNN_OK;
-  pack_rows_kernel<<<(n + 7) / 8, 256, 0, (cudaStream_t)stream>>>(memory, last_update, num_nodes, d, nodes, n, packed, status);
-  const cudaError_t e = cudaGetLastError();
+  const cudaError_t e = launch_rows<true>(memory, nullptr, last_update, nullptr, num_nodes, d, nodes, n, nullptr, packed, status,
+                                          (cudaStream_t)stream);
   if (e != cudaSuccess) return fail(err_host, err_size, TGNN_ECUDA, "tgnn_pack_rows: %s", cudaGetErrorString(e));
   return TGNN_OK;
 }
@@ -180,8 +250,8 @@ int tgnn_unpack_rows(float* memory, double* last_update, int64_t num_nodes, int 
   const int rc = check_rows("tgnn_unpack_rows", memory, last_update, num_nodes, d, nodes, n, packed, status, err_host, err_size);
   if (rc) return rc;
   if (n == 0) return TGNN_OK;
-  unpack_rows_kernel<<<(n + 7) / 8, 256, 0, (cudaStream_t)stream>>>(memory, last_update, num_nodes, d, nodes, n, packed, status);
-  const cudaError_t e = cudaGetLastError();
+  const cudaError_t e = launch_rows<false>(nullptr, memory, nullptr, last_update, num_nodes, d, nodes, n, packed, nullptr, status,
+                                           (cudaStream_t)stream);
   if (e != cudaSuccess) return fail(err_host, err_size, TGNN_ECUDA, "tgnn_unpack_rows: %s", cudaGetErrorString(e));
   return TGNN_OK;
 }
