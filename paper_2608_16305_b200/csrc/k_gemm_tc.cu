@@ -134,14 +134,27 @@ __device__ __forceinline__ void sts_v4(uint32_t addr, uint32_t a, uint32_t b, ui
 // the integer pipe at full rate (the conversion pipe would bound the producers).
 __device__ __forceinline__ uint32_t to_tf32(float x) { return (__float_as_uint(x) + 0x1000u) & 0xffffe000u; }
 
+// One 16-byte chunk of an operand tile.  Single pass: the values rounded to TF32.  Split: the values as they
+// are in the head copy -- the tensor core reads sign, exponent and the upper 10 mantissa bits of a tf32
+// operand and ignores the 13 bits below, so the head it sees is the value truncated -- and the exact
+// remainder (the part it ignores) in the tail copy, of which it again sees the upper bits.  Head + tail then
+// carry 21 mantissa bits; truncation's bias is in the tail's dropped bits only (2^-21 relative).
+__device__ __forceinline__ uint32_t tf32_remainder(float x) {
+  return __float_as_uint(x - __uint_as_float(__float_as_uint(x) & 0xffffe000u));
+}
 template <bool PRECISE>
 __device__ __forceinline__ void store_chunk(uint32_t addr, uint32_t tail_offset, const float4& v) {
-  const uint32_t h0 = to_tf32(v.x), h1 = to_tf32(v.y), h2 = to_tf32(v.z), h3 = to_tf32(v.w);
-  sts_v4(addr, h0, h1, h2, h3);
   if (PRECISE) {
-    sts_v4(addr + tail_offset, to_tf32(v.x - __uint_as_float(h0)), to_tf32(v.y - __uint_as_float(h1)),
-           to_tf32(v.z - __uint_as_float(h2)), to_tf32(v.w - __uint_as_float(h3)));
+    sts_v4(addr, __float_as_uint(v.x), __float_as_uint(v.y), __float_as_uint(v.z), __float_as_uint(v.w));
+    sts_v4(addr + tail_offset, tf32_remainder(v.x), tf32_remainder(v.y), tf32_remainder(v.z), tf32_remainder(v.w));
+  } else {
+    sts_v4(addr, to_tf32(v.x), to_tf32(v.y), to_tf32(v.z), to_tf32(v.w));
   }
+}
+
+// A chunk that a TMA copy left in the head tile as plain fp32 stays there as the head; only its tail is written.
+__device__ __forceinline__ void store_tail_of_raw(uint32_t tail_addr, const float4& v) {
+  sts_v4(tail_addr, tf32_remainder(v.x), tf32_remainder(v.y), tf32_remainder(v.z), tf32_remainder(v.w));
 }
 
 // 64-bit shared-memory matrix descriptor.  layout: 2 = 128-byte swizzle on 16-byte chunks (K-major
@@ -428,7 +441,8 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE, TMA>::THREADS, 1) gemm_tf32
                                 (((cm & 7) ^ ((kk & 3) << 1)) << 4);
           float4 x;
           asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w) : "r"(addr) : "memory");
-          store_chunk<PRECISE>(addr, C_::A_BYTES, x);
+          if (PRECISE) store_tail_of_raw(addr + C_::A_BYTES, x);
+          else store_chunk<PRECISE>(addr, C_::A_BYTES, x);
           if (want_rowsum) { rs.x += x.x; rs.y += x.y; rs.z += x.z; rs.w += x.w; }  // cm == t % 32 for every q
         }
         // B: 32 rows x b_rows values
@@ -438,7 +452,8 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE, TMA>::THREADS, 1) gemm_tf32
                                 (((cm & 7) ^ ((kk & 3) << 1)) << 4);
           float4 x;
           asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w) : "r"(addr) : "memory");
-          store_chunk<PRECISE>(addr, C_::B_BYTES, x);
+          if (PRECISE) store_tail_of_raw(addr + C_::B_BYTES, x);
+          else store_chunk<PRECISE>(addr, C_::B_BYTES, x);
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         mbar_arrive(smem_u32(&s_full[s]));
@@ -489,7 +504,15 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE, TMA>::THREADS, 1) gemm_tf32
           }
           ma = 0xffffffffu;
         }
-        store_regs<BM, PRECISE>(va, ma, a_tile, C_::A_BYTES, MAJOR_K, BM, t, nullptr);
+        if (tile && PRECISE) {  // the landed values stay in place as heads
+#pragma unroll
+          for (int q = 0; q < BM * 8 / GROUP; ++q) {
+            const int idx = t + q * GROUP, r = idx >> 3, c = idx & 7;
+            store_tail_of_raw(a_tile + C_::A_BYTES + r * 128 + ((c ^ (r & 7)) << 4), va[q]);
+          }
+        } else {
+          store_regs<BM, PRECISE>(va, ma, a_tile, C_::A_BYTES, MAJOR_K, BM, t, nullptr);
+        }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         mbar_arrive(smem_u32(&s_full[s]));
       }

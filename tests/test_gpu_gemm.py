@@ -113,3 +113,41 @@ def test_transposed_products_by_tiles(M, N, K, pad):
         assert np.abs(C.cpu().numpy() - (ref + C0)).max() <= 1e-4 * scale
         assert np.abs(rs.cpu().numpy() - A.astype(np.float64).sum(1)).max() <= 1e-4 * max(np.abs(A).sum(1).max(), 1.0)
     lib.close()
+
+
+@pytest.mark.parametrize("layout", [("mn", "mn"), ("k", "k"), ("k", "mn")])
+@pytest.mark.parametrize("low_bits", [0x1fff, 0x1000, 0x0fff])
+def test_operand_split_keeps_the_low_mantissa_bits(layout, low_bits):
+    """Positive operands whose 13 low mantissa bits are all set (or exactly half / just under half an ulp of
+    the 10-bit head): any mismatch between how the head is formed and what the tensor core takes as the head
+    -- rounding on one side, truncation on the other -- shifts every product by up to 2^-10 in the same
+    direction, a relative error near 1e-3 on these all-positive sums.  The split product must stay near the
+    fp32 level instead (the bound leaves room for the accumulator's own rounding over the 96 accumulation
+    steps of K = 256, which on all-positive sums adds up to a few 1e-6)."""
+    from paper_2608_16305_b200 import binding as B
+    M, N, K = 128, 160, 256
+    rng = np.random.default_rng(low_bits)
+    lib = B.Tgnn(B.make_config(100, 32, 16, 10, 2, math_mode=B.TGNN_MATH_TF32))
+
+    def worst(shape):
+        x = (1.0 + rng.random(shape)).astype(np.float32)
+        return ((x.view(np.uint32) & np.uint32(0xffffe000)) | np.uint32(low_bits)).view(np.float32)
+    A, Bm = worst((M, K)), worst((K, N))
+    la, lb = layout
+    if la == "k":
+        A_dev, sa = torch.from_numpy(A).cuda(), (K, 1)
+    else:
+        A_dev, sa = torch.from_numpy(np.ascontiguousarray(A.T)).cuda(), (1, M)
+    if lb == "k":
+        B_dev, sb = torch.from_numpy(np.ascontiguousarray(Bm.T)).cuda(), (1, K)
+    else:
+        B_dev, sb = torch.from_numpy(Bm).cuda(), (N, 1)
+    ref = A.astype(np.float64) @ Bm.astype(np.float64)
+    for acc, split in ((False, 1), (True, 4)):
+        C = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+        lib.debug_gemm(A_dev, *sa, B_dev, *sb, C, N, M, N, K, accumulate=acc, split_k=split, precise=True)
+        torch.cuda.synchronize()
+        assert lib.status() == 0
+        err = np.abs(C.cpu().numpy() - ref).max() / ref.max()
+        assert err <= 2e-5, (layout, hex(low_bits), acc, err)
+    lib.close()
