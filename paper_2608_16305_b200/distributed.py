@@ -82,9 +82,9 @@ class BoundaryRefresh:
     def exchange(self, q: int) -> None:
         """Phase 2: one all-to-all; segment r of send_buf goes to worker r, segment o of recv_buf comes from o."""
         pl, w = self.plan, self.d + 2
-        if pl.P == 1:
-            return                                      # a single worker owns every node
         sc, rc = pl.send_counts(q), pl.recv_counts(q)
+        if pl.P == 1 and sum(sc) == 0 and sum(rc) == 0:
+            return                                      # a single worker owns every node: nothing to move
         dist.all_to_all_single(self.recv_buf[:sum(rc) * w], self.send_buf[:sum(sc) * w],
                                output_split_sizes=[c * w for c in rc], input_split_sizes=[c * w for c in sc],
                                group=self.group)

@@ -210,3 +210,68 @@ def test_refresh_of_emulated_workers_matches_oracle(B):
             mem[me] = mem[me] + np.float32(0.25) * (me + 1)
             mem_dev[me] += 0.25 * (me + 1)
     assert moved > 0
+
+
+def test_nccl_single_rank_moves_rows_and_reduces_the_gradient_buffer():
+    """The collectives of the multi-worker form on a real NCCL communicator (one rank: the only size this
+    machine offers): the all-to-all of packed rows between the library's pack and unpack kernels, the flag
+    broadcast, and an all-reduce directly on the context's gradient buffer followed by the apply call."""
+    import os
+    import socket
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = r"""
+import os, sys, numpy as np, torch, torch.distributed as dist
+sys.path.insert(0, %r)
+from paper_2608_16305_b200 import binding as B, distributed as D, trainer as T, workload as wl
+torch.cuda.set_device(0)
+dist.init_process_group("nccl", rank=0, world_size=1, init_method="tcp://127.0.0.1:" + os.environ["PORT"],
+                        device_id=torch.device("cuda", 0))
+N, d, n = 5000, 100, 1200
+rng = np.random.default_rng(0)
+mem = torch.from_numpy(rng.standard_normal((N, d)).astype(np.float32)).cuda()
+lu = torch.from_numpy(rng.random(N) * 1e5).cuda()
+perm = rng.permutation(N)
+src_nodes, dst_nodes = perm[:n].astype(np.int32), perm[n:2 * n].astype(np.int32)
+# a one-worker plan that sends n rows to itself: rows of src_nodes arrive as the new state of dst_nodes
+plan = D.RefreshPlan.from_lists(torch.from_numpy(dst_nodes[None]).cuda(), np.array([[0, n]]),
+                                torch.from_numpy(src_nodes[None]).cuda(), np.array([[0, n]]), 1, 0)
+ref = D.BoundaryRefresh(plan, d)
+want_m, want_t = mem.clone(), lu.clone()
+want_m[dst_nodes.astype(np.int64)] = mem[src_nodes.astype(np.int64)]
+want_t[dst_nodes.astype(np.int64)] = lu[src_nodes.astype(np.int64)]
+assert D.broadcast_decision(1, torch.device("cuda", 0)) == 1
+ref.run(0, mem, lu)
+torch.cuda.synchronize()
+assert int(ref.status.item()) == 0 and ref.rows_sent == n and ref.rows_received == n
+assert torch.equal(mem, want_m) and torch.equal(lu, want_t)
+# gradient buffer: a deferred step, an all-reduce on the library's own memory, then the apply call
+cfg = wl.scaled(wl.CONFIGS["tiny"], num_events=2000)
+dw = T.DeviceWorkload(wl.make_stream(cfg))
+tr = T.Trainer(dw, wl.make_weights(cfg.d, cfg.d_e, cfg.seed, bias_scale=0.1), math_mode=B.TGNN_MATH_TF32)
+tr.lib.set_grad_sync(True)
+with torch.cuda.stream(tr.stream):
+    for b in range(4):
+        tr.step(b)
+        g = tr.lib.grad_buffer()
+        before = g.clone()
+        dist.all_reduce(g, op=dist.ReduceOp.SUM)
+        torch.cuda.current_stream().synchronize()
+        assert torch.equal(g, before) and float(g.abs().max()) > 0
+        tr.lib.apply_gradient(1.0, tr.gradnorm)
+    torch.cuda.synchronize()
+assert int(tr.step_count.item()) == 4 and tr.lib.status() == 0
+want = float(torch.linalg.vector_norm(tr.lib.grad_buffer().double()))
+assert abs(float(tr.gradnorm.item()) - want) <= 1e-6 * want
+dist.destroy_process_group()
+print("ok")
+""" % root
+    sock = socket.socket()
+    sock.bind(("127.0.0.1", 0))
+    port = sock.getsockname()[1]
+    sock.close()
+    env = dict(os.environ, PORT=str(port), NCCL_NVLS_ENABLE="0")
+    p = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, timeout=300)
+    assert p.returncode == 0, p.stderr.decode()[-3000:]
+    assert b"ok" in p.stdout
