@@ -501,6 +501,7 @@ inline int tg_rows_per_block(int rows) {
 __global__ void __launch_bounds__(256) time_grad_kernel(const float* __restrict__ G, int64_t ldg, int col0,
                                                         const float* __restrict__ S, const float* __restrict__ dt,
                                                         int rows, const int32_t* __restrict__ dev_rows, int d,
+                                                        const float* __restrict__ time_w,
                                                         const float* __restrict__ time_b, double* __restrict__ acc,
                                                         int rows_per_block) {
   extern __shared__ double s_part[];  // [8][2][d]
@@ -510,15 +511,22 @@ __global__ void __launch_bounds__(256) time_grad_kernel(const float* __restrict_
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   // a lane owns columns 4 (lane + 32 v) .. + 3, v = 0, 1 (d <= 256): 128-bit loads of G and S (d, ldg and col0 are
   // multiples of 4 and the rows 16-byte aligned)
+  // Sines: saved rows S; or (S null, dt given) recomputed from the row's dt exactly as the forward pass formed
+  // them -- a row with dt < 0 is an empty slot and contributes nothing; or (both null) the constant sin(b) of dt = 0.
   double gw[2][4], gb[2][4];
-  float4 sb[2];
+  float4 sb[2], wv[2], bv[2];
+  const bool recompute = S == nullptr && dt != nullptr;
 #pragma unroll
   for (int v = 0; v < 2; ++v) {
     const int c = 4 * (lane + 32 * v);
 #pragma unroll
     for (int e = 0; e < 4; ++e) { gw[v][e] = 0.0; gb[v][e] = 0.0; }
-    sb[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (S == nullptr && c < d) sb[v] = make_float4(sinf(time_b[c]), sinf(time_b[c + 1]), sinf(time_b[c + 2]), sinf(time_b[c + 3]));
+    sb[v] = wv[v] = bv[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (S == nullptr && c < d) {
+      bv[v] = make_float4(time_b[c], time_b[c + 1], time_b[c + 2], time_b[c + 3]);
+      if (recompute) wv[v] = make_float4(time_w[c], time_w[c + 1], time_w[c + 2], time_w[c + 3]);
+      else sb[v] = make_float4(sinf(bv[v].x), sinf(bv[v].y), sinf(bv[v].z), sinf(bv[v].w));
+    }
   }
   for (int rb = r0 + wid; rb < r1; rb += 32) {  // rows rb, rb + 8, rb + 16, rb + 24: loads first, sums after
     float4 g[4][2], sn[4][2];
@@ -534,6 +542,25 @@ __global__ void __launch_bounds__(256) time_grad_kernel(const float* __restrict_
         const bool ok = in && c < d;
         g[u][v] = ok ? __ldg(reinterpret_cast<const float4*>(G + (int64_t)r * ldg + col0 + c)) : make_float4(0.f, 0.f, 0.f, 0.f);
         sn[u][v] = ok ? (S ? __ldg(reinterpret_cast<const float4*>(S + (int64_t)r * d + c)) : sb[v]) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+    if (recompute) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const bool live = rb + 8 * u < r1 && dtr[u] >= 0.f;
+#pragma unroll
+        for (int v = 0; v < 2; ++v) {
+          const int c = 4 * (lane + 32 * v);
+          float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (live && c < d) {
+            q.x = __sinf(reduce_two_pi(time_arg(wv[v].x, bv[v].x, dtr[u])));
+            q.y = __sinf(reduce_two_pi(time_arg(wv[v].y, bv[v].y, dtr[u])));
+            q.z = __sinf(reduce_two_pi(time_arg(wv[v].z, bv[v].z, dtr[u])));
+            q.w = __sinf(reduce_two_pi(time_arg(wv[v].w, bv[v].w, dtr[u])));
+          }
+          sn[u][v] = q;
+        }
+        if (!live) dtr[u] = 0.f;
       }
     }
 #pragma unroll
@@ -928,7 +955,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
           KernelScope scope__(ctx, "time_grad_x", s);
           const int rpb = tg_rows_per_block(U_cap);
           time_grad_kernel<<<(U_cap + rpb - 1) / rpb, 256, tg_smem, s>>>(w.dXp, d, 0, w.Xsin, w.x_dt, U_cap,
-                                                                         ctx->upd_n_uniq, d, P + L.time_b, w.tg_acc, rpb);
+                                                                         ctx->upd_n_uniq, d, P + L.time_w, P + L.time_b, w.tg_acc, rpb);
         }
         TGNN_LAUNCH_OK(ctx, "time_grad_x");
       }
@@ -970,7 +997,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       KernelScope scope__(ctx, "time_grad_q", sb);
       const int rpb = tg_rows_per_block(R);
       time_grad_kernel<<<(R + rpb - 1) / rpb, 256, tg_smem, sb>>>(w.dzq, 2 * d, d, nullptr, nullptr, R, nullptr, d,
-                                                                  P + L.time_b, w.tg_acc, rpb);
+                                                                  P + L.time_w, P + L.time_b, w.tg_acc, rpb);
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_q");
     cudaStream_t s_tgz = sb;  // where the time-encoder sum over the neighbor rows runs
@@ -984,7 +1011,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     {
       KernelScope scope__(ctx, "time_grad_z", s_tgz);
       const int rpb = tg_rows_per_block(NB);
-      time_grad_kernel<<<(NB + rpb - 1) / rpb, 256, tg_smem, s_tgz>>>(w.dZmp, 2 * d, d, w.Zsin, w.z_dt, NB, nullptr, d,
+      time_grad_kernel<<<(NB + rpb - 1) / rpb, 256, tg_smem, s_tgz>>>(w.dZmp, 2 * d, d, nullptr, w.z_dt, NB, nullptr, d, P + L.time_w,
                                                                       P + L.time_b, w.tg_acc, rpb);
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_z");
@@ -1023,7 +1050,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
         KernelScope scope__(ctx, "time_grad_x", s);
         const int rpb = tg_rows_per_block(U_cap);
         time_grad_kernel<<<(U_cap + rpb - 1) / rpb, 256, tg_smem, s>>>(w.dXp, d, 0, w.Xsin, w.x_dt, U_cap, ctx->upd_n_uniq,
-                                                                       d, P + L.time_b, w.tg_acc, rpb);
+                                                                       d, P + L.time_w, P + L.time_b, w.tg_acc, rpb);
       }
       TGNN_LAUNCH_OK(ctx, "time_grad_x");
     }

@@ -20,8 +20,15 @@ namespace {
 // neighbors and the parameters, so it can run beside the memory update; the memory part has to wait
 // for it.  One warp per row in both.
 //
-// Static part.  Rows [0, n*k): columns [d, ld) of Z (zero row if the slot is empty), Zsin, z_dt.
+// Static part.  Rows [0, n*k): columns [d, ld) of Z (zero row if the slot is empty), z_dt (-1 if empty).
 // Rows [n*k, n*k + n): the Phi(0) half of z_q.
+// A warp takes ZS_ROWS neighbor rows at a time: their slot records first (one lane per row), then the
+// feature loads of all of them, and only then the conversions, the time encodings and the stores -- the
+// dependent chain slot -> event id -> feature row is paid once per ZS_ROWS rows instead of once per row.
+constexpr int ZS_ROWS = 4;
+constexpr int ZS_FEAT = 8;  // 32-bit feature words per lane and row held in registers: two 16-byte chunks of an
+                            // fp32 row (de <= 256) or four bf16 pairs (de <= 256)
+
 __global__ void __launch_bounds__(256) gather_z_static_kernel(const void* __restrict__ efeat, int feat_bf16,
                                                               const float* __restrict__ time_w,
                                                               const float* __restrict__ time_b, int d, int de, int k,
@@ -30,31 +37,98 @@ __global__ void __launch_bounds__(256) gather_z_static_kernel(const void* __rest
                                                               const int32_t* __restrict__ eid,
                                                               const double* __restrict__ ts, int ld,
                                                               float* __restrict__ Z, float* __restrict__ z_dt,
-                                                              float* __restrict__ Zsin, float* __restrict__ Zq) {
+                                                              float* __restrict__ Zq) {
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   const int nb_rows = n * k;
   const int dkv = 2 * d + de;
-  for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < nb_rows + n; r += warps) {
-    if (r < nb_rows) {
+  const int wrow = feat_bf16 ? (de >> 1) : de;          // 32-bit words per feature row
+  // fp32 rows as 16-byte chunks (rows and the destination columns are 16-byte aligned when d and de are
+  // multiples of 4), bf16 rows as 32-bit pairs; anything wider or ragged goes row by row as before
+  const bool vec4 = !feat_bf16 && (de & 3) == 0 && (d & 3) == 0 && (ld & 3) == 0 && de <= 256 &&
+                    ((((uintptr_t)efeat) | ((uintptr_t)Z)) & 15) == 0;
+  const bool pairs = feat_bf16 && wrow <= 128;
+  const bool regs = vec4 || pairs;
+  const int groups = (nb_rows + ZS_ROWS - 1) / ZS_ROWS;
+  for (int gidx = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; gidx < groups; gidx += warps) {
+    const int r0 = gidx * ZS_ROWS;
+    // slot records: lane j < ZS_ROWS reads row r0 + j
+    int my_nbr = -1, my_eid = 0;
+    float my_dt = 0.f;
+    if (lane < ZS_ROWS && r0 + lane < nb_rows) {
+      const int r = r0 + lane;
+      my_nbr = nbr[r];
+      my_eid = eid[r];
+      my_dt = (float)(times[r / k] - ts[r]);
+    }
+    uint32_t f[ZS_ROWS][ZS_FEAT];
+    int v_nbr[ZS_ROWS];
+    float v_dt[ZS_ROWS];
+#pragma unroll
+    for (int j = 0; j < ZS_ROWS; ++j) {
+      v_nbr[j] = __shfl_sync(0xffffffffu, my_nbr, j);
+      v_dt[j] = __shfl_sync(0xffffffffu, my_dt, j);
+      const int e = __shfl_sync(0xffffffffu, my_eid, j);
+      if (regs && v_nbr[j] >= 0) {
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(efeat) + (int64_t)e * wrow;
+        if (vec4) {
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int q = lane + 32 * u;
+            uint4 x = make_uint4(0u, 0u, 0u, 0u);
+            if (q < (wrow >> 2)) x = __ldg(reinterpret_cast<const uint4*>(src) + q);
+            f[j][4 * u] = x.x; f[j][4 * u + 1] = x.y; f[j][4 * u + 2] = x.z; f[j][4 * u + 3] = x.w;
+          }
+        } else {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int q = lane + 32 * u;
+            f[j][u] = q < wrow ? __ldg(src + q) : 0u;
+          }
+        }
+      } else if (!regs && v_nbr[j] >= 0) {
+        warp_copy_feat(Z + (int64_t)(r0 + j) * ld + d, efeat, feat_bf16, e, de, lane);  // very wide rows: as before
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < ZS_ROWS; ++j) {
+      const int r = r0 + j;
+      if (r >= nb_rows) break;
       float* row = Z + (int64_t)r * ld;
-      if (nbr[r] < 0) {
+      if (v_nbr[j] < 0) {
         for (int q = lane; q < ld; q += 32) row[q] = 0.f;  // the memory part too: nobody else writes this row
-        for (int q = lane; q < d; q += 32) Zsin[(int64_t)r * d + q] = 0.f;
-        if (lane == 0) z_dt[r] = 0.f;
+        if (lane == 0) z_dt[r] = -1.f;  // marks the empty slot for the time-encoder gradient (a real dt is >= 0)
         continue;
       }
-      const float dtf = (float)(times[r / k] - ts[r]);
-      warp_copy_feat(row + d, efeat, feat_bf16, eid[r], de, lane);
+      if (vec4) {
+        uint4* dst = reinterpret_cast<uint4*>(row + d);
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int q = lane + 32 * u;
+          if (q < (wrow >> 2)) dst[q] = make_uint4(f[j][4 * u], f[j][4 * u + 1], f[j][4 * u + 2], f[j][4 * u + 3]);
+        }
+      } else if (pairs) {
+        float* dst = row + d;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int q = lane + 32 * u;
+          if (q < wrow) {
+            dst[2 * q] = __uint_as_float(f[j][u] << 16);
+            dst[2 * q + 1] = __uint_as_float(f[j][u] & 0xffff0000u);
+          }
+        }
+      }
+      const float dtf = v_dt[j];
       float* phi = row + d + de;
-      for (int q = lane; q < d; q += 32) time_encode_sc(time_w[q], time_b[q], dtf, &phi[q], &Zsin[(int64_t)r * d + q]);
+      // the sines the backward pass needs are recomputed there from z_dt (cheaper than 4d bytes out and in again)
+      for (int q = lane; q < d; q += 32) phi[q] = time_encode(time_w[q], time_b[q], dtf);
       for (int q = dkv + lane; q < ld; q += 32) row[q] = 0.f;
       if (lane == 0) z_dt[r] = dtf;
-    } else {
-      const int i = r - nb_rows;
-      for (int q = lane; q < d; q += 32) Zq[(int64_t)i * 2 * d + d + q] = time_encode(time_w[q], time_b[q], 0.f);
     }
   }
+  // the Phi(0) half of z_q
+  for (int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps)
+    for (int q = lane; q < d; q += 32) Zq[(int64_t)i * 2 * d + d + q] = time_encode(time_w[q], time_b[q], 0.f);
 }
 
 // Memory part.  Rows [0, n*k): columns [0, d) of Z for the valid slots.  Rows [n*k, n*k + n): the
@@ -170,12 +244,11 @@ int launch_embed_static(tgnn_ctx* ctx, const double* times, int n, const int32_t
   const tgnn_config& c = ctx->cfg;
   const ParamLayout& L = ctx->L;
   Workspace& w = ctx->ws;
-  const int rows = n * c.k + n;
   {
     KernelScope scope__(ctx, "gather_z_static", s);
-    gather_z_static_kernel<<<(rows + 7) / 8, 256, 0, s>>>(ctx->efeat, c.feat_dtype == TGNN_BF16, ctx->params + L.time_w,
+    gather_z_static_kernel<<<(n * c.k / ZS_ROWS + n + 7) / 8 + 1, 256, 0, s>>>(ctx->efeat, c.feat_dtype == TGNN_BF16, ctx->params + L.time_w,
                                                           ctx->params + L.time_b, c.d, c.d_e, c.k, times, n, nbr, eid, ts,
-                                                          ctx->ld_kv, w.Z, w.z_dt, w.Zsin, w.Zq);
+                                                          ctx->ld_kv, w.Z, w.z_dt, w.Zq);
   }
   TGNN_LAUNCH_OK(ctx, "gather_z_static");
   return TGNN_OK;

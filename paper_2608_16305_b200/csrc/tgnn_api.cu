@@ -124,7 +124,6 @@ size_t carve(tgnn_ctx* ctx, char* base) {
   cv.take(w.g_r, U * d); cv.take(w.g_z, U * d); cv.take(w.g_n, U * d); cv.take(w.g_hn, U * d);
   cv.take(w.Z, NB * ctx->ld_kv);
   cv.take(w.z_dt, NB);
-  cv.take(w.Zsin, NB * d);
   cv.take(w.KV, NB * 2 * d);
   cv.take(w.Zq, R * 2 * d);
   cv.take(w.Q, R * d);

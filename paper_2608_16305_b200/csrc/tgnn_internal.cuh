@@ -57,7 +57,6 @@ struct Workspace {
   // step (5) activations
   float* Z;      // [NB_cap, ld_kv]
   float* z_dt;   // [NB_cap]
-  float* Zsin;   // [NB_cap, d] sin of the time-encoding arguments of Z (zero for empty slots)
   float* KV;     // [NB_cap, 2d]  (K | V)
   float* Zq;     // [R_cap, 2d]
   float* Q;      // [R_cap, d]
