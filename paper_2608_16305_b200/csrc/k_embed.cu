@@ -22,14 +22,14 @@ namespace {
 //
 // Static part.  Rows [0, n*k): columns [d, ld) of Z (zero row if the slot is empty), z_dt (-1 if empty).
 // Rows [n*k, n*k + n): the Phi(0) half of z_q.
-// A warp takes ZS_ROWS neighbor rows at a time: their slot records first (one lane per row), then the
+// A warp takes ZS_ROWS neighbor rows at a time (registers kept to 80 so that three blocks fit an SM): their slot records first (one lane per row), then the
 // feature loads of all of them, and only then the conversions, the time encodings and the stores -- the
 // dependent chain slot -> event id -> feature row is paid once per ZS_ROWS rows instead of once per row.
-constexpr int ZS_ROWS = 4;
+constexpr int ZS_ROWS = 2;
 constexpr int ZS_FEAT = 8;  // 32-bit feature words per lane and row held in registers: two 16-byte chunks of an
                             // fp32 row (de <= 256) or four bf16 pairs (de <= 256)
 
-__global__ void __launch_bounds__(256) gather_z_static_kernel(const void* __restrict__ efeat, int feat_bf16,
+__global__ void __launch_bounds__(256, 3) gather_z_static_kernel(const void* __restrict__ efeat, int feat_bf16,
                                                               const float* __restrict__ time_w,
                                                               const float* __restrict__ time_b, int d, int de, int k,
                                                               const double* __restrict__ times, int n,
@@ -50,6 +50,15 @@ __global__ void __launch_bounds__(256) gather_z_static_kernel(const void* __rest
   const bool pairs = feat_bf16 && wrow <= 128;
   const bool regs = vec4 || pairs;
   const int groups = (nb_rows + ZS_ROWS - 1) / ZS_ROWS;
+  // the encoder's frequencies and phases of this lane's columns stay in registers (d <= 128: four per lane)
+  const bool tw_regs = d <= 128;
+  float tw[4], tb[4];
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const int q = lane + 32 * u;
+    tw[u] = (tw_regs && q < d) ? time_w[q] : 0.f;
+    tb[u] = (tw_regs && q < d) ? time_b[q] : 0.f;
+  }
   for (int gidx = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; gidx < groups; gidx += warps) {
     const int r0 = gidx * ZS_ROWS;
     // slot records: lane j < ZS_ROWS reads row r0 + j
@@ -121,7 +130,16 @@ __global__ void __launch_bounds__(256) gather_z_static_kernel(const void* __rest
       const float dtf = v_dt[j];
       float* phi = row + d + de;
       // the sines the backward pass needs are recomputed there from z_dt (cheaper than 4d bytes out and in again)
-      for (int q = lane; q < d; q += 32) phi[q] = time_encode(time_w[q], time_b[q], dtf);
+      if (tw_regs) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {  // four independent chains per lane
+          const int q = lane + 32 * u;
+          if (q < d) phi[q] = time_encode(tw[u], tb[u], dtf);
+        }
+      } else {
+#pragma unroll 4
+        for (int q = lane; q < d; q += 32) phi[q] = time_encode(time_w[q], time_b[q], dtf);
+      }
       for (int q = dkv + lane; q < ld; q += 32) row[q] = 0.f;
       if (lane == 0) z_dt[r] = dtf;
     }
