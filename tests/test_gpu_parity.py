@@ -302,6 +302,38 @@ def _state_for_parts(r, seed=24):
     return mem, lu
 
 
+def test_time_encoding_over_the_whole_argument_range(B):
+    """Phi(dt) from the message builder for time differences from 0 to 5e7 (the large workload's stream
+    length) under the workloads' frequencies 1 .. 1e-9 and random phases: the kernel's own range reduction
+    followed by the hardware cosine against cos of the same fp32 argument in fp64."""
+    c = wl.scaled(TINY, d_e=0)
+    from paper_2608_16305_b200 import trainer
+    dw = trainer.DeviceWorkload(wl.make_stream(c))
+    W = wl.make_weights(c.d, c.d_e, c.seed, bias_scale=0.0)
+    rng = np.random.default_rng(8)
+    W["time_b"] = (rng.random(c.d) * 6.0 - 3.0).astype(np.float32)
+    tr = trainer.Trainer(dw, W)
+    n, calls = dw.max_mixed, 24                     # the context's batch capacity, many batches
+    dt = np.concatenate([[0.0, 1e-3, 3.14159265, 6.2831853, 5e7], rng.random(n * calls - 5) * 10.0 ** rng.uniform(0, 7.7, n * calls - 5)])
+    src = torch.arange(n, dtype=torch.int32, device="cuda") % c.num_nodes
+    dst = (src + 1) % c.num_nodes
+    eid = torch.zeros(n, dtype=torch.int32, device="cuda")
+    tr.last_update.zero_()
+    parts = []
+    for i in range(calls):
+        msg = torch.zeros((2 * n, c.d_msg), dtype=torch.float32, device="cuda")
+        node = torch.zeros(2 * n, dtype=torch.int32, device="cuda")
+        tr.lib.build_messages(src, dst, dev(dt[i * n:(i + 1) * n].astype(np.float64)), eid, None, msg, node)
+        torch.cuda.synchronize()
+        parts.append(msg.cpu().numpy()[:, 2 * c.d + c.d_e:])
+    phi = np.concatenate(parts)
+    # the argument is one fused multiply-add in fp32: w * dt + b rounded once
+    arg = (W["time_w"].astype(np.float64)[None, :] * np.repeat(dt, 2).astype(np.float32).astype(np.float64)[:, None]
+           + W["time_b"].astype(np.float64)[None, :]).astype(np.float32).astype(np.float64)
+    assert np.abs(arg).max() > 4e7
+    assert np.abs(phi - np.cos(arg)).max() <= 2e-6
+
+
 def test_messages_reduction_and_gru_by_parts(tiny_rig):
     r, o, c = tiny_rig, tiny_rig.oracle, TINY
     tr = r.tr
