@@ -13,7 +13,7 @@ with stand-ins; the defaults are the library's kernels and there is no other imp
 """
 from __future__ import annotations
 
-from typing import Callable, List, Optional, Sequence
+from typing import Callable, List, Optional
 
 import numpy as np
 import torch
