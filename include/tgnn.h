@@ -291,6 +291,8 @@ TGNN_API int tgnn_step_mixed_host(tgnn_ctx* ctx, const int32_t* src_host, const 
 
 /* Copies the parameter gradient of the last tgnn_backward_step to grads_out:f32[param_count]. */
 TGNN_API int tgnn_debug_get_grads(tgnn_ctx* ctx, float* grads_out, void* stream);
+/* Copies the embeddings h of the last tgnn_embed call (or of the last whole step) to h_out:f32[n_roots, d]. */
+TGNN_API int tgnn_debug_get_embeddings(tgnn_ctx* ctx, float* h_out, void* stream);
 /* The ReLU branch each unit took in the last tgnn_embed / tgnn_backward_step pair, as bytes:
  * h_gate_out:uint8[n_roots, d] (1 where h > 0), hid_gate_out:uint8[2 n_q, d] (hidden layer of the
  * link-prediction head, positive pairs first).  A parity check needs them because the derivative
@@ -314,6 +316,21 @@ TGNN_API int tgnn_status(tgnn_ctx* ctx, int32_t* status_host, void* stream);
 /* Number of kernels this context has launched since creation (host counter). */
 TGNN_API int64_t tgnn_kernel_launches(const tgnn_ctx* ctx);
 
+/* The split-bf16 projection kernel on its own, for parity tests (sm_100 tensor cores, any math_mode): the
+ * fp32 operands are first split into two bf16 planes each (hi = bf16(x), lo = bf16(x - hi), 16 mantissa bits
+ * together) inside `scratch` (device, 256-byte aligned, >= 2 * 2 * (rows * ceil8(cols)) bytes per operand plus
+ * 256), then C[M,N] (+)= A B (+ bias[n]) (ReLU) runs as three bf16 passes with fp32 accumulation.  Strides as in
+ * tgnn_debug_gemm, with the restriction that either both operands have the contraction index contiguous
+ * (a_cs = 1, b_rs = 1) or both have the other index contiguous (a_rs = 1, b_cs = 1: C = A^T B over matrix rows).
+ * accumulate / split_k as in tgnn_debug_gemm.  debug_withhold > 0 makes the kernel keep that many shared-memory
+ * slots to itself instead of handing them back, and spin_limit > 0 shortens its bounded waits: together they let
+ * a test make a wait run out (the kernel then records TGNN_ETIMEOUT, stores nothing further, frees its tensor
+ * memory and returns; the context stays usable).  Both 0 in normal use. */
+TGNN_API int tgnn_debug_gemm_split(tgnn_ctx* ctx, const float* A, int64_t a_rs, int64_t a_cs, const float* B, int64_t b_rs,
+                                   int64_t b_cs, float* C, int64_t ldc, int M, int N, int K, const float* bias, int relu,
+                                   int accumulate, int split_k, void* scratch, int64_t scratch_bytes, int debug_withhold,
+                                   uint32_t spin_limit, void* stream);
+
 /* ---- for callers that cannot allocate --------------------------------------- */
 
 /* The paper has no counterpart to this entry point; it exists for hosts that
@@ -333,10 +350,15 @@ TGNN_API int64_t tgnn_kernel_launches(const tgnn_ctx* ctx);
  *   borrowed for the call; stream is a cudaStream_t.
  * num_nodes above TGNN_STATIC_MAX_NODES is refused with TGNN_ECAPACITY.  On any
  * failure a message is written to err_host (host buffer of err_size bytes, may
- * be NULL).
+ * be NULL).  A message whose node id is >= num_nodes is skipped on the device
+ * without being used as an index, and the call then reports it by writing -1 to
+ * n_uniq_out (uniq_out / winner_out are undefined in that case); there is no
+ * status word here, so check n_uniq_out.
  * The first call on each device looks up the array's device address
- * (cudaGetSymbolAddress, with that device current) and keeps it; make that first
- * call before any stream capture begins.
+ * (cudaGetSymbolAddress, with that device current) and keeps it for the life of
+ * the process; make that first call before any stream capture begins.  The kept
+ * address does not survive a cudaDeviceReset of that device: a process that
+ * resets a device must not call this entry point on it afterwards.
  * All calls share the one array and it keeps what the last call left, so the
  * kernel clears the entries it uses before it starts; two calls that overlap
  * on the same GPU (different streams, or two threads) race on it and give

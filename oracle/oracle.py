@@ -199,6 +199,7 @@ class StepResult:
     h: np.ndarray
     uniq: np.ndarray
     winner: np.ndarray
+    gate_overrides: tuple = (0, 0)   # units whose ReLU branch a hint decided against the fp64 sign (output layer, head)
 
 
 def loss_and_grads(cfg, params, memory, last_update, efeat, upd, roots, n_q, loss_mask, want_grads=True,
@@ -231,7 +232,10 @@ def loss_and_grads(cfg, params, memory, last_update, efeat, upd, roots, n_q, los
                              _p(_u8(hid_gate) if hid_gate is not None else None), C.c_double(gate_eps),
                              C.c_int(int(want_grads)), _p(loss), _p(grads), _p(gn),
                              _p(mem_post), _p(lu_post), _p(h), _p(uniq), _p(win), _p(nu))
-    return StepResult(float(loss[0]), float(gn[0]), grads, mem_post, lu_post, h, uniq[:nu[0]].copy(), win[:nu[0]].copy())
+    ov = np.zeros(2, np.int64)
+    lib().orc_last_gate_overrides(_p(ov))
+    return StepResult(float(loss[0]), float(gn[0]), grads, mem_post, lu_post, h, uniq[:nu[0]].copy(), win[:nu[0]].copy(),
+                      (int(ov[0]), int(ov[1])))
 
 
 def adam(cfg, grads, params, m, v, step):

@@ -145,6 +145,10 @@ struct Inputs {
   double gate_eps;
 };
 
+// How many units of the last forward pass took the hinted branch against their own fp64 sign
+// ([0] output layer, [1] head's hidden layer).  Bookkeeping for the tests only: no result depends on it.
+int64_t g_gate_overrides[2] = {0, 0};
+
 struct Tape {
   // messages / reduction / GRU
   std::vector<int32_t> msg_node;  // [2 n_u]
@@ -346,10 +350,12 @@ void embed(const Inputs& in, const Layout& L, const double* P, const double* mem
   double pre_scale = 0;
   for (double v : T.pre_o) pre_scale = std::max(pre_scale, std::fabs(v));
   T.h_on.assign((size_t)R * d, 0);
+  g_gate_overrides[0] = 0;
   for (size_t e = 0; e < (size_t)R * d; ++e) {
     const double a = T.pre_o[e];
     bool on = a > 0;
     if (in.h_gate && std::fabs(a) <= in.gate_eps * pre_scale) on = in.h_gate[e] != 0;
+    if (on != (a > 0)) ++g_gate_overrides[0];
     T.h_on[e] = on;
     T.h[e] = on ? a : 0;
   }
@@ -380,6 +386,7 @@ void loss_forward(const Inputs& in, const Layout& L, const double* P, Tape& T) {
   double scale = 0;
   for (double v : T.pre1) scale = std::max(scale, std::fabs(v));
   double num = 0, den = 0;
+  g_gate_overrides[1] = 0;
   for (int j = 0; j < nq; ++j) {
     for (int pn = 0; pn < 2; ++pn) {
       const size_t p = (size_t)pn * nq + j;
@@ -388,6 +395,7 @@ void loss_forward(const Inputs& in, const Layout& L, const double* P, Tape& T) {
         const double acc = T.pre1[p * d + o];
         bool on = acc > 0;
         if (in.hid_gate && std::fabs(acc) <= in.gate_eps * scale) on = in.hid_gate[p * d + o] != 0;
+        if (on != (acc > 0)) ++g_gate_overrides[1];
         T.hid_on[p * d + o] = on;
         const double hd = on ? acc : 0;
         T.hid1[p * d + o] = hd;
@@ -752,6 +760,10 @@ void orc_loss_and_grads(const orc_config* c, const double* params, const double*
     if (grads_out) std::copy(G.begin(), G.end(), grads_out);
   }
 }
+
+// Units of the last orc_loss_and_grads call whose ReLU branch the hint decided against the fp64 sign:
+// out2[0] output layer of the embedding, out2[1] hidden layer of the head.
+void orc_last_gate_overrides(int64_t* out2) { out2[0] = g_gate_overrides[0]; out2[1] = g_gate_overrides[1]; }
 
 // Adam, no weight decay, no clipping:
 //   step += 1; m = b1 m + (1-b1) g; v = b2 v + (1-b2) g^2;

@@ -36,7 +36,7 @@ EXPORTS = ("tgnn_create", "tgnn_destroy", "tgnn_last_error", "tgnn_param_count",
            "tgnn_controller_create", "tgnn_controller_destroy", "tgnn_controller_begin_batch",
            "tgnn_controller_end_batch", "tgnn_controller_state", "tgnn_backward_scan_scratch", "tgnn_backward_scan",
            "tgnn_build_mixed", "tgnn_set_grad_sync", "tgnn_grad_buffer", "tgnn_apply_gradient", "tgnn_refresh_plan",
-           "tgnn_pack_rows", "tgnn_unpack_rows")
+           "tgnn_pack_rows", "tgnn_unpack_rows", "tgnn_debug_get_embeddings", "tgnn_debug_gemm_split")
 TGNN_STATIC_MAX_NODES = 65536
 
 
@@ -95,6 +95,9 @@ def load_library():
         lib.tgnn_debug_gemm.argtypes = [vp, vp, i64, i64, vp, i64, i64, vp, i64, i32, i32, i32, vp, vp, vp, vp, i32, i32, i32, i32,
                                         vp]
         lib.tgnn_debug_get_gates.argtypes = [vp, vp, vp, vp]
+        lib.tgnn_debug_get_embeddings.argtypes = [vp, vp, vp]
+        lib.tgnn_debug_gemm_split.argtypes = [vp, vp, i64, i64, vp, i64, i64, vp, i64, i32, i32, i32, vp, i32, i32, i32, vp, i64,
+                                              i32, u32, vp]
         lib.tgnn_step_mixed_host.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, i32, u32, u64, i64, vp, vp, vp]
         lib.tgnn_set_graph_replay.argtypes = [vp, i32]
         lib.tgnn_reduce_latest_static.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, vp, vp, i32]
@@ -474,6 +477,20 @@ class Tgnn:
             name, t0, dt = line.rsplit(" ", 2)
             out.append((name, float(t0), float(dt)))
         return out
+
+    def debug_gemm_split(self, A, a_rs, a_cs, Bm, b_rs, b_cs, Cm, ldc, M, N, K, scratch, bias=None, relu=False,
+                         accumulate=False, split_k=1, debug_withhold=0, spin_limit=0, check=True):
+        """The split-bf16 projection kernel on fp32 operands (split inside `scratch`, a uint8 CUDA tensor)."""
+        rc = self.lib.tgnn_debug_gemm_split(self._h, _dp(A, "f32", "A"), a_rs, a_cs, _dp(Bm, "f32", "B"), b_rs, b_cs,
+                                            _dp(Cm, "f32", "C"), ldc, M, N, K, _dp(bias, "f32", "bias"), int(relu),
+                                            int(accumulate), split_k, _dp(scratch, "u8", "scratch"), scratch.numel(),
+                                            debug_withhold, spin_limit, _stream())
+        if check:
+            self._ck(rc)
+        return rc
+
+    def debug_get_embeddings(self, h_out):
+        self._ck(self.lib.tgnn_debug_get_embeddings(self._h, _dp(h_out, "f32", "h_out"), _stream()))
 
     def debug_get_gates(self, h_gate_out, hid_gate_out):
         self._ck(self.lib.tgnn_debug_get_gates(self._h, _dp(h_gate_out, "u8", "h_gate_out"),

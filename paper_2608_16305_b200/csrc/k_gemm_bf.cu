@@ -1,0 +1,520 @@
+// The large projections on the 5th-generation tensor cores with split-bf16 operands (TGNN_MATH_BF16X3).
+//
+// An fp32 value x is held as two bf16 numbers, hi = bf16(x) and lo = bf16(x - hi): together they carry 16
+// mantissa bits (error below 2^-17 relative).  A product A B is then three tensor-core passes at the bf16 rate,
+//   lo(A) hi(B) + hi(A) lo(B) + hi(A) hi(B),
+// with fp32 accumulation in tensor memory -- more accurate than one TF32 pass (10 mantissa bits) at 1.5 times its
+// cost, and half the cost of the three-pass TF32 split.  The operands are STORED split (two bf16 planes of the
+// same shape, written by the kernel that produces the activation), so this kernel never touches operand
+// data with a thread: tiles go from global memory to shared memory by the tensor-memory-access unit,
+// already in the 128-byte-swizzled layout the MMA descriptors expect, and from there into the tensor cores.
+//
+// Roles (320 threads): warp 0 issues the tile copies, warp 1 owns tensor memory and issues the MMAs,
+// warps 2-9 are the epilogue (tensor memory -> registers -> a small staging square -> global memory in
+// whole 64-byte row segments, with bias / ReLU or an atomic accumulate).
+//
+// A CTA is persistent: it walks work items (pair of 128-row tiles, n-tile, contraction split).  The two row
+// tiles of a pair share every B tile, which halves the B traffic per flop; their accumulators sit side by
+// side in tensor memory (2 x 256 columns).  A tiles and B tiles travel through two separate rings of
+// shared-memory slots, each slot with a full (copy landed) and an empty (MMAs that read it retired,
+// signalled by tcgen05.commit) mbarrier, so copies run several slots ahead of the MMAs and across item
+// boundaries.  Every wait is bounded: on expiry the kernel records TGNN_ETIMEOUT, all roles leave their
+// loops, tensor memory is freed and the kernel returns.
+//
+// Operand layouts.  K-major (the contraction index is contiguous in memory: activations [M, K] and weight
+// planes [N, K]): a box of 64 elements x rows lands as rows of 128 bytes, 16-byte chunks XOR-swizzled
+// by (row mod 8); one MMA step (16 elements) advances 32 bytes inside the row.  MN-major (the row / column
+// index of C is contiguous: both operands of a weight gradient, whose contraction runs over matrix rows): a
+// box of 64 columns x 32 contraction rows per 64-column chunk lands the same way with the roles swapped,
+// which is the canonical MN-major layout of the 128-byte swizzle: chunks LBO apart, groups of 8 contraction
+// rows SBO = 1024 bytes apart; one MMA step consumes two such groups.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "tgnn_internal.cuh"
+
+namespace tgnn {
+namespace {
+
+constexpr int BM = 128;           // rows of C per tile (UMMA M)
+constexpr int ACC_STRIDE = 256;   // tensor-memory columns between the two accumulators of a pair
+constexpr int EPI_WARPS = 8;
+constexpr int THREADS = 32 * (2 + EPI_WARPS);
+constexpr int MAX_SLOTS = 8;
+constexpr int STG_PITCH = 20;     // floats between rows of a staged 32 x 16 square (16-byte aligned, bank-staggered)
+constexpr int STG_BYTES = EPI_WARPS * 32 * STG_PITCH * 4;
+constexpr unsigned SPIN_LIMIT = 1u << 22;
+constexpr int SMEM_LIMIT = 227 * 1024;
+
+struct BfArgs {
+  CUtensorMap a_map, b_map;   // three-dimensional: (contiguous index, row, plane)
+  float* C; int64_t ldc;
+  int M, N, K;
+  const float* bias;
+  int relu, accumulate;
+  int mn_major;               // 0: both operands K-major; 1: both MN-major
+  int m_tiles, n_tiles, bn, split_k;
+  int kb_total;               // contraction blocks (64 elements K-major, 32 rows MN-major)
+  int ksteps_total;           // MMA steps of 16 over the whole contraction
+  int a_slot_bytes, b_slot_bytes, n_a_slots, n_b_slots;
+  int b_chunks;               // MN-major: 64-column chunks per B tile
+  int32_t* status;
+  int debug_withhold;         // test hook: the MMA warp skips this many slot releases (an empty-slot wait then expires)
+  unsigned spin_limit;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait on a phase parity; gives up early when another role has already aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned limit, volatile int* abort_flag) {
+  for (unsigned it = 0; it < limit; ++it) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (done) return true;
+    if ((it & 63) == 63 && *abort_flag) return false;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;   // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;   // 128-byte swizzle
+  return d;
+}
+__device__ __forceinline__ void mma_bf16(uint32_t tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void commit_to(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+struct Item {
+  int mt0, tiles, n0, n_valid, kb0, kb1;
+};
+__device__ __forceinline__ Item decode_item(const BfArgs& g, int w) {
+  const int m_pairs = (g.m_tiles + 1) >> 1;
+  const int mp = w % m_pairs, rest = w / m_pairs;
+  const int nt = rest % g.n_tiles, sp = rest / g.n_tiles;
+  Item it;
+  it.mt0 = 2 * mp;
+  it.tiles = min(2, g.m_tiles - it.mt0);
+  it.n0 = nt * g.bn;
+  it.n_valid = min(g.bn, g.N - it.n0);
+  const int per = (g.kb_total + g.split_k - 1) / g.split_k;
+  it.kb0 = sp * per;
+  it.kb1 = min(g.kb_total, it.kb0 + per);
+  return it;
+}
+
+__global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_constant__ BfArgs g) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) uint64_t s_full_a[MAX_SLOTS], s_empty_a[MAX_SLOTS], s_full_b[MAX_SLOTS], s_empty_b[MAX_SLOTS];
+  __shared__ __align__(8) uint64_t s_tmem_full, s_tmem_empty;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t a_ring = smem_u32(smem);
+  const uint32_t b_ring = a_ring + (uint32_t)(g.n_a_slots * g.a_slot_bytes);
+  float* stg_base = reinterpret_cast<float*>(smem + (size_t)g.n_a_slots * g.a_slot_bytes + (size_t)g.n_b_slots * g.b_slot_bytes);
+
+  if (tid == 0) {
+    for (int s = 0; s < MAX_SLOTS; ++s) {
+      mbar_init(smem_u32(&s_full_a[s]), 1); mbar_init(smem_u32(&s_empty_a[s]), 1);
+      mbar_init(smem_u32(&s_full_b[s]), 1); mbar_init(smem_u32(&s_empty_b[s]), 1);
+    }
+    mbar_init(smem_u32(&s_tmem_full), 1);
+    mbar_init(smem_u32(&s_tmem_empty), EPI_WARPS);
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = s_tmem;
+  volatile int* abort_flag = &s_abort;
+  const unsigned limit = g.spin_limit;
+
+  const int m_pairs = (g.m_tiles + 1) >> 1;
+  const int items = m_pairs * g.n_tiles * g.split_k;
+  const int ks_per_kb = g.mn_major ? 2 : 4;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ tile copies
+    if (lane == 0) {
+      uint32_t ca = 0, cb = 0;
+      bool ok = true;
+      const uint32_t a_bytes = (uint32_t)g.a_slot_bytes, b_bytes = (uint32_t)g.b_slot_bytes;
+      const uint32_t a_plane = a_bytes >> 1, b_plane = b_bytes >> 1;
+      for (int w = blockIdx.x; w < items && ok; w += gridDim.x) {
+        const Item it = decode_item(g, w);
+        for (int kb = it.kb0; kb < it.kb1 && ok; ++kb) {
+          {
+            const uint32_t s = cb % (uint32_t)g.n_b_slots;
+            ok = mbar_wait(smem_u32(&s_empty_b[s]), ((cb / (uint32_t)g.n_b_slots) & 1u) ^ 1u, limit, abort_flag);
+            if (!ok) break;
+            const uint32_t bar = smem_u32(&s_full_b[s]), dst = b_ring + s * b_bytes;
+            mbar_expect_tx(bar, b_bytes);
+            if (!g.mn_major) {
+              tma_3d(dst, &g.b_map, kb * 64, it.n0, 0, bar);
+              tma_3d(dst + b_plane, &g.b_map, kb * 64, it.n0, 1, bar);
+            } else {
+              for (int p = 0; p < 2; ++p)
+                for (int c = 0; c < g.b_chunks; ++c) tma_3d(dst + p * b_plane + c * 4096, &g.b_map, it.n0 + 64 * c, kb * 32, p, bar);
+            }
+            ++cb;
+          }
+          for (int t = 0; t < it.tiles && ok; ++t) {
+            const uint32_t s = ca % (uint32_t)g.n_a_slots;
+            ok = mbar_wait(smem_u32(&s_empty_a[s]), ((ca / (uint32_t)g.n_a_slots) & 1u) ^ 1u, limit, abort_flag);
+            if (!ok) break;
+            const uint32_t bar = smem_u32(&s_full_a[s]), dst = a_ring + s * a_bytes;
+            const int m0 = (it.mt0 + t) * BM;
+            mbar_expect_tx(bar, a_bytes);
+            if (!g.mn_major) {
+              tma_3d(dst, &g.a_map, kb * 64, m0, 0, bar);
+              tma_3d(dst + a_plane, &g.a_map, kb * 64, m0, 1, bar);
+            } else {
+              for (int p = 0; p < 2; ++p)
+                for (int c = 0; c < 2; ++c) tma_3d(dst + p * a_plane + c * 4096, &g.a_map, m0 + 64 * c, kb * 32, p, bar);
+            }
+            ++ca;
+          }
+        }
+      }
+      if (!ok) { s_abort = 1; atomicCAS(g.status, 0, TGNN_ETIMEOUT); }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t ca = 0, cb = 0, n_item = 0;
+      int withheld = 0;
+      bool ok = true;
+      const uint32_t a_bytes = (uint32_t)g.a_slot_bytes, b_bytes = (uint32_t)g.b_slot_bytes;
+      const uint32_t a_plane = a_bytes >> 1, b_plane = b_bytes >> 1;
+      const uint32_t mn = g.mn_major ? 1u : 0u;
+      // K-major: 8-row groups 1024 B apart (SBO), a step advances 32 B.  MN-major: 64-column chunks 4096 B apart
+      // (LBO), 8-row contraction groups 1024 B apart (SBO), a step advances two groups.
+      const uint32_t lbo = mn ? 4096u : 16u, sbo = 1024u, kstep_bytes = mn ? 2048u : 32u;
+      for (int w = blockIdx.x; w < items && ok; w += gridDim.x) {
+        const Item it = decode_item(g, w);
+        if (it.kb0 >= it.kb1) continue;   // an empty contraction range: every role skips it
+        ok = mbar_wait(smem_u32(&s_tmem_empty), (n_item & 1u) ^ 1u, limit, abort_flag);   // accumulators drained
+        if (!ok) break;
+        ++n_item;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int n_mma = (it.n_valid + 15) / 16 * 16;
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (mn << 15) | (mn << 16) |
+                               ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+        for (int kb = it.kb0; kb < it.kb1 && ok; ++kb) {
+          const uint32_t sb = cb % (uint32_t)g.n_b_slots;
+          ok = mbar_wait(smem_u32(&s_full_b[sb]), (cb / (uint32_t)g.n_b_slots) & 1u, limit, abort_flag);
+          if (!ok) break;
+          const uint32_t b_addr = b_ring + sb * b_bytes;
+          const int ks_n = min(ks_per_kb, g.ksteps_total - kb * ks_per_kb);
+          for (int t = 0; t < it.tiles && ok; ++t) {
+            const uint32_t sa = ca % (uint32_t)g.n_a_slots;
+            ok = mbar_wait(smem_u32(&s_full_a[sa]), (ca / (uint32_t)g.n_a_slots) & 1u, limit, abort_flag);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a_addr = a_ring + sa * a_bytes;
+            const uint32_t acc = tmem + (uint32_t)(t * ACC_STRIDE);
+            for (int ks = 0; ks < ks_n; ++ks) {
+              const uint64_t da_hi = make_desc(a_addr + ks * kstep_bytes, lbo, sbo);
+              const uint64_t da_lo = make_desc(a_addr + a_plane + ks * kstep_bytes, lbo, sbo);
+              const uint64_t db_hi = make_desc(b_addr + ks * kstep_bytes, lbo, sbo);
+              const uint64_t db_lo = make_desc(b_addr + b_plane + ks * kstep_bytes, lbo, sbo);
+              const uint32_t first = (kb > it.kb0 || ks > 0) ? 1u : 0u;
+              mma_bf16(acc, da_lo, db_hi, idesc, first);
+              mma_bf16(acc, da_hi, db_lo, idesc, 1u);
+              mma_bf16(acc, da_hi, db_hi, idesc, 1u);
+            }
+            if (withheld < g.debug_withhold) ++withheld;   // test hook: this slot is never handed back
+            else commit_to(smem_u32(&s_empty_a[sa]));
+            ++ca;
+          }
+          if (ok) commit_to(smem_u32(&s_empty_b[sb]));
+          ++cb;
+        }
+        if (ok) commit_to(smem_u32(&s_tmem_full));
+      }
+      if (!ok) { s_abort = 1; atomicCAS(g.status, 0, TGNN_ETIMEOUT); }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------ epilogue
+    const int e = warp - 2;
+    const int t = e >> 2;          // which accumulator of the pair
+    const int q4 = warp & 3;       // the tensor-memory lane quarter this warp may read
+    float* stg = stg_base + e * (32 * STG_PITCH);
+    const bool c_vec = (((uintptr_t)g.C & 15) == 0) && (g.ldc % 4 == 0);
+    const int sub = lane >> 2, ch = lane & 3;
+    uint32_t n_item = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < items && ok; w += gridDim.x) {
+      const Item it = decode_item(g, w);
+      if (it.kb0 >= it.kb1) continue;
+      ok = mbar_wait(smem_u32(&s_tmem_full), n_item & 1u, limit, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      ++n_item;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      if (t < it.tiles) {
+        const int m0 = (it.mt0 + t) * BM;
+        const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(t * ACC_STRIDE);
+        const bool with_bias = g.bias != nullptr && it.kb0 == 0;
+        for (int c0 = 0; c0 < it.n_valid; c0 += 32) {
+          uint32_t r[32];
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+              "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+              : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+                "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+                "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+                "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+              : "r"(taddr + (uint32_t)c0));
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const int cb0 = c0 + 16 * h;
+            if (cb0 >= it.n_valid) break;   // warp-uniform
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              *reinterpret_cast<uint4*>(stg + lane * STG_PITCH + 4 * q) =
+                  make_uint4(r[16 * h + 4 * q], r[16 * h + 4 * q + 1], r[16 * h + 4 * q + 2], r[16 * h + 4 * q + 3]);
+            __syncwarp();
+            const int col = cb0 + 4 * ch;   // first of this lane's four columns, relative to the tile
+            float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (with_bias && col < it.n_valid) {
+              const float* bp = g.bias + it.n0 + col;
+              b4.x = bp[0];
+              if (col + 1 < it.n_valid) b4.y = bp[1];
+              if (col + 2 < it.n_valid) b4.z = bp[2];
+              if (col + 3 < it.n_valid) b4.w = bp[3];
+            }
+            const bool full4 = col + 3 < it.n_valid;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int rr = j * 8 + sub;
+              const int row = m0 + q4 * 32 + rr;
+              float4 v = *reinterpret_cast<const float4*>(stg + rr * STG_PITCH + 4 * ch);
+              if (row < g.M && col < it.n_valid) {
+                v.x += b4.x; v.y += b4.y; v.z += b4.z; v.w += b4.w;
+                float* cp = g.C + (int64_t)row * g.ldc + it.n0 + col;
+                if (g.accumulate) {
+                  if (full4 && c_vec) {
+                    atomicAdd(reinterpret_cast<float4*>(cp), v);
+                  } else {
+                    atomicAdd(cp, v.x);
+                    if (col + 1 < it.n_valid) atomicAdd(cp + 1, v.y);
+                    if (col + 2 < it.n_valid) atomicAdd(cp + 2, v.z);
+                    if (col + 3 < it.n_valid) atomicAdd(cp + 3, v.w);
+                  }
+                } else {
+                  if (g.relu) { v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); v.z = fmaxf(v.z, 0.f); v.w = fmaxf(v.w, 0.f); }
+                  if (full4 && c_vec) {
+                    *reinterpret_cast<float4*>(cp) = v;
+                  } else {
+                    cp[0] = v.x;
+                    if (col + 1 < it.n_valid) cp[1] = v.y;
+                    if (col + 2 < it.n_valid) cp[2] = v.z;
+                    if (col + 3 < it.n_valid) cp[3] = v.w;
+                  }
+                }
+              }
+            }
+            __syncwarp();
+          }
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&s_tmem_empty));
+    }
+    if (!ok && lane == 0) { s_abort = 1; atomicCAS(g.status, 0, TGNN_ETIMEOUT); }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (s_abort && warp == 0) {
+    // copies this CTA asked for may still be on their way into its shared memory: give them a bounded while
+    for (int i = 0; i < 64; ++i) __nanosleep(2000);
+  }
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+  }
+}
+
+// fp32 rows -> two bf16 planes (hi, lo).  One thread per 4 consecutive columns; columns in [cols, ld_out) of the
+// planes are written as zeros except column `ones_col` (if >= 0), which is 1 (the bias column of a weight gradient).
+__global__ void __launch_bounds__(256) split_rows_kernel(const float* __restrict__ X, int64_t ld_in, int64_t rows, int cols,
+                                                         const int32_t* __restrict__ dev_rows, __nv_bfloat16* __restrict__ hi,
+                                                         __nv_bfloat16* __restrict__ lo, int64_t ld_out, int ones_col) {
+  const int per_row = (int)(ld_out >> 2);
+  const int64_t n_rows = dev_rows ? min((int64_t)*dev_rows, rows) : rows;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < rows * per_row; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / per_row;
+    const int c = (int)(i - r * per_row) * 4;
+    float v[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int cc = c + e;
+      v[e] = (r < n_rows && cc < cols) ? X[r * ld_in + cc] : ((cc == ones_col && r < n_rows) ? 1.f : 0.f);
+    }
+    __nv_bfloat16 h[4], l[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      h[e] = __float2bfloat16_rn(v[e]);
+      l[e] = __float2bfloat16_rn(v[e] - __bfloat162float(h[e]));
+    }
+    *reinterpret_cast<uint2*>(hi + r * ld_out + c) = *reinterpret_cast<const uint2*>(h);
+    *reinterpret_cast<uint2*>(lo + r * ld_out + c) = *reinterpret_cast<const uint2*>(l);
+  }
+}
+
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+TensorMapEncodeFn encoder() {
+  static TensorMapEncodeFn enc = nullptr;
+  static bool looked = false;
+  if (!looked) {
+    looked = true;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      enc = reinterpret_cast<TensorMapEncodeFn>(fn);
+    (void)cudaGetLastError();
+  }
+  return enc;
+}
+
+// (contiguous index, row, plane) view of a split matrix; box = 64 elements x box_rows x 1 plane, 128-byte swizzle,
+// zeros outside [0, cols) x [0, rows).
+bool encode_split_map(CUtensorMap* map, const SplitMat& m, int box_rows) {
+  const TensorMapEncodeFn enc = encoder();
+  if (!enc || m.rows <= 0 || m.cols <= 0 || box_rows < 1 || box_rows > 256) return false;
+  if (((uintptr_t)m.hi & 15) != 0 || m.ld % 8 != 0 || m.plane_stride % 8 != 0) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)m.cols, (cuuint64_t)m.rows, 2};
+  const cuuint64_t strides[2] = {(cuuint64_t)m.ld * 2, (cuuint64_t)m.plane_stride * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  const cuuint32_t elem[3] = {1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, m.hi, dims, strides, box, elem,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int launch_split_rows(tgnn_ctx* ctx, const float* X, int64_t ld_in, int64_t rows, int cols, const int32_t* dev_rows,
+                      const SplitMat& out, int ones_col, const char* name, cudaStream_t s) {
+  if (rows <= 0) return TGNN_OK;
+  const int64_t work = rows * (out.ld >> 2);
+  const int blocks = (int)((work + 255) / 256 < 148 * 16 ? (work + 255) / 256 : 148 * 16);
+  {
+    KernelScope scope__(ctx, name, s);
+    split_rows_kernel<<<blocks, 256, 0, s>>>(X, ld_in, rows, cols, dev_rows, reinterpret_cast<__nv_bfloat16*>(out.hi),
+                                             reinterpret_cast<__nv_bfloat16*>(out.hi) + out.plane_stride, out.ld, ones_col);
+  }
+  TGNN_LAUNCH_OK(ctx, name);
+  return TGNN_OK;
+}
+
+// C[M,N] (+)= A B (+ bias) (ReLU) from split operands.
+//   mn_major = 0: A is the matrix [M, K], B the matrix [N, K] (both with the contraction index contiguous);
+//   mn_major = 1: A is the matrix [K, M], B the matrix [K, N] (contraction over rows: C = A^T B).
+// split_k > 1 needs accumulate (C holds valid data; partial sums are added atomically).
+int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int mn_major, float* C, int64_t ldc, int M, int N,
+                      int K, const float* bias, int relu, int accumulate, int split_k, const char* name, cudaStream_t s,
+                      int debug_withhold, unsigned spin_limit) {
+  if (M <= 0 || N <= 0) return TGNN_OK;
+  if (K <= 0) return set_error(ctx, TGNN_EINVAL, "gemm %s: empty contraction", name);
+  if (split_k > 1 && !accumulate) return set_error(ctx, TGNN_EINVAL, "gemm %s: split_k needs accumulate", name);
+  BfArgs a = {};
+  a.C = C; a.ldc = ldc; a.M = M; a.N = N; a.K = K; a.bias = bias; a.relu = relu; a.accumulate = accumulate;
+  a.mn_major = mn_major ? 1 : 0;
+  a.status = ctx->ws.status;
+  a.debug_withhold = debug_withhold;
+  a.spin_limit = spin_limit ? spin_limit : SPIN_LIMIT;
+  a.m_tiles = (M + BM - 1) / BM;
+  a.n_tiles = (N + 255) / 256;
+  a.bn = ((N + a.n_tiles - 1) / a.n_tiles + 15) / 16 * 16;
+  const int bke = mn_major ? 32 : 64;
+  a.kb_total = (K + bke - 1) / bke;
+  a.ksteps_total = (K + 15) / 16;
+  a.b_chunks = (a.bn + 63) / 64;
+  a.a_slot_bytes = mn_major ? 2 * 2 * 4096 : 2 * BM * 128;
+  a.b_slot_bytes = mn_major ? 2 * a.b_chunks * 4096 : 2 * a.bn * 128;
+  const int budget = SMEM_LIMIT - 1024 - STG_BYTES - 1024;
+  a.n_b_slots = a.b_slot_bytes > 40 * 1024 ? 2 : (a.b_slot_bytes > 20 * 1024 ? 3 : 4);
+  a.n_a_slots = (budget - a.n_b_slots * a.b_slot_bytes) / a.a_slot_bytes;
+  if (a.n_a_slots > MAX_SLOTS) a.n_a_slots = MAX_SLOTS;
+  if (a.n_a_slots < 2) return set_error(ctx, TGNN_ESHAPE, "gemm %s: tile does not fit shared memory", name);
+  const int m_pairs = (a.m_tiles + 1) / 2;
+  a.split_k = 1;
+  if (accumulate && split_k > 1) {
+    const int base = m_pairs * a.n_tiles;
+    int sp = (148 + base - 1) / base;
+    const int max_s = (a.kb_total + 7) / 8;   // at least 8 contraction blocks per split
+    if (sp > max_s) sp = max_s;
+    if (sp > split_k) sp = split_k;
+    a.split_k = sp < 1 ? 1 : sp;
+  }
+  // the K-major B box is a whole n-tile (bn rows); MN-major boxes are 64 columns x 32 contraction rows
+  if (!encode_split_map(&a.a_map, A, mn_major ? 32 : BM) || !encode_split_map(&a.b_map, B, mn_major ? 32 : a.bn))
+    return set_error(ctx, TGNN_ECUDA, "gemm %s: tensor map encoding failed", name);
+  const int items = m_pairs * a.n_tiles * a.split_k;
+  const int smem = 1024 + a.n_a_slots * a.a_slot_bytes + a.n_b_slots * a.b_slot_bytes + STG_BYTES;
+  static int attr_bytes[64] = {};
+  int dev = 0;
+  TGNN_CUDA_OK(ctx, cudaGetDevice(&dev));
+  if (dev >= 0 && dev < 64 && attr_bytes[dev] < smem) {
+    TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(gemm_bf16s_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT));
+    attr_bytes[dev] = SMEM_LIMIT;
+  }
+  {
+    KernelScope scope__(ctx, name, s);
+    gemm_bf16s_kernel<<<items < 148 ? items : 148, THREADS, smem, s>>>(a);
+  }
+  TGNN_LAUNCH_OK(ctx, name);
+  return TGNN_OK;
+}
+
+}  // namespace tgnn

@@ -59,13 +59,16 @@ __global__ void __launch_bounds__(1024) reduce_latest_static_kernel(const int32_
   int32_t* win_msg = reinterpret_cast<int32_t*>(best_id + kMaxNodes);
   __shared__ int s_warp[32];
   __shared__ int s_total;
+  __shared__ int s_bad;  // a message named a node outside [0, N): it is skipped, never used as an index
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  if (tid == 0) s_bad = 0;
   for (int v = tid; v < N; v += blockDim.x) { best_t[v] = 0ULL; best_id[v] = 0ULL; }
   __syncthreads();
   const int n_round = (n_msg + 31) / 32 * 32;
   for (int j = tid; j < n_round; j += blockDim.x) {
     const int node = j < n_msg ? msg_node[j] : -1;
-    const bool v = node >= 0;
+    if (node >= N) s_bad = 1;
+    const bool v = node >= 0 && node < N;
     const unsigned act = __ballot_sync(FULL, v);
     if (v) {
       const unsigned peers = __match_any_sync(act, node);
@@ -76,7 +79,7 @@ __global__ void __launch_bounds__(1024) reduce_latest_static_kernel(const int32_
   __syncthreads();
   for (int j = tid; j < n_round; j += blockDim.x) {
     const int node = j < n_msg ? msg_node[j] : -1;
-    const bool v = node >= 0 && orderable(t[j >> 1]) == best_t[node];
+    const bool v = node >= 0 && node < N && orderable(t[j >> 1]) == best_t[node];
     const unsigned act = __ballot_sync(FULL, v);
     if (v) {
       const unsigned peers = __match_any_sync(act, node);
@@ -88,7 +91,7 @@ __global__ void __launch_bounds__(1024) reduce_latest_static_kernel(const int32_
   __syncthreads();
   for (int j = tid; j < n_msg; j += blockDim.x) {
     const int node = msg_node[j];
-    if (node < 0) continue;
+    if (node < 0 || node >= N) continue;
     const unsigned long long key = (((unsigned long long)(uint32_t)eid[j >> 1]) << 1 | (unsigned)(j & 1)) + 1ULL;
     if (orderable(t[j >> 1]) == best_t[node] && key == best_id[node]) win_msg[node] = j;
   }
@@ -123,7 +126,7 @@ __global__ void __launch_bounds__(1024) reduce_latest_static_kernel(const int32_
       ++pos;
     }
   }
-  if (tid == 0) *n_uniq_out = s_total;
+  if (tid == 0) *n_uniq_out = s_bad ? -1 : s_total;
 }
 
 int fail(char* err, int err_size, int code, const char* fmt, ...) {

@@ -157,6 +157,15 @@ size_t carve(tgnn_ctx* ctx, char* base) {
 
 inline cudaStream_t S(void* stream) { return reinterpret_cast<cudaStream_t>(stream); }
 
+// Recorded step graphs have the borrowed pointers (state, graph, feature table) and the launch sequence of
+// the current mode baked into their kernel arguments: whenever one of those changes they are dropped and
+// the next steps record new ones.
+void drop_step_graphs(tgnn_ctx* ctx) {
+  for (int i = 0; i < ctx->n_graphs; ++i)
+    if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
+  ctx->n_graphs = 0;
+}
+
 }  // namespace
 }  // namespace tgnn
 
@@ -307,6 +316,7 @@ int tgnn_set_graph(tgnn_ctx* ctx, const int64_t* indptr, const int32_t* nbr, con
   if (!ctx) return TGNN_EINVAL;
   NEED(ctx, indptr && n_entries >= 0, TGNN_EINVAL, "set_graph: null indptr or negative size");
   NEED(ctx, n_entries == 0 || (nbr && eid && ts), TGNN_EINVAL, "set_graph: null adjacency arrays");
+  if (ctx->indptr != indptr || ctx->g_nbr != nbr || ctx->g_eid != eid || ctx->g_ts != ts) drop_step_graphs(ctx);
   ctx->indptr = indptr; ctx->g_nbr = nbr; ctx->g_eid = eid; ctx->g_ts = ts; ctx->n_entries = n_entries;
   return TGNN_OK;
 }
@@ -318,6 +328,7 @@ int tgnn_set_edge_features(tgnn_ctx* ctx, const void* efeat, int dtype, int64_t 
   NEED(ctx, d_e == 0 || efeat, TGNN_EINVAL, "set_edge_features: null table");
   NEED(ctx, num_events >= 0, TGNN_EINVAL, "set_edge_features: negative size");
   NEED(ctx, ((uintptr_t)efeat & 3) == 0, TGNN_EINVAL, "set_edge_features: table must be 4-byte aligned");
+  if (ctx->efeat != efeat) drop_step_graphs(ctx);
   ctx->efeat = efeat; ctx->num_events = num_events;
   return TGNN_OK;
 }
@@ -326,6 +337,9 @@ int tgnn_set_state(tgnn_ctx* ctx, float* memory, double* last_update, float* par
                    int64_t* step) {
   if (!ctx) return TGNN_EINVAL;
   NEED(ctx, memory && last_update && params && adam_m && adam_v && step, TGNN_EINVAL, "set_state: null pointer");
+  if (ctx->memory != memory || ctx->last_update != last_update || ctx->params != params || ctx->adam_m != adam_m ||
+      ctx->adam_v != adam_v || ctx->step != step)
+    drop_step_graphs(ctx);
   ctx->memory = memory; ctx->last_update = last_update; ctx->params = params;
   ctx->adam_m = adam_m; ctx->adam_v = adam_v; ctx->step = step;
   ctx->have_update = false; ctx->have_embed = false; ctx->grads_zeroed = false; ctx->images_fresh = false;
@@ -512,9 +526,7 @@ int tgnn_set_grad_sync(tgnn_ctx* ctx, int defer) {
   if (!ctx) return TGNN_EINVAL;
   if ((defer != 0) == (ctx->defer_adam != 0)) return TGNN_OK;
   // recorded steps end with the fused norm + Adam launch of the other mode: drop them
-  for (int i = 0; i < ctx->n_graphs; ++i)
-    if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
-  ctx->n_graphs = 0;
+  drop_step_graphs(ctx);
   ctx->defer_adam = defer ? 1 : 0;
   ctx->grad_pending = false;
   return TGNN_OK;
@@ -725,6 +737,16 @@ int tgnn_debug_get_grads(tgnn_ctx* ctx, float* grads_out, void* stream) {
   return TGNN_OK;
 }
 
+int tgnn_debug_get_embeddings(tgnn_ctx* ctx, float* h_out, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, h_out, TGNN_EINVAL, "debug_get_embeddings: null pointer");
+  NEED(ctx, ctx->e_h, TGNN_ESTATE, "debug_get_embeddings: no embedding recorded");
+  if (ctx->e_n > 0)
+    TGNN_CUDA_OK(ctx, cudaMemcpyAsync(h_out, ctx->e_h, sizeof(float) * (size_t)ctx->e_n * ctx->cfg.d,
+                                      cudaMemcpyDeviceToDevice, S(stream)));
+  return TGNN_OK;
+}
+
 int tgnn_debug_get_gates(tgnn_ctx* ctx, uint8_t* h_gate_out, uint8_t* hid_gate_out, void* stream) {
   if (!ctx) return TGNN_EINVAL;
   NEED(ctx, h_gate_out && hid_gate_out, TGNN_EINVAL, "debug_get_gates: null pointer");
@@ -743,6 +765,35 @@ int tgnn_debug_gemm(tgnn_ctx* ctx, const float* A, int64_t a_rs, int64_t a_cs, c
   g.M = M; g.N = N; g.K = K; g.dev_M = dev_M; g.dev_K = dev_K; g.bias = bias; g.rowsum_out = rowsum_out;
   g.relu = relu; g.accumulate = accumulate; g.split_k = split_k < 1 ? 1 : split_k; g.precise = precise;
   return launch_gemm(ctx, g, "debug_gemm", S(stream));
+}
+
+int tgnn_debug_gemm_split(tgnn_ctx* ctx, const float* A, int64_t a_rs, int64_t a_cs, const float* B, int64_t b_rs,
+                          int64_t b_cs, float* C, int64_t ldc, int M, int N, int K, const float* bias, int relu,
+                          int accumulate, int split_k, void* scratch, int64_t scratch_bytes, int debug_withhold,
+                          uint32_t spin_limit, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  NEED(ctx, A && B && C && scratch && M > 0 && N > 0 && K > 0, TGNN_EINVAL, "debug_gemm_split: null pointer or empty product");
+  int mn;
+  int64_t lda, ldb, a_rows, a_cols, b_rows, b_cols;
+  if (a_cs == 1 && b_rs == 1) { mn = 0; lda = a_rs; ldb = b_cs; a_rows = M; a_cols = K; b_rows = N; b_cols = K; }
+  else if (a_rs == 1 && b_cs == 1) { mn = 1; lda = a_cs; ldb = b_rs; a_rows = K; a_cols = M; b_rows = K; b_cols = N; }
+  else return set_error(ctx, TGNN_ESHAPE, "debug_gemm_split: operands must both have the contraction index contiguous, or both the other one");
+  const auto up8 = [](int64_t x) { return (x + 7) / 8 * 8; };
+  SplitMat a{nullptr, up8(a_cols), 0, a_rows, a_cols}, b{nullptr, up8(b_cols), 0, b_rows, b_cols};
+  a.plane_stride = a.rows * a.ld;
+  b.plane_stride = b.rows * b.ld;
+  const int64_t a_bytes = (2 * a.plane_stride * 2 + 255) / 256 * 256, b_bytes = 2 * b.plane_stride * 2;
+  NEED(ctx, scratch_bytes >= a_bytes + b_bytes, TGNN_ECAPACITY, "debug_gemm_split: scratch of %lld bytes, %lld needed",
+       (long long)scratch_bytes, (long long)(a_bytes + b_bytes));
+  NEED(ctx, ((uintptr_t)scratch & 255) == 0, TGNN_EINVAL, "debug_gemm_split: scratch must be 256-byte aligned");
+  a.hi = scratch;
+  b.hi = (char*)scratch + a_bytes;
+  int rc = launch_split_rows(ctx, A, lda, a.rows, (int)a.cols, nullptr, a, -1, "split_a", S(stream));
+  if (rc) return rc;
+  rc = launch_split_rows(ctx, B, ldb, b.rows, (int)b.cols, nullptr, b, -1, "split_b", S(stream));
+  if (rc) return rc;
+  return launch_gemm_split(ctx, a, b, mn, C, ldc, M, N, K, bias, relu, accumulate, split_k < 1 ? 1 : split_k, "debug_gemm_split",
+                           S(stream), debug_withhold, spin_limit);
 }
 
 int tgnn_status(tgnn_ctx* ctx, int32_t* status_host, void* stream) {

@@ -325,6 +325,19 @@ struct GemmArgs {
 };
 int launch_gemm(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s);
 int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s);  // k_gemm_tc.cu
+// ---- split-bf16 projections (k_gemm_bf.cu) ----
+// An fp32 matrix stored as two bf16 planes of the same row-major shape: hi = bf16(x) at `hi`, lo = bf16(x - hi)
+// at hi + plane_stride (in bf16 elements).  ld and plane_stride are multiples of 8, `hi` is 16-byte aligned.
+struct SplitMat {
+  void* hi;
+  int64_t ld, plane_stride;
+  int64_t rows, cols;
+};
+int launch_split_rows(tgnn_ctx* ctx, const float* X, int64_t ld_in, int64_t rows, int cols, const int32_t* dev_rows,
+                      const SplitMat& out, int ones_col, const char* name, cudaStream_t s);
+int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int mn_major, float* C, int64_t ldc, int M, int N,
+                      int K, const float* bias, int relu, int accumulate, int split_k, const char* name, cudaStream_t s,
+                      int debug_withhold = 0, unsigned spin_limit = 0);
 size_t plan_weight_sites(tgnn_ctx* ctx);                       // fills ctx->sites, returns the image bytes needed
 int launch_prep_weights(tgnn_ctx* ctx, cudaStream_t s);        // writes all images from the current parameters
 

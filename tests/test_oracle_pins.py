@@ -501,6 +501,52 @@ def test_gradient_against_central_differences(oracle, seed):
     assert abs(base.gradnorm - math.sqrt((base.grads ** 2).sum())) < 1e-14
 
 
+def test_time_encoder_gradient_with_the_fp32_argument(oracle):
+    """The backward pass of the message's time encoding when the argument is fp32 by definition: a hand
+    case with one update event (a self-loop, so a single winner whose gate gradient is the update cell's
+    bias gradient) and roots without neighbors at phase 0 (so the attention side contributes nothing to the
+    encoder).  Then  dL/dw_c = -sin(arg_c) * dt32 * dx_c  and  dL/db_c = -sin(arg_c) * dx_c  with
+    arg_c = w_c * dt32 formed in fp32, dt32 = fp32(16777217) = 16777216, and dx = W_i[:, Phi columns]^T dG
+    computed here from the oracle's own bias gradient.  The fp64 reading (dt = 16777217) gives other sines
+    and another factor, so a backward that forgot either rounding fails."""
+    N, d, k = 5, 4, 3
+    cfg = oracle.make_config(N, d, 0, k, 2, phi_f32=True, round_state_f32=False)
+    W = wl.make_weights(d, 0, 3, bias_scale=0.3)
+    W["time_w"] = np.array([1.0, 0.5, 0.25, 2.0 ** -20], np.float32)
+    W["time_b"] = np.zeros(d, np.float32)
+    P = oracle.pack_params(cfg, W)
+    rng = np.random.default_rng(5)
+    mem = rng.normal(size=(N, d)) * 0.5
+    lu = np.zeros(N)
+    t_ev = 16777217.0                                   # 2^24 + 1: not an fp32 number
+    upd = (np.array([1], np.int32), np.array([1], np.int32), np.array([t_ev]), np.array([0], np.int32), None)
+    nodes = np.array([1, 2, 3], np.int32)
+    times = np.full(3, t_ev + 1.0)
+    none = (np.full((3, k), -1, np.int32), np.full((3, k), -1, np.int32), np.zeros((3, k)), np.zeros(3, np.int32))
+    r = oracle.loss_and_grads(cfg, P, mem, lu, None, upd, (nodes, times) + none, 1, None)
+    assert list(r.uniq) == [1] and list(r.winner) == [1]            # role 1 wins the tie on (t, eid)
+    lay = oracle.param_layout(cfg)
+    dmsg = 3 * d
+    dG = r.grads[lay["gru_b_i"]:lay["gru_b_i"] + 3 * d]             # single winner: the gate gradient itself
+    Wi = np.asarray(W["gru_w_i"], np.float64).reshape(3 * d, dmsg)
+    dx = Wi[:, 2 * d:].T @ dG
+    assert np.abs(dx).min() > 0
+    dt32 = float(np.float32(t_ev))
+    assert dt32 == 16777216.0
+    arg32 = (W["time_w"].astype(np.float32) * np.float32(dt32)).astype(np.float64)   # exact products, phase 0
+    gw, gb = r.grads[lay["time_w"]:lay["time_w"] + d], r.grads[lay["time_b"]:lay["time_b"] + d]
+    assert np.allclose(gb, -np.sin(arg32) * dx, rtol=1e-11, atol=1e-15)
+    assert np.allclose(gw, -np.sin(arg32) * dt32 * dx, rtol=1e-11, atol=1e-9)
+    # the fp64 reading of the same case differs in both factors
+    arg64 = W["time_w"].astype(np.float64) * t_ev
+    assert np.abs(np.sin(arg64) - np.sin(arg32)).max() > 0.1
+    cfg64 = oracle.make_config(N, d, 0, k, 2, phi_f32=False, round_state_f32=False)
+    r64 = oracle.loss_and_grads(cfg64, P, mem, lu, None, upd, (nodes, times) + none, 1, None)
+    dx64 = Wi[:, 2 * d:].T @ r64.grads[lay["gru_b_i"]:lay["gru_b_i"] + 3 * d]
+    assert np.allclose(r64.grads[lay["time_w"]:lay["time_w"] + d], -np.sin(arg64) * t_ev * dx64, rtol=1e-11, atol=1e-9)
+    assert not np.allclose(r64.grads[lay["time_w"]:lay["time_w"] + d], gw, rtol=1e-3)
+
+
 def test_relu_gate_hints_apply_only_inside_the_window(oracle):
     cfg = small_cfg(oracle, N=20, phi_f32=False, round_state_f32=False)
     W = weights(cfg)

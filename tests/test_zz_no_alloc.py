@@ -30,7 +30,7 @@ def _case(rng, N, n, hub):
     return node, t, eid
 
 
-def test_static_reduction_matches_context_backed_one_on_two_calls_in_a_row():
+def test_static_reduction_matches_context_backed_one_on_two_calls_in_a_row(oracle):
     from paper_2608_16305_b200 import binding as B
     rng = np.random.default_rng(31)
     N = 50_000
@@ -56,7 +56,37 @@ def test_static_reduction_matches_context_backed_one_on_two_calls_in_a_row():
         assert np.array_equal(out["ctx"][1], out["static"][1])
         assert np.array_equal(out["ctx"][2], out["static"][2])
         assert np.array_equal(out["static"][1], np.unique(node[node >= 0]))
+        # and both against the CPU oracle's reduction (largest (t, eid, role) per node, ascending nodes)
+        u_ref, w_ref = oracle.reduce_latest(node, t, eid, N_call)
+        assert np.array_equal(out["static"][1], u_ref) and np.array_equal(out["static"][2], w_ref)
     ctx.close()
+
+
+def test_static_reduction_skips_and_reports_a_node_id_beyond_the_graph(oracle):
+    """No status word exists without a context: an id >= num_nodes is never used as an index (the tables
+    beyond num_nodes keep an earlier call's contents) and the call answers n_uniq = -1; the next call with
+    clean inputs is unaffected."""
+    from paper_2608_16305_b200 import binding as B
+    rng = np.random.default_rng(32)
+    N, n = 900, 400
+    node, t, eid = _case(rng, N, n, False)
+    bad = node.copy()
+    bad[11] = N + 5            # inside the built-in array, outside this graph
+    bad[12] = 1 << 30          # far outside the array
+    dev = lambda a: torch.from_numpy(a).cuda()
+    for nodes, expect_bad in [(bad, True), (node, False)]:
+        uniq = torch.full((2 * n,), -7, dtype=torch.int32, device="cuda")
+        win = torch.full((2 * n,), -7, dtype=torch.int32, device="cuda")
+        nu = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+        B.reduce_latest_static(dev(nodes), dev(t), dev(eid), N, uniq, win, nu)
+        torch.cuda.synchronize()
+        if expect_bad:
+            assert int(nu.item()) == -1
+        else:
+            u_ref, w_ref = oracle.reduce_latest(nodes, t, eid, N)
+            U = int(nu.item())
+            assert U == len(u_ref)
+            assert np.array_equal(uniq[:U].cpu().numpy(), u_ref) and np.array_equal(win[:U].cpu().numpy(), w_ref)
 
 
 def test_static_reduction_refuses_graphs_beyond_its_built_in_scratch():
