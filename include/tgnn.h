@@ -313,6 +313,9 @@ TGNN_API int tgnn_debug_gemm(tgnn_ctx* ctx, const float* A, int64_t a_rs, int64_
 /* Device status word (0 or the first TGNN_ETIMEOUT / TGNN_EBOUNDS recorded by a
  * kernel) copied to *status_host.  Synchronises the stream. */
 TGNN_API int tgnn_status(tgnn_ctx* ctx, int32_t* status_host, void* stream);
+/* Resets the device status word to 0 (enqueued on `stream`): after a recorded TGNN_ETIMEOUT / TGNN_EBOUNDS
+ * has been read and dealt with, so that the next one can be seen. */
+TGNN_API int tgnn_clear_status(tgnn_ctx* ctx, void* stream);
 /* Number of kernels this context has launched since creation (host counter). */
 TGNN_API int64_t tgnn_kernel_launches(const tgnn_ctx* ctx);
 

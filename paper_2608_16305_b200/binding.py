@@ -36,7 +36,8 @@ EXPORTS = ("tgnn_create", "tgnn_destroy", "tgnn_last_error", "tgnn_param_count",
            "tgnn_controller_create", "tgnn_controller_destroy", "tgnn_controller_begin_batch",
            "tgnn_controller_end_batch", "tgnn_controller_state", "tgnn_backward_scan_scratch", "tgnn_backward_scan",
            "tgnn_build_mixed", "tgnn_set_grad_sync", "tgnn_grad_buffer", "tgnn_apply_gradient", "tgnn_refresh_plan",
-           "tgnn_pack_rows", "tgnn_unpack_rows", "tgnn_debug_get_embeddings", "tgnn_debug_gemm_split")
+           "tgnn_pack_rows", "tgnn_unpack_rows", "tgnn_debug_get_embeddings", "tgnn_debug_gemm_split",
+           "tgnn_clear_status")
 TGNN_STATIC_MAX_NODES = 65536
 
 
@@ -96,6 +97,7 @@ def load_library():
                                         vp]
         lib.tgnn_debug_get_gates.argtypes = [vp, vp, vp, vp]
         lib.tgnn_debug_get_embeddings.argtypes = [vp, vp, vp]
+        lib.tgnn_clear_status.argtypes = [vp, vp]
         lib.tgnn_debug_gemm_split.argtypes = [vp, vp, i64, i64, vp, i64, i64, vp, i64, i32, i32, i32, vp, i32, i32, i32, vp, i64,
                                               i32, u32, vp]
         lib.tgnn_step_mixed_host.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, i32, u32, u64, i64, vp, vp, vp]
@@ -508,6 +510,9 @@ class Tgnn:
             name, cnt, ms = line.rsplit(" ", 2)
             out[name] = (int(cnt), float(ms))
         return out
+
+    def clear_status(self):
+        self._ck(self.lib.tgnn_clear_status(self._h, _stream()))
 
     def status(self) -> int:
         out = C.c_int32(0)

@@ -506,8 +506,9 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
   int dev = 0;
   TGNN_CUDA_OK(ctx, cudaGetDevice(&dev));
   if (dev >= 0 && dev < 64 && attr_bytes[dev] < smem) {
-    TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(gemm_bf16s_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT));
-    attr_bytes[dev] = SMEM_LIMIT;
+    // the largest dynamic size any shape asks for (the static barriers take a few hundred bytes of the 227 KB)
+    TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(gemm_bf16s_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 1024));
+    attr_bytes[dev] = SMEM_LIMIT - 1024;
   }
   {
     KernelScope scope__(ctx, name, s);

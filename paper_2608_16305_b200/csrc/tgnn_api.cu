@@ -804,6 +804,12 @@ int tgnn_status(tgnn_ctx* ctx, int32_t* status_host, void* stream) {
   return TGNN_OK;
 }
 
+int tgnn_clear_status(tgnn_ctx* ctx, void* stream) {
+  if (!ctx) return TGNN_EINVAL;
+  TGNN_CUDA_OK(ctx, cudaMemsetAsync(ctx->ws.status, 0, sizeof(int32_t), S(stream)));
+  return TGNN_OK;
+}
+
 int tgnn_profile_begin(tgnn_ctx* ctx) {
   if (!ctx) return TGNN_EINVAL;
   ctx->prof.used = 0;
