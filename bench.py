@@ -205,7 +205,8 @@ def run_ours(args, rank, world, device):
     dw = T.DeviceWorkload(stream, device=device, efeat=efeat, batches=range(first - 1, first + span),
                           embed_aux=args.embed_aux)
     weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed, model=args.model)
-    math_mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST}[args.math]
+    math_mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST,
+                 "bf16x3": B.TGNN_MATH_BF16X3}[args.math]
     tr = T.Trainer(dw, weights, math_mode=math_mode, model=args.model)
     if args.no_graph:
         tr.lib.set_graph_replay(False)
@@ -434,7 +435,8 @@ def run_partitioned(args, rank, world, device):
     torch.cuda.synchronize()
     prep_s = time.time() - t0
     weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed, model=args.model)
-    math_mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST}[args.math]
+    math_mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST,
+                 "bf16x3": B.TGNN_MATH_BF16X3}[args.math]
     tr = T.Trainer(dw, weights, math_mode=math_mode, model=args.model)
     tr.lib.set_grad_sync(True)
     ctl = B.Controller(alpha=0.1, beta=0.1, tau_g=1.6, tau_c=0.5, K=K_sync)
@@ -737,7 +739,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--math", default=os.environ.get("TGNN_BENCH_MATH", "tf32"), choices=["fp32", "tf32", "tf32fast"])
+    ap.add_argument("--math", default=os.environ.get("TGNN_BENCH_MATH", "tf32"), choices=["fp32", "tf32", "tf32fast", "bf16x3"])
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--workload", default=WORKLOAD, choices=sorted(wl.CONFIGS),
                     help="default: large, the largest single-GPU configuration (the headline line); the others are parity-test cases")

@@ -66,6 +66,10 @@ enum {
   TGNN_MATH_FP32 = 0,     /* fp32 FMA tiles */
   TGNN_MATH_TF32 = 1,     /* tcgen05 tensor cores: every operand is split into a TF32 head and a TF32
                              tail (3 MMAs per product, fp32 accumulation in TMEM), close to fp32 accuracy */
+  TGNN_MATH_BF16X3 = 3,   /* as TGNN_MATH_TF32, except that the three products over the sampled-neighbor rows (key/value
+                             projection, its input gradient and its weight gradient) hold each fp32 operand as two bf16
+                             numbers (hi + lo, 16 mantissa bits) and run as three bf16 tensor-core passes with fp32
+                             accumulation: more accurate than one TF32 pass, half the tensor time of the TF32 split */
   TGNN_MATH_TF32_FAST = 2 /* tcgen05 tensor cores, single TF32 pass in the forward projections (the gradient
                              products keep the split).  Outputs stay within 2e-3, but gradient tensors whose
                              terms cancel (time encoder, W_k) can be off by ~1e-2 of their largest entry. */

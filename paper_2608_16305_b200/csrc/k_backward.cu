@@ -290,11 +290,15 @@ __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __r
 // One warp per root: backward of the weighted sum, the softmax and the scaled dot products, on the
 // root's K | V rows staged in shared memory.  Lane p < H*k owns the (head, slot) pair p for the
 // probability and logit gradients; afterwards the lanes own columns and write dQ and the dK | dV rows.
+// SPLIT: the key/value gradient rows are written as two bf16 planes (hi, lo; row pitch ld_s, plane_s elements
+// apart) for the split-bf16 products that consume them, instead of as fp32 rows.
+template <bool SPLIT>
 __global__ void __launch_bounds__(256) attention_bwd_kernel(const float* __restrict__ Q, const float* __restrict__ KV,
                                                             const float* __restrict__ alpha,
                                                             const float* __restrict__ dcat_o,
                                                             const int32_t* __restrict__ cnt, int n, int d, int H, int k,
-                                                            float* __restrict__ dQ, float* __restrict__ dKV) {
+                                                            float* __restrict__ dQ, float* __restrict__ dKV,
+                                                            __nv_bfloat16* __restrict__ dkv_hi, int64_t plane_s, int ld_s) {
   extern __shared__ __align__(16) float sm[];
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   const int i = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
@@ -338,23 +342,48 @@ __global__ void __launch_bounds__(256) attention_bwd_kernel(const float* __restr
     dl[p] = g;
   }
   __syncwarp();
-  for (int e = lane; e < d; e += 32) {
-    const int h = e / dh;
-    const float qe = Qs[e], dae = das[e];
-    float dq = 0.f;
-    for (int s = 0; s < k; ++s) {
-      float* row = dKV + ((int64_t)i * k + s) * 2 * d;
-      if (s < c) {
-        const float g = dl[h * k + s];
-        dq = fmaf(g, Ks[s * d + e], dq);
-        row[e] = g * qe;
-        row[d + e] = al[h * k + s] * dae;
-      } else {
-        row[e] = 0.f;
-        row[d + e] = 0.f;
+  if (!SPLIT) {
+    for (int e = lane; e < d; e += 32) {
+      const int h = e / dh;
+      const float qe = Qs[e], dae = das[e];
+      float dq = 0.f;
+      for (int s = 0; s < k; ++s) {
+        float* row = dKV + ((int64_t)i * k + s) * 2 * d;
+        if (s < c) {
+          const float g = dl[h * k + s];
+          dq = fmaf(g, Ks[s * d + e], dq);
+          row[e] = g * qe;
+          row[d + e] = al[h * k + s] * dae;
+        } else {
+          row[e] = 0.f;
+          row[d + e] = 0.f;
+        }
       }
+      dQ[(int64_t)i * d + e] = dq;
     }
-    dQ[(int64_t)i * d + e] = dq;
+  } else {
+    // a lane owns two neighbouring columns (d is even): each (hi, lo) pair goes out as one 32-bit word per plane
+    for (int e = 2 * lane; e < d; e += 64) {
+      const int h0 = e / dh, h1 = (e + 1) / dh;
+      const float q0 = Qs[e], q1 = Qs[e + 1], a0 = das[e], a1 = das[e + 1];
+      float dq0 = 0.f, dq1 = 0.f;
+      for (int s = 0; s < k; ++s) {
+        uint32_t* hi = reinterpret_cast<uint32_t*>(dkv_hi + ((int64_t)i * k + s) * ld_s);
+        uint32_t* lo = reinterpret_cast<uint32_t*>(dkv_hi + plane_s + ((int64_t)i * k + s) * ld_s);
+        uint32_t kh = 0u, kl = 0u, vh = 0u, vl = 0u;
+        if (s < c) {
+          const float g0 = dl[h0 * k + s], g1 = dl[h1 * k + s];
+          dq0 = fmaf(g0, Ks[s * d + e], dq0);
+          dq1 = fmaf(g1, Ks[s * d + e + 1], dq1);
+          split_bf16_pair(g0 * q0, g1 * q1, &kh, &kl);
+          split_bf16_pair(al[h0 * k + s] * a0, al[h1 * k + s] * a1, &vh, &vl);
+        }
+        hi[e >> 1] = kh; lo[e >> 1] = kl;
+        hi[(d + e) >> 1] = vh; lo[(d + e) >> 1] = vl;
+      }
+      dQ[(int64_t)i * d + e] = dq0;
+      dQ[(int64_t)i * d + e + 1] = dq1;
+    }
   }
 }
 
@@ -970,19 +999,36 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       static int attr_bytes = 0;
       const int need = (int)attn_smem_bytes(d, H, k, wpb);
       if (attr_bytes < need) {
-        TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(attention_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, need));
+        TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(attention_bwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, need));
+        TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(attention_bwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, need));
         attr_bytes = need;
       }
     }
+    const bool split = ctx->split_buf != nullptr && ctx->images_fresh;
+    SplitMat dkvs = ctx->dkvs, zs = ctx->zs;
+    dkvs.rows = NB; zs.rows = NB;
     {
       KernelScope scope__(ctx, "attention_bwd", s);
-      attention_bwd_kernel<<<(R + wpb - 1) / wpb, wpb * 32, attn_smem_bytes(d, H, k, wpb), s>>>(
-          w.Q, w.KV, w.alpha, w.dcat_o, ctx->e_cnt, R, d, H, k, w.dQ, w.dKV);
+      if (split)   // the key/value gradient leaves the kernel as bf16 planes, the form its two consumers read
+        attention_bwd_kernel<true><<<(R + wpb - 1) / wpb, wpb * 32, attn_smem_bytes(d, H, k, wpb), s>>>(
+            w.Q, w.KV, w.alpha, w.dcat_o, ctx->e_cnt, R, d, H, k, w.dQ, nullptr, reinterpret_cast<__nv_bfloat16*>(dkvs.hi),
+            dkvs.plane_stride, (int)dkvs.ld);
+      else
+        attention_bwd_kernel<false><<<(R + wpb - 1) / wpb, wpb * 32, attn_smem_bytes(d, H, k, wpb), s>>>(
+            w.Q, w.KV, w.alpha, w.dcat_o, ctx->e_cnt, R, d, H, k, w.dQ, w.dKV, nullptr, 0, 0);
     }
     TGNN_LAUNCH_OK(ctx, "attention_bwd");
     RC(fork_to(ctx, s, sa));
     RC(fork_to(ctx, s, sb));
-    RC(grad_w(ctx, w.dKV, 2 * d, w.Z, ctx->ld_kv, NB, nullptr, 2 * d, (int)L.dkv, G + L.wk, G + L.bk, "dW_kv", sa));
+    if (split) {
+      // dW_kv = dKV^T Z over the neighbor rows; Z's column of ones yields the bias gradient as the last column
+      SplitMat a = dkvs, b = zs;
+      a.rows = NB; a.cols = 2 * d; b.rows = NB; b.cols = L.dkv + 1;
+      RC(launch_gemm_split(ctx, a, b, 1, G + L.wk, L.dkv, 2 * d, (int)L.dkv + 1, NB, nullptr, 0, 1, 1 << 20, "dW_kv", sa, 0, 0,
+                           (int)L.dkv, G + L.bk));
+    } else {
+      RC(grad_w(ctx, w.dKV, 2 * d, w.Z, ctx->ld_kv, NB, nullptr, 2 * d, (int)L.dkv, G + L.wk, G + L.bk, "dW_kv", sa));
+    }
     // time-encoder gradient through the attention inputs (side stream b)
     const size_t tg_smem = (size_t)8 * 2 * d * sizeof(double);
     // gradient w.r.t. the memory columns and the time-encoding columns of Z, side by side in dZmp.  With the
@@ -1001,7 +1047,11 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_q");
     cudaStream_t s_tgz = sb;  // where the time-encoder sum over the neighbor rows runs
-    if (merged_dz) {
+    if (split) {
+      RC(launch_gemm_split(ctx, dkvs, ctx->wz_s, 0, w.dZmp, 2 * d, NB, 2 * d, 2 * d, nullptr, 0, 0, 1, "dZ", s));
+      RC(fork_to(ctx, s, sa));
+      s_tgz = sa;
+    } else if (merged_dz) {
       RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, 0, NB, nullptr, 2 * d, 2 * d, w.dZmp, 2 * d, "dZ", s, SITE_DZ + 1));
       RC(fork_to(ctx, s, sa));
       s_tgz = sa;
@@ -1017,7 +1067,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     TGNN_LAUNCH_OK(ctx, "time_grad_z");
     RC(wait_mark(ctx, s, dzq_done));  // the scatter below needs dzq
     if (ctx->have_update) {
-      if (!merged_dz)
+      if (!merged_dz && !split)
         RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, 0, NB, nullptr, 2 * d, d, w.dZmp, 2 * d, "dZ_mem", s));
       {
         KernelScope scope__(ctx, "scatter_dmem", s);

@@ -149,17 +149,158 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_kernel(const void* __r
     for (int q = lane; q < d; q += 32) Zq[(int64_t)i * 2 * d + d + q] = time_encode(time_w[q], time_b[q], 0.f);
 }
 
+// The static part for the split-bf16 products: the same rows written as two bf16 planes (hi, lo; row pitch ld
+// elements, planes plane_s elements apart) -- columns [d, d + de) edge features, [d + de, dkv) time encoding,
+// column dkv a constant 1 (it turns the weight-gradient product's last column into the bias gradient), zeros up
+// to ld; an empty slot is a row of zeros.  Values travel as pairs of neighbouring columns packed into 32-bit
+// words (d and de are even).  bf16 features are exact in the hi plane; fp32 features and the encodings are split.
+__global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const void* __restrict__ efeat, int feat_bf16,
+                                                                    const float* __restrict__ time_w,
+                                                                    const float* __restrict__ time_b, int d, int de, int k,
+                                                                    const double* __restrict__ times, int n,
+                                                                    const int32_t* __restrict__ nbr,
+                                                                    const int32_t* __restrict__ eid,
+                                                                    const double* __restrict__ ts, int ld,
+                                                                    __nv_bfloat16* __restrict__ z_hi, int64_t plane_s,
+                                                                    float* __restrict__ z_dt, float* __restrict__ Zq) {
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  const int nb_rows = n * k;
+  const int dkv = 2 * d + de;
+  const int fp = de >> 1, tp = d >> 1;          // feature pairs, encoding pairs per row
+  const int groups = (nb_rows + ZS_ROWS - 1) / ZS_ROWS;
+  constexpr int FP_MAX = 4, TP_MAX = 2;         // pairs per lane held in registers: de <= 256, d <= 128
+  const bool regs = fp <= 32 * FP_MAX && tp <= 32 * TP_MAX;
+  float tw[TP_MAX][2], tb[TP_MAX][2];
+#pragma unroll
+  for (int u = 0; u < TP_MAX; ++u) {
+    const int q = 2 * (lane + 32 * u);
+    const bool in = regs && q < d;
+    tw[u][0] = in ? time_w[q] : 0.f; tw[u][1] = in ? time_w[q + 1] : 0.f;
+    tb[u][0] = in ? time_b[q] : 0.f; tb[u][1] = in ? time_b[q + 1] : 0.f;
+  }
+  for (int gidx = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; gidx < groups; gidx += warps) {
+    const int r0 = gidx * ZS_ROWS;
+    int my_nbr = -1, my_eid = 0;
+    float my_dt = 0.f;
+    if (lane < ZS_ROWS && r0 + lane < nb_rows) {
+      const int r = r0 + lane;
+      my_nbr = nbr[r];
+      my_eid = eid[r];
+      my_dt = (float)(times[r / k] - ts[r]);
+    }
+    // feature pairs of both rows first (the dependent chain slot -> event id -> feature row is paid once)
+    uint32_t fa[ZS_ROWS][FP_MAX], fb[ZS_ROWS][FP_MAX];   // bf16 table: fa = the pair as stored; fp32 table: fa, fb = the two floats
+    int v_nbr[ZS_ROWS], v_eid[ZS_ROWS];
+    float v_dt[ZS_ROWS];
+#pragma unroll
+    for (int j = 0; j < ZS_ROWS; ++j) {
+      v_nbr[j] = __shfl_sync(0xffffffffu, my_nbr, j);
+      v_dt[j] = __shfl_sync(0xffffffffu, my_dt, j);
+      v_eid[j] = __shfl_sync(0xffffffffu, my_eid, j);
+      if (regs && v_nbr[j] >= 0) {
+#pragma unroll
+        for (int u = 0; u < FP_MAX; ++u) {
+          const int q = lane + 32 * u;
+          fa[j][u] = 0u; fb[j][u] = 0u;
+          if (q < fp) {
+            if (feat_bf16) {
+              fa[j][u] = __ldg(reinterpret_cast<const uint32_t*>(efeat) + (int64_t)v_eid[j] * fp + q);
+            } else {
+              const uint2 x = __ldg(reinterpret_cast<const uint2*>(efeat) + (int64_t)v_eid[j] * fp + q);
+              fa[j][u] = x.x; fb[j][u] = x.y;
+            }
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < ZS_ROWS; ++j) {
+      const int r = r0 + j;
+      if (r >= nb_rows) break;
+      uint32_t* hi = reinterpret_cast<uint32_t*>(z_hi + (int64_t)r * ld);
+      uint32_t* lo = reinterpret_cast<uint32_t*>(z_hi + plane_s + (int64_t)r * ld);
+      if (v_nbr[j] < 0) {
+        for (int q = lane; q < (ld >> 1); q += 32) { hi[q] = 0u; lo[q] = 0u; }   // the memory part too: nobody else writes this row
+        if (lane == 0) z_dt[r] = -1.f;
+        continue;
+      }
+      const float dtf = v_dt[j];
+      if (regs) {
+#pragma unroll
+        for (int u = 0; u < FP_MAX; ++u) {
+          const int q = lane + 32 * u;
+          if (q < fp) {
+            uint32_t h = fa[j][u], l = 0u;
+            if (!feat_bf16) split_bf16_pair(__uint_as_float(fa[j][u]), __uint_as_float(fb[j][u]), &h, &l);
+            hi[(d >> 1) + q] = h; lo[(d >> 1) + q] = l;
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < TP_MAX; ++u) {
+          const int q = lane + 32 * u;
+          if (q < tp) {
+            uint32_t h, l;
+            split_bf16_pair(time_encode(tw[u][0], tb[u][0], dtf), time_encode(tw[u][1], tb[u][1], dtf), &h, &l);
+            hi[((d + de) >> 1) + q] = h; lo[((d + de) >> 1) + q] = l;
+          }
+        }
+      } else {   // very wide rows: straight from memory, pair by pair
+        for (int q = lane; q < fp; q += 32) {
+          uint32_t h, l = 0u;
+          if (feat_bf16) {
+            h = __ldg(reinterpret_cast<const uint32_t*>(efeat) + (int64_t)v_eid[j] * fp + q);
+          } else {
+            const uint2 x = __ldg(reinterpret_cast<const uint2*>(efeat) + (int64_t)v_eid[j] * fp + q);
+            split_bf16_pair(__uint_as_float(x.x), __uint_as_float(x.y), &h, &l);
+          }
+          hi[(d >> 1) + q] = h; lo[(d >> 1) + q] = l;
+        }
+        for (int q = lane; q < tp; q += 32) {
+          uint32_t h, l;
+          split_bf16_pair(time_encode(time_w[2 * q], time_b[2 * q], dtf), time_encode(time_w[2 * q + 1], time_b[2 * q + 1], dtf), &h, &l);
+          hi[((d + de) >> 1) + q] = h; lo[((d + de) >> 1) + q] = l;
+        }
+      }
+      // column dkv = 1, then zeros up to the row pitch (dkv is even, the pitch a multiple of 8)
+      for (int q = (dkv >> 1) + lane; q < (ld >> 1); q += 32) { hi[q] = q == (dkv >> 1) ? 0x3f80u : 0u; lo[q] = 0u; }
+      if (lane == 0) z_dt[r] = dtf;
+    }
+  }
+  // the Phi(0) half of z_q (fp32: the query projection is not one of the split products)
+  for (int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps)
+    for (int q = lane; q < d; q += 32) Zq[(int64_t)i * 2 * d + d + q] = time_encode(time_w[q], time_b[q], 0.f);
+}
+
 // Memory part.  Rows [0, n*k): columns [0, d) of Z for the valid slots.  Rows [n*k, n*k + n): the
 // memory half of z_q and of cat_o.
+// z_hi != nullptr: the neighbor rows go to the two bf16 planes of the split products instead (pitch ld_s, planes
+// plane_s apart), as pairs of columns packed into 32-bit words.
 __global__ void __launch_bounds__(256) gather_z_memory_kernel(const float* __restrict__ memory, int d, int k,
                                                               const int32_t* __restrict__ nodes, int n,
                                                               const int32_t* __restrict__ nbr, int ld,
                                                               float* __restrict__ Z, float* __restrict__ Zq,
-                                                              float* __restrict__ cat_o) {
+                                                              float* __restrict__ cat_o, __nv_bfloat16* __restrict__ z_hi,
+                                                              int64_t plane_s, int ld_s) {
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   const int nb_rows = n * k;
-  for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < nb_rows + n; r += warps) {
+  if (z_hi != nullptr) {
+    // one thread per pair of columns, rows back to back: every lane of every warp moves data
+    const int hp = d >> 1;
+    const int64_t total = (int64_t)nb_rows * hp;
+    for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+      const int r = (int)(idx / hp), q = (int)(idx - (int64_t)r * hp);
+      const int nb = __ldg(nbr + r);
+      if (nb < 0) continue;
+      const float2 x = __ldg(reinterpret_cast<const float2*>(memory + (int64_t)nb * d) + q);
+      uint32_t h, l;
+      split_bf16_pair(x.x, x.y, &h, &l);
+      reinterpret_cast<uint32_t*>(z_hi + (int64_t)r * ld_s)[q] = h;
+      reinterpret_cast<uint32_t*>(z_hi + plane_s + (int64_t)r * ld_s)[q] = l;
+    }
+  }
+  for (int r = (z_hi != nullptr ? nb_rows : 0) + ((blockIdx.x * blockDim.x + threadIdx.x) >> 5); r < nb_rows + n; r += warps) {
     if (r < nb_rows) {
       const int nb = nbr[r];
       if (nb >= 0) warp_copy_f32(Z + (int64_t)r * ld, memory + (int64_t)nb * d, d, lane);
@@ -264,7 +405,12 @@ int launch_embed_static(tgnn_ctx* ctx, const double* times, int n, const int32_t
   Workspace& w = ctx->ws;
   {
     KernelScope scope__(ctx, "gather_z_static", s);
-    gather_z_static_kernel<<<(n * c.k / ZS_ROWS + n + 7) / 8 + 1, 256, 0, s>>>(ctx->efeat, c.feat_dtype == TGNN_BF16, ctx->params + L.time_w,
+    if (ctx->split_buf != nullptr && ctx->z_split)
+      gather_z_static_split_kernel<<<(n * c.k / ZS_ROWS + n + 7) / 8 + 1, 256, 0, s>>>(
+          ctx->efeat, c.feat_dtype == TGNN_BF16, ctx->params + L.time_w, ctx->params + L.time_b, c.d, c.d_e, c.k, times, n, nbr,
+          eid, ts, (int)ctx->zs.ld, reinterpret_cast<__nv_bfloat16*>(ctx->zs.hi), ctx->zs.plane_stride, w.z_dt, w.Zq);
+    else
+      gather_z_static_kernel<<<(n * c.k / ZS_ROWS + n + 7) / 8 + 1, 256, 0, s>>>(ctx->efeat, c.feat_dtype == TGNN_BF16, ctx->params + L.time_w,
                                                           ctx->params + L.time_b, c.d, c.d_e, c.k, times, n, nbr, eid, ts,
                                                           ctx->ld_kv, w.Z, w.z_dt, w.Zq);
   }
@@ -289,21 +435,28 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
     return TGNN_OK;
   }
   const int rows = n * k + n;
+  // split-bf16 operands: the attention inputs are written as bf16 planes, complete before the product starts
+  const bool split = ctx->split_buf != nullptr && ctx->images_fresh;
   if (!ctx->z_static_done) {
+    ctx->z_split = split;
     const int rc0 = launch_embed_static(ctx, times, n, nbr, eid, ts, s);
     if (rc0) return rc0;
+  } else if (ctx->z_split != split) {
+    return set_error(ctx, TGNN_ESTATE, "embed: the static half of the attention inputs was gathered in the other operand format");
   }
   ctx->z_static_done = false;
   // In the tensor-core modes the key/value projection reads the neighbors' memory rows straight from
   // the table (row-indirect A), so the copy of those rows into Z -- still needed by the backward pass,
   // like the root rows by the query and output projections -- leaves the critical chain for a side stream.
-  const bool indirect = c.math_mode != TGNN_MATH_FP32;
+  const bool indirect = c.math_mode != TGNN_MATH_FP32 && !split;
   int rc = fork_to(ctx, s, ctx->side[0]);
   if (rc) return rc;
   cudaStream_t sg = indirect ? ctx->side[0] : s;
   {
     KernelScope scope__(ctx, "gather_z_memory", sg);
-    gather_z_memory_kernel<<<(rows + 7) / 8, 256, 0, sg>>>(ctx->memory, d, k, nodes, n, nbr, ctx->ld_kv, w.Z, w.Zq, w.cat_o);
+    gather_z_memory_kernel<<<(rows + 7) / 8, 256, 0, sg>>>(ctx->memory, d, k, nodes, n, nbr, ctx->ld_kv, w.Z, w.Zq, w.cat_o,
+                                                           split ? reinterpret_cast<__nv_bfloat16*>(ctx->zs.hi) : nullptr,
+                                                           ctx->zs.plane_stride, (int)ctx->zs.ld);
   }
   TGNN_LAUNCH_OK(ctx, "gather_z_memory");
   if (!indirect) {  // the query projection below runs on the side stream and needs the rows just gathered
@@ -316,7 +469,14 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
   g.C = w.KV; g.ldc = 2 * d; g.M = n * k; g.N = 2 * d; g.K = (int)L.dkv;
   g.bias = ctx->params + L.bk; g.split_k = 1; g.site = SITE_KV + 1;
   if (indirect) { g.a_idx = nbr; g.a_tab = ctx->memory; g.a_tab_cols = d; }
-  rc = launch_gemm(ctx, g, "kv_proj", s);
+  if (split) {
+    SplitMat zs = ctx->zs;
+    zs.rows = n * k;
+    zs.cols = L.dkv;   // the forward product stops before the column of ones
+    rc = launch_gemm_split(ctx, zs, ctx->wkv_s, 0, w.KV, 2 * d, n * k, 2 * d, (int)L.dkv, ctx->params + L.bk, 0, 0, 1, "kv_proj", s);
+  } else {
+    rc = launch_gemm(ctx, g, "kv_proj", s);
+  }
   if (rc) return rc;
   g = GemmArgs{};
   g.A = w.Zq; g.a_rs = 2 * d; g.a_cs = 1;

@@ -91,7 +91,7 @@ int launch_gemm(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t
   if (g.split_k > 1 && !g.accumulate) return set_error(ctx, TGNN_EINVAL, "gemm %s: split_k needs accumulate", name);
   if (ctx->cfg.math_mode != TGNN_MATH_FP32) {
     GemmArgs gp = g;
-    if (ctx->cfg.math_mode == TGNN_MATH_TF32) gp.precise = 1;
+    if (ctx->cfg.math_mode != TGNN_MATH_TF32_FAST) gp.precise = 1;
     const int rc = launch_gemm_tf32(ctx, gp, name, s);
     if (rc != 1) return rc;  // 1: shape not handled by the tensor-core kernel, use the FMA tiles
   }

@@ -58,6 +58,10 @@ struct BfArgs {
   int ksteps_total;           // MMA steps of 16 over the whole contraction
   int a_slot_bytes, b_slot_bytes, n_a_slots, n_b_slots;
   int b_chunks;               // MN-major: 64-column chunks per B tile
+  // accumulate mode: column `extra_col` of the product (if >= 0) is added to extra_out[row] instead of C --
+  // a column of ones appended to B turns that column into the row sums of A, i.e. a bias gradient
+  int extra_col;
+  float* extra_out;
   int32_t* status;
   int debug_withhold;         // test hook: the MMA warp skips this many slot releases (an empty-slot wait then expires)
   unsigned spin_limit;
@@ -327,7 +331,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
               if (col + 2 < it.n_valid) b4.z = bp[2];
               if (col + 3 < it.n_valid) b4.w = bp[3];
             }
-            const bool full4 = col + 3 < it.n_valid;
+            const int xc = g.extra_col - it.n0 - col;   // 0..3: one of this lane's columns is the extra column
+            const bool full4 = col + 3 < it.n_valid && (xc < 0 || xc > 3);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               const int rr = j * 8 + sub;
@@ -340,10 +345,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
                   if (full4 && c_vec) {
                     atomicAdd(reinterpret_cast<float4*>(cp), v);
                   } else {
-                    atomicAdd(cp, v.x);
-                    if (col + 1 < it.n_valid) atomicAdd(cp + 1, v.y);
-                    if (col + 2 < it.n_valid) atomicAdd(cp + 2, v.z);
-                    if (col + 3 < it.n_valid) atomicAdd(cp + 3, v.w);
+                    const float vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int e2 = 0; e2 < 4; ++e2)
+                      if (col + e2 < it.n_valid) atomicAdd(e2 == xc ? g.extra_out + row : cp + e2, vv[e2]);
                   }
                 } else {
                   if (g.relu) { v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); v.z = fmaxf(v.z, 0.f); v.w = fmaxf(v.w, 0.f); }
@@ -408,6 +413,35 @@ __global__ void __launch_bounds__(256) split_rows_kernel(const float* __restrict
   }
 }
 
+// Split planes of the attention layer's key/value weights for this step's two big products:
+//   wkv[n, k] = W_kv[n, k]                      (n < 2d, k < dkv: the forward projection's B operand)
+//   wz[n, k]  = W_kv[k, col(n)]                 (n < 2d, k < 2d: the input gradient toward the memory columns,
+//               col(n) = n for n < d, and the time-encoding columns, col(n) = d + de + (n - d) otherwise)
+// Padding columns of the planes are zero.
+__global__ void __launch_bounds__(256) prep_split_weights_kernel(const float* __restrict__ Wkv, int d, int de,
+                                                                 __nv_bfloat16* __restrict__ wkv_hi, int64_t wkv_plane, int ld_kv,
+                                                                 __nv_bfloat16* __restrict__ wz_hi, int64_t wz_plane, int ld_z) {
+  const int dkv = 2 * d + de, n_rows = 2 * d;
+  const int64_t n_kv = (int64_t)n_rows * ld_kv, n_z = (int64_t)n_rows * ld_z;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n_kv + n_z; i += (int64_t)gridDim.x * blockDim.x) {
+    float v = 0.f;
+    __nv_bfloat16 *hi, *lo;
+    if (i < n_kv) {
+      const int n = (int)(i / ld_kv), k = (int)(i - (int64_t)n * ld_kv);
+      if (k < dkv) v = Wkv[(int64_t)n * dkv + k];
+      hi = wkv_hi + i; lo = wkv_hi + wkv_plane + i;
+    } else {
+      const int64_t j = i - n_kv;
+      const int n = (int)(j / ld_z), k = (int)(j - (int64_t)n * ld_z);
+      if (k < n_rows) v = Wkv[(int64_t)k * dkv + (n < d ? n : d + de + (n - d))];
+      hi = wz_hi + j; lo = wz_hi + wz_plane + j;
+    }
+    const __nv_bfloat16 h = __float2bfloat16_rn(v);
+    *hi = h;
+    *lo = __float2bfloat16_rn(v - __bfloat162float(h));
+  }
+}
+
 typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                       const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                       CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -443,6 +477,20 @@ bool encode_split_map(CUtensorMap* map, const SplitMat& m, int box_rows) {
 
 }  // namespace
 
+int launch_prep_split_weights(tgnn_ctx* ctx, cudaStream_t s) {
+  if (!ctx->split_buf) return TGNN_OK;
+  const int d = ctx->cfg.d, de = ctx->cfg.d_e;
+  {
+    KernelScope scope__(ctx, "prep_split_weights", s);
+    prep_split_weights_kernel<<<148, 256, 0, s>>>(ctx->params + ctx->L.wk, d, de, reinterpret_cast<__nv_bfloat16*>(ctx->wkv_s.hi),
+                                                  ctx->wkv_s.plane_stride, (int)ctx->wkv_s.ld,
+                                                  reinterpret_cast<__nv_bfloat16*>(ctx->wz_s.hi), ctx->wz_s.plane_stride,
+                                                  (int)ctx->wz_s.ld);
+  }
+  TGNN_LAUNCH_OK(ctx, "prep_split_weights");
+  return TGNN_OK;
+}
+
 int launch_split_rows(tgnn_ctx* ctx, const float* X, int64_t ld_in, int64_t rows, int cols, const int32_t* dev_rows,
                       const SplitMat& out, int ones_col, const char* name, cudaStream_t s) {
   if (rows <= 0) return TGNN_OK;
@@ -463,7 +511,7 @@ int launch_split_rows(tgnn_ctx* ctx, const float* X, int64_t ld_in, int64_t rows
 // split_k > 1 needs accumulate (C holds valid data; partial sums are added atomically).
 int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int mn_major, float* C, int64_t ldc, int M, int N,
                       int K, const float* bias, int relu, int accumulate, int split_k, const char* name, cudaStream_t s,
-                      int debug_withhold, unsigned spin_limit) {
+                      int debug_withhold, unsigned spin_limit, int extra_col, float* extra_out) {
   if (M <= 0 || N <= 0) return TGNN_OK;
   if (K <= 0) return set_error(ctx, TGNN_EINVAL, "gemm %s: empty contraction", name);
   if (split_k > 1 && !accumulate) return set_error(ctx, TGNN_EINVAL, "gemm %s: split_k needs accumulate", name);
@@ -471,6 +519,8 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
   a.C = C; a.ldc = ldc; a.M = M; a.N = N; a.K = K; a.bias = bias; a.relu = relu; a.accumulate = accumulate;
   a.mn_major = mn_major ? 1 : 0;
   a.status = ctx->ws.status;
+  a.extra_col = (extra_out && accumulate) ? extra_col : -1;
+  a.extra_out = extra_out;
   a.debug_withhold = debug_withhold;
   a.spin_limit = spin_limit ? spin_limit : SPIN_LIMIT;
   a.m_tiles = (M + BM - 1) / BM;

@@ -913,7 +913,7 @@ namespace tgnn {
 size_t plan_weight_sites(tgnn_ctx* ctx) {
   const ParamLayout& L = ctx->L;
   const int d = (int)L.d, de = (int)L.de;
-  const bool all_precise = ctx->cfg.math_mode == TGNN_MATH_TF32;
+  const bool all_precise = ctx->cfg.math_mode != TGNN_MATH_TF32_FAST;
   struct Def { int id; int64_t w_off, ld; int major, N, K, col0, n_split, col1, M_cap, split_acc, grad; };
   const int U = ctx->U_cap, R = ctx->R_cap, NB = ctx->NB_cap, Q2 = 2 * ctx->nq_cap;
   const int gd = (int)L.gates * d;              // rows of the update cell's matrices
@@ -962,7 +962,7 @@ int launch_prep_weights(tgnn_ctx* ctx, cudaStream_t s) {
     prep_weights_kernel<<<grid, 256, 0, s>>>(ctx->sites_dev, ctx->params, ctx->images);
   }
   TGNN_LAUNCH_OK(ctx, "prep_weights");
-  return TGNN_OK;
+  return launch_prep_split_weights(ctx, s);   // the split planes of the key/value weights, when that mode is on
 }
 
 }  // namespace tgnn

@@ -61,7 +61,8 @@ int check_config(const tgnn_config* c) {
   if (c->k < 1 || c->k > 32 || c->heads * c->k > 1024) return TGNN_ESHAPE;
   if (c->feat_dtype != TGNN_F32 && c->feat_dtype != TGNN_BF16) return TGNN_EINVAL;
   if (c->max_events < 1 || c->max_roots < 3 || c->max_events > (1 << 24) || c->max_roots > (1 << 24)) return TGNN_EINVAL;
-  if (c->math_mode != TGNN_MATH_FP32 && c->math_mode != TGNN_MATH_TF32 && c->math_mode != TGNN_MATH_TF32_FAST) return TGNN_EINVAL;
+  if (c->math_mode != TGNN_MATH_FP32 && c->math_mode != TGNN_MATH_TF32 && c->math_mode != TGNN_MATH_TF32_FAST &&
+      c->math_mode != TGNN_MATH_BF16X3) return TGNN_EINVAL;
   if (c->model != TGNN_MODEL_TGN && c->model != TGNN_MODEL_JODIE) return TGNN_EINVAL;
   if (c->embed_aux != 0 && c->embed_aux != 1) return TGNN_EINVAL;
   if (!(c->lr >= 0.f) || !(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f) || !(c->eps > 0.f))
@@ -262,6 +263,27 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
          cudaMalloc((void**)&ctx->sites_dev, sizeof(ctx->sites)) == cudaSuccess &&
          cudaMemcpy(ctx->sites_dev, ctx->sites, sizeof(ctx->sites), cudaMemcpyHostToDevice) == cudaSuccess;
   }
+  ctx->split_buf = nullptr;
+  if (ok && cfg->math_mode == TGNN_MATH_BF16X3 && cfg->model == TGNN_MODEL_TGN) {
+    const auto up8 = [](int64_t x) { return (x + 7) / 8 * 8; };
+    const int64_t d = cfg->d, dkv = ctx->L.dkv, NB = ctx->NB_cap;
+    ctx->zs = SplitMat{nullptr, up8(dkv + 1), 0, NB, dkv + 1};
+    ctx->dkvs = SplitMat{nullptr, up8(2 * d), 0, NB, 2 * d};
+    ctx->wkv_s = SplitMat{nullptr, up8(dkv), 0, 2 * d, dkv};
+    ctx->wz_s = SplitMat{nullptr, up8(2 * d), 0, 2 * d, 2 * d};
+    SplitMat* ms[4] = {&ctx->zs, &ctx->dkvs, &ctx->wkv_s, &ctx->wz_s};
+    size_t off = 0;
+    for (SplitMat* m : ms) {
+      m->plane_stride = (m->rows * m->ld + 127) / 128 * 128;
+      off += (size_t)(2 * m->plane_stride * 2);
+    }
+    ok = cudaMalloc(&ctx->split_buf, off) == cudaSuccess && cudaMemset(ctx->split_buf, 0, off) == cudaSuccess;
+    off = 0;
+    for (SplitMat* m : ms) {
+      m->hi = (char*)ctx->split_buf + off;
+      off += (size_t)(2 * m->plane_stride * 2);
+    }
+  }
   ctx->ev_next = 0;
   ctx->n_graphs = 0;
   ctx->graphs_enabled = 1;
@@ -272,6 +294,7 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
   if (!ok) {
     cudaGetLastError();
     cudaFree(ctx->images);
+    cudaFree(ctx->split_buf);
     cudaFree(ctx->sites_dev);
     cudaFree(ctx->pack_dev);
     for (int i = 0; i < 2; ++i) if (ctx->pack_host[i]) cudaFreeHost(ctx->pack_host[i]);
@@ -296,6 +319,7 @@ int tgnn_destroy(tgnn_ctx* ctx) {
   for (int i = 0; i < 2; ++i) cudaStreamDestroy(ctx->side[i]);
   for (int i = 0; i < 32; ++i) cudaEventDestroy(ctx->ev[i]);
   cudaFree(ctx->images);
+  cudaFree(ctx->split_buf);
   cudaFree(ctx->sites_dev);
   cudaFree(ctx->pack_dev);
   for (int i = 0; i < 2; ++i) {
@@ -455,6 +479,7 @@ int step_body(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q, bool has_mask, flo
   } side_guard(ctx, S(stream));
   // the weights' B-operand images for this step's projections: written beside the first kernels
   const bool prep = ctx->images != nullptr;
+  ctx->z_split = ctx->split_buf != nullptr && prep;   // the weight planes will be fresh by the time the embedding runs
   if (prep) {
     rc = fork_to(ctx, S(stream), ctx->side[0]);
     if (rc) return rc;

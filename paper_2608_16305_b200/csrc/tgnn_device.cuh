@@ -35,6 +35,19 @@ __device__ __forceinline__ void time_encode_sc(float w, float b, float dtf, floa
   *cos_out = __cosf(r);
 }
 
+// x as two bf16 numbers hi + lo (16 mantissa bits together); pairs of neighbours packed into 32-bit words.
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16* hi, __nv_bfloat16* lo) {
+  *hi = __float2bfloat16_rn(x);
+  *lo = __float2bfloat16_rn(x - __bfloat162float(*hi));
+}
+__device__ __forceinline__ void split_bf16_pair(float x0, float x1, uint32_t* hi, uint32_t* lo) {
+  __nv_bfloat16 h0, l0, h1, l1;
+  split_bf16(x0, &h0, &l0);
+  split_bf16(x1, &h1, &l1);
+  *hi = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+  *lo = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+}
+
 __device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + expf(-x)); }
 __device__ __forceinline__ float softplusf_(float x) { return x > 0.f ? x + log1pf(expf(-x)) : log1pf(expf(x)); }
 

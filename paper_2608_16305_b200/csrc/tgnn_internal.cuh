@@ -118,6 +118,14 @@ struct WeightSite {
   int64_t chunks;            // 16-byte chunks the preparation kernel writes for this site
 };
 
+// An fp32 matrix stored as two bf16 planes of the same row-major shape: hi = bf16(x) at `hi`, lo = bf16(x - hi)
+// at hi + plane_stride (in bf16 elements).  ld and plane_stride are multiples of 8, `hi` is 16-byte aligned.
+struct SplitMat {
+  void* hi;
+  int64_t ld, plane_stride;
+  int64_t rows, cols;
+};
+
 }  // namespace tgnn
 
 struct tgnn_ctx {
@@ -171,6 +179,11 @@ struct tgnn_ctx {
   unsigned char* images;         // device buffer of all sites' images
   size_t images_bytes;
   bool images_fresh;             // images match the current parameters (set by the step, cleared by Adam)
+  // TGNN_MATH_BF16X3: the attention inputs Z (with a column of ones after the last input column), the gradient
+  // of the key/value rows and the key/value weights in their two roles, each as two bf16 planes
+  void* split_buf;
+  tgnn::SplitMat zs, dkvs, wkv_s, wz_s;
+  bool z_split;       // the attention inputs of the current step are (being) written as bf16 planes
   bool z_static_done; // tgnn_train_step already gathered the memory-independent part of the attention inputs
   bool grads_zeroed;  // tgnn_train_step cleared the gradient block ahead of the backward pass
   tgnn::Workspace ws;
@@ -326,18 +339,12 @@ struct GemmArgs {
 int launch_gemm(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s);
 int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s);  // k_gemm_tc.cu
 // ---- split-bf16 projections (k_gemm_bf.cu) ----
-// An fp32 matrix stored as two bf16 planes of the same row-major shape: hi = bf16(x) at `hi`, lo = bf16(x - hi)
-// at hi + plane_stride (in bf16 elements).  ld and plane_stride are multiples of 8, `hi` is 16-byte aligned.
-struct SplitMat {
-  void* hi;
-  int64_t ld, plane_stride;
-  int64_t rows, cols;
-};
+int launch_prep_split_weights(tgnn_ctx* ctx, cudaStream_t s);
 int launch_split_rows(tgnn_ctx* ctx, const float* X, int64_t ld_in, int64_t rows, int cols, const int32_t* dev_rows,
                       const SplitMat& out, int ones_col, const char* name, cudaStream_t s);
 int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int mn_major, float* C, int64_t ldc, int M, int N,
                       int K, const float* bias, int relu, int accumulate, int split_k, const char* name, cudaStream_t s,
-                      int debug_withhold = 0, unsigned spin_limit = 0);
+                      int debug_withhold = 0, unsigned spin_limit = 0, int extra_col = -1, float* extra_out = nullptr);
 size_t plan_weight_sites(tgnn_ctx* ctx);                       // fills ctx->sites, returns the image bytes needed
 int launch_prep_weights(tgnn_ctx* ctx, cudaStream_t s);        // writes all images from the current parameters
 

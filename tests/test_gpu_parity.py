@@ -21,11 +21,11 @@ from paper_2608_16305_b200 import workload as wl
 
 pytestmark = pytest.mark.gpu
 
-TOL = {"fp32": 1e-4, "tf32": 2e-3, "tf32_bf16": 1e-2, "tf32fast": 2e-3, "tf32fast_bf16": 1e-2}
+TOL = {"fp32": 1e-4, "tf32": 2e-3, "tf32_bf16": 1e-2, "tf32fast": 2e-3, "tf32fast_bf16": 1e-2, "bf16x3": 2e-3, "bf16x3_bf16": 1e-2}
 # ReLU's derivative jumps at zero.  A unit whose pre-activation is closer to zero than the kernel's
 # arithmetic resolves may land on either side; for such units (|pre| <= GATE_EPS * max|pre|, nowhere
 # else) the oracle differentiates the branch the kernel took.
-GATE_EPS = {"fp32": 1e-5, "tf32": 2e-4, "tf32fast": 3e-3}
+GATE_EPS = {"fp32": 1e-5, "tf32": 2e-4, "tf32fast": 3e-3, "bf16x3": 2e-4}
 # How many units per step may take the kernel's branch against the oracle's own fp64 sign: a handful, or
 # 2e-5 of the step's ReLU units on the big batches (measured: at most 3 units in any compared step of the
 # five workloads, 1.2 M to 2 M units per step on the batch-4000 ones).
@@ -80,7 +80,8 @@ class Rig:
             self.dw = trainer.PartitionedWorkload(self.stream, *partition, efeat=efeat_dev, embed_aux=embed_aux)
         self.model = model
         self.weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed, bias_scale=bias_scale, model=model)
-        mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST}[math]
+        mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST,
+                "bf16x3": B.TGNN_MATH_BF16X3}[math]
         self.tr = trainer.Trainer(self.dw, self.weights, math_mode=mode, lr=lr, model=model)
         f32 = lambda x: float(np.float32(x))      # the library's configuration holds fp32 hyper-parameters
         self.ocfg = orc_cfg(oracle, cfg, lr=f32(lr), beta1=f32(0.9), beta2=f32(0.999), eps=f32(1e-8))
@@ -520,7 +521,7 @@ def _run_epoch_checks(rig, steps, check_at):
             rig.check_step(b, pre, res, what=f"[{rig.cfg.name} batch {b}]")
 
 
-@pytest.mark.parametrize("math", ["fp32", "tf32"])
+@pytest.mark.parametrize("math", ["fp32", "tf32", "bf16x3"])
 def test_tiny_epoch_teacher_forced(B, oracle, math):
     rig = Rig(B, oracle, TINY, math=math)
     nb = TINY.num_batches
@@ -538,7 +539,7 @@ def _scaled(name, events, **kw):
     return wl.scaled(c, num_events=events, **kw)
 
 
-@pytest.mark.parametrize("math", ["fp32", "tf32"])
+@pytest.mark.parametrize("math", ["fp32", "tf32", "bf16x3"])
 @pytest.mark.parametrize("name,events,at", [
     ("wiki", 6000, {1, 5, 9}),          # 172-d features, d = 100: ragged tiles everywhere
     ("reddit", 9000, {2, 8, 14}),       # replay events + pruning
@@ -597,7 +598,7 @@ def test_head_paths_wide_and_ragged(B, oracle, math, d, batch):
     _run_epoch_checks(rig, range(4), {1, 3})
 
 
-@pytest.mark.parametrize("math", ["fp32", "tf32"])
+@pytest.mark.parametrize("math", ["fp32", "tf32", "bf16x3"])
 def test_bf16_feature_table(B, oracle, math):
     c = wl.scaled(wl.CONFIGS["large"], num_events=20000, num_nodes=3000, batch=1000)
     rig = Rig(B, oracle, c, math=math)
@@ -988,18 +989,20 @@ def _full_size(B, oracle, cfg, check_at, last, math="tf32"):
 
 
 @pytest.mark.slow
-def test_wiki_full_size_graph_replay(B, oracle):
+@pytest.mark.parametrize("math", ["tf32", "bf16x3"])
+def test_wiki_full_size_graph_replay(B, oracle, math):
     cfg = wl.CONFIGS["wiki"]
-    rig = _full_size(B, oracle, cfg, {0, 1, 2, 150, cfg.num_batches - 1}, cfg.num_batches - 1)
+    rig = _full_size(B, oracle, cfg, {0, 1, 2, 150, cfg.num_batches - 1}, cfg.num_batches - 1, math=math)
     # the last batch is ragged (160000 = 266 * 600 + 400): a different shape signature was captured
     assert cfg.num_events % cfg.batch != 0
     assert rig.tr.lib.kernel_launches() > 30 * cfg.num_batches
 
 
 @pytest.mark.slow
-def test_reddit_full_size_replay_and_pruning(B, oracle):
+@pytest.mark.parametrize("math", ["tf32", "bf16x3"])
+def test_reddit_full_size_replay_and_pruning(B, oracle, math):
     cfg = wl.CONFIGS["reddit"]
-    rig = _full_size(B, oracle, cfg, {3, 400}, 400)
+    rig = _full_size(B, oracle, cfg, {3, 400}, 400, math=math)
     heavy = rig.dw.heavy.cpu().numpy()
     keep = rig.dw.mb_keep.cpu().numpy()
     aux = rig.dw.mb_aux.cpu().numpy()
@@ -1007,19 +1010,21 @@ def test_reddit_full_size_replay_and_pruning(B, oracle):
 
 
 @pytest.mark.slow
-def test_lastfm_full_size_hub_contention(B, oracle):
+@pytest.mark.parametrize("math", ["tf32", "bf16x3"])
+def test_lastfm_full_size_hub_contention(B, oracle, math):
     cfg = wl.CONFIGS["lastfm"]
-    rig = _full_size(B, oracle, cfg, {2, 60}, 60)
+    rig = _full_size(B, oracle, cfg, {2, 60}, 60, math=math)
     top = np.bincount(np.concatenate([rig.stream.src, rig.stream.dst])).max() / (2 * cfg.num_events)
     assert top > 0.3                       # one node takes a third of all endpoint slots
 
 
 @pytest.mark.slow
-def test_large_full_size_bf16(B, oracle):
+@pytest.mark.parametrize("math", ["tf32", "bf16x3"])
+def test_large_full_size_bf16(B, oracle, math):
     # 17,000 nodes, 50 M events, 18.6 GB of bf16 edge features resident in HBM (generated on the device),
     # batch 4,000, 20 % replay with pruning; about a minute of host set-up (T-CSR over 10^8 entries).  The
     # feature table is too big for a host copy, so the oracle gets the rows each compared step touches.
     cfg = wl.CONFIGS["large"]
     last = cfg.num_batches - 1
-    rig = _full_size(B, oracle, cfg, {5, last}, last)
+    rig = _full_size(B, oracle, cfg, {5, last}, last, math=math)
     assert rig.compact and rig.efeat_dev.numel() * 2 > 18e9
