@@ -286,18 +286,39 @@ __global__ void __launch_bounds__(256) gather_z_memory_kernel(const float* __res
   const int warps = (gridDim.x * blockDim.x) >> 5;
   const int nb_rows = n * k;
   if (z_hi != nullptr) {
-    // one thread per pair of columns, rows back to back: every lane of every warp moves data
-    const int hp = d >> 1;
-    const int64_t total = (int64_t)nb_rows * hp;
-    for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
-      const int r = (int)(idx / hp), q = (int)(idx - (int64_t)r * hp);
-      const int nb = __ldg(nbr + r);
-      if (nb < 0) continue;
-      const float2 x = __ldg(reinterpret_cast<const float2*>(memory + (int64_t)nb * d) + q);
-      uint32_t h, l;
-      split_bf16_pair(x.x, x.y, &h, &l);
-      reinterpret_cast<uint32_t*>(z_hi + (int64_t)r * ld_s)[q] = h;
-      reinterpret_cast<uint32_t*>(z_hi + plane_s + (int64_t)r * ld_s)[q] = l;
+    // a warp takes four rows at a time: their slot records, then the four table rows (16 bytes per lane), then the
+    // conversions and stores -- four independent round trips in flight per warp instead of a dependent chain per row
+    const int d4 = d >> 2;          // <= 64: two 16-byte pieces per lane at most
+    const int wg = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    for (int r0 = wg * 4; r0 < nb_rows; r0 += warps * 4) {
+      int nb[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) nb[j] = r0 + j < nb_rows ? __ldg(nbr + r0 + j) : -1;
+      float4 x[4][2];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int q = lane + 32 * u;
+          x[j][u] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (nb[j] >= 0 && q < d4) x[j][u] = __ldg(reinterpret_cast<const float4*>(memory + (int64_t)nb[j] * d) + q);
+        }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (nb[j] < 0) continue;
+        uint2* hi = reinterpret_cast<uint2*>(z_hi + (int64_t)(r0 + j) * ld_s);
+        uint2* lo = reinterpret_cast<uint2*>(z_hi + plane_s + (int64_t)(r0 + j) * ld_s);
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int q = lane + 32 * u;
+          if (q < d4) {
+            uint2 h, l;
+            split_bf16_pair(x[j][u].x, x[j][u].y, &h.x, &l.x);
+            split_bf16_pair(x[j][u].z, x[j][u].w, &h.y, &l.y);
+            hi[q] = h; lo[q] = l;
+          }
+        }
+      }
     }
   }
   for (int r = (z_hi != nullptr ? nb_rows : 0) + ((blockIdx.x * blockDim.x + threadIdx.x) >> 5); r < nb_rows + n; r += warps) {
@@ -454,7 +475,9 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
   cudaStream_t sg = indirect ? ctx->side[0] : s;
   {
     KernelScope scope__(ctx, "gather_z_memory", sg);
-    gather_z_memory_kernel<<<(rows + 7) / 8, 256, 0, sg>>>(ctx->memory, d, k, nodes, n, nbr, ctx->ld_kv, w.Z, w.Zq, w.cat_o,
+    // split planes: a grid that fits the machine once (six blocks per SM), rows in groups of four per warp
+    const int gblocks = split ? ((rows + 31) / 32 < 148 * 6 ? (rows + 31) / 32 : 148 * 6) : (rows + 7) / 8;
+    gather_z_memory_kernel<<<gblocks, 256, 0, sg>>>(ctx->memory, d, k, nodes, n, nbr, ctx->ld_kv, w.Z, w.Zq, w.cat_o,
                                                            split ? reinterpret_cast<__nv_bfloat16*>(ctx->zs.hi) : nullptr,
                                                            ctx->zs.plane_stride, (int)ctx->zs.ld);
   }

@@ -63,6 +63,7 @@ struct BfArgs {
   int extra_col;
   float* extra_out;
   int32_t* status;
+  long long* trace;           // debug: clock stamps of CTA 0 (nullptr in normal use)
   int debug_withhold;         // test hook: the MMA warp skips this many slot releases (an empty-slot wait then expires)
   unsigned spin_limit;
 };
@@ -120,22 +121,48 @@ __device__ __forceinline__ void commit_to(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+#define TRACE(slot)                                                          \
+  do {                                                                       \
+    if (g.trace != nullptr && blockIdx.x == 0 && (slot) < 512) g.trace[slot] = clock64(); \
+  } while (0)
+
 struct Item {
   int mt0, tiles, n0, n_valid, kb0, kb1;
 };
-__device__ __forceinline__ Item decode_item(const BfArgs& g, int w) {
-  const int m_pairs = (g.m_tiles + 1) >> 1;
-  const int mp = w % m_pairs, rest = w / m_pairs;
-  const int nt = rest % g.n_tiles, sp = rest / g.n_tiles;
-  Item it;
-  it.mt0 = 2 * mp;
-  it.tiles = min(2, g.m_tiles - it.mt0);
-  it.n0 = nt * g.bn;
-  it.n_valid = min(g.bn, g.N - it.n0);
-  const int per = (g.kb_total + g.split_k - 1) / g.split_k;
-  it.kb0 = sp * per;
-  it.kb1 = min(g.kb_total, it.kb0 + per);
-  return it;
+// A CTA's share of the work: a contiguous range of "tile units" (n-tile / contraction-split combination
+// major, 128-row tile minor), walked in pairs of row tiles that share their B tiles; a pair never spans two
+// combinations, and the last unit of a range may be a single tile.  All roles walk the same sequence.
+struct Walk {
+  int u, u_end;
+};
+__device__ __forceinline__ Walk cta_walk(const BfArgs& g) {
+  const long long T = (long long)g.m_tiles * g.n_tiles * g.split_k;
+  Walk w;
+  w.u = (int)(T * blockIdx.x / gridDim.x);
+  w.u_end = (int)(T * (blockIdx.x + 1) / gridDim.x);
+  return w;
+}
+__device__ __forceinline__ bool next_item(const BfArgs& g, Walk& wk, Item& it) {
+  while (wk.u < wk.u_end) {
+    const int combo = wk.u / g.m_tiles, mt = wk.u - combo * g.m_tiles;
+    it.mt0 = mt;
+    it.tiles = min(2, min(wk.u_end - wk.u, g.m_tiles - mt));
+    wk.u += it.tiles;
+    const int nt = combo % g.n_tiles, sp = combo / g.n_tiles;
+    it.n0 = nt * g.bn;
+    it.n_valid = nt == g.n_tiles - 1 ? g.N - it.n0 : g.bn;
+    const int per = (g.kb_total + g.split_k - 1) / g.split_k;
+    it.kb0 = sp * per;
+    it.kb1 = min(g.kb_total, it.kb0 + per);
+    if (it.kb0 < it.kb1) return true;   // an empty contraction range is skipped by every role alike
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+      : "memory");
 }
 
 __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_constant__ BfArgs g) {
@@ -170,11 +197,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = s_tmem;
+  if (tid == 0) TRACE(0);
   volatile int* abort_flag = &s_abort;
   const unsigned limit = g.spin_limit;
 
-  const int m_pairs = (g.m_tiles + 1) >> 1;
-  const int items = m_pairs * g.n_tiles * g.split_k;
   const int ks_per_kb = g.mn_major ? 2 : 4;
 
   if (warp == 0) {
@@ -183,9 +209,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
       uint32_t ca = 0, cb = 0;
       bool ok = true;
       const uint32_t a_bytes = (uint32_t)g.a_slot_bytes, b_bytes = (uint32_t)g.b_slot_bytes;
-      const uint32_t a_plane = a_bytes >> 1, b_plane = b_bytes >> 1;
-      for (int w = blockIdx.x; w < items && ok; w += gridDim.x) {
-        const Item it = decode_item(g, w);
+      Walk wk = cta_walk(g);
+      Item it;
+      while (ok && next_item(g, wk, it)) {
         for (int kb = it.kb0; kb < it.kb1 && ok; ++kb) {
           {
             const uint32_t s = cb % (uint32_t)g.n_b_slots;
@@ -193,13 +219,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
             if (!ok) break;
             const uint32_t bar = smem_u32(&s_full_b[s]), dst = b_ring + s * b_bytes;
             mbar_expect_tx(bar, b_bytes);
-            if (!g.mn_major) {
-              tma_3d(dst, &g.b_map, kb * 64, it.n0, 0, bar);
-              tma_3d(dst + b_plane, &g.b_map, kb * 64, it.n0, 1, bar);
-            } else {
-              for (int p = 0; p < 2; ++p)
-                for (int c = 0; c < g.b_chunks; ++c) tma_3d(dst + p * b_plane + c * 4096, &g.b_map, it.n0 + 64 * c, kb * 32, p, bar);
-            }
+            // one copy brings both planes of the tile (the box spans the plane dimension)
+            if (!g.mn_major) tma_3d(dst, &g.b_map, kb * 64, it.n0, 0, bar);
+            else tma_4d(dst, &g.b_map, 0, kb * 32, it.n0 >> 6, 0, bar);
             ++cb;
           }
           for (int t = 0; t < it.tiles && ok; ++t) {
@@ -209,13 +231,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
             const uint32_t bar = smem_u32(&s_full_a[s]), dst = a_ring + s * a_bytes;
             const int m0 = (it.mt0 + t) * BM;
             mbar_expect_tx(bar, a_bytes);
-            if (!g.mn_major) {
-              tma_3d(dst, &g.a_map, kb * 64, m0, 0, bar);
-              tma_3d(dst + a_plane, &g.a_map, kb * 64, m0, 1, bar);
-            } else {
-              for (int p = 0; p < 2; ++p)
-                for (int c = 0; c < 2; ++c) tma_3d(dst + p * a_plane + c * 4096, &g.a_map, m0 + 64 * c, kb * 32, p, bar);
-            }
+            if (!g.mn_major) tma_3d(dst, &g.a_map, kb * 64, m0, 0, bar);
+            else tma_4d(dst, &g.a_map, 0, kb * 32, m0 >> 6, 0, bar);
+            TRACE(256 + (int)ca);
             ++ca;
           }
         }
@@ -235,9 +253,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
       // K-major: 8-row groups 1024 B apart (SBO), a step advances 32 B.  MN-major: 64-column chunks 4096 B apart
       // (LBO), 8-row contraction groups 1024 B apart (SBO), a step advances two groups.
       const uint32_t lbo = mn ? 4096u : 16u, sbo = 1024u, kstep_bytes = mn ? 2048u : 32u;
-      for (int w = blockIdx.x; w < items && ok; w += gridDim.x) {
-        const Item it = decode_item(g, w);
-        if (it.kb0 >= it.kb1) continue;   // an empty contraction range: every role skips it
+      Walk wk = cta_walk(g);
+      Item it;
+      while (ok && next_item(g, wk, it)) {
         ok = mbar_wait(smem_u32(&s_tmem_empty), (n_item & 1u) ^ 1u, limit, abort_flag);   // accumulators drained
         if (!ok) break;
         ++n_item;
@@ -256,6 +274,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
             ok = mbar_wait(smem_u32(&s_full_a[sa]), (ca / (uint32_t)g.n_a_slots) & 1u, limit, abort_flag);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            TRACE(16 + 2 * (int)ca);
             const uint32_t a_addr = a_ring + sa * a_bytes;
             const uint32_t acc = tmem + (uint32_t)(t * ACC_STRIDE);
             for (int ks = 0; ks < ks_n; ++ks) {
@@ -268,6 +287,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
               mma_bf16(acc, da_hi, db_lo, idesc, 1u);
               mma_bf16(acc, da_hi, db_hi, idesc, 1u);
             }
+            TRACE(17 + 2 * (int)ca);
             if (withheld < g.debug_withhold) ++withheld;   // test hook: this slot is never handed back
             else commit_to(smem_u32(&s_empty_a[sa]));
             ++ca;
@@ -290,12 +310,13 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
     const int sub = lane >> 2, ch = lane & 3;
     uint32_t n_item = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < items && ok; w += gridDim.x) {
-      const Item it = decode_item(g, w);
-      if (it.kb0 >= it.kb1) continue;
+    Walk wk = cta_walk(g);
+    Item it;
+    while (ok && next_item(g, wk, it)) {
       ok = mbar_wait(smem_u32(&s_tmem_full), n_item & 1u, limit, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
+      if (e == 0 && lane == 0) TRACE(2 + 2 * (int)n_item);
       ++n_item;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       if (t < it.tiles) {
@@ -369,6 +390,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
+      if (e == 0 && lane == 0) TRACE(1 + 2 * (int)n_item);
       if (lane == 0) mbar_arrive(smem_u32(&s_tmem_empty));
     }
     if (!ok && lane == 0) { s_abort = 1; atomicCAS(g.status, 0, TGNN_ETIMEOUT); }
@@ -460,17 +482,35 @@ TensorMapEncodeFn encoder() {
   return enc;
 }
 
-// (contiguous index, row, plane) view of a split matrix; box = 64 elements x box_rows x 1 plane, 128-byte swizzle,
-// zeros outside [0, cols) x [0, rows).
-bool encode_split_map(CUtensorMap* map, const SplitMat& m, int box_rows) {
+// K-major operand: (contiguous index, row, plane) view of a split matrix; box = 64 elements x box_rows x both planes,
+// 128-byte swizzle, zeros outside [0, cols) x [0, rows).
+bool encode_k_map(CUtensorMap* map, const SplitMat& m, int box_rows) {
   const TensorMapEncodeFn enc = encoder();
   if (!enc || m.rows <= 0 || m.cols <= 0 || box_rows < 1 || box_rows > 256) return false;
   if (((uintptr_t)m.hi & 15) != 0 || m.ld % 8 != 0 || m.plane_stride % 8 != 0) return false;
   const cuuint64_t dims[3] = {(cuuint64_t)m.cols, (cuuint64_t)m.rows, 2};
   const cuuint64_t strides[2] = {(cuuint64_t)m.ld * 2, (cuuint64_t)m.plane_stride * 2};
-  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 2};
   const cuuint32_t elem[3] = {1, 1, 1};
   return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, m.hi, dims, strides, box, elem,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// MN-major operand: the matrix [rows = contraction, cols] seen as (element within a 64-column chunk, row, chunk,
+// plane); one box of 64 x 32 rows x `chunks` x both planes lands chunk-major, i.e. as the operand tile's own
+// layout (per chunk 32 rows of 128 bytes, swizzled).  The last chunk of a row may run past the row end into the
+// next row (or, for the last row, up to 126 bytes past the plane): those values only reach rows / columns of C
+// that are never stored, and the buffers end in slack.
+bool encode_mn_map(CUtensorMap* map, const SplitMat& m, int chunks) {
+  const TensorMapEncodeFn enc = encoder();
+  if (!enc || m.rows <= 0 || m.cols <= 0 || chunks < 1 || chunks > 4) return false;
+  if (((uintptr_t)m.hi & 15) != 0 || m.ld % 8 != 0 || m.plane_stride % 8 != 0) return false;
+  const cuuint64_t dims[4] = {64, (cuuint64_t)m.rows, (cuuint64_t)((m.cols + 63) / 64), 2};
+  const cuuint64_t strides[3] = {(cuuint64_t)m.ld * 2, 128, (cuuint64_t)m.plane_stride * 2};
+  const cuuint32_t box[4] = {64, 32, (cuuint32_t)chunks, 2};
+  const cuuint32_t elem[4] = {1, 1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, m.hi, dims, strides, box, elem,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -511,7 +551,7 @@ int launch_split_rows(tgnn_ctx* ctx, const float* X, int64_t ld_in, int64_t rows
 // split_k > 1 needs accumulate (C holds valid data; partial sums are added atomically).
 int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int mn_major, float* C, int64_t ldc, int M, int N,
                       int K, const float* bias, int relu, int accumulate, int split_k, const char* name, cudaStream_t s,
-                      int debug_withhold, unsigned spin_limit, int extra_col, float* extra_out) {
+                      int debug_withhold, unsigned spin_limit, int extra_col, float* extra_out, long long* trace) {
   if (M <= 0 || N <= 0) return TGNN_OK;
   if (K <= 0) return set_error(ctx, TGNN_EINVAL, "gemm %s: empty contraction", name);
   if (split_k > 1 && !accumulate) return set_error(ctx, TGNN_EINVAL, "gemm %s: split_k needs accumulate", name);
@@ -521,17 +561,30 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
   a.status = ctx->ws.status;
   a.extra_col = (extra_out && accumulate) ? extra_col : -1;
   a.extra_out = extra_out;
+  a.trace = trace;
   a.debug_withhold = debug_withhold;
   a.spin_limit = spin_limit ? spin_limit : SPIN_LIMIT;
   a.m_tiles = (M + BM - 1) / BM;
+  // n-tiles: a common stride bn (a multiple of 16; of 64 for MN-major operands, whose tiles start on chunk
+  // boundaries) and the remainder, at most 256 columns, in the last tile
+  const int gran = mn_major ? 64 : 16;
   a.n_tiles = (N + 255) / 256;
-  a.bn = ((N + a.n_tiles - 1) / a.n_tiles + 15) / 16 * 16;
+  int n_last;
+  for (;; ++a.n_tiles) {
+    a.bn = a.n_tiles == 1 ? (N + gran - 1) / gran * gran : (N / a.n_tiles) / gran * gran;
+    if (a.n_tiles > 1 && a.bn < gran) a.bn = gran;
+    n_last = N - (a.n_tiles - 1) * a.bn;
+    if (n_last <= 256) break;
+  }
+  if (n_last <= 0) return set_error(ctx, TGNN_ESHAPE, "gemm %s: n-tiling failed", name);
+  const int n_widest = a.n_tiles == 1 ? N : (a.bn > n_last ? a.bn : n_last);
+  const int b_rows = (n_widest + 15) / 16 * 16;     // K-major B box: rows of the widest n-tile
   const int bke = mn_major ? 32 : 64;
   a.kb_total = (K + bke - 1) / bke;
   a.ksteps_total = (K + 15) / 16;
-  a.b_chunks = (a.bn + 63) / 64;
+  a.b_chunks = (n_widest + 63) / 64;
   a.a_slot_bytes = mn_major ? 2 * 2 * 4096 : 2 * BM * 128;
-  a.b_slot_bytes = mn_major ? 2 * a.b_chunks * 4096 : 2 * a.bn * 128;
+  a.b_slot_bytes = mn_major ? 2 * a.b_chunks * 4096 : 2 * b_rows * 128;
   const int budget = SMEM_LIMIT - 1024 - STG_BYTES - 1024;
   a.n_b_slots = a.b_slot_bytes > 40 * 1024 ? 2 : (a.b_slot_bytes > 20 * 1024 ? 3 : 4);
   a.n_a_slots = (budget - a.n_b_slots * a.b_slot_bytes) / a.a_slot_bytes;
@@ -547,10 +600,11 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
     if (sp > split_k) sp = split_k;
     a.split_k = sp < 1 ? 1 : sp;
   }
-  // the K-major B box is a whole n-tile (bn rows); MN-major boxes are 64 columns x 32 contraction rows
-  if (!encode_split_map(&a.a_map, A, mn_major ? 32 : BM) || !encode_split_map(&a.b_map, B, mn_major ? 32 : a.bn))
-    return set_error(ctx, TGNN_ECUDA, "gemm %s: tensor map encoding failed", name);
-  const int items = m_pairs * a.n_tiles * a.split_k;
+  const bool maps_ok = mn_major ? (encode_mn_map(&a.a_map, A, 2) && encode_mn_map(&a.b_map, B, a.b_chunks))
+                                : (encode_k_map(&a.a_map, A, BM) && encode_k_map(&a.b_map, B, b_rows));
+  if (!maps_ok) return set_error(ctx, TGNN_ECUDA, "gemm %s: tensor map encoding failed", name);
+  const int units = a.m_tiles * a.n_tiles * a.split_k;
+  const int items = (units + 1) / 2;
   const int smem = 1024 + a.n_a_slots * a.a_slot_bytes + a.n_b_slots * a.b_slot_bytes + STG_BYTES;
   static int attr_bytes[64] = {};
   int dev = 0;

@@ -1,6 +1,7 @@
 // C ABI: context life cycle, argument checks, and the sequencing of one training step.
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <new>
@@ -277,6 +278,7 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
       m->plane_stride = (m->rows * m->ld + 127) / 128 * 128;
       off += (size_t)(2 * m->plane_stride * 2);
     }
+    off += 256;   // a chunked tile copy may read up to 126 bytes past the last plane (values that reach no stored output)
     ok = cudaMalloc(&ctx->split_buf, off) == cudaSuccess && cudaMemset(ctx->split_buf, 0, off) == cudaSuccess;
     off = 0;
     for (SplitMat* m : ms) {
@@ -808,7 +810,7 @@ int tgnn_debug_gemm_split(tgnn_ctx* ctx, const float* A, int64_t a_rs, int64_t a
   a.plane_stride = a.rows * a.ld;
   b.plane_stride = b.rows * b.ld;
   const int64_t a_bytes = (2 * a.plane_stride * 2 + 255) / 256 * 256, b_bytes = 2 * b.plane_stride * 2;
-  NEED(ctx, scratch_bytes >= a_bytes + b_bytes, TGNN_ECAPACITY, "debug_gemm_split: scratch of %lld bytes, %lld needed",
+  NEED(ctx, scratch_bytes >= a_bytes + b_bytes + 256, TGNN_ECAPACITY, "debug_gemm_split: scratch of %lld bytes, %lld needed",
        (long long)scratch_bytes, (long long)(a_bytes + b_bytes));
   NEED(ctx, ((uintptr_t)scratch & 255) == 0, TGNN_EINVAL, "debug_gemm_split: scratch must be 256-byte aligned");
   a.hi = scratch;
@@ -817,8 +819,13 @@ int tgnn_debug_gemm_split(tgnn_ctx* ctx, const float* A, int64_t a_rs, int64_t a
   if (rc) return rc;
   rc = launch_split_rows(ctx, B, ldb, b.rows, (int)b.cols, nullptr, b, -1, "split_b", S(stream));
   if (rc) return rc;
+  // TGNN_GEMM_TRACE=1 (debugging aid): the first 4 KB of scratch receive clock stamps of CTA 0 instead of nothing
+  static const bool trace_on = getenv("TGNN_GEMM_TRACE") != nullptr;
+  long long* trace = nullptr;
+  if (trace_on && scratch_bytes >= a_bytes + b_bytes + 256 + 4096 + 256)
+    trace = reinterpret_cast<long long*>((char*)scratch + ((a_bytes + b_bytes + 256 + 255) / 256 * 256));
   return launch_gemm_split(ctx, a, b, mn, C, ldc, M, N, K, bias, relu, accumulate, split_k < 1 ? 1 : split_k, "debug_gemm_split",
-                           S(stream), debug_withhold, spin_limit);
+                           S(stream), debug_withhold, spin_limit, -1, nullptr, trace);
 }
 
 int tgnn_status(tgnn_ctx* ctx, int32_t* status_host, void* stream) {
