@@ -66,10 +66,12 @@ enum {
   TGNN_MATH_FP32 = 0,     /* fp32 FMA tiles */
   TGNN_MATH_TF32 = 1,     /* tcgen05 tensor cores: every operand is split into a TF32 head and a TF32
                              tail (3 MMAs per product, fp32 accumulation in TMEM), close to fp32 accuracy */
-  TGNN_MATH_BF16X3 = 3,   /* as TGNN_MATH_TF32, except that the three products over the sampled-neighbor rows (key/value
-                             projection, its input gradient and its weight gradient) hold each fp32 operand as two bf16
-                             numbers (hi + lo, 16 mantissa bits) and run as three bf16 tensor-core passes with fp32
-                             accumulation: more accurate than one TF32 pass, half the tensor time of the TF32 split */
+  TGNN_MATH_F16X3 = 3,    /* as TGNN_MATH_TF32, except that the three products over the sampled-neighbor rows (key/value
+                             projection, its input gradient and its weight gradient) hold each fp32 operand as two fp16
+                             numbers (hi + lo, 22 mantissa bits; gradients are scaled by a power of two into fp16's
+                             range) and run as three fp16 tensor-core passes with fp32 accumulation: the accuracy of
+                             the TF32 split at half its tensor time.  Edge features and memory values must stay below
+                             fp16's largest number (65504) in magnitude */
   TGNN_MATH_TF32_FAST = 2 /* tcgen05 tensor cores, single TF32 pass in the forward projections (the gradient
                              products keep the split).  Outputs stay within 2e-3, but gradient tensors whose
                              terms cancel (time encoder, W_k) can be off by ~1e-2 of their largest entry. */
@@ -323,10 +325,10 @@ TGNN_API int tgnn_clear_status(tgnn_ctx* ctx, void* stream);
 /* Number of kernels this context has launched since creation (host counter). */
 TGNN_API int64_t tgnn_kernel_launches(const tgnn_ctx* ctx);
 
-/* The split-bf16 projection kernel on its own, for parity tests (sm_100 tensor cores, any math_mode): the
- * fp32 operands are first split into two bf16 planes each (hi = bf16(x), lo = bf16(x - hi), 16 mantissa bits
+/* The split-operand projection kernel on its own, for parity tests (sm_100 tensor cores, any math_mode): the
+ * fp32 operands are first split into two fp16 planes each (hi = fp16(x), lo = fp16(x - hi), 22 mantissa bits
  * together) inside `scratch` (device, 256-byte aligned, >= 2 * 2 * (rows * ceil8(cols)) bytes per operand plus
- * 256), then C[M,N] (+)= A B (+ bias[n]) (ReLU) runs as three bf16 passes with fp32 accumulation.  Strides as in
+ * 256), then C[M,N] (+)= A B (+ bias[n]) (ReLU) runs as three fp16 passes with fp32 accumulation.  Strides as in
  * tgnn_debug_gemm, with the restriction that either both operands have the contraction index contiguous
  * (a_cs = 1, b_rs = 1) or both have the other index contiguous (a_rs = 1, b_cs = 1: C = A^T B over matrix rows).
  * accumulate / split_k as in tgnn_debug_gemm.  debug_withhold > 0 makes the kernel keep that many shared-memory

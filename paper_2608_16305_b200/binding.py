@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libtgnn_b200.so")
 TGNN_OK, TGNN_EINVAL, TGNN_ESHAPE, TGNN_ECAPACITY, TGNN_ESTATE, TGNN_ECUDA, TGNN_ETIMEOUT, TGNN_EBOUNDS = (
     0, -1, -2, -3, -4, -5, -6, -7)
 TGNN_F32, TGNN_BF16 = 0, 1
-TGNN_MATH_FP32, TGNN_MATH_TF32, TGNN_MATH_TF32_FAST, TGNN_MATH_BF16X3 = 0, 1, 2, 3
+TGNN_MATH_FP32, TGNN_MATH_TF32, TGNN_MATH_TF32_FAST, TGNN_MATH_F16X3 = 0, 1, 2, 3
 
 PARAM_NAMES = ("time_w", "time_b", "gru_w_i", "gru_w_h", "gru_b_i", "gru_b_h", "w_q", "b_q", "w_k", "w_v",
                "b_k", "b_v", "w_o", "b_o", "w_1", "b_1", "w_2", "b_2")

@@ -290,15 +290,17 @@ __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __r
 // One warp per root: backward of the weighted sum, the softmax and the scaled dot products, on the
 // root's K | V rows staged in shared memory.  Lane p < H*k owns the (head, slot) pair p for the
 // probability and logit gradients; afterwards the lanes own columns and write dQ and the dK | dV rows.
-// SPLIT: the key/value gradient rows are written as two bf16 planes (hi, lo; row pitch ld_s, plane_s elements
-// apart) for the split-bf16 products that consume them, instead of as fp32 rows.
+// SPLIT: the key/value gradient rows are written as two fp16 planes (hi, lo; row pitch ld_s, plane_s elements
+// apart), multiplied by the power of two gscale so that they sit inside fp16's range, for the split products that
+// consume them (which divide it out again), instead of as fp32 rows.
 template <bool SPLIT>
 __global__ void __launch_bounds__(256) attention_bwd_kernel(const float* __restrict__ Q, const float* __restrict__ KV,
                                                             const float* __restrict__ alpha,
                                                             const float* __restrict__ dcat_o,
                                                             const int32_t* __restrict__ cnt, int n, int d, int H, int k,
                                                             float* __restrict__ dQ, float* __restrict__ dKV,
-                                                            __nv_bfloat16* __restrict__ dkv_hi, int64_t plane_s, int ld_s) {
+                                                            __nv_bfloat16* __restrict__ dkv_hi, int64_t plane_s, int ld_s,
+                                                            float gscale) {
   extern __shared__ __align__(16) float sm[];
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   const int i = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
@@ -311,7 +313,7 @@ __global__ void __launch_bounds__(256) attention_bwd_kernel(const float* __restr
   float* dal = al + H * k;   // d loss / d probability
   float* dl = dal + H * k;   // d loss / d logit, already scaled
   const int dh = d / H;
-  const int c = cnt[i];
+  const int c = max(0, min(cnt[i], k));
   const float scale = rsqrtf((float)dh);
   attn_stage_issue(Ks, Vs, Qs, Q, KV, i, c, d, k, lane);
   {
@@ -375,8 +377,8 @@ __global__ void __launch_bounds__(256) attention_bwd_kernel(const float* __restr
           const float g0 = dl[h0 * k + s], g1 = dl[h1 * k + s];
           dq0 = fmaf(g0, Ks[s * d + e], dq0);
           dq1 = fmaf(g1, Ks[s * d + e + 1], dq1);
-          split_bf16_pair(g0 * q0, g1 * q1, &kh, &kl);
-          split_bf16_pair(al[h0 * k + s] * a0, al[h1 * k + s] * a1, &vh, &vl);
+          split_f16_pair(g0 * q0 * gscale, g1 * q1 * gscale, &kh, &kl);
+          split_f16_pair(al[h0 * k + s] * a0 * gscale, al[h1 * k + s] * a1 * gscale, &vh, &vl);
         }
         hi[e >> 1] = kh; lo[e >> 1] = kl;
         hi[(d + e) >> 1] = vh; lo[(d + e) >> 1] = vl;
@@ -395,7 +397,7 @@ __global__ void __launch_bounds__(256) scatter_dmem_kernel(const float* __restri
                                                            const int32_t* __restrict__ nbr,
                                                            const int32_t* __restrict__ nodes, int n, int k, int d,
                                                            const int32_t* __restrict__ node2slot,
-                                                           float* __restrict__ dMemU) {
+                                                           float* __restrict__ dMemU, int64_t N) {
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   const int nb_rows = n * k;
@@ -421,7 +423,7 @@ __global__ void __launch_bounds__(256) scatter_dmem_kernel(const float* __restri
       }
     }
     const int node = isn ? nbr[r] : nodes[i];
-    if (node < 0) continue;
+    if (node < 0 || node >= N) continue;   // (an id beyond the graph was reported by the forward pass)
     const int slot = node2slot[node];
     if (slot < 0) continue;
     float4* out = reinterpret_cast<float4*>(dMemU + (int64_t)slot * d);
@@ -445,7 +447,7 @@ __global__ void __launch_bounds__(256) scatter_dmem_cached_kernel(const float* _
                                                                   const int32_t* __restrict__ nbr,
                                                                   const int32_t* __restrict__ nodes, int n, int k, int d,
                                                                   const int32_t* __restrict__ node2slot,
-                                                                  float* __restrict__ dMemU) {
+                                                                  float* __restrict__ dMemU, int64_t N) {
   extern __shared__ __align__(16) float s_acc[];  // [SC_WAYS][d]
   __shared__ int s_id[SC_WAYS];
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -474,7 +476,7 @@ __global__ void __launch_bounds__(256) scatter_dmem_cached_kernel(const float* _
       }
     }
     const int node = isn ? nbr[r] : nodes[i];
-    if (node < 0) continue;
+    if (node < 0 || node >= N) continue;
     const int slot = node2slot[node];
     if (slot < 0) continue;
     const int way = slot % SC_WAYS;
@@ -636,7 +638,7 @@ __global__ void __launch_bounds__(256) jodie_embed_bwd_kernel(const float* __res
                                                               const int32_t* __restrict__ nodes,
                                                               const double* __restrict__ times, int n, int d,
                                                               const int32_t* __restrict__ node2slot, int have_update,
-                                                              float* __restrict__ dMemU, double* __restrict__ acc) {
+                                                              float* __restrict__ dMemU, double* __restrict__ acc, int64_t N) {
   extern __shared__ double s_part[];  // [8][2][d]
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   double gw[TG_MAXJ], gb[TG_MAXJ];
@@ -645,6 +647,7 @@ __global__ void __launch_bounds__(256) jodie_embed_bwd_kernel(const float* __res
   const int warps = (gridDim.x * blockDim.x) >> 5;
   for (int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
     const int node = nodes[i];
+    if (node < 0 || node >= N) continue;   // reported by the forward pass; its embedding was zero
     const float dt = (float)(times[i] - last_update[node]);
     const int slot = have_update ? node2slot[node] : -1;
 #pragma unroll
@@ -909,11 +912,8 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     const int relu_out = c.model == TGNN_MODEL_TGN ? 1 : 0;
     const size_t hf_smem = head_fused_smem(d);
     if (hf_smem <= 200 * 1024) {
-      static size_t attr_bytes = 0;
-      if (attr_bytes < hf_smem) {
-        TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(head_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)hf_smem));
-        attr_bytes = hf_smem;
-      }
+      static SmemLimit hf_limit;
+      RC(raise_smem_limit(ctx, head_fused_kernel, (int)hf_smem, hf_limit));
       const int groups = (n_q + HF_EV - 1) / HF_EV;
       {
         KernelScope scope__(ctx, "head_fused", s);
@@ -962,7 +962,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
         KernelScope scope__(ctx, "jodie_embed_bwd", s);
         jodie_embed_bwd_kernel<<<(R + 7) / 8 < 148 ? (R + 7) / 8 : 148, 256, tg_smem, s>>>(
             w.dpre_o, ctx->memory, ctx->last_update, P + L.proj_w, P + L.proj_b, ctx->e_nodes, ctx->e_times, R, d,
-            w.node2slot, ctx->have_update ? 1 : 0, w.dMemU, w.tg_acc + 2 * d);
+            w.node2slot, ctx->have_update ? 1 : 0, w.dMemU, w.tg_acc + 2 * d, c.num_nodes);
       }
       TGNN_LAUNCH_OK(ctx, "jodie_embed_bwd");
       if (ctx->have_update) {
@@ -996,26 +996,23 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     RC(grad_in(ctx, w.dpre_o, d, P + L.wo, 2 * d, 0, R, nullptr, d, 2 * d, w.dcat_o, 2 * d, "dcat_o", s, SITE_DCATO + 1));
     const int wpb = attn_warps_per_block(d, H, k);
     {
-      static int attr_bytes = 0;
+      static SmemLimit lim_f, lim_t;
       const int need = (int)attn_smem_bytes(d, H, k, wpb);
-      if (attr_bytes < need) {
-        TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(attention_bwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, need));
-        TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(attention_bwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, need));
-        attr_bytes = need;
-      }
+      RC(raise_smem_limit(ctx, attention_bwd_kernel<false>, need, lim_f));
+      RC(raise_smem_limit(ctx, attention_bwd_kernel<true>, need, lim_t));
     }
     const bool split = ctx->split_buf != nullptr && ctx->images_fresh;
     SplitMat dkvs = ctx->dkvs, zs = ctx->zs;
     dkvs.rows = NB; zs.rows = NB;
     {
       KernelScope scope__(ctx, "attention_bwd", s);
-      if (split)   // the key/value gradient leaves the kernel as bf16 planes, the form its two consumers read
+      if (split)   // the key/value gradient leaves the kernel as fp16 planes, the form its two consumers read
         attention_bwd_kernel<true><<<(R + wpb - 1) / wpb, wpb * 32, attn_smem_bytes(d, H, k, wpb), s>>>(
             w.Q, w.KV, w.alpha, w.dcat_o, ctx->e_cnt, R, d, H, k, w.dQ, nullptr, reinterpret_cast<__nv_bfloat16*>(dkvs.hi),
-            dkvs.plane_stride, (int)dkvs.ld);
+            dkvs.plane_stride, (int)dkvs.ld, dkvs.scale);
       else
         attention_bwd_kernel<false><<<(R + wpb - 1) / wpb, wpb * 32, attn_smem_bytes(d, H, k, wpb), s>>>(
-            w.Q, w.KV, w.alpha, w.dcat_o, ctx->e_cnt, R, d, H, k, w.dQ, w.dKV, nullptr, 0, 0);
+            w.Q, w.KV, w.alpha, w.dcat_o, ctx->e_cnt, R, d, H, k, w.dQ, w.dKV, nullptr, 0, 0, 1.f);
     }
     TGNN_LAUNCH_OK(ctx, "attention_bwd");
     RC(fork_to(ctx, s, sa));
@@ -1074,10 +1071,10 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
         // many rows per node (small node set, large batch): sum per block first, the hub rows would serialise
         if ((int64_t)NB >= 4 * c.num_nodes)
           scatter_dmem_cached_kernel<<<(NB + R + SC_ROWS - 1) / SC_ROWS, 256, (size_t)SC_WAYS * d * sizeof(float), s>>>(
-              w.dZmp, w.dcat_o, w.dzq, ctx->e_nbr, ctx->e_nodes, R, k, d, w.node2slot, w.dMemU);
+              w.dZmp, w.dcat_o, w.dzq, ctx->e_nbr, ctx->e_nodes, R, k, d, w.node2slot, w.dMemU, c.num_nodes);
         else
           scatter_dmem_kernel<<<(NB + R + 7) / 8, 256, 0, s>>>(w.dZmp, w.dcat_o, w.dzq, ctx->e_nbr, ctx->e_nodes, R, k, d,
-                                                               w.node2slot, w.dMemU);
+                                                               w.node2slot, w.dMemU, c.num_nodes);
       }
       TGNN_LAUNCH_OK(ctx, "scatter_dmem");
       const int U_cap = ctx->upd_cap;

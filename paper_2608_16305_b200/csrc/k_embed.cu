@@ -2,14 +2,12 @@
 #include "tgnn_internal.cuh"
 #include "tgnn_device.cuh"
 
-// Raises a kernel's dynamic shared-memory limit once (the attention kernels stage > 48 KB per block).
-#define RC_ATTR(ctx, kernel, bytes)                                                                                   \
-  do {                                                                                                                \
-    static int done__ = 0;                                                                                            \
-    if (done__ < (int)(bytes)) {                                                                                      \
-      TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(bytes)));     \
-      done__ = (int)(bytes);                                                                                          \
-    }                                                                                                                 \
+// Raises a kernel's dynamic shared-memory limit (the attention kernels stage > 48 KB per block), once per device.
+#define RC_ATTR(ctx, kernel, bytes)                                              \
+  do {                                                                           \
+    static tgnn::SmemLimit lim__;                                                \
+    const int rc__ = tgnn::raise_smem_limit(ctx, kernel, (int)(bytes), lim__);   \
+    if (rc__) return rc__;                                                       \
   } while (0)
 
 namespace tgnn {
@@ -37,7 +35,7 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_kernel(const void* __r
                                                               const int32_t* __restrict__ eid,
                                                               const double* __restrict__ ts, int ld,
                                                               float* __restrict__ Z, float* __restrict__ z_dt,
-                                                              float* __restrict__ Zq) {
+                                                              float* __restrict__ Zq, int64_t N, int64_t E, int32_t* status) {
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   const int nb_rows = n * k;
@@ -69,6 +67,8 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_kernel(const void* __r
       my_nbr = nbr[r];
       my_eid = eid[r];
       my_dt = (float)(times[r / k] - ts[r]);
+      // a slot naming a node or a feature row that does not exist is reported and treated as empty
+      if (my_nbr >= 0 && !(index_ok(my_nbr, N, status) & (de == 0 || index_ok(my_eid, E, status)))) my_nbr = -1;
     }
     uint32_t f[ZS_ROWS][ZS_FEAT];
     int v_nbr[ZS_ROWS];
@@ -149,11 +149,11 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_kernel(const void* __r
     for (int q = lane; q < d; q += 32) Zq[(int64_t)i * 2 * d + d + q] = time_encode(time_w[q], time_b[q], 0.f);
 }
 
-// The static part for the split-bf16 products: the same rows written as two bf16 planes (hi, lo; row pitch ld
+// The static part for the split-operand products: the same rows written as two fp16 planes (hi, lo; row pitch ld
 // elements, planes plane_s elements apart) -- columns [d, d + de) edge features, [d + de, dkv) time encoding,
 // column dkv a constant 1 (it turns the weight-gradient product's last column into the bias gradient), zeros up
 // to ld; an empty slot is a row of zeros.  Values travel as pairs of neighbouring columns packed into 32-bit
-// words (d and de are even).  bf16 features are exact in the hi plane; fp32 features and the encodings are split.
+// words (d and de are even).  Both planes hold fp16 numbers (activations of moderate size: 22 mantissa bits).
 __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const void* __restrict__ efeat, int feat_bf16,
                                                                     const float* __restrict__ time_w,
                                                                     const float* __restrict__ time_b, int d, int de, int k,
@@ -162,7 +162,8 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
                                                                     const int32_t* __restrict__ eid,
                                                                     const double* __restrict__ ts, int ld,
                                                                     __nv_bfloat16* __restrict__ z_hi, int64_t plane_s,
-                                                                    float* __restrict__ z_dt, float* __restrict__ Zq) {
+                                                                    float* __restrict__ z_dt, float* __restrict__ Zq, int64_t N,
+                                                                    int64_t E, int32_t* status) {
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   const int nb_rows = n * k;
@@ -188,6 +189,8 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
       my_nbr = nbr[r];
       my_eid = eid[r];
       my_dt = (float)(times[r / k] - ts[r]);
+      // a slot naming a node or a feature row that does not exist is reported and treated as empty
+      if (my_nbr >= 0 && !(index_ok(my_nbr, N, status) & (de == 0 || index_ok(my_eid, E, status)))) my_nbr = -1;
     }
     // feature pairs of both rows first (the dependent chain slot -> event id -> feature row is paid once)
     uint32_t fa[ZS_ROWS][FP_MAX], fb[ZS_ROWS][FP_MAX];   // bf16 table: fa = the pair as stored; fp32 table: fa, fb = the two floats
@@ -231,8 +234,9 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
         for (int u = 0; u < FP_MAX; ++u) {
           const int q = lane + 32 * u;
           if (q < fp) {
-            uint32_t h = fa[j][u], l = 0u;
-            if (!feat_bf16) split_bf16_pair(__uint_as_float(fa[j][u]), __uint_as_float(fb[j][u]), &h, &l);
+            uint32_t h, l;
+            if (feat_bf16) split_f16_pair(__uint_as_float(fa[j][u] << 16), __uint_as_float(fa[j][u] & 0xffff0000u), &h, &l);
+            else split_f16_pair(__uint_as_float(fa[j][u]), __uint_as_float(fb[j][u]), &h, &l);
             hi[(d >> 1) + q] = h; lo[(d >> 1) + q] = l;
           }
         }
@@ -241,29 +245,30 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
           const int q = lane + 32 * u;
           if (q < tp) {
             uint32_t h, l;
-            split_bf16_pair(time_encode(tw[u][0], tb[u][0], dtf), time_encode(tw[u][1], tb[u][1], dtf), &h, &l);
+            split_f16_pair(time_encode(tw[u][0], tb[u][0], dtf), time_encode(tw[u][1], tb[u][1], dtf), &h, &l);
             hi[((d + de) >> 1) + q] = h; lo[((d + de) >> 1) + q] = l;
           }
         }
       } else {   // very wide rows: straight from memory, pair by pair
         for (int q = lane; q < fp; q += 32) {
-          uint32_t h, l = 0u;
+          uint32_t h, l;
           if (feat_bf16) {
-            h = __ldg(reinterpret_cast<const uint32_t*>(efeat) + (int64_t)v_eid[j] * fp + q);
+            const uint32_t w2 = __ldg(reinterpret_cast<const uint32_t*>(efeat) + (int64_t)v_eid[j] * fp + q);
+            split_f16_pair(__uint_as_float(w2 << 16), __uint_as_float(w2 & 0xffff0000u), &h, &l);
           } else {
             const uint2 x = __ldg(reinterpret_cast<const uint2*>(efeat) + (int64_t)v_eid[j] * fp + q);
-            split_bf16_pair(__uint_as_float(x.x), __uint_as_float(x.y), &h, &l);
+            split_f16_pair(__uint_as_float(x.x), __uint_as_float(x.y), &h, &l);
           }
           hi[(d >> 1) + q] = h; lo[(d >> 1) + q] = l;
         }
         for (int q = lane; q < tp; q += 32) {
           uint32_t h, l;
-          split_bf16_pair(time_encode(time_w[2 * q], time_b[2 * q], dtf), time_encode(time_w[2 * q + 1], time_b[2 * q + 1], dtf), &h, &l);
+          split_f16_pair(time_encode(time_w[2 * q], time_b[2 * q], dtf), time_encode(time_w[2 * q + 1], time_b[2 * q + 1], dtf), &h, &l);
           hi[((d + de) >> 1) + q] = h; lo[((d + de) >> 1) + q] = l;
         }
       }
       // column dkv = 1, then zeros up to the row pitch (dkv is even, the pitch a multiple of 8)
-      for (int q = (dkv >> 1) + lane; q < (ld >> 1); q += 32) { hi[q] = q == (dkv >> 1) ? 0x3f80u : 0u; lo[q] = 0u; }
+      for (int q = (dkv >> 1) + lane; q < (ld >> 1); q += 32) { hi[q] = q == (dkv >> 1) ? 0x3c00u : 0u; lo[q] = 0u; }
       if (lane == 0) z_dt[r] = dtf;
     }
   }
@@ -274,14 +279,14 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
 
 // Memory part.  Rows [0, n*k): columns [0, d) of Z for the valid slots.  Rows [n*k, n*k + n): the
 // memory half of z_q and of cat_o.
-// z_hi != nullptr: the neighbor rows go to the two bf16 planes of the split products instead (pitch ld_s, planes
+// z_hi != nullptr: the neighbor rows go to the two fp16 planes of the split products instead (pitch ld_s, planes
 // plane_s apart), as pairs of columns packed into 32-bit words.
 __global__ void __launch_bounds__(256) gather_z_memory_kernel(const float* __restrict__ memory, int d, int k,
                                                               const int32_t* __restrict__ nodes, int n,
                                                               const int32_t* __restrict__ nbr, int ld,
                                                               float* __restrict__ Z, float* __restrict__ Zq,
                                                               float* __restrict__ cat_o, __nv_bfloat16* __restrict__ z_hi,
-                                                              int64_t plane_s, int ld_s) {
+                                                              int64_t plane_s, int ld_s, int64_t N, int32_t* status) {
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   const int nb_rows = n * k;
@@ -293,7 +298,10 @@ __global__ void __launch_bounds__(256) gather_z_memory_kernel(const float* __res
     for (int r0 = wg * 4; r0 < nb_rows; r0 += warps * 4) {
       int nb[4];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) nb[j] = r0 + j < nb_rows ? __ldg(nbr + r0 + j) : -1;
+      for (int j = 0; j < 4; ++j) {
+        nb[j] = r0 + j < nb_rows ? __ldg(nbr + r0 + j) : -1;
+        if (nb[j] >= N) nb[j] = -1;   // reported by the static half, which left the row empty
+      }
       float4 x[4][2];
 #pragma unroll
       for (int j = 0; j < 4; ++j)
@@ -313,8 +321,8 @@ __global__ void __launch_bounds__(256) gather_z_memory_kernel(const float* __res
           const int q = lane + 32 * u;
           if (q < d4) {
             uint2 h, l;
-            split_bf16_pair(x[j][u].x, x[j][u].y, &h.x, &l.x);
-            split_bf16_pair(x[j][u].z, x[j][u].w, &h.y, &l.y);
+            split_f16_pair(x[j][u].x, x[j][u].y, &h.x, &l.x);
+            split_f16_pair(x[j][u].z, x[j][u].w, &h.y, &l.y);
             hi[q] = h; lo[q] = l;
           }
         }
@@ -324,9 +332,13 @@ __global__ void __launch_bounds__(256) gather_z_memory_kernel(const float* __res
   for (int r = (z_hi != nullptr ? nb_rows : 0) + ((blockIdx.x * blockDim.x + threadIdx.x) >> 5); r < nb_rows + n; r += warps) {
     if (r < nb_rows) {
       const int nb = nbr[r];
-      if (nb >= 0) warp_copy_f32(Z + (int64_t)r * ld, memory + (int64_t)nb * d, d, lane);
+      if (nb >= 0 && nb < N) warp_copy_f32(Z + (int64_t)r * ld, memory + (int64_t)nb * d, d, lane);
     } else {
       const int i = r - nb_rows;
+      if (!index_ok(nodes[i], N, lane == 0 ? status : nullptr)) {   // a root outside the graph: reported, zero rows
+        for (int q = lane; q < d; q += 32) { Zq[(int64_t)i * 2 * d + q] = 0.f; cat_o[(int64_t)i * 2 * d + d + q] = 0.f; }
+        continue;
+      }
       const float* m = memory + (int64_t)nodes[i] * d;
       warp_copy_f32(Zq + (int64_t)i * 2 * d, m, d, lane);
       warp_copy_f32(cat_o + (int64_t)i * 2 * d + d, m, d, lane);
@@ -350,7 +362,7 @@ __global__ void __launch_bounds__(256) attention_fwd_kernel(const float* __restr
   float* al = Qs + 2 * d;  // logits
   float* pr = al + H * k;  // probabilities
   const int dh = d / H;
-  const int c = cnt[i];
+  const int c = max(0, min(cnt[i], k));   // a count outside [0, k] is clamped (the neighbor search never produces one)
   const float scale = rsqrtf((float)dh);
   attn_stage_issue(Ks, Vs, Qs, Q, KV, i, c, d, k, lane);
   attn_stage_wait();
@@ -395,11 +407,15 @@ __global__ void __launch_bounds__(256) jodie_embed_kernel(const float* __restric
                                                           const float* __restrict__ proj_b,
                                                           const int32_t* __restrict__ nodes,
                                                           const double* __restrict__ times, int n, int d,
-                                                          float* __restrict__ h) {
+                                                          float* __restrict__ h, int64_t N, int32_t* status) {
   const int lane = threadIdx.x & 31;
   const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   if (i >= n) return;
   const int node = nodes[i];
+  if (!index_ok(node, N, lane == 0 ? status : nullptr)) {   // reported; the embedding of a node that does not exist is zero
+    for (int q = lane; q < d; q += 32) h[(int64_t)i * d + q] = 0.f;
+    return;
+  }
   const float dt = (float)(times[i] - last_update[node]);
   const float4* m4 = reinterpret_cast<const float4*>(memory + (int64_t)node * d);
   float4* h4 = reinterpret_cast<float4*>(h + (int64_t)i * d);
@@ -429,11 +445,12 @@ int launch_embed_static(tgnn_ctx* ctx, const double* times, int n, const int32_t
     if (ctx->split_buf != nullptr && ctx->z_split)
       gather_z_static_split_kernel<<<(n * c.k / ZS_ROWS + n + 7) / 8 + 1, 256, 0, s>>>(
           ctx->efeat, c.feat_dtype == TGNN_BF16, ctx->params + L.time_w, ctx->params + L.time_b, c.d, c.d_e, c.k, times, n, nbr,
-          eid, ts, (int)ctx->zs.ld, reinterpret_cast<__nv_bfloat16*>(ctx->zs.hi), ctx->zs.plane_stride, w.z_dt, w.Zq);
+          eid, ts, (int)ctx->zs.ld, reinterpret_cast<__nv_bfloat16*>(ctx->zs.hi), ctx->zs.plane_stride, w.z_dt, w.Zq,
+          c.num_nodes, ctx->num_events, w.status);
     else
       gather_z_static_kernel<<<(n * c.k / ZS_ROWS + n + 7) / 8 + 1, 256, 0, s>>>(ctx->efeat, c.feat_dtype == TGNN_BF16, ctx->params + L.time_w,
                                                           ctx->params + L.time_b, c.d, c.d_e, c.k, times, n, nbr, eid, ts,
-                                                          ctx->ld_kv, w.Z, w.z_dt, w.Zq);
+                                                          ctx->ld_kv, w.Z, w.z_dt, w.Zq, c.num_nodes, ctx->num_events, w.status);
   }
   TGNN_LAUNCH_OK(ctx, "gather_z_static");
   return TGNN_OK;
@@ -450,13 +467,13 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
     {
       KernelScope scope__(ctx, "jodie_embed", s);
       jodie_embed_kernel<<<(n + 7) / 8, 256, 0, s>>>(ctx->memory, ctx->last_update, ctx->params + L.proj_w,
-                                                     ctx->params + L.proj_b, nodes, times, n, d, h_out);
+                                                     ctx->params + L.proj_b, nodes, times, n, d, h_out, c.num_nodes, w.status);
     }
     TGNN_LAUNCH_OK(ctx, "jodie_embed");
     return TGNN_OK;
   }
   const int rows = n * k + n;
-  // split-bf16 operands: the attention inputs are written as bf16 planes, complete before the product starts
+  // split operands: the attention inputs are written as fp16 planes, complete before the product starts
   const bool split = ctx->split_buf != nullptr && ctx->images_fresh;
   if (!ctx->z_static_done) {
     ctx->z_split = split;
@@ -479,7 +496,7 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
     const int gblocks = split ? ((rows + 31) / 32 < 148 * 6 ? (rows + 31) / 32 : 148 * 6) : (rows + 7) / 8;
     gather_z_memory_kernel<<<gblocks, 256, 0, sg>>>(ctx->memory, d, k, nodes, n, nbr, ctx->ld_kv, w.Z, w.Zq, w.cat_o,
                                                            split ? reinterpret_cast<__nv_bfloat16*>(ctx->zs.hi) : nullptr,
-                                                           ctx->zs.plane_stride, (int)ctx->zs.ld);
+                                                           ctx->zs.plane_stride, (int)ctx->zs.ld, c.num_nodes, w.status);
   }
   TGNN_LAUNCH_OK(ctx, "gather_z_memory");
   if (!indirect) {  // the query projection below runs on the side stream and needs the rows just gathered
@@ -491,7 +508,7 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
   g.B = ctx->params + L.wk; g.b_rs = 1; g.b_cs = L.dkv;  // rows of [W_k; W_v]
   g.C = w.KV; g.ldc = 2 * d; g.M = n * k; g.N = 2 * d; g.K = (int)L.dkv;
   g.bias = ctx->params + L.bk; g.split_k = 1; g.site = SITE_KV + 1;
-  if (indirect) { g.a_idx = nbr; g.a_tab = ctx->memory; g.a_tab_cols = d; }
+  if (indirect) { g.a_idx = nbr; g.a_tab = ctx->memory; g.a_tab_cols = d; g.a_tab_rows = c.num_nodes; }
   if (split) {
     SplitMat zs = ctx->zs;
     zs.rows = n * k;

@@ -1,6 +1,8 @@
 // Dense projections, fp32 FMA path: a strided tiled GEMM used for every
 // projection and its two gradient products when math_mode is TGNN_MATH_FP32,
 // and for the small products in every mode.
+#include <cstdio>
+
 #include "tgnn_internal.cuh"
 
 namespace tgnn {
@@ -94,6 +96,10 @@ int launch_gemm(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t
     if (ctx->cfg.math_mode != TGNN_MATH_TF32_FAST) gp.precise = 1;
     const int rc = launch_gemm_tf32(ctx, gp, name, s);
     if (rc != 1) return rc;  // 1: shape not handled by the tensor-core kernel, use the FMA tiles
+    // not an error, but not silent either: the note stays in tgnn_last_error and the launches are counted
+    ctx->fma_fallbacks++;
+    snprintf(ctx->err, sizeof(ctx->err), "note: product %s (M=%d N=%d K=%d) does not fit the tensor-core kernel and ran on the "
+             "fp32 FMA tiles (%lld such launches so far)", name, g.M, g.N, g.K, (long long)ctx->fma_fallbacks);
   }
   if (g.a_idx) return set_error(ctx, TGNN_EINVAL, "gemm %s: row-indirect A needs the tensor-core path", name);
   dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.split_k < 1 ? 1 : g.split_k);

@@ -1,24 +1,29 @@
-// The large projections on the 5th-generation tensor cores with split-bf16 operands (TGNN_MATH_BF16X3).
+// The large projections on the 5th-generation tensor cores with split 16-bit operands (TGNN_MATH_F16X3).
 //
-// An fp32 value x is held as two bf16 numbers, hi = bf16(x) and lo = bf16(x - hi): together they carry 16
-// mantissa bits (error below 2^-17 relative).  A product A B is then three tensor-core passes at the bf16 rate,
+// An fp32 value x is held as two 16-bit numbers, hi = r16(x) and lo = r16(x - hi).  With fp16 planes (what the
+// library uses) they carry 22 mantissa bits for values inside fp16's range -- activations and weights as they are,
+// gradients after multiplication by a power of two that the epilogue divides out again; with bf16 planes 16 bits
+// at any range.  A product A B is then three tensor-core passes at the 16-bit rate,
 //   lo(A) hi(B) + hi(A) lo(B) + hi(A) hi(B),
-// with fp32 accumulation in tensor memory -- more accurate than one TF32 pass (10 mantissa bits) at 1.5 times its
-// cost, and half the cost of the three-pass TF32 split.  The operands are STORED split (two bf16 planes of the
-// same shape, written by the kernel that produces the activation), so this kernel never touches operand
-// data with a thread: tiles go from global memory to shared memory by the tensor-memory-access unit,
-// already in the 128-byte-swizzled layout the MMA descriptors expect, and from there into the tensor cores.
+// with fp32 accumulation in tensor memory: the accuracy of the three-pass TF32 split at half its tensor time.  (One
+// MMA cannot mix an fp16 operand with a bf16 one -- the hardware rejects it as an illegal instruction -- so both
+// operands of a product use the same plane format.)  The operands are STORED split (two planes of the same shape,
+// written by the kernel that produces the activation), so this kernel never touches operand data with a thread:
+// tiles go from global memory to shared memory by the tensor-memory-access unit, already in the 128-byte-swizzled
+// layout the MMA descriptors expect, and from there into the tensor cores.
 //
-// Roles (320 threads): warp 0 issues the tile copies, warp 1 owns tensor memory and issues the MMAs,
+// Roles (320 threads): warp 0 issues the tile copies (one per operand tile: the box spans both planes), warp 1 owns tensor memory and issues the MMAs,
 // warps 2-9 are the epilogue (tensor memory -> registers -> a small staging square -> global memory in
 // whole 64-byte row segments, with bias / ReLU or an atomic accumulate).
 //
-// A CTA is persistent: it walks work items (pair of 128-row tiles, n-tile, contraction split).  The two row
-// tiles of a pair share every B tile, which halves the B traffic per flop; their accumulators sit side by
-// side in tensor memory (2 x 256 columns).  A tiles and B tiles travel through two separate rings of
-// shared-memory slots, each slot with a full (copy landed) and an empty (MMAs that read it retired,
-// signalled by tcgen05.commit) mbarrier, so copies run several slots ahead of the MMAs and across item
-// boundaries.  Every wait is bounded: on expiry the kernel records TGNN_ETIMEOUT, all roles leave their
+// A CTA is persistent: it takes a contiguous range of tile units (n-tile / contraction-split combination major,
+// 128-row tile minor).  Activation x weight products walk it one row tile at a time with the accumulator
+// alternating between the two halves of tensor memory, so the epilogue of one tile (a full store of C) runs
+// while the MMAs of the next are issued.  Weight gradients (one long contraction range per CTA) take two row
+// tiles at once, which share every B tile; their accumulators sit side by side.  A tiles and B tiles travel
+// through two separate rings of shared-memory slots, each slot with a full (copy landed) and an empty (MMAs that
+// read it retired, signalled by tcgen05.commit) mbarrier, so copies run several slots ahead of the MMAs and across
+// item boundaries.  Every wait is bounded: on expiry the kernel records TGNN_ETIMEOUT, all roles leave their
 // loops, tensor memory is freed and the kernel returns.
 //
 // Operand layouts.  K-major (the contraction index is contiguous in memory: activations [M, K] and weight
@@ -30,6 +35,7 @@
 // rows SBO = 1024 bytes apart; one MMA step consumes two such groups.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "tgnn_internal.cuh"
 
@@ -53,6 +59,11 @@ struct BfArgs {
   const float* bias;
   int relu, accumulate;
   int mn_major;               // 0: both operands K-major; 1: both MN-major
+  int fp16;                   // both operands' planes hold fp16 numbers (bf16 otherwise; the two may not be mixed)
+  float out_scale;            // the product is multiplied by this (undoes the operands' power-of-two scales)
+  int single;                 // work items are single row tiles whose accumulators alternate between the two halves of
+                              // tensor memory, so that the epilogue of one overlaps the MMAs of the next (B tiles are
+                              // then fetched once per row tile instead of once per pair)
   int m_tiles, n_tiles, bn, split_k;
   int kb_total;               // contraction blocks (64 elements K-major, 32 rows MN-major)
   int ksteps_total;           // MMA steps of 16 over the whole contraction
@@ -109,7 +120,7 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
   d |= (uint64_t)2 << 61;   // 128-byte swizzle
   return d;
 }
-__device__ __forceinline__ void mma_bf16(uint32_t tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+__device__ __forceinline__ void mma_f16(uint32_t tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
@@ -146,7 +157,7 @@ __device__ __forceinline__ bool next_item(const BfArgs& g, Walk& wk, Item& it) {
   while (wk.u < wk.u_end) {
     const int combo = wk.u / g.m_tiles, mt = wk.u - combo * g.m_tiles;
     it.mt0 = mt;
-    it.tiles = min(2, min(wk.u_end - wk.u, g.m_tiles - mt));
+    it.tiles = g.single ? 1 : min(2, min(wk.u_end - wk.u, g.m_tiles - mt));
     wk.u += it.tiles;
     const int nt = combo % g.n_tiles, sp = combo / g.n_tiles;
     it.n0 = nt * g.bn;
@@ -165,10 +176,10 @@ __device__ __forceinline__ void tma_4d(uint32_t dst, const CUtensorMap* map, int
       : "memory");
 }
 
-__global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_constant__ BfArgs g) {
+__global__ void __launch_bounds__(THREADS, 1) gemm_split_kernel(const __grid_constant__ BfArgs g) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t s_full_a[MAX_SLOTS], s_empty_a[MAX_SLOTS], s_full_b[MAX_SLOTS], s_empty_b[MAX_SLOTS];
-  __shared__ __align__(8) uint64_t s_tmem_full, s_tmem_empty;
+  __shared__ __align__(8) uint64_t s_tmem_full[2], s_tmem_empty[2];
   __shared__ uint32_t s_tmem;
   __shared__ int s_abort;
 
@@ -183,8 +194,10 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
       mbar_init(smem_u32(&s_full_a[s]), 1); mbar_init(smem_u32(&s_empty_a[s]), 1);
       mbar_init(smem_u32(&s_full_b[s]), 1); mbar_init(smem_u32(&s_empty_b[s]), 1);
     }
-    mbar_init(smem_u32(&s_tmem_full), 1);
-    mbar_init(smem_u32(&s_tmem_empty), EPI_WARPS);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&s_tmem_full[b]), 1);
+      mbar_init(smem_u32(&s_tmem_empty[b]), EPI_WARPS);
+    }
     s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -256,12 +269,16 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
       Walk wk = cta_walk(g);
       Item it;
       while (ok && next_item(g, wk, it)) {
-        ok = mbar_wait(smem_u32(&s_tmem_empty), (n_item & 1u) ^ 1u, limit, abort_flag);   // accumulators drained
+        const uint32_t buf = g.single ? (n_item & 1u) : 0u, use = g.single ? (n_item >> 1) : n_item;
+        ok = mbar_wait(smem_u32(&s_tmem_empty[buf]), (use & 1u) ^ 1u, limit, abort_flag);   // accumulators drained
         if (!ok) break;
         ++n_item;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int n_mma = (it.n_valid + 15) / 16 * 16;
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (mn << 15) | (mn << 16) |
+        // instruction descriptor: D fp32; A and B formats (the same for both: 1 = bf16, 0 = fp16 -- an MMA that
+        // mixes the two is an illegal instruction); majors; N >> 3; M >> 4
+        const uint32_t fmt = g.fp16 ? 0u : 1u;
+        const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | (mn << 15) | (mn << 16) |
                                ((uint32_t)(n_mma >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
         for (int kb = it.kb0; kb < it.kb1 && ok; ++kb) {
           const uint32_t sb = cb % (uint32_t)g.n_b_slots;
@@ -276,16 +293,16 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             TRACE(16 + 2 * (int)ca);
             const uint32_t a_addr = a_ring + sa * a_bytes;
-            const uint32_t acc = tmem + (uint32_t)(t * ACC_STRIDE);
+            const uint32_t acc = tmem + (uint32_t)((g.single ? (int)buf : t) * ACC_STRIDE);
             for (int ks = 0; ks < ks_n; ++ks) {
               const uint64_t da_hi = make_desc(a_addr + ks * kstep_bytes, lbo, sbo);
               const uint64_t da_lo = make_desc(a_addr + a_plane + ks * kstep_bytes, lbo, sbo);
               const uint64_t db_hi = make_desc(b_addr + ks * kstep_bytes, lbo, sbo);
               const uint64_t db_lo = make_desc(b_addr + b_plane + ks * kstep_bytes, lbo, sbo);
               const uint32_t first = (kb > it.kb0 || ks > 0) ? 1u : 0u;
-              mma_bf16(acc, da_lo, db_hi, idesc, first);
-              mma_bf16(acc, da_hi, db_lo, idesc, 1u);
-              mma_bf16(acc, da_hi, db_hi, idesc, 1u);
+              mma_f16(acc, da_lo, db_hi, idesc, first);
+              mma_f16(acc, da_hi, db_lo, idesc, 1u);
+              mma_f16(acc, da_hi, db_hi, idesc, 1u);
             }
             TRACE(17 + 2 * (int)ca);
             if (withheld < g.debug_withhold) ++withheld;   // test hook: this slot is never handed back
@@ -295,7 +312,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
           if (ok) commit_to(smem_u32(&s_empty_b[sb]));
           ++cb;
         }
-        if (ok) commit_to(smem_u32(&s_tmem_full));
+        if (ok) commit_to(smem_u32(&s_tmem_full[buf]));
       }
       if (!ok) { s_abort = 1; atomicCAS(g.status, 0, TGNN_ETIMEOUT); }
     }
@@ -313,17 +330,22 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
     Walk wk = cta_walk(g);
     Item it;
     while (ok && next_item(g, wk, it)) {
-      ok = mbar_wait(smem_u32(&s_tmem_full), n_item & 1u, limit, abort_flag);
+      const uint32_t buf = g.single ? (n_item & 1u) : 0u, use = g.single ? (n_item >> 1) : n_item;
+      ok = mbar_wait(smem_u32(&s_tmem_full[buf]), use & 1u, limit, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       if (e == 0 && lane == 0) TRACE(2 + 2 * (int)n_item);
       ++n_item;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      if (t < it.tiles) {
-        const int m0 = (it.mt0 + t) * BM;
-        const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(t * ACC_STRIDE);
+      // pairs: warps 2-5 drain the first tile's accumulator, 6-9 the second's.  Single tiles: all eight warps
+      // drain the one accumulator, the two warps of a lane quarter taking alternate 32-column groups.
+      const int acc_i = g.single ? (int)buf : t;
+      const int c_first = g.single ? 32 * t : 0, c_step = g.single ? 64 : 32;
+      if (g.single || t < it.tiles) {
+        const int m0 = (it.mt0 + (g.single ? 0 : t)) * BM;
+        const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(acc_i * ACC_STRIDE);
         const bool with_bias = g.bias != nullptr && it.kb0 == 0;
-        for (int c0 = 0; c0 < it.n_valid; c0 += 32) {
+        for (int c0 = c_first; c0 < it.n_valid; c0 += c_step) {
           uint32_t r[32];
           asm volatile(
               "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
@@ -360,7 +382,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
               const int row = m0 + q4 * 32 + rr;
               float4 v = *reinterpret_cast<const float4*>(stg + rr * STG_PITCH + 4 * ch);
               if (row < g.M && col < it.n_valid) {
-                v.x += b4.x; v.y += b4.y; v.z += b4.z; v.w += b4.w;
+                v.x = fmaf(v.x, g.out_scale, b4.x); v.y = fmaf(v.y, g.out_scale, b4.y);
+                v.z = fmaf(v.z, g.out_scale, b4.z); v.w = fmaf(v.w, g.out_scale, b4.w);
                 float* cp = g.C + (int64_t)row * g.ldc + it.n0 + col;
                 if (g.accumulate) {
                   if (full4 && c_vec) {
@@ -391,7 +414,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (e == 0 && lane == 0) TRACE(1 + 2 * (int)n_item);
-      if (lane == 0) mbar_arrive(smem_u32(&s_tmem_empty));
+      if (lane == 0) mbar_arrive(smem_u32(&s_tmem_empty[buf]));
     }
     if (!ok && lane == 0) { s_abort = 1; atomicCAS(g.status, 0, TGNN_ETIMEOUT); }
   }
@@ -408,11 +431,12 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_bf16s_kernel(const __grid_con
   }
 }
 
-// fp32 rows -> two bf16 planes (hi, lo).  One thread per 4 consecutive columns; columns in [cols, ld_out) of the
+// fp32 rows -> two 16-bit planes (hi, lo), fp16 or bf16, after multiplication by `scale`.  One thread per 4 consecutive columns; columns in [cols, ld_out) of the
 // planes are written as zeros except column `ones_col` (if >= 0), which is 1 (the bias column of a weight gradient).
 __global__ void __launch_bounds__(256) split_rows_kernel(const float* __restrict__ X, int64_t ld_in, int64_t rows, int cols,
                                                          const int32_t* __restrict__ dev_rows, __nv_bfloat16* __restrict__ hi,
-                                                         __nv_bfloat16* __restrict__ lo, int64_t ld_out, int ones_col) {
+                                                         __nv_bfloat16* __restrict__ lo, int64_t ld_out, int ones_col,
+                                                         int fp16, float scale) {
   const int per_row = (int)(ld_out >> 2);
   const int64_t n_rows = dev_rows ? min((int64_t)*dev_rows, rows) : rows;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < rows * per_row; i += (int64_t)gridDim.x * blockDim.x) {
@@ -422,13 +446,20 @@ __global__ void __launch_bounds__(256) split_rows_kernel(const float* __restrict
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const int cc = c + e;
-      v[e] = (r < n_rows && cc < cols) ? X[r * ld_in + cc] : ((cc == ones_col && r < n_rows) ? 1.f : 0.f);
+      v[e] = (r < n_rows && cc < cols) ? scale * X[r * ld_in + cc] : ((cc == ones_col && r < n_rows) ? 1.f : 0.f);
     }
-    __nv_bfloat16 h[4], l[4];
+    unsigned short h[4], l[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      h[e] = __float2bfloat16_rn(v[e]);
-      l[e] = __float2bfloat16_rn(v[e] - __bfloat162float(h[e]));
+      if (fp16) {
+        const __half hh = __float2half_rn(v[e]);
+        h[e] = __half_as_ushort(hh);
+        l[e] = __half_as_ushort(__float2half_rn(v[e] - __half2float(hh)));
+      } else {
+        const __nv_bfloat16 hh = __float2bfloat16_rn(v[e]);
+        h[e] = __bfloat16_as_ushort(hh);
+        l[e] = __bfloat16_as_ushort(__float2bfloat16_rn(v[e] - __bfloat162float(hh)));
+      }
     }
     *reinterpret_cast<uint2*>(hi + r * ld_out + c) = *reinterpret_cast<const uint2*>(h);
     *reinterpret_cast<uint2*>(lo + r * ld_out + c) = *reinterpret_cast<const uint2*>(l);
@@ -439,7 +470,7 @@ __global__ void __launch_bounds__(256) split_rows_kernel(const float* __restrict
 //   wkv[n, k] = W_kv[n, k]                      (n < 2d, k < dkv: the forward projection's B operand)
 //   wz[n, k]  = W_kv[k, col(n)]                 (n < 2d, k < 2d: the input gradient toward the memory columns,
 //               col(n) = n for n < d, and the time-encoding columns, col(n) = d + de + (n - d) otherwise)
-// Padding columns of the planes are zero.
+// Padding columns of the planes are zero.  Both planes hold fp16 numbers.
 __global__ void __launch_bounds__(256) prep_split_weights_kernel(const float* __restrict__ Wkv, int d, int de,
                                                                  __nv_bfloat16* __restrict__ wkv_hi, int64_t wkv_plane, int ld_kv,
                                                                  __nv_bfloat16* __restrict__ wz_hi, int64_t wz_plane, int ld_z) {
@@ -458,9 +489,9 @@ __global__ void __launch_bounds__(256) prep_split_weights_kernel(const float* __
       if (k < n_rows) v = Wkv[(int64_t)k * dkv + (n < d ? n : d + de + (n - d))];
       hi = wz_hi + j; lo = wz_hi + wz_plane + j;
     }
-    const __nv_bfloat16 h = __float2bfloat16_rn(v);
-    *hi = h;
-    *lo = __float2bfloat16_rn(v - __bfloat162float(h));
+    const __half h = __float2half_rn(v);   // weights: two fp16 numbers
+    *reinterpret_cast<__half*>(hi) = h;
+    *reinterpret_cast<__half*>(lo) = __float2half_rn(v - __half2float(h));
   }
 }
 
@@ -539,7 +570,8 @@ int launch_split_rows(tgnn_ctx* ctx, const float* X, int64_t ld_in, int64_t rows
   {
     KernelScope scope__(ctx, name, s);
     split_rows_kernel<<<blocks, 256, 0, s>>>(X, ld_in, rows, cols, dev_rows, reinterpret_cast<__nv_bfloat16*>(out.hi),
-                                             reinterpret_cast<__nv_bfloat16*>(out.hi) + out.plane_stride, out.ld, ones_col);
+                                             reinterpret_cast<__nv_bfloat16*>(out.hi) + out.plane_stride, out.ld, ones_col,
+                                             out.fp16, out.scale);
   }
   TGNN_LAUNCH_OK(ctx, name);
   return TGNN_OK;
@@ -551,13 +583,20 @@ int launch_split_rows(tgnn_ctx* ctx, const float* X, int64_t ld_in, int64_t rows
 // split_k > 1 needs accumulate (C holds valid data; partial sums are added atomically).
 int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int mn_major, float* C, int64_t ldc, int M, int N,
                       int K, const float* bias, int relu, int accumulate, int split_k, const char* name, cudaStream_t s,
-                      int debug_withhold, unsigned spin_limit, int extra_col, float* extra_out, long long* trace) {
+                      int debug_withhold, unsigned spin_limit, int extra_col, float* extra_out, long long* trace, int single) {
   if (M <= 0 || N <= 0) return TGNN_OK;
   if (K <= 0) return set_error(ctx, TGNN_EINVAL, "gemm %s: empty contraction", name);
   if (split_k > 1 && !accumulate) return set_error(ctx, TGNN_EINVAL, "gemm %s: split_k needs accumulate", name);
   BfArgs a = {};
   a.C = C; a.ldc = ldc; a.M = M; a.N = N; a.K = K; a.bias = bias; a.relu = relu; a.accumulate = accumulate;
   a.mn_major = mn_major ? 1 : 0;
+  if ((A.fp16 != 0) != (B.fp16 != 0))
+    return set_error(ctx, TGNN_EINVAL, "gemm %s: one operand is held as fp16 planes and the other as bf16 planes", name);
+  a.fp16 = A.fp16 ? 1 : 0;
+  a.out_scale = 1.f / (A.scale * B.scale);
+  // single row tiles with alternating accumulators for the activation x weight products (their epilogue, a full
+  // store of C, then overlaps the next tile's MMAs); pairs for the weight gradients (one item per CTA, B shared)
+  a.single = single >= 0 ? (single ? 1 : 0) : (mn_major ? 0 : 1);
   a.status = ctx->ws.status;
   a.extra_col = (extra_out && accumulate) ? extra_col : -1;
   a.extra_out = extra_out;
@@ -604,19 +643,16 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
                                 : (encode_k_map(&a.a_map, A, BM) && encode_k_map(&a.b_map, B, b_rows));
   if (!maps_ok) return set_error(ctx, TGNN_ECUDA, "gemm %s: tensor map encoding failed", name);
   const int units = a.m_tiles * a.n_tiles * a.split_k;
-  const int items = (units + 1) / 2;
+  const int items = a.single ? units : (units + 1) / 2;
   const int smem = 1024 + a.n_a_slots * a.a_slot_bytes + a.n_b_slots * a.b_slot_bytes + STG_BYTES;
-  static int attr_bytes[64] = {};
-  int dev = 0;
-  TGNN_CUDA_OK(ctx, cudaGetDevice(&dev));
-  if (dev >= 0 && dev < 64 && attr_bytes[dev] < smem) {
-    // the largest dynamic size any shape asks for (the static barriers take a few hundred bytes of the 227 KB)
-    TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(gemm_bf16s_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 1024));
-    attr_bytes[dev] = SMEM_LIMIT - 1024;
+  static SmemLimit smem_limit;
+  {  // the largest dynamic size any shape asks for (the static barriers take a few hundred bytes of the 227 KB)
+    const int rc = raise_smem_limit(ctx, gemm_split_kernel, SMEM_LIMIT - 1024, smem_limit);
+    if (rc) return rc;
   }
   {
     KernelScope scope__(ctx, name, s);
-    gemm_bf16s_kernel<<<items < 148 ? items : 148, THREADS, smem, s>>>(a);
+    gemm_split_kernel<<<items < 148 ? items : 148, THREADS, smem, s>>>(a);
   }
   TGNN_LAUNCH_OK(ctx, name);
   return TGNN_OK;

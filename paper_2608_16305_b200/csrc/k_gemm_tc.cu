@@ -64,6 +64,7 @@ struct TcArgs {
   const int32_t* a_idx;
   const float* a_tab;
   int a_tab_cols;
+  int64_t a_tab_rows;
   // K-major A as a tiled tensor map (box 32 x 128, 128-byte swizzle): the tensor-memory-access unit brings
   // whole activation tiles into shared memory; a_tma = 0: A goes through registers
   int a_tma;
@@ -385,7 +386,8 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE, TMA>::THREADS, 1) gemm_tf32
 #pragma unroll
       for (int q = 0; q < BM * 8 / GROUP; ++q) {
         const int gr = m0 + ((t + q * GROUP) >> 3);
-        tab_row[q] = gr < M ? g.a_idx[gr] : -1;
+        const int ti = gr < M ? g.a_idx[gr] : -1;
+        tab_row[q] = ti < g.a_tab_rows ? ti : -1;   // an index beyond the table reads as a zero row
       }
       trp = tab_row;
     }
@@ -749,11 +751,10 @@ __global__ void __launch_bounds__(256) prep_weights_kernel(const WeightSite* __r
 template <int BN_T, bool PRECISE, bool FAST, int TMA>
 int launch_tc(tgnn_ctx* ctx, const TcArgs& a, int n_tiles, const char* name, cudaStream_t s) {
   using C_ = Cfg<BN_T, PRECISE, TMA>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(gemm_tf32_kernel<BN_T, PRECISE, FAST, TMA>,
-                                           cudaFuncAttributeMaxDynamicSharedMemorySize, C_::SMEM));
-    attr_set = true;
+  static SmemLimit smem_limit;   // one per template instance
+  {
+    const int rc = raise_smem_limit(ctx, gemm_tf32_kernel<BN_T, PRECISE, FAST, TMA>, C_::SMEM, smem_limit);
+    if (rc) return rc;
   }
   dim3 grid(n_tiles, (a.M + BM - 1) / BM, a.split_k);
   {
@@ -835,6 +836,7 @@ int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStr
   a.status = ctx->ws.status;
   if (g.a_idx && a.a_major == MAJOR_K && g.a_tab_cols % 4 == 0 && (((uintptr_t)g.a_tab & 15) == 0)) {
     a.a_idx = g.a_idx; a.a_tab = g.a_tab; a.a_tab_cols = g.a_tab_cols;
+    a.a_tab_rows = g.a_tab_rows > 0 ? g.a_tab_rows : ((int64_t)1 << 62);
   } else if (g.a_idx) {
     return 1;
   }

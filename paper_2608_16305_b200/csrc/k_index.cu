@@ -2,6 +2,7 @@
 // (step 1), per-node latest-event reduction (step 3).  All results are unique,
 // so they are bit-exact whatever the thread interleaving.
 #include "tgnn_internal.cuh"
+#include "tgnn_device.cuh"
 
 namespace tgnn {
 namespace {
@@ -33,23 +34,25 @@ constexpr int FIRST_VISIT = 0x40000000;
 // Single CTA: the batch has a few thousand events and the histogram lives in L2.
 __global__ void __launch_bounds__(1024) prune_mask_kernel(const int32_t* __restrict__ src, const int32_t* __restrict__ dst,
                                                           const int32_t* __restrict__ eid,
-                                                          const uint8_t* __restrict__ is_aux, int n, int32_t* hist,
-                                                          int force_heavy, uint32_t drop_q32, uint64_t seed,
+                                                          const uint8_t* __restrict__ is_aux, int n, int N,
+                                                          int32_t* status, int32_t* hist, int force_heavy, uint32_t drop_q32, uint64_t seed,
                                                           int64_t batch_idx, uint8_t* __restrict__ keep_out,
                                                           int32_t* __restrict__ heavy_out) {
   __shared__ int s_max, s_touched, s_heavy;
   if (threadIdx.x == 0) { s_max = 0; s_touched = 0; }
   const int n_round = (n + 31) / 32 * 32;
   for (int i = threadIdx.x; i < n_round; i += blockDim.x) {
-    const bool v = i < n;
-    hist_add(hist, v ? src[i] : 0, v);
-    hist_add(hist, v ? dst[i] : 0, v);
+    // an endpoint outside [0, N) is reported and left out of the counts
+    const int a = i < n ? src[i] : 0, b = i < n ? dst[i] : 0;
+    hist_add(hist, a, i < n && index_ok(a, N, status));
+    hist_add(hist, b, i < n && index_ok(b, N, status));
   }
   __syncthreads();
   // max count and number of touched nodes: the first visitor of a node counts it
   int lmax = 0, ltouched = 0;
   for (int i = threadIdx.x; i < 2 * n; i += blockDim.x) {
     const int node = (i & 1) ? dst[i >> 1] : src[i >> 1];
+    if (node < 0 || node >= N) continue;
     const int old = atomicOr(&hist[node], FIRST_VISIT);
     lmax = max(lmax, old & (FIRST_VISIT - 1));
     ltouched += (old & FIRST_VISIT) ? 0 : 1;
@@ -72,8 +75,8 @@ __global__ void __launch_bounds__(1024) prune_mask_kernel(const int32_t* __restr
     bool keep = true;
     if (is_aux[i] && heavy) keep = !(drop_q32 == 0xFFFFFFFFu || hash32(seed, batch_idx, eid[i]) < drop_q32);
     keep_out[i] = keep ? 1 : 0;
-    hist[src[i]] = 0;  // leave the histogram clean for the next call
-    hist[dst[i]] = 0;
+    if (src[i] >= 0 && src[i] < N) hist[src[i]] = 0;  // leave the histogram clean for the next call
+    if (dst[i] >= 0 && dst[i] < N) hist[dst[i]] = 0;
   }
 }
 
@@ -87,13 +90,22 @@ __global__ void __launch_bounds__(256) sample_recent_kernel(const int64_t* __res
                                                             const int32_t* __restrict__ g_eid,
                                                             const double* __restrict__ g_ts,
                                                             const int32_t* __restrict__ nodes,
-                                                            const double* __restrict__ times, int n, int k,
-                                                            int32_t* __restrict__ nbr_out, int32_t* __restrict__ eid_out,
-                                                            double* __restrict__ ts_out, int32_t* __restrict__ cnt_out) {
+                                                            const double* __restrict__ times, int n, int k, int N,
+                                                            int32_t* status, int32_t* __restrict__ nbr_out,
+                                                            int32_t* __restrict__ eid_out, double* __restrict__ ts_out,
+                                                            int32_t* __restrict__ cnt_out) {
   const int lane = threadIdx.x & 31;
   const int root = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
   if (root >= n) return;
   const int node = nodes[root];
+  if (!index_ok(node, N, lane == 0 ? status : nullptr)) {   // a root outside the graph: reported, no neighbors
+    if (lane == 0) cnt_out[root] = 0;
+    if (lane < k) {
+      const int64_t o = (int64_t)root * k + lane;
+      nbr_out[o] = -1; eid_out[o] = -1; ts_out[o] = 0.0;
+    }
+    return;
+  }
   const double t = times[root];
   const int64_t base = indptr[node];
   int64_t lo = base, hi = indptr[node + 1];  // the answer p lies in [lo, hi]
@@ -228,11 +240,21 @@ __device__ __forceinline__ unsigned long long peer_max(unsigned peers, unsigned 
 // Then the touched nodes are compacted in ascending id order by a block scan.
 // msg_node may be null: the node of message j is then read from the event arrays (src for role 0,
 // dst for role 1, none if keep[j>>1] == 0), which saves materialising it.
+// An event that names a node outside [0, N) (or, when E > 0, a feature row outside [0, E)) is reported and sends
+// no message at all, exactly as if its keep flag were 0.
 __device__ __forceinline__ int message_node(const int32_t* __restrict__ msg_node, const int32_t* __restrict__ src,
-                                            const int32_t* __restrict__ dst, const uint8_t* __restrict__ keep, int j) {
-  if (msg_node) return msg_node[j];
-  if (keep && !keep[j >> 1]) return -1;
-  return (j & 1) ? dst[j >> 1] : src[j >> 1];
+                                            const int32_t* __restrict__ dst, const uint8_t* __restrict__ keep,
+                                            const int32_t* __restrict__ eid, int j, int N, int64_t E, int32_t* status) {
+  if (msg_node) {
+    const int node = msg_node[j];
+    if (node < 0) return -1;
+    return index_ok(node, N, status) ? node : -1;
+  }
+  const int i = j >> 1;
+  if (keep && !keep[i]) return -1;
+  const int a = src[i], b = dst[i];
+  if (!(index_ok(a, N, status) & index_ok(b, N, status) & (E <= 0 || index_ok(eid[i], E, status)))) return -1;
+  return (j & 1) ? b : a;
 }
 
 __global__ void __launch_bounds__(1024) reduce_latest_kernel(const int32_t* __restrict__ msg_node,
@@ -245,7 +267,8 @@ __global__ void __launch_bounds__(1024) reduce_latest_kernel(const int32_t* __re
                                                              int32_t* win_msg, int32_t* node2slot, int32_t* prev_uniq,
                                                              int32_t* prev_n_uniq, int32_t* __restrict__ uniq_out,
                                                              int32_t* __restrict__ winner_out,
-                                                             int32_t* __restrict__ n_uniq_out, int smem_nodes) {
+                                                             int32_t* __restrict__ n_uniq_out, int smem_nodes,
+                                                             int32_t* status, int64_t E) {
   extern __shared__ int s_last[];  // [smem_nodes]: last message index per node (fast path)
   __shared__ int s_warp[32];
   __shared__ int s_total;
@@ -266,7 +289,7 @@ __global__ void __launch_bounds__(1024) reduce_latest_kernel(const int32_t* __re
       __syncthreads();
       const int n_round = (n_msg + 31) / 32 * 32;
       for (int j = tid; j < n_round; j += blockDim.x) {
-        const int node = j < n_msg ? message_node(msg_node, ev_src, ev_dst, ev_keep, j) : -1;
+        const int node = j < n_msg ? message_node(msg_node, ev_src, ev_dst, ev_keep, eid, j, N, E, status) : -1;
         const bool v = node >= 0;
         const unsigned act = __ballot_sync(FULL, v);
         if (v) {
@@ -314,7 +337,7 @@ __global__ void __launch_bounds__(1024) reduce_latest_kernel(const int32_t* __re
   }
   const int n_round = (n_msg + 31) / 32 * 32;
   for (int j = tid; j < n_round; j += blockDim.x) {
-    const int node = j < n_msg ? message_node(msg_node, ev_src, ev_dst, ev_keep, j) : -1;
+    const int node = j < n_msg ? message_node(msg_node, ev_src, ev_dst, ev_keep, eid, j, N, E, status) : -1;
     const bool v = node >= 0;
     const unsigned act = __ballot_sync(FULL, v);
     if (v) {
@@ -325,7 +348,7 @@ __global__ void __launch_bounds__(1024) reduce_latest_kernel(const int32_t* __re
   }
   __syncthreads();
   for (int j = tid; j < n_round; j += blockDim.x) {
-    const int node = j < n_msg ? message_node(msg_node, ev_src, ev_dst, ev_keep, j) : -1;
+    const int node = j < n_msg ? message_node(msg_node, ev_src, ev_dst, ev_keep, eid, j, N, E, status) : -1;
     const bool v = node >= 0 && orderable(t[j >> 1]) == best_t[node];
     const unsigned act = __ballot_sync(FULL, v);
     if (v) {
@@ -337,7 +360,7 @@ __global__ void __launch_bounds__(1024) reduce_latest_kernel(const int32_t* __re
   }
   __syncthreads();
   for (int j = tid; j < n_msg; j += blockDim.x) {
-    const int node = message_node(msg_node, ev_src, ev_dst, ev_keep, j);
+    const int node = message_node(msg_node, ev_src, ev_dst, ev_keep, eid, j, N, E, status);
     if (node < 0) continue;
     const unsigned long long key = (((unsigned long long)(uint32_t)eid[j >> 1]) << 1 | (unsigned)(j & 1)) + 1ULL;
     if (orderable(t[j >> 1]) == best_t[node] && key == best_id[node]) win_msg[node] = j;
@@ -388,7 +411,7 @@ int launch_prune_mask(tgnn_ctx* ctx, const int32_t* src, const int32_t* dst, con
                       int32_t* heavy_out, cudaStream_t s) {
   {
     KernelScope scope__(ctx, "prune_mask", s);
-    prune_mask_kernel<<<1, 1024, 0, s>>>(src, dst, eid, is_aux, n, ctx->ws.hist, force_heavy, drop_q32, seed, batch_idx,
+    prune_mask_kernel<<<1, 1024, 0, s>>>(src, dst, eid, is_aux, n, (int)ctx->cfg.num_nodes, ctx->ws.status, ctx->ws.hist, force_heavy, drop_q32, seed, batch_idx,
                                          keep_out, heavy_out);
   }
   TGNN_LAUNCH_OK(ctx, "prune_mask");
@@ -402,7 +425,8 @@ int launch_sample_recent(tgnn_ctx* ctx, const int32_t* nodes, const double* time
   {
     KernelScope scope__(ctx, "sample_recent", s);
     sample_recent_kernel<<<(n + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, s>>>(
-        ctx->indptr, ctx->g_nbr, ctx->g_eid, ctx->g_ts, nodes, times, n, ctx->cfg.k, nbr_out, eid_out, ts_out, cnt_out);
+        ctx->indptr, ctx->g_nbr, ctx->g_eid, ctx->g_ts, nodes, times, n, ctx->cfg.k, (int)ctx->cfg.num_nodes, ctx->ws.status,
+        nbr_out, eid_out, ts_out, cnt_out);
   }
   TGNN_LAUNCH_OK(ctx, "sample_recent");
   return TGNN_OK;
@@ -465,17 +489,18 @@ int launch_reduce_latest_events(tgnn_ctx* ctx, const int32_t* msg_node, const in
   // shared-memory table of the fast path: 4 bytes per node, when it fits
   const int N = (int)ctx->cfg.num_nodes;
   const int smem_nodes = (size_t)N * 4 <= 200 * 1024 ? N : 0;
-  static int attr_bytes = 0;
-  if (smem_nodes * 4 > attr_bytes) {
-    TGNN_CUDA_OK(ctx, cudaFuncSetAttribute(reduce_latest_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_nodes * 4));
-    attr_bytes = smem_nodes * 4;
+  static SmemLimit smem_limit;
+  if (smem_nodes * 4 > 48 * 1024) {
+    const int rc = raise_smem_limit(ctx, reduce_latest_kernel, smem_nodes * 4, smem_limit);
+    if (rc) return rc;
   }
   {
     KernelScope scope__(ctx, "reduce_latest", s);
     reduce_latest_kernel<<<1, 1024, (size_t)smem_nodes * 4, s>>>(msg_node, src, dst, keep, t, eid, n_msg, N, w.best_t,
                                                                  w.best_id, w.win_msg, w.node2slot, w.prev_uniq,
                                                                  w.prev_n_uniq, uniq_out, winner_out, n_uniq_out,
-                                                                 smem_nodes);
+                                                                 smem_nodes, w.status,
+                                                                 ctx->cfg.d_e > 0 && src != nullptr ? ctx->num_events : 0);
   }
   TGNN_LAUNCH_OK(ctx, "reduce_latest");
   return TGNN_OK;

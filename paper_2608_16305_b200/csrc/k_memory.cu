@@ -32,16 +32,22 @@ __global__ void __launch_bounds__(256) build_messages_kernel(const float* __rest
                                                              const int32_t* __restrict__ src,
                                                              const int32_t* __restrict__ dst, const double* __restrict__ t,
                                                              const int32_t* __restrict__ eid,
-                                                             const uint8_t* __restrict__ keep, int n,
-                                                             float* __restrict__ msg_out, int32_t* __restrict__ msg_node_out) {
+                                                             const uint8_t* __restrict__ keep, int n, int64_t N, int64_t E,
+                                                             int32_t* status, float* __restrict__ msg_out,
+                                                             int32_t* __restrict__ msg_node_out) {
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   const int dm = 3 * d + de;
   for (int j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; j < 2 * n; j += warps) {
     const int i = j >> 1, role = j & 1;
-    const bool kept = keep == nullptr || keep[i] != 0;
+    bool kept = keep == nullptr || keep[i] != 0;
     const int self = role ? dst[i] : src[i];
     const int other = role ? src[i] : dst[i];
+    // an event naming a node or a feature row that does not exist is reported and sends no message
+    if (kept) {
+      int32_t* st = lane == 0 ? status : nullptr;
+      kept = index_ok(self, N, st) & index_ok(other, N, st) & (de == 0 || index_ok(eid[i], E, st));
+    }
     if (lane == 0) msg_node_out[j] = kept ? self : -1;
     if (msg_out == nullptr) continue;
     float* row = msg_out + (int64_t)j * dm;
@@ -64,21 +70,33 @@ __global__ void __launch_bounds__(256) gather_winner_kernel(const float* __restr
                                                             const double* __restrict__ t, const int32_t* __restrict__ eid,
                                                             const float* __restrict__ msg, const int32_t* __restrict__ uniq,
                                                             const int32_t* __restrict__ winner,
-                                                            const int32_t* __restrict__ n_uniq, int u_cap, int ld,
+                                                            const int32_t* __restrict__ n_uniq, int u_cap, int n_msg, int64_t N,
+                                                            int64_t E, int32_t* status, int ld,
                                                             float* __restrict__ X, float* __restrict__ x_dt,
                                                             float* __restrict__ Xsin, double* __restrict__ win_t) {
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
-  const int U = min(*n_uniq, u_cap);
+  if (blockIdx.x == 0 && threadIdx.x == 0) index_ok(*n_uniq, (long long)u_cap + 1, status);   // a count beyond the capacity
+  const int U = max(0, min(*n_uniq, u_cap));
   const int dm = 3 * d + de;
   for (int u = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < U; u += warps) {
-    const int j = winner[u], i = j >> 1, role = j & 1;
-    const int self = role ? dst[i] : src[i];
-    const int other = role ? src[i] : dst[i];
-    const double ti = t[i];
-    const float dtf = (float)(ti - last_update[self]);
     float* row = X + (int64_t)u * ld;
     float* sin_row = Xsin + (int64_t)u * d;
+    int32_t* st = lane == 0 ? status : nullptr;
+    const int j = winner[u];
+    bool good = index_ok(j, n_msg, st);
+    const int i = good ? j >> 1 : 0, role = j & 1;
+    const int self = good ? (role ? dst[i] : src[i]) : 0;
+    const int other = good ? (role ? src[i] : dst[i]) : 0;
+    good = good && index_ok(self, N, st) && index_ok(other, N, st) && (de == 0 || msg != nullptr || index_ok(eid[i], E, st));
+    if (!good) {   // reported; the row is zero and the node's update starts from a zero message
+      for (int q = lane; q < ld; q += 32) row[q] = 0.f;
+      for (int q = lane; q < d; q += 32) sin_row[q] = 0.f;
+      if (lane == 0) { x_dt[u] = 0.f; win_t[u] = 0.0; }
+      continue;
+    }
+    const double ti = t[i];
+    const float dtf = (float)(ti - last_update[self]);
     if (msg != nullptr) {
       warp_copy_f32(row, msg + (int64_t)j * dm, dm, lane);
       for (int q = lane; q < d; q += 32) sin_row[q] = sinf(time_arg(time_w[q], time_b[q], dtf));
@@ -97,8 +115,9 @@ __global__ void __launch_bounds__(256) gru_gate_kernel(const float* __restrict__
                                                        const int32_t* __restrict__ n_uniq, int u_cap,
                                                        float* __restrict__ g_r, float* __restrict__ g_z,
                                                        float* __restrict__ g_n, float* __restrict__ g_hn,
-                                                       float* __restrict__ memory, double* __restrict__ last_update) {
-  const int U = min(*n_uniq, u_cap);
+                                                       float* __restrict__ memory, double* __restrict__ last_update,
+                                                       int64_t N, int32_t* status) {
+  const int U = max(0, min(*n_uniq, u_cap));
   const int64_t total = (int64_t)U * d;
   for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
     const int u = (int)(e / d), q = (int)(e % d);
@@ -112,6 +131,7 @@ __global__ void __launch_bounds__(256) gru_gate_kernel(const float* __restrict__
     const float hnew = fmaf(z, h - nn, nn);  // (1 - z) n + z h
     g_r[e] = r; g_z[e] = z; g_n[e] = nn; g_hn[e] = hn;
     const int node = uniq[u];
+    if (!index_ok(node, N, q == 0 ? status : nullptr)) continue;   // reported, nothing written
     memory[(int64_t)node * d + q] = hnew;
     if (q == 0) last_update[node] = win_t[u];
   }
@@ -123,14 +143,15 @@ __global__ void __launch_bounds__(256) rnn_gate_kernel(const float* __restrict__
                                                        const int32_t* __restrict__ uniq, const double* __restrict__ win_t,
                                                        const int32_t* __restrict__ n_uniq, int u_cap,
                                                        float* __restrict__ g_n, float* __restrict__ memory,
-                                                       double* __restrict__ last_update) {
-  const int U = min(*n_uniq, u_cap);
+                                                       double* __restrict__ last_update, int64_t N, int32_t* status) {
+  const int U = max(0, min(*n_uniq, u_cap));
   const int64_t total = (int64_t)U * d;
   for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
     const int u = (int)(e / d), q = (int)(e % d);
     const float hnew = tanhf(Gi[e] + Gh[e]);
     g_n[e] = hnew;
     const int node = uniq[u];
+    if (!index_ok(node, N, q == 0 ? status : nullptr)) continue;
     memory[(int64_t)node * d + q] = hnew;
     if (q == 0) last_update[node] = win_t[u];
   }
@@ -148,7 +169,8 @@ int launch_build_messages(tgnn_ctx* ctx, const int32_t* src, const int32_t* dst,
     KernelScope scope__(ctx, "build_messages", s);
     build_messages_kernel<<<blocks, 256, 0, s>>>(ctx->memory, ctx->last_update, ctx->efeat, c.feat_dtype == TGNN_BF16,
                                                  ctx->params + ctx->L.time_w, ctx->params + ctx->L.time_b, c.d, c.d_e, src,
-                                                 dst, t, eid, keep, n, msg_out, msg_node_out);
+                                                 dst, t, eid, keep, n, c.num_nodes, ctx->num_events, ctx->ws.status, msg_out,
+                                                 msg_node_out);
   }
   TGNN_LAUNCH_OK(ctx, "build_messages");
   return TGNN_OK;
@@ -167,8 +189,8 @@ int launch_memory_update(tgnn_ctx* ctx, const float* msg, const int32_t* uniq, c
     gather_winner_kernel<<<(U_cap + 7) / 8, 256, 0, s>>>(ctx->memory, ctx->last_update, ctx->efeat,
                                                          c.feat_dtype == TGNN_BF16, ctx->params + L.time_w,
                                                          ctx->params + L.time_b, d, c.d_e, ctx->m_src, ctx->m_dst, ctx->m_t,
-                                                         ctx->m_eid, msg, uniq, winner, n_uniq, U_cap, ctx->ld_msg, w.X,
-                                                         w.x_dt, w.Xsin, w.win_t);
+                                                         ctx->m_eid, msg, uniq, winner, n_uniq, U_cap, 2 * ctx->m_n, c.num_nodes,
+                                                         ctx->num_events, w.status, ctx->ld_msg, w.X, w.x_dt, w.Xsin, w.win_t);
   }
   TGNN_LAUNCH_OK(ctx, "gather_winner");
   GemmArgs g = {};
@@ -194,7 +216,7 @@ int launch_memory_update(tgnn_ctx* ctx, const float* msg, const int32_t* uniq, c
     {
       KernelScope scope__(ctx, "rnn_gate", s);
       rnn_gate_kernel<<<(int)((total + 255) / 256), 256, 0, s>>>(w.Gi, w.Gh, d, uniq, w.win_t, n_uniq, U_cap, w.g_n,
-                                                                 ctx->memory, ctx->last_update);
+                                                                 ctx->memory, ctx->last_update, c.num_nodes, w.status);
     }
     TGNN_LAUNCH_OK(ctx, "rnn_gate");
     return TGNN_OK;
@@ -203,7 +225,7 @@ int launch_memory_update(tgnn_ctx* ctx, const float* msg, const int32_t* uniq, c
     KernelScope scope__(ctx, "gru_gate", s);
     gru_gate_kernel<<<(int)((total + 255) / 256), 256, 0, s>>>(w.Gi, w.Gh, w.X, ctx->ld_msg, d, uniq, w.win_t, n_uniq,
                                                                U_cap, w.g_r, w.g_z, w.g_n, w.g_hn, ctx->memory,
-                                                               ctx->last_update);
+                                                               ctx->last_update, c.num_nodes, w.status);
   }
   TGNN_LAUNCH_OK(ctx, "gru_gate");
   return TGNN_OK;

@@ -1,4 +1,5 @@
 // C ABI: context life cycle, argument checks, and the sequencing of one training step.
+#include <cmath>
 #include <cstdarg>
 #include <cstdio>
 #include <cstdlib>
@@ -63,7 +64,7 @@ int check_config(const tgnn_config* c) {
   if (c->feat_dtype != TGNN_F32 && c->feat_dtype != TGNN_BF16) return TGNN_EINVAL;
   if (c->max_events < 1 || c->max_roots < 3 || c->max_events > (1 << 24) || c->max_roots > (1 << 24)) return TGNN_EINVAL;
   if (c->math_mode != TGNN_MATH_FP32 && c->math_mode != TGNN_MATH_TF32 && c->math_mode != TGNN_MATH_TF32_FAST &&
-      c->math_mode != TGNN_MATH_BF16X3) return TGNN_EINVAL;
+      c->math_mode != TGNN_MATH_F16X3) return TGNN_EINVAL;
   if (c->model != TGNN_MODEL_TGN && c->model != TGNN_MODEL_JODIE) return TGNN_EINVAL;
   if (c->embed_aux != 0 && c->embed_aux != 1) return TGNN_EINVAL;
   if (!(c->lr >= 0.f) || !(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f) || !(c->eps > 0.f))
@@ -265,13 +266,15 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
          cudaMemcpy(ctx->sites_dev, ctx->sites, sizeof(ctx->sites), cudaMemcpyHostToDevice) == cudaSuccess;
   }
   ctx->split_buf = nullptr;
-  if (ok && cfg->math_mode == TGNN_MATH_BF16X3 && cfg->model == TGNN_MODEL_TGN) {
+  if (ok && cfg->math_mode == TGNN_MATH_F16X3 && cfg->model == TGNN_MODEL_TGN) {
     const auto up8 = [](int64_t x) { return (x + 7) / 8 * 8; };
     const int64_t d = cfg->d, dkv = ctx->L.dkv, NB = ctx->NB_cap;
-    ctx->zs = SplitMat{nullptr, up8(dkv + 1), 0, NB, dkv + 1};
-    ctx->dkvs = SplitMat{nullptr, up8(2 * d), 0, NB, 2 * d};
-    ctx->wkv_s = SplitMat{nullptr, up8(dkv), 0, 2 * d, dkv};
-    ctx->wz_s = SplitMat{nullptr, up8(2 * d), 0, 2 * d, 2 * d};
+    // every operand as two fp16 numbers (22 mantissa bits); the gradient rows, whose entries are far below fp16's
+    // normal range, multiplied by 2^12 first (the products divide it out again)
+    ctx->zs = SplitMat{nullptr, up8(dkv + 1), 0, NB, dkv + 1, 1, 1.f};
+    ctx->dkvs = SplitMat{nullptr, up8(2 * d), 0, NB, 2 * d, 1, 4096.f};
+    ctx->wkv_s = SplitMat{nullptr, up8(dkv), 0, 2 * d, dkv, 1, 1.f};
+    ctx->wz_s = SplitMat{nullptr, up8(2 * d), 0, 2 * d, 2 * d, 1, 1.f};
     SplitMat* ms[4] = {&ctx->zs, &ctx->dkvs, &ctx->wkv_s, &ctx->wz_s};
     size_t off = 0;
     for (SplitMat* m : ms) {
@@ -806,7 +809,10 @@ int tgnn_debug_gemm_split(tgnn_ctx* ctx, const float* A, int64_t a_rs, int64_t a
   else if (a_rs == 1 && b_cs == 1) { mn = 1; lda = a_cs; ldb = b_rs; a_rows = K; a_cols = M; b_rows = K; b_cols = N; }
   else return set_error(ctx, TGNN_ESHAPE, "debug_gemm_split: operands must both have the contraction index contiguous, or both the other one");
   const auto up8 = [](int64_t x) { return (x + 7) / 8 * 8; };
-  SplitMat a{nullptr, up8(a_cols), 0, a_rows, a_cols}, b{nullptr, up8(b_cols), 0, b_rows, b_cols};
+  // TGNN_GEMM_BF16=1 (debugging aid): bf16 planes instead of fp16 planes; TGNN_GEMM_SCALE=s: A is scaled by 2^s
+  const int f16 = getenv("TGNN_GEMM_BF16") && atoi(getenv("TGNN_GEMM_BF16")) ? 0 : 1;
+  const float sc = getenv("TGNN_GEMM_SCALE") ? ldexpf(1.f, atoi(getenv("TGNN_GEMM_SCALE"))) : 1.f;
+  SplitMat a{nullptr, up8(a_cols), 0, a_rows, a_cols, f16, sc}, b{nullptr, up8(b_cols), 0, b_rows, b_cols, f16, 1.f};
   a.plane_stride = a.rows * a.ld;
   b.plane_stride = b.rows * b.ld;
   const int64_t a_bytes = (2 * a.plane_stride * 2 + 255) / 256 * 256, b_bytes = 2 * b.plane_stride * 2;
@@ -825,7 +831,8 @@ int tgnn_debug_gemm_split(tgnn_ctx* ctx, const float* A, int64_t a_rs, int64_t a
   if (trace_on && scratch_bytes >= a_bytes + b_bytes + 256 + 4096 + 256)
     trace = reinterpret_cast<long long*>((char*)scratch + ((a_bytes + b_bytes + 256 + 255) / 256 * 256));
   return launch_gemm_split(ctx, a, b, mn, C, ldc, M, N, K, bias, relu, accumulate, split_k < 1 ? 1 : split_k, "debug_gemm_split",
-                           S(stream), debug_withhold, spin_limit, -1, nullptr, trace);
+                           S(stream), debug_withhold, spin_limit, -1, nullptr, trace,
+                           getenv("TGNN_GEMM_SINGLE") ? atoi(getenv("TGNN_GEMM_SINGLE")) : -1);
 }
 
 int tgnn_status(tgnn_ctx* ctx, int32_t* status_host, void* stream) {

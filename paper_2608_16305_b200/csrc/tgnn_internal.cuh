@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
 #include <vector>
 
 #include "../../include/tgnn.h"
@@ -118,12 +119,16 @@ struct WeightSite {
   int64_t chunks;            // 16-byte chunks the preparation kernel writes for this site
 };
 
-// An fp32 matrix stored as two bf16 planes of the same row-major shape: hi = bf16(x) at `hi`, lo = bf16(x - hi)
-// at hi + plane_stride (in bf16 elements).  ld and plane_stride are multiples of 8, `hi` is 16-byte aligned.
+// An fp32 matrix stored as two 16-bit planes of the same row-major shape: hi = r16(scale * x) at `hi`,
+// lo = r16(scale * x - hi) at hi + plane_stride (in elements), r16 rounding to fp16 (fp16 = 1: 22 mantissa bits
+// together, values must stay inside fp16's range, hence the power-of-two `scale` for gradients) or to bf16
+// (fp16 = 0: 16 bits, any range).  ld and plane_stride are multiples of 8, `hi` is 16-byte aligned.
 struct SplitMat {
   void* hi;
   int64_t ld, plane_stride;
   int64_t rows, cols;
+  int fp16;
+  float scale;
 };
 
 }  // namespace tgnn
@@ -179,11 +184,11 @@ struct tgnn_ctx {
   unsigned char* images;         // device buffer of all sites' images
   size_t images_bytes;
   bool images_fresh;             // images match the current parameters (set by the step, cleared by Adam)
-  // TGNN_MATH_BF16X3: the attention inputs Z (with a column of ones after the last input column), the gradient
-  // of the key/value rows and the key/value weights in their two roles, each as two bf16 planes
+  // TGNN_MATH_F16X3: the attention inputs Z (with a column of ones after the last input column), the gradient
+  // of the key/value rows and the key/value weights in their two roles, each as two fp16 planes
   void* split_buf;
   tgnn::SplitMat zs, dkvs, wkv_s, wz_s;
-  bool z_split;       // the attention inputs of the current step are (being) written as bf16 planes
+  bool z_split;       // the attention inputs of the current step are (being) written as fp16 planes
   bool z_static_done; // tgnn_train_step already gathered the memory-independent part of the attention inputs
   bool grads_zeroed;  // tgnn_train_step cleared the gradient block ahead of the backward pass
   tgnn::Workspace ws;
@@ -213,6 +218,7 @@ struct tgnn_ctx {
   int defer_adam;
   bool grad_pending;
   int64_t launches;
+  int64_t fma_fallbacks;   // products that a tensor-core mode had to run on the fp32 FMA tiles
   tgnn::Profiler prof;
   char err[256];
 };
@@ -231,6 +237,25 @@ int set_error(tgnn_ctx* ctx, int code, const char* fmt, ...);
     cudaError_t e__ = cudaGetLastError();                                                    \
     if (e__ != cudaSuccess) return tgnn::set_error(ctx, TGNN_ECUDA, "launch %s: %s", name, cudaGetErrorString(e__)); \
   } while (0)
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize is a setting per device (and the library may serve several devices
+// from several threads of one process): each kernel keeps one of these to remember what it has raised where.
+struct SmemLimit {
+  int bytes[64] = {};
+  std::mutex lock;
+};
+template <typename F>
+inline int raise_smem_limit(tgnn_ctx* ctx, F kernel, int bytes, SmemLimit& st) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
+    return set_error(ctx, TGNN_ECUDA, "cudaGetDevice failed or device index above 63");
+  std::lock_guard<std::mutex> g(st.lock);
+  if (st.bytes[dev] >= bytes) return TGNN_OK;
+  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return set_error(ctx, TGNN_ECUDA, "cudaFuncSetAttribute(%d bytes): %s", bytes, cudaGetErrorString(e));
+  st.bytes[dev] = bytes;
+  return TGNN_OK;
+}
 
 // side[i] waits for everything enqueued so far on `from`.
 inline int fork_to(tgnn_ctx* ctx, cudaStream_t from, cudaStream_t to) {
@@ -331,6 +356,7 @@ struct GemmArgs {
   const int32_t* a_idx;   // optional (tensor-core path, K-major A): leading a_tab_cols columns of row m come from
   const float* a_tab;     //   a_tab[a_idx[m] * a_tab_cols + k] (zero row if a_idx[m] < 0) instead of A
   int a_tab_cols;
+  int64_t a_tab_rows;     //   rows of a_tab: an index at or beyond it reads as a zero row
   int site;               // WeightSiteId + 1 when B is that weight matrix (0: none); lets the kernel use its image
   int precise;            // tensor-core mode only: 3xTF32 head/tail split, close to fp32 accuracy
   int tail_slack;         // both operands live in the workspace arena: a tiled load may read up to 124 bytes past
@@ -338,13 +364,14 @@ struct GemmArgs {
 };
 int launch_gemm(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s);
 int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStream_t s);  // k_gemm_tc.cu
-// ---- split-bf16 projections (k_gemm_bf.cu) ----
+// ---- split-operand projections (k_gemm_split.cu) ----
 int launch_prep_split_weights(tgnn_ctx* ctx, cudaStream_t s);
 int launch_split_rows(tgnn_ctx* ctx, const float* X, int64_t ld_in, int64_t rows, int cols, const int32_t* dev_rows,
-                      const SplitMat& out, int ones_col, const char* name, cudaStream_t s);
+                      const SplitMat& out, int ones_col, const char* name, cudaStream_t s);   // honours out.fp16, out.scale
 int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int mn_major, float* C, int64_t ldc, int M, int N,
                       int K, const float* bias, int relu, int accumulate, int split_k, const char* name, cudaStream_t s,
-                      int debug_withhold = 0, unsigned spin_limit = 0, int extra_col = -1, float* extra_out = nullptr, long long* trace = nullptr);
+                      int debug_withhold = 0, unsigned spin_limit = 0, int extra_col = -1, float* extra_out = nullptr, long long* trace = nullptr,
+                      int single = -1);
 size_t plan_weight_sites(tgnn_ctx* ctx);                       // fills ctx->sites, returns the image bytes needed
 int launch_prep_weights(tgnn_ctx* ctx, cudaStream_t s);        // writes all images from the current parameters
 

@@ -1,7 +1,8 @@
-"""The split-bf16 projection kernel (two bf16 planes per fp32 operand, three tensor-core passes, fp32
+"""The split-operand projection kernel (two 16-bit planes per fp32 operand, three tensor-core passes, fp32
 accumulation) against the plain definition C = A B (+ bias, ReLU, accumulate) computed in fp64 by numpy.
-Two bf16 terms carry 16 mantissa bits, so the result must sit within 1e-4 of the largest |C| (a single
-bf16 pass would be off by 4e-3, one TF32 pass by 1e-3).  Also: a bounded wait that is made to run out."""
+Two fp16 terms carry 22 mantissa bits (two bf16 terms 16), so the result must sit within 1e-4 of the largest
+|C| whichever planes are used (a single bf16 pass would be off by 4e-3, one TF32 pass by 1e-3).  Also: a
+bounded wait that is made to run out."""
 import numpy as np
 import pytest
 import torch
@@ -79,6 +80,39 @@ def test_split_projection_matches_definition(lib, shape):
     err = np.abs(got[:, :N] - (C0[:, :N] + ref)).max() / scale
     assert err <= 1e-4, f"accumulate mode err {err}"
     assert np.array_equal(got[:, N:], C0[:, N:])                    # the padding columns are not touched
+
+
+@pytest.mark.parametrize("shape", [(1800, 200, 372, "k"), (200, 387, 5000, "mn")])
+def test_fp16_planes_beat_bf16_planes_and_scaling_keeps_gradients_in_range(lib, shape, monkeypatch):
+    """The library holds its operands as two fp16 numbers (22 mantissa bits); the kernel also takes bf16 planes
+    (16 bits, any range).  fp16 planes must be the more accurate of the two.  Gradient-sized entries (1e-6) lie
+    below fp16's normal range: scaled by 2^12 on the way in (and back in the epilogue) they keep full accuracy."""
+    M, N, K, lay = shape
+    rng = np.random.default_rng(77)
+    A, Bm, A_dev, sa, B_dev, sb = _operands(rng, M, N, K, lay)
+    ref = A.astype(np.float64) @ Bm.astype(np.float64)
+    scr = _scratch(M, N, K)
+    errs = {}
+    for bf in ("0", "1"):
+        monkeypatch.setenv("TGNN_GEMM_BF16", bf)
+        C = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+        lib.debug_gemm_split(A_dev, *sa, B_dev, *sb, C, N, M, N, K, scr)
+        torch.cuda.synchronize()
+        assert lib.status() == 0
+        errs[bf] = np.abs(C.cpu().numpy() - ref).max() / np.abs(ref).max()
+    # (over a contraction of thousands of terms the fp32 accumulator's own rounding, ~2e-5, hides the difference)
+    assert errs["0"] <= 3e-5 and errs["1"] <= 1e-4 and (K > 1000 or errs["0"] < 0.5 * errs["1"]), errs
+    monkeypatch.setenv("TGNN_GEMM_BF16", "0")
+    small = (A_dev * 1e-6).contiguous()
+    for shift, bound in (("0", None), ("12", 5e-6)):
+        monkeypatch.setenv("TGNN_GEMM_SCALE", shift)
+        C = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+        lib.debug_gemm_split(small, *sa, B_dev, *sb, C, N, M, N, K, scr)
+        torch.cuda.synchronize()
+        errs[shift] = np.abs(C.cpu().numpy() - 1e-6 * ref).max() / np.abs(1e-6 * ref).max()
+        if bound:
+            assert errs[shift] <= (3e-5 if K > 1000 else bound), errs
+    assert errs["12"] < errs["0"], errs          # unscaled, the small entries lose their remainder plane
 
 
 def test_every_tile_lands_where_the_definition_puts_it(lib):

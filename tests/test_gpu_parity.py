@@ -21,11 +21,11 @@ from paper_2608_16305_b200 import workload as wl
 
 pytestmark = pytest.mark.gpu
 
-TOL = {"fp32": 1e-4, "tf32": 2e-3, "tf32_bf16": 1e-2, "tf32fast": 2e-3, "tf32fast_bf16": 1e-2, "bf16x3": 2e-3, "bf16x3_bf16": 1e-2}
+TOL = {"fp32": 1e-4, "tf32": 2e-3, "tf32_bf16": 1e-2, "tf32fast": 2e-3, "tf32fast_bf16": 1e-2, "f16x3": 2e-3, "f16x3_bf16": 1e-2}
 # ReLU's derivative jumps at zero.  A unit whose pre-activation is closer to zero than the kernel's
 # arithmetic resolves may land on either side; for such units (|pre| <= GATE_EPS * max|pre|, nowhere
 # else) the oracle differentiates the branch the kernel took.
-GATE_EPS = {"fp32": 1e-5, "tf32": 2e-4, "tf32fast": 3e-3, "bf16x3": 2e-4}
+GATE_EPS = {"fp32": 1e-5, "tf32": 2e-4, "tf32fast": 3e-3, "f16x3": 2e-4}
 # How many units per step may take the kernel's branch against the oracle's own fp64 sign: a handful, or
 # 2e-5 of the step's ReLU units on the big batches (measured: at most 3 units in any compared step of the
 # five workloads, 1.2 M to 2 M units per step on the batch-4000 ones).
@@ -81,7 +81,7 @@ class Rig:
         self.model = model
         self.weights = wl.make_weights(cfg.d, cfg.d_e, cfg.seed, bias_scale=bias_scale, model=model)
         mode = {"fp32": B.TGNN_MATH_FP32, "tf32": B.TGNN_MATH_TF32, "tf32fast": B.TGNN_MATH_TF32_FAST,
-                "bf16x3": B.TGNN_MATH_BF16X3}[math]
+                "f16x3": B.TGNN_MATH_F16X3}[math]
         self.tr = trainer.Trainer(self.dw, self.weights, math_mode=mode, lr=lr, model=model)
         f32 = lambda x: float(np.float32(x))      # the library's configuration holds fp32 hyper-parameters
         self.ocfg = orc_cfg(oracle, cfg, lr=f32(lr), beta1=f32(0.9), beta2=f32(0.999), eps=f32(1e-8))
@@ -521,7 +521,7 @@ def _run_epoch_checks(rig, steps, check_at):
             rig.check_step(b, pre, res, what=f"[{rig.cfg.name} batch {b}]")
 
 
-@pytest.mark.parametrize("math", ["fp32", "tf32", "bf16x3"])
+@pytest.mark.parametrize("math", ["fp32", "tf32", "f16x3"])
 def test_tiny_epoch_teacher_forced(B, oracle, math):
     rig = Rig(B, oracle, TINY, math=math)
     nb = TINY.num_batches
@@ -539,7 +539,7 @@ def _scaled(name, events, **kw):
     return wl.scaled(c, num_events=events, **kw)
 
 
-@pytest.mark.parametrize("math", ["fp32", "tf32", "bf16x3"])
+@pytest.mark.parametrize("math", ["fp32", "tf32", "f16x3"])
 @pytest.mark.parametrize("name,events,at", [
     ("wiki", 6000, {1, 5, 9}),          # 172-d features, d = 100: ragged tiles everywhere
     ("reddit", 9000, {2, 8, 14}),       # replay events + pruning
@@ -598,7 +598,7 @@ def test_head_paths_wide_and_ragged(B, oracle, math, d, batch):
     _run_epoch_checks(rig, range(4), {1, 3})
 
 
-@pytest.mark.parametrize("math", ["fp32", "tf32", "bf16x3"])
+@pytest.mark.parametrize("math", ["fp32", "tf32", "f16x3"])
 def test_bf16_feature_table(B, oracle, math):
     c = wl.scaled(wl.CONFIGS["large"], num_events=20000, num_nodes=3000, batch=1000)
     rig = Rig(B, oracle, c, math=math)
@@ -970,6 +970,74 @@ def test_argument_errors_are_reported_not_launched(B):
     lib.close()
 
 
+def test_indices_beyond_the_graph_are_reported_and_never_used(B, oracle):
+    """Every gather and scatter checks its indices.  An update event that names a node beyond the graph or a
+    feature row beyond the table is reported through the status word (TGNN_EBOUNDS) and treated exactly as if its
+    keep flag were 0: the step's result equals, bit for bit, that of a second context given the same batch with
+    those events masked out.  A root beyond the graph and a node count beyond the capacity are reported too, and
+    nothing outside the arrays involved is touched."""
+    cfg = _scaled("wiki", 6000)
+    a = Rig(B, oracle, cfg, math="fp32")
+    a.tr.lib.set_graph_replay(False)
+    for step in range(3):
+        a.tr.step(step)
+    torch.cuda.synchronize()
+    N, E = cfg.num_nodes, cfg.num_events
+    u = a.dw.mb_slice(2)
+    src, dst, t, eid = (x[u].clone() for x in (a.dw.mb_src, a.dw.mb_dst, a.dw.mb_t, a.dw.mb_eid))
+    keep = torch.ones(src.numel(), dtype=torch.uint8, device="cuda")
+    bad_src, bad_dst, bad_eid = src.clone(), dst.clone(), eid.clone()
+    bad_src[3] = N + 7
+    bad_dst[11] = 1 << 30
+    bad_eid[5] = E + 3
+    masked = keep.clone()
+    masked[[3, 5, 11]] = 0
+    q = a.dw.targets(3)
+    state = (a.tr.memory, a.tr.last_update, a.tr.params, a.tr.adam_m, a.tr.adam_v, a.tr.step_count)
+    saved = [x.clone() for x in state]
+    a.tr.lib.train_step(bad_src, bad_dst, t, bad_eid, keep, *q, None, a.tr.loss, a.tr.gradnorm)
+    torch.cuda.synchronize()
+    assert a.tr.lib.status() == B.TGNN_EBOUNDS
+    got = [x.clone() for x in state] + [a.tr.loss.clone()]
+    a.tr.lib.clear_status()
+    for x, y in zip(state, saved):
+        x.copy_(y)
+    a.tr.lib.train_step(src, dst, t, eid, masked, *q, None, a.tr.loss, a.tr.gradnorm)
+    torch.cuda.synchronize()
+    assert a.tr.lib.status() == 0
+    assert torch.equal(got[1], a.tr.last_update)                                  # the same nodes were updated
+    assert relerr(got[0].cpu().numpy(), a.tr.memory.cpu().numpy()) <= 1e-6        # (atomic summation order differs)
+    assert abs(float(got[6].item()) - float(a.tr.loss.item())) <= 1e-6 * abs(float(a.tr.loss.item()))
+    a.tr.lib.clear_status()
+    # a root beyond the graph: reported, the step completes with finite numbers
+    qs, qd, qn, qt = (x.clone() for x in a.dw.targets(4))
+    qd[7] = N
+    v = a.dw.mb_slice(3)
+    a.tr.lib.train_step(a.dw.mb_src[v], a.dw.mb_dst[v], a.dw.mb_t[v], a.dw.mb_eid[v], None, qs, qd, qn, qt, None, a.tr.loss,
+                        a.tr.gradnorm)
+    torch.cuda.synchronize()
+    assert a.tr.lib.status() == B.TGNN_EBOUNDS
+    assert bool(torch.isfinite(a.tr.loss).all()) and bool(torch.isfinite(a.tr.memory).all())
+    a.tr.lib.clear_status()
+    # a device-side node count beyond the capacity of the arrays it describes: clamped and reported
+    lib = a.tr.lib
+    n = 40
+    node = torch.zeros(2 * n, dtype=torch.int32, device="cuda")
+    lib.build_messages(src[:n], dst[:n], t[:n], eid[:n], None, None, node)
+    uniq = torch.zeros(2 * n, dtype=torch.int32, device="cuda")
+    win = torch.zeros(2 * n, dtype=torch.int32, device="cuda")
+    nu = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lib.reduce_latest(node, t[:n], eid[:n], uniq, win, nu)
+    before = a.tr.memory.clone()
+    nu.fill_(1_000_000)
+    lib.memory_update(None, uniq, win, nu)
+    torch.cuda.synchronize()
+    assert lib.status() == B.TGNN_EBOUNDS
+    touched = torch.zeros(N, dtype=torch.bool, device="cuda")
+    touched[uniq.long()] = True
+    assert torch.equal(a.tr.memory[~touched], before[~touched])
+
+
 # ------------------------------------------ full-size workloads, bench launch configuration
 # The same teacher-forced comparison at the full sizes of the named workloads, driven the way bench.py drives
 # it: tensor-core mode, the whole step replayed as a CUDA graph on a capturable stream.  The oracle
@@ -989,7 +1057,7 @@ def _full_size(B, oracle, cfg, check_at, last, math="tf32"):
 
 
 @pytest.mark.slow
-@pytest.mark.parametrize("math", ["tf32", "bf16x3"])
+@pytest.mark.parametrize("math", ["tf32", "f16x3"])
 def test_wiki_full_size_graph_replay(B, oracle, math):
     cfg = wl.CONFIGS["wiki"]
     rig = _full_size(B, oracle, cfg, {0, 1, 2, 150, cfg.num_batches - 1}, cfg.num_batches - 1, math=math)
@@ -999,7 +1067,7 @@ def test_wiki_full_size_graph_replay(B, oracle, math):
 
 
 @pytest.mark.slow
-@pytest.mark.parametrize("math", ["tf32", "bf16x3"])
+@pytest.mark.parametrize("math", ["tf32", "f16x3"])
 def test_reddit_full_size_replay_and_pruning(B, oracle, math):
     cfg = wl.CONFIGS["reddit"]
     rig = _full_size(B, oracle, cfg, {3, 400}, 400, math=math)
@@ -1010,7 +1078,7 @@ def test_reddit_full_size_replay_and_pruning(B, oracle, math):
 
 
 @pytest.mark.slow
-@pytest.mark.parametrize("math", ["tf32", "bf16x3"])
+@pytest.mark.parametrize("math", ["tf32", "f16x3"])
 def test_lastfm_full_size_hub_contention(B, oracle, math):
     cfg = wl.CONFIGS["lastfm"]
     rig = _full_size(B, oracle, cfg, {2, 60}, 60, math=math)
@@ -1019,7 +1087,7 @@ def test_lastfm_full_size_hub_contention(B, oracle, math):
 
 
 @pytest.mark.slow
-@pytest.mark.parametrize("math", ["tf32", "bf16x3"])
+@pytest.mark.parametrize("math", ["tf32", "f16x3"])
 def test_large_full_size_bf16(B, oracle, math):
     # 17,000 nodes, 50 M events, 18.6 GB of bf16 edge features resident in HBM (generated on the device),
     # batch 4,000, 20 % replay with pruning; about a minute of host set-up (T-CSR over 10^8 entries).  The
