@@ -1,5 +1,7 @@
 // Step (6): masked link-prediction loss (Eq. 13), exact backward of steps (4)-(5),
 // gradient norm g_r and the Adam update.
+#include <cstdlib>
+
 #include "tgnn_internal.cuh"
 #include "tgnn_device.cuh"
 
@@ -1017,15 +1019,10 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     TGNN_LAUNCH_OK(ctx, "attention_bwd");
     RC(fork_to(ctx, s, sa));
     RC(fork_to(ctx, s, sb));
-    if (split) {
-      // dW_kv = dKV^T Z over the neighbor rows; Z's column of ones yields the bias gradient as the last column
-      SplitMat a = dkvs, b = zs;
-      a.rows = NB; a.cols = 2 * d; b.rows = NB; b.cols = L.dkv + 1;
-      RC(launch_gemm_split(ctx, a, b, 1, G + L.wk, L.dkv, 2 * d, (int)L.dkv + 1, NB, nullptr, 0, 1, 1 << 20, "dW_kv", sa, 0, 0,
-                           (int)L.dkv, G + L.bk));
-    } else {
+    // dW_kv is a leaf of the chain, its input-gradient sibling dZ is on it, and the split kernel is persistent (a
+    // launch fills the machine until it ends): in that mode the weight gradient is issued after dZ, further down.
+    if (!split)
       RC(grad_w(ctx, w.dKV, 2 * d, w.Z, ctx->ld_kv, NB, nullptr, 2 * d, (int)L.dkv, G + L.wk, G + L.bk, "dW_kv", sa));
-    }
     // time-encoder gradient through the attention inputs (side stream b)
     const size_t tg_smem = (size_t)8 * 2 * d * sizeof(double);
     // gradient w.r.t. the memory columns and the time-encoding columns of Z, side by side in dZmp.  With the
@@ -1047,7 +1044,14 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     if (split) {
       RC(launch_gemm_split(ctx, dkvs, ctx->wz_s, 0, w.dZmp, 2 * d, NB, 2 * d, 2 * d, nullptr, 0, 0, 1, "dZ", s));
       RC(fork_to(ctx, s, sa));
-      s_tgz = sa;
+      RC(fork_to(ctx, s, sb));
+      // dW_kv = dKV^T Z over the neighbor rows; Z's column of ones yields the bias gradient as the last column.  It
+      // starts when dZ has finished and runs beside the rest of the chain (scatter, cell backward, ...).
+      SplitMat a = dkvs, b = zs;
+      a.rows = NB; a.cols = 2 * d; b.rows = NB; b.cols = L.dkv + 1;
+      RC(launch_gemm_split(ctx, a, b, 1, G + L.wk, L.dkv, 2 * d, (int)L.dkv + 1, NB, nullptr, 0, 1, 1 << 20, "dW_kv", sa, 0, 0,
+                           (int)L.dkv, G + L.bk));
+      s_tgz = sb;
     } else if (merged_dz) {
       RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, 0, NB, nullptr, 2 * d, 2 * d, w.dZmp, 2 * d, "dZ", s, SITE_DZ + 1));
       RC(fork_to(ctx, s, sa));
@@ -1069,7 +1073,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       {
         KernelScope scope__(ctx, "scatter_dmem", s);
         // many rows per node (small node set, large batch): sum per block first, the hub rows would serialise
-        if ((int64_t)NB >= 4 * c.num_nodes)
+        if ((int64_t)NB >= (getenv("TGNN_SC") ? atoi(getenv("TGNN_SC")) : 4) * c.num_nodes)
           scatter_dmem_cached_kernel<<<(NB + R + SC_ROWS - 1) / SC_ROWS, 256, (size_t)SC_WAYS * d * sizeof(float), s>>>(
               w.dZmp, w.dcat_o, w.dzq, ctx->e_nbr, ctx->e_nodes, R, k, d, w.node2slot, w.dMemU, c.num_nodes);
         else

@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
                                                                     const double* __restrict__ ts, int ld,
                                                                     __nv_bfloat16* __restrict__ z_hi, int64_t plane_s,
                                                                     float* __restrict__ z_dt, float* __restrict__ Zq, int64_t N,
-                                                                    int64_t E, int32_t* status) {
+                                                                    int64_t E, int32_t* status, int g_begin, int g_end) {
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   const int nb_rows = n * k;
@@ -180,7 +180,8 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
     tw[u][0] = in ? time_w[q] : 0.f; tw[u][1] = in ? time_w[q + 1] : 0.f;
     tb[u][0] = in ? time_b[q] : 0.f; tb[u][1] = in ? time_b[q + 1] : 0.f;
   }
-  for (int gidx = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; gidx < groups; gidx += warps) {
+  // this launch covers the row groups [g_begin, g_end) (the gather goes out as several launches, see the launcher)
+  for (int gidx = g_begin + ((blockIdx.x * blockDim.x + threadIdx.x) >> 5); gidx < min(groups, g_end); gidx += warps) {
     const int r0 = gidx * ZS_ROWS;
     int my_nbr = -1, my_eid = 0;
     float my_dt = 0.f;
@@ -272,7 +273,8 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
       if (lane == 0) z_dt[r] = dtf;
     }
   }
-  // the Phi(0) half of z_q (fp32: the query projection is not one of the split products)
+  // the Phi(0) half of z_q (fp32: the query projection is not one of the split products); with the first launch
+  if (g_begin == 0)
   for (int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps)
     for (int q = lane; q < d; q += 32) Zq[(int64_t)i * 2 * d + d + q] = time_encode(time_w[q], time_b[q], 0.f);
 }
@@ -442,12 +444,20 @@ int launch_embed_static(tgnn_ctx* ctx, const double* times, int n, const int32_t
   Workspace& w = ctx->ws;
   {
     KernelScope scope__(ctx, "gather_z_static", s);
-    if (ctx->split_buf != nullptr && ctx->z_split)
-      gather_z_static_split_kernel<<<(n * c.k / ZS_ROWS + n + 7) / 8 + 1, 256, 0, s>>>(
-          ctx->efeat, c.feat_dtype == TGNN_BF16, ctx->params + L.time_w, ctx->params + L.time_b, c.d, c.d_e, c.k, times, n, nbr,
-          eid, ts, (int)ctx->zs.ld, reinterpret_cast<__nv_bfloat16*>(ctx->zs.hi), ctx->zs.plane_stride, w.z_dt, w.Zq,
-          c.num_nodes, ctx->num_events, w.status);
-    else
+    if (ctx->split_buf != nullptr && ctx->z_split) {
+      // In three pieces: the gather runs on a low-priority side stream beside the memory update, whose
+      // products need whole SMs; between two pieces the SMs that drain go to those kernels first.
+      const int groups = (n * c.k + ZS_ROWS - 1) / ZS_ROWS, per = (groups + 2) / 3 > 0 ? (groups + 2) / 3 : 1;
+      for (int g0 = 0; g0 < groups; g0 += per) {
+        const int g1 = g0 + per < groups ? g0 + per : groups;
+        gather_z_static_split_kernel<<<(g1 - g0 + 7) / 8 + 1, 256, 0, s>>>(
+            ctx->efeat, c.feat_dtype == TGNN_BF16, ctx->params + L.time_w, ctx->params + L.time_b, c.d, c.d_e, c.k, times, n,
+            nbr, eid, ts, (int)ctx->zs.ld, reinterpret_cast<__nv_bfloat16*>(ctx->zs.hi), ctx->zs.plane_stride, w.z_dt, w.Zq,
+            c.num_nodes, ctx->num_events, w.status, g0, g1);
+        ctx->launches++;
+      }
+      ctx->launches--;
+    } else
       gather_z_static_kernel<<<(n * c.k / ZS_ROWS + n + 7) / 8 + 1, 256, 0, s>>>(ctx->efeat, c.feat_dtype == TGNN_BF16, ctx->params + L.time_w,
                                                           ctx->params + L.time_b, c.d, c.d_e, c.k, times, n, nbr, eid, ts,
                                                           ctx->ld_kv, w.Z, w.z_dt, w.Zq, c.num_nodes, ctx->num_events, w.status);

@@ -66,6 +66,7 @@ struct BfArgs {
                               // then fetched once per row tile instead of once per pair)
   int m_tiles, n_tiles, bn, split_k;
   int kb_total;               // contraction blocks (64 elements K-major, 32 rows MN-major)
+  int kb_begin, kb_end;       // the part of them this launch covers (a long weight gradient goes out as several launches)
   int ksteps_total;           // MMA steps of 16 over the whole contraction
   int a_slot_bytes, b_slot_bytes, n_a_slots, n_b_slots;
   int b_chunks;               // MN-major: 64-column chunks per B tile
@@ -162,9 +163,9 @@ __device__ __forceinline__ bool next_item(const BfArgs& g, Walk& wk, Item& it) {
     const int nt = combo % g.n_tiles, sp = combo / g.n_tiles;
     it.n0 = nt * g.bn;
     it.n_valid = nt == g.n_tiles - 1 ? g.N - it.n0 : g.bn;
-    const int per = (g.kb_total + g.split_k - 1) / g.split_k;
-    it.kb0 = sp * per;
-    it.kb1 = min(g.kb_total, it.kb0 + per);
+    const int per = (g.kb_end - g.kb_begin + g.split_k - 1) / g.split_k;
+    it.kb0 = g.kb_begin + sp * per;
+    it.kb1 = min(g.kb_end, it.kb0 + per);
     if (it.kb0 < it.kb1) return true;   // an empty contraction range is skipped by every role alike
   }
   return false;
@@ -344,7 +345,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_split_kernel(const __grid_con
       if (g.single || t < it.tiles) {
         const int m0 = (it.mt0 + (g.single ? 0 : t)) * BM;
         const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(acc_i * ACC_STRIDE);
-        const bool with_bias = g.bias != nullptr && it.kb0 == 0;
+        const bool with_bias = g.bias != nullptr && it.kb0 == 0;   // (the bias goes in with the first contraction block)
         for (int c0 = c_first; c0 < it.n_valid; c0 += c_step) {
           uint32_t r[32];
           asm volatile(
@@ -583,7 +584,8 @@ int launch_split_rows(tgnn_ctx* ctx, const float* X, int64_t ld_in, int64_t rows
 // split_k > 1 needs accumulate (C holds valid data; partial sums are added atomically).
 int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int mn_major, float* C, int64_t ldc, int M, int N,
                       int K, const float* bias, int relu, int accumulate, int split_k, const char* name, cudaStream_t s,
-                      int debug_withhold, unsigned spin_limit, int extra_col, float* extra_out, long long* trace, int single) {
+                      int debug_withhold, unsigned spin_limit, int extra_col, float* extra_out, long long* trace, int single,
+                      int launches) {
   if (M <= 0 || N <= 0) return TGNN_OK;
   if (K <= 0) return set_error(ctx, TGNN_EINVAL, "gemm %s: empty contraction", name);
   if (split_k > 1 && !accumulate) return set_error(ctx, TGNN_EINVAL, "gemm %s: split_k needs accumulate", name);
@@ -650,11 +652,21 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
     const int rc = raise_smem_limit(ctx, gemm_split_kernel, SMEM_LIMIT - 1024, smem_limit);
     if (rc) return rc;
   }
-  {
-    KernelScope scope__(ctx, name, s);
-    gemm_split_kernel<<<items < 148 ? items : 148, THREADS, smem, s>>>(a);
+  // A long accumulating product may go out as several launches over consecutive parts of the contraction: a
+  // persistent launch holds every SM until it ends, and the boundaries between the parts are where kernels of
+  // the step's critical chain (higher stream priority) get in.
+  int parts = (accumulate && launches > 1) ? launches : 1;
+  if (parts > a.kb_total / (4 * a.split_k)) parts = a.kb_total / (4 * a.split_k);
+  if (parts < 1) parts = 1;
+  for (int p = 0; p < parts; ++p) {
+    a.kb_begin = (int)((long long)a.kb_total * p / parts);
+    a.kb_end = (int)((long long)a.kb_total * (p + 1) / parts);
+    {
+      KernelScope scope__(ctx, name, s);
+      gemm_split_kernel<<<items < 148 ? items : 148, THREADS, smem, s>>>(a);
+    }
+    TGNN_LAUNCH_OK(ctx, name);
   }
-  TGNN_LAUNCH_OK(ctx, name);
   return TGNN_OK;
 }
 

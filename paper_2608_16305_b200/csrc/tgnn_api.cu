@@ -294,7 +294,14 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
   ctx->graphs_enabled = 1;
   ctx->defer_adam = 0;
   ctx->grad_pending = false;
-  for (int i = 0; ok && i < 2; ++i) ok = cudaStreamCreateWithFlags(&ctx->side[i], cudaStreamNonBlocking) == cudaSuccess;
+  {
+    // the side streams carry work that is off the step's critical chain: lowest priority, so that a kernel of the
+    // chain (the caller's stream) gets the next free SM slots when both have blocks waiting
+    int least = 0, greatest = 0;
+    ok = ok && cudaDeviceGetStreamPriorityRange(&least, &greatest) == cudaSuccess;
+    for (int i = 0; ok && i < 2; ++i)
+      ok = cudaStreamCreateWithPriority(&ctx->side[i], cudaStreamNonBlocking, least) == cudaSuccess;
+  }
   for (int i = 0; ok && i < 32; ++i) ok = cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
@@ -644,7 +651,8 @@ int tgnn_train_step(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, c
   }
   e->kernels = ctx->launches - l0;
   cudaGraphExec_t exec = nullptr;
-  const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
+  // node priorities as captured (side-stream kernels low, the caller's stream as it is) instead of one priority for all
+  const cudaError_t ie = cudaGraphInstantiate(&exec, graph, cudaGraphInstantiateFlagUseNodePriority);
   cudaGraphDestroy(graph);
   if (ie != cudaSuccess || !exec) {
     cudaGetLastError();
