@@ -525,13 +525,14 @@ __global__ void __launch_bounds__(256) scatter_dmem_cached_kernel(const float* _
 // (dw) and acc[d:2d] (db).  Dynamic shared memory: 8 * 2 * d doubles.
 constexpr int TG_MAXJ = 8;
 // Rows per block: every block ends with one fp64 atomic per column onto the same 2d addresses, and those
-// serialise, so the grid is kept to about one block per SM (rows per block a multiple of the 8 warps);
-// inside a block each warp walks its rows four at a time so that their loads overlap.
+// serialise, so the grid is kept to about two blocks per SM, as many as fit at once (rows per block a multiple
+// of the 8 warps); inside a block each warp walks its rows two at a time so that their loads overlap.
+constexpr int TG_U = 2;   // rows a warp has in flight (more would cost the registers that let two blocks share an SM)
 inline int tg_rows_per_block(int rows) {
-  const int r = (rows + 147) / 148;
+  const int r = (rows + 295) / 296;
   return r < 8 ? 8 : (r + 7) / 8 * 8;
 }
-__global__ void __launch_bounds__(256) time_grad_kernel(const float* __restrict__ G, int64_t ldg, int col0,
+__global__ void __launch_bounds__(256, 2) time_grad_kernel(const float* __restrict__ G, int64_t ldg, int col0,
                                                         const float* __restrict__ S, const float* __restrict__ dt,
                                                         int rows, const int32_t* __restrict__ dev_rows, int d,
                                                         const float* __restrict__ time_w,
@@ -561,11 +562,11 @@ __global__ void __launch_bounds__(256) time_grad_kernel(const float* __restrict_
       else sb[v] = make_float4(sinf(bv[v].x), sinf(bv[v].y), sinf(bv[v].z), sinf(bv[v].w));
     }
   }
-  for (int rb = r0 + wid; rb < r1; rb += 32) {  // rows rb, rb + 8, rb + 16, rb + 24: loads first, sums after
-    float4 g[4][2], sn[4][2];
-    float dtr[4];
+  for (int rb = r0 + wid; rb < r1; rb += 8 * TG_U) {  // rows rb, rb + 8, ...: loads first, sums after
+    float4 g[TG_U][2], sn[TG_U][2];
+    float dtr[TG_U];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < TG_U; ++u) {
       const int r = rb + 8 * u;
       const bool in = r < r1;
       dtr[u] = (in && dt) ? dt[r] : 0.f;
@@ -579,7 +580,7 @@ __global__ void __launch_bounds__(256) time_grad_kernel(const float* __restrict_
     }
     if (recompute) {
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < TG_U; ++u) {
         const bool live = rb + 8 * u < r1 && dtr[u] >= 0.f;
 #pragma unroll
         for (int v = 0; v < 2; ++v) {
@@ -597,7 +598,7 @@ __global__ void __launch_bounds__(256) time_grad_kernel(const float* __restrict_
       }
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < TG_U; ++u) {
 #pragma unroll
       for (int v = 0; v < 2; ++v) {
         const float ge[4] = {g[u][v].x, g[u][v].y, g[u][v].z, g[u][v].w};
@@ -882,6 +883,20 @@ int launch_get_gates(tgnn_ctx* ctx, uint8_t* h_gate_out, uint8_t* hid_gate_out, 
   return TGNN_OK;
 }
 
+// G[wk + r * dkv + c] += pad[r * ld + c] for c < dkv, G[bk + r] += pad[r * ld + dkv]: the weight gradient of the
+// key/value projection is accumulated in a copy with 16-byte aligned rows (vector atomics from every contraction
+// split instead of four scalar ones) and folded into the flat gradient once.
+__global__ void __launch_bounds__(256) fold_dwkv_kernel(const float* __restrict__ pad, int ld, int rows, int dkv,
+                                                        float* __restrict__ g_w, float* __restrict__ g_b) {
+  const int total = rows * (dkv + 1);
+  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
+    const int r = e / (dkv + 1), c = e - r * (dkv + 1);
+    const float v = pad[(int64_t)r * ld + c];
+    if (c < dkv) g_w[(int64_t)r * dkv + c] += v;
+    else g_b[r] += v;
+  }
+}
+
 #define RC(x)            \
   do {                   \
     int rc__ = (x);      \
@@ -1049,8 +1064,12 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       // starts when dZ has finished and runs beside the rest of the chain (scatter, cell backward, ...).
       SplitMat a = dkvs, b = zs;
       a.rows = NB; a.cols = 2 * d; b.rows = NB; b.cols = L.dkv + 1;
-      RC(launch_gemm_split(ctx, a, b, 1, G + L.wk, L.dkv, 2 * d, (int)L.dkv + 1, NB, nullptr, 0, 1, 1 << 20, "dW_kv", sa, 0, 0,
-                           (int)L.dkv, G + L.bk));
+      RC(launch_gemm_split(ctx, a, b, 1, w.dWkv_pad, ctx->ld_wkv, 2 * d, (int)L.dkv + 1, NB, nullptr, 0, 1, 1 << 20, "dW_kv", sa));
+      {
+        KernelScope scope__(ctx, "fold_dW_kv", sa);
+        fold_dwkv_kernel<<<148, 256, 0, sa>>>(w.dWkv_pad, ctx->ld_wkv, 2 * d, (int)L.dkv, G + L.wk, G + L.bk);
+      }
+      TGNN_LAUNCH_OK(ctx, "fold_dW_kv");
       s_tgz = sb;
     } else if (merged_dz) {
       RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, 0, NB, nullptr, 2 * d, 2 * d, w.dZmp, 2 * d, "dZ", s, SITE_DZ + 1));

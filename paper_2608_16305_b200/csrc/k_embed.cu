@@ -445,9 +445,10 @@ int launch_embed_static(tgnn_ctx* ctx, const double* times, int n, const int32_t
   {
     KernelScope scope__(ctx, "gather_z_static", s);
     if (ctx->split_buf != nullptr && ctx->z_split) {
-      // In three pieces: the gather runs on a low-priority side stream beside the memory update, whose
+      // Large batches in three pieces: the gather runs on a low-priority side stream beside the memory update, whose
       // products need whole SMs; between two pieces the SMs that drain go to those kernels first.
-      const int groups = (n * c.k + ZS_ROWS - 1) / ZS_ROWS, per = (groups + 2) / 3 > 0 ? (groups + 2) / 3 : 1;
+      const int groups = (n * c.k + ZS_ROWS - 1) / ZS_ROWS;
+      const int per = groups >= 32768 ? (groups + 2) / 3 : groups;   // (small batches: one launch)
       for (int g0 = 0; g0 < groups; g0 += per) {
         const int g1 = g0 + per < groups ? g0 + per : groups;
         gather_z_static_split_kernel<<<(g1 - g0 + 7) / 8 + 1, 256, 0, s>>>(

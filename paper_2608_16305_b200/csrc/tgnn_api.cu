@@ -148,8 +148,9 @@ size_t carve(tgnn_ctx* ctx, char* base) {
   cv.take(w.adam_sc, 4);
   cv.take(w.counters, 4);
   cv.take(w.status, 4);
-  // cleared together at the start of every backward pass: keep these five adjacent and in this order
+  // cleared together at the start of every backward pass: keep these six adjacent and in this order
   cv.take(w.grads, (size_t)ctx->L.total);
+  cv.take_packed(w.dWkv_pad, (size_t)2 * d * ctx->ld_wkv);
   cv.take_packed(w.dMemU, U * d);
   cv.take_packed(w.red, 4);
   cv.take_packed(w.tg_acc, 4 * d);  // time encoder dw | db, time projection dw_p | db_p
@@ -216,6 +217,7 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
   ctx->nq_cap = cfg->max_roots / 3;
   ctx->ld_msg = (int)((ctx->L.dmsg + 31) / 32 * 32);
   ctx->ld_kv = (int)((ctx->L.dkv + 31) / 32 * 32);
+  ctx->ld_wkv = (int)((ctx->L.dkv + 1 + 3) / 4 * 4);
   ctx->arena_bytes = carve(ctx, nullptr);
   if (cudaMalloc(&ctx->arena, ctx->arena_bytes) != cudaSuccess) {
     cudaGetLastError();

@@ -78,6 +78,7 @@ struct Workspace {
   float* dGi;     // [U_cap, 3d]
   float* dGh;     // [U_cap, 3d]
   float* dXp;     // [U_cap, d]   grad wrt the time-encoding part of the winners' messages
+  float* dWkv_pad;  // [2d, ld_wkv] W_kv's gradient (and, in column dkv, its bias gradient) with 16-byte aligned rows
   float* grads;   // [P]
   double* red;    // [4] sum of squares, spare
   double* tg_acc; // [2d] fp64 sums of the time-encoder gradient (dw | db)
@@ -138,6 +139,7 @@ struct tgnn_ctx {
   tgnn::ParamLayout L;
   int U_cap, R_cap, NB_cap, nq_cap;
   int ld_msg, ld_kv;  // padded leading dimensions of X and Z
+  int ld_wkv;         // row pitch of the padded W_kv gradient: dkv + 1 rounded up to a multiple of 4
   // borrowed
   const int64_t* indptr;
   const int32_t *g_nbr, *g_eid;
