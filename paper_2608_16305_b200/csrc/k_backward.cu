@@ -1092,7 +1092,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       {
         KernelScope scope__(ctx, "scatter_dmem", s);
         // many rows per node (small node set, large batch): sum per block first, the hub rows would serialise
-        if ((int64_t)NB >= (getenv("TGNN_SC") ? atoi(getenv("TGNN_SC")) : 4) * c.num_nodes)
+        if ((int64_t)NB >= 4 * (int64_t)c.num_nodes)
           scatter_dmem_cached_kernel<<<(NB + R + SC_ROWS - 1) / SC_ROWS, 256, (size_t)SC_WAYS * d * sizeof(float), s>>>(
               w.dZmp, w.dcat_o, w.dzq, ctx->e_nbr, ctx->e_nodes, R, k, d, w.node2slot, w.dMemU, c.num_nodes);
         else
