@@ -334,7 +334,11 @@ TGNN_API int64_t tgnn_kernel_launches(const tgnn_ctx* ctx);
  * accumulate / split_k as in tgnn_debug_gemm.  debug_withhold > 0 makes the kernel keep that many shared-memory
  * slots to itself instead of handing them back, and spin_limit > 0 shortens its bounded waits: together they let
  * a test make a wait run out (the kernel then records TGNN_ETIMEOUT, stores nothing further, frees its tensor
- * memory and returns; the context stays usable).  Both 0 in normal use. */
+ * memory and returns; the context stays usable).  Both 0 in normal use.  Environment switches read by this call
+ * only: TGNN_GEMM_PAIR=0|1 forces the one-CTA-per-tile form or the CTA-pair form (one 256-row MMA across two SMs,
+ * each loading half of the B tile; default: pairs for K-major products of 32 row tiles and more),
+ * TGNN_GEMM_SINGLE=0|1 the walk by pairs of row tiles or by single tiles, TGNN_GEMM_BF16=1 bf16 planes,
+ * TGNN_GEMM_SCALE=s a scale of 2^s on A. */
 TGNN_API int tgnn_debug_gemm_split(tgnn_ctx* ctx, const float* A, int64_t a_rs, int64_t a_cs, const float* B, int64_t b_rs,
                                    int64_t b_cs, float* C, int64_t ldc, int M, int N, int K, const float* bias, int relu,
                                    int accumulate, int split_k, void* scratch, int64_t scratch_bytes, int debug_withhold,

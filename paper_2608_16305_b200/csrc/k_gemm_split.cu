@@ -70,6 +70,7 @@ struct BfArgs {
   int ksteps_total;           // MMA steps of 16 over the whole contraction
   int a_slot_bytes, b_slot_bytes, n_a_slots, n_b_slots;
   int b_chunks;               // MN-major: 64-column chunks per B tile
+  int stage_bytes, n_stages;  // CTA-pair kernel: one ring of stages, each an A tile (both planes) followed by this CTA's half of the B tile
   // accumulate mode: column `extra_col` of the product (if >= 0) is added to extra_out[row] instead of C --
   // a column of ones appended to B turns that column into the row sums of A, i.e. a bias gradient
   int extra_col;
@@ -175,6 +176,80 @@ __device__ __forceinline__ void tma_4d(uint32_t dst, const CUtensorMap* map, int
       "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
       : "memory");
+}
+
+// One epilogue warp's share of a finished 128-row accumulator: columns c_first, c_first + c_step, ... (groups of 32)
+// of the lane quarter q4, from tensor memory through the warp's staging square to C (bias / ReLU / scale, or an
+// atomic accumulate).
+__device__ __forceinline__ void drain_tile(const BfArgs& g, const Item& it, int m0, uint32_t taddr, int c_first, int c_step,
+                                           float* stg, int lane, int q4, bool c_vec) {
+  const int sub = lane >> 2, ch = lane & 3;
+  const bool with_bias = g.bias != nullptr && it.kb0 == 0;   // (the bias goes in with the first contraction block)
+  for (int c0 = c_first; c0 < it.n_valid; c0 += c_step) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr + (uint32_t)c0));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int cb0 = c0 + 16 * h;
+      if (cb0 >= it.n_valid) break;   // warp-uniform
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        *reinterpret_cast<uint4*>(stg + lane * STG_PITCH + 4 * q) =
+            make_uint4(r[16 * h + 4 * q], r[16 * h + 4 * q + 1], r[16 * h + 4 * q + 2], r[16 * h + 4 * q + 3]);
+      __syncwarp();
+      const int col = cb0 + 4 * ch;   // first of this lane's four columns, relative to the tile
+      float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (with_bias && col < it.n_valid) {
+        const float* bp = g.bias + it.n0 + col;
+        b4.x = bp[0];
+        if (col + 1 < it.n_valid) b4.y = bp[1];
+        if (col + 2 < it.n_valid) b4.z = bp[2];
+        if (col + 3 < it.n_valid) b4.w = bp[3];
+      }
+      const int xc = g.extra_col - it.n0 - col;   // 0..3: one of this lane's columns is the extra column
+      const bool full4 = col + 3 < it.n_valid && (xc < 0 || xc > 3);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int rr = j * 8 + sub;
+        const int row = m0 + q4 * 32 + rr;
+        float4 v = *reinterpret_cast<const float4*>(stg + rr * STG_PITCH + 4 * ch);
+        if (row < g.M && col < it.n_valid) {
+          v.x = fmaf(v.x, g.out_scale, b4.x); v.y = fmaf(v.y, g.out_scale, b4.y);
+          v.z = fmaf(v.z, g.out_scale, b4.z); v.w = fmaf(v.w, g.out_scale, b4.w);
+          float* cp = g.C + (int64_t)row * g.ldc + it.n0 + col;
+          if (g.accumulate) {
+            if (full4 && c_vec) {
+              atomicAdd(reinterpret_cast<float4*>(cp), v);
+            } else {
+              const float vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+              for (int e2 = 0; e2 < 4; ++e2)
+                if (col + e2 < it.n_valid) atomicAdd(e2 == xc ? g.extra_out + row : cp + e2, vv[e2]);
+            }
+          } else {
+            if (g.relu) { v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); v.z = fmaxf(v.z, 0.f); v.w = fmaxf(v.w, 0.f); }
+            if (full4 && c_vec) {
+              *reinterpret_cast<float4*>(cp) = v;
+            } else {
+              cp[0] = v.x;
+              if (col + 1 < it.n_valid) cp[1] = v.y;
+              if (col + 2 < it.n_valid) cp[2] = v.z;
+              if (col + 3 < it.n_valid) cp[3] = v.w;
+            }
+          }
+        }
+      }
+      __syncwarp();
+    }
+  }
 }
 
 __global__ void __launch_bounds__(THREADS, 1) gemm_split_kernel(const __grid_constant__ BfArgs g) {
@@ -325,7 +400,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_split_kernel(const __grid_con
     const int q4 = warp & 3;       // the tensor-memory lane quarter this warp may read
     float* stg = stg_base + e * (32 * STG_PITCH);
     const bool c_vec = (((uintptr_t)g.C & 15) == 0) && (g.ldc % 4 == 0);
-    const int sub = lane >> 2, ch = lane & 3;
     uint32_t n_item = 0;
     bool ok = true;
     Walk wk = cta_walk(g);
@@ -345,72 +419,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_split_kernel(const __grid_con
       if (g.single || t < it.tiles) {
         const int m0 = (it.mt0 + (g.single ? 0 : t)) * BM;
         const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(acc_i * ACC_STRIDE);
-        const bool with_bias = g.bias != nullptr && it.kb0 == 0;   // (the bias goes in with the first contraction block)
-        for (int c0 = c_first; c0 < it.n_valid; c0 += c_step) {
-          uint32_t r[32];
-          asm volatile(
-              "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-              "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-              : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-                "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-                "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-                "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-              : "r"(taddr + (uint32_t)c0));
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const int cb0 = c0 + 16 * h;
-            if (cb0 >= it.n_valid) break;   // warp-uniform
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-              *reinterpret_cast<uint4*>(stg + lane * STG_PITCH + 4 * q) =
-                  make_uint4(r[16 * h + 4 * q], r[16 * h + 4 * q + 1], r[16 * h + 4 * q + 2], r[16 * h + 4 * q + 3]);
-            __syncwarp();
-            const int col = cb0 + 4 * ch;   // first of this lane's four columns, relative to the tile
-            float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (with_bias && col < it.n_valid) {
-              const float* bp = g.bias + it.n0 + col;
-              b4.x = bp[0];
-              if (col + 1 < it.n_valid) b4.y = bp[1];
-              if (col + 2 < it.n_valid) b4.z = bp[2];
-              if (col + 3 < it.n_valid) b4.w = bp[3];
-            }
-            const int xc = g.extra_col - it.n0 - col;   // 0..3: one of this lane's columns is the extra column
-            const bool full4 = col + 3 < it.n_valid && (xc < 0 || xc > 3);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const int rr = j * 8 + sub;
-              const int row = m0 + q4 * 32 + rr;
-              float4 v = *reinterpret_cast<const float4*>(stg + rr * STG_PITCH + 4 * ch);
-              if (row < g.M && col < it.n_valid) {
-                v.x = fmaf(v.x, g.out_scale, b4.x); v.y = fmaf(v.y, g.out_scale, b4.y);
-                v.z = fmaf(v.z, g.out_scale, b4.z); v.w = fmaf(v.w, g.out_scale, b4.w);
-                float* cp = g.C + (int64_t)row * g.ldc + it.n0 + col;
-                if (g.accumulate) {
-                  if (full4 && c_vec) {
-                    atomicAdd(reinterpret_cast<float4*>(cp), v);
-                  } else {
-                    const float vv[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                    for (int e2 = 0; e2 < 4; ++e2)
-                      if (col + e2 < it.n_valid) atomicAdd(e2 == xc ? g.extra_out + row : cp + e2, vv[e2]);
-                  }
-                } else {
-                  if (g.relu) { v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); v.z = fmaxf(v.z, 0.f); v.w = fmaxf(v.w, 0.f); }
-                  if (full4 && c_vec) {
-                    *reinterpret_cast<float4*>(cp) = v;
-                  } else {
-                    cp[0] = v.x;
-                    if (col + 1 < it.n_valid) cp[1] = v.y;
-                    if (col + 2 < it.n_valid) cp[2] = v.z;
-                    if (col + 3 < it.n_valid) cp[3] = v.w;
-                  }
-                }
-              }
-            }
-            __syncwarp();
-          }
-        }
+        drain_tile(g, it, m0, taddr, c_first, c_step, stg, lane, q4, c_vec);
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
@@ -429,6 +438,248 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_split_kernel(const __grid_con
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+  }
+}
+
+// ---- CTA pairs (a cluster of two CTAs on the two SMs of one processing cluster, one 256-row MMA across both) ----
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// the shared::cluster address of the same shared-memory location in the CTA of rank `rank`
+__device__ __forceinline__ uint32_t peer_addr(uint32_t local, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+// tile copy into this CTA's shared memory whose completion is counted on a barrier of the pair's leader
+__device__ __forceinline__ void tma_3d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t cluster_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(cluster_bar)
+      : "memory");
+}
+__device__ __forceinline__ void mma_f16_pair(uint32_t tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// arrives on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs issued so far have retired
+__device__ __forceinline__ void commit_to_pair(uint32_t bar) {
+  const uint16_t both = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(both) : "memory");
+}
+
+// The walk of a CTA pair: a contiguous range of units (n-tile major, 256-row tile minor), one unit per item.
+__device__ __forceinline__ Walk pair_walk(const BfArgs& g) {
+  const long long T = (long long)g.m_tiles * g.n_tiles;
+  const unsigned c = blockIdx.x >> 1, nc = gridDim.x >> 1;
+  Walk w;
+  w.u = (int)(T * c / nc);
+  w.u_end = (int)(T * (c + 1) / nc);
+  return w;
+}
+__device__ __forceinline__ bool next_pair_item(const BfArgs& g, Walk& wk, Item& it) {
+  if (wk.u >= wk.u_end) return false;
+  const int nt = wk.u / g.m_tiles;
+  it.mt0 = wk.u - nt * g.m_tiles;
+  it.tiles = 1;
+  ++wk.u;
+  it.n0 = nt * g.bn;
+  it.n_valid = nt == g.n_tiles - 1 ? g.N - it.n0 : g.bn;
+  it.kb0 = 0;
+  it.kb1 = g.kb_total;
+  return true;
+}
+
+// K-major products with many row tiles, on pairs of CTAs.  A work item is a 256-row tile of C: each CTA of the
+// pair loads its own 128 rows of A and HALF of the B tile (the leader the first n/2 rows of the [n, K] operand,
+// its peer the second half), the leader issues one MMA of 256 rows for both, and each CTA finds its 128 rows of
+// the accumulator in its own tensor memory and stores them.  Per flop a CTA pulls 58 KB instead of 84 KB through
+// its shared memory for a 208-column tile, and the accumulators still alternate between two halves of tensor
+// memory so that a tile's epilogue runs beside the next tile's MMAs.  Barriers: a stage's full barrier lives in the
+// leader and counts the bytes of both CTAs' copies; its empty barrier and the accumulator-full barriers live in
+// both CTAs and are signalled together by a multicast commit; the accumulator-empty barriers live in the leader
+// and collect the epilogue warps of both CTAs.  Every wait is bounded as in the single-CTA kernel; a CTA that gives
+// up also raises its peer's abort flag, and both meet at the cluster barrier before tensor memory is freed.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_split_pair_kernel(const __grid_constant__ BfArgs g) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) uint64_t s_full[MAX_SLOTS], s_empty[MAX_SLOTS];
+  __shared__ __align__(8) uint64_t s_tmem_full[2], s_tmem_empty[2];
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_rank();
+  const bool leader = rank == 0;
+  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t ring = smem_u32(smem);
+  float* stg_base = reinterpret_cast<float*>(smem + (size_t)g.n_stages * g.stage_bytes);
+
+  if (tid == 0) {
+    for (int s = 0; s < MAX_SLOTS; ++s) {
+      mbar_init(smem_u32(&s_full[s]), 1);    // the leader's own arrive with the byte count of both CTAs' copies
+      mbar_init(smem_u32(&s_empty[s]), 1);   // one multicast commit
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&s_tmem_full[b]), 1);
+      mbar_init(smem_u32(&s_tmem_empty[b]), 2 * EPI_WARPS);   // (used in the leader: epilogue warps of both CTAs)
+    }
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {   // both CTAs of the pair take part in the pair-wide allocation
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync_all();   // the peer's barriers are initialised before anything is counted on them
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = s_tmem;
+  volatile int* abort_flag = &s_abort;
+  const unsigned limit = g.spin_limit;
+  const uint32_t stage_bytes = (uint32_t)g.stage_bytes, n_stages = (uint32_t)g.n_stages;
+  const uint32_t a_bytes = 2u * BM * 128u;                 // both planes of the A tile
+  const uint32_t b_plane = (stage_bytes - a_bytes) >> 1;   // one plane of this CTA's half of the B tile
+  const int b_rows = (int)(b_plane >> 7);                  // rows of the copied half (the widest n-tile's)
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ tile copies (each CTA its own)
+    if (lane == 0) {
+      uint32_t c = 0;
+      bool ok = true;
+      Walk wk = pair_walk(g);
+      Item it;
+      (void)b_rows;
+      while (ok && next_pair_item(g, wk, it)) {
+        const int n_mma = (it.n_valid + 15) / 16 * 16;
+        const int m0 = (2 * it.mt0 + (int)rank) * BM;
+        const int nb0 = it.n0 + (int)rank * (n_mma >> 1);   // first B row of this CTA's half
+        for (int kb = it.kb0; kb < it.kb1 && ok; ++kb) {
+          const uint32_t s = c % n_stages;
+          ok = mbar_wait(smem_u32(&s_empty[s]), ((c / n_stages) & 1u) ^ 1u, limit, abort_flag);
+          if (!ok) break;
+          const uint32_t dst = ring + s * stage_bytes;
+          const uint32_t bar = peer_addr(smem_u32(&s_full[s]), 0);
+          if (leader) mbar_expect_tx(smem_u32(&s_full[s]), 2u * stage_bytes);
+          tma_3d_pair(dst, &g.a_map, kb * 64, m0, 0, bar);
+          tma_3d_pair(dst + a_bytes, &g.b_map, kb * 64, nb0, 0, bar);
+          ++c;
+        }
+      }
+      if (!ok) {
+        s_abort = 1;
+        asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_addr(smem_u32(&s_abort), rank ^ 1u)), "r"(1) : "memory");
+        atomicCAS(g.status, 0, TGNN_ETIMEOUT);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (the leader's, for both CTAs)
+    if (lane == 0 && leader) {
+      uint32_t c = 0, n_item = 0;
+      int withheld = 0;
+      bool ok = true;
+      Walk wk = pair_walk(g);
+      Item it;
+      while (ok && next_pair_item(g, wk, it)) {
+        const uint32_t buf = n_item & 1u, use = n_item >> 1;
+        ok = mbar_wait(smem_u32(&s_tmem_empty[buf]), (use & 1u) ^ 1u, limit, abort_flag);   // drained in both CTAs
+        if (!ok) break;
+        ++n_item;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int n_mma = (it.n_valid + 15) / 16 * 16;
+        const uint32_t fmt = g.fp16 ? 0u : 1u;
+        const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(n_mma >> 3) << 17) |
+                               ((uint32_t)((2 * BM) >> 4) << 24);
+        const uint32_t acc = tmem + buf * (uint32_t)ACC_STRIDE;
+        for (int kb = it.kb0; kb < it.kb1 && ok; ++kb) {
+          const uint32_t s = c % n_stages;
+          ok = mbar_wait(smem_u32(&s_full[s]), (c / n_stages) & 1u, limit, abort_flag);
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t a_addr = ring + s * stage_bytes, b_addr = a_addr + a_bytes;
+          const int ks_n = min(4, g.ksteps_total - kb * 4);
+          for (int ks = 0; ks < ks_n; ++ks) {
+            const uint64_t da_hi = make_desc(a_addr + ks * 32u, 16u, 1024u);
+            const uint64_t da_lo = make_desc(a_addr + (a_bytes >> 1) + ks * 32u, 16u, 1024u);
+            const uint64_t db_hi = make_desc(b_addr + ks * 32u, 16u, 1024u);
+            const uint64_t db_lo = make_desc(b_addr + b_plane + ks * 32u, 16u, 1024u);
+            const uint32_t first = (kb > it.kb0 || ks > 0) ? 1u : 0u;
+            mma_f16_pair(acc, da_lo, db_hi, idesc, first);
+            mma_f16_pair(acc, da_hi, db_lo, idesc, 1u);
+            mma_f16_pair(acc, da_hi, db_hi, idesc, 1u);
+          }
+          if (withheld < g.debug_withhold) ++withheld;   // test hook: this stage is never handed back
+          else commit_to_pair(smem_u32(&s_empty[s]));
+          ++c;
+        }
+        if (ok) commit_to_pair(smem_u32(&s_tmem_full[buf]));
+      }
+      if (!ok) {
+        s_abort = 1;
+        asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_addr(smem_u32(&s_abort), 1u)), "r"(1) : "memory");
+        atomicCAS(g.status, 0, TGNN_ETIMEOUT);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------ epilogue (each CTA its own 128 rows)
+    const int e = warp - 2;
+    const int t = e >> 2;
+    const int q4 = warp & 3;
+    float* stg = stg_base + e * (32 * STG_PITCH);
+    const bool c_vec = (((uintptr_t)g.C & 15) == 0) && (g.ldc % 4 == 0);
+    const uint32_t empty0 = peer_addr(smem_u32(&s_tmem_empty[0]), 0), empty1 = peer_addr(smem_u32(&s_tmem_empty[1]), 0);
+    uint32_t n_item = 0;
+    bool ok = true;
+    Walk wk = pair_walk(g);
+    Item it;
+    while (ok && next_pair_item(g, wk, it)) {
+      const uint32_t buf = n_item & 1u, use = n_item >> 1;
+      ok = mbar_wait(smem_u32(&s_tmem_full[buf]), use & 1u, limit, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      ++n_item;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int m0 = (2 * it.mt0 + (int)rank) * BM;
+      const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16) + buf * (uint32_t)ACC_STRIDE;
+      drain_tile(g, it, m0, taddr, 32 * t, 64, stg, lane, q4, c_vec);
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(buf ? empty1 : empty0);
+    }
+    if (!ok && lane == 0) {
+      s_abort = 1;
+      asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_addr(smem_u32(&s_abort), rank ^ 1u)), "r"(1) : "memory");
+      atomicCAS(g.status, 0, TGNN_ETIMEOUT);
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (s_abort && warp == 0) {
+    // copies this CTA asked for may still be on their way into its shared memory: give them a bounded while
+    for (int i = 0; i < 64; ++i) __nanosleep(2000);
+  }
+  __syncthreads();
+  // neither CTA frees tensor memory or leaves while its peer's MMAs, commits or arrivals may still touch it
+  cluster_sync_all();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
   }
 }
 
@@ -585,7 +836,7 @@ int launch_split_rows(tgnn_ctx* ctx, const float* X, int64_t ld_in, int64_t rows
 int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int mn_major, float* C, int64_t ldc, int M, int N,
                       int K, const float* bias, int relu, int accumulate, int split_k, const char* name, cudaStream_t s,
                       int debug_withhold, unsigned spin_limit, int extra_col, float* extra_out, long long* trace, int single,
-                      int launches) {
+                      int launches, int pair) {
   if (M <= 0 || N <= 0) return TGNN_OK;
   if (K <= 0) return set_error(ctx, TGNN_EINVAL, "gemm %s: empty contraction", name);
   if (split_k > 1 && !accumulate) return set_error(ctx, TGNN_EINVAL, "gemm %s: split_k needs accumulate", name);
@@ -644,6 +895,33 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
   const bool maps_ok = mn_major ? (encode_mn_map(&a.a_map, A, 2) && encode_mn_map(&a.b_map, B, a.b_chunks))
                                 : (encode_k_map(&a.a_map, A, BM) && encode_k_map(&a.b_map, B, b_rows));
   if (!maps_ok) return set_error(ctx, TGNN_ECUDA, "gemm %s: tensor map encoding failed", name);
+  // K-major products with more than a handful of row tiles: pairs of CTAs, each loading half of every B tile
+  // (`pair` = 0 / 1 overrides the default).
+  const bool can_pair = !mn_major && a.split_k == 1 && a.extra_col < 0 && M > BM;
+  if (can_pair && (pair > 0 || (pair < 0 && a.m_tiles >= 32))) {
+    const int n_mma = (n_widest + 15) / 16 * 16, bh = n_mma / 2;
+    a.m_tiles = (M + 2 * BM - 1) / (2 * BM);
+    a.stage_bytes = 2 * BM * 128 + 2 * bh * 128;
+    a.n_stages = (SMEM_LIMIT - 1024 - STG_BYTES - 1024) / a.stage_bytes;
+    if (a.n_stages > MAX_SLOTS) a.n_stages = MAX_SLOTS;
+    if (a.n_stages >= 2 && encode_k_map(&a.b_map, B, bh)) {
+      a.kb_begin = 0; a.kb_end = a.kb_total;
+      const int units = a.m_tiles * a.n_tiles;
+      const int clusters = units < 74 ? units : 74;
+      const int smem = 1024 + a.n_stages * a.stage_bytes + STG_BYTES;
+      static SmemLimit pair_limit;
+      const int rc = raise_smem_limit(ctx, gemm_split_pair_kernel, SMEM_LIMIT - 1024, pair_limit);
+      if (rc) return rc;
+      {
+        KernelScope scope__(ctx, name, s);
+        gemm_split_pair_kernel<<<2 * clusters, THREADS, smem, s>>>(a);
+      }
+      TGNN_LAUNCH_OK(ctx, name);
+      return TGNN_OK;
+    }
+    a.m_tiles = (M + BM - 1) / BM;   // (does not fit: the single-CTA kernel below)
+    if (!encode_k_map(&a.b_map, B, b_rows)) return set_error(ctx, TGNN_ECUDA, "gemm %s: tensor map encoding failed", name);
+  }
   const int units = a.m_tiles * a.n_tiles * a.split_k;
   const int items = a.single ? units : (units + 1) / 2;
   const int smem = 1024 + a.n_a_slots * a.a_slot_bytes + a.n_b_slots * a.b_slot_bytes + STG_BYTES;

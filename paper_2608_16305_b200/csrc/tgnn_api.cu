@@ -842,7 +842,8 @@ int tgnn_debug_gemm_split(tgnn_ctx* ctx, const float* A, int64_t a_rs, int64_t a
     trace = reinterpret_cast<long long*>((char*)scratch + ((a_bytes + b_bytes + 256 + 255) / 256 * 256));
   return launch_gemm_split(ctx, a, b, mn, C, ldc, M, N, K, bias, relu, accumulate, split_k < 1 ? 1 : split_k, "debug_gemm_split",
                            S(stream), debug_withhold, spin_limit, -1, nullptr, trace,
-                           getenv("TGNN_GEMM_SINGLE") ? atoi(getenv("TGNN_GEMM_SINGLE")) : -1);
+                           getenv("TGNN_GEMM_SINGLE") ? atoi(getenv("TGNN_GEMM_SINGLE")) : -1, 1,
+                           getenv("TGNN_GEMM_PAIR") ? atoi(getenv("TGNN_GEMM_PAIR")) : -1);
 }
 
 int tgnn_status(tgnn_ctx* ctx, int32_t* status_host, void* stream) {

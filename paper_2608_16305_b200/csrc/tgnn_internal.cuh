@@ -373,7 +373,7 @@ int launch_split_rows(tgnn_ctx* ctx, const float* X, int64_t ld_in, int64_t rows
 int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int mn_major, float* C, int64_t ldc, int M, int N,
                       int K, const float* bias, int relu, int accumulate, int split_k, const char* name, cudaStream_t s,
                       int debug_withhold = 0, unsigned spin_limit = 0, int extra_col = -1, float* extra_out = nullptr, long long* trace = nullptr,
-                      int single = -1, int launches = 1);
+                      int single = -1, int launches = 1, int pair = -1);
 size_t plan_weight_sites(tgnn_ctx* ctx);                       // fills ctx->sites, returns the image bytes needed
 int launch_prep_weights(tgnn_ctx* ctx, cudaStream_t s);        // writes all images from the current parameters
 

@@ -1,8 +1,9 @@
 """The split-operand projection kernel (two 16-bit planes per fp32 operand, three tensor-core passes, fp32
 accumulation) against the plain definition C = A B (+ bias, ReLU, accumulate) computed in fp64 by numpy.
 Two fp16 terms carry 22 mantissa bits (two bf16 terms 16), so the result must sit within 1e-4 of the largest
-|C| whichever planes are used (a single bf16 pass would be off by 4e-3, one TF32 pass by 1e-3).  Also: a
-bounded wait that is made to run out."""
+|C| whichever planes are used (a single bf16 pass would be off by 4e-3, one TF32 pass by 1e-3).  K-major products are run on both
+forms of the kernel: one CTA per row tile, and pairs of CTAs that share each B tile (one 256-row MMA across two
+SMs).  Also: a bounded wait that is made to run out, in either form."""
 import numpy as np
 import pytest
 import torch
@@ -52,9 +53,19 @@ def lib():
     l.close()
 
 
-@pytest.mark.parametrize("shape", SHAPES)
-def test_split_projection_matches_definition(lib, shape):
-    M, N, K, lay = shape
+PAIR_SHAPES = [
+    (300, 200, 386, "k"),        # one 256-row tile and a ragged one whose second half is empty
+    (1800, 200, 372, "k"),       # 8 tiles of 256 rows, the last with 8 valid rows
+    (513, 300, 472, "k"),        # two n-tiles of different widths; the third tile holds one row
+    (40000, 200, 386, "k"),      # 157 tiles over 74 pairs: the persistent walk, accumulators alternating
+    (129, 16, 16, "k"),          # narrowest MMA, one contraction step
+]
+
+
+@pytest.mark.parametrize("shape", SHAPES + [s + ("pair",) for s in PAIR_SHAPES])
+def test_split_projection_matches_definition(lib, shape, monkeypatch):
+    M, N, K, lay = shape[:4]
+    monkeypatch.setenv("TGNN_GEMM_PAIR", "1" if len(shape) > 4 else "0")
     rng = np.random.default_rng(M * 1000003 + N * 1009 + K)
     A, Bm, A_dev, sa, B_dev, sb = _operands(rng, M, N, K, lay)
     ref = A.astype(np.float64) @ Bm.astype(np.float64)
@@ -73,7 +84,8 @@ def test_split_projection_matches_definition(lib, shape):
     ldc = N + 5
     C0 = rng.normal(size=(M, ldc)).astype(np.float32)
     C = torch.from_numpy(C0.copy()).cuda()
-    lib.debug_gemm_split(A_dev, *sa, B_dev, *sb, C, ldc, M, N, K, scr, accumulate=True, split_k=64)
+    lib.debug_gemm_split(A_dev, *sa, B_dev, *sb, C, ldc, M, N, K, scr, accumulate=True,
+                         split_k=1 if len(shape) > 4 else 64)      # (pairs of CTAs do not split the contraction)
     torch.cuda.synchronize()
     assert lib.status() == 0
     got = C.cpu().numpy()
@@ -136,13 +148,17 @@ def test_every_tile_lands_where_the_definition_puts_it(lib):
         assert np.array_equal(C.cpu().numpy(), want), lay
 
 
-def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable(lib):
+@pytest.mark.parametrize("pair", [0, 1])
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable(lib, pair, monkeypatch):
     """The kernel's waits are bounded.  With one shared-memory slot withheld (a debug hook: the MMA warp does
     not hand it back) and a short limit, the copy warp's wait for that slot runs out: the kernel records
     TGNN_ETIMEOUT in the status word, stores nothing, frees its tensor memory and returns.  A normal launch
-    right after it (which needs that tensor memory) gives the right answer."""
+    right after it (which needs that tensor memory) gives the right answer.  In the paired form both CTAs' copy
+    warps run out, each raises the other's abort flag, and the two meet at the cluster barrier before they free
+    tensor memory."""
     from paper_2608_16305_b200 import binding as B
-    M, N, K = 128, 64, 4096                       # one work item, 64 contraction blocks: more than the ring holds
+    monkeypatch.setenv("TGNN_GEMM_PAIR", str(pair))
+    M, N, K = 128 * (1 + pair), 64, 4096          # one work item, 64 contraction blocks: more than the ring holds
     rng = np.random.default_rng(5)
     A, Bm, A_dev, sa, B_dev, sb = _operands(rng, M, N, K, "k")
     scr = _scratch(M, N, K)
