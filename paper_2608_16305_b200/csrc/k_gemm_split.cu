@@ -48,12 +48,16 @@ constexpr int EPI_WARPS = 8;
 constexpr int THREADS = 32 * (2 + EPI_WARPS);
 constexpr int MAX_SLOTS = 8;
 constexpr int STG_PITCH = 20;     // floats between rows of a staged 32 x 16 square (16-byte aligned, bank-staggered)
-constexpr int STG_BYTES = EPI_WARPS * 32 * STG_PITCH * 4;
+constexpr int STG_WARP_BYTES = 4096;   // per epilogue warp: a 32 x 32 fp32 square for a bulk store (or the 32 x 16 square of the plain path)
+constexpr int STG_BYTES = EPI_WARPS * STG_WARP_BYTES;
 constexpr unsigned SPIN_LIMIT = 1u << 22;
 constexpr int SMEM_LIMIT = 227 * 1024;
 
 struct BfArgs {
   CUtensorMap a_map, b_map;   // three-dimensional: (contiguous index, row, plane)
+  CUtensorMap c_map;          // C as (column, row) in boxes of 32 x 32 fp32 values, 128-byte swizzle (valid when c_bulk)
+  int c_bulk;                 // C is 16-byte aligned with a pitch that is a multiple of 16 bytes: the epilogue stores (or
+                              // reduces) whole 32 x 32 squares from shared memory with the tensor-memory-access unit
   float* C; int64_t ldc;
   int M, N, K;
   const float* bias;
@@ -185,6 +189,7 @@ __device__ __forceinline__ void drain_tile(const BfArgs& g, const Item& it, int 
                                            float* stg, int lane, int q4, bool c_vec) {
   const int sub = lane >> 2, ch = lane & 3;
   const bool with_bias = g.bias != nullptr && it.kb0 == 0;   // (the bias goes in with the first contraction block)
+  const bool edge_tile = it.n0 + it.n_valid >= g.N;          // columns past n_valid lie outside C (and are clipped)
   for (int c0 = c_first; c0 < it.n_valid; c0 += c_step) {
     uint32_t r[32];
     asm volatile(
@@ -196,6 +201,49 @@ __device__ __forceinline__ void drain_tile(const BfArgs& g, const Item& it, int 
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr + (uint32_t)c0));
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+    if (g.c_bulk && (edge_tile || c0 + 32 <= it.n_valid)) {
+      // Bulk path: the lane holds 32 consecutive columns of its row; it finishes them (scale, bias, ReLU) and
+      // writes them as one 128-byte row of a swizzled 32 x 32 square, which one bulk tensor store (or fp32
+      // add-reduction) moves to C; rows past M and columns past N are clipped by the tensor map.
+      if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the square is free again
+      __syncwarp();
+      float* row_p = stg + lane * 32;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        float4 v = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]),
+                               __uint_as_float(r[4 * q + 3]));
+        float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (with_bias) {
+          const int col = c0 + 4 * q;
+          const float* bp = g.bias + it.n0 + col;
+          if (col < it.n_valid) b4.x = __ldg(bp);
+          if (col + 1 < it.n_valid) b4.y = __ldg(bp + 1);
+          if (col + 2 < it.n_valid) b4.z = __ldg(bp + 2);
+          if (col + 3 < it.n_valid) b4.w = __ldg(bp + 3);
+        }
+        v.x = fmaf(v.x, g.out_scale, b4.x); v.y = fmaf(v.y, g.out_scale, b4.y);
+        v.z = fmaf(v.z, g.out_scale, b4.z); v.w = fmaf(v.w, g.out_scale, b4.w);
+        if (g.relu && !g.accumulate) { v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); v.z = fmaxf(v.z, 0.f); v.w = fmaxf(v.w, 0.f); }
+        *reinterpret_cast<float4*>(row_p + 4 * (q ^ (lane & 7))) = v;
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) {
+        const int x = it.n0 + c0, y = m0 + q4 * 32;
+        if (g.accumulate)
+          asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+                       ::"l"(&g.c_map), "r"(x), "r"(y), "r"(smem_u32(stg)) : "memory");
+        else
+          asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                       ::"l"(&g.c_map), "r"(x), "r"(y), "r"(smem_u32(stg)) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      }
+      continue;
+    }
+    if (g.c_bulk) {   // the plain path reuses the square: an earlier bulk store must have read it
+      if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      __syncwarp();
+    }
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       const int cb0 = c0 + 16 * h;
@@ -398,7 +446,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_split_kernel(const __grid_con
     const int e = warp - 2;
     const int t = e >> 2;          // which accumulator of the pair
     const int q4 = warp & 3;       // the tensor-memory lane quarter this warp may read
-    float* stg = stg_base + e * (32 * STG_PITCH);
+    float* stg = stg_base + e * (STG_WARP_BYTES / 4);
     const bool c_vec = (((uintptr_t)g.C & 15) == 0) && (g.ldc % 4 == 0);
     uint32_t n_item = 0;
     bool ok = true;
@@ -426,6 +474,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_split_kernel(const __grid_con
       if (e == 0 && lane == 0) TRACE(1 + 2 * (int)n_item);
       if (lane == 0) mbar_arrive(smem_u32(&s_tmem_empty[buf]));
     }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // this warp's bulk stores have landed
     if (!ok && lane == 0) { s_abort = 1; atomicCAS(g.status, 0, TGNN_ETIMEOUT); }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -464,6 +513,13 @@ __device__ __forceinline__ void tma_3d_pair(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%2, %3, %4}], [%5];"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(cluster_bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_4d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                            uint32_t cluster_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.cta_group::2 [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(cluster_bar)
       : "memory");
 }
 __device__ __forceinline__ void mma_f16_pair(uint32_t tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
@@ -549,6 +605,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
   cluster_sync_all();   // the peer's barriers are initialised before anything is counted on them
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = s_tmem;
+  if (tid == 0) TRACE(0);
   volatile int* abort_flag = &s_abort;
   const unsigned limit = g.spin_limit;
   const uint32_t stage_bytes = (uint32_t)g.stage_bytes, n_stages = (uint32_t)g.n_stages;
@@ -577,6 +634,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
           if (leader) mbar_expect_tx(smem_u32(&s_full[s]), 2u * stage_bytes);
           tma_3d_pair(dst, &g.a_map, kb * 64, m0, 0, bar);
           tma_3d_pair(dst + a_bytes, &g.b_map, kb * 64, nb0, 0, bar);
+          TRACE(256 + (int)c);
           ++c;
         }
       }
@@ -611,6 +669,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
           ok = mbar_wait(smem_u32(&s_full[s]), (c / n_stages) & 1u, limit, abort_flag);
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          TRACE(16 + 2 * (int)c);
           const uint32_t a_addr = ring + s * stage_bytes, b_addr = a_addr + a_bytes;
           const int ks_n = min(4, g.ksteps_total - kb * 4);
           for (int ks = 0; ks < ks_n; ++ks) {
@@ -623,6 +682,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
             mma_f16_pair(acc, da_hi, db_lo, idesc, 1u);
             mma_f16_pair(acc, da_hi, db_hi, idesc, 1u);
           }
+          TRACE(17 + 2 * (int)c);
           if (withheld < g.debug_withhold) ++withheld;   // test hook: this stage is never handed back
           else commit_to_pair(smem_u32(&s_empty[s]));
           ++c;
@@ -641,7 +701,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
     const int e = warp - 2;
     const int t = e >> 2;
     const int q4 = warp & 3;
-    float* stg = stg_base + e * (32 * STG_PITCH);
+    float* stg = stg_base + e * (STG_WARP_BYTES / 4);
     const bool c_vec = (((uintptr_t)g.C & 15) == 0) && (g.ldc % 4 == 0);
     const uint32_t empty0 = peer_addr(smem_u32(&s_tmem_empty[0]), 0), empty1 = peer_addr(smem_u32(&s_tmem_empty[1]), 0);
     uint32_t n_item = 0;
@@ -653,6 +713,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
       ok = mbar_wait(smem_u32(&s_tmem_full[buf]), use & 1u, limit, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
+      if (e == 0 && lane == 0) TRACE(2 + 2 * (int)n_item);
       ++n_item;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int m0 = (2 * it.mt0 + (int)rank) * BM;
@@ -660,8 +721,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
       drain_tile(g, it, m0, taddr, 32 * t, 64, stg, lane, q4, c_vec);
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
+      if (e == 0 && lane == 0) TRACE(1 + 2 * (int)n_item);
       if (lane == 0) mbar_arrive_cluster(buf ? empty1 : empty0);
     }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // this warp's bulk stores have landed
     if (!ok && lane == 0) {
       s_abort = 1;
       asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_addr(smem_u32(&s_abort), rank ^ 1u)), "r"(1) : "memory");
@@ -676,6 +739,195 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
   }
   __syncthreads();
   // neither CTA frees tensor memory or leaves while its peer's MMAs, commits or arrivals may still touch it
+  cluster_sync_all();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+  }
+}
+
+// Weight gradients (both operands MN-major, C = A^T B accumulated over a long contraction) on pairs of CTAs.
+// A pair owns a 256-row tile of C -- all of it, up to 512 columns, as two accumulators of 256 columns side by side
+// in each CTA's tensor memory -- and a range of the contraction.  Per block of 32 contraction rows a CTA loads its
+// own 128 columns of A (its rows of C) once, and from B only the 128 columns per accumulator that are its half of
+// the MMA's B tile: every operand byte is fetched by exactly one CTA of the pair, where the single-CTA kernel
+// fetches A once per n-tile.  Barriers and bounded waits as in gemm_split_pair_kernel.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_split_pair_mn_kernel(const __grid_constant__ BfArgs g) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) uint64_t s_full[MAX_SLOTS], s_empty[MAX_SLOTS];
+  __shared__ __align__(8) uint64_t s_tmem_full, s_tmem_empty;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_abort;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_rank();
+  const bool leader = rank == 0;
+  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t ring = smem_u32(smem);
+  float* stg_base = reinterpret_cast<float*>(smem + (size_t)g.n_stages * g.stage_bytes);
+
+  if (tid == 0) {
+    for (int s = 0; s < MAX_SLOTS; ++s) {
+      mbar_init(smem_u32(&s_full[s]), 1);
+      mbar_init(smem_u32(&s_empty[s]), 1);
+    }
+    mbar_init(smem_u32(&s_tmem_full), 1);
+    mbar_init(smem_u32(&s_tmem_empty), 2 * EPI_WARPS);
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync_all();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = s_tmem;
+  if (tid == 0) TRACE(0);
+  volatile int* abort_flag = &s_abort;
+  const unsigned limit = g.spin_limit;
+  const uint32_t stage_bytes = (uint32_t)g.stage_bytes, n_stages = (uint32_t)g.n_stages;
+  constexpr uint32_t TILE = 2u * 2u * 4096u;   // 128 columns x 32 contraction rows, both planes (plane, chunk, row, 64 elements)
+  const int n_sub = g.n_tiles;                  // accumulators (256 columns of C each): 1 or 2
+
+  // the pair's units: (256-row tile of C, part of the contraction), contiguous per pair
+  const int T = g.m_tiles * g.split_k;
+  const int u_begin = (int)((long long)T * (blockIdx.x >> 1) / (gridDim.x >> 1));
+  const int u_end = (int)((long long)T * ((blockIdx.x >> 1) + 1) / (gridDim.x >> 1));
+  const int per = (g.kb_total + g.split_k - 1) / g.split_k;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ tile copies (each CTA its own)
+    if (lane == 0) {
+      uint32_t c = 0;
+      bool ok = true;
+      for (int u = u_begin; u < u_end && ok; ++u) {
+        const int ms = u % g.m_tiles, sp = u / g.m_tiles;
+        const int kb0 = sp * per, kb1 = min(g.kb_total, kb0 + per);
+        const int a_chunk = ms * 4 + (int)rank * 2;
+        for (int kb = kb0; kb < kb1 && ok; ++kb) {
+          const uint32_t s = c % n_stages;
+          ok = mbar_wait(smem_u32(&s_empty[s]), ((c / n_stages) & 1u) ^ 1u, limit, abort_flag);
+          if (!ok) break;
+          const uint32_t dst = ring + s * stage_bytes;
+          const uint32_t bar = peer_addr(smem_u32(&s_full[s]), 0);
+          if (leader) mbar_expect_tx(smem_u32(&s_full[s]), 2u * stage_bytes);
+          tma_4d_pair(dst, &g.a_map, 0, kb * 32, a_chunk, 0, bar);
+          for (int j = 0; j < n_sub; ++j) tma_4d_pair(dst + TILE * (uint32_t)(1 + j), &g.b_map, 0, kb * 32, j * 4 + (int)rank * 2, 0, bar);
+          TRACE(256 + (int)c);
+          ++c;
+        }
+      }
+      if (!ok) {
+        s_abort = 1;
+        asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_addr(smem_u32(&s_abort), rank ^ 1u)), "r"(1) : "memory");
+        atomicCAS(g.status, 0, TGNN_ETIMEOUT);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (the leader's, for both CTAs)
+    if (lane == 0 && leader) {
+      uint32_t c = 0, n_item = 0;
+      int withheld = 0;
+      bool ok = true;
+      const uint32_t fmt = g.fp16 ? 0u : 1u;
+      // D fp32; both operands MN-major; N = 256; M = 256 across the pair
+      const uint32_t idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | (1u << 15) | (1u << 16) | ((256u >> 3) << 17) |
+                             ((uint32_t)((2 * BM) >> 4) << 24);
+      for (int u = u_begin; u < u_end && ok; ++u) {
+        const int sp = u / g.m_tiles;
+        const int kb0 = sp * per, kb1 = min(g.kb_total, kb0 + per);
+        if (kb0 >= kb1) continue;
+        ok = mbar_wait(smem_u32(&s_tmem_empty), (n_item & 1u) ^ 1u, limit, abort_flag);   // drained in both CTAs
+        if (!ok) break;
+        ++n_item;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        for (int kb = kb0; kb < kb1 && ok; ++kb) {
+          const uint32_t s = c % n_stages;
+          ok = mbar_wait(smem_u32(&s_full[s]), (c / n_stages) & 1u, limit, abort_flag);
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          TRACE(16 + 2 * (int)c);
+          const uint32_t a_addr = ring + s * stage_bytes;
+          const int ks_n = min(2, g.ksteps_total - kb * 2);
+          for (int j = 0; j < n_sub; ++j) {
+            const uint32_t b_addr = a_addr + TILE * (uint32_t)(1 + j);
+            const uint32_t acc = tmem + (uint32_t)(j * ACC_STRIDE);
+            for (int ks = 0; ks < ks_n; ++ks) {
+              const uint64_t da_hi = make_desc(a_addr + ks * 2048u, 4096u, 1024u);
+              const uint64_t da_lo = make_desc(a_addr + (TILE >> 1) + ks * 2048u, 4096u, 1024u);
+              const uint64_t db_hi = make_desc(b_addr + ks * 2048u, 4096u, 1024u);
+              const uint64_t db_lo = make_desc(b_addr + (TILE >> 1) + ks * 2048u, 4096u, 1024u);
+              const uint32_t first = (kb > kb0 || ks > 0) ? 1u : 0u;
+              mma_f16_pair(acc, da_lo, db_hi, idesc, first);
+              mma_f16_pair(acc, da_hi, db_lo, idesc, 1u);
+              mma_f16_pair(acc, da_hi, db_hi, idesc, 1u);
+            }
+          }
+          TRACE(17 + 2 * (int)c);
+          if (withheld < g.debug_withhold) ++withheld;   // test hook: this stage is never handed back
+          else commit_to_pair(smem_u32(&s_empty[s]));
+          ++c;
+        }
+        if (ok) commit_to_pair(smem_u32(&s_tmem_full));
+      }
+      if (!ok) {
+        s_abort = 1;
+        asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_addr(smem_u32(&s_abort), 1u)), "r"(1) : "memory");
+        atomicCAS(g.status, 0, TGNN_ETIMEOUT);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------ epilogue (each CTA its own 128 rows)
+    const int e = warp - 2;
+    const int t = e >> 2;          // warps 2-5 drain the first accumulator, 6-9 the second (all eight the only one)
+    const int q4 = warp & 3;
+    float* stg = stg_base + e * (STG_WARP_BYTES / 4);
+    const bool c_vec = (((uintptr_t)g.C & 15) == 0) && (g.ldc % 4 == 0);
+    const uint32_t empty_bar = peer_addr(smem_u32(&s_tmem_empty), 0);
+    uint32_t n_item = 0;
+    bool ok = true;
+    for (int u = u_begin; u < u_end && ok; ++u) {
+      const int ms = u % g.m_tiles, sp = u / g.m_tiles;
+      const int kb0 = sp * per, kb1 = min(g.kb_total, kb0 + per);
+      if (kb0 >= kb1) continue;
+      ok = mbar_wait(smem_u32(&s_tmem_full), n_item & 1u, limit, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      if (e == 0 && lane == 0) TRACE(2 + 2 * (int)n_item);
+      ++n_item;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int m0 = (2 * ms + (int)rank) * BM;
+      const int j = n_sub == 2 ? t : 0;
+      Item it;
+      it.mt0 = ms; it.tiles = 1; it.kb0 = kb0; it.kb1 = kb1;
+      it.n0 = j * 256;
+      it.n_valid = min(256, g.N - it.n0);
+      const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(j * ACC_STRIDE);
+      drain_tile(g, it, m0, taddr, n_sub == 2 ? 0 : 32 * t, n_sub == 2 ? 32 : 64, stg, lane, q4, c_vec);
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (e == 0 && lane == 0) TRACE(1 + 2 * (int)n_item);
+      if (lane == 0) mbar_arrive_cluster(empty_bar);
+    }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // this warp's bulk stores have landed
+    if (!ok && lane == 0) {
+      s_abort = 1;
+      asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_addr(smem_u32(&s_abort), rank ^ 1u)), "r"(1) : "memory");
+      atomicCAS(g.status, 0, TGNN_ETIMEOUT);
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (s_abort && warp == 0) {
+    for (int i = 0; i < 64; ++i) __nanosleep(2000);   // copies still on their way into this CTA's shared memory
+  }
+  __syncthreads();
   cluster_sync_all();
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -798,6 +1050,18 @@ bool encode_mn_map(CUtensorMap* map, const SplitMat& m, int chunks) {
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// C [M, N] fp32 with pitch ldc as (column, row); boxes of 32 x 32 values, 128-byte swizzle in shared memory.
+bool encode_c_map(CUtensorMap* map, float* C, int64_t ldc, int M, int N) {
+  const TensorMapEncodeFn enc = encoder();
+  if (!enc || ((uintptr_t)C & 15) != 0 || ldc % 4 != 0) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)ldc * 4};
+  const cuuint32_t box[2] = {32, 32};
+  const cuuint32_t elem[2] = {1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 int launch_prep_split_weights(tgnn_ctx* ctx, cudaStream_t s) {
@@ -853,6 +1117,7 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
   a.status = ctx->ws.status;
   a.extra_col = (extra_out && accumulate) ? extra_col : -1;
   a.extra_out = extra_out;
+  a.c_bulk = a.extra_col < 0 && encode_c_map(&a.c_map, C, ldc, M, N) ? 1 : 0;
   a.trace = trace;
   a.debug_withhold = debug_withhold;
   a.spin_limit = spin_limit ? spin_limit : SPIN_LIMIT;
@@ -921,6 +1186,37 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
     }
     a.m_tiles = (M + BM - 1) / BM;   // (does not fit: the single-CTA kernel below)
     if (!encode_k_map(&a.b_map, B, b_rows)) return set_error(ctx, TGNN_ECUDA, "gemm %s: tensor map encoding failed", name);
+  }
+  // Weight gradients whose tile of C is more than 128 rows and at most 512 columns: pairs of CTAs, each operand
+  // byte fetched once per pair.
+  if (mn_major && accumulate && split_k > 1 && a.extra_col < 0 && M > BM && N <= 512 && (pair > 0 || pair < 0)) {
+    BfArgs b = a;
+    b.m_tiles = (M + 2 * BM - 1) / (2 * BM);
+    b.n_tiles = (N + 255) / 256;
+    b.bn = 256;
+    b.stage_bytes = 16384 * (1 + b.n_tiles);
+    b.n_stages = (SMEM_LIMIT - 1024 - STG_BYTES - 1024) / b.stage_bytes;
+    if (b.n_stages > MAX_SLOTS) b.n_stages = MAX_SLOTS;
+    int sp = 74 / b.m_tiles;
+    const int max_s = (b.kb_total + 7) / 8;
+    if (sp > max_s) sp = max_s;
+    if (sp > split_k) sp = split_k;
+    b.split_k = sp < 1 ? 1 : sp;
+    b.kb_begin = 0; b.kb_end = b.kb_total;
+    if (b.n_stages >= 2 && encode_mn_map(&b.a_map, A, 2) && encode_mn_map(&b.b_map, B, 2)) {
+      const int units = b.m_tiles * b.split_k;
+      const int clusters = units < 74 ? units : 74;
+      const int smem = 1024 + b.n_stages * b.stage_bytes + STG_BYTES;
+      static SmemLimit pair_mn_limit;
+      const int rc = raise_smem_limit(ctx, gemm_split_pair_mn_kernel, SMEM_LIMIT - 1024, pair_mn_limit);
+      if (rc) return rc;
+      {
+        KernelScope scope__(ctx, name, s);
+        gemm_split_pair_mn_kernel<<<2 * clusters, THREADS, smem, s>>>(b);
+      }
+      TGNN_LAUNCH_OK(ctx, name);
+      return TGNN_OK;
+    }
   }
   const int units = a.m_tiles * a.n_tiles * a.split_k;
   const int items = a.single ? units : (units + 1) / 2;

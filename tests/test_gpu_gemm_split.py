@@ -59,6 +59,10 @@ PAIR_SHAPES = [
     (513, 300, 472, "k"),        # two n-tiles of different widths; the third tile holds one row
     (40000, 200, 386, "k"),      # 157 tiles over 74 pairs: the persistent walk, accumulators alternating
     (129, 16, 16, "k"),          # narrowest MMA, one contraction step
+    (200, 387, 5000, "mn"),      # weight gradient on pairs: two accumulators, 74 parts of the contraction
+    (200, 201, 3000, "mn"),      # one accumulator, drained by all eight epilogue warps
+    (300, 100, 40, "mn"),        # two 256-row tiles of C, contraction of two blocks
+    (256, 512, 777, "mn"),       # the widest C a pair holds; ragged contraction
 ]
 
 
@@ -85,7 +89,7 @@ def test_split_projection_matches_definition(lib, shape, monkeypatch):
     C0 = rng.normal(size=(M, ldc)).astype(np.float32)
     C = torch.from_numpy(C0.copy()).cuda()
     lib.debug_gemm_split(A_dev, *sa, B_dev, *sb, C, ldc, M, N, K, scr, accumulate=True,
-                         split_k=1 if len(shape) > 4 else 64)      # (pairs of CTAs do not split the contraction)
+                         split_k=1 if len(shape) > 4 and lay == "k" else 64)   # (K-major pairs do not split the contraction)
     torch.cuda.synchronize()
     assert lib.status() == 0
     got = C.cpu().numpy()
