@@ -469,8 +469,12 @@ int launch_embed_static(tgnn_ctx* ctx, const double* times, int n, const int32_t
 
 int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n, const int32_t* nbr,
                  const int32_t* eid, const double* ts, const int32_t* cnt, float* h_out, cudaStream_t s) {
-  if (n == 0) return TGNN_OK;
   const tgnn_config& c = ctx->cfg;
+  // tgnn_train_step left work on its side stream; it is waited for where it is first needed
+  const bool pending = ctx->side_pending;
+  ctx->side_pending = false;
+  if (pending && (n == 0 || c.model == TGNN_MODEL_JODIE)) TGNN_CUDA_OK(ctx, cudaStreamWaitEvent(s, ctx->ev_side_done, 0));
+  if (n == 0) return TGNN_OK;
   const ParamLayout& L = ctx->L;
   Workspace& w = ctx->ws;
   const int d = c.d, k = c.k, H = c.heads;
@@ -513,6 +517,12 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
   if (!indirect) {  // the query projection below runs on the side stream and needs the rows just gathered
     rc = fork_to(ctx, s, ctx->side[0]);
     if (rc) return rc;
+  }
+  // the static half of the attention inputs (the side stream's work) is needed from here on: by the key/value
+  // projection and, through the time encoding of the roots, by the query projection on side[0]
+  if (pending) {
+    TGNN_CUDA_OK(ctx, cudaStreamWaitEvent(s, ctx->ev_side_done, 0));
+    TGNN_CUDA_OK(ctx, cudaStreamWaitEvent(ctx->side[0], ctx->ev_side_done, 0));
   }
   GemmArgs g = {};
   g.A = w.Z; g.a_rs = ctx->ld_kv; g.a_cs = 1;

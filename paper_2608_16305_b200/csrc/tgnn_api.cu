@@ -305,6 +305,9 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
       ok = cudaStreamCreateWithPriority(&ctx->side[i], cudaStreamNonBlocking, least) == cudaSuccess;
   }
   for (int i = 0; ok && i < 32; ++i) ok = cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming) == cudaSuccess;
+  ctx->side_pending = false;
+  ok = ok && cudaEventCreateWithFlags(&ctx->ev_search, cudaEventDisableTiming) == cudaSuccess &&
+       cudaEventCreateWithFlags(&ctx->ev_side_done, cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     cudaFree(ctx->images);
@@ -332,6 +335,7 @@ int tgnn_destroy(tgnn_ctx* ctx) {
     if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
   for (int i = 0; i < 2; ++i) cudaStreamDestroy(ctx->side[i]);
   for (int i = 0; i < 32; ++i) cudaEventDestroy(ctx->ev[i]);
+  cudaEventDestroy(ctx->ev_search); cudaEventDestroy(ctx->ev_side_done);
   cudaFree(ctx->images);
   cudaFree(ctx->split_buf);
   cudaFree(ctx->sites_dev);
@@ -504,22 +508,27 @@ int step_body(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q, bool has_mask, flo
   cudaStream_t side = ctx->side[1];
   rc = fork_to(ctx, S(stream), side);
   if (rc) return rc;
-  {  // clear the gradient block off the critical chain (grads | dMemU | red | tg_acc | scalars, contiguous)
-    const size_t zero_bytes = (size_t)((char*)(w.st_scalars + 4) - (char*)w.grads);
-    TGNN_CUDA_OK(ctx, cudaMemsetAsync(w.grads, 0, zero_bytes, side));
-    ctx->grads_zeroed = true;
-  }
   rc = launch_make_roots(ctx, w.st_q_src, w.st_q_dst, w.st_q_neg, w.st_q_t, n_q, side);
   if (rc) return rc;
   NEED(ctx, ctx->cfg.d_e == 0 || ctx->efeat, TGNN_ESTATE, "train_step: tgnn_set_edge_features has not been called");
+  TGNN_CUDA_OK(ctx, cudaEventRecord(ctx->ev_search, side));
   if (ctx->cfg.model == TGNN_MODEL_TGN) {  // the time-projected embedding samples no neighbors
     rc = tgnn_sample_recent(ctx, w.r_node, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, w.nb_cnt, side);
     if (rc) return rc;
+    TGNN_CUDA_OK(ctx, cudaEventRecord(ctx->ev_search, side));
     // edge features and time encodings of the sampled neighbors do not depend on memory either
     rc = launch_embed_static(ctx, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, side);
     if (rc) return rc;
     ctx->z_static_done = true;
   }
+  {  // clear the gradient block off the critical chain (grads | dMemU | red | tg_acc | scalars, contiguous); the
+     // backward pass is its first reader, so it goes behind the gathers, which the embedding waits for
+    const size_t zero_bytes = (size_t)((char*)(w.st_scalars + 4) - (char*)w.grads);
+    TGNN_CUDA_OK(ctx, cudaMemsetAsync(w.grads, 0, zero_bytes, side));
+    ctx->grads_zeroed = true;
+  }
+  TGNN_CUDA_OK(ctx, cudaEventRecord(ctx->ev_side_done, side));
+  ctx->side_pending = true;
   if (n_u > 0) {
     // messages stay virtual: the reduction reads the event arrays, the memory update gathers the winners
     ctx->m_src = w.st_u_src; ctx->m_dst = w.st_u_dst; ctx->m_t = w.st_u_t; ctx->m_eid = w.st_u_eid;
@@ -539,8 +548,9 @@ int step_body(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q, bool has_mask, flo
     if (rc) return rc;
     ctx->images_fresh = true;
   }
-  rc = fork_to(ctx, side, S(stream));  // join
-  if (rc) return rc;
+  // the embedding waits for the side stream's pieces where it first needs each: roots and neighbor lists here, the
+  // static half of its inputs before the key/value projection
+  TGNN_CUDA_OK(ctx, cudaStreamWaitEvent(S(stream), ctx->ev_search, 0));
   rc = tgnn_embed(ctx, w.r_node, w.r_time, 3 * n_q, w.nb_node, w.nb_eid, w.nb_ts, w.nb_cnt, w.h, stream);
   if (rc) return rc;
   return tgnn_backward_step(ctx, n_q, has_mask ? w.st_mask : nullptr, loss_out, gradnorm_out, stream);

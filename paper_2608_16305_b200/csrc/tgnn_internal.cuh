@@ -201,6 +201,11 @@ struct tgnn_ctx {
   // back into the caller's stream with events, so the caller still sees one ordered stream of work.
   cudaStream_t side[2];
   cudaEvent_t ev[32];
+  // tgnn_train_step's side stream, recorded after the neighbor search and after everything else it carries (the static
+  // half of the attention inputs, the clear of the gradient block); the embedding waits for each where it first
+  // needs it (side_pending: recorded and not yet waited for)
+  cudaEvent_t ev_search, ev_side_done;
+  bool side_pending;
   int ev_next;
   // Replay of a whole training step as a CUDA graph: tgnn_train_step copies its inputs into the
   // fixed staging buffers and, for a shape signature it has already run once, captures the launch
