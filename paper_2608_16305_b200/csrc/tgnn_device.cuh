@@ -61,11 +61,14 @@ __device__ __forceinline__ void split_bf16_pair(float x0, float x1, uint32_t* hi
 
 // The same as two fp16 numbers: 22 mantissa bits together for values inside fp16's range (|x| < 65504; below
 // 6e-5 the absolute error is 3e-8).  Used for operands of moderate size; gradients are scaled into range first.
+// (Packed conversions: one instruction rounds both values and leaves them in place, and the way back is an fp16
+// add unit operation; the scalar conversions would queue on the special-function pipe beside the cosines.)
 __device__ __forceinline__ void split_f16_pair(float x0, float x1, uint32_t* hi, uint32_t* lo) {
-  const __half h0 = __float2half_rn(x0), h1 = __float2half_rn(x1);
-  const __half l0 = __float2half_rn(x0 - __half2float(h0)), l1 = __float2half_rn(x1 - __half2float(h1));
-  *hi = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
-  *lo = (uint32_t)__half_as_ushort(l0) | ((uint32_t)__half_as_ushort(l1) << 16);
+  const __half2 h = __floats2half2_rn(x0, x1);             // .x = x0 in the low half
+  const float2 hf = __half22float2(h);
+  const __half2 l = __floats2half2_rn(x0 - hf.x, x1 - hf.y);
+  *hi = *reinterpret_cast<const uint32_t*>(&h);
+  *lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
 __device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + expf(-x)); }
