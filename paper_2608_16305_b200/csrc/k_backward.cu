@@ -916,7 +916,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
   // sequential and stays on the caller's stream s.  Weight-gradient products and time-encoder sums
   // are leaves of that chain: they go to the two side streams as soon as their operands exist and
   // are joined back before the gradient norm.
-  cudaStream_t sa = ctx->side[0], sb = ctx->side[1];
+  cudaStream_t sa = ctx->side[0], sb = ctx->side[1], sc = ctx->side[2];
   // grads | dMemU | red | tg_acc | st_scalars are contiguous in the arena: one memset clears them all
   if (!ctx->grads_zeroed) {
     const size_t zero_bytes = (size_t)((char*)(w.st_scalars + 4) - (char*)w.grads);
@@ -1056,10 +1056,11 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_q");
     cudaStream_t s_tgz = sb;  // where the time-encoder sum over the neighbor rows runs
+    bool join_sc = false;
     if (split) {
       RC(launch_gemm_split(ctx, dkvs, ctx->wz_s, 0, w.dZmp, 2 * d, NB, 2 * d, 2 * d, nullptr, 0, 0, 1, "dZ", s));
       RC(fork_to(ctx, s, sa));
-      RC(fork_to(ctx, s, sb));
+      RC(fork_to(ctx, s, sc));
       // dW_kv = dKV^T Z over the neighbor rows; Z's column of ones yields the bias gradient as the last column.  It
       // starts when dZ has finished and runs beside the rest of the chain (scatter, cell backward, ...).
       SplitMat a = dkvs, b = zs;
@@ -1070,7 +1071,10 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
         fold_dwkv_kernel<<<148, 256, 0, sa>>>(w.dWkv_pad, ctx->ld_wkv, 2 * d, (int)L.dkv, G + L.wk, G + L.bk);
       }
       TGNN_LAUNCH_OK(ctx, "fold_dW_kv");
-      s_tgz = sb;
+      // The time-encoder sum needs little shared memory and fits beside the weight gradient's CTAs; on side stream
+      // b it would queue behind the query-side products, which wait for a whole SM each.
+      s_tgz = sc;
+      join_sc = true;
     } else if (merged_dz) {
       RC(grad_in(ctx, w.dKV, 2 * d, P + L.wk, L.dkv, 0, NB, nullptr, 2 * d, 2 * d, w.dZmp, 2 * d, "dZ", s, SITE_DZ + 1));
       RC(fork_to(ctx, s, sa));
@@ -1126,6 +1130,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     }
     RC(fork_to(ctx, sa, s));  // join
     RC(fork_to(ctx, sb, s));
+    if (join_sc) RC(fork_to(ctx, sc, s));
     }  // attention model
   }
   {

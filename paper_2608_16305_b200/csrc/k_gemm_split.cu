@@ -1197,6 +1197,9 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
     b.stage_bytes = 16384 * (1 + b.n_tiles);
     b.n_stages = (SMEM_LIMIT - 1024 - STG_BYTES - 1024) / b.stage_bytes;
     if (b.n_stages > MAX_SLOTS) b.n_stages = MAX_SLOTS;
+    // three stages feed the MMAs as well as four do, and leave 48 KB of the SM's shared memory to blocks of the
+    // kernels that run beside a weight gradient (gradient scatter, time-encoder sums): measured 11 us per step
+    if (b.n_stages > 3) b.n_stages = 3;
     int sp = 74 / b.m_tiles;
     const int max_s = (b.kb_total + 7) / 8;
     if (sp > max_s) sp = max_s;
