@@ -273,10 +273,8 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
       if (lane == 0) z_dt[r] = dtf;
     }
   }
-  // the Phi(0) half of z_q (fp32: the query projection is not one of the split products); with the first launch
-  if (g_begin == 0)
-  for (int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps)
-    for (int q = lane; q < d; q += 32) Zq[(int64_t)i * 2 * d + d + q] = time_encode(time_w[q], time_b[q], 0.f);
+  // (the Phi(0) half of z_q is written with the roots' memory rows, by gather_z_memory_kernel)
+  (void)Zq;
 }
 
 // Memory part.  Rows [0, n*k): columns [0, d) of Z for the valid slots.  Rows [n*k, n*k + n): the
@@ -288,11 +286,15 @@ __global__ void __launch_bounds__(256) gather_z_memory_kernel(const float* __res
                                                               const int32_t* __restrict__ nbr, int ld,
                                                               float* __restrict__ Z, float* __restrict__ Zq,
                                                               float* __restrict__ cat_o, __nv_bfloat16* __restrict__ z_hi,
-                                                              int64_t plane_s, int ld_s, int64_t N, int32_t* status) {
+                                                              int64_t plane_s, int ld_s, int64_t N, int32_t* status,
+                                                              int part, const float* __restrict__ time_w,
+                                                              const float* __restrict__ time_b) {
+  // part: bit 0 = the neighbor rows, bit 1 = the root rows (with time_w != nullptr also their Phi(0) half of z_q, so
+  // that the query projection depends on this launch alone)
   const int lane = threadIdx.x & 31;
   const int warps = (gridDim.x * blockDim.x) >> 5;
   const int nb_rows = n * k;
-  if (z_hi != nullptr) {
+  if (z_hi != nullptr && (part & 1)) {
     // a warp takes four rows at a time: their slot records, then the four table rows (16 bytes per lane), then the
     // conversions and stores -- four independent round trips in flight per warp instead of a dependent chain per row
     const int d4 = d >> 2;          // <= 64: two 16-byte pieces per lane at most
@@ -331,7 +333,8 @@ __global__ void __launch_bounds__(256) gather_z_memory_kernel(const float* __res
       }
     }
   }
-  for (int r = (z_hi != nullptr ? nb_rows : 0) + ((blockIdx.x * blockDim.x + threadIdx.x) >> 5); r < nb_rows + n; r += warps) {
+  const int r_first = (z_hi != nullptr || !(part & 1)) ? nb_rows : 0, r_last = (part & 2) ? nb_rows + n : nb_rows;
+  for (int r = r_first + ((blockIdx.x * blockDim.x + threadIdx.x) >> 5); r < r_last; r += warps) {
     if (r < nb_rows) {
       const int nb = nbr[r];
       if (nb >= 0 && nb < N) warp_copy_f32(Z + (int64_t)r * ld, memory + (int64_t)nb * d, d, lane);
@@ -344,6 +347,10 @@ __global__ void __launch_bounds__(256) gather_z_memory_kernel(const float* __res
       const float* m = memory + (int64_t)nodes[i] * d;
       warp_copy_f32(Zq + (int64_t)i * 2 * d, m, d, lane);
       warp_copy_f32(cat_o + (int64_t)i * 2 * d + d, m, d, lane);
+    }
+    if (r >= nb_rows && time_w != nullptr) {
+      const int i = r - nb_rows;
+      for (int q = lane; q < d; q += 32) Zq[(int64_t)i * 2 * d + d + q] = time_encode(time_w[q], time_b[q], 0.f);
     }
   }
 }
@@ -507,25 +514,47 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
   const bool indirect = c.math_mode != TGNN_MATH_FP32 && !split;
   int rc = fork_to(ctx, s, ctx->side[0]);
   if (rc) return rc;
-  cudaStream_t sg = indirect ? ctx->side[0] : s;
-  {
-    KernelScope scope__(ctx, "gather_z_memory", sg);
-    // split planes: a grid that fits the machine once (six blocks per SM), rows in groups of four per warp
-    const int gblocks = split ? ((rows + 31) / 32 < 148 * 6 ? (rows + 31) / 32 : 148 * 6) : (rows + 7) / 8;
-    gather_z_memory_kernel<<<gblocks, 256, 0, sg>>>(ctx->memory, d, k, nodes, n, nbr, ctx->ld_kv, w.Z, w.Zq, w.cat_o,
-                                                           split ? reinterpret_cast<__nv_bfloat16*>(ctx->zs.hi) : nullptr,
-                                                           ctx->zs.plane_stride, (int)ctx->zs.ld, c.num_nodes, w.status);
-  }
-  TGNN_LAUNCH_OK(ctx, "gather_z_memory");
-  if (!indirect) {  // the query projection below runs on the side stream and needs the rows just gathered
-    rc = fork_to(ctx, s, ctx->side[0]);
-    if (rc) return rc;
-  }
-  // the static half of the attention inputs (the side stream's work) is needed from here on: by the key/value
-  // projection and, through the time encoding of the roots, by the query projection on side[0]
-  if (pending) {
-    TGNN_CUDA_OK(ctx, cudaStreamWaitEvent(s, ctx->ev_side_done, 0));
-    TGNN_CUDA_OK(ctx, cudaStreamWaitEvent(ctx->side[0], ctx->ev_side_done, 0));
+  if (split) {
+    // root rows (both halves of z_q, the memory half of cat_o) on the side stream, where the query projection
+    // follows them at once; the neighbor rows -- planes the key/value projection reads -- on this one
+    {
+      KernelScope scope__(ctx, "gather_roots", ctx->side[0]);
+      gather_z_memory_kernel<<<(n + 7) / 8, 256, 0, ctx->side[0]>>>(ctx->memory, d, k, nodes, n, nbr, ctx->ld_kv, w.Z, w.Zq, w.cat_o,
+                                                                   reinterpret_cast<__nv_bfloat16*>(ctx->zs.hi), ctx->zs.plane_stride,
+                                                                   (int)ctx->zs.ld, c.num_nodes, w.status, 2,
+                                                                   ctx->params + L.time_w, ctx->params + L.time_b);
+    }
+    TGNN_LAUNCH_OK(ctx, "gather_roots");
+    {
+      KernelScope scope__(ctx, "gather_z_memory", s);
+      // a grid that fits the machine once (six blocks per SM), rows in groups of four per warp
+      const int nbr_rows = n * k;
+      const int gblocks = (nbr_rows + 31) / 32 < 148 * 6 ? (nbr_rows + 31) / 32 : 148 * 6;
+      gather_z_memory_kernel<<<gblocks, 256, 0, s>>>(ctx->memory, d, k, nodes, n, nbr, ctx->ld_kv, w.Z, w.Zq, w.cat_o,
+                                                    reinterpret_cast<__nv_bfloat16*>(ctx->zs.hi), ctx->zs.plane_stride,
+                                                    (int)ctx->zs.ld, c.num_nodes, w.status, 1, nullptr, nullptr);
+    }
+    TGNN_LAUNCH_OK(ctx, "gather_z_memory");
+    // the static half of the attention inputs (the step's side stream) is needed from here on
+    if (pending) TGNN_CUDA_OK(ctx, cudaStreamWaitEvent(s, ctx->ev_side_done, 0));
+  } else {
+    cudaStream_t sg = indirect ? ctx->side[0] : s;
+    {
+      KernelScope scope__(ctx, "gather_z_memory", sg);
+      gather_z_memory_kernel<<<(rows + 7) / 8, 256, 0, sg>>>(ctx->memory, d, k, nodes, n, nbr, ctx->ld_kv, w.Z, w.Zq, w.cat_o, nullptr,
+                                                            0, 0, c.num_nodes, w.status, 3, nullptr, nullptr);
+    }
+    TGNN_LAUNCH_OK(ctx, "gather_z_memory");
+    if (!indirect) {  // the query projection below runs on the side stream and needs the rows just gathered
+      rc = fork_to(ctx, s, ctx->side[0]);
+      if (rc) return rc;
+    }
+    // the static half of the attention inputs (the step's side stream) is needed from here on: by the key/value
+    // projection and, through the time encoding of the roots, by the query projection on side[0]
+    if (pending) {
+      TGNN_CUDA_OK(ctx, cudaStreamWaitEvent(s, ctx->ev_side_done, 0));
+      TGNN_CUDA_OK(ctx, cudaStreamWaitEvent(ctx->side[0], ctx->ev_side_done, 0));
+    }
   }
   GemmArgs g = {};
   g.A = w.Z; g.a_rs = ctx->ld_kv; g.a_cs = 1;
