@@ -71,7 +71,9 @@ enum {
                              numbers (hi + lo, 22 mantissa bits; gradients are scaled by a power of two into fp16's
                              range) and run as three fp16 tensor-core passes with fp32 accumulation: the accuracy of
                              the TF32 split at half its tensor time.  Edge features and memory values must stay below
-                             fp16's largest number (65504) in magnitude */
+                             fp16's largest number (65504) in magnitude.  With a bf16 edge-feature table (tolerance
+                             1e-2) the weight gradient of the key/value projection, a leaf of the backward pass, reads
+                             only the hi numbers (one pass) */
   TGNN_MATH_TF32_FAST = 2 /* tcgen05 tensor cores, single TF32 pass in the forward projections (the gradient
                              products keep the split).  Outputs stay within 2e-3, but gradient tensors whose
                              terms cancel (time encoder, W_k) can be off by ~1e-2 of their largest entry. */
@@ -338,7 +340,8 @@ TGNN_API int64_t tgnn_kernel_launches(const tgnn_ctx* ctx);
  * only: TGNN_GEMM_PAIR=0|1 forces the one-CTA-per-tile form or the CTA-pair form (one 256-row MMA across two SMs,
  * each loading half of the B tile; default: pairs for K-major products of 32 row tiles and more),
  * TGNN_GEMM_SINGLE=0|1 the walk by pairs of row tiles or by single tiles, TGNN_GEMM_BF16=1 bf16 planes,
- * TGNN_GEMM_SCALE=s a scale of 2^s on A. */
+ * TGNN_GEMM_SCALE=s a scale of 2^s on A, TGNN_GEMM_PASSES=1 only the hi planes (one pass, 11-bit operands: the
+ * form the step uses for the key/value weight gradient when the feature table is bf16). */
 TGNN_API int tgnn_debug_gemm_split(tgnn_ctx* ctx, const float* A, int64_t a_rs, int64_t a_cs, const float* B, int64_t b_rs,
                                    int64_t b_cs, float* C, int64_t ldc, int M, int N, int K, const float* bias, int relu,
                                    int accumulate, int split_k, void* scratch, int64_t scratch_bytes, int debug_withhold,

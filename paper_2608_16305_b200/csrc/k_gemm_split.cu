@@ -64,6 +64,7 @@ struct BfArgs {
   int relu, accumulate;
   int mn_major;               // 0: both operands K-major; 1: both MN-major
   int fp16;                   // both operands' planes hold fp16 numbers (bf16 otherwise; the two may not be mixed)
+  int planes;                 // 2: hi and lo planes, three passes per product; 1: only the hi planes are read, one pass
   float out_scale;            // the product is multiplied by this (undoes the operands' power-of-two scales)
   int single;                 // work items are single row tiles whose accumulators alternate between the two halves of
                               // tensor memory, so that the epilogue of one overlaps the MMAs of the next (B tiles are
@@ -385,7 +386,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_split_kernel(const __grid_con
       int withheld = 0;
       bool ok = true;
       const uint32_t a_bytes = (uint32_t)g.a_slot_bytes, b_bytes = (uint32_t)g.b_slot_bytes;
-      const uint32_t a_plane = a_bytes >> 1, b_plane = b_bytes >> 1;
+      const uint32_t a_plane = a_bytes / (uint32_t)g.planes, b_plane = b_bytes / (uint32_t)g.planes;
+      const bool three = g.planes == 2;
       const uint32_t mn = g.mn_major ? 1u : 0u;
       // K-major: 8-row groups 1024 B apart (SBO), a step advances 32 B.  MN-major: 64-column chunks 4096 B apart
       // (LBO), 8-row contraction groups 1024 B apart (SBO), a step advances two groups.
@@ -424,9 +426,11 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_split_kernel(const __grid_con
               const uint64_t db_hi = make_desc(b_addr + ks * kstep_bytes, lbo, sbo);
               const uint64_t db_lo = make_desc(b_addr + b_plane + ks * kstep_bytes, lbo, sbo);
               const uint32_t first = (kb > it.kb0 || ks > 0) ? 1u : 0u;
-              mma_f16(acc, da_lo, db_hi, idesc, first);
-              mma_f16(acc, da_hi, db_lo, idesc, 1u);
-              mma_f16(acc, da_hi, db_hi, idesc, 1u);
+              if (three) {
+                mma_f16(acc, da_lo, db_hi, idesc, first);
+                mma_f16(acc, da_hi, db_lo, idesc, 1u);
+              }
+              mma_f16(acc, da_hi, db_hi, idesc, three ? 1u : first);
             }
             TRACE(17 + 2 * (int)ca);
             if (withheld < g.debug_withhold) ++withheld;   // test hook: this slot is never handed back
@@ -609,8 +613,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
   volatile int* abort_flag = &s_abort;
   const unsigned limit = g.spin_limit;
   const uint32_t stage_bytes = (uint32_t)g.stage_bytes, n_stages = (uint32_t)g.n_stages;
-  const uint32_t a_bytes = 2u * BM * 128u;                 // both planes of the A tile
-  const uint32_t b_plane = (stage_bytes - a_bytes) >> 1;   // one plane of this CTA's half of the B tile
+  const uint32_t planes = (uint32_t)g.planes;
+  const uint32_t a_bytes = planes * BM * 128u;                  // the A tile (all its planes)
+  const uint32_t b_plane = (stage_bytes - a_bytes) / planes;    // one plane of this CTA's half of the B tile
   const int b_rows = (int)(b_plane >> 7);                  // rows of the copied half (the widest n-tile's)
 
   if (warp == 0) {
@@ -674,13 +679,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
           const int ks_n = min(4, g.ksteps_total - kb * 4);
           for (int ks = 0; ks < ks_n; ++ks) {
             const uint64_t da_hi = make_desc(a_addr + ks * 32u, 16u, 1024u);
-            const uint64_t da_lo = make_desc(a_addr + (a_bytes >> 1) + ks * 32u, 16u, 1024u);
+            const uint64_t da_lo = make_desc(a_addr + BM * 128u + ks * 32u, 16u, 1024u);
             const uint64_t db_hi = make_desc(b_addr + ks * 32u, 16u, 1024u);
             const uint64_t db_lo = make_desc(b_addr + b_plane + ks * 32u, 16u, 1024u);
             const uint32_t first = (kb > it.kb0 || ks > 0) ? 1u : 0u;
-            mma_f16_pair(acc, da_lo, db_hi, idesc, first);
-            mma_f16_pair(acc, da_hi, db_lo, idesc, 1u);
-            mma_f16_pair(acc, da_hi, db_hi, idesc, 1u);
+            if (planes == 2u) {
+              mma_f16_pair(acc, da_lo, db_hi, idesc, first);
+              mma_f16_pair(acc, da_hi, db_lo, idesc, 1u);
+            }
+            mma_f16_pair(acc, da_hi, db_hi, idesc, planes == 2u ? 1u : first);
           }
           TRACE(17 + 2 * (int)c);
           if (withheld < g.debug_withhold) ++withheld;   // test hook: this stage is never handed back
@@ -790,7 +797,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
   volatile int* abort_flag = &s_abort;
   const unsigned limit = g.spin_limit;
   const uint32_t stage_bytes = (uint32_t)g.stage_bytes, n_stages = (uint32_t)g.n_stages;
-  constexpr uint32_t TILE = 2u * 2u * 4096u;   // 128 columns x 32 contraction rows, both planes (plane, chunk, row, 64 elements)
+  const uint32_t PLANE = 2u * 4096u;                 // one plane of an operand tile: 128 columns x 32 contraction rows
+  const uint32_t TILE = (uint32_t)g.planes * PLANE;  // (plane, chunk, row, 64 elements)
   const int n_sub = g.n_tiles;                  // accumulators (256 columns of C each): 1 or 2
 
   // the pair's units: (256-row tile of C, part of the contraction), contiguous per pair
@@ -859,13 +867,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
             const uint32_t acc = tmem + (uint32_t)(j * ACC_STRIDE);
             for (int ks = 0; ks < ks_n; ++ks) {
               const uint64_t da_hi = make_desc(a_addr + ks * 2048u, 4096u, 1024u);
-              const uint64_t da_lo = make_desc(a_addr + (TILE >> 1) + ks * 2048u, 4096u, 1024u);
+              const uint64_t da_lo = make_desc(a_addr + PLANE + ks * 2048u, 4096u, 1024u);
               const uint64_t db_hi = make_desc(b_addr + ks * 2048u, 4096u, 1024u);
-              const uint64_t db_lo = make_desc(b_addr + (TILE >> 1) + ks * 2048u, 4096u, 1024u);
+              const uint64_t db_lo = make_desc(b_addr + PLANE + ks * 2048u, 4096u, 1024u);
               const uint32_t first = (kb > kb0 || ks > 0) ? 1u : 0u;
-              mma_f16_pair(acc, da_lo, db_hi, idesc, first);
-              mma_f16_pair(acc, da_hi, db_lo, idesc, 1u);
-              mma_f16_pair(acc, da_hi, db_hi, idesc, 1u);
+              if (g.planes == 2) {
+                mma_f16_pair(acc, da_lo, db_hi, idesc, first);
+                mma_f16_pair(acc, da_hi, db_lo, idesc, 1u);
+              }
+              mma_f16_pair(acc, da_hi, db_hi, idesc, g.planes == 2 ? 1u : first);
             }
           }
           TRACE(17 + 2 * (int)c);
@@ -940,7 +950,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
 __global__ void __launch_bounds__(256) split_rows_kernel(const float* __restrict__ X, int64_t ld_in, int64_t rows, int cols,
                                                          const int32_t* __restrict__ dev_rows, __nv_bfloat16* __restrict__ hi,
                                                          __nv_bfloat16* __restrict__ lo, int64_t ld_out, int ones_col,
-                                                         int fp16, float scale) {
+                                                         int fp16, float scale, int planes) {
   const int per_row = (int)(ld_out >> 2);
   const int64_t n_rows = dev_rows ? min((int64_t)*dev_rows, rows) : rows;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < rows * per_row; i += (int64_t)gridDim.x * blockDim.x) {
@@ -966,7 +976,7 @@ __global__ void __launch_bounds__(256) split_rows_kernel(const float* __restrict
       }
     }
     *reinterpret_cast<uint2*>(hi + r * ld_out + c) = *reinterpret_cast<const uint2*>(h);
-    *reinterpret_cast<uint2*>(lo + r * ld_out + c) = *reinterpret_cast<const uint2*>(l);
+    if (planes == 2) *reinterpret_cast<uint2*>(lo + r * ld_out + c) = *reinterpret_cast<const uint2*>(l);
   }
 }
 
@@ -977,7 +987,8 @@ __global__ void __launch_bounds__(256) split_rows_kernel(const float* __restrict
 // Padding columns of the planes are zero.  Both planes hold fp16 numbers.
 __global__ void __launch_bounds__(256) prep_split_weights_kernel(const float* __restrict__ Wkv, int d, int de,
                                                                  __nv_bfloat16* __restrict__ wkv_hi, int64_t wkv_plane, int ld_kv,
-                                                                 __nv_bfloat16* __restrict__ wz_hi, int64_t wz_plane, int ld_z) {
+                                                                 __nv_bfloat16* __restrict__ wz_hi, int64_t wz_plane, int ld_z,
+                                                                 int planes) {
   const int dkv = 2 * d + de, n_rows = 2 * d;
   const int64_t n_kv = (int64_t)n_rows * ld_kv, n_z = (int64_t)n_rows * ld_z;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n_kv + n_z; i += (int64_t)gridDim.x * blockDim.x) {
@@ -995,7 +1006,7 @@ __global__ void __launch_bounds__(256) prep_split_weights_kernel(const float* __
     }
     const __half h = __float2half_rn(v);   // weights: two fp16 numbers
     *reinterpret_cast<__half*>(hi) = h;
-    *reinterpret_cast<__half*>(lo) = __float2half_rn(v - __half2float(h));
+    if (planes == 2) *reinterpret_cast<__half*>(lo) = __float2half_rn(v - __half2float(h));
   }
 }
 
@@ -1021,11 +1032,11 @@ TensorMapEncodeFn encoder() {
 // 128-byte swizzle, zeros outside [0, cols) x [0, rows).
 bool encode_k_map(CUtensorMap* map, const SplitMat& m, int box_rows) {
   const TensorMapEncodeFn enc = encoder();
-  if (!enc || m.rows <= 0 || m.cols <= 0 || box_rows < 1 || box_rows > 256) return false;
+  if (!enc || m.rows <= 0 || m.cols <= 0 || box_rows < 1 || box_rows > 256 || m.planes < 1 || m.planes > 2) return false;
   if (((uintptr_t)m.hi & 15) != 0 || m.ld % 8 != 0 || m.plane_stride % 8 != 0) return false;
-  const cuuint64_t dims[3] = {(cuuint64_t)m.cols, (cuuint64_t)m.rows, 2};
+  const cuuint64_t dims[3] = {(cuuint64_t)m.cols, (cuuint64_t)m.rows, (cuuint64_t)m.planes};
   const cuuint64_t strides[2] = {(cuuint64_t)m.ld * 2, (cuuint64_t)m.plane_stride * 2};
-  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)m.planes};
   const cuuint32_t elem[3] = {1, 1, 1};
   return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, m.hi, dims, strides, box, elem,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -1039,11 +1050,11 @@ bool encode_k_map(CUtensorMap* map, const SplitMat& m, int box_rows) {
 // that are never stored, and the buffers end in slack.
 bool encode_mn_map(CUtensorMap* map, const SplitMat& m, int chunks) {
   const TensorMapEncodeFn enc = encoder();
-  if (!enc || m.rows <= 0 || m.cols <= 0 || chunks < 1 || chunks > 4) return false;
+  if (!enc || m.rows <= 0 || m.cols <= 0 || chunks < 1 || chunks > 4 || m.planes < 1 || m.planes > 2) return false;
   if (((uintptr_t)m.hi & 15) != 0 || m.ld % 8 != 0 || m.plane_stride % 8 != 0) return false;
-  const cuuint64_t dims[4] = {64, (cuuint64_t)m.rows, (cuuint64_t)((m.cols + 63) / 64), 2};
+  const cuuint64_t dims[4] = {64, (cuuint64_t)m.rows, (cuuint64_t)((m.cols + 63) / 64), (cuuint64_t)m.planes};
   const cuuint64_t strides[3] = {(cuuint64_t)m.ld * 2, 128, (cuuint64_t)m.plane_stride * 2};
-  const cuuint32_t box[4] = {64, 32, (cuuint32_t)chunks, 2};
+  const cuuint32_t box[4] = {64, 32, (cuuint32_t)chunks, (cuuint32_t)m.planes};
   const cuuint32_t elem[4] = {1, 1, 1, 1};
   return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, m.hi, dims, strides, box, elem,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -1072,7 +1083,7 @@ int launch_prep_split_weights(tgnn_ctx* ctx, cudaStream_t s) {
     prep_split_weights_kernel<<<148, 256, 0, s>>>(ctx->params + ctx->L.wk, d, de, reinterpret_cast<__nv_bfloat16*>(ctx->wkv_s.hi),
                                                   ctx->wkv_s.plane_stride, (int)ctx->wkv_s.ld,
                                                   reinterpret_cast<__nv_bfloat16*>(ctx->wz_s.hi), ctx->wz_s.plane_stride,
-                                                  (int)ctx->wz_s.ld);
+                                                  (int)ctx->wz_s.ld, ctx->wkv_s.planes);
   }
   TGNN_LAUNCH_OK(ctx, "prep_split_weights");
   return TGNN_OK;
@@ -1087,7 +1098,7 @@ int launch_split_rows(tgnn_ctx* ctx, const float* X, int64_t ld_in, int64_t rows
     KernelScope scope__(ctx, name, s);
     split_rows_kernel<<<blocks, 256, 0, s>>>(X, ld_in, rows, cols, dev_rows, reinterpret_cast<__nv_bfloat16*>(out.hi),
                                              reinterpret_cast<__nv_bfloat16*>(out.hi) + out.plane_stride, out.ld, ones_col,
-                                             out.fp16, out.scale);
+                                             out.fp16, out.scale, out.planes);
   }
   TGNN_LAUNCH_OK(ctx, name);
   return TGNN_OK;
@@ -1110,6 +1121,9 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
   if ((A.fp16 != 0) != (B.fp16 != 0))
     return set_error(ctx, TGNN_EINVAL, "gemm %s: one operand is held as fp16 planes and the other as bf16 planes", name);
   a.fp16 = A.fp16 ? 1 : 0;
+  if (A.planes != B.planes) return set_error(ctx, TGNN_EINVAL, "gemm %s: the operands differ in their number of planes", name);
+  a.planes = A.planes == 1 ? 1 : 2;
+  const int planes = a.planes;
   a.out_scale = 1.f / (A.scale * B.scale);
   // single row tiles with alternating accumulators for the activation x weight products (their epilogue, a full
   // store of C, then overlaps the next tile's MMAs); pairs for the weight gradients (one item per CTA, B shared)
@@ -1140,8 +1154,8 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
   a.kb_total = (K + bke - 1) / bke;
   a.ksteps_total = (K + 15) / 16;
   a.b_chunks = (n_widest + 63) / 64;
-  a.a_slot_bytes = mn_major ? 2 * 2 * 4096 : 2 * BM * 128;
-  a.b_slot_bytes = mn_major ? 2 * a.b_chunks * 4096 : 2 * b_rows * 128;
+  a.a_slot_bytes = mn_major ? planes * 2 * 4096 : planes * BM * 128;
+  a.b_slot_bytes = mn_major ? planes * a.b_chunks * 4096 : planes * b_rows * 128;
   const int budget = SMEM_LIMIT - 1024 - STG_BYTES - 1024;
   a.n_b_slots = a.b_slot_bytes > 40 * 1024 ? 2 : (a.b_slot_bytes > 20 * 1024 ? 3 : 4);
   a.n_a_slots = (budget - a.n_b_slots * a.b_slot_bytes) / a.a_slot_bytes;
@@ -1166,7 +1180,7 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
   if (can_pair && (pair > 0 || (pair < 0 && a.m_tiles >= 32))) {
     const int n_mma = (n_widest + 15) / 16 * 16, bh = n_mma / 2;
     a.m_tiles = (M + 2 * BM - 1) / (2 * BM);
-    a.stage_bytes = 2 * BM * 128 + 2 * bh * 128;
+    a.stage_bytes = planes * (BM * 128 + bh * 128);
     a.n_stages = (SMEM_LIMIT - 1024 - STG_BYTES - 1024) / a.stage_bytes;
     if (a.n_stages > MAX_SLOTS) a.n_stages = MAX_SLOTS;
     if (a.n_stages >= 2 && encode_k_map(&a.b_map, B, bh)) {
@@ -1194,12 +1208,12 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
     b.m_tiles = (M + 2 * BM - 1) / (2 * BM);
     b.n_tiles = (N + 255) / 256;
     b.bn = 256;
-    b.stage_bytes = 16384 * (1 + b.n_tiles);
+    b.stage_bytes = planes * 8192 * (1 + b.n_tiles);
     b.n_stages = (SMEM_LIMIT - 1024 - STG_BYTES - 1024) / b.stage_bytes;
     if (b.n_stages > MAX_SLOTS) b.n_stages = MAX_SLOTS;
     // three stages feed the MMAs as well as four do, and leave 48 KB of the SM's shared memory to blocks of the
     // kernels that run beside a weight gradient (gradient scatter, time-encoder sums): measured 11 us per step
-    if (b.n_stages > 3) b.n_stages = 3;
+    if (b.n_stages > 6 / planes) b.n_stages = 6 / planes;   // (144 KB of stages in either form)
     int sp = 74 / b.m_tiles;
     const int max_s = (b.kb_total + 7) / 8;
     if (sp > max_s) sp = max_s;

@@ -273,22 +273,23 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
     const int64_t d = cfg->d, dkv = ctx->L.dkv, NB = ctx->NB_cap;
     // every operand as two fp16 numbers (22 mantissa bits); the gradient rows, whose entries are far below fp16's
     // normal range, multiplied by 2^12 first (the products divide it out again)
-    ctx->zs = SplitMat{nullptr, up8(dkv + 1), 0, NB, dkv + 1, 1, 1.f};
-    ctx->dkvs = SplitMat{nullptr, up8(2 * d), 0, NB, 2 * d, 1, 4096.f};
-    ctx->wkv_s = SplitMat{nullptr, up8(dkv), 0, 2 * d, dkv, 1, 1.f};
-    ctx->wz_s = SplitMat{nullptr, up8(2 * d), 0, 2 * d, 2 * d, 1, 1.f};
+    const int planes = 2;   // hi and lo (a product that can do with one pass reads the hi planes alone)
+    ctx->zs = SplitMat{nullptr, up8(dkv + 1), 0, NB, dkv + 1, 1, 1.f, planes};
+    ctx->dkvs = SplitMat{nullptr, up8(2 * d), 0, NB, 2 * d, 1, 4096.f, planes};
+    ctx->wkv_s = SplitMat{nullptr, up8(dkv), 0, 2 * d, dkv, 1, 1.f, planes};
+    ctx->wz_s = SplitMat{nullptr, up8(2 * d), 0, 2 * d, 2 * d, 1, 1.f, planes};
     SplitMat* ms[4] = {&ctx->zs, &ctx->dkvs, &ctx->wkv_s, &ctx->wz_s};
     size_t off = 0;
     for (SplitMat* m : ms) {
       m->plane_stride = (m->rows * m->ld + 127) / 128 * 128;
-      off += (size_t)(2 * m->plane_stride * 2);
+      off += (size_t)(planes * m->plane_stride * 2);
     }
     off += 256;   // a chunked tile copy may read up to 126 bytes past the last plane (values that reach no stored output)
     ok = cudaMalloc(&ctx->split_buf, off) == cudaSuccess && cudaMemset(ctx->split_buf, 0, off) == cudaSuccess;
     off = 0;
     for (SplitMat* m : ms) {
       m->hi = (char*)ctx->split_buf + off;
-      off += (size_t)(2 * m->plane_stride * 2);
+      off += (size_t)(planes * m->plane_stride * 2);
     }
   }
   ctx->ev_next = 0;
@@ -832,7 +833,9 @@ int tgnn_debug_gemm_split(tgnn_ctx* ctx, const float* A, int64_t a_rs, int64_t a
   // TGNN_GEMM_BF16=1 (debugging aid): bf16 planes instead of fp16 planes; TGNN_GEMM_SCALE=s: A is scaled by 2^s
   const int f16 = getenv("TGNN_GEMM_BF16") && atoi(getenv("TGNN_GEMM_BF16")) ? 0 : 1;
   const float sc = getenv("TGNN_GEMM_SCALE") ? ldexpf(1.f, atoi(getenv("TGNN_GEMM_SCALE"))) : 1.f;
-  SplitMat a{nullptr, up8(a_cols), 0, a_rows, a_cols, f16, sc}, b{nullptr, up8(b_cols), 0, b_rows, b_cols, f16, 1.f};
+  // TGNN_GEMM_PASSES=1 (debugging aid): hi planes only, one pass
+  const int planes = getenv("TGNN_GEMM_PASSES") && atoi(getenv("TGNN_GEMM_PASSES")) == 1 ? 1 : 2;
+  SplitMat a{nullptr, up8(a_cols), 0, a_rows, a_cols, f16, sc, planes}, b{nullptr, up8(b_cols), 0, b_rows, b_cols, f16, 1.f, planes};
   a.plane_stride = a.rows * a.ld;
   b.plane_stride = b.rows * b.ld;
   const int64_t a_bytes = (2 * a.plane_stride * 2 + 255) / 256 * 256, b_bytes = 2 * b.plane_stride * 2;

@@ -130,6 +130,7 @@ struct SplitMat {
   int64_t rows, cols;
   int fp16;
   float scale;
+  int planes;   // 2: hi and lo planes (three passes per product); 1: only the hi plane is read (one pass, 11-bit operands)
 };
 
 }  // namespace tgnn

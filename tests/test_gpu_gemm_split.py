@@ -131,6 +131,36 @@ def test_fp16_planes_beat_bf16_planes_and_scaling_keeps_gradients_in_range(lib, 
     assert errs["12"] < errs["0"], errs          # unscaled, the small entries lose their remainder plane
 
 
+@pytest.mark.parametrize("shape", [(300, 200, 386, "k"), (1800, 200, 372, "k"), (40000, 200, 386, "k"), (513, 300, 472, "k"),
+                                   (200, 387, 5000, "mn"), (100, 200, 777, "mn"), (256, 512, 777, "mn")])
+def test_single_pass_products_hold_fp16_accuracy(lib, shape, monkeypatch):
+    """One plane per operand (the hi numbers only) and one tensor-core pass: the form TGNN_MATH_F16X1 uses.  Eleven
+    mantissa bits per operand: the product of random operands stays within 1e-3 of the largest |C| (three passes:
+    1e-4), through every kernel form the launcher picks for the shape."""
+    M, N, K, lay = shape
+    monkeypatch.setenv("TGNN_GEMM_PASSES", "1")
+    monkeypatch.delenv("TGNN_GEMM_PAIR", raising=False)
+    rng = np.random.default_rng(M + 7 * N + 13 * K)
+    A, Bm, A_dev, sa, B_dev, sb = _operands(rng, M, N, K, lay)
+    ref = A.astype(np.float64) @ Bm.astype(np.float64)
+    scr = _scratch(M, N, K)
+    bias = rng.normal(size=N).astype(np.float32)
+    C = torch.full((M, N), 7.0, dtype=torch.float32, device="cuda")
+    lib.debug_gemm_split(A_dev, *sa, B_dev, *sb, C, N, M, N, K, scr, bias=torch.from_numpy(bias).cuda())
+    torch.cuda.synchronize()
+    assert lib.status() == 0
+    err = np.abs(C.cpu().numpy() - (ref + bias)).max() / np.abs(ref).max()
+    assert 1e-6 < err <= 1e-3, err          # (far above the three-pass error: the lo planes really are not used)
+    ldc = (N + 3) // 4 * 4
+    C0 = rng.normal(size=(M, ldc)).astype(np.float32)
+    C = torch.from_numpy(C0.copy()).cuda()
+    lib.debug_gemm_split(A_dev, *sa, B_dev, *sb, C, ldc, M, N, K, scr, accumulate=True, split_k=64 if lay == "mn" else 1)
+    torch.cuda.synchronize()
+    assert lib.status() == 0
+    err = np.abs(C.cpu().numpy()[:, :N] - (C0[:, :N] + ref)).max() / np.abs(ref).max()
+    assert err <= 1e-3, err
+
+
 def test_every_tile_lands_where_the_definition_puts_it(lib):
     """Index-valued operands: A picks row m of B scaled by a small integer, so every C entry names the (row
     tile, n-tile, column) it came from exactly (all values are small integers, exact in bf16)."""
