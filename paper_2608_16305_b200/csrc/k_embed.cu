@@ -458,10 +458,11 @@ int launch_embed_static(tgnn_ctx* ctx, const double* times, int n, const int32_t
       const int per = groups >= 32768 ? (groups + 2) / 3 : groups;   // (small batches: one launch)
       for (int g0 = 0; g0 < groups; g0 += per) {
         const int g1 = g0 + per < groups ? g0 + per : groups;
-        // a resident grid (three blocks per SM) whose warps walk the groups: the encoder's frequencies and phases are
-        // loaded once per warp, not once per pair of rows
+        // a grid of four waves (three blocks per SM at a time) whose warps walk the groups: the encoder's frequencies
+        // and phases are loaded once per warp for several pairs of rows, and blocks still end often enough for the
+        // kernels of the chain (higher priority) to find room between them
         const int want = (g1 - g0 + 7) / 8 + 1;
-        gather_z_static_split_kernel<<<want < 148 * 3 ? want : 148 * 3, 256, 0, s>>>(
+        gather_z_static_split_kernel<<<want < 148 * 12 ? want : 148 * 12, 256, 0, s>>>(
             ctx->efeat, c.feat_dtype == TGNN_BF16, ctx->params + L.time_w, ctx->params + L.time_b, c.d, c.d_e, c.k, times, n,
             nbr, eid, ts, (int)ctx->zs.ld, reinterpret_cast<__nv_bfloat16*>(ctx->zs.hi), ctx->zs.plane_stride, w.z_dt, w.Zq,
             c.num_nodes, ctx->num_events, w.status, g0, g1);
