@@ -526,8 +526,8 @@ __global__ void __launch_bounds__(256) scatter_dmem_cached_kernel(const float* _
 constexpr int TG_MAXJ = 8;
 // Rows per block: every block ends with one fp64 atomic per column onto the same 2d addresses, and those
 // serialise, so the grid is kept to about two blocks per SM, as many as fit at once (rows per block a multiple
-// of the 8 warps); inside a block each warp walks its rows two at a time so that their loads overlap.
-constexpr int TG_U = 2;   // rows a warp has in flight (more would cost the registers that let two blocks share an SM)
+// of the 8 warps); inside a block each warp walks its rows three at a time so that their loads overlap.
+constexpr int TG_U = 3;   // rows a warp has in flight (four spill at the 128 registers that let two blocks share an SM)
 inline int tg_rows_per_block(int rows) {
   const int r = (rows + 295) / 296;
   return r < 8 ? 8 : (r + 7) / 8 * 8;
