@@ -134,7 +134,8 @@ def test_fp16_planes_beat_bf16_planes_and_scaling_keeps_gradients_in_range(lib, 
 @pytest.mark.parametrize("shape", [(300, 200, 386, "k"), (1800, 200, 372, "k"), (40000, 200, 386, "k"), (513, 300, 472, "k"),
                                    (200, 387, 5000, "mn"), (100, 200, 777, "mn"), (256, 512, 777, "mn")])
 def test_single_pass_products_hold_fp16_accuracy(lib, shape, monkeypatch):
-    """One plane per operand (the hi numbers only) and one tensor-core pass: the form TGNN_MATH_F16X1 uses.  Eleven
+    """Only the hi plane of each operand and one tensor-core pass: the form the step uses for the key/value weight
+    gradient when the feature table is bf16 (tolerance 1e-2).  Eleven
     mantissa bits per operand: the product of random operands stays within 1e-3 of the largest |C| (three passes:
     1e-4), through every kernel form the launcher picks for the shape."""
     M, N, K, lay = shape
