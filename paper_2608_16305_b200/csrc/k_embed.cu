@@ -169,6 +169,9 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
   const int nb_rows = n * k;
   const int dkv = 2 * d + de;
   const int fp = de >> 1, tp = d >> 1;          // feature pairs, encoding pairs per row
+  // words written per row: the dkv + 1 columns rounded up to 8 (the rest of the pitch, padding that keeps rows on
+  // 128-byte lines, is never read: tile copies stop at the matrix's column count)
+  const int zero_end = min(ld, (dkv + 1 + 7) / 8 * 8) >> 1;
   const int groups = (nb_rows + ZS_ROWS - 1) / ZS_ROWS;
   constexpr int FP_MAX = 4, TP_MAX = 2;         // pairs per lane held in registers: de <= 256, d <= 128
   const bool regs = fp <= 32 * FP_MAX && tp <= 32 * TP_MAX;
@@ -225,7 +228,7 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
       uint32_t* hi = reinterpret_cast<uint32_t*>(z_hi + (int64_t)r * ld);
       uint32_t* lo = reinterpret_cast<uint32_t*>(z_hi + plane_s + (int64_t)r * ld);
       if (v_nbr[j] < 0) {
-        for (int q = lane; q < (ld >> 1); q += 32) { hi[q] = 0u; lo[q] = 0u; }   // the memory part too: nobody else writes this row
+        for (int q = lane; q < zero_end; q += 32) { hi[q] = 0u; lo[q] = 0u; }   // the memory part too: nobody else writes this row
         if (lane == 0) z_dt[r] = -1.f;
         continue;
       }
@@ -269,7 +272,7 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
         }
       }
       // column dkv = 1, then zeros up to the row pitch (dkv is even, the pitch a multiple of 8)
-      for (int q = (dkv >> 1) + lane; q < (ld >> 1); q += 32) { hi[q] = q == (dkv >> 1) ? 0x3c00u : 0u; lo[q] = 0u; }
+      for (int q = (dkv >> 1) + lane; q < zero_end; q += 32) { hi[q] = q == (dkv >> 1) ? 0x3c00u : 0u; lo[q] = 0u; }
       if (lane == 0) z_dt[r] = dtf;
     }
   }

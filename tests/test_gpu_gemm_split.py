@@ -59,6 +59,7 @@ PAIR_SHAPES = [
     (513, 300, 472, "k"),        # two n-tiles of different widths; the third tile holds one row
     (40000, 200, 386, "k"),      # 157 tiles over 74 pairs: the persistent walk, accumulators alternating
     (129, 16, 16, "k"),          # narrowest MMA, one contraction step
+    (40000, 200, 200, "k"),      # short contraction (the input gradient's shape): tiles of four blocks on a ring of three stages
     (200, 387, 5000, "mn"),      # weight gradient on pairs: two accumulators, 74 parts of the contraction
     (200, 201, 3000, "mn"),      # one accumulator, drained by all eight epilogue warps
     (300, 100, 40, "mn"),        # two 256-row tiles of C, contraction of two blocks
