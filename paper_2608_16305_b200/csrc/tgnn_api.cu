@@ -667,7 +667,9 @@ int tgnn_train_step(tgnn_ctx* ctx, const int32_t* u_src, const int32_t* u_dst, c
   e->kernels = ctx->launches - l0;
   cudaGraphExec_t exec = nullptr;
   // node priorities as captured (side-stream kernels low, the caller's stream as it is) instead of one priority for all
-  const cudaError_t ie = cudaGraphInstantiate(&exec, graph, cudaGraphInstantiateFlagUseNodePriority);
+  // (the attention model only: in the short chain of the time-projection model the side streams' kernels are on the
+  // critical path themselves, and ranking them below the chain cost 9 % there)
+  const cudaError_t ie = cudaGraphInstantiate(&exec, graph, ctx->cfg.model == TGNN_MODEL_TGN ? cudaGraphInstantiateFlagUseNodePriority : 0);
   cudaGraphDestroy(graph);
   if (ie != cudaSuccess || !exec) {
     cudaGetLastError();
