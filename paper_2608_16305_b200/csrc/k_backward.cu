@@ -1,7 +1,5 @@
 // Step (6): masked link-prediction loss (Eq. 13), exact backward of steps (4)-(5),
 // gradient norm g_r and the Adam update.
-#include <cstdlib>
-
 #include "tgnn_internal.cuh"
 #include "tgnn_device.cuh"
 
@@ -282,6 +280,266 @@ __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __r
   }
   __syncthreads();  // both teams are through: the block's sums are complete
   for (int q = tid; q < d; q += blockDim.x)
+    if (gw2[q] != 0.f) atomicAdd(&g_w2[q], gw2[q]);
+  if (tid == 0) {
+    if (s_gb2 != 0.f) atomicAdd(g_b2, s_gb2);
+    if (s_loss != 0.f) atomicAdd(loss_acc, s_loss);
+  }
+}
+
+// The same head on tiles of TE events per block with register-blocked products (the form used when the model's
+// width allows: d a multiple of 4 and both halves of W_1, transposed, fit in shared memory beside the tile).
+// Rows of a tile: [0, TE) sources, [TE, 2TE) destinations, [2TE, 3TE) negatives; pairs: [0, TE) positive, [TE, 2TE)
+// negative.  Shared memory, all c-major / j-major so that the inner loops read 16 bytes per operand:
+//   WaT[c][j] = W_1[j][c], WbT[c][j] = W_1[j][d + c]   (pitch LDW)
+//   HT[c][r]   embedding rows, transposed             (pitch RP = 3 TE + 4)
+//   PT[j][r]   W_1a h_r (sources) or W_1b h_r         (pitch RP)
+//   D1T[j][p]  d loss / d pre1, transposed            (pitch PP = 2 TE + 4)
+// Hidden layer: a thread owns a 4 x 4 block of (hidden unit, row) and walks the d input columns (two 16-byte loads
+// per 16 FMAs).  Input gradient: a thread owns 4 events x {positive, negative} x 4 input columns and walks the hidden
+// units four at a time (twelve 16-byte loads per 128 FMAs); it holds both pairs of its events, so the source rows'
+// two contributions meet in registers.  Everything else (scores, loss, dw_2, db_2, gate bytes) as in head_fused_kernel.
+template <int TE>
+struct HeadTile {
+  static constexpr int ROWS = 3 * TE, PAIRS = 2 * TE, RP = ROWS + 4, PP = PAIRS + 4;
+  static constexpr int THREADS = 416;
+  static __host__ __device__ int ldw(int d) { return (d + 3) & ~3; }
+  static __host__ __device__ size_t smem_floats(int d) { return (size_t)2 * d * ldw(d) + (size_t)2 * d * RP + (size_t)d * PP + 3 * (size_t)ldw(d); }
+};
+
+template <int TE>
+__global__ void __launch_bounds__(HeadTile<TE>::THREADS) head_tile_kernel(const float* __restrict__ h, const float* __restrict__ W1,
+                                                                        const float* __restrict__ b1, const float* __restrict__ w2,
+                                                                        const float* __restrict__ b2,
+                                                                        const uint8_t* __restrict__ loss_mask, int nq, int d,
+                                                                        float* __restrict__ cat1, float* __restrict__ dpre1,
+                                                                        uint8_t* __restrict__ hid_gate, float* __restrict__ dpre_o,
+                                                                        float* __restrict__ g_w2, float* __restrict__ g_b2,
+                                                                        float* __restrict__ loss_acc, int relu_out) {
+  using HT_ = HeadTile<TE>;
+  constexpr int ROWS = HT_::ROWS, PAIRS = HT_::PAIRS, RP = HT_::RP, PP = HT_::PP, T = HT_::THREADS;
+  extern __shared__ __align__(16) float sm[];
+  __shared__ float s_msum, s_gb2, s_loss;
+  const int LDW = HT_::ldw(d);
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  float* WaT = sm;
+  float* WbT = WaT + (size_t)d * LDW;
+  float* HTs = WbT + (size_t)d * LDW;
+  float* PTs = HTs + (size_t)d * RP;
+  float* D1T = PTs + (size_t)d * RP;
+  float* b1s = D1T + (size_t)d * PP;
+  float* w2s = b1s + LDW;
+  float* gw2 = w2s + LDW;
+  {  // W_1 [d][2d] -> the two transposed halves: a thread reads 4 rows of one column (coalesced over columns) and
+     // writes them as one 16-byte piece
+    // a warp owns four hidden units j at a time, its lanes walk the 2d columns: coalesced 4-byte loads of four rows
+    // of W_1, one 16-byte store per column into the transposed half; two columns per lane in flight
+    const int d4 = d >> 2, nw = T >> 5;
+    for (int j4 = wid; j4 < d4; j4 += nw) {
+      const float* w0 = W1 + (int64_t)(4 * j4) * 2 * d;
+      for (int c2 = lane; c2 < 2 * d; c2 += 64) {
+        float4 v[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int cc = c2 + 32 * u;
+          if (cc < 2 * d) {
+            v[u].x = __ldg(w0 + cc); v[u].y = __ldg(w0 + 2 * d + cc);
+            v[u].z = __ldg(w0 + 4 * d + cc); v[u].w = __ldg(w0 + 6 * d + cc);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int cc = c2 + 32 * u;
+          if (cc < 2 * d) {
+            float* dst = cc < d ? WaT + (size_t)cc * LDW : WbT + (size_t)(cc - d) * LDW;
+            *reinterpret_cast<float4*>(dst + 4 * j4) = v[u];
+          }
+        }
+      }
+    }
+  }
+  for (int q = tid; q < d; q += T) { b1s[q] = b1[q]; w2s[q] = w2[q]; gw2[q] = 0.f; }
+  if (tid == 0) { s_msum = 0.f; s_gb2 = 0.f; s_loss = 0.f; }
+  __syncthreads();
+  {  // every block counts the whole mask (a few KB)
+    int c = 0;
+    for (int j = tid; j < nq; j += T) c += loss_mask ? (loss_mask[j] != 0) : 1;
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(FULL, c, o);
+    if (lane == 0 && c) atomicAdd(&s_msum, (float)c);
+  }
+  __syncthreads();
+  const float msum = s_msum;
+  const float bias2 = b2[0];
+  const int tiles = (nq + TE - 1) / TE;
+  for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    const int ev0 = tile * TE;
+    // ---- embedding rows -> HT (transposed) and cat1 ----
+    // a warp owns rows r = wid, wid + warps, ...; its lanes walk the d columns (up to eight loads per lane in flight)
+    for (int r = wid; r < ROWS; r += (T >> 5)) {
+      const int blk = r / TE, ev = ev0 + (r - blk * TE);   // (TE is a compile-time constant)
+      const bool in = ev < nq;
+      const float* src = h + ((int64_t)blk * nq + (in ? ev : 0)) * d;
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int c = lane + 32 * u;
+        v[u] = (in && c < d) ? __ldg(src + c) : 0.f;
+      }
+      float* o0 = nullptr;   // where this row goes in cat1 (sources go to two rows)
+      float* o1 = nullptr;
+      if (in) {
+        if (blk == 0) { o0 = cat1 + (int64_t)ev * 2 * d; o1 = cat1 + (int64_t)(nq + ev) * 2 * d; }
+        else if (blk == 1) o0 = cat1 + (int64_t)ev * 2 * d + d;
+        else o0 = cat1 + (int64_t)(nq + ev) * 2 * d + d;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int c = lane + 32 * u;
+        if (c < d) {
+          if (o0) o0[c] = v[u];
+          if (o1) o1[c] = v[u];
+          HTs[c * RP + r] = v[u];
+        }
+      }
+    }
+    __syncthreads();
+    // ---- hidden layer: PT[j][r] = sum_c W[j][c] h_r[c] ----
+    {
+      const int ntj = d >> 2, ntr = ROWS >> 2;
+      for (int t = tid; t < ntj * ntr; t += T) {
+        const int tj = t % ntj, tr = t / ntj;
+        const float* Wp = (4 * tr < TE ? WaT : WbT) + 4 * tj;   // (TE is a multiple of 4: a row block lies in one part)
+        const float* Hp = HTs + 4 * tr;
+        float acc[4][4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+#pragma unroll 4
+        for (int c = 0; c < d; ++c) {
+          const float4 wv = *reinterpret_cast<const float4*>(Wp + (size_t)c * LDW);
+          const float4 hv = *reinterpret_cast<const float4*>(Hp + c * RP);
+          const float wj[4] = {wv.x, wv.y, wv.z, wv.w};
+          const float hr[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+          for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(wj[a], hr[b], acc[a][b]);
+        }
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+          *reinterpret_cast<float4*>(PTs + (4 * tj + a) * RP + 4 * tr) = make_float4(acc[a][0], acc[a][1], acc[a][2], acc[a][3]);
+      }
+    }
+    __syncthreads();
+    // ---- scores, loss terms, d loss / d pre1: one warp per pair ----
+    {
+      float gw2r[8];   // this lane's hidden units j = lane + 32 u (d <= 256)
+#pragma unroll
+      for (int u = 0; u < 8; ++u) gw2r[u] = 0.f;
+      for (int p = wid; p < PAIRS; p += (T >> 5)) {
+        const int half = p / TE, e = p - half * TE, ev = ev0 + e;
+        const bool valid = ev < nq;
+        const int s_col = e, o_col = TE + TE * half + e;
+        float sc = 0.f;
+        for (int q = lane; q < d; q += 32) {
+          const float a = fmaxf(PTs[q * RP + s_col] + PTs[q * RP + o_col] + b1s[q], 0.f);
+          sc = fmaf(w2s[q], a, sc);
+        }
+        for (int o = 16; o > 0; o >>= 1) sc += __shfl_xor_sync(FULL, sc, o);
+        sc += bias2;
+        const float m = valid && (loss_mask ? (loss_mask[ev] != 0) : true) ? 1.f : 0.f;
+        const float wj = msum > 0.f ? m / msum : 0.f;
+        const float ds = half == 0 ? -wj * sigmoidf_(-sc) : wj * sigmoidf_(sc);
+        if (lane == 0 && wj != 0.f) {
+          atomicAdd(&s_loss, wj * (half == 0 ? softplusf_(-sc) : softplusf_(sc)));
+          atomicAdd(&s_gb2, ds);
+        }
+        const int64_t row = (int64_t)half * nq + ev;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int q = lane + 32 * u;
+          if (q < d) {
+            const float a = fmaxf(PTs[q * RP + s_col] + PTs[q * RP + o_col] + b1s[q], 0.f);
+            gw2r[u] = fmaf(ds, a, gw2r[u]);
+            const float dv = a > 0.f ? ds * w2s[q] : 0.f;
+            D1T[q * PP + p] = dv;
+            if (valid) {
+              dpre1[row * d + q] = dv;
+              hid_gate[row * d + q] = a > 0.f;
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int q = lane + 32 * u;
+        if (q < d && gw2r[u] != 0.f) atomicAdd(&gw2[q], gw2r[u]);
+      }
+    }
+    __syncthreads();
+    // ---- input gradient: dC[p][c2] = sum_j dh1[p][j] W_1[j][c2], both pairs of 4 events x 4 columns per thread ----
+    {
+      const int ntp = TE >> 2, ntc = (2 * d) >> 2;
+      for (int t = tid; t < ntp * ntc; t += T) {
+        const int tp = t % ntp, tc = t / ntp;
+        const int c2 = 4 * tc;
+        const bool lower = c2 < d;
+        const float* Wp = lower ? WaT + (size_t)c2 * LDW : WbT + (size_t)(c2 - d) * LDW;
+        const float* Dp = D1T + 4 * tp;
+        float aP[4][4], aN[4][4];   // [event][column]
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int b = 0; b < 4; ++b) { aP[a][b] = 0.f; aN[a][b] = 0.f; }
+        for (int j0 = 0; j0 < d; j0 += 4) {
+          float4 w4[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) w4[i] = *reinterpret_cast<const float4*>(Wp + (size_t)i * LDW + j0);
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) {
+            const float4 dp = *reinterpret_cast<const float4*>(Dp + (j0 + jj) * PP);
+            const float4 dn = *reinterpret_cast<const float4*>(Dp + (j0 + jj) * PP + TE);
+            const float de[4] = {dp.x, dp.y, dp.z, dp.w};
+            const float dm[4] = {dn.x, dn.y, dn.z, dn.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float wv = jj == 0 ? w4[i].x : (jj == 1 ? w4[i].y : (jj == 2 ? w4[i].z : w4[i].w));
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                aP[e][i] = fmaf(de[e], wv, aP[e][i]);
+                aN[e][i] = fmaf(dm[e], wv, aN[e][i]);
+              }
+            }
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int el = 4 * tp + e, ev = ev0 + el;
+          if (ev >= nq) continue;
+          if (lower) {   // source rows collect their positive and their negative pair
+            float o[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              o[i] = (!relu_out || HTs[(c2 + i) * RP + el] > 0.f) ? aP[e][i] + aN[e][i] : 0.f;
+            *reinterpret_cast<float4*>(dpre_o + (int64_t)ev * d + c2) = make_float4(o[0], o[1], o[2], o[3]);
+          } else {
+            const int cc = c2 - d;
+            float o[4], n[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              o[i] = (!relu_out || HTs[(cc + i) * RP + TE + el] > 0.f) ? aP[e][i] : 0.f;
+              n[i] = (!relu_out || HTs[(cc + i) * RP + 2 * TE + el] > 0.f) ? aN[e][i] : 0.f;
+            }
+            *reinterpret_cast<float4*>(dpre_o + ((int64_t)nq + ev) * d + cc) = make_float4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<float4*>(dpre_o + ((int64_t)2 * nq + ev) * d + cc) = make_float4(n[0], n[1], n[2], n[3]);
+          }
+        }
+      }
+    }
+    __syncthreads();
+  }
+  for (int q = tid; q < d; q += T)
     if (gw2[q] != 0.f) atomicAdd(&g_w2[q], gw2[q]);
   if (tid == 0) {
     if (s_gb2 != 0.f) atomicAdd(g_b2, s_gb2);
@@ -928,7 +1186,23 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     // beside the staging rows; wider models take the projections through the GEMM path instead.
     const int relu_out = c.model == TGNN_MODEL_TGN ? 1 : 0;
     const size_t hf_smem = head_fused_smem(d);
-    if (hf_smem <= 200 * 1024) {
+    // Large batches: tiles of 32 events per block with register-blocked products (one round of blocks from 2 400
+    // events up; below that the groups of four of head_fused_kernel spread over more SMs and are faster).
+    const size_t ht32 = HeadTile<32>::smem_floats(d) * sizeof(float);
+    if (d % 4 == 0 && d <= 256 && ht32 <= 225 * 1024 && n_q >= 32 * 74) {
+      static SmemLimit ht32_limit;
+      RC(raise_smem_limit(ctx, head_tile_kernel<32>, (int)ht32, ht32_limit));
+      const int tiles = (n_q + 31) / 32;
+      {
+        KernelScope scope__(ctx, "head_fused", s);
+        head_tile_kernel<32><<<tiles < 148 ? tiles : 148, HeadTile<32>::THREADS, ht32, s>>>(
+            ctx->e_h, P + L.w1, P + L.b1, P + L.w2, P + L.b2, loss_mask, n_q, d, w.cat1, w.hid1, w.hid_gate, w.dpre_o,
+            G + L.w2, G + L.b2, w.st_scalars, relu_out);
+      }
+      TGNN_LAUNCH_OK(ctx, "head_fused");
+      RC(fork_to(ctx, s, sa));
+      RC(grad_w(ctx, w.hid1, d, w.cat1, 2 * d, 2 * n_q, nullptr, d, 2 * d, G + L.w1, G + L.b1, "dW_1", sa));
+    } else if (hf_smem <= 200 * 1024) {
       static SmemLimit hf_limit;
       RC(raise_smem_limit(ctx, head_fused_kernel, (int)hf_smem, hf_limit));
       const int groups = (n_q + HF_EV - 1) / HF_EV;
