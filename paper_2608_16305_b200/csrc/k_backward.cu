@@ -1186,18 +1186,35 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     // beside the staging rows; wider models take the projections through the GEMM path instead.
     const int relu_out = c.model == TGNN_MODEL_TGN ? 1 : 0;
     const size_t hf_smem = head_fused_smem(d);
-    // Large batches: tiles of 32 events per block with register-blocked products (one round of blocks from 2 400
-    // events up; below that the groups of four of head_fused_kernel spread over more SMs and are faster).
+    // Large batches: tiles of TE events per block with register-blocked products (from 2 400 events up; below that
+    // the groups of four of head_fused_kernel spread over more SMs and are faster).  TE is the tile size whose
+    // rounds of 148 blocks cost least: 4 000 events are 143 tiles of 28 -- one round on 143 SMs -- where tiles of 32
+    // would leave 23 SMs idle for a longer round.
     const size_t ht32 = HeadTile<32>::smem_floats(d) * sizeof(float);
     if (d % 4 == 0 && d <= 256 && ht32 <= 225 * 1024 && n_q >= 32 * 74) {
-      static SmemLimit ht32_limit;
-      RC(raise_smem_limit(ctx, head_tile_kernel<32>, (int)ht32, ht32_limit));
-      const int tiles = (n_q + 31) / 32;
+      int te = 32, best = 1 << 30;
+      for (int cand = 32; cand >= 20; cand -= 4) {
+        const int tiles = (n_q + cand - 1) / cand, cost = ((tiles + 147) / 148) * cand;
+        if (cost < best) { best = cost; te = cand; }
+      }
+      const int tiles = (n_q + te - 1) / te;
+      const int grid = tiles < 148 ? tiles : 148;
       {
         KernelScope scope__(ctx, "head_fused", s);
-        head_tile_kernel<32><<<tiles < 148 ? tiles : 148, HeadTile<32>::THREADS, ht32, s>>>(
-            ctx->e_h, P + L.w1, P + L.b1, P + L.w2, P + L.b2, loss_mask, n_q, d, w.cat1, w.hid1, w.hid_gate, w.dpre_o,
-            G + L.w2, G + L.b2, w.st_scalars, relu_out);
+#define TGNN_HEAD_TILE(TE_)                                                                                              \
+  do {                                                                                                                   \
+    static SmemLimit lim__;                                                                                              \
+    const size_t bytes__ = HeadTile<TE_>::smem_floats(d) * sizeof(float);                                                \
+    RC(raise_smem_limit(ctx, head_tile_kernel<TE_>, (int)bytes__, lim__));                                               \
+    head_tile_kernel<TE_><<<grid, HeadTile<TE_>::THREADS, bytes__, s>>>(                                                 \
+        ctx->e_h, P + L.w1, P + L.b1, P + L.w2, P + L.b2, loss_mask, n_q, d, w.cat1, w.hid1, w.hid_gate, w.dpre_o,      \
+        G + L.w2, G + L.b2, w.st_scalars, relu_out);                                                                    \
+  } while (0)
+        if (te == 32) TGNN_HEAD_TILE(32);
+        else if (te == 28) TGNN_HEAD_TILE(28);
+        else if (te == 24) TGNN_HEAD_TILE(24);
+        else TGNN_HEAD_TILE(20);
+#undef TGNN_HEAD_TILE
       }
       TGNN_LAUNCH_OK(ctx, "head_fused");
       RC(fork_to(ctx, s, sa));
