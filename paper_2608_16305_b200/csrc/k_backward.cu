@@ -297,12 +297,12 @@ __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __r
 //   D1T[j][p]  d loss / d pre1, transposed            (pitch PP = 2 TE + 4)
 // Hidden layer: a thread owns a 4 x 4 block of (hidden unit, row) and walks the d input columns (two 16-byte loads
 // per 16 FMAs).  Input gradient: a thread owns 4 events x {positive, negative} x 4 input columns and walks the hidden
-// units four at a time (twelve 16-byte loads per 128 FMAs); it holds both pairs of its events, so the source rows'
-// two contributions meet in registers.  Everything else (scores, loss, dw_2, db_2, gate bytes) as in head_fused_kernel.
+// units four at a time; it holds both pairs of its two events, so the source rows' two contributions meet in
+// registers.  Everything else (scores, loss, dw_2, db_2, gate bytes) as in head_fused_kernel.
 template <int TE>
 struct HeadTile {
   static constexpr int ROWS = 3 * TE, PAIRS = 2 * TE, RP = ROWS + 4, PP = PAIRS + 4;
-  static constexpr int THREADS = 416;
+  static constexpr int THREADS = 832;   // 26 warps: the products' loops wait on shared-memory loads, and more warps hide that
   static __host__ __device__ int ldw(int d) { return (d + 3) & ~3; }
   static __host__ __device__ size_t smem_floats(int d) { return (size_t)2 * d * ldw(d) + (size_t)2 * d * RP + (size_t)d * PP + 3 * (size_t)ldw(d); }
 };
@@ -478,18 +478,18 @@ __global__ void __launch_bounds__(HeadTile<TE>::THREADS) head_tile_kernel(const 
       }
     }
     __syncthreads();
-    // ---- input gradient: dC[p][c2] = sum_j dh1[p][j] W_1[j][c2], both pairs of 4 events x 4 columns per thread ----
+    // ---- input gradient: dC[p][c2] = sum_j dh1[p][j] W_1[j][c2], both pairs of 2 events x 4 columns per thread ----
     {
-      const int ntp = TE >> 2, ntc = (2 * d) >> 2;
+      const int ntp = TE >> 1, ntc = (2 * d) >> 2;
       for (int t = tid; t < ntp * ntc; t += T) {
         const int tp = t % ntp, tc = t / ntp;
         const int c2 = 4 * tc;
         const bool lower = c2 < d;
         const float* Wp = lower ? WaT + (size_t)c2 * LDW : WbT + (size_t)(c2 - d) * LDW;
-        const float* Dp = D1T + 4 * tp;
-        float aP[4][4], aN[4][4];   // [event][column]
+        const float* Dp = D1T + 2 * tp;
+        float aP[2][4], aN[2][4];   // [event][column]
 #pragma unroll
-        for (int a = 0; a < 4; ++a)
+        for (int a = 0; a < 2; ++a)
 #pragma unroll
           for (int b = 0; b < 4; ++b) { aP[a][b] = 0.f; aN[a][b] = 0.f; }
         for (int j0 = 0; j0 < d; j0 += 4) {
@@ -498,15 +498,15 @@ __global__ void __launch_bounds__(HeadTile<TE>::THREADS) head_tile_kernel(const 
           for (int i = 0; i < 4; ++i) w4[i] = *reinterpret_cast<const float4*>(Wp + (size_t)i * LDW + j0);
 #pragma unroll
           for (int jj = 0; jj < 4; ++jj) {
-            const float4 dp = *reinterpret_cast<const float4*>(Dp + (j0 + jj) * PP);
-            const float4 dn = *reinterpret_cast<const float4*>(Dp + (j0 + jj) * PP + TE);
-            const float de[4] = {dp.x, dp.y, dp.z, dp.w};
-            const float dm[4] = {dn.x, dn.y, dn.z, dn.w};
+            const float2 dp = *reinterpret_cast<const float2*>(Dp + (j0 + jj) * PP);
+            const float2 dn = *reinterpret_cast<const float2*>(Dp + (j0 + jj) * PP + TE);
+            const float de[2] = {dp.x, dp.y};
+            const float dm[2] = {dn.x, dn.y};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               const float wv = jj == 0 ? w4[i].x : (jj == 1 ? w4[i].y : (jj == 2 ? w4[i].z : w4[i].w));
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
+              for (int e = 0; e < 2; ++e) {
                 aP[e][i] = fmaf(de[e], wv, aP[e][i]);
                 aN[e][i] = fmaf(dm[e], wv, aN[e][i]);
               }
@@ -514,8 +514,8 @@ __global__ void __launch_bounds__(HeadTile<TE>::THREADS) head_tile_kernel(const 
           }
         }
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int el = 4 * tp + e, ev = ev0 + el;
+        for (int e = 0; e < 2; ++e) {
+          const int el = 2 * tp + e, ev = ev0 + el;
           if (ev >= nq) continue;
           if (lower) {   // source rows collect their positive and their negative pair
             float o[4];
