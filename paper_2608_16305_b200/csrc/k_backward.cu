@@ -287,6 +287,20 @@ __global__ void __launch_bounds__(HF_THREADS) head_fused_kernel(const float* __r
   }
 }
 
+// W_1 [d][2d] -> WT[c2][j] = W_1[j][c2] (row pitch ldw): both halves transposed, the layout head_tile_kernel keeps in
+// shared memory.  A warp owns four hidden units, its lanes walk the columns.
+__global__ void __launch_bounds__(256) prep_head_wt_kernel(const float* __restrict__ W1, int d, int ldw, float* __restrict__ WT) {
+  const int lane = threadIdx.x & 31, wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nw = (gridDim.x * blockDim.x) >> 5;
+  for (int j4 = wid; j4 < (d >> 2); j4 += nw) {
+    const float* w0 = W1 + (int64_t)(4 * j4) * 2 * d;
+    for (int c2 = lane; c2 < 2 * d; c2 += 32) {
+      float4 v;
+      v.x = __ldg(w0 + c2); v.y = __ldg(w0 + 2 * d + c2); v.z = __ldg(w0 + 4 * d + c2); v.w = __ldg(w0 + 6 * d + c2);
+      *reinterpret_cast<float4*>(WT + (size_t)c2 * ldw + 4 * j4) = v;
+    }
+  }
+}
+
 // The same head on tiles of TE events per block with register-blocked products (the form used when the model's
 // width allows: d a multiple of 4 and both halves of W_1, transposed, fit in shared memory beside the tile).
 // Rows of a tile: [0, TE) sources, [TE, 2TE) destinations, [2TE, 3TE) negatives; pairs: [0, TE) positive, [TE, 2TE)
@@ -308,7 +322,7 @@ struct HeadTile {
 };
 
 template <int TE>
-__global__ void __launch_bounds__(HeadTile<TE>::THREADS) head_tile_kernel(const float* __restrict__ h, const float* __restrict__ W1,
+__global__ void __launch_bounds__(HeadTile<TE>::THREADS) head_tile_kernel(const float* __restrict__ h, const float* __restrict__ WT,
                                                                         const float* __restrict__ b1, const float* __restrict__ w2,
                                                                         const float* __restrict__ b2,
                                                                         const uint8_t* __restrict__ loss_mask, int nq, int d,
@@ -330,33 +344,11 @@ __global__ void __launch_bounds__(HeadTile<TE>::THREADS) head_tile_kernel(const 
   float* b1s = D1T + (size_t)d * PP;
   float* w2s = b1s + LDW;
   float* gw2 = w2s + LDW;
-  {  // W_1 [d][2d] -> the two transposed halves: a thread reads 4 rows of one column (coalesced over columns) and
-     // writes them as one 16-byte piece
-    // a warp owns four hidden units j at a time, its lanes walk the 2d columns: coalesced 4-byte loads of four rows
-    // of W_1, one 16-byte store per column into the transposed half; two columns per lane in flight
-    const int d4 = d >> 2, nw = T >> 5;
-    for (int j4 = wid; j4 < d4; j4 += nw) {
-      const float* w0 = W1 + (int64_t)(4 * j4) * 2 * d;
-      for (int c2 = lane; c2 < 2 * d; c2 += 64) {
-        float4 v[2];
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const int cc = c2 + 32 * u;
-          if (cc < 2 * d) {
-            v[u].x = __ldg(w0 + cc); v[u].y = __ldg(w0 + 2 * d + cc);
-            v[u].z = __ldg(w0 + 4 * d + cc); v[u].w = __ldg(w0 + 6 * d + cc);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const int cc = c2 + 32 * u;
-          if (cc < 2 * d) {
-            float* dst = cc < d ? WaT + (size_t)cc * LDW : WbT + (size_t)(cc - d) * LDW;
-            *reinterpret_cast<float4*>(dst + 4 * j4) = v[u];
-          }
-        }
-      }
-    }
+  {  // both transposed halves of W_1 (prepared once per step in this layout): a straight 16-byte copy
+    const int n4 = (2 * d * LDW) >> 2;
+    const float4* src = reinterpret_cast<const float4*>(WT);
+    float4* dst = reinterpret_cast<float4*>(WaT);
+    for (int i = tid; i < n4; i += T) dst[i] = __ldg(src + i);
   }
   for (int q = tid; q < d; q += T) { b1s[q] = b1[q]; w2s[q] = w2[q]; gw2[q] = 0.f; }
   if (tid == 0) { s_msum = 0.f; s_gb2 = 0.f; s_loss = 0.f; }
@@ -1130,6 +1122,17 @@ int grad_in(tgnn_ctx* ctx, const float* dY, int64_t ld_dy, const float* W, int64
 
 }  // namespace
 
+int launch_prep_head(tgnn_ctx* ctx, cudaStream_t s) {
+  const int d = ctx->cfg.d;
+  if (d % 4 != 0 || d > 256) return TGNN_OK;   // (the tile head is not used for such widths)
+  {
+    KernelScope scope__(ctx, "prep_head", s);
+    prep_head_wt_kernel<<<(d / 4 + 7) / 8, 256, 0, s>>>(ctx->params + ctx->L.w1, d, (d + 3) / 4 * 4, ctx->ws.head_wT);
+  }
+  TGNN_LAUNCH_OK(ctx, "prep_head");
+  return TGNN_OK;
+}
+
 int launch_get_gates(tgnn_ctx* ctx, uint8_t* h_gate_out, uint8_t* hid_gate_out, cudaStream_t s) {
   const int64_t n = (int64_t)ctx->e_n * ctx->cfg.d;
   if (n > 0) {
@@ -1199,6 +1202,9 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       }
       const int tiles = (n_q + te - 1) / te;
       const int grid = tiles < 148 ? tiles : 148;
+      // W_1 transposed: written with the weight images at the start of the step; otherwise (fp32 mode, or the
+      // backward step called on its own after the parameters changed) here
+      if (!(ctx->images != nullptr && ctx->images_fresh)) RC(launch_prep_head(ctx, s));
       {
         KernelScope scope__(ctx, "head_fused", s);
 #define TGNN_HEAD_TILE(TE_)                                                                                              \
@@ -1207,7 +1213,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     const size_t bytes__ = HeadTile<TE_>::smem_floats(d) * sizeof(float);                                                \
     RC(raise_smem_limit(ctx, head_tile_kernel<TE_>, (int)bytes__, lim__));                                               \
     head_tile_kernel<TE_><<<grid, HeadTile<TE_>::THREADS, bytes__, s>>>(                                                 \
-        ctx->e_h, P + L.w1, P + L.b1, P + L.w2, P + L.b2, loss_mask, n_q, d, w.cat1, w.hid1, w.hid_gate, w.dpre_o,      \
+        ctx->e_h, w.head_wT, P + L.b1, P + L.w2, P + L.b2, loss_mask, n_q, d, w.cat1, w.hid1, w.hid_gate, w.dpre_o,      \
         G + L.w2, G + L.b2, w.st_scalars, relu_out);                                                                    \
   } while (0)
         if (te == 32) TGNN_HEAD_TILE(32);

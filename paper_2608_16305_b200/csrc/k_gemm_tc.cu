@@ -964,6 +964,8 @@ int launch_prep_weights(tgnn_ctx* ctx, cudaStream_t s) {
     prep_weights_kernel<<<grid, 256, 0, s>>>(ctx->sites_dev, ctx->params, ctx->images);
   }
   TGNN_LAUNCH_OK(ctx, "prep_weights");
+  const int rch = launch_prep_head(ctx, s);    // W_1 transposed, for the tile form of the link-prediction head
+  if (rch) return rch;
   return launch_prep_split_weights(ctx, s);   // the split planes of the key/value weights, when that mode is on
 }
 

@@ -132,6 +132,7 @@ size_t carve(tgnn_ctx* ctx, char* base) {
   cv.take(w.Q, R * d);
   cv.take(w.alpha, R * H * k);
   cv.take(w.cat_o, R * 2 * d);
+  cv.take(w.head_wT, 2 * d * ((d + 3) / 4 * 4));
   cv.take(w.cat1, 2 * nq * 2 * d);
   cv.take(w.hid1, 2 * nq * d);
   cv.take(w.hid_gate, 2 * nq * d);

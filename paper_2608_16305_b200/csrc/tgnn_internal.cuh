@@ -64,6 +64,7 @@ struct Workspace {
   float* alpha;  // [R_cap, H, k]
   float* cat_o;  // [R_cap, 2d]  (a | m_root)
   // step (6)
+  float* head_wT; // [2d, up4(d)] W_1's two halves transposed ([c][j]) for the tile head, rewritten with the weight images
   float* cat1;    // [2*nq_cap, 2d]
   float* hid1;    // [2*nq_cap, d]  ReLU(pre1); overwritten by dpre1
   uint8_t* hid_gate;  // [2*nq_cap, d] 1 where the head's hidden unit was active
@@ -383,5 +384,6 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
                       int single = -1, int launches = 1, int pair = -1);
 size_t plan_weight_sites(tgnn_ctx* ctx);                       // fills ctx->sites, returns the image bytes needed
 int launch_prep_weights(tgnn_ctx* ctx, cudaStream_t s);        // writes all images from the current parameters
+int launch_prep_head(tgnn_ctx* ctx, cudaStream_t s);           // k_backward.cu: W_1 transposed for the tile head
 
 }  // namespace tgnn
