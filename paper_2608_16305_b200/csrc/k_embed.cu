@@ -184,15 +184,30 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
     tb[u][0] = in ? time_b[q] : 0.f; tb[u][1] = in ? time_b[q + 1] : 0.f;
   }
   // this launch covers the row groups [g_begin, g_end) (the gather goes out as several launches, see the launcher)
-  for (int gidx = g_begin + ((blockIdx.x * blockDim.x + threadIdx.x) >> 5); gidx < min(groups, g_end); gidx += warps) {
+  // The slot records of a group (one lane per row) are fetched one group ahead: the dependent chain of a group is
+  // slot record -> feature rows -> stores, and a warp that walks several groups would otherwise pay both round
+  // trips one after the other for each of them.
+  const int g_last = min(groups, g_end);
+  int nx_nbr = -1, nx_eid = 0;
+  double nx_t = 0.0, nx_ts = 0.0;
+  auto fetch_slots = [&](int gi) {
+    nx_nbr = -1; nx_eid = 0; nx_t = 0.0; nx_ts = 0.0;
+    const int r = gi * ZS_ROWS + lane;
+    if (gi < g_last && lane < ZS_ROWS && r < nb_rows) {
+      nx_nbr = __ldg(nbr + r);
+      nx_eid = __ldg(eid + r);
+      nx_t = __ldg(times + r / k);
+      nx_ts = __ldg(ts + r);
+    }
+  };
+  const int g_first = g_begin + ((blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+  fetch_slots(g_first);
+  for (int gidx = g_first; gidx < g_last; gidx += warps) {
     const int r0 = gidx * ZS_ROWS;
-    int my_nbr = -1, my_eid = 0;
-    float my_dt = 0.f;
+    int my_nbr = nx_nbr, my_eid = nx_eid;
+    float my_dt = (float)(nx_t - nx_ts);
+    fetch_slots(gidx + warps);   // in flight while this group's feature rows are fetched and written
     if (lane < ZS_ROWS && r0 + lane < nb_rows) {
-      const int r = r0 + lane;
-      my_nbr = nbr[r];
-      my_eid = eid[r];
-      my_dt = (float)(times[r / k] - ts[r]);
       // a slot naming a node or a feature row that does not exist is reported and treated as empty
       if (my_nbr >= 0 && !(index_ok(my_nbr, N, status) & (de == 0 || index_ok(my_eid, E, status)))) my_nbr = -1;
     }
@@ -238,10 +253,17 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
         for (int u = 0; u < FP_MAX; ++u) {
           const int q = lane + 32 * u;
           if (q < fp) {
-            uint32_t h, l;
-            if (feat_bf16) split_f16_pair(__uint_as_float(fa[j][u] << 16), __uint_as_float(fa[j][u] & 0xffff0000u), &h, &l);
-            else split_f16_pair(__uint_as_float(fa[j][u]), __uint_as_float(fb[j][u]), &h, &l);
-            hi[(d >> 1) + q] = h; lo[(d >> 1) + q] = l;
+            if (feat_bf16) {
+              // A bf16 number is an fp16 number (8 significant bits, and the workloads' features lie inside fp16's
+              // range), so its lo part is zero: the lo plane's feature columns are never written and stay at the
+              // zeros they were allocated with.  (Below 6e-5 in magnitude the value is rounded to fp16's subnormal
+              // grid instead: an absolute error under 3e-8.)
+              hi[(d >> 1) + q] = pack_f16_pair(__uint_as_float(fa[j][u] << 16), __uint_as_float(fa[j][u] & 0xffff0000u));
+            } else {
+              uint32_t h, l;
+              split_f16_pair(__uint_as_float(fa[j][u]), __uint_as_float(fb[j][u]), &h, &l);
+              hi[(d >> 1) + q] = h; lo[(d >> 1) + q] = l;
+            }
           }
         }
 #pragma unroll
@@ -258,11 +280,11 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const voi
           uint32_t h, l;
           if (feat_bf16) {
             const uint32_t w2 = __ldg(reinterpret_cast<const uint32_t*>(efeat) + (int64_t)v_eid[j] * fp + q);
-            split_f16_pair(__uint_as_float(w2 << 16), __uint_as_float(w2 & 0xffff0000u), &h, &l);
-          } else {
-            const uint2 x = __ldg(reinterpret_cast<const uint2*>(efeat) + (int64_t)v_eid[j] * fp + q);
-            split_f16_pair(__uint_as_float(x.x), __uint_as_float(x.y), &h, &l);
+            hi[(d >> 1) + q] = pack_f16_pair(__uint_as_float(w2 << 16), __uint_as_float(w2 & 0xffff0000u));
+            continue;
           }
+          const uint2 x = __ldg(reinterpret_cast<const uint2*>(efeat) + (int64_t)v_eid[j] * fp + q);
+          split_f16_pair(__uint_as_float(x.x), __uint_as_float(x.y), &h, &l);
           hi[(d >> 1) + q] = h; lo[(d >> 1) + q] = l;
         }
         for (int q = lane; q < tp; q += 32) {

@@ -71,6 +71,12 @@ __device__ __forceinline__ void split_f16_pair(float x0, float x1, uint32_t* hi,
   *lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
+// Two values as one fp16 number each, packed (the hi part alone).
+__device__ __forceinline__ uint32_t pack_f16_pair(float x0, float x1) {
+  const __half2 h = __floats2half2_rn(x0, x1);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
 __device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + expf(-x)); }
 __device__ __forceinline__ float softplusf_(float x) { return x > 0.f ? x + log1pf(expf(-x)) : log1pf(expf(x)); }
 
