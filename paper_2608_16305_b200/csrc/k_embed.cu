@@ -154,7 +154,7 @@ __global__ void __launch_bounds__(256, 3) gather_z_static_kernel(const void* __r
 // column dkv a constant 1 (it turns the weight-gradient product's last column into the bias gradient), zeros up
 // to ld; an empty slot is a row of zeros.  Values travel as pairs of neighbouring columns packed into 32-bit
 // words (d and de are even).  Both planes hold fp16 numbers (activations of moderate size: 22 mantissa bits).
-__global__ void __launch_bounds__(256, 3) gather_z_static_split_kernel(const void* __restrict__ efeat, int feat_bf16,
+__global__ void __launch_bounds__(256, 4) gather_z_static_split_kernel(const void* __restrict__ efeat, int feat_bf16,
                                                                     const float* __restrict__ time_w,
                                                                     const float* __restrict__ time_b, int d, int de, int k,
                                                                     const double* __restrict__ times, int n,
