@@ -688,82 +688,115 @@ __global__ void __launch_bounds__(256) scatter_dmem_kernel(const float* __restri
 }
 
 // The same scatter for batches in which many rows hit few nodes (hub nodes: tens of thousands of rows onto one
-// updated row serialise on its atomics).  A block takes SC_ROWS consecutive rows and first sums them per slot in
-// a small shared-memory table (SC_WAYS entries, claimed by compare-and-swap; a row whose slot finds its entry
-// taken by another slot goes to global memory directly), then adds every claimed entry to dMemU once.
-// Dynamic shared memory: SC_WAYS * d floats.
-constexpr int SC_ROWS = 128, SC_WAYS = 16;
-__global__ void __launch_bounds__(256) scatter_dmem_cached_kernel(const float* __restrict__ dZm,
-                                                                  const float* __restrict__ dcat_o,
-                                                                  const float* __restrict__ dzq,
-                                                                  const int32_t* __restrict__ nbr,
-                                                                  const int32_t* __restrict__ nodes, int n, int k, int d,
-                                                                  const int32_t* __restrict__ node2slot,
-                                                                  float* __restrict__ dMemU, int64_t N) {
-  extern __shared__ __align__(16) float s_acc[];  // [SC_WAYS][d]
-  __shared__ int s_id[SC_WAYS];
+// updated row serialise on its atomics).  A block takes SC_ROWS consecutive rows.  One thread per row first
+// resolves row -> node -> slot and files the row under one of SC_WAYS lists (a list belongs to the first slot that
+// claims it by compare-and-swap; a row whose list belongs to another slot goes to a list of singles).  The lists
+// are then laid end to end, so that rows of one slot are neighbours, and every warp walks an equal share of that
+// sequence, 8 / U row loads in flight: it sums in registers while the slot stays the same and adds the sum to
+// dMemU when it changes.  Rows whose node was not updated are never read.
+constexpr int SC_ROWS = 256, SC_WAYS = 32;  // 256 rows, 256 threads: the whole batch is one wave of blocks
+template <int U>  // 16-byte pieces of a row per lane: 1 (d <= 128) or 2
+__global__ void __launch_bounds__(256, 4) scatter_dmem_cached_kernel(const float* __restrict__ dZm,
+                                                                     const float* __restrict__ dcat_o,
+                                                                     const float* __restrict__ dzq,
+                                                                     const int32_t* __restrict__ nbr,
+                                                                     const int32_t* __restrict__ nodes, int n, int k, int d,
+                                                                     const int32_t* __restrict__ node2slot,
+                                                                     float* __restrict__ dMemU, int64_t N) {
+  static_assert(SC_WAYS == 32, "one lane per list in the offset scan");
+  static_assert(SC_ROWS == 256, "one thread per row, row numbers kept in a byte");
+  __shared__ int s_id[SC_WAYS], s_cnt[SC_WAYS + 1], s_off[SC_WAYS + 1], s_slot[SC_ROWS];
+  __shared__ unsigned char s_seq[SC_ROWS];
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const int nb_rows = n * k, total = nb_rows + n;
-  const int d4 = d >> 2;
-  for (int e = threadIdx.x; e < SC_WAYS * d; e += blockDim.x) s_acc[e] = 0.f;
+  const int d4 = d >> 2;  // <= 32 U
+  const int r_base = blockIdx.x * SC_ROWS;
   if (threadIdx.x < SC_WAYS) s_id[threadIdx.x] = -1;
+  if (threadIdx.x <= SC_WAYS) s_cnt[threadIdx.x] = 0;  // (entry SC_WAYS: the singles)
   __syncthreads();
-  const int r_end = min(total, (int)(blockIdx.x + 1) * SC_ROWS);
-  for (int r = blockIdx.x * SC_ROWS + wid; r < r_end; r += 8) {
-    const bool isn = r < nb_rows;
-    const int i = r - nb_rows;
-    float4 g[2];
+  int way = -1, pos = 0;
+  if (r_base + threadIdx.x < total) {
+    const int r = r_base + threadIdx.x;
+    const int node = r < nb_rows ? nbr[r] : nodes[r - nb_rows];
+    int slot = -1;
+    if (node >= 0 && node < N) slot = node2slot[node];  // (an id beyond the graph was reported by the forward pass)
+    s_slot[threadIdx.x] = slot;
+    if (slot >= 0) {
+      way = slot % SC_WAYS;
+      const int owner = atomicCAS(&s_id[way], -1, slot);
+      if (owner != -1 && owner != slot) way = SC_WAYS;
+      pos = atomicAdd(&s_cnt[way], 1);
+    }
+  }
+  __syncthreads();
+  if (wid == 0) {  // exclusive scan of the list lengths
+    const int c = s_cnt[lane];
+    int incl = c;
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(FULL, incl, o);
+      if (lane >= o) incl += t;
+    }
+    s_off[lane] = incl - c;
+    if (lane == 31) s_off[SC_WAYS] = incl;
+  }
+  __syncthreads();
+  if (way >= 0) s_seq[s_off[way] + pos] = (unsigned char)threadIdx.x;
+  __syncthreads();
+  const int n_live = s_off[SC_WAYS] + s_cnt[SC_WAYS];
+  const int share = (n_live + 7) >> 3;
+  const int e_end = min(n_live, (wid + 1) * share);
+  constexpr int V = 8 / U;
+  int cur = -1;
+  float4 acc[U];
+#pragma unroll
+  for (int u = 0; u < U; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+  auto flush = [&]() {
+    if (cur < 0) return;
+    float4* out = reinterpret_cast<float4*>(dMemU + (int64_t)cur * d);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
       const int q4 = lane + 32 * u;
-      g[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (q4 < d4) {
-        if (isn) {
-          g[u] = __ldg(reinterpret_cast<const float4*>(dZm + (int64_t)r * 2 * d) + q4);
-        } else {
-          const float4 a = __ldg(reinterpret_cast<const float4*>(dcat_o + (int64_t)i * 2 * d + d) + q4);
-          const float4 b = __ldg(reinterpret_cast<const float4*>(dzq + (int64_t)i * 2 * d) + q4);
-          g[u] = make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
-        }
-      }
+      if (q4 < d4) atomicAdd(out + q4, acc[u]);
+      acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    const int node = isn ? nbr[r] : nodes[i];
-    if (node < 0 || node >= N) continue;
-    const int slot = node2slot[node];
-    if (slot < 0) continue;
-    const int way = slot % SC_WAYS;
-    int owner = 0;
-    if (lane == 0) {
-      owner = atomicCAS(&s_id[way], -1, slot);
-      if (owner == -1) owner = slot;  // claimed now
-    }
-    owner = __shfl_sync(FULL, owner, 0);
-    if (owner == slot) {
-      float* acc = s_acc + way * d;
+  };
+  for (int e = wid * share; e < e_end; e += V) {
+    float4 g[V][U];
+    int t[V];
 #pragma unroll
-      for (int u = 0; u < 2; ++u) {
+    for (int v = 0; v < V; ++v) {
+      t[v] = e + v < e_end ? (int)s_seq[e + v] : -1;
+      if (t[v] < 0) continue;
+      const int r = r_base + t[v];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
         const int q4 = lane + 32 * u;
+        g[v][u] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (q4 < d4) {
-          atomicAdd(acc + 4 * q4, g[u].x); atomicAdd(acc + 4 * q4 + 1, g[u].y);
-          atomicAdd(acc + 4 * q4 + 2, g[u].z); atomicAdd(acc + 4 * q4 + 3, g[u].w);
+          if (r < nb_rows) {
+            g[v][u] = __ldg(reinterpret_cast<const float4*>(dZm + (int64_t)r * 2 * d) + q4);  // memory half of the row
+          } else {
+            const int i = r - nb_rows;
+            const float4 a = __ldg(reinterpret_cast<const float4*>(dcat_o + (int64_t)i * 2 * d + d) + q4);
+            const float4 b = __ldg(reinterpret_cast<const float4*>(dzq + (int64_t)i * 2 * d) + q4);
+            g[v][u] = make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+          }
         }
       }
-    } else {
-      float4* out = reinterpret_cast<float4*>(dMemU + (int64_t)slot * d);
+    }
 #pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        const int q4 = lane + 32 * u;
-        if (q4 < d4) atomicAdd(out + q4, g[u]);
+    for (int v = 0; v < V; ++v) {
+      if (t[v] < 0) continue;  // (uniform over the warp)
+      const int slot = s_slot[t[v]];
+      if (slot != cur) { flush(); cur = slot; }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        acc[u].x += g[v][u].x; acc[u].y += g[v][u].y; acc[u].z += g[v][u].z; acc[u].w += g[v][u].w;
       }
     }
   }
-  __syncthreads();
-  for (int w = wid; w < SC_WAYS; w += 8) {
-    const int slot = s_id[w];
-    if (slot < 0) continue;
-    float4* out = reinterpret_cast<float4*>(dMemU + (int64_t)slot * d);
-    for (int q4 = lane; q4 < d4; q4 += 32) atomicAdd(out + q4, *reinterpret_cast<const float4*>(s_acc + w * d + 4 * q4));
-  }
+  flush();
 }
 
 // Time-encoder gradient: G[r, col0 + c] is d loss / d Phi(dt_r)_c and S[r, c] = sin(arg) was kept by
@@ -1399,12 +1432,17 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       {
         KernelScope scope__(ctx, "scatter_dmem", s);
         // many rows per node (small node set, large batch): sum per block first, the hub rows would serialise
-        if ((int64_t)NB >= 4 * (int64_t)c.num_nodes)
-          scatter_dmem_cached_kernel<<<(NB + R + SC_ROWS - 1) / SC_ROWS, 256, (size_t)SC_WAYS * d * sizeof(float), s>>>(
+        if ((int64_t)NB >= 4 * (int64_t)c.num_nodes) {
+          if (d <= 128)
+          scatter_dmem_cached_kernel<1><<<(NB + R + SC_ROWS - 1) / SC_ROWS, 256, 0, s>>>(
               w.dZmp, w.dcat_o, w.dzq, ctx->e_nbr, ctx->e_nodes, R, k, d, w.node2slot, w.dMemU, c.num_nodes);
         else
+          scatter_dmem_cached_kernel<2><<<(NB + R + SC_ROWS - 1) / SC_ROWS, 256, 0, s>>>(
+              w.dZmp, w.dcat_o, w.dzq, ctx->e_nbr, ctx->e_nodes, R, k, d, w.node2slot, w.dMemU, c.num_nodes);
+        } else {
           scatter_dmem_kernel<<<(NB + R + 7) / 8, 256, 0, s>>>(w.dZmp, w.dcat_o, w.dzq, ctx->e_nbr, ctx->e_nodes, R, k, d,
                                                                w.node2slot, w.dMemU, c.num_nodes);
+        }
       }
       TGNN_LAUNCH_OK(ctx, "scatter_dmem");
       const int U_cap = ctx->upd_cap;
