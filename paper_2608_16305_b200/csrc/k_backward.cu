@@ -692,11 +692,11 @@ __global__ void __launch_bounds__(256) scatter_dmem_kernel(const float* __restri
 // resolves row -> node -> slot and files the row under one of SC_WAYS lists (a list belongs to the first slot that
 // claims it by compare-and-swap; a row whose list belongs to another slot goes to a list of singles).  The lists
 // are then laid end to end, so that rows of one slot are neighbours, and every warp walks an equal share of that
-// sequence, 8 / U row loads in flight: it sums in registers while the slot stays the same and adds the sum to
+// sequence, 6 / U row loads in flight: it sums in registers while the slot stays the same and adds the sum to
 // dMemU when it changes.  Rows whose node was not updated are never read.
 constexpr int SC_ROWS = 256, SC_WAYS = 32;  // 256 rows, 256 threads: the whole batch is one wave of blocks
 template <int U>  // 16-byte pieces of a row per lane: 1 (d <= 128) or 2
-__global__ void __launch_bounds__(256, 4) scatter_dmem_cached_kernel(const float* __restrict__ dZm,
+__global__ void __launch_bounds__(256, 5) scatter_dmem_cached_kernel(const float* __restrict__ dZm,
                                                                      const float* __restrict__ dcat_o,
                                                                      const float* __restrict__ dzq,
                                                                      const int32_t* __restrict__ nbr,
@@ -746,7 +746,7 @@ __global__ void __launch_bounds__(256, 4) scatter_dmem_cached_kernel(const float
   const int n_live = s_off[SC_WAYS] + s_cnt[SC_WAYS];
   const int share = (n_live + 7) >> 3;
   const int e_end = min(n_live, (wid + 1) * share);
-  constexpr int V = 8 / U;
+  constexpr int V = 6 / U;  // (48 registers: five blocks share an SM, or fewer beside a persistent product)
   int cur = -1;
   float4 acc[U];
 #pragma unroll
@@ -815,7 +815,8 @@ inline int tg_rows_per_block(int rows) {
   const int r = (rows + 295) / 296;
   return r < 8 ? 8 : (r + 7) / 8 * 8;
 }
-__global__ void __launch_bounds__(256, 2) time_grad_kernel(const float* __restrict__ G, int64_t ldg, int col0,
+template <int V>  // 16-byte column pieces per lane: 1 (d <= 128: half the registers, four blocks share an SM) or 2
+__global__ void __launch_bounds__(256, V == 1 ? 4 : 2) time_grad_kernel(const float* __restrict__ G, int64_t ldg, int col0,
                                                         const float* __restrict__ S, const float* __restrict__ dt,
                                                         int rows, const int32_t* __restrict__ dev_rows, int d,
                                                         const float* __restrict__ time_w,
@@ -826,15 +827,15 @@ __global__ void __launch_bounds__(256, 2) time_grad_kernel(const float* __restri
   const int r0 = blockIdx.x * rows_per_block, r1 = min(R, r0 + rows_per_block);
   if (r0 >= r1) return;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  // a lane owns columns 4 (lane + 32 v) .. + 3, v = 0, 1 (d <= 256): 128-bit loads of G and S (d, ldg and col0 are
+  // a lane owns columns 4 (lane + 32 v) .. + 3, v < V (d <= 128 V): 128-bit loads of G and S (d, ldg and col0 are
   // multiples of 4 and the rows 16-byte aligned)
   // Sines: saved rows S; or (S null, dt given) recomputed from the row's dt exactly as the forward pass formed
   // them -- a row with dt < 0 is an empty slot and contributes nothing; or (both null) the constant sin(b) of dt = 0.
-  double gw[2][4], gb[2][4];
-  float4 sb[2], wv[2], bv[2];
+  double gw[V][4], gb[V][4];
+  float4 sb[V], wv[V], bv[V];
   const bool recompute = S == nullptr && dt != nullptr;
 #pragma unroll
-  for (int v = 0; v < 2; ++v) {
+  for (int v = 0; v < V; ++v) {
     const int c = 4 * (lane + 32 * v);
 #pragma unroll
     for (int e = 0; e < 4; ++e) { gw[v][e] = 0.0; gb[v][e] = 0.0; }
@@ -846,7 +847,7 @@ __global__ void __launch_bounds__(256, 2) time_grad_kernel(const float* __restri
     }
   }
   for (int rb = r0 + wid; rb < r1; rb += 8 * TG_U) {  // rows rb, rb + 8, ...: loads first, sums after
-    float4 g[TG_U][2], sn[TG_U][2];
+    float4 g[TG_U][V], sn[TG_U][V];
     float dtr[TG_U];
 #pragma unroll
     for (int u = 0; u < TG_U; ++u) {
@@ -854,7 +855,7 @@ __global__ void __launch_bounds__(256, 2) time_grad_kernel(const float* __restri
       const bool in = r < r1;
       dtr[u] = (in && dt) ? dt[r] : 0.f;
 #pragma unroll
-      for (int v = 0; v < 2; ++v) {
+      for (int v = 0; v < V; ++v) {
         const int c = 4 * (lane + 32 * v);
         const bool ok = in && c < d;
         g[u][v] = ok ? __ldg(reinterpret_cast<const float4*>(G + (int64_t)r * ldg + col0 + c)) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -866,7 +867,7 @@ __global__ void __launch_bounds__(256, 2) time_grad_kernel(const float* __restri
       for (int u = 0; u < TG_U; ++u) {
         const bool live = rb + 8 * u < r1 && dtr[u] >= 0.f;
 #pragma unroll
-        for (int v = 0; v < 2; ++v) {
+        for (int v = 0; v < V; ++v) {
           const int c = 4 * (lane + 32 * v);
           float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
           if (live && c < d) {
@@ -883,7 +884,7 @@ __global__ void __launch_bounds__(256, 2) time_grad_kernel(const float* __restri
 #pragma unroll
     for (int u = 0; u < TG_U; ++u) {
 #pragma unroll
-      for (int v = 0; v < 2; ++v) {
+      for (int v = 0; v < V; ++v) {
         const float ge[4] = {g[u][v].x, g[u][v].y, g[u][v].z, g[u][v].w};
         const float se[4] = {sn[u][v].x, sn[u][v].y, sn[u][v].z, sn[u][v].w};
 #pragma unroll
@@ -896,7 +897,7 @@ __global__ void __launch_bounds__(256, 2) time_grad_kernel(const float* __restri
     }
   }
 #pragma unroll
-  for (int v = 0; v < 2; ++v) {
+  for (int v = 0; v < V; ++v) {
     const int c = 4 * (lane + 32 * v);
     if (c < d) {
 #pragma unroll
@@ -909,6 +910,15 @@ __global__ void __launch_bounds__(256, 2) time_grad_kernel(const float* __restri
     for (int w = 0; w < 8; ++w) t += s_part[w * 2 * d + e];
     if (t != 0.0) atomicAdd(&acc[e], t);
   }
+}
+
+inline void time_grad_launch(int grid, size_t smem, cudaStream_t st, const float* G, int64_t ldg, int col0, const float* S,
+                             const float* dt, int rows, const int32_t* dev_rows, int d, const float* time_w,
+                             const float* time_b, double* acc, int rows_per_block) {
+  if (d <= 128)
+    time_grad_kernel<1><<<grid, 256, smem, st>>>(G, ldg, col0, S, dt, rows, dev_rows, d, time_w, time_b, acc, rows_per_block);
+  else
+    time_grad_kernel<2><<<grid, 256, smem, st>>>(G, ldg, col0, S, dt, rows, dev_rows, d, time_w, time_b, acc, rows_per_block);
 }
 
 // Backward of the time-projected embedding h = m * (1 + dt w_p + b_p), one warp per root:
@@ -1330,7 +1340,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
         {
           KernelScope scope__(ctx, "time_grad_x", s);
           const int rpb = tg_rows_per_block(U_cap);
-          time_grad_kernel<<<(U_cap + rpb - 1) / rpb, 256, tg_smem, s>>>(w.dXp, d, 0, w.Xsin, w.x_dt, U_cap,
+          time_grad_launch((U_cap + rpb - 1) / rpb, tg_smem, s, w.dXp, d, 0, w.Xsin, w.x_dt, U_cap,
                                                                          ctx->upd_n_uniq, d, P + L.time_w, P + L.time_b, w.tg_acc, rpb);
         }
         TGNN_LAUNCH_OK(ctx, "time_grad_x");
@@ -1381,7 +1391,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     {
       KernelScope scope__(ctx, "time_grad_q", sb);
       const int rpb = tg_rows_per_block(R);
-      time_grad_kernel<<<(R + rpb - 1) / rpb, 256, tg_smem, sb>>>(w.dzq, 2 * d, d, nullptr, nullptr, R, nullptr, d,
+      time_grad_launch((R + rpb - 1) / rpb, tg_smem, sb, w.dzq, 2 * d, d, nullptr, nullptr, R, nullptr, d,
                                                                   P + L.time_w, P + L.time_b, w.tg_acc, rpb);
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_q");
@@ -1421,7 +1431,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     {
       KernelScope scope__(ctx, "time_grad_z", s_tgz);
       const int rpb = tg_rows_per_block(NB);
-      time_grad_kernel<<<(NB + rpb - 1) / rpb, 256, tg_smem, s_tgz>>>(w.dZmp, 2 * d, d, nullptr, w.z_dt, NB, nullptr, d, P + L.time_w,
+      time_grad_launch((NB + rpb - 1) / rpb, tg_smem, s_tgz, w.dZmp, 2 * d, d, nullptr, w.z_dt, NB, nullptr, d, P + L.time_w,
                                                                       P + L.time_b, w.tg_acc, rpb);
     }
     TGNN_LAUNCH_OK(ctx, "time_grad_z");
@@ -1464,7 +1474,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
       {
         KernelScope scope__(ctx, "time_grad_x", s);
         const int rpb = tg_rows_per_block(U_cap);
-        time_grad_kernel<<<(U_cap + rpb - 1) / rpb, 256, tg_smem, s>>>(w.dXp, d, 0, w.Xsin, w.x_dt, U_cap, ctx->upd_n_uniq,
+        time_grad_launch((U_cap + rpb - 1) / rpb, tg_smem, s, w.dXp, d, 0, w.Xsin, w.x_dt, U_cap, ctx->upd_n_uniq,
                                                                        d, P + L.time_w, P + L.time_b, w.tg_acc, rpb);
       }
       TGNN_LAUNCH_OK(ctx, "time_grad_x");

@@ -759,7 +759,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
 // own 128 columns of A (its rows of C) once, and from B only the 128 columns per accumulator that are its half of
 // the MMA's B tile: every operand byte is fetched by exactly one CTA of the pair, where the single-CTA kernel
 // fetches A once per n-tile.  Barriers and bounded waits as in gemm_split_pair_kernel.
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_split_pair_mn_kernel(const __grid_constant__ BfArgs g) {
+// EPI epilogue warps (4 or 8): a unit's accumulators are drained once, at the end of a long contraction, so four warps
+// (one per tensor-memory lane quarter) cost little -- and the CTA then holds 6 warps' registers instead of 10, which
+// leaves room on every SM sub-partition for blocks of the kernels that run beside it.
+template <int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(32 * (2 + EPI), 1) gemm_split_pair_mn_kernel(const __grid_constant__ BfArgs g) {
+  static_assert(EPI == 4 || EPI == 8, "one or two warps per lane quarter");
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t s_full[MAX_SLOTS], s_empty[MAX_SLOTS];
   __shared__ __align__(8) uint64_t s_tmem_full, s_tmem_empty;
@@ -779,7 +784,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
       mbar_init(smem_u32(&s_empty[s]), 1);
     }
     mbar_init(smem_u32(&s_tmem_full), 1);
-    mbar_init(smem_u32(&s_tmem_empty), 2 * EPI_WARPS);
+    mbar_init(smem_u32(&s_tmem_empty), 2 * EPI);
     s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -895,7 +900,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
   } else {
     // ------------------------------------------------------------ epilogue (each CTA its own 128 rows)
     const int e = warp - 2;
-    const int t = e >> 2;          // warps 2-5 drain the first accumulator, 6-9 the second (all eight the only one)
+    const int t = e >> 2;          // EPI = 8: warps 2-5 drain the first accumulator, 6-9 the second (all eight the only one)
     const int q4 = warp & 3;
     float* stg = stg_base + e * (STG_WARP_BYTES / 4);
     const bool c_vec = (((uintptr_t)g.C & 15) == 0) && (g.ldc % 4 == 0);
@@ -913,13 +918,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1) gemm_spl
       ++n_item;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int m0 = (2 * ms + (int)rank) * BM;
-      const int j = n_sub == 2 ? t : 0;
-      Item it;
-      it.mt0 = ms; it.tiles = 1; it.kb0 = kb0; it.kb1 = kb1;
-      it.n0 = j * 256;
-      it.n_valid = min(256, g.N - it.n0);
-      const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(j * ACC_STRIDE);
-      drain_tile(g, it, m0, taddr, n_sub == 2 ? 0 : 32 * t, n_sub == 2 ? 32 : 64, stg, lane, q4, c_vec);
+      for (int j = (EPI == 8 && n_sub == 2) ? t : 0; j < n_sub; ++j) {
+        Item it;
+        it.mt0 = ms; it.tiles = 1; it.kb0 = kb0; it.kb1 = kb1;
+        it.n0 = j * 256;
+        it.n_valid = min(256, g.N - it.n0);
+        const uint32_t taddr = tmem + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(j * ACC_STRIDE);
+        if (EPI == 8) {
+          drain_tile(g, it, m0, taddr, n_sub == 2 ? 0 : 32 * t, n_sub == 2 ? 32 : 64, stg, lane, q4, c_vec);
+          break;
+        }
+        drain_tile(g, it, m0, taddr, 0, 32, stg, lane, q4, c_vec);
+      }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (e == 0 && lane == 0) TRACE(1 + 2 * (int)n_item);
@@ -1225,11 +1235,11 @@ int launch_gemm_split(tgnn_ctx* ctx, const SplitMat& A, const SplitMat& B, int m
       const int clusters = units < 74 ? units : 74;
       const int smem = 1024 + b.n_stages * b.stage_bytes + STG_BYTES;
       static SmemLimit pair_mn_limit;
-      const int rc = raise_smem_limit(ctx, gemm_split_pair_mn_kernel, SMEM_LIMIT - 1024, pair_mn_limit);
+      const int rc = raise_smem_limit(ctx, gemm_split_pair_mn_kernel<4>, SMEM_LIMIT - 1024, pair_mn_limit);
       if (rc) return rc;
       {
         KernelScope scope__(ctx, name, s);
-        gemm_split_pair_mn_kernel<<<2 * clusters, THREADS, smem, s>>>(b);
+        gemm_split_pair_mn_kernel<4><<<2 * clusters, 32 * (2 + 4), smem, s>>>(b);
       }
       TGNN_LAUNCH_OK(ctx, name);
       return TGNN_OK;

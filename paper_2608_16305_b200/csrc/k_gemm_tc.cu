@@ -864,9 +864,13 @@ int launch_gemm_tf32(tgnn_ctx* ctx, const GemmArgs& g, const char* name, cudaStr
   }
   // whole-chunk operands: 16-byte aligned rows, and the dimension the 16-byte chunks run along is a
   // multiple of 4 and known on the host
-  const auto whole = [](const float* p, int64_t ld, int major, int k, const int* dev_k, int mn, const int* dev_mn) {
+  // (An MN-major operand of a workspace buffer may end inside a chunk when its row pitch covers the chunk: the
+  // values read past the end only reach rows or columns of C beyond M or N, which are not stored.)
+  const bool slack = g.tail_slack != 0;
+  const auto whole = [slack](const float* p, int64_t ld, int major, int k, const int* dev_k, int mn, const int* dev_mn) {
     if (((uintptr_t)p & 15) != 0 || ld % 4 != 0) return false;
-    return major == MAJOR_K ? (k % 4 == 0 && dev_k == nullptr) : (mn % 4 == 0 && dev_mn == nullptr);
+    return major == MAJOR_K ? (k % 4 == 0 && dev_k == nullptr)
+                            : ((mn % 4 == 0 || (slack && (mn + 3) / 4 * 4 <= ld)) && dev_mn == nullptr);
   };
   const bool fast = whole(a.A, a.lda, a.a_major, a.K, a.dev_K, a.M, a.dev_M) &&
                     (a.b_image != nullptr || whole(a.B, a.ldb, a.b_major, a.K, a.dev_K, a.N, nullptr));
