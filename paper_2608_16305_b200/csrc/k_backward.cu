@@ -1220,7 +1220,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
   // sequential and stays on the caller's stream s.  Weight-gradient products and time-encoder sums
   // are leaves of that chain: they go to the two side streams as soon as their operands exist and
   // are joined back before the gradient norm.
-  cudaStream_t sa = ctx->side[0], sb = ctx->side[1], sc = ctx->side[2];
+  cudaStream_t sa = ctx->side[0], sb = ctx->side[1], sc = ctx->side[2], sd = ctx->side[3];
   // grads | dMemU | red | tg_acc | st_scalars are contiguous in the arena: one memset clears them all
   if (!ctx->grads_zeroed) {
     const size_t zero_bytes = (size_t)((char*)(w.st_scalars + 4) - (char*)w.grads);
@@ -1463,10 +1463,12 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
                                                                       w.g_hn, ctx->upd_n_uniq, U_cap, w.dGi, w.dGh);
       }
       TGNN_LAUNCH_OK(ctx, "gru_bwd_gate");
-      RC(fork_to(ctx, s, sa));
+      // (split mode: side stream a carries the persistent key/value weight gradient, which ends late)
+      cudaStream_t s_wi = split ? sd : sa;
+      RC(fork_to(ctx, s, s_wi));
       RC(fork_to(ctx, s, sb));
       RC(grad_w(ctx, w.dGi, 3 * d, w.X, ctx->ld_msg, U_cap, ctx->upd_n_uniq, 3 * d, (int)L.dmsg, G + L.gru_wi,
-                G + L.gru_bi, "dW_i", sa));
+                G + L.gru_bi, "dW_i", s_wi));
       RC(grad_w(ctx, w.dGh, 3 * d, w.X, ctx->ld_msg, U_cap, ctx->upd_n_uniq, 3 * d, d, G + L.gru_wh, G + L.gru_bh,
                 "dW_h", sb));
       RC(grad_in(ctx, w.dGi, 3 * d, P + L.gru_wi, L.dmsg, 2 * d + de, U_cap, ctx->upd_n_uniq, 3 * d, d, w.dXp, d,
@@ -1478,6 +1480,7 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
                                                                        d, P + L.time_w, P + L.time_b, w.tg_acc, rpb);
       }
       TGNN_LAUNCH_OK(ctx, "time_grad_x");
+      if (split) RC(fork_to(ctx, sd, s));  // join
     }
     RC(fork_to(ctx, sa, s));  // join
     RC(fork_to(ctx, sb, s));

@@ -690,8 +690,9 @@ __global__ void __launch_bounds__(Cfg<BN_T, PRECISE, TMA>::THREADS, 1) gemm_tf32
 void tile_plan(int M, int N, bool split_accumulate, int* n_tiles, int* bn) {
   int nt = (N + 255) / 256;
   const int m_tiles = (M + BM - 1) / BM;
+  // (only while the narrower tiles still make one wave of CTAs: a CTA takes a whole SM)
   if (!split_accumulate)
-    while (m_tiles * nt < 96 && ((N + nt - 1) / nt + 31) / 32 * 32 > 64) ++nt;
+    while (m_tiles * (nt + 1) <= 148 && ((N + nt - 1) / nt + 31) / 32 * 32 > 64) ++nt;
   *n_tiles = nt;
   *bn = ((N + nt - 1) / nt + 31) / 32 * 32;
 }

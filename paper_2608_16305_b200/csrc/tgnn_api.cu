@@ -305,7 +305,7 @@ int tgnn_create(const tgnn_config* cfg, tgnn_ctx** out) {
     // chain (the caller's stream) gets the next free SM slots when both have blocks waiting
     int least = 0, greatest = 0;
     ok = ok && cudaDeviceGetStreamPriorityRange(&least, &greatest) == cudaSuccess;
-    for (int i = 0; ok && i < 3; ++i)
+    for (int i = 0; ok && i < 4; ++i)
       ok = cudaStreamCreateWithPriority(&ctx->side[i], cudaStreamNonBlocking, least) == cudaSuccess;
   }
   for (int i = 0; ok && i < 32; ++i) ok = cudaEventCreateWithFlags(&ctx->ev[i], cudaEventDisableTiming) == cudaSuccess;
@@ -337,7 +337,7 @@ int tgnn_destroy(tgnn_ctx* ctx) {
   }
   for (int i = 0; i < ctx->n_graphs; ++i)
     if (ctx->graphs[i].exec) cudaGraphExecDestroy(ctx->graphs[i].exec);
-  for (int i = 0; i < 3; ++i) cudaStreamDestroy(ctx->side[i]);
+  for (int i = 0; i < 4; ++i) cudaStreamDestroy(ctx->side[i]);
   for (int i = 0; i < 32; ++i) cudaEventDestroy(ctx->ev[i]);
   cudaEventDestroy(ctx->ev_search); cudaEventDestroy(ctx->ev_side_done);
   cudaFree(ctx->images);
@@ -493,11 +493,11 @@ int step_body(tgnn_ctx* ctx, int n_u, bool has_keep, int n_q, bool has_mask, flo
   // launch then times that kernel alone instead of the kernel plus whatever shares the machine with it.
   struct SideGuard {
     tgnn_ctx* c;
-    cudaStream_t s0, s1, s2;
-    SideGuard(tgnn_ctx* c_, cudaStream_t main) : c(c_), s0(c_->side[0]), s1(c_->side[1]), s2(c_->side[2]) {
-      if (c->prof.on) c->side[0] = c->side[1] = c->side[2] = main;
+    cudaStream_t s0, s1, s2, s3;
+    SideGuard(tgnn_ctx* c_, cudaStream_t main) : c(c_), s0(c_->side[0]), s1(c_->side[1]), s2(c_->side[2]), s3(c_->side[3]) {
+      if (c->prof.on) c->side[0] = c->side[1] = c->side[2] = c->side[3] = main;
     }
-    ~SideGuard() { c->side[0] = s0; c->side[1] = s1; c->side[2] = s2; }
+    ~SideGuard() { c->side[0] = s0; c->side[1] = s1; c->side[2] = s2; c->side[3] = s3; }
   } side_guard(ctx, S(stream));
   // the weights' B-operand images for this step's projections: written beside the first kernels
   const bool prep = ctx->images != nullptr;

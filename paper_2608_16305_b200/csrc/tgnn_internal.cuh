@@ -201,8 +201,9 @@ struct tgnn_ctx {
   // Two internal streams for kernels that do not lie on the step's critical chain (weight-gradient
   // products, the neighbor search next to the memory update, ...).  They are forked from and joined
   // back into the caller's stream with events, so the caller still sees one ordered stream of work.
-  cudaStream_t side[3];   // [2]: the time-encoder sum over the neighbor rows in the split mode (it must not queue behind
-                          // products that wait for a whole SM's shared memory)
+  cudaStream_t side[4];   // [2]: the time-encoder sum over the neighbor rows in the split mode (it must not queue behind
+                          // products that wait for a whole SM's shared memory); [3]: the update cell's input-weight
+                          // gradient in that mode (it must not queue behind the persistent weight gradient on [0])
   cudaEvent_t ev[32];
   // tgnn_train_step's side stream, recorded after the neighbor search and after everything else it carries (the static
   // half of the attention inputs, the clear of the gradient block); the embedding waits for each where it first
