@@ -198,7 +198,7 @@ struct tgnn_ctx {
   tgnn::Workspace ws;
   void* arena;
   size_t arena_bytes;
-  // Two internal streams for kernels that do not lie on the step's critical chain (weight-gradient
+  // Internal streams for kernels that do not lie on the step's critical chain (weight-gradient
   // products, the neighbor search next to the memory update, ...).  They are forked from and joined
   // back into the caller's stream with events, so the caller still sees one ordered stream of work.
   cudaStream_t side[4];   // [2]: the time-encoder sum over the neighbor rows in the split mode (it must not queue behind
