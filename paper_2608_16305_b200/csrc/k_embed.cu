@@ -433,6 +433,94 @@ __global__ void __launch_bounds__(256) attention_fwd_kernel(const float* __restr
   }
 }
 
+// The same kernel for compile-time shapes (D columns, H heads, KS slots; D / H even, H * KS <= 32): the generic
+// kernel above spends 1 900 instructions per root, mostly loop control and scalar shared-memory loads, and is bound
+// by instruction issue.  Here the dot products read pairs of columns, the exponentials are formed once per (head,
+// slot) and shared through shared memory, and the weighted sum of V runs on four columns per lane.  Every sum keeps
+// the generic kernel's order of operations, so the two give the same bits.
+template <int D, int H, int KS>
+__global__ void __launch_bounds__(256) attention_fwd_fixed_kernel(const float* __restrict__ Q, const float* __restrict__ KV,
+                                                                  const int32_t* __restrict__ cnt, int n,
+                                                                  float* __restrict__ alpha, float* __restrict__ cat_o) {
+  constexpr int DH = D / H, D4 = D / 4, P = H * KS;
+  static_assert(D % 4 == 0 && DH % 2 == 0 && P <= 32 && D4 <= 32, "shape not covered by the fixed kernel");
+  extern __shared__ __align__(16) float sm[];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int i = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+  if (i >= n) return;
+  float* Ks = sm + wib * attn_warp_floats(D, H, KS);
+  float* Vs = Ks + KS * D;
+  float* Qs = Vs + KS * D;
+  float* al = Qs + 2 * D;  // logits
+  float* pr = al + P;      // exponentials, then probabilities
+  const int c = max(0, min(cnt[i], KS));   // a count outside [0, k] is clamped (the neighbor search never produces one)
+  const float scale = rsqrtf((float)DH);
+  {
+    const float* q = Q + (int64_t)i * D;
+    if (lane < D4) cp_async16(Qs + 4 * lane, q + 4 * lane);
+    const float* kv = KV + (int64_t)i * KS * 2 * D;
+    for (int e = lane; e < c * 2 * D4; e += 32) {
+      const int sl = e / (2 * D4), r = e - sl * 2 * D4;
+      cp_async16(r < D4 ? Ks + sl * D + 4 * r : Vs + sl * D + 4 * (r - D4), kv + 4 * e);
+    }
+  }
+  attn_stage_wait();
+  const int h = lane / KS, sl = lane - h * KS;
+  const bool live = lane < P && sl < c;
+  float a = 0.f;
+  if (live) {
+    const float2* kr = reinterpret_cast<const float2*>(Ks + sl * D + h * DH);
+    const float2* qr = reinterpret_cast<const float2*>(Qs + h * DH);
+#pragma unroll
+    for (int e = 0; e < DH / 2; ++e) {
+      const float2 qv = qr[e], kv2 = kr[e];
+      a = fmaf(qv.x, kv2.x, a);
+      a = fmaf(qv.y, kv2.y, a);
+    }
+    a *= scale;
+  }
+  if (lane < P) al[lane] = a;
+  __syncwarp();
+  float ex = 0.f;
+  if (live) {
+    float mx = -INFINITY;
+#pragma unroll
+    for (int t = 0; t < KS; ++t)
+      if (t < c) mx = fmaxf(mx, al[h * KS + t]);
+    ex = expf(a - mx);
+  }
+  if (lane < P) pr[lane] = ex;
+  __syncwarp();
+  float out = 0.f;
+  if (live) {
+    float den = 0.f;
+#pragma unroll
+    for (int t = 0; t < KS; ++t)
+      if (t < c) den += pr[h * KS + t];
+    out = ex / den;
+  }
+  __syncwarp();   // every lane has read the exponentials
+  if (lane < P) {
+    pr[lane] = out;
+    alpha[(int64_t)i * P + lane] = out;
+  }
+  __syncwarp();
+  if (lane < D4) {
+    const int h0 = (4 * lane) / DH, h1 = (4 * lane + 2) / DH;   // columns 4l, 4l+1 share a head, and so do 4l+2, 4l+3
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int t = 0; t < KS; ++t) {
+      if (t < c) {
+        const float p0 = pr[h0 * KS + t], p1 = pr[h1 * KS + t];
+        const float4 v = *reinterpret_cast<const float4*>(Vs + t * D + 4 * lane);
+        acc.x = fmaf(p0, v.x, acc.x); acc.y = fmaf(p0, v.y, acc.y);
+        acc.z = fmaf(p1, v.z, acc.z); acc.w = fmaf(p1, v.w, acc.w);
+      }
+    }
+    *reinterpret_cast<float4*>(cat_o + (int64_t)i * 2 * D + 4 * lane) = acc;
+  }
+}
+
 // Time-projected embedding: h[i] = memory[node_i] * (1 + dt_i w_p + b_p), dt_i = fp32(t_i - last_update[node_i]).
 // One warp per root, 128-bit accesses (d is a multiple of 4, rows 16-byte aligned).
 __global__ void __launch_bounds__(256) jodie_embed_kernel(const float* __restrict__ memory,
@@ -606,11 +694,17 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
   rc = fork_to(ctx, ctx->side[0], s);
   if (rc) return rc;
   const int wpb = attn_warps_per_block(d, H, k);
-  RC_ATTR(ctx, attention_fwd_kernel, attn_smem_bytes(d, H, k, wpb));
+  const bool fixed_shape = d == 100 && H == 2 && k == 10;   // the paper's configuration
+  if (fixed_shape) RC_ATTR(ctx, (attention_fwd_fixed_kernel<100, 2, 10>), attn_smem_bytes(d, H, k, wpb));
+  else RC_ATTR(ctx, attention_fwd_kernel, attn_smem_bytes(d, H, k, wpb));
   {
     KernelScope scope__(ctx, "attention_fwd", s);
-    attention_fwd_kernel<<<(n + wpb - 1) / wpb, wpb * 32, attn_smem_bytes(d, H, k, wpb), s>>>(w.Q, w.KV, cnt, n, d, H, k,
-                                                                                           w.alpha, w.cat_o);
+    if (fixed_shape)
+      attention_fwd_fixed_kernel<100, 2, 10><<<(n + wpb - 1) / wpb, wpb * 32, attn_smem_bytes(d, H, k, wpb), s>>>(w.Q, w.KV, cnt, n,
+                                                                                                              w.alpha, w.cat_o);
+    else
+      attention_fwd_kernel<<<(n + wpb - 1) / wpb, wpb * 32, attn_smem_bytes(d, H, k, wpb), s>>>(w.Q, w.KV, cnt, n, d, H, k,
+                                                                                             w.alpha, w.cat_o);
   }
   TGNN_LAUNCH_OK(ctx, "attention_fwd");
   g = GemmArgs{};
