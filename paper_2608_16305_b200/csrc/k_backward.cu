@@ -641,6 +641,103 @@ __global__ void __launch_bounds__(256) attention_bwd_kernel(const float* __restr
   }
 }
 
+// The split form of the kernel above for compile-time shapes (D columns, H heads, KS slots; D / H even, H * KS <= 32,
+// D <= 128).  The generic kernel is bound by instruction issue (2 800 instructions per root: loop control, scalar
+// shared-memory loads, 32-bit plane stores); here the dot products read pairs of columns, a lane owns four
+// neighbouring columns of the key / value gradient rows and writes them as one 64-bit word per plane and row.  Every
+// sum keeps the generic kernel's order of operations.
+template <int D, int H, int KS>
+__global__ void __launch_bounds__(256) attention_bwd_fixed_kernel(const float* __restrict__ Q, const float* __restrict__ KV,
+                                                                  const float* __restrict__ alpha,
+                                                                  const float* __restrict__ dcat_o,
+                                                                  const int32_t* __restrict__ cnt, int n,
+                                                                  float* __restrict__ dQ, __nv_bfloat16* __restrict__ dkv_hi,
+                                                                  int64_t plane_s, int ld_s, float gscale) {
+  constexpr int DH = D / H, D4 = D / 4, P = H * KS;
+  static_assert(D % 4 == 0 && DH % 2 == 0 && P <= 32 && D4 <= 32, "shape not covered by the fixed kernel");
+  extern __shared__ __align__(16) float sm[];
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int i = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
+  if (i >= n) return;
+  float* Ks = sm + wib * attn_warp_floats(D, H, KS);
+  float* Vs = Ks + KS * D;
+  float* Qs = Vs + KS * D;
+  float* das = Qs + D;       // d loss / d a
+  float* al = das + D;       // probabilities
+  float* dal = al + P;       // d loss / d probability
+  float* dl = dal + P;       // d loss / d logit, already scaled
+  const int c = max(0, min(cnt[i], KS));
+  const float scale = rsqrtf((float)DH);
+  {
+    const float* q = Q + (int64_t)i * D;
+    const float* g = dcat_o + (int64_t)i * 2 * D;
+    if (lane < D4) {
+      cp_async16(Qs + 4 * lane, q + 4 * lane);
+      cp_async16(das + 4 * lane, g + 4 * lane);
+    }
+    const float* kv = KV + (int64_t)i * KS * 2 * D;
+    for (int e = lane; e < c * 2 * D4; e += 32) {
+      const int sl = e / (2 * D4), r = e - sl * 2 * D4;
+      cp_async16(r < D4 ? Ks + sl * D + 4 * r : Vs + sl * D + 4 * (r - D4), kv + 4 * e);
+    }
+    if (lane < P) al[lane] = alpha[(int64_t)i * P + lane];
+  }
+  attn_stage_wait();
+  const int h = lane / KS, sl = lane - h * KS;
+  const bool live = lane < P && sl < c;
+  float a = 0.f;
+  if (live) {
+    const float2* vr = reinterpret_cast<const float2*>(Vs + sl * D + h * DH);
+    const float2* gr = reinterpret_cast<const float2*>(das + h * DH);
+#pragma unroll
+    for (int e = 0; e < DH / 2; ++e) {
+      const float2 gv = gr[e], vv = vr[e];
+      a = fmaf(gv.x, vv.x, a);
+      a = fmaf(gv.y, vv.y, a);
+    }
+  }
+  if (lane < P) dal[lane] = a;
+  __syncwarp();
+  float gl = 0.f;
+  if (live) {
+    float dot = 0.f;
+#pragma unroll
+    for (int t = 0; t < KS; ++t)
+      if (t < c) dot = fmaf(al[h * KS + t], dal[h * KS + t], dot);
+    gl = al[lane] * (a - dot) * scale;
+  }
+  if (lane < P) dl[lane] = gl;
+  __syncwarp();
+  if (lane < D4) {
+    const int h0 = (4 * lane) / DH, h1 = (4 * lane + 2) / DH;   // columns 4l, 4l+1 share a head, and so do 4l+2, 4l+3
+    const float4 q4 = *reinterpret_cast<const float4*>(Qs + 4 * lane);
+    const float4 a4 = *reinterpret_cast<const float4*>(das + 4 * lane);
+    float4 dq = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int t = 0; t < KS; ++t) {
+      __nv_bfloat16* hi_row = dkv_hi + ((int64_t)i * KS + t) * ld_s + 4 * lane;
+      __nv_bfloat16* lo_row = hi_row + plane_s;
+      uint2 kh = make_uint2(0u, 0u), kl = kh, vh = kh, vl = kh;
+      if (t < c) {
+        const float g0 = dl[h0 * KS + t], g1 = dl[h1 * KS + t];
+        const float p0 = al[h0 * KS + t], p1 = al[h1 * KS + t];
+        const float4 kv4 = *reinterpret_cast<const float4*>(Ks + t * D + 4 * lane);
+        dq.x = fmaf(g0, kv4.x, dq.x); dq.y = fmaf(g0, kv4.y, dq.y);
+        dq.z = fmaf(g1, kv4.z, dq.z); dq.w = fmaf(g1, kv4.w, dq.w);
+        split_f16_pair(g0 * q4.x * gscale, g0 * q4.y * gscale, &kh.x, &kl.x);
+        split_f16_pair(g1 * q4.z * gscale, g1 * q4.w * gscale, &kh.y, &kl.y);
+        split_f16_pair(p0 * a4.x * gscale, p0 * a4.y * gscale, &vh.x, &vl.x);
+        split_f16_pair(p1 * a4.z * gscale, p1 * a4.w * gscale, &vh.y, &vl.y);
+      }
+      *reinterpret_cast<uint2*>(hi_row) = kh;
+      *reinterpret_cast<uint2*>(lo_row) = kl;
+      *reinterpret_cast<uint2*>(hi_row + D) = vh;
+      *reinterpret_cast<uint2*>(lo_row + D) = vl;
+    }
+    *reinterpret_cast<float4*>(dQ + (int64_t)i * D + 4 * lane) = dq;
+  }
+}
+
 // Gradient rows flowing into memory rows that the last memory update wrote: one warp per
 // source row, added into dMemU[node2slot[node]].  Rows [0, nb_rows): dZm with node = nbr;
 // rows [nb_rows, nb_rows + n): the root's own row, dcat_o[:, d:] + dzq[:, :d].
@@ -1353,17 +1450,24 @@ int launch_backward(tgnn_ctx* ctx, int n_q, const uint8_t* loss_mask, float* los
     RC(grad_in(ctx, w.dpre_o, d, P + L.wo, 2 * d, 0, R, nullptr, d, 2 * d, w.dcat_o, 2 * d, "dcat_o", s, SITE_DCATO + 1));
     const int wpb = attn_warps_per_block(d, H, k);
     {
-      static SmemLimit lim_f, lim_t;
+      static SmemLimit lim_f, lim_t, lim_x;
       const int need = (int)attn_smem_bytes(d, H, k, wpb);
       RC(raise_smem_limit(ctx, attention_bwd_kernel<false>, need, lim_f));
       RC(raise_smem_limit(ctx, attention_bwd_kernel<true>, need, lim_t));
+      if (d == 100 && H == 2 && k == 10) RC(raise_smem_limit(ctx, (attention_bwd_fixed_kernel<100, 2, 10>), need, lim_x));
     }
     const bool split = ctx->split_buf != nullptr && ctx->images_fresh;
     SplitMat dkvs = ctx->dkvs, zs = ctx->zs;
     dkvs.rows = NB; zs.rows = NB;
     {
       KernelScope scope__(ctx, "attention_bwd", s);
-      if (split)   // the key/value gradient leaves the kernel as fp16 planes, the form its two consumers read
+      // (8-byte plane stores: row pitch and plane distance multiples of 4 elements)
+      const bool fixed_shape = split && d == 100 && H == 2 && k == 10 && dkvs.ld % 4 == 0 && dkvs.plane_stride % 4 == 0;
+      if (fixed_shape)   // the paper's configuration
+        attention_bwd_fixed_kernel<100, 2, 10><<<(R + wpb - 1) / wpb, wpb * 32, attn_smem_bytes(d, H, k, wpb), s>>>(
+            w.Q, w.KV, w.alpha, w.dcat_o, ctx->e_cnt, R, w.dQ, reinterpret_cast<__nv_bfloat16*>(dkvs.hi), dkvs.plane_stride,
+            (int)dkvs.ld, dkvs.scale);
+      else if (split)   // the key/value gradient leaves the kernel as fp16 planes, the form its two consumers read
         attention_bwd_kernel<true><<<(R + wpb - 1) / wpb, wpb * 32, attn_smem_bytes(d, H, k, wpb), s>>>(
             w.Q, w.KV, w.alpha, w.dcat_o, ctx->e_cnt, R, d, H, k, w.dQ, nullptr, reinterpret_cast<__nv_bfloat16*>(dkvs.hi),
             dkvs.plane_stride, (int)dkvs.ld, dkvs.scale);
