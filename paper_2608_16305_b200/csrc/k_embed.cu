@@ -458,10 +458,17 @@ __global__ void __launch_bounds__(256) attention_fwd_fixed_kernel(const float* _
   {
     const float* q = Q + (int64_t)i * D;
     if (lane < D4) cp_async16(Qs + 4 * lane, q + 4 * lane);
-    const float* kv = KV + (int64_t)i * KS * 2 * D;
-    for (int e = lane; e < c * 2 * D4; e += 32) {
-      const int sl = e / (2 * D4), r = e - sl * 2 * D4;
-      cp_async16(r < D4 ? Ks + sl * D + 4 * r : Vs + sl * D + 4 * (r - D4), kv + 4 * e);
+    // lane l < D / 4 copies chunk l of every valid row's K half and V half: constant offsets from two pointers
+    const float* kv = KV + (int64_t)i * KS * 2 * D + 4 * lane;
+    float* kd = Ks + 4 * lane;
+    if (lane < D4) {
+#pragma unroll
+      for (int t = 0; t < KS; ++t) {
+        if (t < c) {
+          cp_async16(kd + t * D, kv + t * 2 * D);
+          cp_async16(kd + (KS + t) * D, kv + t * 2 * D + D);   // (Vs = Ks + KS * D)
+        }
+      }
     }
   }
   attn_stage_wait();
