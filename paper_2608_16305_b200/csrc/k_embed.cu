@@ -439,37 +439,32 @@ __global__ void __launch_bounds__(256) attention_fwd_kernel(const float* __restr
 // slot) and shared through shared memory, and the weighted sum of V runs on four columns per lane.  Every sum keeps
 // the generic kernel's order of operations, so the two give the same bits.
 template <int D, int H, int KS>
-__global__ void __launch_bounds__(256) attention_fwd_fixed_kernel(const float* __restrict__ Q, const float* __restrict__ KV,
-                                                                  const int32_t* __restrict__ cnt, int n,
-                                                                  float* __restrict__ alpha, float* __restrict__ cat_o) {
+__host__ __device__ constexpr int attn_fwd_fixed_floats() { return (KS * D + D + 2 * H * KS + 3) & ~3; }   // K rows, query, two scratch vectors
+template <int D, int H, int KS>
+__global__ void __launch_bounds__(256, 5) attention_fwd_fixed_kernel(const float* __restrict__ Q, const float* __restrict__ KV,
+                                                                     const int32_t* __restrict__ cnt, int n,
+                                                                     float* __restrict__ alpha, float* __restrict__ cat_o) {
   constexpr int DH = D / H, D4 = D / 4, P = H * KS;
   static_assert(D % 4 == 0 && DH % 2 == 0 && P <= 32 && D4 <= 32, "shape not covered by the fixed kernel");
   extern __shared__ __align__(16) float sm[];
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   const int i = (int)((blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5);
   if (i >= n) return;
-  float* Ks = sm + wib * attn_warp_floats(D, H, KS);
-  float* Vs = Ks + KS * D;
-  float* Qs = Vs + KS * D;
-  float* al = Qs + 2 * D;  // logits
+  // Only the K halves and the query are staged (4.6 KB per warp: five blocks per SM instead of three); the V halves
+  // are read once, column-wise, straight from global memory in the last phase.
+  float* Ks = sm + wib * attn_fwd_fixed_floats<D, H, KS>();
+  float* Qs = Ks + KS * D;
+  float* al = Qs + D;      // logits
   float* pr = al + P;      // exponentials, then probabilities
   const int c = max(0, min(cnt[i], KS));   // a count outside [0, k] is clamped (the neighbor search never produces one)
   const float scale = rsqrtf((float)DH);
-  {
-    const float* q = Q + (int64_t)i * D;
-    if (lane < D4) cp_async16(Qs + 4 * lane, q + 4 * lane);
-    // lane l < D / 4 copies chunk l of every valid row's K half and V half: constant offsets from two pointers
-    const float* kv = KV + (int64_t)i * KS * 2 * D + 4 * lane;
+  const float* kv = KV + (int64_t)i * KS * 2 * D + 4 * lane;
+  if (lane < D4) {
+    cp_async16(Qs + 4 * lane, Q + (int64_t)i * D + 4 * lane);
     float* kd = Ks + 4 * lane;
-    if (lane < D4) {
 #pragma unroll
-      for (int t = 0; t < KS; ++t) {
-        if (t < c) {
-          cp_async16(kd + t * D, kv + t * 2 * D);
-          cp_async16(kd + (KS + t) * D, kv + t * 2 * D + D);   // (Vs = Ks + KS * D)
-        }
-      }
-    }
+    for (int t = 0; t < KS; ++t)
+      if (t < c) cp_async16(kd + t * D, kv + t * 2 * D);
   }
   attn_stage_wait();
   const int h = lane / KS, sl = lane - h * KS;
@@ -515,13 +510,21 @@ __global__ void __launch_bounds__(256) attention_fwd_fixed_kernel(const float* _
   if (lane < D4) {
     const int h0 = (4 * lane) / DH, h1 = (4 * lane + 2) / DH;   // columns 4l, 4l+1 share a head, and so do 4l+2, 4l+3
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    constexpr int HALF = (KS + 1) / 2;   // the rows' loads go out in two rounds (registers)
 #pragma unroll
-    for (int t = 0; t < KS; ++t) {
-      if (t < c) {
-        const float p0 = pr[h0 * KS + t], p1 = pr[h1 * KS + t];
-        const float4 v = *reinterpret_cast<const float4*>(Vs + t * D + 4 * lane);
-        acc.x = fmaf(p0, v.x, acc.x); acc.y = fmaf(p0, v.y, acc.y);
-        acc.z = fmaf(p1, v.z, acc.z); acc.w = fmaf(p1, v.w, acc.w);
+    for (int t0 = 0; t0 < KS; t0 += HALF) {
+      float4 v[HALF];
+#pragma unroll
+      for (int u = 0; u < HALF; ++u)
+        if (t0 + u < KS && t0 + u < c) v[u] = __ldg(reinterpret_cast<const float4*>(kv + (t0 + u) * 2 * D + D));
+#pragma unroll
+      for (int u = 0; u < HALF; ++u) {
+        const int t = t0 + u;
+        if (t < KS && t < c) {
+          const float p0 = pr[h0 * KS + t], p1 = pr[h1 * KS + t];
+          acc.x = fmaf(p0, v[u].x, acc.x); acc.y = fmaf(p0, v[u].y, acc.y);
+          acc.z = fmaf(p1, v[u].z, acc.z); acc.w = fmaf(p1, v[u].w, acc.w);
+        }
       }
     }
     *reinterpret_cast<float4*>(cat_o + (int64_t)i * 2 * D + 4 * lane) = acc;
@@ -702,13 +705,13 @@ int launch_embed(tgnn_ctx* ctx, const int32_t* nodes, const double* times, int n
   if (rc) return rc;
   const int wpb = attn_warps_per_block(d, H, k);
   const bool fixed_shape = d == 100 && H == 2 && k == 10;   // the paper's configuration
-  if (fixed_shape) RC_ATTR(ctx, (attention_fwd_fixed_kernel<100, 2, 10>), attn_smem_bytes(d, H, k, wpb));
+  constexpr int fixed_smem = 8 * attn_fwd_fixed_floats<100, 2, 10>() * 4;   // eight warps per block
+  if (fixed_shape) RC_ATTR(ctx, (attention_fwd_fixed_kernel<100, 2, 10>), fixed_smem);
   else RC_ATTR(ctx, attention_fwd_kernel, attn_smem_bytes(d, H, k, wpb));
   {
     KernelScope scope__(ctx, "attention_fwd", s);
     if (fixed_shape)
-      attention_fwd_fixed_kernel<100, 2, 10><<<(n + wpb - 1) / wpb, wpb * 32, attn_smem_bytes(d, H, k, wpb), s>>>(w.Q, w.KV, cnt, n,
-                                                                                                              w.alpha, w.cat_o);
+      attention_fwd_fixed_kernel<100, 2, 10><<<(n + 7) / 8, 256, fixed_smem, s>>>(w.Q, w.KV, cnt, n, w.alpha, w.cat_o);
     else
       attention_fwd_kernel<<<(n + wpb - 1) / wpb, wpb * 32, attn_smem_bytes(d, H, k, wpb), s>>>(w.Q, w.KV, cnt, n, d, H, k,
                                                                                              w.alpha, w.cat_o);
